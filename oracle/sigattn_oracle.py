@@ -1,0 +1,179 @@
+"""Plain float64 definition of sigmoid self-attention and of its analytic gradient.
+
+TEST INFRASTRUCTURE ONLY: imported by tests, by the smoke check and by the
+benchmark's CPU-baseline leg, never by the product path.  No code is shared with
+the CUDA kernels; this file depends on numpy alone.
+
+What it computes, per (batch, head), all in float64:
+
+  forward (Eq. 3 of Section 2; Algorithm 1 of Appendix F reaches the same result,
+  tiling only reorders the sums)
+      x_ij = scale * <q_i, k_j> + b - m_h * |i - j|
+      P_ij = sigmoid(x_ij),  set to 0 where causal and j > i
+      O    = P V
+
+  backward (sigmoid column of the forward/backward table in Appendix F.1;
+  Algorithm 2 reaches the same result)
+      dV = P^T dO
+      dP = dO V^T
+      dS = P * (1 - P) * dP          (0 where masked)
+      dQ = scale * dS K
+      dK = scale * dS^T Q
+
+Readings of the paper taken here
+  * The bias b is added after the 1/sqrt(d) scaling, once per logit (Eq. 3 defines
+    sigma(u) = sigmoid(u + b) with u the scaled logit).
+  * The causal mask multiplies sigma(.) and keeps the diagonal (the n = 3 example in
+    the sequence-length-normalisation ablation, Appendix G): a masked weight is
+    exactly 0, not sigmoid(b), and passes no gradient.
+  * The table in Appendix F.1 and Algorithm 2 print the factor sqrt(d) in dQ and dK.
+    The chain rule through S = Q K^T / sqrt(d) gives 1/sqrt(d) = scale; central finite
+    differences (tests) confirm scale and reject sqrt(d).  Algorithm 2 also swaps
+    indices in its dV and dP lines; the table's dV = P^T dO and dP = dO V^T are used.
+  * The paper prints no ALiBi formula.  The linear-bias form it cites is used: the
+    head's positive slope m_h times the distance |i - j| is subtracted from the scaled
+    logit (not multiplied by scale); for causal calls only j <= i survives, which is
+    the usual m_h * (i - j).
+
+Every function is pinned by tests that do not call back into this file's own
+formulae (closed forms, brute-force loops, finite differences, the paper's second
+form of the forward, the printed n = 3 mask): there is no "parity unpinned" part.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+__all__ = [
+    "sigmoid",
+    "causal_mask",
+    "position_bias",
+    "attention_weights",
+    "sigattn_fwd",
+    "sigattn_bwd",
+    "sigattn_fwd_sequence_form",
+]
+
+
+def sigmoid(x):
+    """sigmoid(x) = 1 / (1 + exp(-x)) (Eq. 3), evaluated without overflow.
+
+    For x >= 0 the definition is used as printed; for x < 0 the algebraically equal
+    exp(x) / (1 + exp(x)) is used so that exp never sees a large positive argument.
+    """
+    x = np.asarray(x, dtype=np.float64)
+    out = np.empty_like(x)
+    pos = x >= 0
+    out[pos] = 1.0 / (1.0 + np.exp(-x[pos]))
+    e = np.exp(x[~pos])
+    out[~pos] = e / (1.0 + e)
+    return out
+
+
+def causal_mask(n: int, i0: int = 0, i1: int | None = None):
+    """Rows i0..i1-1 of the n x n lower-triangular 0/1 matrix, diagonal included
+    (the matrix M printed for n = 3 in Appendix G's normalisation ablation)."""
+    i1 = n if i1 is None else i1
+    i = np.arange(i0, i1)[:, None]
+    j = np.arange(n)[None, :]
+    return (j <= i).astype(np.float64)
+
+
+def position_bias(n: int, slope: float, i0: int = 0, i1: int | None = None):
+    """Additive linear position bias -slope * |i - j| for rows i0..i1-1 (Appendix F.4
+    names ALiBi; see the module header for the reading)."""
+    i1 = n if i1 is None else i1
+    i = np.arange(i0, i1, dtype=np.float64)[:, None]
+    j = np.arange(n, dtype=np.float64)[None, :]
+    return -float(slope) * np.abs(i - j)
+
+
+def attention_weights(q, k, scale, bias, causal, slope=0.0, i0=0, i1=None):
+    """P for query rows i0..i1-1 of one head: sigmoid(scale * q k^T + b + position
+    bias), times the causal mask.  q, k: [n, d] float64."""
+    n = q.shape[0]
+    i1 = n if i1 is None else i1
+    x = scale * (q[i0:i1] @ k.T) + bias
+    if slope != 0.0:
+        x = x + position_bias(n, slope, i0, i1)
+    p = sigmoid(x)
+    if causal:
+        p = p * causal_mask(n, i0, i1)
+    return p
+
+
+def _as_f64(*arrays):
+    return [np.ascontiguousarray(a, dtype=np.float64) for a in arrays]
+
+
+def _slopes(alibi_slopes, num_heads):
+    if alibi_slopes is None:
+        return np.zeros(num_heads, dtype=np.float64)
+    s = np.asarray(alibi_slopes, dtype=np.float64).reshape(-1)
+    if s.shape[0] != num_heads:
+        raise ValueError("alibi_slopes must hold one slope per head")
+    return s
+
+
+def _row_ranges(n, row_block):
+    """Query rows are independent in the forward and enter dK, dV only through a sum
+    over rows, so they may be visited in slabs to bound memory (an n x n float64 matrix
+    is 2 GiB at n = 16384).  row_block=None visits all rows at once."""
+    step = n if not row_block else int(row_block)
+    return [(a, min(n, a + step)) for a in range(0, n, step)]
+
+
+def sigattn_fwd(q, k, v, scale, bias, causal=False, alibi_slopes=None, row_block=None):
+    """O = sigmoid(scale * Q K^T + b [+ position bias]) [* causal mask] V  (Eq. 3).
+
+    q, k, v: [B, H, N, D] arrays (any float dtype; converted to float64).
+    Returns O as float64 [B, H, N, D].
+    """
+    q, k, v = _as_f64(q, k, v)
+    B, H, N, D = q.shape
+    slopes = _slopes(alibi_slopes, H)
+    o = np.zeros((B, H, N, D), dtype=np.float64)
+    for b in range(B):
+        for h in range(H):
+            for i0, i1 in _row_ranges(N, row_block):
+                p = attention_weights(q[b, h], k[b, h], scale, bias, causal, slopes[h], i0, i1)
+                o[b, h, i0:i1] = p @ v[b, h]
+    return o
+
+
+def sigattn_bwd(q, k, v, d_o, scale, bias, causal=False, alibi_slopes=None, row_block=None):
+    """Gradients of L = sum(O * dO) with respect to Q, K, V (sigmoid column of the
+    forward/backward table in Appendix F.1, with the 1/sqrt(d) factor; see header).
+
+    Returns (dQ, dK, dV), float64 [B, H, N, D] each.
+    """
+    q, k, v, d_o = _as_f64(q, k, v, d_o)
+    B, H, N, D = q.shape
+    slopes = _slopes(alibi_slopes, H)
+    dq = np.zeros_like(q)
+    dk = np.zeros_like(q)
+    dv = np.zeros_like(q)
+    for b in range(B):
+        for h in range(H):
+            for i0, i1 in _row_ranges(N, row_block):
+                p = attention_weights(q[b, h], k[b, h], scale, bias, causal, slopes[h], i0, i1)
+                do_rows = d_o[b, h, i0:i1]
+                dv[b, h] += p.T @ do_rows
+                dp = do_rows @ v[b, h].T
+                ds = p * (1.0 - p) * dp
+                dq[b, h, i0:i1] = scale * (ds @ k[b, h])
+                dk[b, h] += scale * (ds.T @ q[b, h, i0:i1])
+    return dq, dk, dv
+
+
+def sigattn_fwd_sequence_form(q, k, v, scale, n_bias):
+    """Second form of the forward, valid at b = -log(n_bias), non-causal, no position
+    bias (Eq. 4): y_i = sum_j exp(s_ij) / (exp(s_ij) + n_bias) v_j with s the scaled
+    logit.  Kept separate from sigattn_fwd on purpose: it never calls sigmoid()."""
+    q, k, v = _as_f64(q, k, v)
+    B, H, N, D = q.shape
+    o = np.zeros((B, H, N, D), dtype=np.float64)
+    for b in range(B):
+        for h in range(H):
+            e = np.exp(scale * (q[b, h] @ k[b, h].T))
+            o[b, h] = (e / (e + float(n_bias))) @ v[b, h]
+    return o

@@ -1,0 +1,309 @@
+"""Pins for the float64 oracle: closed forms, brute force, finite differences and the
+paper's printed facts.  None of these re-use the oracle's own formulae, so a dropped
+term, a wrong sign or index, or a transposed operand in oracle/ fails at least one."""
+import math
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def rnd(shape, seed, std=1.0):
+    return std * np.random.default_rng(seed).standard_normal(shape)
+
+
+def scalar_sigmoid(x):
+    """Textbook definition with math.exp, independent of oracle.sigmoid."""
+    if x >= 0:
+        return 1.0 / (1.0 + math.exp(-x))
+    e = math.exp(x)
+    return e / (1.0 + e)
+
+
+def brute_forward(q, k, v, scale, bias, causal, slopes):
+    """Pure-Python loops over every (b, h, i, j, d): the definition, element by element."""
+    B, H, N, D = q.shape
+    o = np.zeros((B, H, N, D))
+    for b in range(B):
+        for h in range(H):
+            m = 0.0 if slopes is None else float(slopes[h])
+            for i in range(N):
+                for j in range(N):
+                    if causal and j > i:
+                        continue
+                    s = 0.0
+                    for d in range(D):
+                        s += q[b, h, i, d] * k[b, h, j, d]
+                    x = scale * s + bias - m * abs(i - j)
+                    p = scalar_sigmoid(x)
+                    for d in range(D):
+                        o[b, h, i, d] += p * v[b, h, j, d]
+    return o
+
+
+# ----------------------------------------------------------------------------- sigmoid
+
+
+def test_sigmoid_identities():
+    x = np.linspace(-40, 40, 2001)
+    s = oracle.sigmoid(x)
+    assert np.all(np.isfinite(s))
+    np.testing.assert_allclose(s + oracle.sigmoid(-x), 1.0, rtol=0, atol=2.3e-16)  # 1 ulp
+    assert oracle.sigmoid(np.array([0.0]))[0] == 0.5
+    assert np.all(np.diff(s) >= 0)
+    # Section 4: sigmoid(x) = 0.5 * (1 + tanh(0.5 x))
+    np.testing.assert_allclose(s, 0.5 * (1.0 + np.tanh(0.5 * x)), rtol=0, atol=2.3e-16)
+    ref = np.array([scalar_sigmoid(t) for t in x])
+    np.testing.assert_allclose(s, ref, rtol=1e-15, atol=0)
+
+
+def test_sigmoid_extremes():
+    s = oracle.sigmoid(np.array([-1e4, -745.0, 745.0, 1e4]))
+    assert s[0] == 0.0 and s[-1] == 1.0
+    assert np.all(np.isfinite(s))
+
+
+def test_sigmoid_derivative_is_p_times_one_minus_p():
+    # Appendix E: d p / d z = p (1 - p)
+    z = np.linspace(-6, 6, 25)
+    h = 1e-6
+    fd = (oracle.sigmoid(z + h) - oracle.sigmoid(z - h)) / (2 * h)
+    p = oracle.sigmoid(z)
+    np.testing.assert_allclose(fd, p * (1 - p), rtol=1e-7, atol=1e-10)  # fd truncation + rounding at h = 1e-6
+
+
+# ------------------------------------------------------------------------------ masks
+
+
+def test_causal_mask_matches_printed_n3_example():
+    golden = np.loadtxt(os.path.join(GOLDEN, "causal_mask_n3.txt"))
+    np.testing.assert_array_equal(oracle.causal_mask(3), golden)
+    np.testing.assert_array_equal(oracle.causal_mask(3, 1, 3), golden[1:3])
+
+
+def test_position_bias_is_minus_slope_times_distance():
+    pb = oracle.position_bias(5, 0.25)
+    for i in range(5):
+        for j in range(5):
+            assert pb[i, j] == -0.25 * abs(i - j)
+    np.testing.assert_array_equal(oracle.position_bias(5, 0.25, 2, 4), pb[2:4])
+
+
+# ---------------------------------------------------------------------------- forward
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_forward_q_zero_closed_form(causal):
+    B, H, N, D = 2, 3, 17, 8
+    k, v = rnd((B, H, N, D), 1), rnd((B, H, N, D), 2)
+    q = np.zeros((B, H, N, D))
+    b = -math.log(N)
+    o = oracle.sigattn_fwd(q, k, v, 1 / math.sqrt(D), b, causal)
+    sb = scalar_sigmoid(b)
+    if causal:
+        expect = sb * np.cumsum(v, axis=2)
+    else:
+        expect = np.broadcast_to(sb * v.sum(axis=2, keepdims=True), v.shape)
+    np.testing.assert_allclose(o, expect, rtol=1e-13, atol=1e-14)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_forward_bias_limits(causal):
+    B, H, N, D = 1, 2, 9, 4
+    q, k, v = rnd((B, H, N, D), 3), rnd((B, H, N, D), 4), rnd((B, H, N, D), 5)
+    o_lo = oracle.sigattn_fwd(q, k, v, 0.5, -1e4, causal)
+    assert np.all(o_lo == 0.0)
+    o_hi = oracle.sigattn_fwd(q, k, v, 0.5, 1e4, causal)
+    expect = np.cumsum(v, axis=2) if causal else np.broadcast_to(v.sum(axis=2, keepdims=True), v.shape)
+    np.testing.assert_allclose(o_hi, expect, rtol=1e-14, atol=1e-14)
+
+
+def test_forward_single_token():
+    D = 6
+    q, k, v = rnd((1, 1, 1, D), 6), rnd((1, 1, 1, D), 7), rnd((1, 1, 1, D), 8)
+    scale, b = 0.37, -0.8
+    for causal in (False, True):
+        o = oracle.sigattn_fwd(q, k, v, scale, b, causal, alibi_slopes=[0.5])
+        p = scalar_sigmoid(scale * float(q[0, 0, 0] @ k[0, 0, 0]) + b)
+        np.testing.assert_allclose(o[0, 0, 0], p * v[0, 0, 0], rtol=1e-15)
+
+
+def test_forward_complement_identity():
+    # sigmoid(x) + sigmoid(-x) = 1  =>  O(Q, b) + O(-Q, -b) = column sum of V
+    B, H, N, D = 2, 2, 11, 5
+    q, k, v = rnd((B, H, N, D), 9), rnd((B, H, N, D), 10), rnd((B, H, N, D), 11)
+    o1 = oracle.sigattn_fwd(q, k, v, 0.4, -1.3)
+    o2 = oracle.sigattn_fwd(-q, k, v, 0.4, 1.3)
+    np.testing.assert_allclose(o1 + o2, np.broadcast_to(v.sum(2, keepdims=True), v.shape), rtol=1e-13, atol=1e-13)
+
+
+def test_forward_matches_sequence_form_and_direct_formula():
+    # Eq. 4: at b = -log n the weights are exp(s) / (exp(s) + n)
+    B, H, N, D = 1, 2, 13, 8
+    q, k, v = rnd((B, H, N, D), 12), rnd((B, H, N, D), 13), rnd((B, H, N, D), 14)
+    scale = 1 / math.sqrt(D)
+    o = oracle.sigattn_fwd(q, k, v, scale, -math.log(N))
+    np.testing.assert_allclose(o, oracle.sigattn_fwd_sequence_form(q, k, v, scale, N), rtol=1e-13, atol=1e-15)
+    # the same second form retyped here with einsum, so the pin does not lean on oracle/
+    e = np.exp(scale * np.einsum("bhid,bhjd->bhij", q, k))
+    np.testing.assert_allclose(o, np.einsum("bhij,bhjd->bhid", e / (e + N), v), rtol=1e-13, atol=1e-15)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("with_slopes", [False, True])
+def test_forward_brute_force(causal, with_slopes):
+    B, H, N, D = 2, 2, 7, 3
+    q, k, v = rnd((B, H, N, D), 15), rnd((B, H, N, D), 16), rnd((B, H, N, D), 17)
+    slopes = np.array([0.5, 0.0625]) if with_slopes else None
+    scale, b = 0.61, -1.1
+    o = oracle.sigattn_fwd(q, k, v, scale, b, causal, slopes)
+    np.testing.assert_allclose(o, brute_forward(q, k, v, scale, b, causal, slopes), rtol=1e-13, atol=1e-14)
+
+
+def test_forward_causal_first_and_last_rows():
+    B, H, N, D = 1, 1, 10, 4
+    q, k, v = rnd((B, H, N, D), 18), rnd((B, H, N, D), 19), rnd((B, H, N, D), 20)
+    scale, b = 0.5, -0.3
+    oc = oracle.sigattn_fwd(q, k, v, scale, b, True)
+    of = oracle.sigattn_fwd(q, k, v, scale, b, False)
+    p00 = scalar_sigmoid(scale * float(q[0, 0, 0] @ k[0, 0, 0]) + b)
+    np.testing.assert_allclose(oc[0, 0, 0], p00 * v[0, 0, 0], rtol=1e-14)
+    np.testing.assert_allclose(oc[0, 0, -1], of[0, 0, -1], rtol=1e-14)
+    assert not np.allclose(oc[0, 0, 3], of[0, 0, 3])
+
+
+def test_forward_huge_slope_keeps_only_the_diagonal():
+    B, H, N, D = 1, 2, 6, 4
+    q, k, v = rnd((B, H, N, D), 21), rnd((B, H, N, D), 22), rnd((B, H, N, D), 23)
+    scale, b = 0.5, 0.2
+    o = oracle.sigattn_fwd(q, k, v, scale, b, True, alibi_slopes=[1e4, 1e4])
+    for h in range(H):
+        for i in range(N):
+            p = scalar_sigmoid(scale * float(q[0, h, i] @ k[0, h, i]) + b)
+            np.testing.assert_allclose(o[0, h, i], p * v[0, h, i], rtol=1e-13)
+
+
+def test_forward_structure_properties():
+    B, H, N, D = 2, 3, 9, 4
+    q, k, v = rnd((B, H, N, D), 24), rnd((B, H, N, D), 25), rnd((B, H, N, D), 26)
+    scale, b = 0.45, -1.0
+    o = oracle.sigattn_fwd(q, k, v, scale, b)
+    # zero slopes == no slopes
+    np.testing.assert_array_equal(o, oracle.sigattn_fwd(q, k, v, scale, b, alibi_slopes=np.zeros(H)))
+    # joint permutation of keys and values leaves O unchanged; permuting queries permutes O
+    perm = np.random.default_rng(0).permutation(N)
+    np.testing.assert_allclose(o, oracle.sigattn_fwd(q, k[:, :, perm], v[:, :, perm], scale, b), rtol=1e-13, atol=1e-14)
+    np.testing.assert_allclose(o[:, :, perm], oracle.sigattn_fwd(q[:, :, perm], k, v, scale, b), rtol=1e-13, atol=1e-14)
+    # linear in V
+    v2 = rnd((B, H, N, D), 27)
+    np.testing.assert_allclose(
+        oracle.sigattn_fwd(q, k, 2 * v - 3 * v2, scale, b),
+        2 * o - 3 * oracle.sigattn_fwd(q, k, v2, scale, b), rtol=1e-12, atol=1e-13)
+    # heads and batches are independent; each head uses its own slope
+    slopes = np.array([0.5, 0.25, 0.125])
+    os_ = oracle.sigattn_fwd(q, k, v, scale, b, True, slopes)
+    for bb in range(B):
+        for h in range(H):
+            one = oracle.sigattn_fwd(q[bb:bb + 1, h:h + 1], k[bb:bb + 1, h:h + 1], v[bb:bb + 1, h:h + 1],
+                                     scale, b, True, slopes[h:h + 1])
+            np.testing.assert_array_equal(os_[bb, h], one[0, 0])
+    # row slabs give the same result as all rows at once
+    np.testing.assert_allclose(os_, oracle.sigattn_fwd(q, k, v, scale, b, True, slopes, row_block=4), rtol=1e-14, atol=1e-15)
+
+
+# --------------------------------------------------------------------------- backward
+
+
+def loss(q, k, v, d_o, scale, b, causal, slopes):
+    return float(np.sum(oracle.sigattn_fwd(q, k, v, scale, b, causal, slopes) * d_o))
+
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("with_slopes", [False, True])
+def test_backward_finite_differences(causal, with_slopes):
+    """Central differences of L = sum(O * dO).  This is what settles the 1/sqrt(d)
+    factor in dQ, dK against the sqrt(d) printed in Appendix F.1."""
+    B, H, N, D = 1, 2, 6, 4
+    q, k, v, d_o = (rnd((B, H, N, D), s) for s in (30, 31, 32, 33))
+    slopes = np.array([0.5, 0.125]) if with_slopes else None
+    scale, b = 1 / math.sqrt(D), -math.log(N)
+    dq, dk, dv = oracle.sigattn_bwd(q, k, v, d_o, scale, b, causal, slopes)
+    h = 1e-6
+    for name, x, g in (("q", q, dq), ("k", k, dk), ("v", v, dv)):
+        fd = np.zeros_like(x)
+        it = np.nditer(x, flags=["multi_index"])
+        for _ in it:
+            idx = it.multi_index
+            old = x[idx]
+            x[idx] = old + h
+            lp = loss(q, k, v, d_o, scale, b, causal, slopes)
+            x[idx] = old - h
+            lm = loss(q, k, v, d_o, scale, b, causal, slopes)
+            x[idx] = old
+            fd[idx] = (lp - lm) / (2 * h)
+        err = np.linalg.norm(fd - g) / np.linalg.norm(fd)
+        assert err < 1e-7, (name, err)
+        if name in ("q", "k"):
+            # the printed sqrt(d) factor would be off by exactly d
+            assert np.linalg.norm(fd - D * g) / np.linalg.norm(fd) > 1.0
+
+
+def test_backward_single_token_closed_form():
+    D = 5
+    q, k, v, d_o = (rnd((1, 1, 1, D), s) for s in (40, 41, 42, 43))
+    scale, b = 0.3, -0.4
+    dq, dk, dv = oracle.sigattn_bwd(q, k, v, d_o, scale, b, True)
+    p = scalar_sigmoid(scale * float(q[0, 0, 0] @ k[0, 0, 0]) + b)
+    ds = float(d_o[0, 0, 0] @ v[0, 0, 0]) * p * (1 - p)
+    np.testing.assert_allclose(dv[0, 0, 0], p * d_o[0, 0, 0], rtol=1e-14)
+    np.testing.assert_allclose(dq[0, 0, 0], scale * ds * k[0, 0, 0], rtol=1e-14)
+    np.testing.assert_allclose(dk[0, 0, 0], scale * ds * q[0, 0, 0], rtol=1e-14)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_backward_brute_force_loops(causal):
+    B, H, N, D = 1, 2, 5, 3
+    q, k, v, d_o = (rnd((B, H, N, D), s) for s in (50, 51, 52, 53))
+    slopes = np.array([0.25, 0.5])
+    scale, b = 0.7, -0.9
+    dq, dk, dv = oracle.sigattn_bwd(q, k, v, d_o, scale, b, causal, slopes)
+    rq, rk, rv = np.zeros_like(q), np.zeros_like(q), np.zeros_like(q)
+    for h in range(H):
+        for i in range(N):
+            for j in range(N):
+                if causal and j > i:
+                    continue
+                x = scale * float(q[0, h, i] @ k[0, h, j]) + b - slopes[h] * abs(i - j)
+                p = scalar_sigmoid(x)
+                dp = float(d_o[0, h, i] @ v[0, h, j])
+                ds = p * (1 - p) * dp
+                rv[0, h, j] += p * d_o[0, h, i]
+                rq[0, h, i] += scale * ds * k[0, h, j]
+                rk[0, h, j] += scale * ds * q[0, h, i]
+    np.testing.assert_allclose(dq, rq, rtol=1e-13, atol=1e-15)
+    np.testing.assert_allclose(dk, rk, rtol=1e-13, atol=1e-15)
+    np.testing.assert_allclose(dv, rv, rtol=1e-13, atol=1e-15)
+
+
+def test_backward_structure_properties():
+    B, H, N, D = 2, 2, 8, 4
+    q, k, v, d_o = (rnd((B, H, N, D), s) for s in (60, 61, 62, 63))
+    scale, b = 0.5, -1.2
+    # Q = 0 => dK = 0 ; dV linear in dO ; row slabs agree
+    _, dk0, _ = oracle.sigattn_bwd(np.zeros_like(q), k, v, d_o, scale, b, True)
+    assert np.all(dk0 == 0.0)
+    g1 = oracle.sigattn_bwd(q, k, v, d_o, scale, b, True)
+    g2 = oracle.sigattn_bwd(q, k, v, 3.0 * d_o, scale, b, True)
+    for a, c in zip(g1, g2):
+        np.testing.assert_allclose(3.0 * a, c, rtol=1e-13, atol=1e-15)
+    g3 = oracle.sigattn_bwd(q, k, v, d_o, scale, b, True, row_block=3)
+    for a, c in zip(g1, g3):
+        np.testing.assert_allclose(a, c, rtol=1e-13, atol=1e-15)
+    # causal: the last key receives gradient only from the last query
+    dq, dk, dv = g1
+    p = scalar_sigmoid(scale * float(q[0, 0, -1] @ k[0, 0, -1]) + b)
+    np.testing.assert_allclose(dv[0, 0, -1], p * d_o[0, 0, -1], rtol=1e-13)
