@@ -1,0 +1,118 @@
+/*
+ * sigattn — fused sigmoid self-attention, forward and backward, for NVIDIA B200 (sm_100a).
+ *
+ * C ABI of libsigattn.so.  Plain pointers and sizes only; no framework types.
+ *
+ * Operation (Section 2, Eq. 3 of "Theory, Analysis, and Best Practices for Sigmoid
+ * Self-Attention"; tiled forward = Algorithm 1, tiled backward = Algorithm 2 of
+ * Appendix F.1), per batch b and head h, with i the query row and j the key row:
+ *
+ *     x_ij = scale * <Q_i, K_j> + bias - slope_h * |i - j|
+ *     P_ij = sigmoid(x_ij), and P_ij = 0 where causal != 0 and j > i
+ *     O    = P V
+ *
+ *     dV = P^T dO,  dP = dO V^T,  dS = P * (1 - P) * dP,
+ *     dQ = scale * dS K,  dK = scale * dS^T Q
+ *
+ * The factor in dQ and dK is `scale` (= 1/sqrt(D) in the paper's use), the derivative
+ * of the scaled logit; the sqrt(d) printed in the paper's table is a typo.  No row
+ * maximum, row sum, log-sum-exp or rowsum(dO * O) exists anywhere: the backward
+ * recomputes P from Q, K alone (activation recomputation, Section 4).
+ *
+ * Layout.  Every tensor is contiguous row-major [B, H, N, D], D innermost.
+ * dtype 0: bfloat16 tensors, tensor-core path (tcgen05 MMA, fp32 accumulation).
+ * dtype 1: float32 tensors, CUDA-core debug path (exact expf and division).
+ * D must be 64 or 128.  Base pointers must be 16-byte aligned.  `alibi_slopes` is
+ * NULL or a device pointer to H floats (the positive slope of each head, shared by
+ * all batches); NULL behaves like all-zero slopes.
+ *
+ * Ownership.  All pointers are DEVICE pointers owned by the caller, except where a
+ * function says "host".  The library allocates no device memory on these calls; the
+ * backward's fp32 dQ accumulator lives in the caller's `workspace`.  Outputs are
+ * overwritten in full; inputs are never written.
+ *
+ * Asynchrony.  Work is enqueued on `stream` (a cudaStream_t; NULL = default stream)
+ * and the call returns without synchronising.
+ *
+ * Errors.  Return value 0 = success; negative = error, nothing was launched:
+ *   -1 null pointer            -2 unsupported shape (D not 64/128, a size < 1, too large)
+ *   -3 misaligned pointer      -4 bad dtype or flag
+ *   -5 workspace too small     -6 device is not sm_100
+ *   -7 CUDA runtime/driver error at set-up or launch (see sigattn_last_cuda_error)
+ *   -8 a bounded device-side wait expired in an earlier launch (reported by sigattn_check)
+ * Arguments are validated before anything is enqueued.
+ */
+#ifndef SIGATTN_H_
+#define SIGATTN_H_
+
+#include <stddef.h>
+
+#if defined(__GNUC__)
+#define SIGATTN_API __attribute__((visibility("default")))
+#else
+#define SIGATTN_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SIGATTN_OK 0
+#define SIGATTN_ERR_NULL (-1)
+#define SIGATTN_ERR_SHAPE (-2)
+#define SIGATTN_ERR_ALIGN (-3)
+#define SIGATTN_ERR_FLAG (-4)
+#define SIGATTN_ERR_WORKSPACE (-5)
+#define SIGATTN_ERR_ARCH (-6)
+#define SIGATTN_ERR_CUDA (-7)
+#define SIGATTN_ERR_DEVICE_TIMEOUT (-8)
+
+#define SIGATTN_DTYPE_BF16 0
+#define SIGATTN_DTYPE_FP32 1
+
+/* Forward (Eq. 3; Algorithm 1).  q, k, v: inputs; o: output; all [B, H, N, D]. */
+SIGATTN_API int sigattn_fwd(const void* q, const void* k, const void* v, void* o,
+                int B, int H, int N, int D,
+                float scale, float bias, int causal,
+                const float* alibi_slopes, int dtype, void* stream);
+
+/* Backward (sigmoid column of the forward/backward table, Appendix F.1; Algorithm 2).
+ * q, k, v, d_o: inputs; dq, dk, dv: outputs; all [B, H, N, D].
+ * workspace: device scratch of at least sigattn_bwd_workspace_bytes(...) bytes,
+ * 256-byte aligned; its contents on entry are irrelevant and on exit unspecified.
+ * Two calls that share a workspace must not overlap on the device.
+ * dQ sums contributions of different key tiles with floating-point atomics, so its
+ * low-order bits may differ from run to run; dK and dV are deterministic. */
+SIGATTN_API int sigattn_bwd(const void* q, const void* k, const void* v, const void* d_o,
+                void* dq, void* dk, void* dv,
+                int B, int H, int N, int D,
+                float scale, float bias, int causal,
+                const float* alibi_slopes, int dtype,
+                void* workspace, size_t workspace_bytes, void* stream);
+
+/* Bytes of scratch sigattn_bwd needs for this problem (0 for the fp32 debug path).
+ * Returns 0 for invalid shapes as well; sigattn_bwd reports those. */
+SIGATTN_API size_t sigattn_bwd_workspace_bytes(int B, int H, int N, int D, int dtype);
+
+/* Synchronises `stream`, then returns 0 or SIGATTN_ERR_DEVICE_TIMEOUT if any kernel of
+ * this library gave up a bounded wait on the current device since the last check
+ * (the flag is cleared), or SIGATTN_ERR_CUDA if the stream reports a CUDA error. */
+SIGATTN_API int sigattn_check(void* stream);
+
+/* Text for an error code (static storage, never NULL). */
+SIGATTN_API const char* sigattn_strerror(int code);
+
+/* cudaGetErrorString of the CUDA error behind the last SIGATTN_ERR_CUDA on this thread. */
+SIGATTN_API const char* sigattn_last_cuda_error(void);
+
+/* Library version: major * 10000 + minor * 100 + patch. */
+SIGATTN_API int sigattn_version(void);
+
+/* Number of kernels of this library launched by this process so far (all threads). */
+SIGATTN_API unsigned long long sigattn_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+
+#endif /* SIGATTN_H_ */

@@ -1,0 +1,31 @@
+"""Fused sigmoid self-attention (forward + backward) for NVIDIA B200.
+
+The computation lives in libsigattn.so (hand-written CUDA for sm_100a, C ABI declared
+in include/sigattn.h).  This package is the thin Python binding plus the seeded
+synthetic-input recipes used by the tests and the benchmark.
+
+The binding is imported on first use of one of its names, so that
+`python -m paper_2409_04431_b200.build` can run before the library exists; using any
+operation without the built library raises ImportError (there is no fallback).
+"""
+_BINDING_NAMES = (
+    "DTYPE_BF16",
+    "DTYPE_FP32",
+    "SigattnError",
+    "sigattn_bwd",
+    "sigattn_bwd_workspace_bytes",
+    "sigattn_check",
+    "sigattn_fwd",
+    "sigattn_launch_count",
+    "sigattn_strerror",
+    "sigattn_version",
+)
+
+__all__ = list(_BINDING_NAMES)
+
+
+def __getattr__(name):
+    if name in _BINDING_NAMES:
+        from . import binding
+        return getattr(binding, name)
+    raise AttributeError(f"module {__name__!r} has no attribute {name!r}")

@@ -1,0 +1,174 @@
+"""ctypes binding of libsigattn.so: argument marshalling only.
+
+Every step of the attention path runs inside the library's CUDA kernels.  PyTorch is
+used for device memory and streams, nothing else.  There is no CPU or PyTorch
+fallback: if the shared library is missing, importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+_PKG_DIR = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG_DIR, "libsigattn.so")
+
+DTYPE_BF16 = 0
+DTYPE_FP32 = 1
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing. Build it with `python -m paper_2409_04431_b200.build` "
+        "(needs nvcc); there is no fallback implementation."
+    )
+
+_lib = ctypes.CDLL(LIB_PATH)
+
+_c = ctypes
+_lib.sigattn_fwd.restype = _c.c_int
+_lib.sigattn_fwd.argtypes = [_c.c_void_p] * 4 + [_c.c_int] * 4 + [_c.c_float, _c.c_float, _c.c_int,
+                                                                    _c.c_void_p, _c.c_int, _c.c_void_p]
+_lib.sigattn_bwd.restype = _c.c_int
+_lib.sigattn_bwd.argtypes = [_c.c_void_p] * 7 + [_c.c_int] * 4 + [_c.c_float, _c.c_float, _c.c_int,
+                                                                    _c.c_void_p, _c.c_int, _c.c_void_p,
+                                                                    _c.c_size_t, _c.c_void_p]
+_lib.sigattn_bwd_workspace_bytes.restype = _c.c_size_t
+_lib.sigattn_bwd_workspace_bytes.argtypes = [_c.c_int] * 5
+_lib.sigattn_check.restype = _c.c_int
+_lib.sigattn_check.argtypes = [_c.c_void_p]
+_lib.sigattn_strerror.restype = _c.c_char_p
+_lib.sigattn_strerror.argtypes = [_c.c_int]
+_lib.sigattn_last_cuda_error.restype = _c.c_char_p
+_lib.sigattn_last_cuda_error.argtypes = []
+_lib.sigattn_version.restype = _c.c_int
+_lib.sigattn_version.argtypes = []
+_lib.sigattn_launch_count.restype = _c.c_ulonglong
+_lib.sigattn_launch_count.argtypes = []
+
+EXPORTED = [
+    "sigattn_fwd", "sigattn_bwd", "sigattn_bwd_workspace_bytes", "sigattn_check",
+    "sigattn_strerror", "sigattn_last_cuda_error", "sigattn_version", "sigattn_launch_count",
+]
+
+
+class SigattnError(RuntimeError):
+    def __init__(self, code: int):
+        self.code = code
+        msg = _lib.sigattn_strerror(code).decode()
+        if code == -7:
+            msg += ": " + _lib.sigattn_last_cuda_error().decode()
+        super().__init__(f"sigattn error {code}: {msg}")
+
+
+def lib():
+    """The loaded ctypes library (raw C-ABI access, e.g. for error-path tests)."""
+    return _lib
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    return t.data_ptr()
+
+
+def _stream_ptr(stream):
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+def _dtype_code(t) -> int:
+    import torch
+    if t.dtype == torch.bfloat16:
+        return DTYPE_BF16
+    if t.dtype == torch.float32:
+        return DTYPE_FP32
+    raise TypeError(f"sigattn supports bfloat16 and float32 tensors, got {t.dtype}")
+
+
+def _check_same(ts, names):
+    import torch
+    ref = ts[0]
+    if ref.dim() != 4:
+        raise ValueError("tensors must be [B, H, N, D]")
+    for t, n in zip(ts, names):
+        if not isinstance(t, torch.Tensor) or not t.is_cuda:
+            raise ValueError(f"{n} must be a CUDA tensor")
+        if t.shape != ref.shape or t.dtype != ref.dtype or t.device != ref.device:
+            raise ValueError(f"{n} must match q in shape, dtype and device")
+        if not t.is_contiguous():
+            raise ValueError(f"{n} must be contiguous [B, H, N, D]")
+
+
+def sigattn_version() -> int:
+    return _lib.sigattn_version()
+
+
+def sigattn_launch_count() -> int:
+    return int(_lib.sigattn_launch_count())
+
+
+def sigattn_strerror(code: int) -> str:
+    return _lib.sigattn_strerror(code).decode()
+
+
+def sigattn_bwd_workspace_bytes(B, H, N, D, dtype_code) -> int:
+    return int(_lib.sigattn_bwd_workspace_bytes(B, H, N, D, dtype_code))
+
+
+def sigattn_check(stream=None) -> None:
+    rc = _lib.sigattn_check(_stream_ptr(stream))
+    if rc != 0:
+        raise SigattnError(rc)
+
+
+def sigattn_fwd(q, k, v, scale, bias, causal=False, alibi_slopes=None, out=None, stream=None):
+    """O = sigmoid(scale * Q K^T + bias [- slope * |i - j|]) [causal-masked] V.
+
+    q, k, v: contiguous CUDA tensors [B, H, N, D], bfloat16 (tensor-core path) or
+    float32 (debug path).  alibi_slopes: None or a float32 CUDA tensor of H slopes.
+    Returns `out` (allocated if None).  Enqueues on the current stream; does not sync.
+    """
+    import torch
+    _check_same([q, k, v], ["q", "k", "v"])
+    if out is None:
+        out = torch.empty_like(q)
+    else:
+        _check_same([q, out], ["q", "out"])
+    B, H, N, D = q.shape
+    with torch.cuda.device(q.device):
+        rc = _lib.sigattn_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, H, N, D, float(scale), float(bias),
+                              int(bool(causal)), _ptr(alibi_slopes), _dtype_code(q), _stream_ptr(stream))
+    if rc != 0:
+        raise SigattnError(rc)
+    return out
+
+
+def sigattn_bwd(q, k, v, d_o, scale, bias, causal=False, alibi_slopes=None, workspace=None, out=None, stream=None):
+    """(dQ, dK, dV) of L = sum(O * dO).  `workspace`: optional uint8 CUDA tensor of at
+    least sigattn_bwd_workspace_bytes bytes (allocated if None).  `out`: optional
+    (dq, dk, dv) tuple to write into."""
+    import torch
+    _check_same([q, k, v, d_o], ["q", "k", "v", "d_o"])
+    B, H, N, D = q.shape
+    code = _dtype_code(q)
+    if out is None:
+        dq, dk, dv = torch.empty_like(q), torch.empty_like(q), torch.empty_like(q)
+    else:
+        dq, dk, dv = out
+        _check_same([q, dq, dk, dv], ["q", "dq", "dk", "dv"])
+    need = sigattn_bwd_workspace_bytes(B, H, N, D, code)
+    if workspace is None and need > 0:
+        workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    with torch.cuda.device(q.device):
+        rc = _lib.sigattn_bwd(_ptr(q), _ptr(k), _ptr(v), _ptr(d_o), _ptr(dq), _ptr(dk), _ptr(dv), B, H, N, D,
+                              float(scale), float(bias), int(bool(causal)), _ptr(alibi_slopes), code,
+                              _ptr(workspace), ws_bytes, _stream_ptr(stream))
+    if rc != 0:
+        raise SigattnError(rc)
+    return dq, dk, dv

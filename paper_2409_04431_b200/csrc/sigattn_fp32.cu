@@ -1,0 +1,167 @@
+// float32 debug path on CUDA cores: the definition evaluated with exact expf and a
+// true division, fp32 FMA accumulation, no tensor cores (TF32 would cost 1e-3 of
+// accuracy).  One thread block per query row (forward, dQ) or per key row (dK, dV);
+// nothing is shared between blocks, so every output is deterministic.
+//
+// Forward: Eq. 3 / Algorithm 1.  Backward: the sigmoid column of the forward/backward
+// table in Appendix F.1 / Algorithm 2, with the factor scale = 1/sqrt(d) in dQ and dK.
+#include "sigattn_internal.h"
+#include "../../include/sigattn.h"
+
+namespace sigattn {
+namespace {
+
+constexpr int kThreads = 128;
+
+__device__ __forceinline__ float sigmoid_exact(float x) { return 1.0f / (1.0f + expf(-x)); }
+
+__device__ __forceinline__ float dot_row(const float* __restrict__ a_smem, const float* __restrict__ b, int D) {
+  float s = 0.0f;
+  for (int d = 0; d < D; ++d) s = fmaf(a_smem[d], b[d], s);
+  return s;
+}
+
+// grid (N, B*H); block 128.  Thread t handles key j0 + t, then output column t.
+__global__ void fwd_fp32_kernel(const float* __restrict__ q, const float* __restrict__ k,
+                                const float* __restrict__ v, float* __restrict__ o, int H, int N, int D,
+                                float scale, float bias, int causal, const float* __restrict__ slopes) {
+  __shared__ float sq[128];
+  __shared__ float sp[kThreads];
+  const int i = blockIdx.x, bh = blockIdx.y, t = threadIdx.x;
+  const size_t base = static_cast<size_t>(bh) * N * D;
+  const float slope = slopes ? slopes[bh % H] : 0.0f;
+  if (t < D) sq[t] = q[base + static_cast<size_t>(i) * D + t];
+  __syncthreads();
+  const int jend = causal ? i + 1 : N;
+  float acc = 0.0f;
+  for (int j0 = 0; j0 < jend; j0 += kThreads) {
+    const int j = j0 + t;
+    float p = 0.0f;
+    if (j < jend) {
+      const float s = dot_row(sq, k + base + static_cast<size_t>(j) * D, D);
+      const float x = fmaf(scale, s, bias) - slope * fabsf(static_cast<float>(i - j));
+      p = sigmoid_exact(x);
+    }
+    sp[t] = p;
+    __syncthreads();
+    if (t < D) {
+      const int cnt = min(kThreads, jend - j0);
+      for (int jj = 0; jj < cnt; ++jj) acc = fmaf(sp[jj], v[base + static_cast<size_t>(j0 + jj) * D + t], acc);
+    }
+    __syncthreads();
+  }
+  if (t < D) o[base + static_cast<size_t>(i) * D + t] = acc;
+}
+
+// dQ_i = scale * sum_j dS_ij K_j.  grid (N, B*H).
+__global__ void bwd_dq_fp32_kernel(const float* __restrict__ q, const float* __restrict__ k,
+                                   const float* __restrict__ v, const float* __restrict__ d_o,
+                                   float* __restrict__ dq, int H, int N, int D, float scale, float bias,
+                                   int causal, const float* __restrict__ slopes) {
+  __shared__ float sq[128];
+  __shared__ float sdo[128];
+  __shared__ float sds[kThreads];
+  const int i = blockIdx.x, bh = blockIdx.y, t = threadIdx.x;
+  const size_t base = static_cast<size_t>(bh) * N * D;
+  const float slope = slopes ? slopes[bh % H] : 0.0f;
+  if (t < D) {
+    sq[t] = q[base + static_cast<size_t>(i) * D + t];
+    sdo[t] = d_o[base + static_cast<size_t>(i) * D + t];
+  }
+  __syncthreads();
+  const int jend = causal ? i + 1 : N;
+  float acc = 0.0f;
+  for (int j0 = 0; j0 < jend; j0 += kThreads) {
+    const int j = j0 + t;
+    float ds = 0.0f;
+    if (j < jend) {
+      const float s = dot_row(sq, k + base + static_cast<size_t>(j) * D, D);
+      const float x = fmaf(scale, s, bias) - slope * fabsf(static_cast<float>(i - j));
+      const float p = sigmoid_exact(x);
+      const float dp = dot_row(sdo, v + base + static_cast<size_t>(j) * D, D);
+      ds = p * (1.0f - p) * dp;
+    }
+    sds[t] = ds;
+    __syncthreads();
+    if (t < D) {
+      const int cnt = min(kThreads, jend - j0);
+      for (int jj = 0; jj < cnt; ++jj) acc = fmaf(sds[jj], k[base + static_cast<size_t>(j0 + jj) * D + t], acc);
+    }
+    __syncthreads();
+  }
+  if (t < D) dq[base + static_cast<size_t>(i) * D + t] = scale * acc;
+}
+
+// dV_j = sum_i P_ij dO_i ; dK_j = scale * sum_i dS_ij Q_i.  grid (N, B*H), one key row each.
+__global__ void bwd_dkdv_fp32_kernel(const float* __restrict__ q, const float* __restrict__ k,
+                                     const float* __restrict__ v, const float* __restrict__ d_o,
+                                     float* __restrict__ dk, float* __restrict__ dv, int H, int N, int D,
+                                     float scale, float bias, int causal, const float* __restrict__ slopes) {
+  __shared__ float sk[128];
+  __shared__ float sv[128];
+  __shared__ float sp[kThreads];
+  __shared__ float sds[kThreads];
+  const int j = blockIdx.x, bh = blockIdx.y, t = threadIdx.x;
+  const size_t base = static_cast<size_t>(bh) * N * D;
+  const float slope = slopes ? slopes[bh % H] : 0.0f;
+  if (t < D) {
+    sk[t] = k[base + static_cast<size_t>(j) * D + t];
+    sv[t] = v[base + static_cast<size_t>(j) * D + t];
+  }
+  __syncthreads();
+  const int ibeg = causal ? j : 0;
+  float acc_k = 0.0f, acc_v = 0.0f;
+  for (int i0 = ibeg; i0 < N; i0 += kThreads) {
+    const int i = i0 + t;
+    float p = 0.0f, ds = 0.0f;
+    if (i < N) {
+      const float s = dot_row(sk, q + base + static_cast<size_t>(i) * D, D);
+      const float x = fmaf(scale, s, bias) - slope * fabsf(static_cast<float>(i - j));
+      p = sigmoid_exact(x);
+      const float dp = dot_row(sv, d_o + base + static_cast<size_t>(i) * D, D);
+      ds = p * (1.0f - p) * dp;
+    }
+    sp[t] = p;
+    sds[t] = ds;
+    __syncthreads();
+    if (t < D) {
+      const int cnt = min(kThreads, N - i0);
+      for (int ii = 0; ii < cnt; ++ii) {
+        const size_t row = base + static_cast<size_t>(i0 + ii) * D + t;
+        acc_v = fmaf(sp[ii], d_o[row], acc_v);
+        acc_k = fmaf(sds[ii], q[row], acc_k);
+      }
+    }
+    __syncthreads();
+  }
+  if (t < D) {
+    dv[base + static_cast<size_t>(j) * D + t] = acc_v;
+    dk[base + static_cast<size_t>(j) * D + t] = scale * acc_k;
+  }
+}
+
+}  // namespace
+
+int launch_fwd_fp32(const float* q, const float* k, const float* v, float* o, const Problem& p,
+                    cudaStream_t stream, unsigned long long* launches, cudaError_t* cuda_err) {
+  dim3 grid(p.N, p.B * p.H);
+  fwd_fp32_kernel<<<grid, kThreads, 0, stream>>>(q, k, v, o, p.H, p.N, p.D, p.scale, p.bias, p.causal, p.slopes);
+  *launches += 1;
+  *cuda_err = cudaGetLastError();
+  return *cuda_err == cudaSuccess ? SIGATTN_OK : SIGATTN_ERR_CUDA;
+}
+
+int launch_bwd_fp32(const float* q, const float* k, const float* v, const float* d_o, float* dq, float* dk,
+                    float* dv, const Problem& p, cudaStream_t stream, unsigned long long* launches,
+                    cudaError_t* cuda_err) {
+  dim3 grid(p.N, p.B * p.H);
+  bwd_dq_fp32_kernel<<<grid, kThreads, 0, stream>>>(q, k, v, d_o, dq, p.H, p.N, p.D, p.scale, p.bias, p.causal,
+                                                    p.slopes);
+  bwd_dkdv_fp32_kernel<<<grid, kThreads, 0, stream>>>(q, k, v, d_o, dk, dv, p.H, p.N, p.D, p.scale, p.bias,
+                                                      p.causal, p.slopes);
+  *launches += 2;
+  *cuda_err = cudaGetLastError();
+  return *cuda_err == cudaSuccess ? SIGATTN_OK : SIGATTN_ERR_CUDA;
+}
+
+}  // namespace sigattn

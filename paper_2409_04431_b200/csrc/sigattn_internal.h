@@ -1,0 +1,38 @@
+// Internal interface between the C-ABI layer and the kernel launchers.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+namespace sigattn {
+
+struct Problem {
+  int B, H, N, D;
+  float scale, bias;
+  int causal;
+  const float* slopes;  // device pointer to H floats, or nullptr
+};
+
+// Every launcher enqueues on `stream`, adds the number of kernels it launched to
+// *launches and returns a SIGATTN_* code; on SIGATTN_ERR_CUDA it stores the CUDA error
+// in *cuda_err.  `status` is the device-side status word that kernels set when a
+// bounded wait expires.
+
+int launch_fwd_fp32(const float* q, const float* k, const float* v, float* o, const Problem& p,
+                    cudaStream_t stream, unsigned long long* launches, cudaError_t* cuda_err);
+
+int launch_bwd_fp32(const float* q, const float* k, const float* v, const float* d_o, float* dq, float* dk,
+                    float* dv, const Problem& p, cudaStream_t stream, unsigned long long* launches,
+                    cudaError_t* cuda_err);
+
+int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const Problem& p, int* status,
+                    cudaStream_t stream, unsigned long long* launches, cudaError_t* cuda_err);
+
+int launch_bwd_bf16(const void* q, const void* k, const void* v, const void* d_o, void* dq, void* dk, void* dv,
+                    const Problem& p, void* workspace, int* status, cudaStream_t stream,
+                    unsigned long long* launches, cudaError_t* cuda_err);
+
+size_t bwd_bf16_workspace_bytes(int B, int H, int N, int D);
+
+}  // namespace sigattn

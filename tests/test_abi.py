@@ -1,0 +1,126 @@
+"""Host-only checks of the C-ABI library: it loads without a GPU, exports every symbol
+the header declares, validates arguments before touching a device, and the Python
+binding marshals to the same names."""
+import ctypes
+import math
+import os
+import re
+
+import numpy as np
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "sigattn.h")
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2409_04431_b200 import build
+    build.build()
+    from paper_2409_04431_b200 import binding
+    return binding.lib()
+
+
+def declared_symbols():
+    text = open(HEADER).read()
+    return re.findall(r"SIGATTN_API\s+[\w\s\*]+?\b(sigattn_\w+)\s*\(", text)
+
+
+def test_header_declares_the_boundary():
+    names = declared_symbols()
+    for required in ("sigattn_fwd", "sigattn_bwd", "sigattn_bwd_workspace_bytes", "sigattn_check",
+                     "sigattn_strerror", "sigattn_version"):
+        assert required in names
+
+
+def test_library_exports_every_declared_symbol(lib):
+    from paper_2409_04431_b200 import binding
+    for name in declared_symbols():
+        assert hasattr(lib, name), name
+        assert name in binding.EXPORTED, name
+    raw = ctypes.CDLL(binding.LIB_PATH)
+    for name in declared_symbols():
+        getattr(raw, name)
+
+
+def test_version_and_error_strings(lib):
+    assert lib.sigattn_version() >= 100
+    seen = set()
+    for code in range(0, -9, -1):
+        s = lib.sigattn_strerror(code).decode()
+        assert s and s not in seen
+        seen.add(s)
+    assert "unknown" in lib.sigattn_strerror(-99).decode()
+
+
+def test_workspace_bytes(lib):
+    # fp32 dQ accumulator [B, H, N, D] at least; 0 for the fp32 path and for bad shapes
+    assert lib.sigattn_bwd_workspace_bytes(2, 16, 4096, 128, 0) >= 2 * 16 * 4096 * 128 * 4
+    assert lib.sigattn_bwd_workspace_bytes(2, 16, 4096, 128, 1) == 0
+    assert lib.sigattn_bwd_workspace_bytes(2, 16, 4096, 96, 0) == 0
+    assert lib.sigattn_bwd_workspace_bytes(0, 16, 4096, 128, 0) == 0
+
+
+def test_argument_validation_happens_before_any_device_work(lib):
+    """These calls must return their error codes on a machine without a GPU."""
+    buf = np.zeros(4096, dtype=np.uint8)
+    p = buf.ctypes.data
+    p = (p + 255) & ~255
+    ok = dict(B=1, H=1, N=4, D=64)
+    f = lib.sigattn_fwd
+    assert f(None, p, p, p, 1, 1, 4, 64, 0.125, 0.0, 0, None, 0, None) == -1
+    assert f(p, p, p, None, 1, 1, 4, 64, 0.125, 0.0, 0, None, 0, None) == -1
+    assert f(p, p, p, p, 1, 1, 4, 96, 0.125, 0.0, 0, None, 0, None) == -2
+    assert f(p, p, p, p, 1, 1, 0, 64, 0.125, 0.0, 0, None, 0, None) == -2
+    assert f(p, p, p, p, 0, 1, 4, 64, 0.125, 0.0, 0, None, 0, None) == -2
+    assert f(p, p, p, p, 70000, 1, 4, 64, 0.125, 0.0, 0, None, 0, None) == -2
+    assert f(p + 2, p, p, p, 1, 1, 4, 64, 0.125, 0.0, 0, None, 0, None) == -3
+    assert f(p, p, p, p, 1, 1, 4, 64, 0.125, 0.0, 0, None, 7, None) == -4
+    assert f(p, p, p, p, 1, 1, 4, 64, 0.125, 0.0, 2, None, 0, None) == -4
+    g = lib.sigattn_bwd
+    assert g(p, p, p, p, p, p, None, 1, 1, 4, 64, 0.125, 0.0, 0, None, 0, p, 4096, None) == -1
+    assert g(p, p, p, p, p, p, p, 1, 1, 4, 48, 0.125, 0.0, 0, None, 0, p, 4096, None) == -2
+    assert g(p, p, p, p, p, p, p + 8, 1, 1, 4, 64, 0.125, 0.0, 0, None, 0, p, 4096, None) == -3
+    assert g(p, p, p, p, p, p, p, 1, 1, 4, 64, 0.125, 0.0, 0, None, 0, None, 0, None) == -1      # workspace missing
+    assert g(p, p, p, p, p, p, p, 1, 1, 4, 64, 0.125, 0.0, 0, None, 0, p + 16, 4096, None) == -3  # workspace alignment
+    assert g(p, p, p, p, p, p, p, 1, 1, 4, 64, 0.125, 0.0, 0, None, 0, p, 16, None) == -5
+    assert g(p, p, p, p, p, p, p, 1, 1, 4, 64, 0.125, 0.0, 0, None, 3, p, 4096, None) == -4
+
+
+def test_input_recipes():
+    from paper_2409_04431_b200 import inputs
+    cfg = inputs.CONFIGS["c4"]
+    q, k, v, d_o = inputs.make_inputs(cfg, heads=1, batch=1)
+    assert q.shape == (1, 1, 4096, 128) and q.dtype == np.float32
+    # qk-norm recipe: rows of q, k have L2 norm sqrt(D) up to bf16 rounding
+    np.testing.assert_allclose(np.linalg.norm(q, axis=-1), math.sqrt(128), rtol=2e-3)
+    np.testing.assert_allclose(np.linalg.norm(k, axis=-1), math.sqrt(128), rtol=2e-3)
+    # values are exactly representable in bf16, and the generator is reproducible
+    for t in (q, k, v, d_o):
+        np.testing.assert_array_equal(inputs.round_to_bf16(t), t)
+    q2, *_ = inputs.make_inputs(cfg, heads=1, batch=1)
+    np.testing.assert_array_equal(q, q2)
+    c3 = inputs.CONFIGS["c3"]
+    np.testing.assert_allclose(c3.slopes(), [2.0 ** (-8 * h / 16) for h in range(1, 17)], rtol=1e-6)
+    assert abs(inputs.CONFIGS["c5"].bias + math.log(16384)) < 1e-12
+    # FLOP model: c = (n + 1) / (2 n) equals the unmasked fraction of the n x n matrix
+    n = 37
+    assert inputs.causal_fraction(n, True) == np.tril(np.ones((n, n))).sum() / n ** 2
+    assert cfg.flops_fwd() == 4 * inputs.causal_fraction(4096, True) * 2 * 16 * 4096 ** 2 * 128
+    assert cfg.flops_bwd() == 2.5 * cfg.flops_fwd()
+
+
+def test_bf16_rounding_is_round_to_nearest_even():
+    from paper_2409_04431_b200 import inputs
+    x = np.array([1.0, 1.00390625, 1.01171875, -2.5, 3.14159, 1e-30, 65504.0], dtype=np.float32)
+    bits = inputs.f32_to_bf16_bits(x)
+    back = inputs.bf16_bits_to_f32(bits)
+    # 1 + 2^-8 is a tie between 1 and 1 + 2^-7 -> even mantissa (1.0); 1 + 3*2^-8 -> 1 + 2^-6
+    assert back[1] == 1.0 and back[2] == 1.015625
+    assert np.all(np.abs(back - x) <= np.abs(x) * 2.0 ** -8)
+    try:
+        import torch
+        t = torch.from_numpy(x).to(torch.bfloat16).to(torch.float32).numpy()
+        np.testing.assert_array_equal(back, t)
+    except ImportError:
+        pass

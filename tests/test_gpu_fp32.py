@@ -1,0 +1,49 @@
+"""fp32 debug path (CUDA cores, exact expf) against the float64 oracle, through the C ABI."""
+import math
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2409_04431_b200 import inputs
+from parity_util import assert_fp32_close, to_device, to_host
+
+pytestmark = pytest.mark.gpu
+
+
+def run_case(q, k, v, d_o, scale, bias, causal, slopes):
+    import torch
+    import paper_2409_04431_b200 as sa
+    dq_, dk_, dv_, do_ = (to_device(t, "fp32") for t in (q, k, v, d_o))
+    sl = None if slopes is None else torch.from_numpy(np.asarray(slopes, dtype=np.float32)).cuda()
+    o = sa.sigattn_fwd(dq_, dk_, dv_, scale, bias, causal, sl)
+    gq, gk, gv = sa.sigattn_bwd(dq_, dk_, dv_, do_, scale, bias, causal, sl)
+    sa.sigattn_check()
+    ref_o = oracle.sigattn_fwd(q, k, v, scale, bias, causal, slopes)
+    ref_q, ref_k, ref_v = oracle.sigattn_bwd(q, k, v, d_o, scale, bias, causal, slopes)
+    assert_fp32_close(to_host(o), ref_o, "O")
+    assert_fp32_close(to_host(gq), ref_q, "dQ")
+    assert_fp32_close(to_host(gk), ref_k, "dK")
+    assert_fp32_close(to_host(gv), ref_v, "dV")
+
+
+def test_config1_fp32():
+    cfg = inputs.CONFIGS["c1"]
+    q, k, v, d_o = inputs.make_inputs(cfg)
+    run_case(q, k, v, d_o, cfg.scale, cfg.bias, cfg.causal, cfg.slopes())
+
+
+@pytest.mark.parametrize("N", [1, 2, 63, 129, 300])
+@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("causal", [False, True])
+def test_fp32_edge_shapes(N, D, causal):
+    B, H = 2, 3
+    q, k, v, d_o = inputs.random_case(B, H, N, D, seed=1000 + N + D, dtype="fp32")
+    slopes = np.array([0.5, 0.25, 0.0625], dtype=np.float32) if (N % 2) else None
+    run_case(q, k, v, d_o, 1 / math.sqrt(D), -math.log(max(N, 2)), causal, slopes)
+
+
+@pytest.mark.parametrize("bias", [0.0, -30.0, 30.0])
+def test_fp32_bias_extremes(bias):
+    q, k, v, d_o = inputs.random_case(1, 2, 70, 64, seed=77, dtype="fp32")
+    run_case(q, k, v, d_o, 0.125, bias, True, None)
