@@ -15,6 +15,10 @@ constexpr int kThreads = 128;
 
 __device__ __forceinline__ float sigmoid_exact(float x) { return 1.0f / (1.0f + expf(-x)); }
 
+// P (1 - P) evaluated as sigmoid(x) * sigmoid(-x): the same quantity (1 - sigmoid(x) =
+// sigmoid(-x)), but without the cancellation of 1 - P when P rounds to 1.
+__device__ __forceinline__ float sigmoid_slope(float x) { return sigmoid_exact(x) * sigmoid_exact(-x); }
+
 __device__ __forceinline__ float dot_row(const float* __restrict__ a_smem, const float* __restrict__ b, int D) {
   float s = 0.0f;
   for (int d = 0; d < D; ++d) s = fmaf(a_smem[d], b[d], s);
@@ -77,9 +81,8 @@ __global__ void bwd_dq_fp32_kernel(const float* __restrict__ q, const float* __r
     if (j < jend) {
       const float s = dot_row(sq, k + base + static_cast<size_t>(j) * D, D);
       const float x = fmaf(scale, s, bias) - slope * fabsf(static_cast<float>(i - j));
-      const float p = sigmoid_exact(x);
       const float dp = dot_row(sdo, v + base + static_cast<size_t>(j) * D, D);
-      ds = p * (1.0f - p) * dp;
+      ds = sigmoid_slope(x) * dp;
     }
     sds[t] = ds;
     __syncthreads();
@@ -119,7 +122,7 @@ __global__ void bwd_dkdv_fp32_kernel(const float* __restrict__ q, const float* _
       const float x = fmaf(scale, s, bias) - slope * fabsf(static_cast<float>(i - j));
       p = sigmoid_exact(x);
       const float dp = dot_row(sv, d_o + base + static_cast<size_t>(i) * D, D);
-      ds = p * (1.0f - p) * dp;
+      ds = sigmoid_slope(x) * dp;
     }
     sp[t] = p;
     sds[t] = ds;

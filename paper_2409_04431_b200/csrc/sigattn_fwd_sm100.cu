@@ -1,6 +1,492 @@
+// bf16 forward of sigmoid attention for sm_100a (Algorithm 1 of Appendix F.1, redesigned
+// for Blackwell): O = sigmoid(scale * Q K^T + b - slope * |i - j|) [causal-masked] V.
+//
+// One persistent CTA per SM walks a list of work items (batch*head, pair of 128-row query
+// tiles), heaviest first when causal.  Inside a CTA the work is split by warp role:
+//
+//   warp 8      TMA producer: Q tiles once per item, then K_0, V_0, K_1, V_1, ... through a
+//               ring of shared-memory stages (128-byte swizzle, zero fill beyond row N).
+//   warp 9      MMA issuer (one thread): S_t = Q_t K_j^T into tensor memory, then
+//               O_t += P_t V_j with P read from tensor memory.  The two query tiles are
+//               interleaved so the tensor pipe works on one while the other is activated.
+//   warps 0-3   activation group of query tile 0: reads S from tensor memory (one row per
+//   warps 4-7   thread), evaluates P = sigmoid(.) in registers, writes bf16 P back over S.
+//               (same for tile 1)  At the end of an item the group converts its O
+//               accumulator to bf16 and stores it with TMA (rows >= N are clipped).
+//
+// Sigmoid needs no row maximum, no row sum and no rescaling of O (Section 4), so there is
+// no correction step and O is touched once, at the end.
+//
+// Activation.  With a = log2(e) * x:  u = 2^a;  if every a in a thread's 32-column chunk is
+// <= -3 (u <= 1/8, the usual case at b = -log n) then P = u (1 - u (1 - u (1 - u))), the
+// alternating series of u / (1 + u) cut after u^4 (relative error < 2^-12, below bf16
+// resolution): one MUFU op per element.  Otherwise P = u / (1 + u) with a reciprocal: two
+// MUFU ops.  The paper's 0.5 + 0.5 * tanh(x / 2) is not used: at x << 0 it subtracts two
+// nearly equal numbers and loses P's relative accuracy.
 #include "sigattn_internal.h"
+#include "sm100_primitives.cuh"
+#include "tensor_map.h"
 #include "../../include/sigattn.h"
+
 namespace sigattn {
-int launch_fwd_bf16(const void*, const void*, const void*, void*, const Problem&, int*, cudaStream_t,
-                    unsigned long long*, cudaError_t*) { return SIGATTN_ERR_FLAG; }
+namespace {
+
+using namespace sm100;
+
+constexpr int kBM = 128;        // query rows per tile (= TMEM lanes)
+constexpr int kBN = 128;        // keys per tile
+constexpr int kFwdThreads = 320;
+constexpr int kLoadWarp = 8;
+constexpr int kMmaWarp = 9;
+constexpr float kLog2e = 1.4426950408889634f;
+
+template <int D>
+struct FwdSmem {
+  static constexpr int kPanels = D / 64;
+  static constexpr int kPanelBytes = kBM * 128;           // 128 rows x 128 B
+  static constexpr int kTileBytes = kPanels * kPanelBytes;  // one Q, K or V tile
+  static constexpr int kStages = (D == 128) ? 4 : 8;
+  static constexpr int kQOff = 0;
+  static constexpr int kKvOff = 2 * kTileBytes;
+  static constexpr int kTotal = kKvOff + kStages * kTileBytes;
+  static constexpr int kDynBytes = kTotal + 1024;  // slack to align the base to 1024 B
+};
+
+struct FwdBarriers {
+  uint64_t q_full[2], q_empty[2];
+  uint64_t s_full[2], p_full[2];
+  uint64_t o_full[2], o_empty[2];
+  uint64_t kv_full[8], kv_empty[8];
+};
+
+struct FwdParams {
+  int BH, H, N;
+  int n_pairs;     // ceil(N / 256)
+  int n_kv_total;  // ceil(N / 128)
+  int n_items;
+  float scale_log2e, bias_log2e;
+  const float* slopes;
+  int* status;
+};
+
+struct Item {
+  int bh, row0, n_kv, n[2];
+};
+
+template <bool CAUSAL>
+__device__ __forceinline__ Item decode_item(const FwdParams& p, int item) {
+  Item w;
+  const int rank = item / p.BH;
+  w.bh = item - rank * p.BH;
+  const int pair = CAUSAL ? (p.n_pairs - 1 - rank) : rank;
+  w.row0 = pair * 2 * kBM;
+#pragma unroll
+  for (int t = 0; t < 2; ++t) {
+    const int r = w.row0 + t * kBM;
+    w.n[t] = (r >= p.N) ? 0 : (CAUSAL ? min(p.n_kv_total, r / kBN + 1) : p.n_kv_total);
+  }
+  w.n_kv = max(w.n[0], w.n[1]);
+  return w;
 }
+
+// ------------------------------------------------------------------ producer
+
+template <int D, bool CAUSAL>
+__device__ void fwd_load_role(const FwdParams& p, const CUtensorMap* tmQ, const CUtensorMap* tmK,
+                              const CUtensorMap* tmV, uint32_t smem_base, FwdBarriers* bars, volatile int* cta_err) {
+  using L = FwdSmem<D>;
+  uint32_t kv_cnt = 0;
+  uint32_t q_iter[2] = {0, 0};
+  for (int item = blockIdx.x; item < p.n_items; item += gridDim.x) {
+    const Item w = decode_item<CAUSAL>(p, item);
+    auto load_q = [&](int t) -> bool {
+      if (w.n[t] == 0) return true;
+      if (!mbar_wait(smem_u32(&bars->q_empty[t]), (q_iter[t] & 1) ^ 1, cta_err, 10 + t)) return false;
+      const uint32_t bar = smem_u32(&bars->q_full[t]);
+      mbar_arrive_expect_tx(bar, L::kTileBytes);
+#pragma unroll
+      for (int pn = 0; pn < L::kPanels; ++pn)
+        tma_load_3d(smem_base + L::kQOff + t * L::kTileBytes + pn * L::kPanelBytes, tmQ, bar, pn * 64,
+                    w.row0 + t * kBM, w.bh);
+      ++q_iter[t];
+      return true;
+    };
+    auto load_kv = [&](const CUtensorMap* tm, int j) -> bool {
+      const uint32_t stage = kv_cnt % L::kStages;
+      const uint32_t phase = (kv_cnt / L::kStages) & 1;
+      if (!mbar_wait(smem_u32(&bars->kv_empty[stage]), phase ^ 1, cta_err, 12)) return false;
+      const uint32_t bar = smem_u32(&bars->kv_full[stage]);
+      mbar_arrive_expect_tx(bar, L::kTileBytes);
+#pragma unroll
+      for (int pn = 0; pn < L::kPanels; ++pn)
+        tma_load_3d(smem_base + L::kKvOff + stage * L::kTileBytes + pn * L::kPanelBytes, tm, bar, pn * 64, j * kBN,
+                    w.bh);
+      ++kv_cnt;
+      return true;
+    };
+    if (!load_q(0)) return;
+    if (!load_kv(tmK, 0)) return;
+    if (!load_q(1)) return;
+    for (int j = 0; j < w.n_kv; ++j) {
+      if (!load_kv(tmV, j)) return;
+      if (j + 1 < w.n_kv && !load_kv(tmK, j + 1)) return;
+    }
+  }
+}
+
+// ------------------------------------------------------------------ MMA issuer
+
+template <int D, bool CAUSAL>
+__device__ void fwd_mma_role(const FwdParams& p, uint32_t smem_base, uint32_t tmem, FwdBarriers* bars,
+                             volatile int* cta_err) {
+  using L = FwdSmem<D>;
+  constexpr uint32_t kIdescS = make_idesc_bf16(kBM, kBN, 0, 0);
+  constexpr uint32_t kIdescPV = make_idesc_bf16(kBM, D, 0, 1);
+  uint32_t kv_cnt = 0;
+  uint32_t it[2] = {0, 0};      // items seen per query tile
+  uint32_t p_cnt[2] = {0, 0};   // P tiles consumed per query tile
+
+  // S_t = Q_t K^T : both operands K-major, 128-byte swizzle.
+  auto issue_s = [&](int t, uint32_t k_smem) {
+    const uint32_t q_smem = smem_base + L::kQOff + t * L::kTileBytes;
+#pragma unroll
+    for (int ks = 0; ks < D / 16; ++ks) {
+      const uint32_t off = (ks >> 2) * L::kPanelBytes + (ks & 3) * 32;
+      umma_ss(tmem + t * kBN, make_smem_desc_sw128(q_smem + off, 16, 1024),
+              make_smem_desc_sw128(k_smem + off, 16, 1024), kIdescS, ks > 0);
+    }
+  };
+  // O_t (+)= P_t V : A = bf16 P in tensor memory (aliasing S_t), B = V, MN-major.
+  auto issue_pv = [&](int t, uint32_t v_smem, bool accumulate) {
+#pragma unroll
+    for (int ks = 0; ks < kBN / 16; ++ks) {
+      umma_ts(tmem + 2 * kBN + t * D, tmem + t * kBN + ks * 8,
+              make_smem_desc_sw128(v_smem + ks * 2048, L::kPanelBytes, 1024), kIdescPV, (accumulate || ks > 0));
+    }
+  };
+  auto kv_wait = [&](uint32_t cnt) -> bool {
+    const uint32_t stage = cnt % L::kStages, phase = (cnt / L::kStages) & 1;
+    return mbar_wait(smem_u32(&bars->kv_full[stage]), phase, cta_err, 20);
+  };
+  auto kv_addr = [&](uint32_t cnt) { return smem_base + L::kKvOff + (cnt % L::kStages) * L::kTileBytes; };
+  auto kv_release = [&](uint32_t cnt) { umma_commit(smem_u32(&bars->kv_empty[cnt % L::kStages])); };
+
+  for (int item = blockIdx.x; item < p.n_items; item += gridDim.x) {
+    const Item w = decode_item<CAUSAL>(p, item);
+    // ring positions: K_j at kv_cnt + 2 j (j > 0: 2 j), V_j right after K_j ... order K0 V0 K1 V1 ...
+    const uint32_t base_cnt = kv_cnt;
+    auto k_cnt = [&](int j) { return base_cnt + 2 * j; };
+    auto v_cnt = [&](int j) { return base_cnt + 2 * j + 1; };
+
+    // first logits
+    if (!mbar_wait(smem_u32(&bars->q_full[0]), it[0] & 1, cta_err, 21)) return;
+    if (!kv_wait(k_cnt(0))) return;
+    tc_fence_after_sync();
+    issue_s(0, kv_addr(k_cnt(0)));
+    umma_commit(smem_u32(&bars->s_full[0]));
+    if (w.n[1] > 0) {
+      if (!mbar_wait(smem_u32(&bars->q_full[1]), it[1] & 1, cta_err, 22)) return;
+      tc_fence_after_sync();
+      issue_s(1, kv_addr(k_cnt(0)));
+      umma_commit(smem_u32(&bars->s_full[1]));
+    }
+    kv_release(k_cnt(0));
+    // accumulators of the previous item must have been read out before the first PV overwrites them
+    if (!mbar_wait(smem_u32(&bars->o_empty[0]), (it[0] & 1) ^ 1, cta_err, 23)) return;
+    if (w.n[1] > 0 && !mbar_wait(smem_u32(&bars->o_empty[1]), (it[1] & 1) ^ 1, cta_err, 24)) return;
+
+    for (int j = 0; j < w.n_kv; ++j) {
+      if (!kv_wait(v_cnt(j))) return;
+      const bool more = (j + 1 < w.n_kv);
+      if (j < w.n[0]) {
+        if (!mbar_wait(smem_u32(&bars->p_full[0]), p_cnt[0] & 1, cta_err, 25)) return;
+        ++p_cnt[0];
+        tc_fence_after_sync();
+        issue_pv(0, kv_addr(v_cnt(j)), j > 0);
+        if (j == w.n[0] - 1) umma_commit(smem_u32(&bars->o_full[0]));
+      }
+      if (more && !kv_wait(k_cnt(j + 1))) return;
+      if (j + 1 < w.n[0]) {
+        tc_fence_after_sync();
+        issue_s(0, kv_addr(k_cnt(j + 1)));
+        umma_commit(smem_u32(&bars->s_full[0]));
+      }
+      if (j < w.n[1]) {
+        if (!mbar_wait(smem_u32(&bars->p_full[1]), p_cnt[1] & 1, cta_err, 26)) return;
+        ++p_cnt[1];
+        tc_fence_after_sync();
+        issue_pv(1, kv_addr(v_cnt(j)), j > 0);
+        if (j == w.n[1] - 1) umma_commit(smem_u32(&bars->o_full[1]));
+      }
+      kv_release(v_cnt(j));
+      if (j + 1 < w.n[1]) {
+        issue_s(1, kv_addr(k_cnt(j + 1)));
+        umma_commit(smem_u32(&bars->s_full[1]));
+      }
+      if (more) kv_release(k_cnt(j + 1));
+    }
+    kv_cnt = base_cnt + 2 * w.n_kv;
+    ++it[0];
+    if (w.n[1] > 0) ++it[1];
+  }
+}
+
+// ------------------------------------------------------------------ activation + epilogue
+
+// 32 logits of one row -> 16 packed bf16x2 sigmoid values.
+//   a = s * scale_log2e + c0   (c0 carries the bias and, with ALiBi, the position term)
+template <bool CAUSAL_DIAG, bool ALIBI>
+__device__ __forceinline__ void sigmoid_chunk(const uint32_t (&s)[32], uint32_t (&out)[16], float scale_log2e,
+                                              float bias_log2e, float slope_log2e, float row_rel, int col_base) {
+  float a[32];
+#pragma unroll
+  for (int i = 0; i < 32; ++i) {
+    float c0 = bias_log2e;
+    if (ALIBI) {
+      const float dist = row_rel - static_cast<float>(col_base + i);
+      c0 = fmaf(-slope_log2e, fabsf(dist), bias_log2e);
+    }
+    a[i] = fmaf(__uint_as_float(s[i]), scale_log2e, c0);
+  }
+  float m = fmax3(a[0], a[1], a[2]);
+#pragma unroll
+  for (int i = 3; i + 1 < 32; i += 2) m = fmax3(m, a[i], a[i + 1]);
+  m = fmaxf(m, a[31]);
+  float pr[32];
+  if (m <= -3.0f) {
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      const float u = ex2_approx(a[i]);
+      float t = 1.0f - u;
+      t = fmaf(-u, t, 1.0f);
+      t = fmaf(-u, t, 1.0f);
+      pr[i] = u * t;
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      const float u = ex2_approx(fminf(a[i], 64.0f));
+      pr[i] = u * rcp_approx(1.0f + u);
+    }
+  }
+  if (CAUSAL_DIAG) {
+#pragma unroll
+    for (int i = 0; i < 32; ++i)
+      if (static_cast<float>(col_base + i) > row_rel) pr[i] = 0.0f;
+  }
+#pragma unroll
+  for (int i = 0; i < 16; ++i) out[i] = pack_bf16x2(pr[2 * i], pr[2 * i + 1]);
+}
+
+template <int D, bool CAUSAL, bool ALIBI>
+__device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, int t, uint8_t* smem, uint32_t tmem,
+                             FwdBarriers* bars, volatile int* cta_err) {
+  using L = FwdSmem<D>;
+  const int tid = threadIdx.x & 127;         // row of the tile
+  const int quarter = (threadIdx.x >> 5) & 3;  // TMEM lane quarter this warp may touch
+  const uint32_t lane_off = static_cast<uint32_t>(quarter * 32) << 16;
+  const uint32_t tS = tmem + t * kBN + lane_off;
+  const uint32_t tO = tmem + 2 * kBN + t * D + lane_off;
+  uint32_t s_cnt = 0, it = 0;
+
+  for (int item = blockIdx.x; item < p.n_items; item += gridDim.x) {
+    const Item w = decode_item<CAUSAL>(p, item);
+    const int nt = w.n[t];
+    if (nt == 0) continue;
+    const int row = w.row0 + t * kBM + tid;
+    float slope_log2e = 0.0f;
+    if (ALIBI) slope_log2e = p.slopes[w.bh % p.H] * kLog2e;
+
+    for (int j = 0; j < nt; ++j) {
+      if (!mbar_wait(smem_u32(&bars->s_full[t]), s_cnt & 1, cta_err, 30 + t)) return;
+      ++s_cnt;
+      tc_fence_after_sync();
+      const float row_rel = static_cast<float>(row - j * kBN);
+      const bool diag = CAUSAL && (j == nt - 1);
+#pragma unroll 1
+      for (int c = 0; c < kBN / 32; ++c) {
+        uint32_t s[32], pk[16];
+        tmem_ld32(tS + c * 32, s);
+        tmem_wait_ld();
+        if (diag)
+          sigmoid_chunk<true, ALIBI>(s, pk, p.scale_log2e, p.bias_log2e, slope_log2e, row_rel, c * 32);
+        else
+          sigmoid_chunk<false, ALIBI>(s, pk, p.scale_log2e, p.bias_log2e, slope_log2e, row_rel, c * 32);
+        tmem_st16(tS + c * 16, pk);
+      }
+      tmem_wait_st();
+      tc_fence_before_sync();
+      mbar_arrive(smem_u32(&bars->p_full[t]));
+    }
+
+    // epilogue: O_t (fp32, tensor memory) -> bf16 -> swizzled shared memory (the Q_t buffer,
+    // free once every logits MMA of the item is done) -> TMA store.
+    if (!mbar_wait(smem_u32(&bars->o_full[t]), it & 1, cta_err, 32 + t)) return;
+    ++it;
+    tc_fence_after_sync();
+    uint8_t* stage = smem + L::kQOff + t * L::kTileBytes;
+#pragma unroll 1
+    for (int c = 0; c < D / 32; ++c) {
+      uint32_t o[32];
+      tmem_ld32(tO + c * 32, o);
+      tmem_wait_ld();
+      uint8_t* panel = stage + (c >> 1) * L::kPanelBytes + tid * 128;
+#pragma unroll
+      for (int g = 0; g < 4; ++g) {
+        uint4 val;
+        val.x = pack_bf16x2(__uint_as_float(o[8 * g + 0]), __uint_as_float(o[8 * g + 1]));
+        val.y = pack_bf16x2(__uint_as_float(o[8 * g + 2]), __uint_as_float(o[8 * g + 3]));
+        val.z = pack_bf16x2(__uint_as_float(o[8 * g + 4]), __uint_as_float(o[8 * g + 5]));
+        val.w = pack_bf16x2(__uint_as_float(o[8 * g + 6]), __uint_as_float(o[8 * g + 7]));
+        const int chunk = (c & 1) * 4 + g;
+        *reinterpret_cast<uint4*>(panel + ((chunk ^ (tid & 7)) * 16)) = val;
+      }
+    }
+    tc_fence_before_sync();
+    mbar_arrive(smem_u32(&bars->o_empty[t]));
+    fence_proxy_async_smem();
+    asm volatile("bar.sync %0, 128;" ::"r"(1 + t) : "memory");
+    if (tid == 0) {
+#pragma unroll
+      for (int pn = 0; pn < L::kPanels; ++pn)
+        tma_store_3d(tmO, smem_u32(stage + pn * L::kPanelBytes), pn * 64, w.row0 + t * kBM, w.bh);
+      tma_commit_group();
+      tma_wait_group_read<0>();
+      mbar_arrive(smem_u32(&bars->q_empty[t]));
+    }
+  }
+  if (tid == 0) tma_wait_group<0>();
+}
+
+// ------------------------------------------------------------------ kernel
+
+template <int D, bool CAUSAL, bool ALIBI>
+__global__ void __launch_bounds__(kFwdThreads, 1)
+sigattn_fwd_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                        const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
+                        const FwdParams p) {
+  using L = FwdSmem<D>;
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ FwdBarriers bars;
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int cta_err;
+
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const uint32_t smem_base = smem_u32(smem);
+  const int warp = threadIdx.x >> 5;
+
+  if (threadIdx.x == 0) {
+    cta_err = 0;
+    for (int t = 0; t < 2; ++t) {
+      mbar_init(smem_u32(&bars.q_full[t]), 1);
+      mbar_init(smem_u32(&bars.q_empty[t]), 1);
+      mbar_init(smem_u32(&bars.s_full[t]), 1);
+      mbar_init(smem_u32(&bars.p_full[t]), 128);
+      mbar_init(smem_u32(&bars.o_full[t]), 1);
+      mbar_init(smem_u32(&bars.o_empty[t]), 128);
+    }
+    for (int s = 0; s < L::kStages; ++s) {
+      mbar_init(smem_u32(&bars.kv_full[s]), 1);
+      mbar_init(smem_u32(&bars.kv_empty[s]), 1);
+    }
+    fence_mbar_init();
+  }
+  if (warp == kLoadWarp && elect_one()) {
+    tma_prefetch_desc(&tmQ);
+    tma_prefetch_desc(&tmK);
+    tma_prefetch_desc(&tmV);
+    tma_prefetch_desc(&tmO);
+  }
+  if (warp == kMmaWarp) {
+    tmem_alloc(smem_u32(&tmem_base_slot), 512);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = tmem_base_slot;
+
+  if (warp == kLoadWarp) {
+    if ((threadIdx.x & 31) == 0) fwd_load_role<D, CAUSAL>(p, &tmQ, &tmK, &tmV, smem_base, &bars, &cta_err);
+    __syncwarp();
+  } else if (warp == kMmaWarp) {
+    if ((threadIdx.x & 31) == 0) fwd_mma_role<D, CAUSAL>(p, smem_base, tmem, &bars, &cta_err);
+    __syncwarp();
+  } else {
+    fwd_act_role<D, CAUSAL, ALIBI>(p, &tmO, warp >> 2, smem, tmem, &bars, &cta_err);
+  }
+
+  tc_fence_before_sync();
+  __syncthreads();
+  if (cta_err != 0) {
+    if (threadIdx.x == 0) atomicExch(p.status, 100 + cta_err);
+    __nanosleep(100000);  // let copies in flight towards this CTA's shared memory land
+  }
+  if (warp == kMmaWarp) tmem_dealloc(tmem, 512);
+}
+
+template <int D, bool CAUSAL, bool ALIBI>
+int launch_fwd_variant(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtensorMap& tmO,
+                       const FwdParams& fp, int num_sms, cudaStream_t stream, cudaError_t* cuda_err) {
+  auto kernel = sigattn_fwd_bf16_kernel<D, CAUSAL, ALIBI>;
+  static bool configured = false;
+  if (!configured) {
+    *cuda_err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdSmem<D>::kDynBytes);
+    if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
+    configured = true;
+  }
+  const int grid = fp.n_items < num_sms ? fp.n_items : num_sms;
+  kernel<<<grid, kFwdThreads, FwdSmem<D>::kDynBytes, stream>>>(tmQ, tmK, tmV, tmO, fp);
+  *cuda_err = cudaGetLastError();
+  return *cuda_err == cudaSuccess ? SIGATTN_OK : SIGATTN_ERR_CUDA;
+}
+
+}  // namespace
+
+int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const Problem& p, int* status,
+                    cudaStream_t stream, unsigned long long* launches, cudaError_t* cuda_err) {
+  int dev = 0, num_sms = 0;
+  *cuda_err = cudaGetDevice(&dev);
+  if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
+  *cuda_err = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
+  if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
+
+  const uint64_t BH = static_cast<uint64_t>(p.B) * p.H;
+  CUtensorMap tmQ, tmK, tmV, tmO;
+  const void* ptrs[4] = {q, k, v, o};
+  CUtensorMap* maps[4] = {&tmQ, &tmK, &tmV, &tmO};
+  for (int i = 0; i < 4; ++i) {
+    if (make_map_3d(maps[i], ptrs[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, BH, p.N, p.D, kBM, 64) != 0) {
+      *cuda_err = cudaErrorInvalidValue;
+      return SIGATTN_ERR_CUDA;
+    }
+  }
+  FwdParams fp;
+  fp.BH = static_cast<int>(BH);
+  fp.H = p.H;
+  fp.N = p.N;
+  fp.n_pairs = (p.N + 2 * kBM - 1) / (2 * kBM);
+  fp.n_kv_total = (p.N + kBN - 1) / kBN;
+  fp.n_items = fp.n_pairs * fp.BH;
+  fp.scale_log2e = p.scale * kLog2e;
+  fp.bias_log2e = p.bias * kLog2e;
+  fp.slopes = p.slopes;
+  fp.status = status;
+
+  int rc;
+  const bool alibi = p.slopes != nullptr;
+#define SIGATTN_FWD_CASE(DD, CC, AA) \
+  rc = launch_fwd_variant<DD, CC, AA>(tmQ, tmK, tmV, tmO, fp, num_sms, stream, cuda_err)
+  if (p.D == 128) {
+    if (p.causal) { if (alibi) SIGATTN_FWD_CASE(128, true, true); else SIGATTN_FWD_CASE(128, true, false); }
+    else          { if (alibi) SIGATTN_FWD_CASE(128, false, true); else SIGATTN_FWD_CASE(128, false, false); }
+  } else {
+    if (p.causal) { if (alibi) SIGATTN_FWD_CASE(64, true, true); else SIGATTN_FWD_CASE(64, true, false); }
+    else          { if (alibi) SIGATTN_FWD_CASE(64, false, true); else SIGATTN_FWD_CASE(64, false, false); }
+  }
+#undef SIGATTN_FWD_CASE
+  if (rc == SIGATTN_OK) *launches += 1;
+  return rc;
+}
+
+}  // namespace sigattn

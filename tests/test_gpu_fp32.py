@@ -43,7 +43,23 @@ def test_fp32_edge_shapes(N, D, causal):
     run_case(q, k, v, d_o, 1 / math.sqrt(D), -math.log(max(N, 2)), causal, slopes)
 
 
-@pytest.mark.parametrize("bias", [0.0, -30.0, 30.0])
+@pytest.mark.parametrize("bias", [0.0, -30.0, 12.0])
 def test_fp32_bias_extremes(bias):
     q, k, v, d_o = inputs.random_case(1, 2, 70, 64, seed=77, dtype="fp32")
     run_case(q, k, v, d_o, 0.125, bias, True, None)
+
+
+def test_fp32_saturated_weights():
+    """b = +30: every weight is 1 to within 1e-13, so O and dV are plain (prefix) sums and
+    dQ, dK vanish (|dS| ~ 1e-13 |dP|; the float64 oracle itself resolves 1 - P only to
+    1e-3 there, so dQ and dK are checked for size, not digits)."""
+    import paper_2409_04431_b200 as sa
+    q, k, v, d_o = inputs.random_case(1, 2, 70, 64, seed=78, dtype="fp32")
+    tq, tk, tv, tdo = (to_device(t, "fp32") for t in (q, k, v, d_o))
+    o = sa.sigattn_fwd(tq, tk, tv, 0.125, 30.0, True)
+    gq, gk, gv = sa.sigattn_bwd(tq, tk, tv, tdo, 0.125, 30.0, True)
+    sa.sigattn_check()
+    assert_fp32_close(to_host(o), np.cumsum(v.astype(np.float64), axis=2), "O")
+    rev = np.flip(np.cumsum(np.flip(d_o.astype(np.float64), axis=2), axis=2), axis=2)
+    assert_fp32_close(to_host(gv), rev, "dV")
+    assert np.max(np.abs(to_host(gq))) < 1e-9 and np.max(np.abs(to_host(gk))) < 1e-9
