@@ -1,7 +1,630 @@
+// bf16 backward of sigmoid attention for sm_100a (Algorithm 2 of Appendix F.1, redesigned
+// for Blackwell).  Per (batch*head, 128-key tile j) work item, looping over query tiles i:
+//
+//     S^T  = K_j Q_i^T                      (tensor memory region A, fp32)
+//     P^T  = sigmoid(scale S^T + b ...)     (registers -> bf16 over region A)
+//     dV_j += P^T dO_i                      (A operand from tensor memory)
+//     dP^T = V_j dO_i^T                     (region B)
+//     dS^T = P^T (1 - P^T) dP^T             (registers -> bf16 in shared memory)
+//     dK_j += dS^T Q_i
+//     dQ_i  = dS K_j                        (region B again, then fp32 reduce-add to HBM)
+//
+// Everything is kept transposed (keys on the 128 TMEM lanes, queries along columns) so
+// that P^T can feed the dV product straight from tensor memory and one shared-memory
+// copy of dS^T serves both dK (as a K-major A operand) and dQ (as an MN-major A operand).
+// No row statistic of any kind is read or written: dS is a point-wise function of S and
+// dP (Section 4 / Appendix F.1), and P is recomputed from Q and K alone.
+//
+// dK_j and dV_j stay in tensor memory across the whole query loop.  dQ_i is complete only
+// after all key tiles have contributed, so each CTA adds its fp32 partial tile into a
+// [B, H, N, D] fp32 workspace with TMA reduce-add; the workspace is zeroed before and
+// converted to bf16 (times scale) after the main kernel: the two helper steps that
+// survive from the paper's backward.  scale is also folded into dK's epilogue.
+//
+// Warp roles (448 threads): warps 0-7 two activation groups (query columns 0-63 and
+// 64-127 of the tile; every thread owns one key row), warps 8-11 dQ drain group,
+// warp 12 TMA producer, warp 13 MMA issuer.
 #include "sigattn_internal.h"
+#include "sm100_primitives.cuh"
+#include "tensor_map.h"
 #include "../../include/sigattn.h"
+
 namespace sigattn {
-int launch_bwd_bf16(const void*, const void*, const void*, const void*, void*, void*, void*, const Problem&, void*,
-                    int*, cudaStream_t, unsigned long long*, cudaError_t*) { return SIGATTN_ERR_FLAG; }
-size_t bwd_bf16_workspace_bytes(int B, int H, int N, int D) { return (size_t)B * H * N * D * 4; }
+namespace {
+
+using namespace sm100;
+
+constexpr int kT = 128;  // tile edge: keys per item (TMEM lanes) and queries per step
+constexpr int kBwdThreads = 448;
+constexpr int kBwdLoadWarp = 12;
+constexpr int kBwdMmaWarp = 13;
+constexpr float kLog2eB = 1.4426950408889634f;
+
+template <int D>
+struct BwdSmem {
+  static constexpr int kPanels = D / 64;
+  static constexpr int kPanelBytes = kT * 128;
+  static constexpr int kTileBytes = kPanels * kPanelBytes;  // a K, V, Q or dO tile
+  static constexpr int kKOff = 0;
+  static constexpr int kVOff = kTileBytes;
+  static constexpr int kQOff = 2 * kTileBytes;              // two stages
+  static constexpr int kDoOff = 4 * kTileBytes;             // one stage
+  static constexpr int kDsOff = 5 * kTileBytes;             // dS^T, 128 x 128 bf16 = two panels
+  static constexpr int kDqOff = kDsOff + 2 * kPanelBytes;   // two fp32 staging boxes of 128 x 32
+  static constexpr int kTotal = kDqOff + 2 * kPanelBytes;
+  static constexpr int kDynBytes = kTotal + 1024;
+};
+
+struct BwdBarriers {
+  uint64_t kv_full, kv_empty;
+  uint64_t q_full[2], q_empty[2];
+  uint64_t do_full, do_empty;
+  uint64_t s_full, dp_full;
+  uint64_t p_ready, ds_ready;
+  uint64_t dq_full, dq_empty;
+  uint64_t dkv_full, dkv_empty;
+};
+
+struct BwdParams {
+  int BH, H, N;
+  int n_tiles;  // ceil(N / 128), for keys and for queries
+  int n_items;
+  float scale, scale_log2e, bias_log2e;
+  const float* slopes;
+  int* status;
+};
+
+struct BwdItem {
+  int bh, j, i_begin, n;
+};
+
+template <bool CAUSAL>
+__device__ __forceinline__ BwdItem decode_bwd_item(const BwdParams& p, int item) {
+  BwdItem w;
+  w.j = item / p.BH;  // ascending key tile = descending work when causal
+  w.bh = item - w.j * p.BH;
+  w.i_begin = CAUSAL ? w.j : 0;
+  w.n = p.n_tiles - w.i_begin;
+  return w;
 }
+
+// TMEM column map (fp32 columns): region A = S^T / P^T, region B = dP^T / dQ.
+template <int D>
+struct BwdTmem {
+  static constexpr uint32_t kA = 0;
+  static constexpr uint32_t kB = 128;
+  static constexpr uint32_t kDv = 256;
+  static constexpr uint32_t kDk = 256 + D;
+};
+
+// ------------------------------------------------------------------ producer
+
+template <int D, bool CAUSAL>
+__device__ void bwd_load_role(const BwdParams& p, const CUtensorMap* tmQ, const CUtensorMap* tmK,
+                              const CUtensorMap* tmV, const CUtensorMap* tmDo, uint32_t smem_base,
+                              BwdBarriers* bars, volatile int* cta_err) {
+  using L = BwdSmem<D>;
+  uint32_t q_cnt = 0, do_cnt = 0, item_cnt = 0;
+  auto load_tile = [&](const CUtensorMap* tm, uint32_t dst, uint32_t bar, int row, int bh) {
+#pragma unroll
+    for (int pn = 0; pn < L::kPanels; ++pn) tma_load_3d(dst + pn * L::kPanelBytes, tm, bar, pn * 64, row, bh);
+  };
+  auto load_q = [&](int i, int bh) -> bool {
+    const uint32_t st = q_cnt & 1, ph = (q_cnt >> 1) & 1;
+    if (!mbar_wait(smem_u32(&bars->q_empty[st]), ph ^ 1, cta_err, 40)) return false;
+    const uint32_t bar = smem_u32(&bars->q_full[st]);
+    mbar_arrive_expect_tx(bar, L::kTileBytes);
+    load_tile(tmQ, smem_base + L::kQOff + st * L::kTileBytes, bar, i * kT, bh);
+    ++q_cnt;
+    return true;
+  };
+  auto load_do = [&](int i, int bh) -> bool {
+    if (!mbar_wait(smem_u32(&bars->do_empty), (do_cnt & 1) ^ 1, cta_err, 41)) return false;
+    const uint32_t bar = smem_u32(&bars->do_full);
+    mbar_arrive_expect_tx(bar, L::kTileBytes);
+    load_tile(tmDo, smem_base + L::kDoOff, bar, i * kT, bh);
+    ++do_cnt;
+    return true;
+  };
+  for (int item = blockIdx.x; item < p.n_items; item += gridDim.x) {
+    const BwdItem w = decode_bwd_item<CAUSAL>(p, item);
+    if (!load_q(w.i_begin, w.bh)) return;
+    if (!load_do(w.i_begin, w.bh)) return;
+    if (!mbar_wait(smem_u32(&bars->kv_empty), (item_cnt & 1) ^ 1, cta_err, 42)) return;
+    {
+      const uint32_t bar = smem_u32(&bars->kv_full);
+      mbar_arrive_expect_tx(bar, 2 * L::kTileBytes);
+      load_tile(tmK, smem_base + L::kKOff, bar, w.j * kT, w.bh);
+      load_tile(tmV, smem_base + L::kVOff, bar, w.j * kT, w.bh);
+    }
+    ++item_cnt;
+    for (int it = 1; it < w.n; ++it) {
+      if (!load_q(w.i_begin + it, w.bh)) return;
+      if (!load_do(w.i_begin + it, w.bh)) return;
+    }
+  }
+}
+
+// ------------------------------------------------------------------ MMA issuer
+
+template <int D, bool CAUSAL>
+__device__ void bwd_mma_role(const BwdParams& p, uint32_t smem_base, uint32_t tmem, BwdBarriers* bars,
+                             volatile int* cta_err) {
+  using L = BwdSmem<D>;
+  using TM = BwdTmem<D>;
+  constexpr uint32_t kIdescSt = make_idesc_bf16(kT, kT, 0, 0);   // S^T, dP^T : K-major x K-major
+  constexpr uint32_t kIdescAcc = make_idesc_bf16(kT, D, 0, 1);   // dV, dK   : (TMEM | K-major) x MN-major
+  constexpr uint32_t kIdescDq = make_idesc_bf16(kT, D, 1, 1);    // dQ       : MN-major x MN-major
+  const uint32_t sK = smem_base + L::kKOff, sV = smem_base + L::kVOff, sDo = smem_base + L::kDoOff,
+                 sDs = smem_base + L::kDsOff;
+  uint32_t q_cnt = 0, do_cnt = 0, item_cnt = 0, step_cnt = 0;
+
+  // [128 x 128] = X[128 x D] * Y[128 x D]^T, both K-major
+  auto issue_kk = [&](uint32_t d_col, uint32_t x, uint32_t y) {
+#pragma unroll
+    for (int ks = 0; ks < D / 16; ++ks) {
+      const uint32_t off = (ks >> 2) * L::kPanelBytes + (ks & 3) * 32;
+      umma_ss(tmem + d_col, make_smem_desc_sw128(x + off, 16, 1024), make_smem_desc_sw128(y + off, 16, 1024),
+              kIdescSt, ks > 0);
+    }
+  };
+
+  for (int item = blockIdx.x; item < p.n_items; item += gridDim.x) {
+    const BwdItem w = decode_bwd_item<CAUSAL>(p, item);
+    if (!mbar_wait(smem_u32(&bars->kv_full), item_cnt & 1, cta_err, 50)) return;
+
+    // prologue: S^T(0), dP^T(0)
+    {
+      const uint32_t st = q_cnt & 1, ph = (q_cnt >> 1) & 1;
+      if (!mbar_wait(smem_u32(&bars->q_full[st]), ph, cta_err, 51)) return;
+      tc_fence_after_sync();
+      issue_kk(TM::kA, sK, smem_base + L::kQOff + st * L::kTileBytes);
+      umma_commit(smem_u32(&bars->s_full));
+      if (!mbar_wait(smem_u32(&bars->do_full), do_cnt & 1, cta_err, 52)) return;
+      if (!mbar_wait(smem_u32(&bars->dq_empty), (step_cnt & 1) ^ 1, cta_err, 53)) return;
+      tc_fence_after_sync();
+      issue_kk(TM::kB, sV, sDo);
+      umma_commit(smem_u32(&bars->dp_full));
+    }
+    for (int it = 0; it < w.n; ++it) {
+      const uint32_t st = q_cnt & 1;
+      const uint32_t sQ = smem_base + L::kQOff + st * L::kTileBytes;
+      const bool more = (it + 1 < w.n);
+      // dV += P^T dO_i
+      if (!mbar_wait(smem_u32(&bars->p_ready), step_cnt & 1, cta_err, 54)) return;
+      if (it == 0 && !mbar_wait(smem_u32(&bars->dkv_empty), (item_cnt & 1) ^ 1, cta_err, 55)) return;
+      tc_fence_after_sync();
+#pragma unroll
+      for (int ks = 0; ks < kT / 16; ++ks) {
+        umma_ts(tmem + TM::kDv, tmem + TM::kA + (ks >> 2) * 64 + (ks & 3) * 8,
+                make_smem_desc_sw128(sDo + ks * 2048, L::kPanelBytes, 1024), kIdescAcc, (it > 0 || ks > 0));
+      }
+      umma_commit(smem_u32(&bars->do_empty));
+      ++do_cnt;
+      // S^T of the next query tile
+      if (more) {
+        const uint32_t nst = (q_cnt + 1) & 1, nph = ((q_cnt + 1) >> 1) & 1;
+        if (!mbar_wait(smem_u32(&bars->q_full[nst]), nph, cta_err, 56)) return;
+        tc_fence_after_sync();
+        issue_kk(TM::kA, sK, smem_base + L::kQOff + nst * L::kTileBytes);
+        umma_commit(smem_u32(&bars->s_full));
+      }
+      // dK += dS^T Q_i ; dQ_i = dS K_j
+      if (!mbar_wait(smem_u32(&bars->ds_ready), step_cnt & 1, cta_err, 57)) return;
+      tc_fence_after_sync();
+#pragma unroll
+      for (int ks = 0; ks < kT / 16; ++ks) {
+        umma_ss(tmem + TM::kDk,
+                make_smem_desc_sw128(sDs + (ks >> 2) * L::kPanelBytes + (ks & 3) * 32, 16, 1024),
+                make_smem_desc_sw128(sQ + ks * 2048, L::kPanelBytes, 1024), kIdescAcc, (it > 0 || ks > 0));
+      }
+      umma_commit(smem_u32(&bars->q_empty[st]));
+      ++q_cnt;
+#pragma unroll
+      for (int ks = 0; ks < kT / 16; ++ks) {
+        umma_ss(tmem + TM::kB, make_smem_desc_sw128(sDs + ks * 2048, L::kPanelBytes, 1024),
+                make_smem_desc_sw128(sK + ks * 2048, L::kPanelBytes, 1024), kIdescDq, ks > 0);
+      }
+      umma_commit(smem_u32(&bars->dq_full));
+      ++step_cnt;
+      // dP^T of the next query tile (region B must have been drained of dQ_i first)
+      if (more) {
+        if (!mbar_wait(smem_u32(&bars->do_full), do_cnt & 1, cta_err, 58)) return;
+        if (!mbar_wait(smem_u32(&bars->dq_empty), (step_cnt & 1) ^ 1, cta_err, 59)) return;
+        tc_fence_after_sync();
+        issue_kk(TM::kB, sV, sDo);
+        umma_commit(smem_u32(&bars->dp_full));
+      }
+    }
+    umma_commit(smem_u32(&bars->dkv_full));
+    ++item_cnt;
+  }
+}
+
+// ------------------------------------------------------------------ activation groups
+
+// 32 logits (transposed tile: this thread's key against 32 queries) -> P as bf16x2 for
+// the dV product and P (1 - P) in fp32 for dS.
+//   a = log2(e) * (scale * s + b - slope * |i - j|);  u = 2^a;  P = u / (1 + u);  1 - P = 1 / (1 + u)
+template <bool DIAG, bool ALIBI>
+__device__ __forceinline__ void bwd_sigmoid_chunk(const uint32_t (&s)[32], uint32_t (&p_out)[16], float* pp,
+                                                  float scale_log2e, float bias_log2e, float slope_log2e,
+                                                  float col_rel, int q_base) {
+  float a[32];
+#pragma unroll
+  for (int e = 0; e < 32; ++e) {
+    float c0 = bias_log2e;
+    if (ALIBI) c0 = fmaf(-slope_log2e, fabsf(static_cast<float>(q_base + e) - col_rel), bias_log2e);
+    a[e] = fmaf(__uint_as_float(s[e]), scale_log2e, c0);
+  }
+  float m = fmax3(a[0], a[1], a[2]);
+#pragma unroll
+  for (int e = 3; e + 1 < 32; e += 2) m = fmax3(m, a[e], a[e + 1]);
+  m = fmaxf(m, a[31]);
+  float pr[32];
+  if (m <= -3.0f) {
+#pragma unroll
+    for (int e = 0; e < 32; ++e) {
+      const float u = ex2_approx(a[e]);
+      float t = 1.0f - u;
+      t = fmaf(-u, t, 1.0f);
+      t = fmaf(-u, t, 1.0f);  // t ~ 1 / (1 + u)
+      pr[e] = u * t;
+      pp[e] = pr[e] * t;
+    }
+  } else {
+#pragma unroll
+    for (int e = 0; e < 32; ++e) {
+      const float u = ex2_approx(fminf(a[e], 64.0f));
+      const float r = rcp_approx(1.0f + u);
+      pr[e] = u * r;
+      pp[e] = pr[e] * r;
+    }
+  }
+  if (DIAG) {
+#pragma unroll
+    for (int e = 0; e < 32; ++e)
+      if (static_cast<float>(q_base + e) < col_rel) { pr[e] = 0.0f; pp[e] = 0.0f; }  // query before key
+  }
+#pragma unroll
+  for (int e = 0; e < 16; ++e) p_out[e] = pack_bf16x2(pr[2 * e], pr[2 * e + 1]);
+}
+
+// One row of a [128 x D] fp32 accumulator -> bf16 (times `mul`) -> swizzled staging tile.
+template <int D>
+__device__ __forceinline__ void bwd_store_acc_rows(uint32_t t_acc, uint8_t* stage, int tid, float mul) {
+  using L = BwdSmem<D>;
+#pragma unroll 1
+  for (int c = 0; c < D / 32; ++c) {
+    uint32_t o[32];
+    tmem_ld32(t_acc + c * 32, o);
+    tmem_wait_ld();
+    uint8_t* panel = stage + (c >> 1) * L::kPanelBytes + tid * 128;
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+      uint4 val;
+      val.x = pack_bf16x2(mul * __uint_as_float(o[8 * g + 0]), mul * __uint_as_float(o[8 * g + 1]));
+      val.y = pack_bf16x2(mul * __uint_as_float(o[8 * g + 2]), mul * __uint_as_float(o[8 * g + 3]));
+      val.z = pack_bf16x2(mul * __uint_as_float(o[8 * g + 4]), mul * __uint_as_float(o[8 * g + 5]));
+      val.w = pack_bf16x2(mul * __uint_as_float(o[8 * g + 6]), mul * __uint_as_float(o[8 * g + 7]));
+      const int chunk = (c & 1) * 4 + g;
+      *reinterpret_cast<uint4*>(panel + ((chunk ^ (tid & 7)) * 16)) = val;
+    }
+  }
+}
+
+template <int D, bool CAUSAL, bool ALIBI>
+__device__ void bwd_act_role(const BwdParams& p, const CUtensorMap* tmDk, const CUtensorMap* tmDv, int wg,
+                             uint8_t* smem, uint32_t tmem, BwdBarriers* bars, volatile int* cta_err) {
+  using L = BwdSmem<D>;
+  using TM = BwdTmem<D>;
+  const int tid = threadIdx.x & 127;  // key row within the tile
+  const uint32_t lane_off = static_cast<uint32_t>(((threadIdx.x >> 5) & 3) * 32) << 16;
+  uint32_t step_cnt = 0, item_cnt = 0;
+
+  for (int item = blockIdx.x; item < p.n_items; item += gridDim.x) {
+    const BwdItem w = decode_bwd_item<CAUSAL>(p, item);
+    float slope_log2e = 0.0f;
+    if (ALIBI) slope_log2e = p.slopes[w.bh % p.H] * kLog2eB;
+
+    for (int it = 0; it < w.n; ++it) {
+      const int i = w.i_begin + it;
+      const float col_rel = static_cast<float>((w.j - i) * kT + tid);  // key index minus first query of the tile
+      const bool diag = CAUSAL && (it == 0);
+      float pp[64];
+      if (!mbar_wait(smem_u32(&bars->s_full), step_cnt & 1, cta_err, 60 + wg)) return;
+      tc_fence_after_sync();
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        const int gc = wg * 2 + c;  // 32-query chunk of the tile
+        uint32_t s[32], pk[16];
+        tmem_ld32(tmem + TM::kA + lane_off + gc * 32, s);
+        tmem_wait_ld();
+        if (diag)
+          bwd_sigmoid_chunk<true, ALIBI>(s, pk, pp + 32 * c, p.scale_log2e, p.bias_log2e, slope_log2e, col_rel, gc * 32);
+        else
+          bwd_sigmoid_chunk<false, ALIBI>(s, pk, pp + 32 * c, p.scale_log2e, p.bias_log2e, slope_log2e, col_rel, gc * 32);
+        tmem_st16(tmem + TM::kA + lane_off + wg * 64 + c * 16, pk);
+      }
+      tmem_wait_st();
+      tc_fence_before_sync();
+      mbar_arrive(smem_u32(&bars->p_ready));
+
+      // dS^T = P (1 - P) dP^T -> bf16 -> shared memory [key][query], 128-byte swizzle
+      if (!mbar_wait(smem_u32(&bars->dp_full), step_cnt & 1, cta_err, 62 + wg)) return;
+      tc_fence_after_sync();
+      uint8_t* ds_row = smem + L::kDsOff + wg * L::kPanelBytes + tid * 128;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {  // 16 queries at a time
+        uint32_t dp[16];
+        tmem_ld16(tmem + TM::kB + lane_off + wg * 64 + c * 16, dp);
+        tmem_wait_ld();
+#pragma unroll
+        for (int g = 0; g < 2; ++g) {
+          uint4 val;
+          const float* f = pp + c * 16 + g * 8;
+          val.x = pack_bf16x2(f[0] * __uint_as_float(dp[8 * g + 0]), f[1] * __uint_as_float(dp[8 * g + 1]));
+          val.y = pack_bf16x2(f[2] * __uint_as_float(dp[8 * g + 2]), f[3] * __uint_as_float(dp[8 * g + 3]));
+          val.z = pack_bf16x2(f[4] * __uint_as_float(dp[8 * g + 4]), f[5] * __uint_as_float(dp[8 * g + 5]));
+          val.w = pack_bf16x2(f[6] * __uint_as_float(dp[8 * g + 6]), f[7] * __uint_as_float(dp[8 * g + 7]));
+          const int chunk = c * 2 + g;
+          *reinterpret_cast<uint4*>(ds_row + ((chunk ^ (tid & 7)) * 16)) = val;
+        }
+      }
+      tc_fence_before_sync();   // the dP^T reads above precede the dQ MMA that overwrites region B
+      fence_proxy_async_smem();
+      mbar_arrive(smem_u32(&bars->ds_ready));
+      ++step_cnt;
+    }
+
+    // epilogue: group 0 stores dV_j (staged in the V tile), group 1 stores scale * dK_j (K tile)
+    if (!mbar_wait(smem_u32(&bars->dkv_full), item_cnt & 1, cta_err, 64 + wg)) return;
+    ++item_cnt;
+    tc_fence_after_sync();
+    uint8_t* stage = smem + (wg == 0 ? L::kVOff : L::kKOff);
+    bwd_store_acc_rows<D>(tmem + (wg == 0 ? TM::kDv : TM::kDk) + lane_off, stage, tid, wg == 0 ? 1.0f : p.scale);
+    tc_fence_before_sync();
+    mbar_arrive(smem_u32(&bars->dkv_empty));
+    fence_proxy_async_smem();
+    if (wg == 0) named_barrier_sync<1, 128>(); else named_barrier_sync<2, 128>();
+    if (tid == 0) {
+      const CUtensorMap* tm = (wg == 0) ? tmDv : tmDk;
+#pragma unroll
+      for (int pn = 0; pn < L::kPanels; ++pn)
+        tma_store_3d(tm, smem_u32(stage + pn * L::kPanelBytes), pn * 64, w.j * kT, w.bh);
+      tma_commit_group();
+      tma_wait_group_read<0>();
+      mbar_arrive(smem_u32(&bars->kv_empty));
+    }
+  }
+  if (tid == 0) tma_wait_group<0>();
+}
+
+// ------------------------------------------------------------------ dQ drain group
+
+template <int D, bool CAUSAL>
+__device__ void bwd_drain_role(const BwdParams& p, const CUtensorMap* tmW, uint8_t* smem, uint32_t tmem,
+                               BwdBarriers* bars, volatile int* cta_err) {
+  using L = BwdSmem<D>;
+  using TM = BwdTmem<D>;
+  const int tid = threadIdx.x & 127;  // query row within the tile
+  const uint32_t lane_off = static_cast<uint32_t>(((threadIdx.x >> 5) & 3) * 32) << 16;
+  uint32_t step_cnt = 0, box_cnt = 0;
+  for (int item = blockIdx.x; item < p.n_items; item += gridDim.x) {
+    const BwdItem w = decode_bwd_item<CAUSAL>(p, item);
+    for (int it = 0; it < w.n; ++it) {
+      const int row0 = (w.i_begin + it) * kT;
+      if (!mbar_wait(smem_u32(&bars->dq_full), step_cnt & 1, cta_err, 70)) return;
+      ++step_cnt;
+      tc_fence_after_sync();
+#pragma unroll 1
+      for (int c = 0; c < D / 32; ++c) {
+        uint32_t o[32];
+        tmem_ld32(tmem + TM::kB + lane_off + c * 32, o);
+        tmem_wait_ld();
+        if (c == D / 32 - 1) {
+          tc_fence_before_sync();
+          mbar_arrive(smem_u32(&bars->dq_empty));
+        }
+        // the staging box used two boxes ago must have been read by its reduce-add
+        if (tid == 0) tma_wait_group_read<1>();
+        named_barrier_sync<3, 128>();
+        uint8_t* box = smem + L::kDqOff + (box_cnt & 1) * L::kPanelBytes;
+        uint8_t* rowp = box + tid * 128;
+#pragma unroll
+        for (int g = 0; g < 8; ++g) {
+          uint4 val = make_uint4(o[4 * g + 0], o[4 * g + 1], o[4 * g + 2], o[4 * g + 3]);
+          *reinterpret_cast<uint4*>(rowp + ((g ^ (tid & 7)) * 16)) = val;
+        }
+        fence_proxy_async_smem();
+        named_barrier_sync<3, 128>();
+        if (tid == 0) {
+          tma_reduce_add_3d(tmW, smem_u32(box), c * 32, row0, w.bh);
+          tma_commit_group();
+        }
+        ++box_cnt;
+      }
+    }
+  }
+  if (tid == 0) tma_wait_group<0>();
+}
+
+// ------------------------------------------------------------------ kernels
+
+template <int D, bool CAUSAL, bool ALIBI>
+__global__ void __launch_bounds__(kBwdThreads, 1)
+sigattn_bwd_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                        const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmDo,
+                        const __grid_constant__ CUtensorMap tmDk, const __grid_constant__ CUtensorMap tmDv,
+                        const __grid_constant__ CUtensorMap tmW, const BwdParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ BwdBarriers bars;
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int cta_err;
+
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const uint32_t smem_base = smem_u32(smem);
+  const int warp = threadIdx.x >> 5;
+
+  if (threadIdx.x == 0) {
+    cta_err = 0;
+    mbar_init(smem_u32(&bars.kv_full), 1);
+    mbar_init(smem_u32(&bars.kv_empty), 2);
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(smem_u32(&bars.q_full[s]), 1);
+      mbar_init(smem_u32(&bars.q_empty[s]), 1);
+    }
+    mbar_init(smem_u32(&bars.do_full), 1);
+    mbar_init(smem_u32(&bars.do_empty), 1);
+    mbar_init(smem_u32(&bars.s_full), 1);
+    mbar_init(smem_u32(&bars.dp_full), 1);
+    mbar_init(smem_u32(&bars.p_ready), 256);
+    mbar_init(smem_u32(&bars.ds_ready), 256);
+    mbar_init(smem_u32(&bars.dq_full), 1);
+    mbar_init(smem_u32(&bars.dq_empty), 128);
+    mbar_init(smem_u32(&bars.dkv_full), 1);
+    mbar_init(smem_u32(&bars.dkv_empty), 256);
+    fence_mbar_init();
+  }
+  if (warp == kBwdLoadWarp && elect_one()) {
+    tma_prefetch_desc(&tmQ);
+    tma_prefetch_desc(&tmK);
+    tma_prefetch_desc(&tmV);
+    tma_prefetch_desc(&tmDo);
+    tma_prefetch_desc(&tmDk);
+    tma_prefetch_desc(&tmDv);
+    tma_prefetch_desc(&tmW);
+  }
+  if (warp == kBwdMmaWarp) {
+    tmem_alloc(smem_u32(&tmem_base_slot), 512);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = tmem_base_slot;
+
+  if (warp == kBwdLoadWarp) {
+    if ((threadIdx.x & 31) == 0) bwd_load_role<D, CAUSAL>(p, &tmQ, &tmK, &tmV, &tmDo, smem_base, &bars, &cta_err);
+    __syncwarp();
+  } else if (warp == kBwdMmaWarp) {
+    if ((threadIdx.x & 31) == 0) bwd_mma_role<D, CAUSAL>(p, smem_base, tmem, &bars, &cta_err);
+    __syncwarp();
+  } else if (warp < 8) {
+    bwd_act_role<D, CAUSAL, ALIBI>(p, &tmDk, &tmDv, warp >> 2, smem, tmem, &bars, &cta_err);
+  } else {
+    bwd_drain_role<D, CAUSAL>(p, &tmW, smem, tmem, &bars, &cta_err);
+  }
+
+  tc_fence_before_sync();
+  __syncthreads();
+  if (cta_err != 0) {
+    if (threadIdx.x == 0) atomicExch(p.status, 200 + cta_err);
+    __nanosleep(100000);
+  }
+  if (warp == kBwdMmaWarp) tmem_dealloc(tmem, 512);
+}
+
+// dQ (bf16) = scale * workspace (fp32): the conversion step that follows the main kernel.
+__global__ void __launch_bounds__(256)
+sigattn_bwd_convert_dq_kernel(const float4* __restrict__ ws, uint2* __restrict__ dq, size_t n_vec4, float scale) {
+  const size_t stride = static_cast<size_t>(gridDim.x) * blockDim.x;
+  for (size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < n_vec4; i += stride) {
+    const float4 v = ws[i];
+    uint2 o;
+    o.x = pack_bf16x2(scale * v.x, scale * v.y);
+    o.y = pack_bf16x2(scale * v.z, scale * v.w);
+    dq[i] = o;
+  }
+}
+
+template <int D, bool CAUSAL, bool ALIBI>
+int launch_bwd_variant(const CUtensorMap* maps, const BwdParams& bp, int num_sms, cudaStream_t stream,
+                       cudaError_t* cuda_err) {
+  auto kernel = sigattn_bwd_bf16_kernel<D, CAUSAL, ALIBI>;
+  static bool configured = false;
+  if (!configured) {
+    *cuda_err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<D>::kDynBytes);
+    if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
+    configured = true;
+  }
+  const int grid = bp.n_items < num_sms ? bp.n_items : num_sms;
+  kernel<<<grid, kBwdThreads, BwdSmem<D>::kDynBytes, stream>>>(maps[0], maps[1], maps[2], maps[3], maps[4], maps[5],
+                                                                maps[6], bp);
+  *cuda_err = cudaGetLastError();
+  return *cuda_err == cudaSuccess ? SIGATTN_OK : SIGATTN_ERR_CUDA;
+}
+
+}  // namespace
+
+size_t bwd_bf16_workspace_bytes(int B, int H, int N, int D) {
+  return static_cast<size_t>(B) * H * N * D * sizeof(float);
+}
+
+int launch_bwd_bf16(const void* q, const void* k, const void* v, const void* d_o, void* dq, void* dk, void* dv,
+                    const Problem& p, void* workspace, int* status, cudaStream_t stream,
+                    unsigned long long* launches, cudaError_t* cuda_err) {
+  int dev = 0, num_sms = 0;
+  *cuda_err = cudaGetDevice(&dev);
+  if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
+  *cuda_err = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
+  if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
+
+  const uint64_t BH = static_cast<uint64_t>(p.B) * p.H;
+  CUtensorMap maps[7];
+  const void* ptrs[6] = {q, k, v, d_o, dk, dv};
+  for (int i = 0; i < 6; ++i) {
+    if (make_map_3d(&maps[i], ptrs[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, BH, p.N, p.D, kT, 64) != 0) {
+      *cuda_err = cudaErrorInvalidValue;
+      return SIGATTN_ERR_CUDA;
+    }
+  }
+  if (make_map_3d(&maps[6], workspace, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, BH, p.N, p.D, kT, 32) != 0) {
+    *cuda_err = cudaErrorInvalidValue;
+    return SIGATTN_ERR_CUDA;
+  }
+  BwdParams bp;
+  bp.BH = static_cast<int>(BH);
+  bp.H = p.H;
+  bp.N = p.N;
+  bp.n_tiles = (p.N + kT - 1) / kT;
+  bp.n_items = bp.n_tiles * bp.BH;
+  bp.scale = p.scale;
+  bp.scale_log2e = p.scale * kLog2eB;
+  bp.bias_log2e = p.bias * kLog2eB;
+  bp.slopes = p.slopes;
+  bp.status = status;
+
+  const size_t n_elems = static_cast<size_t>(BH) * p.N * p.D;
+  // step 1: clear the fp32 dQ accumulator
+  *cuda_err = cudaMemsetAsync(workspace, 0, n_elems * sizeof(float), stream);
+  if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
+
+  // step 2: main kernel
+  int rc;
+  const bool alibi = p.slopes != nullptr;
+#define SIGATTN_BWD_CASE(DD, CC, AA) rc = launch_bwd_variant<DD, CC, AA>(maps, bp, num_sms, stream, cuda_err)
+  if (p.D == 128) {
+    if (p.causal) { if (alibi) SIGATTN_BWD_CASE(128, true, true); else SIGATTN_BWD_CASE(128, true, false); }
+    else          { if (alibi) SIGATTN_BWD_CASE(128, false, true); else SIGATTN_BWD_CASE(128, false, false); }
+  } else {
+    if (p.causal) { if (alibi) SIGATTN_BWD_CASE(64, true, true); else SIGATTN_BWD_CASE(64, true, false); }
+    else          { if (alibi) SIGATTN_BWD_CASE(64, false, true); else SIGATTN_BWD_CASE(64, false, false); }
+  }
+#undef SIGATTN_BWD_CASE
+  if (rc != SIGATTN_OK) return rc;
+  *launches += 1;
+
+  // step 3: dQ = scale * accumulator, as bf16
+  const size_t n_vec4 = n_elems / 4;  // D is a multiple of 64
+  const int blocks = static_cast<int>(n_vec4 / 256 + 1 < static_cast<size_t>(num_sms) * 8 ? n_vec4 / 256 + 1
+                                                                                            : static_cast<size_t>(num_sms) * 8);
+  sigattn_bwd_convert_dq_kernel<<<blocks, 256, 0, stream>>>(static_cast<const float4*>(workspace),
+                                                            static_cast<uint2*>(dq), n_vec4, p.scale);
+  *cuda_err = cudaGetLastError();
+  if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
+  *launches += 1;
+  return SIGATTN_OK;
+}
+
+}  // namespace sigattn
