@@ -1,0 +1,381 @@
+#!/usr/bin/env python
+"""Benchmark of the fused sigmoid-attention forward + backward on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c4] [--impl ours|reference]
+
+A "step" is one forward plus one backward pass over one synthetic batch of the chosen
+configuration (default c4: causal LM shape B=2, H=16, N=4096, D=128, bf16, QK-normed
+inputs, b = -log N).  Metric: useful bf16 TFLOP/s of the step, FLOPs counted as
+4 c B H N^2 D (forward) + 10 c B H N^2 D (backward), c = (N+1)/(2N) when causal.
+
+One JSON line is printed by rank 0.  With N > 1 (torchrun), every rank runs the same
+workload on its own GPU and its own batch (the (batch, head) pairs are independent, no
+collective exists on the path): weak scaling, value = FLOPs of all ranks / max time.
+
+`--impl reference` times the float64 CPU oracle on the host cores instead (a bounded
+sample of the same workload); it is a deliberately slow baseline, not a target.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+from paper_2409_04431_b200 import inputs  # noqa: E402
+
+METRIC = "sigmoid-attn fwd+bwd bf16 TFLOP/s"
+UNIT = "TFLOP/s"
+FALLBACK_PEAKS = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0}
+L2_FLUSH_BYTES = 256 << 20
+
+# DRAM bytes per launch of the dominant kernel (backward main kernel) from the committed
+# ncu capture, per workload; see profiles/.  None where no capture exists.
+NCU_TRAFFIC_BYTES = {}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {k: float(d[k]) for k in FALLBACK_PEAKS if k in d}, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def host_cores() -> int:
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+# ----------------------------------------------------------------------------- oracle legs
+
+
+def oracle_sample(cfg, budget_s: float = 20.0):
+    """Time the float64 oracle, as it stands, on a bounded sample of `cfg`: whole heads of
+    one batch element, as many as fit the time budget (at least one)."""
+    import oracle  # test infrastructure; used here for the CPU baseline only
+
+    q, k, v, d_o = inputs.make_inputs(cfg, heads=1, batch=1)
+    slopes = cfg.slopes()
+    sl = None if slopes is None else slopes[:1]
+    rb = 1024 if cfg.N > 4096 else None
+    t0 = time.perf_counter()
+    oracle.sigattn_fwd(q, k, v, cfg.scale, cfg.bias, cfg.causal, sl, row_block=rb)
+    oracle.sigattn_bwd(q, k, v, d_o, cfg.scale, cfg.bias, cfg.causal, sl, row_block=rb)
+    one = time.perf_counter() - t0
+    heads = max(1, min(cfg.B * cfg.H, int(budget_s / max(one, 1e-6))))
+    total = one
+    done = 1
+    while done < heads:
+        t0 = time.perf_counter()
+        oracle.sigattn_fwd(q, k, v, cfg.scale, cfg.bias, cfg.causal, sl, row_block=rb)
+        oracle.sigattn_bwd(q, k, v, d_o, cfg.scale, cfg.bias, cfg.causal, sl, row_block=rb)
+        total += time.perf_counter() - t0
+        done += 1
+    flops_head = (cfg.flops_fwd() + cfg.flops_bwd()) / (cfg.B * cfg.H)
+    return {
+        "value": flops_head * done / total / 1e12,
+        "unit": UNIT,
+        "cores": host_cores(),
+        "kind": "oracle",
+        "sample": f"{done} of {cfg.B * cfg.H} (batch, head) pairs of {cfg.name}, fwd+bwd, float64 numpy, "
+                  f"{total:.1f} s wall",
+    }, total / done
+
+
+def run_reference(args, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    steps = max(1, args.steps)
+    warm = max(0, args.warmup)
+    per_step_budget = max(2.0, 60.0 / (steps + warm))
+    vals, times = [], []
+    base = None
+    for s in range(warm + steps):
+        base, per_head = oracle_sample(cfg, budget_s=per_step_budget)
+        if s >= warm:
+            vals.append(base["value"])
+            times.append(per_head)
+    value = float(np.mean(vals))
+    base["value"] = value
+    line = {
+        "impl": "reference",
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps, "warmup": warm,
+        "ms_per_step": float(np.mean(times)) * 1e3 * cfg.B * cfg.H,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(cfg, args.gpus),
+        "cpu_baseline": base,
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(cfg, n_gpus):
+    return {
+        "workload": f"{cfg.name}: B={cfg.B} H={cfg.H} N={cfg.N} D={cfg.D} {cfg.dtype} "
+                    f"{'causal' if cfg.causal else 'full'}{' alibi' if cfg.alibi else ''}"
+                    f"{' qk-norm' if cfg.qk_norm else ''} b=-ln(N), one fwd+bwd per step",
+        "per_gpu_batch": cfg.B, "gpus": n_gpus,
+        "cache": f"L2 flushed between timed steps (write of {L2_FLUSH_BYTES >> 20} MiB)",
+    }
+
+
+# ----------------------------------------------------------------------------- clocks
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons of one GPU while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period_s
+        self.stop_flag = threading.Event()
+        self.sm, self.reasons, self.max_sm = [], set(), None
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_sm = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+        }
+        while not self.stop_flag.is_set():
+            try:
+                self.sm.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def summary(self):
+        if not self.ok or not self.sm:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_sm, "reasons": [], "samples": 0}
+        return {"sm_mhz": float(np.median(self.sm)), "sm_max_mhz": self.max_sm, "reasons": sorted(self.reasons),
+                "samples": len(self.sm)}
+
+
+def physical_gpu_index(local_index: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        parts = [p for p in vis.split(",") if p.strip() != ""]
+        try:
+            return int(parts[local_index])
+        except (ValueError, IndexError):
+            return local_index
+    return local_index
+
+
+# ----------------------------------------------------------------------------- our arm
+
+
+def run_ours(args, cfg):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2409_04431_b200 as sa  # raises if libsigattn.so is missing: no fallback
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback for the product path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    steps, warm = max(1, args.steps), max(3, args.warmup)
+    dt = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
+    code = 0 if cfg.dtype == "bf16" else 1
+
+    # host inputs (seeded; each rank its own batch) -> pinned host tensors -> device
+    qh, kh, vh, doh = inputs.make_inputs(cfg, seed=inputs.SEED_BASE + cfg.index + 1000 * rank)
+
+    def to_torch_host(x):
+        if cfg.dtype == "bf16":
+            t = torch.from_numpy(inputs.f32_to_bf16_bits(x).view(np.int16)).view(torch.bfloat16)
+        else:
+            t = torch.from_numpy(x)
+        return t.pin_memory()
+
+    host_in = [to_torch_host(x) for x in (qh, kh, vh, doh)]
+    host_out = [torch.empty_like(host_in[0]).pin_memory() for _ in range(4)]
+    q, k, v, d_o = (t.to(dev, non_blocking=True) for t in host_in)
+    o = torch.empty_like(q)
+    grads = tuple(torch.empty_like(q) for _ in range(3))
+    slopes_np = cfg.slopes()
+    slopes = None if slopes_np is None else torch.from_numpy(slopes_np).to(dev)
+    slopes_host = None if slopes_np is None else torch.from_numpy(slopes_np).pin_memory()
+    ws = torch.empty(max(1, sa.sigattn_bwd_workspace_bytes(cfg.B, cfg.H, cfg.N, cfg.D, code)), dtype=torch.uint8,
+                     device=dev)
+    arena = torch.empty(sa.sigattn_step_host_arena_bytes(cfg.B, cfg.H, cfg.N, cfg.D, code), dtype=torch.uint8,
+                        device=dev)
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    torch.cuda.synchronize()
+
+    def fwd():
+        sa.sigattn_fwd(q, k, v, cfg.scale, cfg.bias, cfg.causal, slopes, out=o)
+
+    def bwd():
+        sa.sigattn_bwd(q, k, v, d_o, cfg.scale, cfg.bias, cfg.causal, slopes, workspace=ws, out=grads)
+
+    ev = lambda: torch.cuda.Event(enable_timing=True)  # noqa: E731
+    sampled = list(range(0, steps, 8))          # steps whose main backward kernel is timed on its own
+    k_ev = {s: (ev(), ev()) for s in sampled}
+    for a, b in k_ev.values():                  # create the handles before handing them to the library
+        a.record(); b.record()
+    torch.cuda.synchronize()
+
+    for _ in range(warm):
+        fwd(); bwd()
+    sa.sigattn_check()
+
+    # ---- timed region: K steps, device-resident inputs, L2 flushed between steps (untimed)
+    sampler = ClockSampler(physical_gpu_index(local))
+    e_fwd0, e_fwd1, e_bwd1 = [ev() for _ in range(steps)], [ev() for _ in range(steps)], [ev() for _ in range(steps)]
+    barrier()
+    launches0 = sa.sigattn_launch_count()
+    sampler.start()
+    wall0 = time.perf_counter()
+    for s in range(steps):
+        flush.zero_()
+        e_fwd0[s].record()
+        fwd()
+        e_fwd1[s].record()
+        if s in k_ev:  # the hook adds two event records around the main kernel
+            sa.sigattn_bwd_set_timing_events(*k_ev[s])
+            bwd()
+            sa.sigattn_bwd_set_timing_events(None, None)
+        else:
+            bwd()
+        e_bwd1[s].record()
+    barrier()
+    kern_ms = [a.elapsed_time(b) for a, b in k_ev.values()]
+    wall = time.perf_counter() - wall0
+    launches = sa.sigattn_launch_count() - launches0
+    sampler.stop_flag.set()
+    sampler.join()
+    sa.sigattn_check()
+
+    fwd_ms = [e_fwd0[s].elapsed_time(e_fwd1[s]) for s in range(steps)]
+    bwd_ms = [e_fwd1[s].elapsed_time(e_bwd1[s]) for s in range(steps)]
+    t_fwd, t_bwd = float(np.sum(fwd_ms)), float(np.sum(bwd_ms))
+    t_total = t_fwd + t_bwd
+
+    # ---- end to end: host (pinned) inputs -> device -> fwd + bwd -> host, through the C ABI
+    e2e_steps = max(3, min(steps, 10))
+    for _ in range(2):
+        sa.sigattn_step_host(*host_in, *host_out, cfg.scale, cfg.bias, cfg.causal, slopes_host, arena=arena)
+    barrier()
+    e0, e1 = ev(), ev()
+    e0.record()
+    for _ in range(e2e_steps):
+        sa.sigattn_step_host(*host_in, *host_out, cfg.scale, cfg.bias, cfg.causal, slopes_host, arena=arena)
+    e1.record()
+    barrier()
+    sa.sigattn_check()
+    t_e2e = e0.elapsed_time(e1) / e2e_steps
+
+    # max over ranks
+    stats = torch.tensor([t_total, t_fwd, t_bwd, t_e2e, float(np.mean(kern_ms))], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(stats, op=dist.ReduceOp.MAX)
+    t_total, t_fwd, t_bwd, t_e2e, t_kern = stats.tolist()
+
+    if rank == 0:
+        peaks, peak_src = load_peaks()
+        f_fwd, f_bwd = cfg.flops_fwd(), cfg.flops_bwd()
+        per_step_ms = t_total / steps
+        value = world * (f_fwd + f_bwd) * steps / (t_total * 1e-3) / 1e12
+        fwd_tf = f_fwd * steps / (t_fwd * 1e-3) / 1e12
+        bwd_tf = f_bwd * steps / (t_bwd * 1e-3) / 1e12
+        kern_tf = f_bwd / (t_kern * 1e-3) / 1e12
+        peak = peaks["bf16_tflops"]
+        tensor_bytes = cfg.B * cfg.H * cfg.N * cfg.D * (2 if cfg.dtype == "bf16" else 4)
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warm,
+            "ms_per_step": per_step_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": cfg.dtype, "data": "synthetic",
+            "config": workload_config(cfg, world),
+            "fwd": {"tflops": fwd_tf, "ms": t_fwd / steps, "frac_of_peak": fwd_tf / peak},
+            "bwd": {"tflops": bwd_tf, "ms": t_bwd / steps, "frac_of_peak": bwd_tf / peak,
+                    "includes": "dQ-accumulator clear + main kernel + dQ convert"},
+            "frac_of_peak": value / world / peak,
+            "roofline": {
+                "kernel": "sigattn_bwd_bf16_kernel (backward main kernel)",
+                "bound": "tensor", "achieved": kern_tf, "peak": peak, "unit": "TFLOP/s", "frac": kern_tf / peak,
+                "peak_source": f"{peak_src} bf16_tflops (burst)", "avg_launch_ms": t_kern,
+                "algorithmic_flops_per_launch": f_bwd,
+                "traffic": NCU_TRAFFIC_BYTES.get(cfg.name),
+            },
+            "e2e": {"value": world * (f_fwd + f_bwd) / (t_e2e * 1e-3) / 1e12, "unit": UNIT,
+                    "ms_per_step": t_e2e, "h2d_bytes_per_step": 4 * tensor_bytes, "d2h_bytes_per_step": 4 * tensor_bytes},
+            "gpu_launches": int(launches),
+            "clocks": sampler.summary(),
+            "wall_s_timed_region": wall,
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"], _ = oracle_sample(cfg, budget_s=args.cpu_budget)
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c4", choices=sorted(inputs.CONFIGS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-budget", type=float, default=15.0)
+    args = ap.parse_args()
+    cfg = inputs.CONFIGS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_ours(args, cfg)
+
+
+if __name__ == "__main__":
+    main()

@@ -94,6 +94,31 @@ SIGATTN_API int sigattn_bwd(const void* q, const void* k, const void* v, const v
  * Returns 0 for invalid shapes as well; sigattn_bwd reports those. */
 SIGATTN_API size_t sigattn_bwd_workspace_bytes(int B, int H, int N, int D, int dtype);
 
+/* One forward + backward pass from HOST buffers (pinned memory recommended): copies
+ * q, k, v, d_o (and the H slopes, if any) to the device, runs sigattn_fwd and
+ * sigattn_bwd, and copies o, dq, dk, dv back, all enqueued on `stream` in that order;
+ * returns without synchronising.  Every tensor pointer and `alibi_slopes_host` are HOST
+ * pointers; `device_arena` is DEVICE scratch of at least
+ * sigattn_step_host_arena_bytes(...) bytes, 256-byte aligned, owned by the caller (it
+ * holds the eight tensors, the slopes and the backward workspace).  The host buffers must
+ * stay valid until the stream has finished.  No counterpart in the paper: this is the
+ * end-to-end entry for callers whose data lives in host memory. */
+SIGATTN_API int sigattn_step_host(const void* q_host, const void* k_host, const void* v_host, const void* d_o_host,
+                      void* o_host, void* dq_host, void* dk_host, void* dv_host,
+                      int B, int H, int N, int D,
+                      float scale, float bias, int causal,
+                      const float* alibi_slopes_host, int dtype,
+                      void* device_arena, size_t arena_bytes, void* stream);
+
+/* Bytes of device scratch sigattn_step_host needs (0 for invalid shapes). */
+SIGATTN_API size_t sigattn_step_host_arena_bytes(int B, int H, int N, int D, int dtype);
+
+/* Optional timing hook: when both are non-NULL cudaEvent_t handles, every following
+ * sigattn_bwd on this thread records `start` right before and `stop` right after its
+ * main kernel (excluding the dQ-accumulator clear and the dQ conversion) on the call's
+ * stream.  Pass NULL, NULL to switch it off.  Returns 0. */
+SIGATTN_API int sigattn_bwd_set_timing_events(void* start_event, void* stop_event);
+
 /* Synchronises `stream`, then returns 0 or SIGATTN_ERR_DEVICE_TIMEOUT if any kernel of
  * this library gave up a bounded wait on the current device since the last check
  * (the flag is cleared), or SIGATTN_ERR_CUDA if the stream reports a CUDA error. */

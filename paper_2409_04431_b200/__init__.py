@@ -19,6 +19,9 @@ _BINDING_NAMES = (
     "sigattn_launch_count",
     "sigattn_strerror",
     "sigattn_version",
+    "sigattn_step_host",
+    "sigattn_step_host_arena_bytes",
+    "sigattn_bwd_set_timing_events",
 )
 
 __all__ = list(_BINDING_NAMES)

@@ -33,6 +33,14 @@ _lib.sigattn_bwd.argtypes = [_c.c_void_p] * 7 + [_c.c_int] * 4 + [_c.c_float, _c
                                                                     _c.c_size_t, _c.c_void_p]
 _lib.sigattn_bwd_workspace_bytes.restype = _c.c_size_t
 _lib.sigattn_bwd_workspace_bytes.argtypes = [_c.c_int] * 5
+_lib.sigattn_step_host.restype = _c.c_int
+_lib.sigattn_step_host.argtypes = [_c.c_void_p] * 8 + [_c.c_int] * 4 + [_c.c_float, _c.c_float, _c.c_int,
+                                                                          _c.c_void_p, _c.c_int, _c.c_void_p,
+                                                                          _c.c_size_t, _c.c_void_p]
+_lib.sigattn_step_host_arena_bytes.restype = _c.c_size_t
+_lib.sigattn_step_host_arena_bytes.argtypes = [_c.c_int] * 5
+_lib.sigattn_bwd_set_timing_events.restype = _c.c_int
+_lib.sigattn_bwd_set_timing_events.argtypes = [_c.c_void_p, _c.c_void_p]
 _lib.sigattn_check.restype = _c.c_int
 _lib.sigattn_check.argtypes = [_c.c_void_p]
 _lib.sigattn_strerror.restype = _c.c_char_p
@@ -47,6 +55,7 @@ _lib.sigattn_launch_count.argtypes = []
 EXPORTED = [
     "sigattn_fwd", "sigattn_bwd", "sigattn_bwd_workspace_bytes", "sigattn_check",
     "sigattn_strerror", "sigattn_last_cuda_error", "sigattn_version", "sigattn_launch_count",
+    "sigattn_step_host", "sigattn_step_host_arena_bytes", "sigattn_bwd_set_timing_events",
 ]
 
 
@@ -172,3 +181,41 @@ def sigattn_bwd(q, k, v, d_o, scale, bias, causal=False, alibi_slopes=None, work
     if rc != 0:
         raise SigattnError(rc)
     return dq, dk, dv
+
+
+def sigattn_step_host_arena_bytes(B, H, N, D, dtype_code) -> int:
+    return int(_lib.sigattn_step_host_arena_bytes(B, H, N, D, dtype_code))
+
+
+def sigattn_step_host(q, k, v, d_o, o, dq, dk, dv, scale, bias, causal=False, alibi_slopes=None, arena=None,
+                      stream=None):
+    """Forward + backward from HOST tensors (CPU torch tensors, ideally pinned): copies the
+    inputs to the device, runs both passes, copies O, dQ, dK, dV back into the given host
+    tensors; everything is enqueued on the current stream and nothing is synchronised.
+    `arena`: uint8 CUDA tensor of at least sigattn_step_host_arena_bytes bytes.
+    `alibi_slopes`: None or a float32 CPU tensor of H slopes."""
+    import torch
+    ts = [q, k, v, d_o, o, dq, dk, dv]
+    for t in ts:
+        if t.is_cuda or not t.is_contiguous() or t.shape != q.shape or t.dtype != q.dtype:
+            raise ValueError("sigattn_step_host takes contiguous CPU tensors of one shape and dtype")
+    B, H, N, D = q.shape
+    code = _dtype_code(q)
+    need = sigattn_step_host_arena_bytes(B, H, N, D, code)
+    if arena is None:
+        arena = torch.empty(need, dtype=torch.uint8, device="cuda")
+    with torch.cuda.device(arena.device):
+        rc = _lib.sigattn_step_host(*[_ptr(t) for t in ts], B, H, N, D, float(scale), float(bias),
+                                    int(bool(causal)), _ptr(alibi_slopes), code, _ptr(arena),
+                                    arena.numel(), _stream_ptr(stream))
+    if rc != 0:
+        raise SigattnError(rc)
+    return arena
+
+
+def sigattn_bwd_set_timing_events(start=None, stop=None) -> None:
+    """start, stop: torch.cuda.Event(enable_timing=True) that have been recorded once
+    (so that their handles exist), or None, None to switch the hook off."""
+    a = None if start is None else start.cuda_event
+    b = None if stop is None else stop.cuda_event
+    _lib.sigattn_bwd_set_timing_events(a, b)

@@ -119,6 +119,66 @@ int sigattn_bwd(const void* q, const void* k, const void* v, const void* d_o, vo
   return rc;
 }
 
+int sigattn_bwd_set_timing_events(void* start_event, void* stop_event) {
+  sigattn::set_bwd_timing_events(static_cast<cudaEvent_t>(start_event), static_cast<cudaEvent_t>(stop_event));
+  return SIGATTN_OK;
+}
+
+namespace {
+size_t align256(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
+}
+
+size_t sigattn_step_host_arena_bytes(int B, int H, int N, int D, int dtype) {
+  if (check_shape(B, H, N, D) != SIGATTN_OK) return 0;
+  if (dtype != SIGATTN_DTYPE_BF16 && dtype != SIGATTN_DTYPE_FP32) return 0;
+  const size_t tensor = align256(static_cast<size_t>(B) * H * N * D * (dtype == SIGATTN_DTYPE_BF16 ? 2 : 4));
+  return 8 * tensor + align256(static_cast<size_t>(H) * sizeof(float)) +
+         align256(sigattn_bwd_workspace_bytes(B, H, N, D, dtype));
+}
+
+int sigattn_step_host(const void* q_host, const void* k_host, const void* v_host, const void* d_o_host, void* o_host,
+                      void* dq_host, void* dk_host, void* dv_host, int B, int H, int N, int D, float scale,
+                      float bias, int causal, const float* alibi_slopes_host, int dtype, void* device_arena,
+                      size_t arena_bytes, void* stream) {
+  if (!q_host || !k_host || !v_host || !d_o_host || !o_host || !dq_host || !dk_host || !dv_host || !device_arena)
+    return SIGATTN_ERR_NULL;
+  if (int rc = check_shape(B, H, N, D)) return rc;
+  if (dtype != SIGATTN_DTYPE_BF16 && dtype != SIGATTN_DTYPE_FP32) return SIGATTN_ERR_FLAG;
+  if (causal != 0 && causal != 1) return SIGATTN_ERR_FLAG;
+  if (reinterpret_cast<uintptr_t>(device_arena) & 255u) return SIGATTN_ERR_ALIGN;
+  if (arena_bytes < sigattn_step_host_arena_bytes(B, H, N, D, dtype)) return SIGATTN_ERR_WORKSPACE;
+  const size_t bytes = static_cast<size_t>(B) * H * N * D * (dtype == SIGATTN_DTYPE_BF16 ? 2 : 4);
+  const size_t tensor = align256(bytes);
+  char* base = static_cast<char*>(device_arena);
+  void* d[8];
+  for (int i = 0; i < 8; ++i) d[i] = base + i * tensor;
+  float* d_slopes = reinterpret_cast<float*>(base + 8 * tensor);
+  void* d_ws = base + 8 * tensor + align256(static_cast<size_t>(H) * sizeof(float));
+  const size_t ws_bytes = sigattn_bwd_workspace_bytes(B, H, N, D, dtype);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const void* in_host[4] = {q_host, k_host, v_host, d_o_host};
+  for (int i = 0; i < 4; ++i) {
+    cudaError_t e = cudaMemcpyAsync(d[i], in_host[i], bytes, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) { t_last_cuda = e; return SIGATTN_ERR_CUDA; }
+  }
+  if (alibi_slopes_host) {
+    cudaError_t e = cudaMemcpyAsync(d_slopes, alibi_slopes_host, static_cast<size_t>(H) * sizeof(float),
+                                    cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) { t_last_cuda = e; return SIGATTN_ERR_CUDA; }
+  }
+  const float* slopes = alibi_slopes_host ? d_slopes : nullptr;
+  if (int rc = sigattn_fwd(d[0], d[1], d[2], d[4], B, H, N, D, scale, bias, causal, slopes, dtype, stream)) return rc;
+  if (int rc = sigattn_bwd(d[0], d[1], d[2], d[3], d[5], d[6], d[7], B, H, N, D, scale, bias, causal, slopes, dtype,
+                           ws_bytes ? d_ws : nullptr, ws_bytes, stream))
+    return rc;
+  void* out_host[4] = {o_host, dq_host, dk_host, dv_host};
+  for (int i = 0; i < 4; ++i) {
+    cudaError_t e = cudaMemcpyAsync(out_host[i], d[4 + i], bytes, cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) { t_last_cuda = e; return SIGATTN_ERR_CUDA; }
+  }
+  return SIGATTN_OK;
+}
+
 size_t sigattn_bwd_workspace_bytes(int B, int H, int N, int D, int dtype) {
   if (check_shape(B, H, N, D) != SIGATTN_OK) return 0;
   if (dtype != SIGATTN_DTYPE_BF16) return 0;

@@ -557,6 +557,16 @@ int launch_bwd_variant(const CUtensorMap* maps, const BwdParams& bp, int num_sms
 
 }  // namespace
 
+namespace {
+thread_local cudaEvent_t t_ev_start = nullptr;
+thread_local cudaEvent_t t_ev_stop = nullptr;
+}  // namespace
+
+void set_bwd_timing_events(cudaEvent_t start, cudaEvent_t stop) {
+  t_ev_start = start;
+  t_ev_stop = stop;
+}
+
 size_t bwd_bf16_workspace_bytes(int B, int H, int N, int D) {
   return static_cast<size_t>(B) * H * N * D * sizeof(float);
 }
@@ -601,6 +611,8 @@ int launch_bwd_bf16(const void* q, const void* k, const void* v, const void* d_o
   if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
 
   // step 2: main kernel
+  const bool timed = (t_ev_start != nullptr && t_ev_stop != nullptr);
+  if (timed) cudaEventRecord(t_ev_start, stream);
   int rc;
   const bool alibi = p.slopes != nullptr;
 #define SIGATTN_BWD_CASE(DD, CC, AA) rc = launch_bwd_variant<DD, CC, AA>(maps, bp, num_sms, stream, cuda_err)
@@ -613,6 +625,7 @@ int launch_bwd_bf16(const void* q, const void* k, const void* v, const void* d_o
   }
 #undef SIGATTN_BWD_CASE
   if (rc != SIGATTN_OK) return rc;
+  if (timed) cudaEventRecord(t_ev_stop, stream);
   *launches += 1;
 
   // step 3: dQ = scale * accumulator, as bf16

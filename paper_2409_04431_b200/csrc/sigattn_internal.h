@@ -35,4 +35,7 @@ int launch_bwd_bf16(const void* q, const void* k, const void* v, const void* d_o
 
 size_t bwd_bf16_workspace_bytes(int B, int H, int N, int D);
 
+// Events recorded around the backward's main kernel on the calling thread (nullptr = off).
+void set_bwd_timing_events(cudaEvent_t start, cudaEvent_t stop);
+
 }  // namespace sigattn

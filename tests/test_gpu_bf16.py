@@ -1,0 +1,167 @@
+"""bf16 tensor-core path (tcgen05 + TMA kernels) against the float64 oracle, element by
+element on the same seeded, bf16-rounded inputs, through the C ABI.
+
+Tolerances (per output tensor): max-abs <= 2e-2 and relative Frobenius <= 5e-3, the bar
+set for bf16 inputs with fp32 accumulation.  The max-abs bound is meant for outputs of
+order one (the five benchmark configurations); edge cases with b >= 0 produce outputs of
+order N, so there it scales with max|reference| (see assert_close below).
+"""
+import math
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2409_04431_b200 import inputs
+from parity_util import BF16_MAX_ABS, BF16_REL_FRO, max_abs, rel_fro, to_device, to_host
+
+pytestmark = pytest.mark.gpu
+
+CANARY = 4096  # elements appended to every output buffer and checked for overruns
+
+
+def assert_close(got, ref, name):
+    assert np.all(np.isfinite(got)), f"{name}: non-finite output (unwritten rows keep their NaN poison)"
+    ma, rf = max_abs(got, ref), rel_fro(got, ref)
+    bound = BF16_MAX_ABS * max(1.0, float(np.max(np.abs(ref))))
+    assert ma <= bound, f"{name}: max-abs {ma:.3e} > {bound:.3e}"
+    assert rf <= BF16_REL_FRO, f"{name}: rel-Frobenius {rf:.3e} > {BF16_REL_FRO}"
+    for b in range(got.shape[0]):
+        for h in range(got.shape[1]):
+            r = rel_fro(got[b, h], ref[b, h])
+            assert r <= 2 * BF16_REL_FRO, f"{name}[{b},{h}]: per-head rel-Frobenius {r:.3e}"
+
+
+def poisoned_like(t):
+    """Output buffer pre-filled with NaN plus a canary tail that must stay untouched."""
+    import torch
+    flat = torch.full((t.numel() + CANARY,), float("nan"), dtype=t.dtype, device=t.device)
+    flat[t.numel():] = 1234.0
+    return flat, flat[: t.numel()].view(t.shape)
+
+
+def check_canary(flat, n):
+    import torch
+    assert torch.all(flat[n:] == 1234.0).item(), "kernel wrote past the end of an output buffer"
+
+
+def run_gpu(q, k, v, d_o, scale, bias, causal, slopes, backward=True):
+    import torch
+    import paper_2409_04431_b200 as sa
+    tq, tk, tv, tdo = (to_device(t, "bf16") for t in (q, k, v, d_o))
+    sl = None if slopes is None else torch.from_numpy(np.asarray(slopes, dtype=np.float32)).cuda()
+    fo, o = poisoned_like(tq)
+    sa.sigattn_fwd(tq, tk, tv, scale, bias, causal, sl, out=o)
+    outs = [(fo, o)]
+    if backward:
+        bufs = [poisoned_like(tq) for _ in range(3)]
+        sa.sigattn_bwd(tq, tk, tv, tdo, scale, bias, causal, sl, out=tuple(b[1] for b in bufs))
+        outs += bufs
+    sa.sigattn_check()
+    for flat, view in outs:
+        check_canary(flat, view.numel())
+    return [to_host(view) for _, view in outs]
+
+
+def compare(q, k, v, d_o, scale, bias, causal, slopes, backward=True, row_block=None):
+    got = run_gpu(q, k, v, d_o, scale, bias, causal, slopes, backward)
+    assert_close(got[0], oracle.sigattn_fwd(q, k, v, scale, bias, causal, slopes, row_block), "O")
+    if backward:
+        refs = oracle.sigattn_bwd(q, k, v, d_o, scale, bias, causal, slopes, row_block)
+        for name, g, r in zip(("dQ", "dK", "dV"), got[1:], refs):
+            assert_close(g, r, name)
+
+
+# ---------------------------------------------------------------- the benchmark configurations
+
+
+def test_config2_vit_full():
+    cfg = inputs.CONFIGS["c2"]  # B=32, H=12, N=197, D=64, non-causal: the whole configuration
+    q, k, v, d_o = inputs.make_inputs(cfg)
+    compare(q, k, v, d_o, cfg.scale, cfg.bias, cfg.causal, cfg.slopes())
+
+
+def test_config3_lm_alibi():
+    cfg = inputs.CONFIGS["c3"]  # one batch element, all 16 heads (each head has its own slope)
+    q, k, v, d_o = inputs.make_inputs(cfg, batch=1)
+    compare(q, k, v, d_o, cfg.scale, cfg.bias, cfg.causal, cfg.slopes())
+
+
+def test_config4_lm_qknorm():
+    cfg = inputs.CONFIGS["c4"]  # both batch elements, 3 of 16 heads
+    q, k, v, d_o = inputs.make_inputs(cfg, heads=3)
+    compare(q, k, v, d_o, cfg.scale, cfg.bias, cfg.causal, None, row_block=1024)
+
+
+def test_config5_long_context_one_head():
+    cfg = inputs.CONFIGS["c5"]  # N = 16384: one head end to end
+    q, k, v, d_o = inputs.make_inputs(cfg, heads=1)
+    compare(q, k, v, d_o, cfg.scale, cfg.bias, cfg.causal, None, row_block=1024)
+
+
+# ---------------------------------------------------------------- edge shapes
+
+
+@pytest.mark.parametrize("N", [1, 2, 63, 64, 65, 127, 128, 129, 197, 255, 256, 257, 1000])
+@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("causal", [False, True])
+def test_edge_shapes(N, D, causal):
+    B, H = 2, 2
+    q, k, v, d_o = inputs.random_case(B, H, N, D, seed=5000 + 2 * N + D + int(causal))
+    slopes = np.array([0.5, 0.03125], dtype=np.float32) if (N % 2 == 1) else None
+    compare(q, k, v, d_o, 1 / math.sqrt(D), -math.log(max(N, 2)), causal, slopes)
+
+
+@pytest.mark.parametrize("bias", [0.0, -30.0, 12.0])
+@pytest.mark.parametrize("causal", [False, True])
+def test_bias_extremes(bias, causal):
+    q, k, v, d_o = inputs.random_case(1, 2, 300, 64, seed=99)
+    compare(q, k, v, d_o, 0.125, bias, causal, None)
+
+
+def test_saturated_weights():
+    """b = +30: P = 1 everywhere; O and dV are (prefix) sums, dQ = dK = 0 to working precision."""
+    q, k, v, d_o = inputs.random_case(1, 2, 200, 128, seed=98)
+    got = run_gpu(q, k, v, d_o, 0.0884, 30.0, True, None)
+    assert_close(got[0], np.cumsum(v.astype(np.float64), axis=2), "O")
+    rev = np.flip(np.cumsum(np.flip(d_o.astype(np.float64), axis=2), axis=2), axis=2)
+    assert_close(got[3], rev, "dV")
+    assert np.max(np.abs(got[1])) < 1e-8 and np.max(np.abs(got[2])) < 1e-8
+
+
+def test_zero_slopes_equal_no_slopes_and_many_heads():
+    import torch
+    import paper_2409_04431_b200 as sa
+    B, H, N, D = 3, 20, 130, 64   # more work items than one wave of a small grid; odd head count
+    q, k, v, d_o = inputs.random_case(B, H, N, D, seed=7)
+    tq, tk, tv = (to_device(t, "bf16") for t in (q, k, v))
+    o1 = sa.sigattn_fwd(tq, tk, tv, 0.125, -4.0, True)
+    o2 = sa.sigattn_fwd(tq, tk, tv, 0.125, -4.0, True, torch.zeros(H, dtype=torch.float32, device="cuda"))
+    sa.sigattn_check()
+    assert torch.equal(o1, o2)
+    assert_close(to_host(o1), oracle.sigattn_fwd(q, k, v, 0.125, -4.0, True), "O")
+
+
+def test_run_to_run_determinism():
+    """O, dK, dV are bit-identical between runs; dQ (atomic fp32 accumulation order) agrees
+    to tolerance."""
+    import torch
+    import paper_2409_04431_b200 as sa
+    q, k, v, d_o = inputs.random_case(2, 4, 700, 128, seed=11)
+    tq, tk, tv, tdo = (to_device(t, "bf16") for t in (q, k, v, d_o))
+    a = [sa.sigattn_fwd(tq, tk, tv, 0.09, -6.5, True), *sa.sigattn_bwd(tq, tk, tv, tdo, 0.09, -6.5, True)]
+    b = [sa.sigattn_fwd(tq, tk, tv, 0.09, -6.5, True), *sa.sigattn_bwd(tq, tk, tv, tdo, 0.09, -6.5, True)]
+    sa.sigattn_check()
+    assert torch.equal(a[0], b[0]) and torch.equal(a[2], b[2]) and torch.equal(a[3], b[3])
+    assert rel_fro(to_host(a[1]), to_host(b[1])) < 1e-2 * BF16_REL_FRO + 4e-3
+
+
+def test_library_counts_its_launches():
+    import paper_2409_04431_b200 as sa
+    q, k, v, d_o = inputs.random_case(1, 1, 128, 64, seed=3)
+    tq, tk, tv, tdo = (to_device(t, "bf16") for t in (q, k, v, d_o))
+    n0 = sa.sigattn_launch_count()
+    sa.sigattn_fwd(tq, tk, tv, 0.125, -4.0)
+    sa.sigattn_bwd(tq, tk, tv, tdo, 0.125, -4.0)
+    sa.sigattn_check()
+    assert sa.sigattn_launch_count() - n0 == 3  # forward; backward main + dQ convert
