@@ -78,6 +78,17 @@ struct BwdItem {
   int bh, j, i_begin, n;
 };
 
+// Ranks are ordered by decreasing cost; rounds alternate direction over the CTAs so that
+// expensive and cheap items pair up (static stand-in for longest-first scheduling).
+__device__ __forceinline__ int bwd_snake_rank(int round, int n_items) {
+  const int g = gridDim.x;
+  const int c = (round & 1) ? (g - 1 - static_cast<int>(blockIdx.x)) : static_cast<int>(blockIdx.x);
+  const int rank = round * g + c;
+  return rank < n_items ? rank : -1;
+}
+
+__device__ __forceinline__ int bwd_num_rounds(int n_items) { return (n_items + gridDim.x - 1) / gridDim.x; }
+
 template <bool CAUSAL>
 __device__ __forceinline__ BwdItem decode_bwd_item(const BwdParams& p, int item) {
   BwdItem w;
@@ -126,7 +137,9 @@ __device__ void bwd_load_role(const BwdParams& p, const CUtensorMap* tmQ, const 
     ++do_cnt;
     return true;
   };
-  for (int item = blockIdx.x; item < p.n_items; item += gridDim.x) {
+  for (int round = 0, rounds = bwd_num_rounds(p.n_items); round < rounds; ++round) {
+    const int item = bwd_snake_rank(round, p.n_items);
+    if (item < 0) continue;
     const BwdItem w = decode_bwd_item<CAUSAL>(p, item);
     if (!load_q(w.i_begin, w.bh)) return;
     if (!load_do(w.i_begin, w.bh)) return;
@@ -169,7 +182,9 @@ __device__ void bwd_mma_role(const BwdParams& p, uint32_t smem_base, uint32_t tm
     }
   };
 
-  for (int item = blockIdx.x; item < p.n_items; item += gridDim.x) {
+  for (int round = 0, rounds = bwd_num_rounds(p.n_items); round < rounds; ++round) {
+    const int item = bwd_snake_rank(round, p.n_items);
+    if (item < 0) continue;
     const BwdItem w = decode_bwd_item<CAUSAL>(p, item);
     if (!mbar_wait(smem_u32(&bars->kv_full), item_cnt & 1, cta_err, 50)) return;
 
@@ -209,9 +224,15 @@ __device__ void bwd_mma_role(const BwdParams& p, uint32_t smem_base, uint32_t tm
         issue_kk(TM::kA, sK, smem_base + L::kQOff + nst * L::kTileBytes);
         umma_commit(smem_u32(&bars->s_full));
       }
-      // dK += dS^T Q_i ; dQ_i = dS K_j
+      // dQ_i = dS K_j first (its drain is on the critical path), then dK += dS^T Q_i
       if (!mbar_wait(smem_u32(&bars->ds_ready), step_cnt & 1, cta_err, 57)) return;
       tc_fence_after_sync();
+#pragma unroll
+      for (int ks = 0; ks < kT / 16; ++ks) {
+        umma_ss(tmem + TM::kB, make_smem_desc_sw128(sDs + ks * 2048, L::kPanelBytes, 1024),
+                make_smem_desc_sw128(sK + ks * 2048, L::kPanelBytes, 1024), kIdescDq, ks > 0);
+      }
+      umma_commit(smem_u32(&bars->dq_full));
 #pragma unroll
       for (int ks = 0; ks < kT / 16; ++ks) {
         umma_ss(tmem + TM::kDk,
@@ -220,12 +241,6 @@ __device__ void bwd_mma_role(const BwdParams& p, uint32_t smem_base, uint32_t tm
       }
       umma_commit(smem_u32(&bars->q_empty[st]));
       ++q_cnt;
-#pragma unroll
-      for (int ks = 0; ks < kT / 16; ++ks) {
-        umma_ss(tmem + TM::kB, make_smem_desc_sw128(sDs + ks * 2048, L::kPanelBytes, 1024),
-                make_smem_desc_sw128(sK + ks * 2048, L::kPanelBytes, 1024), kIdescDq, ks > 0);
-      }
-      umma_commit(smem_u32(&bars->dq_full));
       ++step_cnt;
       // dP^T of the next query tile (region B must have been drained of dQ_i first)
       if (more) {
@@ -322,7 +337,9 @@ __device__ void bwd_act_role(const BwdParams& p, const CUtensorMap* tmDk, const 
   const uint32_t lane_off = static_cast<uint32_t>(((threadIdx.x >> 5) & 3) * 32) << 16;
   uint32_t step_cnt = 0, item_cnt = 0;
 
-  for (int item = blockIdx.x; item < p.n_items; item += gridDim.x) {
+  for (int round = 0, rounds = bwd_num_rounds(p.n_items); round < rounds; ++round) {
+    const int item = bwd_snake_rank(round, p.n_items);
+    if (item < 0) continue;
     const BwdItem w = decode_bwd_item<CAUSAL>(p, item);
     float slope_log2e = 0.0f;
     if (ALIBI) slope_log2e = p.slopes[w.bh % p.H] * kLog2eB;
@@ -409,40 +426,47 @@ __device__ void bwd_drain_role(const BwdParams& p, const CUtensorMap* tmW, uint8
   using TM = BwdTmem<D>;
   const int tid = threadIdx.x & 127;  // query row within the tile
   const uint32_t lane_off = static_cast<uint32_t>(((threadIdx.x >> 5) & 3) * 32) << 16;
-  uint32_t step_cnt = 0, box_cnt = 0;
-  for (int item = blockIdx.x; item < p.n_items; item += gridDim.x) {
+  uint32_t step_cnt = 0;
+  for (int round = 0, rounds = bwd_num_rounds(p.n_items); round < rounds; ++round) {
+    const int item = bwd_snake_rank(round, p.n_items);
+    if (item < 0) continue;
     const BwdItem w = decode_bwd_item<CAUSAL>(p, item);
     for (int it = 0; it < w.n; ++it) {
       const int row0 = (w.i_begin + it) * kT;
       if (!mbar_wait(smem_u32(&bars->dq_full), step_cnt & 1, cta_err, 70)) return;
       ++step_cnt;
       tc_fence_after_sync();
+      // 64 columns per round: both staging boxes are filled from registers, so region B is
+      // released right after the last TMEM read instead of after the last reduce-add.
 #pragma unroll 1
-      for (int c = 0; c < D / 32; ++c) {
-        uint32_t o[32];
-        tmem_ld32(tmem + TM::kB + lane_off + c * 32, o);
+      for (int r = 0; r < D / 64; ++r) {
+        uint32_t o0[32], o1[32];
+        tmem_ld32(tmem + TM::kB + lane_off + r * 64, o0);
+        tmem_ld32(tmem + TM::kB + lane_off + r * 64 + 32, o1);
         tmem_wait_ld();
-        if (c == D / 32 - 1) {
+        if (r == D / 64 - 1) {
           tc_fence_before_sync();
           mbar_arrive(smem_u32(&bars->dq_empty));
         }
-        // the staging box used two boxes ago must have been read by its reduce-add
-        if (tid == 0) tma_wait_group_read<1>();
+        // both staging boxes must have been read by the reduce-adds issued earlier
+        if (tid == 0) tma_wait_group_read<0>();
         named_barrier_sync<3, 128>();
-        uint8_t* box = smem + L::kDqOff + (box_cnt & 1) * L::kPanelBytes;
-        uint8_t* rowp = box + tid * 128;
+        uint8_t* row0p = smem + L::kDqOff + tid * 128;
+        uint8_t* row1p = row0p + L::kPanelBytes;
 #pragma unroll
         for (int g = 0; g < 8; ++g) {
-          uint4 val = make_uint4(o[4 * g + 0], o[4 * g + 1], o[4 * g + 2], o[4 * g + 3]);
-          *reinterpret_cast<uint4*>(rowp + ((g ^ (tid & 7)) * 16)) = val;
+          *reinterpret_cast<uint4*>(row0p + ((g ^ (tid & 7)) * 16)) =
+              make_uint4(o0[4 * g + 0], o0[4 * g + 1], o0[4 * g + 2], o0[4 * g + 3]);
+          *reinterpret_cast<uint4*>(row1p + ((g ^ (tid & 7)) * 16)) =
+              make_uint4(o1[4 * g + 0], o1[4 * g + 1], o1[4 * g + 2], o1[4 * g + 3]);
         }
         fence_proxy_async_smem();
         named_barrier_sync<3, 128>();
         if (tid == 0) {
-          tma_reduce_add_3d(tmW, smem_u32(box), c * 32, row0, w.bh);
+          tma_reduce_add_3d(tmW, smem_u32(smem + L::kDqOff), r * 64, row0, w.bh);
+          tma_reduce_add_3d(tmW, smem_u32(smem + L::kDqOff + L::kPanelBytes), r * 64 + 32, row0, w.bh);
           tma_commit_group();
         }
-        ++box_cnt;
       }
     }
   }

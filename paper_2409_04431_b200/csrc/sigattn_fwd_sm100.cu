@@ -73,6 +73,19 @@ struct Item {
   int bh, row0, n_kv, n[2];
 };
 
+// Work items are ranked by decreasing cost (causal: later query tiles see more keys).
+// Round r of the persistent loop hands ranks [r G, (r + 1) G) to the G CTAs, forwards in
+// even rounds and backwards in odd rounds, so a CTA that drew an expensive item in one
+// round draws a cheap one in the next (a static stand-in for longest-first scheduling).
+__device__ __forceinline__ int snake_rank(int round, int n_items) {
+  const int g = gridDim.x;
+  const int c = (round & 1) ? (g - 1 - static_cast<int>(blockIdx.x)) : static_cast<int>(blockIdx.x);
+  const int rank = round * g + c;
+  return rank < n_items ? rank : -1;
+}
+
+__device__ __forceinline__ int num_rounds(int n_items) { return (n_items + gridDim.x - 1) / gridDim.x; }
+
 template <bool CAUSAL>
 __device__ __forceinline__ Item decode_item(const FwdParams& p, int item) {
   Item w;
@@ -97,7 +110,9 @@ __device__ void fwd_load_role(const FwdParams& p, const CUtensorMap* tmQ, const 
   using L = FwdSmem<D>;
   uint32_t kv_cnt = 0;
   uint32_t q_iter[2] = {0, 0};
-  for (int item = blockIdx.x; item < p.n_items; item += gridDim.x) {
+  for (int round = 0, rounds = num_rounds(p.n_items); round < rounds; ++round) {
+    const int item = snake_rank(round, p.n_items);
+    if (item < 0) continue;
     const Item w = decode_item<CAUSAL>(p, item);
     auto load_q = [&](int t) -> bool {
       if (w.n[t] == 0) return true;
@@ -171,7 +186,9 @@ __device__ void fwd_mma_role(const FwdParams& p, uint32_t smem_base, uint32_t tm
   auto kv_addr = [&](uint32_t cnt) { return smem_base + L::kKvOff + (cnt % L::kStages) * L::kTileBytes; };
   auto kv_release = [&](uint32_t cnt) { umma_commit(smem_u32(&bars->kv_empty[cnt % L::kStages])); };
 
-  for (int item = blockIdx.x; item < p.n_items; item += gridDim.x) {
+  for (int round = 0, rounds = num_rounds(p.n_items); round < rounds; ++round) {
+    const int item = snake_rank(round, p.n_items);
+    if (item < 0) continue;
     const Item w = decode_item<CAUSAL>(p, item);
     // ring positions: K_j at kv_cnt + 2 j (j > 0: 2 j), V_j right after K_j ... order K0 V0 K1 V1 ...
     const uint32_t base_cnt = kv_cnt;
@@ -289,7 +306,9 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, int t, 
   const uint32_t tO = tmem + 2 * kBN + t * D + lane_off;
   uint32_t s_cnt = 0, it = 0;
 
-  for (int item = blockIdx.x; item < p.n_items; item += gridDim.x) {
+  for (int round = 0, rounds = num_rounds(p.n_items); round < rounds; ++round) {
+    const int item = snake_rank(round, p.n_items);
+    if (item < 0) continue;
     const Item w = decode_item<CAUSAL>(p, item);
     const int nt = w.n[t];
     if (nt == 0) continue;
