@@ -25,6 +25,7 @@
 // 64-127 of the tile; every thread owns one key row), warps 8-11 dQ drain group,
 // warp 12 TMA producer, warp 13 MMA issuer.
 #include "sigattn_internal.h"
+#include "sigattn_activation.cuh"
 #include "sm100_primitives.cuh"
 #include "tensor_map.h"
 #include "../../include/sigattn.h"
@@ -262,7 +263,7 @@ __device__ void bwd_mma_role(const BwdParams& p, uint32_t smem_base, uint32_t tm
 // the dV product and P (1 - P) in fp32 for dS.
 //   a = log2(e) * (scale * s + b - slope * |i - j|);  u = 2^a;  P = u / (1 + u);  1 - P = 1 / (1 + u)
 template <bool DIAG, bool ALIBI>
-__device__ __forceinline__ void bwd_sigmoid_chunk(const uint32_t (&s)[32], uint32_t (&p_out)[16], float* pp,
+__device__ __forceinline__ void bwd_sigmoid_chunk(const uint32_t (&s)[32], uint32_t (&p_out)[16], float (&pp)[32],
                                                   float scale_log2e, float bias_log2e, float slope_log2e,
                                                   float col_rel, int q_base) {
   float a[32];
@@ -272,30 +273,8 @@ __device__ __forceinline__ void bwd_sigmoid_chunk(const uint32_t (&s)[32], uint3
     if (ALIBI) c0 = fmaf(-slope_log2e, fabsf(static_cast<float>(q_base + e) - col_rel), bias_log2e);
     a[e] = fmaf(__uint_as_float(s[e]), scale_log2e, c0);
   }
-  float m = fmax3(a[0], a[1], a[2]);
-#pragma unroll
-  for (int e = 3; e + 1 < 32; e += 2) m = fmax3(m, a[e], a[e + 1]);
-  m = fmaxf(m, a[31]);
   float pr[32];
-  if (m <= -3.0f) {
-#pragma unroll
-    for (int e = 0; e < 32; ++e) {
-      const float u = ex2_approx(a[e]);
-      float t = 1.0f - u;
-      t = fmaf(-u, t, 1.0f);
-      t = fmaf(-u, t, 1.0f);  // t ~ 1 / (1 + u)
-      pr[e] = u * t;
-      pp[e] = pr[e] * t;
-    }
-  } else {
-#pragma unroll
-    for (int e = 0; e < 32; ++e) {
-      const float u = ex2_approx(fminf(a[e], 64.0f));
-      const float r = rcp_approx(1.0f + u);
-      pr[e] = u * r;
-      pp[e] = pr[e] * r;
-    }
-  }
+  sigmoid_block<32, true, false>(a, pr, pp);
   if (DIAG) {
 #pragma unroll
     for (int e = 0; e < 32; ++e)
@@ -348,7 +327,7 @@ __device__ void bwd_act_role(const BwdParams& p, const CUtensorMap* tmDk, const 
       const int i = w.i_begin + it;
       const float col_rel = static_cast<float>((w.j - i) * kT + tid);  // key index minus first query of the tile
       const bool diag = CAUSAL && (it == 0);
-      float pp[64];
+      float pp0[32], pp1[32];
       if (!mbar_wait(smem_u32(&bars->s_full), step_cnt & 1, cta_err, 60 + wg)) return;
       tc_fence_after_sync();
 #pragma unroll
@@ -357,10 +336,11 @@ __device__ void bwd_act_role(const BwdParams& p, const CUtensorMap* tmDk, const 
         uint32_t s[32], pk[16];
         tmem_ld32(tmem + TM::kA + lane_off + gc * 32, s);
         tmem_wait_ld();
+        float(&ppc)[32] = (c == 0) ? pp0 : pp1;
         if (diag)
-          bwd_sigmoid_chunk<true, ALIBI>(s, pk, pp + 32 * c, p.scale_log2e, p.bias_log2e, slope_log2e, col_rel, gc * 32);
+          bwd_sigmoid_chunk<true, ALIBI>(s, pk, ppc, p.scale_log2e, p.bias_log2e, slope_log2e, col_rel, gc * 32);
         else
-          bwd_sigmoid_chunk<false, ALIBI>(s, pk, pp + 32 * c, p.scale_log2e, p.bias_log2e, slope_log2e, col_rel, gc * 32);
+          bwd_sigmoid_chunk<false, ALIBI>(s, pk, ppc, p.scale_log2e, p.bias_log2e, slope_log2e, col_rel, gc * 32);
         tmem_st16(tmem + TM::kA + lane_off + wg * 64 + c * 16, pk);
       }
       tmem_wait_st();
@@ -379,7 +359,7 @@ __device__ void bwd_act_role(const BwdParams& p, const CUtensorMap* tmDk, const 
 #pragma unroll
         for (int g = 0; g < 2; ++g) {
           uint4 val;
-          const float* f = pp + c * 16 + g * 8;
+          const float* f = ((c < 2) ? pp0 : pp1) + (c & 1) * 16 + g * 8;
           val.x = pack_bf16x2(f[0] * __uint_as_float(dp[8 * g + 0]), f[1] * __uint_as_float(dp[8 * g + 1]));
           val.y = pack_bf16x2(f[2] * __uint_as_float(dp[8 * g + 2]), f[3] * __uint_as_float(dp[8 * g + 3]));
           val.z = pack_bf16x2(f[4] * __uint_as_float(dp[8 * g + 4]), f[5] * __uint_as_float(dp[8 * g + 5]));

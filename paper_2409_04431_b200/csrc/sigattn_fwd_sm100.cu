@@ -17,13 +17,11 @@
 // Sigmoid needs no row maximum, no row sum and no rescaling of O (Section 4), so there is
 // no correction step and O is touched once, at the end.
 //
-// Activation.  With a = log2(e) * x:  u = 2^a;  if every a in a thread's 32-column chunk is
-// <= -3 (u <= 1/8, the usual case at b = -log n) then P = u (1 - u (1 - u (1 - u))), the
-// alternating series of u / (1 + u) cut after u^4 (relative error < 2^-12, below bf16
-// resolution): one MUFU op per element.  Otherwise P = u / (1 + u) with a reciprocal: two
-// MUFU ops.  The paper's 0.5 + 0.5 * tanh(x / 2) is not used: at x << 0 it subtracts two
-// nearly equal numbers and loses P's relative accuracy.
+// Activation: P = u / (1 + u) with u = 2^(log2(e) x), one MUFU op per element in the
+// common case; see sigattn_activation.cuh for the evaluation and for why the paper's
+// tanh form is not used.
 #include "sigattn_internal.h"
+#include "sigattn_activation.cuh"
 #include "sm100_primitives.cuh"
 #include "tensor_map.h"
 #include "../../include/sigattn.h"
@@ -39,6 +37,29 @@ constexpr int kFwdThreads = 320;
 constexpr int kLoadWarp = 8;
 constexpr int kMmaWarp = 9;
 constexpr float kLog2e = 1.4426950408889634f;
+constexpr int kTurnBarrier = 4;  // named barriers 4 and 5: activation turn of group 0 / 1
+#ifndef SIGATTN_FWD_PINGPONG
+#define SIGATTN_FWD_PINGPONG 0
+#endif
+
+#ifdef SIGATTN_TRACE
+// Development aid: one thread per role of CTA 0 logs (event id, clock) pairs into shared
+// memory; the log is copied to a global buffer when the kernel ends.
+__device__ long long g_trace[4][512];
+__device__ int g_trace_n[4];
+__shared__ long long s_trace[3][512];
+__shared__ int s_trace_n[3];
+#define TRACE(slot, ev)                                                         \
+  do {                                                                          \
+    if (blockIdx.x == 0) {                                                      \
+      const long long c_ = clock64();                                           \
+      const int n_ = s_trace_n[slot];                                           \
+      if (n_ < 255) { s_trace[slot][2 * n_] = (ev); s_trace[slot][2 * n_ + 1] = c_; s_trace_n[slot] = n_ + 1; } \
+    }                                                                           \
+  } while (0)
+#else
+#define TRACE(slot, ev) do {} while (0)
+#endif
 
 template <int D>
 struct FwdSmem {
@@ -218,6 +239,7 @@ __device__ void fwd_mma_role(const FwdParams& p, uint32_t smem_base, uint32_t tm
       if (j < w.n[0]) {
         if (!mbar_wait(smem_u32(&bars->p_full[0]), p_cnt[0] & 1, cta_err, 25)) return;
         ++p_cnt[0];
+        TRACE(2, 10);
         tc_fence_after_sync();
         issue_pv(0, kv_addr(v_cnt(j)), j > 0);
         if (j == w.n[0] - 1) umma_commit(smem_u32(&bars->o_full[0]));
@@ -231,6 +253,7 @@ __device__ void fwd_mma_role(const FwdParams& p, uint32_t smem_base, uint32_t tm
       if (j < w.n[1]) {
         if (!mbar_wait(smem_u32(&bars->p_full[1]), p_cnt[1] & 1, cta_err, 26)) return;
         ++p_cnt[1];
+        TRACE(2, 11);
         tc_fence_after_sync();
         issue_pv(1, kv_addr(v_cnt(j)), j > 0);
         if (j == w.n[1] - 1) umma_commit(smem_u32(&bars->o_full[1]));
@@ -250,49 +273,31 @@ __device__ void fwd_mma_role(const FwdParams& p, uint32_t smem_base, uint32_t tm
 
 // ------------------------------------------------------------------ activation + epilogue
 
-// 32 logits of one row -> 16 packed bf16x2 sigmoid values.
+// 64 logits of one row (two 32-column TMEM loads) -> 32 packed bf16x2 sigmoid values.
 //   a = s * scale_log2e + c0   (c0 carries the bias and, with ALiBi, the position term)
-template <bool CAUSAL_DIAG, bool ALIBI>
-__device__ __forceinline__ void sigmoid_chunk(const uint32_t (&s)[32], uint32_t (&out)[16], float scale_log2e,
-                                              float bias_log2e, float slope_log2e, float row_rel, int col_base) {
-  float a[32];
+template <bool ALIBI>
+__device__ __forceinline__ void sigmoid_block64(const uint32_t (&s0)[32], const uint32_t (&s1)[32],
+                                                uint32_t (&out)[32], float scale_log2e, float bias_log2e,
+                                                float slope_log2e, float row_rel, int col_base, bool causal_diag) {
+  float a[64];
 #pragma unroll
-  for (int i = 0; i < 32; ++i) {
+  for (int i = 0; i < 64; ++i) {
     float c0 = bias_log2e;
     if (ALIBI) {
       const float dist = row_rel - static_cast<float>(col_base + i);
       c0 = fmaf(-slope_log2e, fabsf(dist), bias_log2e);
     }
-    a[i] = fmaf(__uint_as_float(s[i]), scale_log2e, c0);
+    a[i] = fmaf(__uint_as_float(i < 32 ? s0[i & 31] : s1[i & 31]), scale_log2e, c0);
   }
-  float m = fmax3(a[0], a[1], a[2]);
+  float pr[64];
+  sigmoid_block<64, false, true>(a, pr, nullptr);
+  if (causal_diag) {  // keys after the query get weight 0 (only on the diagonal tile)
 #pragma unroll
-  for (int i = 3; i + 1 < 32; i += 2) m = fmax3(m, a[i], a[i + 1]);
-  m = fmaxf(m, a[31]);
-  float pr[32];
-  if (m <= -3.0f) {
-#pragma unroll
-    for (int i = 0; i < 32; ++i) {
-      const float u = ex2_approx(a[i]);
-      float t = 1.0f - u;
-      t = fmaf(-u, t, 1.0f);
-      t = fmaf(-u, t, 1.0f);
-      pr[i] = u * t;
-    }
-  } else {
-#pragma unroll
-    for (int i = 0; i < 32; ++i) {
-      const float u = ex2_approx(fminf(a[i], 64.0f));
-      pr[i] = u * rcp_approx(1.0f + u);
-    }
-  }
-  if (CAUSAL_DIAG) {
-#pragma unroll
-    for (int i = 0; i < 32; ++i)
+    for (int i = 0; i < 64; ++i)
       if (static_cast<float>(col_base + i) > row_rel) pr[i] = 0.0f;
   }
 #pragma unroll
-  for (int i = 0; i < 16; ++i) out[i] = pack_bf16x2(pr[2 * i], pr[2 * i + 1]);
+  for (int i = 0; i < 32; ++i) out[i] = pack_bf16x2(pr[2 * i], pr[2 * i + 1]);
 }
 
 template <int D, bool CAUSAL, bool ALIBI>
@@ -305,6 +310,7 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, int t, 
   const uint32_t tS = tmem + t * kBN + lane_off;
   const uint32_t tO = tmem + 2 * kBN + t * D + lane_off;
   uint32_t s_cnt = 0, it = 0;
+  if (SIGATTN_FWD_PINGPONG && t == 1) named_barrier_arrive<256>(kTurnBarrier);  // group 0 holds the first turn
 
   for (int round = 0, rounds = num_rounds(p.n_items); round < rounds; ++round) {
     const int item = snake_rank(round, p.n_items);
@@ -316,26 +322,34 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, int t, 
     float slope_log2e = 0.0f;
     if (ALIBI) slope_log2e = p.slopes[w.bh % p.H] * kLog2e;
 
+    const int n_pingpong = min(w.n[0], w.n[1]);
     for (int j = 0; j < nt; ++j) {
       if (!mbar_wait(smem_u32(&bars->s_full[t]), s_cnt & 1, cta_err, 30 + t)) return;
       ++s_cnt;
+      if (tid == 0) TRACE(t, 1);
+      // The two groups take turns on the MUFU pipe: while one evaluates its tile the tensor
+      // pipe works for the other.  Group 0 goes first; each hands the turn over when done.
+      if (SIGATTN_FWD_PINGPONG && j < n_pingpong) named_barrier_sync_id<256>(kTurnBarrier + t);
+      if (tid == 0) TRACE(t, 2);
       tc_fence_after_sync();
       const float row_rel = static_cast<float>(row - j * kBN);
       const bool diag = CAUSAL && (j == nt - 1);
+      // Two blocks of 64 columns; P (bf16) goes back over the columns already consumed.
 #pragma unroll 1
-      for (int c = 0; c < kBN / 32; ++c) {
-        uint32_t s[32], pk[16];
-        tmem_ld32(tS + c * 32, s);
+      for (int h = 0; h < kBN / 64; ++h) {
+        uint32_t s0[32], s1[32], pk[32];
+        tmem_ld32(tS + h * 64, s0);
+        tmem_ld32(tS + h * 64 + 32, s1);
         tmem_wait_ld();
-        if (diag)
-          sigmoid_chunk<true, ALIBI>(s, pk, p.scale_log2e, p.bias_log2e, slope_log2e, row_rel, c * 32);
-        else
-          sigmoid_chunk<false, ALIBI>(s, pk, p.scale_log2e, p.bias_log2e, slope_log2e, row_rel, c * 32);
-        tmem_st16(tS + c * 16, pk);
+        sigmoid_block64<ALIBI>(s0, s1, pk, p.scale_log2e, p.bias_log2e, slope_log2e, row_rel, h * 64, diag);
+        tmem_st32(tS + h * 32, pk);
       }
+      if (SIGATTN_FWD_PINGPONG && j < n_pingpong) named_barrier_arrive<256>(kTurnBarrier + (t ^ 1));
+      if (tid == 0) TRACE(t, 7);
       tmem_wait_st();
       tc_fence_before_sync();
       mbar_arrive(smem_u32(&bars->p_full[t]));
+      if (tid == 0) TRACE(t, 3);
     }
 
     // epilogue: O_t (fp32, tensor memory) -> bf16 -> swizzled shared memory (the Q_t buffer,
@@ -394,6 +408,9 @@ sigattn_fwd_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
   const uint32_t smem_base = smem_u32(smem);
   const int warp = threadIdx.x >> 5;
 
+#ifdef SIGATTN_TRACE
+  if (threadIdx.x < 3) s_trace_n[threadIdx.x] = 0;
+#endif
   if (threadIdx.x == 0) {
     cta_err = 0;
     for (int t = 0; t < 2; ++t) {
@@ -437,6 +454,12 @@ sigattn_fwd_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
 
   tc_fence_before_sync();
   __syncthreads();
+#ifdef SIGATTN_TRACE
+  if (blockIdx.x == 0) {
+    for (int i = threadIdx.x; i < 3 * 512; i += blockDim.x) g_trace[i / 512][i % 512] = s_trace[i / 512][i % 512];
+    if (threadIdx.x < 3) g_trace_n[threadIdx.x] = s_trace_n[threadIdx.x];
+  }
+#endif
   if (cta_err != 0) {
     if (threadIdx.x == 0) atomicExch(p.status, 100 + cta_err);
     __nanosleep(100000);  // let copies in flight towards this CTA's shared memory land
@@ -509,3 +532,16 @@ int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const 
 }
 
 }  // namespace sigattn
+
+#ifdef SIGATTN_TRACE
+extern "C" __attribute__((visibility("default"))) int sigattn_trace_dump(long long* out, int* counts, int reset) {
+  cudaDeviceSynchronize();
+  cudaMemcpyFromSymbol(out, sigattn::g_trace, sizeof(long long) * 4 * 512);
+  cudaMemcpyFromSymbol(counts, sigattn::g_trace_n, sizeof(int) * 4);
+  if (reset) {
+    int z[4] = {0, 0, 0, 0};
+    cudaMemcpyToSymbol(sigattn::g_trace_n, z, sizeof(z));
+  }
+  return 0;
+}
+#endif
