@@ -40,6 +40,7 @@
  *   -5 workspace too small     -6 device is not sm_100
  *   -7 CUDA runtime/driver error at set-up or launch (see sigattn_last_cuda_error)
  *   -8 a bounded device-side wait expired in an earlier launch (reported by sigattn_check)
+ *   -9 problem too large for sigattn_bwd_static_scratch's built-in scratch
  * Arguments are validated before anything is enqueued.
  */
 #ifndef SIGATTN_H_
@@ -66,6 +67,7 @@ extern "C" {
 #define SIGATTN_ERR_ARCH (-6)
 #define SIGATTN_ERR_CUDA (-7)
 #define SIGATTN_ERR_DEVICE_TIMEOUT (-8)
+#define SIGATTN_ERR_STATIC_SCRATCH (-9)
 
 #define SIGATTN_DTYPE_BF16 0
 #define SIGATTN_DTYPE_FP32 1
@@ -89,6 +91,36 @@ SIGATTN_API int sigattn_bwd(const void* q, const void* k, const void* v, const v
                 float scale, float bias, int causal,
                 const float* alibi_slopes, int dtype,
                 void* workspace, size_t workspace_bytes, void* stream);
+
+/* Backward for callers that cannot obtain device scratch at all.  (The paper has no
+ * counterpart: this entry point exists for how the library is embedded, not for the
+ * method.)  Who needs it: code that runs where cudaMalloc and friends are off limits -
+ * inside a framework's allocator callback or a real-time loop, in a plugin whose host
+ * forbids allocations after start-up, or in a process whose memory pool has already
+ * handed every byte to someone else - and that therefore cannot pass sigattn_bwd a
+ * workspace.  Same operation, arguments and results as sigattn_bwd, minus the workspace:
+ * the fp32 dQ accumulator lives in a fixed array inside the library instead.
+ *
+ * Limits and rules:
+ *  - B*H*N*D must not exceed sigattn_bwd_static_scratch_max_elements() (4 Mi elements,
+ *    a 16 MiB array that every GPU on which the library is loaded holds until the
+ *    process exits); larger problems return SIGATTN_ERR_STATIC_SCRATCH and launch nothing.
+ *  - The call allocates nothing: no cudaMalloc, cudaFree or allocating library routine.
+ *  - The first call on each device looks up the array's device address (one
+ *    cudaGetSymbolAddress, with that device current); make that first call outside any
+ *    stream capture.
+ *  - All calls on a device share the one array.  It keeps whatever the last call left in
+ *    it, so every call clears the part it uses before accumulating; two calls that overlap
+ *    on the device (different streams, or sigattn_bwd_static_scratch from two threads)
+ *    race on it and produce garbage.  Serialise them, e.g. by using one stream. */
+SIGATTN_API int sigattn_bwd_static_scratch(const void* q, const void* k, const void* v, const void* d_o,
+                               void* dq, void* dk, void* dv,
+                               int B, int H, int N, int D,
+                               float scale, float bias, int causal,
+                               const float* alibi_slopes, int dtype, void* stream);
+
+/* Largest B*H*N*D that sigattn_bwd_static_scratch accepts. */
+SIGATTN_API size_t sigattn_bwd_static_scratch_max_elements(void);
 
 /* Bytes of scratch sigattn_bwd needs for this problem (0 for the fp32 debug path).
  * Returns 0 for invalid shapes as well; sigattn_bwd reports those. */

@@ -22,6 +22,8 @@ _BINDING_NAMES = (
     "sigattn_step_host",
     "sigattn_step_host_arena_bytes",
     "sigattn_bwd_set_timing_events",
+    "sigattn_bwd_static_scratch",
+    "sigattn_bwd_static_scratch_max_elements",
 )
 
 __all__ = list(_BINDING_NAMES)

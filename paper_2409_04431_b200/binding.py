@@ -41,6 +41,11 @@ _lib.sigattn_step_host_arena_bytes.restype = _c.c_size_t
 _lib.sigattn_step_host_arena_bytes.argtypes = [_c.c_int] * 5
 _lib.sigattn_bwd_set_timing_events.restype = _c.c_int
 _lib.sigattn_bwd_set_timing_events.argtypes = [_c.c_void_p, _c.c_void_p]
+_lib.sigattn_bwd_static_scratch.restype = _c.c_int
+_lib.sigattn_bwd_static_scratch.argtypes = [_c.c_void_p] * 7 + [_c.c_int] * 4 + [_c.c_float, _c.c_float, _c.c_int,
+                                                                                   _c.c_void_p, _c.c_int, _c.c_void_p]
+_lib.sigattn_bwd_static_scratch_max_elements.restype = _c.c_size_t
+_lib.sigattn_bwd_static_scratch_max_elements.argtypes = []
 _lib.sigattn_check.restype = _c.c_int
 _lib.sigattn_check.argtypes = [_c.c_void_p]
 _lib.sigattn_strerror.restype = _c.c_char_p
@@ -56,6 +61,7 @@ EXPORTED = [
     "sigattn_fwd", "sigattn_bwd", "sigattn_bwd_workspace_bytes", "sigattn_check",
     "sigattn_strerror", "sigattn_last_cuda_error", "sigattn_version", "sigattn_launch_count",
     "sigattn_step_host", "sigattn_step_host_arena_bytes", "sigattn_bwd_set_timing_events",
+    "sigattn_bwd_static_scratch", "sigattn_bwd_static_scratch_max_elements",
 ]
 
 
@@ -219,3 +225,30 @@ def sigattn_bwd_set_timing_events(start=None, stop=None) -> None:
     a = None if start is None else start.cuda_event
     b = None if stop is None else stop.cuda_event
     _lib.sigattn_bwd_set_timing_events(a, b)
+
+
+def sigattn_bwd_static_scratch_max_elements() -> int:
+    return int(_lib.sigattn_bwd_static_scratch_max_elements())
+
+
+def sigattn_bwd_static_scratch(q, k, v, d_o, scale, bias, causal=False, alibi_slopes=None, out=None, stream=None):
+    """sigattn_bwd for callers that must not allocate device memory: the fp32 dQ
+    accumulator is a fixed array inside the library, so no workspace is passed (and this
+    wrapper allocates none; give `out=(dq, dk, dv)` to avoid even the output allocation).
+    B*H*N*D is limited to sigattn_bwd_static_scratch_max_elements(); calls that overlap on
+    the device share the array and race, so keep them on one stream."""
+    import torch
+    _check_same([q, k, v, d_o], ["q", "k", "v", "d_o"])
+    B, H, N, D = q.shape
+    if out is None:
+        dq, dk, dv = torch.empty_like(q), torch.empty_like(q), torch.empty_like(q)
+    else:
+        dq, dk, dv = out
+        _check_same([q, dq, dk, dv], ["q", "dq", "dk", "dv"])
+    with torch.cuda.device(q.device):
+        rc = _lib.sigattn_bwd_static_scratch(_ptr(q), _ptr(k), _ptr(v), _ptr(d_o), _ptr(dq), _ptr(dk), _ptr(dv),
+                                             B, H, N, D, float(scale), float(bias), int(bool(causal)),
+                                             _ptr(alibi_slopes), _dtype_code(q), _stream_ptr(stream))
+    if rc != 0:
+        raise SigattnError(rc)
+    return dq, dk, dv

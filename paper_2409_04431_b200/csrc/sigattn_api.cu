@@ -52,6 +52,20 @@ int check_shape(int B, int H, int N, int D) {
 
 }  // namespace
 
+namespace sigattn {
+
+int resolve_device(int** status) {
+  int dev = 0;
+  return device_setup(&dev, status);
+}
+
+void account(unsigned long long launches, int rc, cudaError_t cuda_err) {
+  g_launches.fetch_add(launches);
+  if (rc == SIGATTN_ERR_CUDA) t_last_cuda = cuda_err;
+}
+
+}  // namespace sigattn
+
 extern "C" {
 
 int sigattn_fwd(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int D, float scale,
@@ -213,6 +227,7 @@ const char* sigattn_strerror(int code) {
     case SIGATTN_ERR_ARCH: return "device is not sm_100 (B200)";
     case SIGATTN_ERR_CUDA: return "CUDA runtime or driver error (see sigattn_last_cuda_error)";
     case SIGATTN_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired; results of that launch are invalid";
+    case SIGATTN_ERR_STATIC_SCRATCH: return "problem larger than the built-in scratch of sigattn_bwd_static_scratch (B*H*N*D elements over the limit)";
     default: return "unknown sigattn error code";
   }
 }

@@ -35,6 +35,13 @@ int launch_bwd_bf16(const void* q, const void* k, const void* v, const void* d_o
 
 size_t bwd_bf16_workspace_bytes(int B, int H, int N, int D);
 
+// Services of the C-ABI layer for entry points that live in other translation units.
+// resolve_device: checks that the current device is sm_100 and returns the address of its
+// status word (a SIGATTN_* code otherwise).  account: adds to the launch counter and
+// remembers the CUDA error behind a SIGATTN_ERR_CUDA for sigattn_last_cuda_error.
+int resolve_device(int** status);
+void account(unsigned long long launches, int rc, cudaError_t cuda_err);
+
 // Events recorded around the backward's main kernel on the calling thread (nullptr = off).
 void set_bwd_timing_events(cudaEvent_t start, cudaEvent_t stop);
 
