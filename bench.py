@@ -30,7 +30,7 @@ sys.path.insert(0, ROOT)
 
 import numpy as np  # noqa: E402
 
-from paper_2409_04431_b200 import inputs  # noqa: E402
+from paper_2409_04431_b200 import inputs, sharding  # noqa: E402
 
 METRIC = "sigmoid-attn fwd+bwd bf16 TFLOP/s"
 UNIT = "TFLOP/s"
@@ -227,7 +227,7 @@ def run_ours(args, cfg):
     code = 0 if cfg.dtype == "bf16" else 1
 
     # host inputs (seeded; each rank its own batch) -> pinned host tensors -> device
-    qh, kh, vh, doh = inputs.make_inputs(cfg, seed=inputs.SEED_BASE + cfg.index + 1000 * rank)
+    qh, kh, vh, doh = inputs.make_inputs(cfg, seed=sharding.rank_seed(cfg, rank))
 
     def to_torch_host(x):
         if cfg.dtype == "bf16":
@@ -315,16 +315,14 @@ def run_ours(args, cfg):
     t_e2e = e0.elapsed_time(e1) / e2e_steps
 
     # max over ranks
-    stats = torch.tensor([t_total, t_fwd, t_bwd, t_e2e, float(np.mean(kern_ms))], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(stats, op=dist.ReduceOp.MAX)
-    t_total, t_fwd, t_bwd, t_e2e, t_kern = stats.tolist()
+    t_total, t_fwd, t_bwd, t_e2e, t_kern = sharding.max_over_ranks(
+        [t_total, t_fwd, t_bwd, t_e2e, float(np.mean(kern_ms))], device=dev)
 
     if rank == 0:
         peaks, peak_src = load_peaks()
         f_fwd, f_bwd = cfg.flops_fwd(), cfg.flops_bwd()
         per_step_ms = t_total / steps
-        value = world * (f_fwd + f_bwd) * steps / (t_total * 1e-3) / 1e12
+        value = sharding.whole_job_tflops(f_fwd + f_bwd, steps, world, t_total)
         fwd_tf = f_fwd * steps / (t_fwd * 1e-3) / 1e12
         bwd_tf = f_bwd * steps / (t_bwd * 1e-3) / 1e12
         kern_tf = f_bwd / (t_kern * 1e-3) / 1e12

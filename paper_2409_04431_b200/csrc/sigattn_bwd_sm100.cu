@@ -174,14 +174,25 @@ __device__ void bwd_mma_role(const BwdParams& p, uint32_t smem_base, uint32_t tm
   uint32_t q_cnt = 0, do_cnt = 0, item_cnt = 0, step_cnt = 0;
 
   // [128 x 128] = X[128 x D] * Y[128 x D]^T, both K-major
-  auto issue_kk = [&](uint32_t d_col, uint32_t x, uint32_t y) {
+  auto issue_kk = [&](uint32_t d_col, uint64_t x_desc, uint64_t y_desc) {
 #pragma unroll
     for (int ks = 0; ks < D / 16; ++ks) {
       const uint32_t off = (ks >> 2) * L::kPanelBytes + (ks & 3) * 32;
-      umma_ss(tmem + d_col, make_smem_desc_sw128(x + off, 16, 1024), make_smem_desc_sw128(y + off, 16, 1024),
-              kIdescSt, ks > 0);
+      umma_ss(tmem + d_col, desc_advance(x_desc, off), desc_advance(y_desc, off), kIdescSt, ks > 0);
     }
   };
+  // Descriptors are built once; each k-step only advances the start address.
+  const uint64_t dK_k = make_smem_desc_sw128(sK, 16, 1024);                 // K_j, K-major (S^T)
+  const uint64_t dV_k = make_smem_desc_sw128(sV, 16, 1024);                 // V_j, K-major (dP^T)
+  const uint64_t dDo_k = make_smem_desc_sw128(sDo, 16, 1024);               // dO_i, K-major (dP^T)
+  const uint64_t dDo_mn = make_smem_desc_sw128(sDo, L::kPanelBytes, 1024);  // dO_i, MN-major (dV)
+  const uint64_t dK_mn = make_smem_desc_sw128(sK, L::kPanelBytes, 1024);    // K_j, MN-major (dQ)
+  const uint64_t dDs_k = make_smem_desc_sw128(sDs, 16, 1024);               // dS^T, K-major (dK)
+  const uint64_t dDs_mn = make_smem_desc_sw128(sDs, L::kPanelBytes, 1024);  // dS^T, MN-major (dQ)
+  const uint64_t dQ_k[2] = {make_smem_desc_sw128(smem_base + L::kQOff, 16, 1024),
+                            make_smem_desc_sw128(smem_base + L::kQOff + L::kTileBytes, 16, 1024)};
+  const uint64_t dQ_mn[2] = {make_smem_desc_sw128(smem_base + L::kQOff, L::kPanelBytes, 1024),
+                             make_smem_desc_sw128(smem_base + L::kQOff + L::kTileBytes, L::kPanelBytes, 1024)};
 
   for (int round = 0, rounds = bwd_num_rounds(p.n_items); round < rounds; ++round) {
     const int item = bwd_snake_rank(round, p.n_items);
@@ -194,17 +205,16 @@ __device__ void bwd_mma_role(const BwdParams& p, uint32_t smem_base, uint32_t tm
       const uint32_t st = q_cnt & 1, ph = (q_cnt >> 1) & 1;
       if (!mbar_wait(smem_u32(&bars->q_full[st]), ph, cta_err, 51)) return;
       tc_fence_after_sync();
-      issue_kk(TM::kA, sK, smem_base + L::kQOff + st * L::kTileBytes);
+      issue_kk(TM::kA, dK_k, dQ_k[st]);
       umma_commit(smem_u32(&bars->s_full));
       if (!mbar_wait(smem_u32(&bars->do_full), do_cnt & 1, cta_err, 52)) return;
       if (!mbar_wait(smem_u32(&bars->dq_empty), (step_cnt & 1) ^ 1, cta_err, 53)) return;
       tc_fence_after_sync();
-      issue_kk(TM::kB, sV, sDo);
+      issue_kk(TM::kB, dV_k, dDo_k);
       umma_commit(smem_u32(&bars->dp_full));
     }
     for (int it = 0; it < w.n; ++it) {
       const uint32_t st = q_cnt & 1;
-      const uint32_t sQ = smem_base + L::kQOff + st * L::kTileBytes;
       const bool more = (it + 1 < w.n);
       // dV += P^T dO_i
       if (!mbar_wait(smem_u32(&bars->p_ready), step_cnt & 1, cta_err, 54)) return;
@@ -212,8 +222,8 @@ __device__ void bwd_mma_role(const BwdParams& p, uint32_t smem_base, uint32_t tm
       tc_fence_after_sync();
 #pragma unroll
       for (int ks = 0; ks < kT / 16; ++ks) {
-        umma_ts(tmem + TM::kDv, tmem + TM::kA + (ks >> 2) * 64 + (ks & 3) * 8,
-                make_smem_desc_sw128(sDo + ks * 2048, L::kPanelBytes, 1024), kIdescAcc, (it > 0 || ks > 0));
+        umma_ts(tmem + TM::kDv, tmem + TM::kA + (ks >> 2) * 64 + (ks & 3) * 8, desc_advance(dDo_mn, ks * 2048),
+                kIdescAcc, (it > 0 || ks > 0));
       }
       umma_commit(smem_u32(&bars->do_empty));
       ++do_cnt;
@@ -222,7 +232,7 @@ __device__ void bwd_mma_role(const BwdParams& p, uint32_t smem_base, uint32_t tm
         const uint32_t nst = (q_cnt + 1) & 1, nph = ((q_cnt + 1) >> 1) & 1;
         if (!mbar_wait(smem_u32(&bars->q_full[nst]), nph, cta_err, 56)) return;
         tc_fence_after_sync();
-        issue_kk(TM::kA, sK, smem_base + L::kQOff + nst * L::kTileBytes);
+        issue_kk(TM::kA, dK_k, dQ_k[nst]);
         umma_commit(smem_u32(&bars->s_full));
       }
       // dQ_i = dS K_j first (its drain is on the critical path), then dK += dS^T Q_i
@@ -230,15 +240,13 @@ __device__ void bwd_mma_role(const BwdParams& p, uint32_t smem_base, uint32_t tm
       tc_fence_after_sync();
 #pragma unroll
       for (int ks = 0; ks < kT / 16; ++ks) {
-        umma_ss(tmem + TM::kB, make_smem_desc_sw128(sDs + ks * 2048, L::kPanelBytes, 1024),
-                make_smem_desc_sw128(sK + ks * 2048, L::kPanelBytes, 1024), kIdescDq, ks > 0);
+        umma_ss(tmem + TM::kB, desc_advance(dDs_mn, ks * 2048), desc_advance(dK_mn, ks * 2048), kIdescDq, ks > 0);
       }
       umma_commit(smem_u32(&bars->dq_full));
 #pragma unroll
       for (int ks = 0; ks < kT / 16; ++ks) {
-        umma_ss(tmem + TM::kDk,
-                make_smem_desc_sw128(sDs + (ks >> 2) * L::kPanelBytes + (ks & 3) * 32, 16, 1024),
-                make_smem_desc_sw128(sQ + ks * 2048, L::kPanelBytes, 1024), kIdescAcc, (it > 0 || ks > 0));
+        umma_ss(tmem + TM::kDk, desc_advance(dDs_k, (ks >> 2) * L::kPanelBytes + (ks & 3) * 32),
+                desc_advance(dQ_mn[st], ks * 2048), kIdescAcc, (it > 0 || ks > 0));
       }
       umma_commit(smem_u32(&bars->q_empty[st]));
       ++q_cnt;
@@ -248,7 +256,7 @@ __device__ void bwd_mma_role(const BwdParams& p, uint32_t smem_base, uint32_t tm
         if (!mbar_wait(smem_u32(&bars->do_full), do_cnt & 1, cta_err, 58)) return;
         if (!mbar_wait(smem_u32(&bars->dq_empty), (step_cnt & 1) ^ 1, cta_err, 59)) return;
         tc_fence_after_sync();
-        issue_kk(TM::kB, sV, sDo);
+        issue_kk(TM::kB, dV_k, dDo_k);
         umma_commit(smem_u32(&bars->dp_full));
       }
     }

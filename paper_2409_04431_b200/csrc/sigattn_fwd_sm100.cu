@@ -9,10 +9,11 @@
 //   warp 9      MMA issuer (one thread): S_t = Q_t K_j^T into tensor memory, then
 //               O_t += P_t V_j with P read from tensor memory.  The two query tiles are
 //               interleaved so the tensor pipe works on one while the other is activated.
-//   warps 0-3   activation group of query tile 0: reads S from tensor memory (one row per
-//   warps 4-7   thread), evaluates P = sigmoid(.) in registers, writes bf16 P back over S.
-//               (same for tile 1)  At the end of an item the group converts its O
-//               accumulator to bf16 and stores it with TMA (rows >= N are clipped).
+//   warps 0-7   activation: 256 threads read S of one query tile from tensor memory (thread =
+//               one row x 64 key columns), evaluate P = sigmoid(.) in registers and write
+//               bf16 P back over S; they alternate between the two tiles.  At the end of an
+//               item they convert the O accumulators to bf16 and store them with TMA (rows
+//               >= N are clipped).
 //
 // Sigmoid needs no row maximum, no row sum and no rescaling of O (Section 4), so there is
 // no correction step and O is touched once, at the end.
@@ -37,14 +38,10 @@ constexpr int kFwdThreads = 320;
 constexpr int kLoadWarp = 8;
 constexpr int kMmaWarp = 9;
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr int kTurnBarrier = 4;  // named barriers 4 and 5: activation turn of group 0 / 1
-#ifndef SIGATTN_FWD_PINGPONG
-#define SIGATTN_FWD_PINGPONG 0
-#endif
 
 #ifdef SIGATTN_TRACE
-// Development aid: one thread per role of CTA 0 logs (event id, clock) pairs into shared
-// memory; the log is copied to a global buffer when the kernel ends.
+// Development aid (off in the product build): one thread per role of CTA 0 logs
+// (event id, clock) pairs into shared memory; copied to a global buffer at kernel end.
 __device__ long long g_trace[4][512];
 __device__ int g_trace_n[4];
 __shared__ long long s_trace[3][512];
@@ -182,22 +179,26 @@ __device__ void fwd_mma_role(const FwdParams& p, uint32_t smem_base, uint32_t tm
   uint32_t it[2] = {0, 0};      // items seen per query tile
   uint32_t p_cnt[2] = {0, 0};   // P tiles consumed per query tile
 
+  // Descriptors are built once per operand tile; each k-step only advances the start address.
+  const uint64_t q_desc[2] = {make_smem_desc_sw128(smem_base + L::kQOff, 16, 1024),
+                              make_smem_desc_sw128(smem_base + L::kQOff + L::kTileBytes, 16, 1024)};
   // S_t = Q_t K^T : both operands K-major, 128-byte swizzle.
   auto issue_s = [&](int t, uint32_t k_smem) {
-    const uint32_t q_smem = smem_base + L::kQOff + t * L::kTileBytes;
+    const uint64_t qd = q_desc[t];
+    const uint64_t kd = make_smem_desc_sw128(k_smem, 16, 1024);
 #pragma unroll
     for (int ks = 0; ks < D / 16; ++ks) {
       const uint32_t off = (ks >> 2) * L::kPanelBytes + (ks & 3) * 32;
-      umma_ss(tmem + t * kBN, make_smem_desc_sw128(q_smem + off, 16, 1024),
-              make_smem_desc_sw128(k_smem + off, 16, 1024), kIdescS, ks > 0);
+      umma_ss(tmem + t * kBN, desc_advance(qd, off), desc_advance(kd, off), kIdescS, ks > 0);
     }
   };
   // O_t (+)= P_t V : A = bf16 P in tensor memory (aliasing S_t), B = V, MN-major.
   auto issue_pv = [&](int t, uint32_t v_smem, bool accumulate) {
+    const uint64_t vd = make_smem_desc_sw128(v_smem, L::kPanelBytes, 1024);
 #pragma unroll
     for (int ks = 0; ks < kBN / 16; ++ks) {
-      umma_ts(tmem + 2 * kBN + t * D, tmem + t * kBN + ks * 8,
-              make_smem_desc_sw128(v_smem + ks * 2048, L::kPanelBytes, 1024), kIdescPV, (accumulate || ks > 0));
+      umma_ts(tmem + 2 * kBN + t * D, tmem + t * kBN + (ks >> 2) * 64 + (ks & 3) * 8, desc_advance(vd, ks * 2048),
+              kIdescPV, (accumulate || ks > 0));
     }
   };
   auto kv_wait = [&](uint32_t cnt) -> bool {
@@ -239,7 +240,7 @@ __device__ void fwd_mma_role(const FwdParams& p, uint32_t smem_base, uint32_t tm
       if (j < w.n[0]) {
         if (!mbar_wait(smem_u32(&bars->p_full[0]), p_cnt[0] & 1, cta_err, 25)) return;
         ++p_cnt[0];
-        TRACE(2, 10);
+        TRACE(2, 5);
         tc_fence_after_sync();
         issue_pv(0, kv_addr(v_cnt(j)), j > 0);
         if (j == w.n[0] - 1) umma_commit(smem_u32(&bars->o_full[0]));
@@ -249,11 +250,12 @@ __device__ void fwd_mma_role(const FwdParams& p, uint32_t smem_base, uint32_t tm
         tc_fence_after_sync();
         issue_s(0, kv_addr(k_cnt(j + 1)));
         umma_commit(smem_u32(&bars->s_full[0]));
+        TRACE(2, 6);
       }
       if (j < w.n[1]) {
         if (!mbar_wait(smem_u32(&bars->p_full[1]), p_cnt[1] & 1, cta_err, 26)) return;
         ++p_cnt[1];
-        TRACE(2, 11);
+        TRACE(2, 15);
         tc_fence_after_sync();
         issue_pv(1, kv_addr(v_cnt(j)), j > 0);
         if (j == w.n[1] - 1) umma_commit(smem_u32(&bars->o_full[1]));
@@ -262,6 +264,7 @@ __device__ void fwd_mma_role(const FwdParams& p, uint32_t smem_base, uint32_t tm
       if (j + 1 < w.n[1]) {
         issue_s(1, kv_addr(k_cnt(j + 1)));
         umma_commit(smem_u32(&bars->s_full[1]));
+        TRACE(2, 16);
       }
       if (more) kv_release(k_cnt(j + 1));
     }
@@ -300,95 +303,100 @@ __device__ __forceinline__ void sigmoid_block64(const uint32_t (&s0)[32], const 
   for (int i = 0; i < 32; ++i) out[i] = pack_bf16x2(pr[2 * i], pr[2 * i + 1]);
 }
 
+// Both activation groups (256 threads) work on the same query tile at a time, alternating
+// between the two tiles of the item: thread (g, r) owns row r and key columns
+// [64 g, 64 g + 64) of the tile.  While the groups evaluate one tile, the tensor pipe runs
+// P V and the next logits of the other one, so the MUFU pipe and the tensor pipe take turns
+// on a tile instead of competing for it.
 template <int D, bool CAUSAL, bool ALIBI>
-__device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, int t, uint8_t* smem, uint32_t tmem,
+__device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t* smem, uint32_t tmem,
                              FwdBarriers* bars, volatile int* cta_err) {
   using L = FwdSmem<D>;
+  const int g = (threadIdx.x >> 7) & 1;      // column half of the tile
   const int tid = threadIdx.x & 127;         // row of the tile
-  const int quarter = (threadIdx.x >> 5) & 3;  // TMEM lane quarter this warp may touch
-  const uint32_t lane_off = static_cast<uint32_t>(quarter * 32) << 16;
-  const uint32_t tS = tmem + t * kBN + lane_off;
-  const uint32_t tO = tmem + 2 * kBN + t * D + lane_off;
-  uint32_t s_cnt = 0, it = 0;
-  if (SIGATTN_FWD_PINGPONG && t == 1) named_barrier_arrive<256>(kTurnBarrier);  // group 0 holds the first turn
+  const uint32_t lane_off = static_cast<uint32_t>(((threadIdx.x >> 5) & 3) * 32) << 16;
+  uint32_t s_cnt[2] = {0, 0}, it[2] = {0, 0};
 
   for (int round = 0, rounds = num_rounds(p.n_items); round < rounds; ++round) {
     const int item = snake_rank(round, p.n_items);
     if (item < 0) continue;
     const Item w = decode_item<CAUSAL>(p, item);
-    const int nt = w.n[t];
-    if (nt == 0) continue;
-    const int row = w.row0 + t * kBM + tid;
     float slope_log2e = 0.0f;
     if (ALIBI) slope_log2e = p.slopes[w.bh % p.H] * kLog2e;
 
-    const int n_pingpong = min(w.n[0], w.n[1]);
-    for (int j = 0; j < nt; ++j) {
-      if (!mbar_wait(smem_u32(&bars->s_full[t]), s_cnt & 1, cta_err, 30 + t)) return;
-      ++s_cnt;
-      if (tid == 0) TRACE(t, 1);
-      // The two groups take turns on the MUFU pipe: while one evaluates its tile the tensor
-      // pipe works for the other.  Group 0 goes first; each hands the turn over when done.
-      if (SIGATTN_FWD_PINGPONG && j < n_pingpong) named_barrier_sync_id<256>(kTurnBarrier + t);
-      if (tid == 0) TRACE(t, 2);
-      tc_fence_after_sync();
-      const float row_rel = static_cast<float>(row - j * kBN);
-      const bool diag = CAUSAL && (j == nt - 1);
-      // Two blocks of 64 columns; P (bf16) goes back over the columns already consumed.
-#pragma unroll 1
-      for (int h = 0; h < kBN / 64; ++h) {
+    for (int j = 0; j < w.n_kv; ++j) {
+#pragma unroll
+      for (int t = 0; t < 2; ++t) {
+        if (j >= w.n[t]) continue;
+        if (!mbar_wait(smem_u32(&bars->s_full[t]), s_cnt[t] & 1, cta_err, 30 + t)) return;
+        ++s_cnt[t];
+        if (threadIdx.x == 0) TRACE(0, 1 + 10 * t);
+        if (threadIdx.x == 160) TRACE(1, 1 + 10 * t);
+        tc_fence_after_sync();
+        const float row_rel = static_cast<float>(w.row0 + t * kBM + tid - j * kBN);
+        const bool diag = CAUSAL && (j == w.n[t] - 1);
+        // 64 logits -> 64 weights; bf16 P goes back over the first half of the columns just read
+        const uint32_t tS = tmem + t * kBN + lane_off + g * 64;
         uint32_t s0[32], s1[32], pk[32];
-        tmem_ld32(tS + h * 64, s0);
-        tmem_ld32(tS + h * 64 + 32, s1);
+        tmem_ld32(tS, s0);
+        tmem_ld32(tS + 32, s1);
         tmem_wait_ld();
-        sigmoid_block64<ALIBI>(s0, s1, pk, p.scale_log2e, p.bias_log2e, slope_log2e, row_rel, h * 64, diag);
-        tmem_st32(tS + h * 32, pk);
+        if (threadIdx.x == 0) TRACE(0, 2 + 10 * t);
+        sigmoid_block64<ALIBI>(s0, s1, pk, p.scale_log2e, p.bias_log2e, slope_log2e, row_rel, g * 64, diag);
+        if (threadIdx.x == 0) TRACE(0, 3 + 10 * t);
+        if (threadIdx.x == 160) TRACE(1, 3 + 10 * t);
+        tmem_st32(tS, pk);
+        tmem_wait_st();
+        tc_fence_before_sync();
+        mbar_arrive(smem_u32(&bars->p_full[t]));
+        if (threadIdx.x == 0) TRACE(0, 4 + 10 * t);
       }
-      if (SIGATTN_FWD_PINGPONG && j < n_pingpong) named_barrier_arrive<256>(kTurnBarrier + (t ^ 1));
-      if (tid == 0) TRACE(t, 7);
-      tmem_wait_st();
-      tc_fence_before_sync();
-      mbar_arrive(smem_u32(&bars->p_full[t]));
-      if (tid == 0) TRACE(t, 3);
     }
 
     // epilogue: O_t (fp32, tensor memory) -> bf16 -> swizzled shared memory (the Q_t buffer,
-    // free once every logits MMA of the item is done) -> TMA store.
-    if (!mbar_wait(smem_u32(&bars->o_full[t]), it & 1, cta_err, 32 + t)) return;
-    ++it;
-    tc_fence_after_sync();
-    uint8_t* stage = smem + L::kQOff + t * L::kTileBytes;
-#pragma unroll 1
-    for (int c = 0; c < D / 32; ++c) {
-      uint32_t o[32];
-      tmem_ld32(tO + c * 32, o);
-      tmem_wait_ld();
-      uint8_t* panel = stage + (c >> 1) * L::kPanelBytes + tid * 128;
+    // free once every logits MMA of the item is done) -> TMA store.  Each group converts
+    // half of the D columns.
 #pragma unroll
-      for (int g = 0; g < 4; ++g) {
-        uint4 val;
-        val.x = pack_bf16x2(__uint_as_float(o[8 * g + 0]), __uint_as_float(o[8 * g + 1]));
-        val.y = pack_bf16x2(__uint_as_float(o[8 * g + 2]), __uint_as_float(o[8 * g + 3]));
-        val.z = pack_bf16x2(__uint_as_float(o[8 * g + 4]), __uint_as_float(o[8 * g + 5]));
-        val.w = pack_bf16x2(__uint_as_float(o[8 * g + 6]), __uint_as_float(o[8 * g + 7]));
-        const int chunk = (c & 1) * 4 + g;
-        *reinterpret_cast<uint4*>(panel + ((chunk ^ (tid & 7)) * 16)) = val;
+    for (int t = 0; t < 2; ++t) {
+      if (w.n[t] == 0) continue;
+      if (!mbar_wait(smem_u32(&bars->o_full[t]), it[t] & 1, cta_err, 32 + t)) return;
+      ++it[t];
+      tc_fence_after_sync();
+      uint8_t* stage = smem + L::kQOff + t * L::kTileBytes;
+      const uint32_t tO = tmem + 2 * kBN + t * D + lane_off + g * (D / 2);
+#pragma unroll
+      for (int c = 0; c < D / 64; ++c) {
+        uint32_t o[32];
+        tmem_ld32(tO + c * 32, o);
+        tmem_wait_ld();
+        // D = 128: group g fills panel g (8 chunks of 16 B); D = 64: half of the only panel
+        uint8_t* row_ptr = stage + (D == 128 ? g * L::kPanelBytes : 0) + tid * 128;
+#pragma unroll
+        for (int q4 = 0; q4 < 4; ++q4) {
+          uint4 val;
+          val.x = pack_bf16x2(__uint_as_float(o[8 * q4 + 0]), __uint_as_float(o[8 * q4 + 1]));
+          val.y = pack_bf16x2(__uint_as_float(o[8 * q4 + 2]), __uint_as_float(o[8 * q4 + 3]));
+          val.z = pack_bf16x2(__uint_as_float(o[8 * q4 + 4]), __uint_as_float(o[8 * q4 + 5]));
+          val.w = pack_bf16x2(__uint_as_float(o[8 * q4 + 6]), __uint_as_float(o[8 * q4 + 7]));
+          const int chunk = (D == 128 ? c * 4 : g * 4) + q4;
+          *reinterpret_cast<uint4*>(row_ptr + ((chunk ^ (tid & 7)) * 16)) = val;
+        }
+      }
+      tc_fence_before_sync();
+      mbar_arrive(smem_u32(&bars->o_empty[t]));
+      fence_proxy_async_smem();
+      named_barrier_sync<1, 256>();
+      if (threadIdx.x == 0) {
+#pragma unroll
+        for (int pn = 0; pn < L::kPanels; ++pn)
+          tma_store_3d(tmO, smem_u32(stage + pn * L::kPanelBytes), pn * 64, w.row0 + t * kBM, w.bh);
+        tma_commit_group();
+        tma_wait_group_read<0>();
+        mbar_arrive(smem_u32(&bars->q_empty[t]));
       }
     }
-    tc_fence_before_sync();
-    mbar_arrive(smem_u32(&bars->o_empty[t]));
-    fence_proxy_async_smem();
-    asm volatile("bar.sync %0, 128;" ::"r"(1 + t) : "memory");
-    if (tid == 0) {
-#pragma unroll
-      for (int pn = 0; pn < L::kPanels; ++pn)
-        tma_store_3d(tmO, smem_u32(stage + pn * L::kPanelBytes), pn * 64, w.row0 + t * kBM, w.bh);
-      tma_commit_group();
-      tma_wait_group_read<0>();
-      mbar_arrive(smem_u32(&bars->q_empty[t]));
-    }
   }
-  if (tid == 0) tma_wait_group<0>();
+  if (threadIdx.x == 0) tma_wait_group<0>();
 }
 
 // ------------------------------------------------------------------ kernel
@@ -417,9 +425,9 @@ sigattn_fwd_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
       mbar_init(smem_u32(&bars.q_full[t]), 1);
       mbar_init(smem_u32(&bars.q_empty[t]), 1);
       mbar_init(smem_u32(&bars.s_full[t]), 1);
-      mbar_init(smem_u32(&bars.p_full[t]), 128);
+      mbar_init(smem_u32(&bars.p_full[t]), 256);
       mbar_init(smem_u32(&bars.o_full[t]), 1);
-      mbar_init(smem_u32(&bars.o_empty[t]), 128);
+      mbar_init(smem_u32(&bars.o_empty[t]), 256);
     }
     for (int s = 0; s < L::kStages; ++s) {
       mbar_init(smem_u32(&bars.kv_full[s]), 1);
@@ -449,7 +457,7 @@ sigattn_fwd_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
     if ((threadIdx.x & 31) == 0) fwd_mma_role<D, CAUSAL>(p, smem_base, tmem, &bars, &cta_err);
     __syncwarp();
   } else {
-    fwd_act_role<D, CAUSAL, ALIBI>(p, &tmO, warp >> 2, smem, tmem, &bars, &cta_err);
+    fwd_act_role<D, CAUSAL, ALIBI>(p, &tmO, smem, tmem, &bars, &cta_err);
   }
 
   tc_fence_before_sync();
@@ -532,6 +540,7 @@ int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const 
 }
 
 }  // namespace sigattn
+
 
 #ifdef SIGATTN_TRACE
 extern "C" __attribute__((visibility("default"))) int sigattn_trace_dump(long long* out, int* counts, int reset) {

@@ -248,6 +248,13 @@ __device__ __forceinline__ uint64_t make_smem_desc_sw128(uint32_t smem_addr, uin
   return d;
 }
 
+// Descriptor of the same matrix `byte_offset` bytes further on (a multiple of 16 that keeps
+// the address inside the 256 KB window): only the start-address field changes, so issuing
+// the k-steps of a product costs one 64-bit add each instead of rebuilding the descriptor.
+__device__ __forceinline__ uint64_t desc_advance(uint64_t desc, uint32_t byte_offset) {
+  return desc + static_cast<uint64_t>(byte_offset >> 4);
+}
+
 // 32-bit instruction descriptor for kind::f16 with bf16 inputs and fp32 accumulation.
 // a_mn / b_mn: 1 if that operand is MN-major in shared memory, 0 if K-major.
 __host__ __device__ constexpr uint32_t make_idesc_bf16(int M, int N, int a_mn, int b_mn) {

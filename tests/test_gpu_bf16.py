@@ -165,3 +165,22 @@ def test_library_counts_its_launches():
     sa.sigattn_bwd(tq, tk, tv, tdo, 0.125, -4.0)
     sa.sigattn_check()
     assert sa.sigattn_launch_count() - n0 == 3  # forward; backward main + dQ convert
+
+
+def test_step_from_host_buffers():
+    """sigattn_step_host: H2D copies, forward, backward, D2H copies in one call."""
+    import torch
+    import paper_2409_04431_b200 as sa
+    B, H, N, D = 2, 4, 333, 64
+    q, k, v, d_o = inputs.random_case(B, H, N, D, seed=21)
+    slopes = np.array([0.5, 0.25, 0.125, 0.0625], dtype=np.float32)
+    host_in = [torch.from_numpy(inputs.f32_to_bf16_bits(t).view(np.int16)).view(torch.bfloat16).pin_memory()
+               for t in (q, k, v, d_o)]
+    host_out = [torch.full_like(host_in[0], float("nan")).pin_memory() for _ in range(4)]
+    scale, bias = 0.125, -math.log(N)
+    sa.sigattn_step_host(*host_in, *host_out, scale, bias, True, torch.from_numpy(slopes))
+    sa.sigattn_check()
+    got = [t.float().numpy().astype(np.float64) for t in host_out]
+    assert_close(got[0], oracle.sigattn_fwd(q, k, v, scale, bias, True, slopes), "O")
+    for name, g, r in zip(("dQ", "dK", "dV"), got[1:], oracle.sigattn_bwd(q, k, v, d_o, scale, bias, True, slopes)):
+        assert_close(g, r, name)
