@@ -3,14 +3,13 @@
 // With a = log2(e) * x and u = 2^a the weight is P = u / (1 + u) and 1 - P = 1 / (1 + u).
 // Both kernels work on a block of 32 or 64 logits of one thread at a time and evaluate
 //
-//   fast path   t = 1 - u + u^2,  P = u t,  P (1 - P) = P t
-//               (the alternating series of 1 / (1 + u) cut after u^2: relative error
-//               u^3 <= 2^-12 for a <= -4, i.e. below bf16 resolution; one MUFU op per
-//               element).  It is computed unconditionally, so that nothing waits on the
-//               reduction that decides whether it was allowed.
-//   exact path  e = 2^-a,  r = 1 / (1 + e),  P = r,  P (1 - P) = r e r  (two MUFU ops),
-//               taken afterwards if any logit of the block has a > -4.  At b = -log n almost
-//               no chunk needs it.
+//   common path  P = u - u^2 + u^3, the alternating series of u / (1 + u) (relative error
+//                u^3 <= 2^-12 for a <= -4, below bf16 resolution), and P (1 - P) = P - P^2;
+//                one exponential per element, a fixed share of them evaluated on the FMA
+//                pipe (ex2_emulated) instead of the MUFU pipe.
+//   exact path   e = 2^-a,  r = 1 / (1 + e),  P = r,  P (1 - P) = r e r  (two MUFU ops),
+//                taken if any logit of the block has a > -4.  At b = -log n almost no block
+//                needs it.
 //
 // The paper evaluates sigmoid as 0.5 (1 + tanh(x / 2)) with the hardware tanh (Section 4).
 // On B200 tanh.approx.f32 followed by 0.5 + 0.5 t loses P's relative accuracy for x << 0
@@ -50,32 +49,61 @@ __device__ __forceinline__ float max_tree(const float (&a)[N]) {
   return m[0];
 }
 
-// a[N] (already scaled by log2 e) -> P[N]; if WITH_SLOPE also P (1 - P) in pp[N].
-// SPECULATE = true evaluates the fast path before the decision is known (shortest
-// dependency chain, more live registers); false decides first.
-template <int N, bool WITH_SLOPE, bool SPECULATE>
-__device__ __forceinline__ void sigmoid_block(const float (&a)[N], float (&pr)[N], float* pp) {
-  bool exact;
-  if (!SPECULATE) exact = max_tree<N>(a) > kFastPathMaxA;
-  if (SPECULATE || !exact) {
+// 2^a on the FMA and ALU pipes instead of the MUFU pipe: a = n + f with n = round(a),
+// 2^f from a cubic on [-0.5, 0.5] (relative error 7.5e-5 = 2^-13.7, fitted for this
+// interval), 2^n by adding n to the exponent field.  Valid for -120 <= a (clamped) and
+// a < 100.  Used for a fixed share of the elements to take load off the MUFU pipe, which
+// otherwise bounds the activation at 16 elements per clock per SM.
+__device__ __forceinline__ float ex2_emulated(float a) {
+  a = fmaxf(a, -120.0f);
+  const float t = a + 12582912.0f;  // 1.5 * 2^23: the rounded integer lands in the low mantissa bits
+  const float f = a - (t - 12582912.0f);
+  float p = fmaf(0.05517145885f, f, 0.2426108620f);
+  p = fmaf(p, f, 0.6932609924f);
+  p = fmaf(p, f, 0.9999280895f);
+  return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
+}
+
+constexpr int kEmulateEvery = 4;  // every 4th exponential of the common path is emulated
+
+// Common path: u / (1 + u) = u - u^2 + u^3 - ..., cut after u^3 and evaluated as
+// u - u (u - u^2): two FMAs; relative error u^3 <= 2^-12 for a <= -4.
+template <int N, bool WITH_SLOPE, bool EMULATE>
+__device__ __forceinline__ void sigmoid_common(const float (&a)[N], float (&pr)[N], float* pp) {
 #pragma unroll
-    for (int i = 0; i < N; ++i) {
-      const float u = sm100::ex2_approx(a[i]);
-      float t = 1.0f - u;
-      t = fmaf(u, u, t);
-      pr[i] = u * t;
-      if (WITH_SLOPE) pp[i] = pr[i] * t;
-    }
+  for (int i = 0; i < N; ++i) {
+    const float u = (EMULATE && i % kEmulateEvery == kEmulateEvery - 1) ? ex2_emulated(a[i]) : sm100::ex2_approx(a[i]);
+    const float w = fmaf(-u, u, u);
+    pr[i] = fmaf(-u, w, u);
+    if (WITH_SLOPE) pp[i] = fmaf(-pr[i], pr[i], pr[i]);  // P <= 1/17 here: no cancellation in P - P^2
   }
-  if (SPECULATE) exact = max_tree<N>(a) > kFastPathMaxA;
-  if (exact) {
+}
+
+// Exact path: r = 1 / (1 + 2^-a) = P, and 1 - P = 2^-a r (no subtraction from a rounded P).
+template <int N, bool WITH_SLOPE>
+__device__ __forceinline__ void sigmoid_exact(const float (&a)[N], float (&pr)[N], float* pp) {
 #pragma unroll
-    for (int i = 0; i < N; ++i) {
-      const float e = sm100::ex2_approx(fminf(-a[i], 120.0f));
-      const float r = sm100::rcp_approx(1.0f + e);
-      pr[i] = r;
-      if (WITH_SLOPE) pp[i] = r * (e * r);
-    }
+  for (int i = 0; i < N; ++i) {
+    const float e = sm100::ex2_approx(fminf(-a[i], 120.0f));
+    const float r = sm100::rcp_approx(1.0f + e);
+    pr[i] = r;
+    if (WITH_SLOPE) pp[i] = r * (e * r);
+  }
+}
+
+// a[N] (already scaled by log2 e) -> P[N]; if WITH_SLOPE also P (1 - P) in pp[N].
+// SPECULATE = true evaluates the common path before the decision is known (shortest
+// dependency chain, more live registers) and redoes the block on the exact path if needed;
+// false decides first.  EMULATE moves every kEmulateEvery-th exponential of the common path
+// to the FMA pipe.
+template <int N, bool WITH_SLOPE, bool SPECULATE, bool EMULATE>
+__device__ __forceinline__ void sigmoid_block(const float (&a)[N], float (&pr)[N], float* pp) {
+  if (SPECULATE) {
+    sigmoid_common<N, WITH_SLOPE, EMULATE>(a, pr, pp);
+    if (max_tree<N>(a) > kFastPathMaxA) sigmoid_exact<N, WITH_SLOPE>(a, pr, pp);
+  } else {
+    if (max_tree<N>(a) <= kFastPathMaxA) sigmoid_common<N, WITH_SLOPE, EMULATE>(a, pr, pp);
+    else sigmoid_exact<N, WITH_SLOPE>(a, pr, pp);
   }
 }
 

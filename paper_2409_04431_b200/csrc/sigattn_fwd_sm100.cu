@@ -9,11 +9,12 @@
 //   warp 9      MMA issuer (one thread): S_t = Q_t K_j^T into tensor memory, then
 //               O_t += P_t V_j with P read from tensor memory.  The two query tiles are
 //               interleaved so the tensor pipe works on one while the other is activated.
-//   warps 0-7   activation: 256 threads read S of one query tile from tensor memory (thread =
-//               one row x 64 key columns), evaluate P = sigmoid(.) in registers and write
-//               bf16 P back over S; they alternate between the two tiles.  At the end of an
-//               item they convert the O accumulators to bf16 and store them with TMA (rows
-//               >= N are clipped).
+//   warps 0-7   activation: threads read S from tensor memory (one row each), evaluate
+//               P = sigmoid(.) in registers and write bf16 P back over S.  All 256 threads
+//               work on one query tile (64 key columns each) and alternate between the two
+//               tiles, so the MUFU pipe and the tensor pipe take turns on a tile.  At the end
+//               of an item they convert the O accumulators to bf16 and store them with TMA
+//               (rows >= N are clipped).
 //
 // Sigmoid needs no row maximum, no row sum and no rescaling of O (Section 4), so there is
 // no correction step and O is touched once, at the end.
@@ -39,24 +40,14 @@ constexpr int kLoadWarp = 8;
 constexpr int kMmaWarp = 9;
 constexpr float kLog2e = 1.4426950408889634f;
 
-#ifdef SIGATTN_TRACE
-// Development aid (off in the product build): one thread per role of CTA 0 logs
-// (event id, clock) pairs into shared memory; copied to a global buffer at kernel end.
-__device__ long long g_trace[4][512];
-__device__ int g_trace_n[4];
-__shared__ long long s_trace[3][512];
-__shared__ int s_trace_n[3];
-#define TRACE(slot, ev)                                                         \
-  do {                                                                          \
-    if (blockIdx.x == 0) {                                                      \
-      const long long c_ = clock64();                                           \
-      const int n_ = s_trace_n[slot];                                           \
-      if (n_ < 255) { s_trace[slot][2 * n_] = (ev); s_trace[slot][2 * n_ + 1] = c_; s_trace_n[slot] = n_ + 1; } \
-    }                                                                           \
-  } while (0)
-#else
-#define TRACE(slot, ev) do {} while (0)
+// Build-time switches of the forward activation (defaults = the measured best):
+#ifndef SIGATTN_FWD_SPECULATE
+#define SIGATTN_FWD_SPECULATE 0   // evaluate the common path before the block maximum is known
 #endif
+#ifndef SIGATTN_FWD_EMULATE
+#define SIGATTN_FWD_EMULATE 1     // every 4th exponential on the FMA pipe
+#endif
+
 
 template <int D>
 struct FwdSmem {
@@ -197,8 +188,10 @@ __device__ void fwd_mma_role(const FwdParams& p, uint32_t smem_base, uint32_t tm
     const uint64_t vd = make_smem_desc_sw128(v_smem, L::kPanelBytes, 1024);
 #pragma unroll
     for (int ks = 0; ks < kBN / 16; ++ks) {
-      umma_ts(tmem + 2 * kBN + t * D, tmem + t * kBN + (ks >> 2) * 64 + (ks & 3) * 8, desc_advance(vd, ks * 2048),
-              kIdescPV, (accumulate || ks > 0));
+      // bf16 P sits at columns [0, 32) (group 0) and [64, 96) (group 1) of S_t
+      const uint32_t p_col = (ks >> 2) * 64 + (ks & 3) * 8;
+      umma_ts(tmem + 2 * kBN + t * D, tmem + t * kBN + p_col, desc_advance(vd, ks * 2048), kIdescPV,
+              (accumulate || ks > 0));
     }
   };
   auto kv_wait = [&](uint32_t cnt) -> bool {
@@ -240,7 +233,6 @@ __device__ void fwd_mma_role(const FwdParams& p, uint32_t smem_base, uint32_t tm
       if (j < w.n[0]) {
         if (!mbar_wait(smem_u32(&bars->p_full[0]), p_cnt[0] & 1, cta_err, 25)) return;
         ++p_cnt[0];
-        TRACE(2, 5);
         tc_fence_after_sync();
         issue_pv(0, kv_addr(v_cnt(j)), j > 0);
         if (j == w.n[0] - 1) umma_commit(smem_u32(&bars->o_full[0]));
@@ -250,12 +242,10 @@ __device__ void fwd_mma_role(const FwdParams& p, uint32_t smem_base, uint32_t tm
         tc_fence_after_sync();
         issue_s(0, kv_addr(k_cnt(j + 1)));
         umma_commit(smem_u32(&bars->s_full[0]));
-        TRACE(2, 6);
       }
       if (j < w.n[1]) {
         if (!mbar_wait(smem_u32(&bars->p_full[1]), p_cnt[1] & 1, cta_err, 26)) return;
         ++p_cnt[1];
-        TRACE(2, 15);
         tc_fence_after_sync();
         issue_pv(1, kv_addr(v_cnt(j)), j > 0);
         if (j == w.n[1] - 1) umma_commit(smem_u32(&bars->o_full[1]));
@@ -264,7 +254,6 @@ __device__ void fwd_mma_role(const FwdParams& p, uint32_t smem_base, uint32_t tm
       if (j + 1 < w.n[1]) {
         issue_s(1, kv_addr(k_cnt(j + 1)));
         umma_commit(smem_u32(&bars->s_full[1]));
-        TRACE(2, 16);
       }
       if (more) kv_release(k_cnt(j + 1));
     }
@@ -293,7 +282,7 @@ __device__ __forceinline__ void sigmoid_block64(const uint32_t (&s0)[32], const 
     a[i] = fmaf(__uint_as_float(i < 32 ? s0[i & 31] : s1[i & 31]), scale_log2e, c0);
   }
   float pr[64];
-  sigmoid_block<64, false, true>(a, pr, nullptr);
+  sigmoid_block<64, false, SIGATTN_FWD_SPECULATE != 0, SIGATTN_FWD_EMULATE != 0>(a, pr, nullptr);
   if (causal_diag) {  // keys after the query get weight 0 (only on the diagonal tile)
 #pragma unroll
     for (int i = 0; i < 64; ++i)
@@ -315,7 +304,7 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
   const int g = (threadIdx.x >> 7) & 1;      // column half of the tile
   const int tid = threadIdx.x & 127;         // row of the tile
   const uint32_t lane_off = static_cast<uint32_t>(((threadIdx.x >> 5) & 3) * 32) << 16;
-  uint32_t s_cnt[2] = {0, 0}, it[2] = {0, 0};
+  uint32_t s_cnt0 = 0, s_cnt1 = 0, it[2] = {0, 0};
 
   for (int round = 0, rounds = num_rounds(p.n_items); round < rounds; ++round) {
     const int item = snake_rank(round, p.n_items);
@@ -324,32 +313,29 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
     float slope_log2e = 0.0f;
     if (ALIBI) slope_log2e = p.slopes[w.bh % p.H] * kLog2e;
 
+    // Tile-steps are visited in the order (j, tile 0), (j, tile 1), (j + 1, tile 0), ...
     for (int j = 0; j < w.n_kv; ++j) {
 #pragma unroll
       for (int t = 0; t < 2; ++t) {
         if (j >= w.n[t]) continue;
-        if (!mbar_wait(smem_u32(&bars->s_full[t]), s_cnt[t] & 1, cta_err, 30 + t)) return;
-        ++s_cnt[t];
-        if (threadIdx.x == 0) TRACE(0, 1 + 10 * t);
-        if (threadIdx.x == 160) TRACE(1, 1 + 10 * t);
+        uint32_t& cnt = t ? s_cnt1 : s_cnt0;
+        if (!mbar_wait(smem_u32(&bars->s_full[t]), cnt & 1, cta_err, 30 + t)) return;
+        ++cnt;
         tc_fence_after_sync();
         const float row_rel = static_cast<float>(w.row0 + t * kBM + tid - j * kBN);
         const bool diag = CAUSAL && (j == w.n[t] - 1);
-        // 64 logits -> 64 weights; bf16 P goes back over the first half of the columns just read
+        // bf16 P goes back over the first half of the 64 columns this thread has just read
         const uint32_t tS = tmem + t * kBN + lane_off + g * 64;
-        uint32_t s0[32], s1[32], pk[32];
+        uint32_t s0[32], s1[32];
         tmem_ld32(tS, s0);
         tmem_ld32(tS + 32, s1);
         tmem_wait_ld();
-        if (threadIdx.x == 0) TRACE(0, 2 + 10 * t);
+        uint32_t pk[32];
         sigmoid_block64<ALIBI>(s0, s1, pk, p.scale_log2e, p.bias_log2e, slope_log2e, row_rel, g * 64, diag);
-        if (threadIdx.x == 0) TRACE(0, 3 + 10 * t);
-        if (threadIdx.x == 160) TRACE(1, 3 + 10 * t);
         tmem_st32(tS, pk);
         tmem_wait_st();
         tc_fence_before_sync();
         mbar_arrive(smem_u32(&bars->p_full[t]));
-        if (threadIdx.x == 0) TRACE(0, 4 + 10 * t);
       }
     }
 
@@ -416,9 +402,6 @@ sigattn_fwd_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
   const uint32_t smem_base = smem_u32(smem);
   const int warp = threadIdx.x >> 5;
 
-#ifdef SIGATTN_TRACE
-  if (threadIdx.x < 3) s_trace_n[threadIdx.x] = 0;
-#endif
   if (threadIdx.x == 0) {
     cta_err = 0;
     for (int t = 0; t < 2; ++t) {
@@ -462,12 +445,6 @@ sigattn_fwd_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
 
   tc_fence_before_sync();
   __syncthreads();
-#ifdef SIGATTN_TRACE
-  if (blockIdx.x == 0) {
-    for (int i = threadIdx.x; i < 3 * 512; i += blockDim.x) g_trace[i / 512][i % 512] = s_trace[i / 512][i % 512];
-    if (threadIdx.x < 3) g_trace_n[threadIdx.x] = s_trace_n[threadIdx.x];
-  }
-#endif
   if (cta_err != 0) {
     if (threadIdx.x == 0) atomicExch(p.status, 100 + cta_err);
     __nanosleep(100000);  // let copies in flight towards this CTA's shared memory land
@@ -542,15 +519,3 @@ int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const 
 }  // namespace sigattn
 
 
-#ifdef SIGATTN_TRACE
-extern "C" __attribute__((visibility("default"))) int sigattn_trace_dump(long long* out, int* counts, int reset) {
-  cudaDeviceSynchronize();
-  cudaMemcpyFromSymbol(out, sigattn::g_trace, sizeof(long long) * 4 * 512);
-  cudaMemcpyFromSymbol(counts, sigattn::g_trace_n, sizeof(int) * 4);
-  if (reset) {
-    int z[4] = {0, 0, 0, 0};
-    cudaMemcpyToSymbol(sigattn::g_trace_n, z, sizeof(z));
-  }
-  return 0;
-}
-#endif
