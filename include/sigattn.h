@@ -156,6 +156,14 @@ SIGATTN_API int sigattn_bwd_set_timing_events(void* start_event, void* stop_even
  * (the flag is cleared), or SIGATTN_ERR_CUDA if the stream reports a CUDA error. */
 SIGATTN_API int sigattn_check(void* stream);
 
+/* Self-test of the failure path: launches one small kernel whose only thread group waits,
+ * with the same bounded wait the attention kernels use but a limit of `limit_us`
+ * microseconds (1 .. 100000), on a barrier that nothing ever signals.  The wait gives up,
+ * the kernel ends normally and records the event, so the next sigattn_check(stream) must
+ * return SIGATTN_ERR_DEVICE_TIMEOUT while the context stays usable.  Returns 0 if the
+ * kernel was enqueued.  No counterpart in the paper. */
+SIGATTN_API int sigattn_selftest_bounded_wait(int limit_us, void* stream);
+
 /* Text for an error code (static storage, never NULL). */
 SIGATTN_API const char* sigattn_strerror(int code);
 

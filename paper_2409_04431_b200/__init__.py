@@ -24,6 +24,7 @@ _BINDING_NAMES = (
     "sigattn_bwd_set_timing_events",
     "sigattn_bwd_static_scratch",
     "sigattn_bwd_static_scratch_max_elements",
+    "sigattn_selftest_bounded_wait",
 )
 
 __all__ = list(_BINDING_NAMES)

@@ -46,6 +46,8 @@ _lib.sigattn_bwd_static_scratch.argtypes = [_c.c_void_p] * 7 + [_c.c_int] * 4 + 
                                                                                    _c.c_void_p, _c.c_int, _c.c_void_p]
 _lib.sigattn_bwd_static_scratch_max_elements.restype = _c.c_size_t
 _lib.sigattn_bwd_static_scratch_max_elements.argtypes = []
+_lib.sigattn_selftest_bounded_wait.restype = _c.c_int
+_lib.sigattn_selftest_bounded_wait.argtypes = [_c.c_int, _c.c_void_p]
 _lib.sigattn_check.restype = _c.c_int
 _lib.sigattn_check.argtypes = [_c.c_void_p]
 _lib.sigattn_strerror.restype = _c.c_char_p
@@ -62,6 +64,7 @@ EXPORTED = [
     "sigattn_strerror", "sigattn_last_cuda_error", "sigattn_version", "sigattn_launch_count",
     "sigattn_step_host", "sigattn_step_host_arena_bytes", "sigattn_bwd_set_timing_events",
     "sigattn_bwd_static_scratch", "sigattn_bwd_static_scratch_max_elements",
+    "sigattn_selftest_bounded_wait",
 ]
 
 
@@ -252,3 +255,11 @@ def sigattn_bwd_static_scratch(q, k, v, d_o, scale, bias, causal=False, alibi_sl
     if rc != 0:
         raise SigattnError(rc)
     return dq, dk, dv
+
+
+def sigattn_selftest_bounded_wait(limit_us: int = 2000, stream=None) -> None:
+    """Enqueue the failure-path self-test: a kernel whose bounded wait must expire after
+    `limit_us` microseconds.  The following sigattn_check() raises SigattnError(-8)."""
+    rc = _lib.sigattn_selftest_bounded_wait(int(limit_us), _stream_ptr(stream))
+    if rc != 0:
+        raise SigattnError(rc)

@@ -5,6 +5,7 @@
 
 #include "../../include/sigattn.h"
 #include "sigattn_internal.h"
+#include "sm100_primitives.cuh"
 
 namespace {
 
@@ -16,6 +17,22 @@ thread_local cudaError_t t_last_cuda = cudaSuccess;
 constexpr int kMaxDevices = 64;
 int* g_status_ptr[kMaxDevices] = {nullptr};
 int g_arch_ok[kMaxDevices] = {0};  // 0 unknown, 1 sm_100, -1 other
+
+// One warp waits on a barrier that is never signalled; the bounded wait must expire, the
+// kernel must return, and the status word must say so.
+__global__ void selftest_bounded_wait_kernel(long long limit_cycles, int* status) {
+  __shared__ uint64_t bar;
+  __shared__ int cta_err;
+  if (threadIdx.x == 0) {
+    cta_err = 0;
+    sm100::mbar_init(sm100::smem_u32(&bar), 1);
+    sm100::fence_mbar_init();
+  }
+  __syncthreads();
+  const bool ok = sm100::mbar_wait_limit(sm100::smem_u32(&bar), 0, &cta_err, 1, limit_cycles);
+  __syncthreads();
+  if (threadIdx.x == 0 && (!ok || cta_err != 0)) atomicExch(status, 900 + cta_err);
+}
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -213,6 +230,22 @@ int sigattn_check(void* stream) {
     if (e != cudaSuccess) { t_last_cuda = e; return SIGATTN_ERR_CUDA; }
     return SIGATTN_ERR_DEVICE_TIMEOUT;
   }
+  return SIGATTN_OK;
+}
+
+int sigattn_selftest_bounded_wait(int limit_us, void* stream) {
+  if (limit_us < 1 || limit_us > 100000) return SIGATTN_ERR_FLAG;
+  int dev = 0;
+  int* status = nullptr;
+  if (int rc = device_setup(&dev, &status)) return rc;
+  int khz = 0;
+  cudaError_t e = cudaDeviceGetAttribute(&khz, cudaDevAttrClockRate, dev);
+  if (e != cudaSuccess) { t_last_cuda = e; return SIGATTN_ERR_CUDA; }
+  const long long limit_cycles = static_cast<long long>(limit_us) * khz / 1000;
+  selftest_bounded_wait_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(limit_cycles, status);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) { t_last_cuda = e; return SIGATTN_ERR_CUDA; }
+  g_launches.fetch_add(1);
   return SIGATTN_OK;
 }
 

@@ -64,7 +64,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // tear-down, so the kernel always terminates and frees its tensor memory.
 constexpr long long kWaitLimitCycles = 2000000000LL;  // about one second
 
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* cta_error, int where) {
+__device__ __forceinline__ bool mbar_wait_limit(uint32_t bar, uint32_t parity, volatile int* cta_error, int where,
+                                                long long limit_cycles) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   while (true) {
@@ -72,11 +73,15 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       if (mbar_try_wait(bar, parity)) return true;
     }
     if (*cta_error != 0) return false;
-    if (clock64() - t0 > kWaitLimitCycles) {
+    if (clock64() - t0 > limit_cycles) {
       *cta_error = where;
       return false;
     }
   }
+}
+
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* cta_error, int where) {
+  return mbar_wait_limit(bar, parity, cta_error, where, kWaitLimitCycles);
 }
 
 // ------------------------------------------------------------------ proxies and fences

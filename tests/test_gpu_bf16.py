@@ -184,3 +184,108 @@ def test_step_from_host_buffers():
     assert_close(got[0], oracle.sigattn_fwd(q, k, v, scale, bias, True, slopes), "O")
     for name, g, r in zip(("dQ", "dK", "dV"), got[1:], oracle.sigattn_bwd(q, k, v, d_o, scale, bias, True, slopes)):
         assert_close(g, r, name)
+
+
+# ---------------------------------------------------------------- full-size launches, sampled heads
+
+
+def _full_size_sampled(cfg_name, heads_to_check):
+    """Run the GPU on the whole configuration (the launch the benchmark times) and compare
+    the sampled (batch, head) pairs with the oracle, which computes each pair on its own."""
+    import torch
+    import paper_2409_04431_b200 as sa
+    cfg = inputs.CONFIGS[cfg_name]
+    q, k, v, d_o = inputs.make_inputs(cfg)
+    tq, tk, tv, tdo = (to_device(t, "bf16") for t in (q, k, v, d_o))
+    slopes = cfg.slopes()
+    sl = None if slopes is None else torch.from_numpy(slopes).cuda()
+    o = sa.sigattn_fwd(tq, tk, tv, cfg.scale, cfg.bias, cfg.causal, sl)
+    dq, dk, dv = sa.sigattn_bwd(tq, tk, tv, tdo, cfg.scale, cfg.bias, cfg.causal, sl)
+    sa.sigattn_check()
+    for t in (o, dq, dk, dv):
+        assert torch.isfinite(t.float()).all().item()
+    rb = 1024 if cfg.N > 4096 else None
+    for b, h in heads_to_check:
+        sel = (slice(b, b + 1), slice(h, h + 1))
+        s1 = None if slopes is None else slopes[h:h + 1]
+        ref_o = oracle.sigattn_fwd(q[sel], k[sel], v[sel], cfg.scale, cfg.bias, cfg.causal, s1, rb)
+        refs = oracle.sigattn_bwd(q[sel], k[sel], v[sel], d_o[sel], cfg.scale, cfg.bias, cfg.causal, s1, rb)
+        assert_close(to_host(o[sel]), ref_o, f"O[{b},{h}]")
+        for name, g, r in zip(("dQ", "dK", "dV"), (dq, dk, dv), refs):
+            assert_close(to_host(g[sel]), r, f"{name}[{b},{h}]")
+
+
+def test_config3_full_launch_sampled_heads():
+    _full_size_sampled("c3", [(0, 0), (3, 7), (7, 15)])
+
+
+def test_config4_full_launch_sampled_heads():
+    _full_size_sampled("c4", [(0, 0), (1, 15)])
+
+
+def test_config5_full_launch_sampled_head():
+    _full_size_sampled("c5", [(0, 31)])
+
+
+def test_non_default_stream_and_back_to_back_calls():
+    """Calls enqueue on the caller's stream without synchronising; results of interleaved
+    calls on one stream are those of the calls run one by one."""
+    import torch
+    import paper_2409_04431_b200 as sa
+    q, k, v, d_o = inputs.random_case(2, 2, 384, 128, seed=31)
+    tq, tk, tv, tdo = (to_device(t, "bf16") for t in (q, k, v, d_o))
+    ref_o = sa.sigattn_fwd(tq, tk, tv, 0.09, -5.9, True)
+    ref_g = sa.sigattn_bwd(tq, tk, tv, tdo, 0.09, -5.9, True)
+    sa.sigattn_check()
+    st = torch.cuda.Stream()
+    st.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(st):
+        outs = []
+        for _ in range(3):
+            o = sa.sigattn_fwd(tq, tk, tv, 0.09, -5.9, True)
+            g = sa.sigattn_bwd(tq, tk, tv, tdo, 0.09, -5.9, True)
+            outs.append((o, g))
+        sa.sigattn_check(st)
+    for o, g in outs:
+        assert torch.equal(o, ref_o) and torch.equal(g[1], ref_g[1]) and torch.equal(g[2], ref_g[2])
+        assert rel_fro(to_host(g[0]), to_host(ref_g[0])) < 1e-3
+
+
+def test_device_side_argument_errors():
+    """Misaligned device pointers and a short workspace are refused before any launch."""
+    import torch
+    import paper_2409_04431_b200 as sa
+    from paper_2409_04431_b200 import binding
+    lib = binding.lib()
+    t = torch.zeros(1 * 1 * 128 * 64 + 64, dtype=torch.bfloat16, device="cuda")
+    p = t.data_ptr()
+    ws = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")
+    n0 = sa.sigattn_launch_count()
+    assert lib.sigattn_fwd(p + 2, p, p, p, 1, 1, 128, 64, 0.125, 0.0, 0, None, 0, None) == -3
+    assert lib.sigattn_bwd(p, p, p, p, p, p, p, 1, 1, 128, 64, 0.125, 0.0, 0, None, 0, ws.data_ptr(), 1024, None) == -5
+    assert lib.sigattn_bwd(p, p, p, p, p, p, p, 1, 1, 128, 64, 0.125, 0.0, 0, None, 0, ws.data_ptr() + 64, 1 << 19, None) == -3
+    assert sa.sigattn_launch_count() == n0
+    sa.sigattn_check()
+
+
+def test_bounded_wait_expires_and_is_reported():
+    """Failure detection without a GPU fault: a wait on a barrier nothing signals gives up
+    after its limit, the kernel returns, sigattn_check reports -8 once, and the context is
+    still usable afterwards."""
+    import time
+    import torch
+    import paper_2409_04431_b200 as sa
+    sa.sigattn_check()
+    t0 = time.perf_counter()
+    sa.sigattn_selftest_bounded_wait(limit_us=3000)
+    with pytest.raises(sa.SigattnError) as err:
+        sa.sigattn_check()
+    elapsed = time.perf_counter() - t0
+    assert err.value.code == -8
+    assert elapsed < 2.0, "the wait must end by its limit, not by a watchdog"
+    sa.sigattn_check()  # the flag is cleared by the failing check
+    q, k, v, _ = inputs.random_case(1, 1, 130, 64, seed=1)
+    tq, tk, tv = (to_device(t, "bf16") for t in (q, k, v))
+    o = sa.sigattn_fwd(tq, tk, tv, 0.125, -4.0)
+    sa.sigattn_check()
+    assert torch.isfinite(o.float()).all().item()
