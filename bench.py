@@ -100,7 +100,7 @@ def run_reference(args, cfg):
         return
     steps = max(1, args.steps)
     warm = max(0, args.warmup)
-    per_step_budget = max(2.0, 60.0 / (steps + warm))
+    per_step_budget = 90.0 / (steps + warm)   # whole run: about 1.5 minutes plus one head per step at least
     vals, times = [], []
     base = None
     for s in range(warm + steps):

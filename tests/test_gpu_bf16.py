@@ -289,3 +289,43 @@ def test_bounded_wait_expires_and_is_reported():
     o = sa.sigattn_fwd(tq, tk, tv, 0.125, -4.0)
     sa.sigattn_check()
     assert torch.isfinite(o.float()).all().item()
+
+
+def test_long_sequence_closed_form():
+    """N = 32768 (far beyond what the oracle can do head by head in seconds): with Q = 0 every
+    unmasked weight is sigmoid(b), so O, dV, dK and dQ have closed forms (prefix / suffix sums)
+    that hold at any size.  Exercises 256 key tiles, the causal tile skipping and the dQ
+    accumulation across all of them."""
+    import torch
+    import paper_2409_04431_b200 as sa
+    B, H, N, D = 1, 2, 32768, 64
+    rng = np.random.default_rng(77)
+    k = inputs.round_to_bf16(rng.standard_normal((B, H, N, D), dtype=np.float32))
+    v = inputs.round_to_bf16(rng.standard_normal((B, H, N, D), dtype=np.float32) / 16)
+    d_o = inputs.round_to_bf16(rng.standard_normal((B, H, N, D), dtype=np.float32) / 16)
+    q = np.zeros_like(k)
+    bias, scale = -2.0, 0.125
+    sb = 1.0 / (1.0 + math.exp(-bias))
+    tq, tk, tv, tdo = (to_device(t, "bf16") for t in (q, k, v, d_o))
+    o = to_host(sa.sigattn_fwd(tq, tk, tv, scale, bias, True))
+    dq, dk, dv = (to_host(t) for t in sa.sigattn_bwd(tq, tk, tv, tdo, scale, bias, True))
+    sa.sigattn_check()
+    v64, do64, k64 = v.astype(np.float64), d_o.astype(np.float64), k.astype(np.float64)
+    # the GPU rounds P = sigmoid(b) to bf16 before the second product; use that value in the closed forms
+    sb_bf16 = float(inputs.round_to_bf16(np.array([sb], dtype=np.float32))[0])
+    ref_o = sb_bf16 * np.cumsum(v64, axis=2)
+    assert rel_fro(o, ref_o) < 3e-3 and np.all(np.isfinite(o))
+    ref_dv = sb_bf16 * np.flip(np.cumsum(np.flip(do64, axis=2), axis=2), axis=2)
+    assert rel_fro(dv, ref_dv) < 3e-3
+    assert np.max(np.abs(dk)) == 0.0          # dK = scale * dS^T Q with Q = 0
+    # dQ_i = scale * sb (1 - sb) * (sum_{j <= i} k_j v_j^T) dO_i on sampled rows
+    c = scale * sb * (1.0 - sb)
+    for h in range(H):
+        m = np.zeros((D, D))
+        rows = {5, 127, 128, 4095, 20000, N - 1}
+        for i in range(N):
+            m += np.outer(k64[0, h, i], v64[0, h, i])
+            if i in rows:
+                ref = c * (m @ do64[0, h, i])
+                err = np.linalg.norm(dq[0, h, i] - ref) / np.linalg.norm(ref)
+                assert err < 2e-2, (h, i, err)  # one row: bf16 rounding of dS and of the output, no averaging
