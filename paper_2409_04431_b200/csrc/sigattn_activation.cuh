@@ -92,19 +92,12 @@ __device__ __forceinline__ void sigmoid_exact(const float (&a)[N], float (&pr)[N
 }
 
 // a[N] (already scaled by log2 e) -> P[N]; if WITH_SLOPE also P (1 - P) in pp[N].
-// SPECULATE = true evaluates the common path before the decision is known (shortest
-// dependency chain, more live registers) and redoes the block on the exact path if needed;
-// false decides first.  EMULATE moves every kEmulateEvery-th exponential of the common path
-// to the FMA pipe.
-template <int N, bool WITH_SLOPE, bool SPECULATE, bool EMULATE>
+// The block's largest a decides between the two paths before anything else is evaluated.
+// EMULATE moves every kEmulateEvery-th exponential of the common path to the FMA pipe.
+template <int N, bool WITH_SLOPE, bool EMULATE>
 __device__ __forceinline__ void sigmoid_block(const float (&a)[N], float (&pr)[N], float* pp) {
-  if (SPECULATE) {
-    sigmoid_common<N, WITH_SLOPE, EMULATE>(a, pr, pp);
-    if (max_tree<N>(a) > kFastPathMaxA) sigmoid_exact<N, WITH_SLOPE>(a, pr, pp);
-  } else {
-    if (max_tree<N>(a) <= kFastPathMaxA) sigmoid_common<N, WITH_SLOPE, EMULATE>(a, pr, pp);
-    else sigmoid_exact<N, WITH_SLOPE>(a, pr, pp);
-  }
+  if (max_tree<N>(a) <= kFastPathMaxA) sigmoid_common<N, WITH_SLOPE, EMULATE>(a, pr, pp);
+  else sigmoid_exact<N, WITH_SLOPE>(a, pr, pp);
 }
 
 }  // namespace sigattn

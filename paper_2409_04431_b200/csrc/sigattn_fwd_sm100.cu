@@ -40,10 +40,7 @@ constexpr int kLoadWarp = 8;
 constexpr int kMmaWarp = 9;
 constexpr float kLog2e = 1.4426950408889634f;
 
-// Build-time switches of the forward activation (defaults = the measured best):
-#ifndef SIGATTN_FWD_SPECULATE
-#define SIGATTN_FWD_SPECULATE 0   // evaluate the common path before the block maximum is known
-#endif
+// Build-time switch of the forward activation (default = the measured best):
 #ifndef SIGATTN_FWD_EMULATE
 #define SIGATTN_FWD_EMULATE 1     // every 4th exponential on the FMA pipe
 #endif
@@ -282,7 +279,7 @@ __device__ __forceinline__ void sigmoid_block64(const uint32_t (&s0)[32], const 
     a[i] = fmaf(__uint_as_float(i < 32 ? s0[i & 31] : s1[i & 31]), scale_log2e, c0);
   }
   float pr[64];
-  sigmoid_block<64, false, SIGATTN_FWD_SPECULATE != 0, SIGATTN_FWD_EMULATE != 0>(a, pr, nullptr);
+  sigmoid_block<64, false, SIGATTN_FWD_EMULATE != 0>(a, pr, nullptr);
   if (causal_diag) {  // keys after the query get weight 0 (only on the diagonal tile)
 #pragma unroll
     for (int i = 0; i < 64; ++i)

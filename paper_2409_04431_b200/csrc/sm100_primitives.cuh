@@ -115,14 +115,6 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst_smem, const CUtensorMap
       : "memory");
 }
 
-// global -> L2 only: warms the cache for a tile that will be loaded later.
-__device__ __forceinline__ void tma_prefetch_l2_3d(const CUtensorMap* m, int c0, int c1, int c2) {
-  asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global [%0, {%1, %2, %3}];"
-               :
-               : "l"(reinterpret_cast<uint64_t>(m)), "r"(c0), "r"(c1), "r"(c2)
-               : "memory");
-}
-
 // shared -> global, 3-D tile (rows beyond the tensor's extent are clipped by the hardware).
 __device__ __forceinline__ void tma_store_3d(const CUtensorMap* m, uint32_t src_smem, int c0, int c1, int c2) {
   asm volatile(
@@ -227,17 +219,6 @@ __device__ __forceinline__ void named_barrier_sync() {
   asm volatile("bar.sync %0, %1;" ::"n"(ID), "n"(COUNT) : "memory");
 }
 
-// Non-blocking arrival on a named barrier that COUNT threads (arrivers + waiters) share.
-template <int COUNT>
-__device__ __forceinline__ void named_barrier_arrive(int id) {
-  asm volatile("bar.arrive %0, %1;" ::"r"(id), "n"(COUNT) : "memory");
-}
-
-template <int COUNT>
-__device__ __forceinline__ void named_barrier_sync_id(int id) {
-  asm volatile("bar.sync %0, %1;" ::"r"(id), "n"(COUNT) : "memory");
-}
-
 // ------------------------------------------------------------------ tcgen05 MMA
 
 // 64-bit shared-memory matrix descriptor (sm_100 format): start address, leading and
@@ -309,15 +290,6 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
-// fp32 add of four consecutive floats into global memory (16-byte aligned), no return value.
-__device__ __forceinline__ void red_add_v4(float* addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};"
-               :
-               : "l"(addr), "f"(__uint_as_float(a)), "f"(__uint_as_float(b)), "f"(__uint_as_float(c)),
-                 "f"(__uint_as_float(d))
-               : "memory");
-}
-
 // ------------------------------------------------------------------ arithmetic helpers
 
 __device__ __forceinline__ float ex2_approx(float x) {
@@ -329,12 +301,6 @@ __device__ __forceinline__ float ex2_approx(float x) {
 __device__ __forceinline__ float rcp_approx(float x) {
   float y;
   asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-
-__device__ __forceinline__ float tanh_approx(float x) {
-  float y;
-  asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
 
