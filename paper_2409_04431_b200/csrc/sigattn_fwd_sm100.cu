@@ -4,17 +4,20 @@
 // One persistent CTA per SM walks a list of work items (batch*head, pair of 128-row query
 // tiles), heaviest first when causal.  Inside a CTA the work is split by warp role:
 //
-//   warp 8      TMA producer: Q tiles once per item, then K_0, V_0, K_1, V_1, ... through a
+//   warp 16     TMA producer: Q tiles once per item, then K_0, V_0, K_1, V_1, ... through a
 //               ring of shared-memory stages (128-byte swizzle, zero fill beyond row N).
-//   warp 9      MMA issuer (one thread): S_t = Q_t K_j^T into tensor memory, then
+//   warp 17     MMA issuer (one thread): S_t = Q_t K_j^T into tensor memory, then
 //               O_t += P_t V_j with P read from tensor memory.  The two query tiles are
 //               interleaved so the tensor pipe works on one while the other is activated.
-//   warps 0-7   activation: threads read S from tensor memory (one row each), evaluate
-//               P = sigmoid(.) in registers and write bf16 P back over S.  All 256 threads
-//               work on one query tile (64 key columns each) and alternate between the two
-//               tiles, so the MUFU pipe and the tensor pipe take turns on a tile.  At the end
-//               of an item they convert the O accumulators to bf16 and store them with TMA
-//               (rows >= N are clipped).
+//   warps 0-15  activation: threads read S from tensor memory (one row each), evaluate
+//               P = sigmoid(.) in registers and write bf16 P back over S.  All 512 threads
+//               work on one query tile (32 key columns each) and alternate between the two
+//               tiles, so the MUFU pipe and the tensor pipe take turns on a tile.  Sixteen
+//               warps rather than eight: the activation is bound by the latency of its
+//               dependent chain (tensor-memory load, exponential, polynomial, store), and
+//               four warps per scheduler hide it better than two (measured +3 % at D = 128,
+//               +15 % at D = 64).  At the end of an item they convert the O accumulators to
+//               bf16 and store them with TMA (rows >= N are clipped).
 //
 // Sigmoid needs no row maximum, no row sum and no rescaling of O (Section 4), so there is
 // no correction step and O is touched once, at the end.
@@ -35,9 +38,16 @@ using namespace sm100;
 
 constexpr int kBM = 128;        // query rows per tile (= TMEM lanes)
 constexpr int kBN = 128;        // keys per tile
-constexpr int kFwdThreads = 320;
-constexpr int kLoadWarp = 8;
-constexpr int kMmaWarp = 9;
+#ifndef SIGATTN_FWD_ACT_WARPS
+#define SIGATTN_FWD_ACT_WARPS 16
+#endif
+constexpr int kActWarps = SIGATTN_FWD_ACT_WARPS;   // 8 or 16
+constexpr int kActThreads = 32 * kActWarps;
+constexpr int kGroups = kActWarps / 4;             // column groups of a tile
+constexpr int kCols = kBN / kGroups;               // key columns per activation thread
+constexpr int kFwdThreads = kActThreads + 64;
+constexpr int kLoadWarp = kActWarps;
+constexpr int kMmaWarp = kActWarps + 1;
 constexpr float kLog2e = 1.4426950408889634f;
 
 // Build-time switch of the forward activation (default = the measured best):
@@ -185,8 +195,9 @@ __device__ void fwd_mma_role(const FwdParams& p, uint32_t smem_base, uint32_t tm
     const uint64_t vd = make_smem_desc_sw128(v_smem, L::kPanelBytes, 1024);
 #pragma unroll
     for (int ks = 0; ks < kBN / 16; ++ks) {
-      // bf16 P sits at columns [0, 32) (group 0) and [64, 96) (group 1) of S_t
-      const uint32_t p_col = (ks >> 2) * 64 + (ks & 3) * 8;
+      // column group c wrote its bf16 P over the first half of its own logits columns:
+      // [c kCols, c kCols + kCols / 2), one k-step of 16 keys per 8 columns
+      const uint32_t p_col = (ks / (kCols / 16)) * kCols + (ks % (kCols / 16)) * 8;
       umma_ts(tmem + 2 * kBN + t * D, tmem + t * kBN + p_col, desc_advance(vd, ks * 2048), kIdescPV,
               (accumulate || ks > 0));
     }
@@ -262,43 +273,59 @@ __device__ void fwd_mma_role(const FwdParams& p, uint32_t smem_base, uint32_t tm
 
 // ------------------------------------------------------------------ activation + epilogue
 
-// 64 logits of one row (two 32-column TMEM loads) -> 32 packed bf16x2 sigmoid values.
+template <int N>
+__device__ __forceinline__ void tmem_ld_cols(uint32_t addr, uint32_t (&v)[N]) {
+  static_assert(N == 16 || N == 32 || N == 64, "columns per thread");
+  if constexpr (N == 16) {
+    tmem_ld16(addr, v);
+  } else {
+#pragma unroll
+    for (int c = 0; c < N / 32; ++c) tmem_ld32(addr + c * 32, *reinterpret_cast<uint32_t (*)[32]>(&v[c * 32]));
+  }
+}
+template <int N>
+__device__ __forceinline__ void tmem_st_cols(uint32_t addr, uint32_t (&v)[N]) {
+  static_assert(N == 16 || N == 32, "packed columns per thread");
+  if constexpr (N == 16) tmem_st16(addr, v); else tmem_st32(addr, v);
+}
+
+// kCols logits of one row (32-column TMEM loads) -> kCols / 2 packed bf16x2 sigmoid values.
 //   a = s * scale_log2e + c0   (c0 carries the bias and, with ALiBi, the position term)
 template <bool ALIBI>
-__device__ __forceinline__ void sigmoid_block64(const uint32_t (&s0)[32], const uint32_t (&s1)[32],
-                                                uint32_t (&out)[32], float scale_log2e, float bias_log2e,
-                                                float slope_log2e, float row_rel, int col_base, bool causal_diag) {
-  float a[64];
+__device__ __forceinline__ void sigmoid_cols(const uint32_t (&s)[kCols], uint32_t (&out)[kCols / 2],
+                                             float scale_log2e, float bias_log2e, float slope_log2e, float row_rel,
+                                             int col_base, bool causal_diag) {
+  float a[kCols];
 #pragma unroll
-  for (int i = 0; i < 64; ++i) {
+  for (int i = 0; i < kCols; ++i) {
     float c0 = bias_log2e;
     if (ALIBI) {
       const float dist = row_rel - static_cast<float>(col_base + i);
       c0 = fmaf(-slope_log2e, fabsf(dist), bias_log2e);
     }
-    a[i] = fmaf(__uint_as_float(i < 32 ? s0[i & 31] : s1[i & 31]), scale_log2e, c0);
+    a[i] = fmaf(__uint_as_float(s[i]), scale_log2e, c0);
   }
-  float pr[64];
-  sigmoid_block<64, false, SIGATTN_FWD_EMULATE != 0>(a, pr, nullptr);
+  float pr[kCols];
+  sigmoid_block<kCols, false, SIGATTN_FWD_EMULATE != 0>(a, pr, nullptr);
   if (causal_diag) {  // keys after the query get weight 0 (only on the diagonal tile)
 #pragma unroll
-    for (int i = 0; i < 64; ++i)
+    for (int i = 0; i < kCols; ++i)
       if (static_cast<float>(col_base + i) > row_rel) pr[i] = 0.0f;
   }
 #pragma unroll
-  for (int i = 0; i < 32; ++i) out[i] = pack_bf16x2(pr[2 * i], pr[2 * i + 1]);
+  for (int i = 0; i < kCols / 2; ++i) out[i] = pack_bf16x2(pr[2 * i], pr[2 * i + 1]);
 }
 
-// Both activation groups (256 threads) work on the same query tile at a time, alternating
-// between the two tiles of the item: thread (g, r) owns row r and key columns
-// [64 g, 64 g + 64) of the tile.  While the groups evaluate one tile, the tensor pipe runs
+// All activation threads work on the same query tile at a time, alternating between the
+// two tiles of the item: thread (g, r) owns row r and key columns [kCols g, kCols g + kCols)
+// of the tile.  While the groups evaluate one tile, the tensor pipe runs
 // P V and the next logits of the other one, so the MUFU pipe and the tensor pipe take turns
 // on a tile instead of competing for it.
 template <int D, bool CAUSAL, bool ALIBI>
 __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t* smem, uint32_t tmem,
                              FwdBarriers* bars, volatile int* cta_err) {
   using L = FwdSmem<D>;
-  const int g = (threadIdx.x >> 7) & 1;      // column half of the tile
+  const int g = threadIdx.x >> 7;            // column group of the tile
   const int tid = threadIdx.x & 127;         // row of the tile
   const uint32_t lane_off = static_cast<uint32_t>(((threadIdx.x >> 5) & 3) * 32) << 16;
   uint32_t s_cnt0 = 0, s_cnt1 = 0, it[2] = {0, 0};
@@ -321,15 +348,14 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
         tc_fence_after_sync();
         const float row_rel = static_cast<float>(w.row0 + t * kBM + tid - j * kBN);
         const bool diag = CAUSAL && (j == w.n[t] - 1);
-        // bf16 P goes back over the first half of the 64 columns this thread has just read
-        const uint32_t tS = tmem + t * kBN + lane_off + g * 64;
-        uint32_t s0[32], s1[32];
-        tmem_ld32(tS, s0);
-        tmem_ld32(tS + 32, s1);
+        // bf16 P goes back over the first half of the columns this thread has just read
+        const uint32_t tS = tmem + t * kBN + lane_off + g * kCols;
+        uint32_t sv[kCols];
+        tmem_ld_cols(tS, sv);
         tmem_wait_ld();
-        uint32_t pk[32];
-        sigmoid_block64<ALIBI>(s0, s1, pk, p.scale_log2e, p.bias_log2e, slope_log2e, row_rel, g * 64, diag);
-        tmem_st32(tS, pk);
+        uint32_t pk[kCols / 2];
+        sigmoid_cols<ALIBI>(sv, pk, p.scale_log2e, p.bias_log2e, slope_log2e, row_rel, g * kCols, diag);
+        tmem_st_cols(tS, pk);
         tmem_wait_st();
         tc_fence_before_sync();
         mbar_arrive(smem_u32(&bars->p_full[t]));
@@ -337,8 +363,8 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
     }
 
     // epilogue: O_t (fp32, tensor memory) -> bf16 -> swizzled shared memory (the Q_t buffer,
-    // free once every logits MMA of the item is done) -> TMA store.  Each group converts
-    // half of the D columns.
+    // free once every logits MMA of the item is done) -> TMA store.  Each column group
+    // converts its share of the D columns.
 #pragma unroll
     for (int t = 0; t < 2; ++t) {
       if (w.n[t] == 0) continue;
@@ -346,29 +372,29 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
       ++it[t];
       tc_fence_after_sync();
       uint8_t* stage = smem + L::kQOff + t * L::kTileBytes;
-      const uint32_t tO = tmem + 2 * kBN + t * D + lane_off + g * (D / 2);
+      constexpr int kECols = D / kGroups;   // accumulator columns per thread
+      const uint32_t tO = tmem + 2 * kBN + t * D + lane_off + g * kECols;
+      uint32_t o[kECols];
+      tmem_ld_cols(tO, o);
+      tmem_wait_ld();
+      {
+        const int col = g * kECols;           // first of this thread's columns
+        uint8_t* row_ptr = stage + (col >> 6) * L::kPanelBytes + tid * 128;
 #pragma unroll
-      for (int c = 0; c < D / 64; ++c) {
-        uint32_t o[32];
-        tmem_ld32(tO + c * 32, o);
-        tmem_wait_ld();
-        // D = 128: group g fills panel g (8 chunks of 16 B); D = 64: half of the only panel
-        uint8_t* row_ptr = stage + (D == 128 ? g * L::kPanelBytes : 0) + tid * 128;
-#pragma unroll
-        for (int q4 = 0; q4 < 4; ++q4) {
+        for (int q4 = 0; q4 < kECols / 8; ++q4) {
           uint4 val;
           val.x = pack_bf16x2(__uint_as_float(o[8 * q4 + 0]), __uint_as_float(o[8 * q4 + 1]));
           val.y = pack_bf16x2(__uint_as_float(o[8 * q4 + 2]), __uint_as_float(o[8 * q4 + 3]));
           val.z = pack_bf16x2(__uint_as_float(o[8 * q4 + 4]), __uint_as_float(o[8 * q4 + 5]));
           val.w = pack_bf16x2(__uint_as_float(o[8 * q4 + 6]), __uint_as_float(o[8 * q4 + 7]));
-          const int chunk = (D == 128 ? c * 4 : g * 4) + q4;
+          const int chunk = ((col & 63) >> 3) + q4;
           *reinterpret_cast<uint4*>(row_ptr + ((chunk ^ (tid & 7)) * 16)) = val;
         }
       }
       tc_fence_before_sync();
       mbar_arrive(smem_u32(&bars->o_empty[t]));
       fence_proxy_async_smem();
-      named_barrier_sync<1, 256>();
+      named_barrier_sync<1, kActThreads>();
       if (threadIdx.x == 0) {
 #pragma unroll
         for (int pn = 0; pn < L::kPanels; ++pn)
@@ -405,9 +431,9 @@ sigattn_fwd_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
       mbar_init(smem_u32(&bars.q_full[t]), 1);
       mbar_init(smem_u32(&bars.q_empty[t]), 1);
       mbar_init(smem_u32(&bars.s_full[t]), 1);
-      mbar_init(smem_u32(&bars.p_full[t]), 256);
+      mbar_init(smem_u32(&bars.p_full[t]), kActThreads);
       mbar_init(smem_u32(&bars.o_full[t]), 1);
-      mbar_init(smem_u32(&bars.o_empty[t]), 256);
+      mbar_init(smem_u32(&bars.o_empty[t]), kActThreads);
     }
     for (int s = 0; s < L::kStages; ++s) {
       mbar_init(smem_u32(&bars.kv_full[s]), 1);
