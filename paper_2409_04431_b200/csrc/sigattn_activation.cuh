@@ -5,8 +5,8 @@
 //
 //   common path  P = u - u^2 + u^3, the alternating series of u / (1 + u) (relative error
 //                u^3 <= 2^-12 for a <= -4, below bf16 resolution), and P (1 - P) = P - P^2;
-//                one exponential per element, a fixed share of them evaluated on the FMA
-//                pipe (ex2_emulated) instead of the MUFU pipe.
+//                one exponential per element; where the MUFU pipe is the bound (forward at
+//                D = 64) a fixed share of them is evaluated on the FMA pipe (ex2_emulated).
 //   exact path   e = 2^-a,  r = 1 / (1 + e),  P = r,  P (1 - P) = r e r  (two MUFU ops),
 //                taken if any logit of the block has a > -4.  At b = -log n almost no block
 //                needs it.
@@ -64,15 +64,15 @@ __device__ __forceinline__ float ex2_emulated(float a) {
   return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
 }
 
-constexpr int kEmulateEvery = 4;  // every 4th exponential of the common path is emulated
-
 // Common path: u / (1 + u) = u - u^2 + u^3 - ..., cut after u^3 and evaluated as
 // u - u (u - u^2): two FMAs; relative error u^3 <= 2^-12 for a <= -4.
-template <int N, bool WITH_SLOPE, bool EMULATE>
+// EMULATE_EVERY = m > 0 evaluates every m-th exponential on the FMA pipe, 0 none.
+template <int N, bool WITH_SLOPE, int EMULATE_EVERY>
 __device__ __forceinline__ void sigmoid_common(const float (&a)[N], float (&pr)[N], float* pp) {
 #pragma unroll
   for (int i = 0; i < N; ++i) {
-    const float u = (EMULATE && i % kEmulateEvery == kEmulateEvery - 1) ? ex2_emulated(a[i]) : sm100::ex2_approx(a[i]);
+    const bool emulate = EMULATE_EVERY > 0 && i % (EMULATE_EVERY > 0 ? EMULATE_EVERY : 1) == EMULATE_EVERY - 1;
+    const float u = emulate ? ex2_emulated(a[i]) : sm100::ex2_approx(a[i]);
     const float w = fmaf(-u, u, u);
     pr[i] = fmaf(-u, w, u);
     if (WITH_SLOPE) pp[i] = fmaf(-pr[i], pr[i], pr[i]);  // P <= 1/17 here: no cancellation in P - P^2
@@ -93,10 +93,9 @@ __device__ __forceinline__ void sigmoid_exact(const float (&a)[N], float (&pr)[N
 
 // a[N] (already scaled by log2 e) -> P[N]; if WITH_SLOPE also P (1 - P) in pp[N].
 // The block's largest a decides between the two paths before anything else is evaluated.
-// EMULATE moves every kEmulateEvery-th exponential of the common path to the FMA pipe.
-template <int N, bool WITH_SLOPE, bool EMULATE>
+template <int N, bool WITH_SLOPE, int EMULATE_EVERY>
 __device__ __forceinline__ void sigmoid_block(const float (&a)[N], float (&pr)[N], float* pp) {
-  if (max_tree<N>(a) <= kFastPathMaxA) sigmoid_common<N, WITH_SLOPE, EMULATE>(a, pr, pp);
+  if (max_tree<N>(a) <= kFastPathMaxA) sigmoid_common<N, WITH_SLOPE, EMULATE_EVERY>(a, pr, pp);
   else sigmoid_exact<N, WITH_SLOPE>(a, pr, pp);
 }
 

@@ -282,7 +282,7 @@ __device__ __forceinline__ void bwd_sigmoid_chunk(const uint32_t (&s)[32], uint3
     a[e] = fmaf(__uint_as_float(s[e]), scale_log2e, c0);
   }
   float pr[32];
-  sigmoid_block<32, true, false>(a, pr, pp);
+  sigmoid_block<32, true, 0>(a, pr, pp);
   if (DIAG) {
 #pragma unroll
     for (int e = 0; e < 32; ++e)

@@ -50,9 +50,15 @@ constexpr int kLoadWarp = kActWarps;
 constexpr int kMmaWarp = kActWarps + 1;
 constexpr float kLog2e = 1.4426950408889634f;
 
-// Build-time switch of the forward activation (default = the measured best):
-#ifndef SIGATTN_FWD_EMULATE
-#define SIGATTN_FWD_EMULATE 1     // every 4th exponential on the FMA pipe
+// Share of the forward's exponentials evaluated on the FMA pipe (every m-th, 0 = none).
+// At D = 128 the shorter instruction stream wins (emulating every 4th measured -6 %); at
+// D = 64, where a tile step has half the tensor work per exponential, unloading the MUFU
+// pipe gains 1-2 %.
+#ifndef SIGATTN_FWD_EMULATE_D64
+#define SIGATTN_FWD_EMULATE_D64 8
+#endif
+#ifndef SIGATTN_FWD_EMULATE_D128
+#define SIGATTN_FWD_EMULATE_D128 0
 #endif
 
 
@@ -291,7 +297,7 @@ __device__ __forceinline__ void tmem_st_cols(uint32_t addr, uint32_t (&v)[N]) {
 
 // kCols logits of one row (32-column TMEM loads) -> kCols / 2 packed bf16x2 sigmoid values.
 //   a = s * scale_log2e + c0   (c0 carries the bias and, with ALiBi, the position term)
-template <bool ALIBI>
+template <bool ALIBI, int EMULATE_EVERY>
 __device__ __forceinline__ void sigmoid_cols(const uint32_t (&s)[kCols], uint32_t (&out)[kCols / 2],
                                              float scale_log2e, float bias_log2e, float slope_log2e, float row_rel,
                                              int col_base, bool causal_diag) {
@@ -306,7 +312,7 @@ __device__ __forceinline__ void sigmoid_cols(const uint32_t (&s)[kCols], uint32_
     a[i] = fmaf(__uint_as_float(s[i]), scale_log2e, c0);
   }
   float pr[kCols];
-  sigmoid_block<kCols, false, SIGATTN_FWD_EMULATE != 0>(a, pr, nullptr);
+  sigmoid_block<kCols, false, EMULATE_EVERY>(a, pr, nullptr);
   if (causal_diag) {  // keys after the query get weight 0 (only on the diagonal tile)
 #pragma unroll
     for (int i = 0; i < kCols; ++i)
@@ -354,7 +360,9 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
         tmem_ld_cols(tS, sv);
         tmem_wait_ld();
         uint32_t pk[kCols / 2];
-        sigmoid_cols<ALIBI>(sv, pk, p.scale_log2e, p.bias_log2e, slope_log2e, row_rel, g * kCols, diag);
+        constexpr int kEmulateEvery = (D == 128) ? SIGATTN_FWD_EMULATE_D128 : SIGATTN_FWD_EMULATE_D64;
+        sigmoid_cols<ALIBI, kEmulateEvery>(sv, pk, p.scale_log2e, p.bias_log2e, slope_log2e, row_rel, g * kCols,
+                                           diag);
         tmem_st_cols(tS, pk);
         tmem_wait_st();
         tc_fence_before_sync();
