@@ -128,8 +128,12 @@ SIGATTN_API size_t sigattn_bwd_workspace_bytes(int B, int H, int N, int D, int d
 
 /* One forward + backward pass from HOST buffers (pinned memory recommended): copies
  * q, k, v, d_o (and the H slopes, if any) to the device, runs sigattn_fwd and
- * sigattn_bwd, and copies o, dq, dk, dv back, all enqueued on `stream` in that order;
- * returns without synchronising.  Every tensor pointer and `alibi_slopes_host` are HOST
+ * sigattn_bwd, and copies o, dq, dk, dv back; returns without synchronising.  The work is
+ * ordered after everything enqueued on `stream` before the call, and whatever is enqueued
+ * on `stream` afterwards is ordered after it.  In between, the problem is cut into chunks
+ * of whole heads whose copies in, kernels and copies out run on three streams owned by the
+ * library (created on the first call on a device), so that both directions of the host
+ * link and the kernels overlap; that overlap needs pinned host buffers.  Every tensor pointer and `alibi_slopes_host` are HOST
  * pointers; `device_arena` is DEVICE scratch of at least
  * sigattn_step_host_arena_bytes(...) bytes, 256-byte aligned, owned by the caller (it
  * holds the eight tensors, the slopes and the backward workspace).  The host buffers must

@@ -1,6 +1,7 @@
 // C-ABI layer of libsigattn.so: argument validation, dispatch by dtype, device-side
 // status word, error strings.  See include/sigattn.h for the contract.
 #include <atomic>
+#include <mutex>
 #include <stdint.h>
 
 #include "../../include/sigattn.h"
@@ -157,6 +158,62 @@ int sigattn_bwd_set_timing_events(void* start_event, void* stop_event) {
 
 namespace {
 size_t align256(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
+
+// sigattn_step_host splits the problem into chunks of whole heads and runs copy-in, kernels
+// and copy-out of different chunks on three streams of its own, so that the two directions
+// of the host link and the kernels overlap.  Streams and events are created once per device.
+constexpr int kHostStepEvents = 64;   // events per kind; head chunking never forms more chunks than this
+struct HostStepPipeline {
+  cudaStream_t in = nullptr, compute = nullptr, out = nullptr;
+  cudaEvent_t start = nullptr, done = nullptr;
+  cudaEvent_t in_done[kHostStepEvents] = {}, computed[kHostStepEvents] = {};
+  bool ready = false;
+};
+HostStepPipeline g_host_step[kMaxDevices];
+std::mutex g_host_step_mutex;
+
+int host_step_pipeline(int dev, HostStepPipeline** out) {
+  std::lock_guard<std::mutex> lock(g_host_step_mutex);
+  HostStepPipeline& p = g_host_step[dev];
+  if (!p.ready) {
+    cudaError_t e = cudaSuccess;
+    auto stream = [&](cudaStream_t* s) { if (e == cudaSuccess) e = cudaStreamCreateWithFlags(s, cudaStreamNonBlocking); };
+    auto event = [&](cudaEvent_t* ev) { if (e == cudaSuccess) e = cudaEventCreateWithFlags(ev, cudaEventDisableTiming); };
+    stream(&p.in); stream(&p.compute); stream(&p.out);
+    event(&p.start); event(&p.done);
+    for (int i = 0; i < kHostStepEvents; ++i) { event(&p.in_done[i]); event(&p.computed[i]); }
+    if (e != cudaSuccess) { t_last_cuda = e; return SIGATTN_ERR_CUDA; }
+    p.ready = true;
+  }
+  *out = &p;
+  return SIGATTN_OK;
+}
+
+// A chunk is either a group of whole batch entries or, within one batch entry, a group of
+// heads whose size divides H (so a chunk never straddles two batch entries and the ALiBi slope
+// of a head is found at a fixed offset).  About eight chunks are formed, none below 1 MiB per
+// tensor unless the whole problem is.
+struct HostStepChunking {
+  int batches;   // batch entries per chunk (>= 1); heads == H if > 1
+  int heads;     // heads per chunk
+};
+HostStepChunking host_step_chunking(int B, int H, size_t head_bytes) {
+  const size_t min_bytes = 1u << 20;
+  if (B >= 2 && static_cast<size_t>(H) * head_bytes * B >= 2 * min_bytes && (B >= 8 || H * head_bytes < 8 * min_bytes)) {
+    int nb = (B + 7) / 8;
+    while (static_cast<size_t>(nb) * H * head_bytes < min_bytes && nb < B) ++nb;
+    return {nb, H};
+  }
+  int best = H;
+  for (int d = H; d >= 1; --d) {
+    if (H % d != 0) continue;
+    if (d * head_bytes < min_bytes && d != H) break;
+    if (static_cast<long long>(B) * (H / d) > kHostStepEvents) break;
+    best = d;
+    if (static_cast<long long>(B) * (H / d) >= 8) break;
+  }
+  return {1, best};
+}
 }
 
 size_t sigattn_step_host_arena_bytes(int B, int H, int N, int D, int dtype) {
@@ -178,35 +235,75 @@ int sigattn_step_host(const void* q_host, const void* k_host, const void* v_host
   if (causal != 0 && causal != 1) return SIGATTN_ERR_FLAG;
   if (reinterpret_cast<uintptr_t>(device_arena) & 255u) return SIGATTN_ERR_ALIGN;
   if (arena_bytes < sigattn_step_host_arena_bytes(B, H, N, D, dtype)) return SIGATTN_ERR_WORKSPACE;
-  const size_t bytes = static_cast<size_t>(B) * H * N * D * (dtype == SIGATTN_DTYPE_BF16 ? 2 : 4);
-  const size_t tensor = align256(bytes);
+  int dev = 0;
+  int* status = nullptr;
+  if (int rc = device_setup(&dev, &status)) return rc;
+  HostStepPipeline* pipe = nullptr;
+  if (int rc = host_step_pipeline(dev, &pipe)) return rc;
+
+  const size_t elem = (dtype == SIGATTN_DTYPE_BF16) ? 2 : 4;
+  const size_t head_bytes = static_cast<size_t>(N) * D * elem;   // one (batch, head) slab of a tensor
+  const size_t tensor = align256(static_cast<size_t>(B) * H * head_bytes);
   char* base = static_cast<char*>(device_arena);
-  void* d[8];
-  for (int i = 0; i < 8; ++i) d[i] = base + i * tensor;
   float* d_slopes = reinterpret_cast<float*>(base + 8 * tensor);
-  void* d_ws = base + 8 * tensor + align256(static_cast<size_t>(H) * sizeof(float));
-  const size_t ws_bytes = sigattn_bwd_workspace_bytes(B, H, N, D, dtype);
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  char* d_ws = base + 8 * tensor + align256(static_cast<size_t>(H) * sizeof(float));
+  const HostStepChunking ck = host_step_chunking(B, H, head_bytes);
+  const int chunks_per_batch = H / ck.heads;                       // 1 if chunks are whole batch entries
+  const int n_chunks = (ck.batches > 1 || ck.heads == H) ? (B + ck.batches - 1) / ck.batches : B * chunks_per_batch;
+  cudaStream_t caller = static_cast<cudaStream_t>(stream);
   const void* in_host[4] = {q_host, k_host, v_host, d_o_host};
-  for (int i = 0; i < 4; ++i) {
-    cudaError_t e = cudaMemcpyAsync(d[i], in_host[i], bytes, cudaMemcpyHostToDevice, st);
-    if (e != cudaSuccess) { t_last_cuda = e; return SIGATTN_ERR_CUDA; }
-  }
-  if (alibi_slopes_host) {
-    cudaError_t e = cudaMemcpyAsync(d_slopes, alibi_slopes_host, static_cast<size_t>(H) * sizeof(float),
-                                    cudaMemcpyHostToDevice, st);
-    if (e != cudaSuccess) { t_last_cuda = e; return SIGATTN_ERR_CUDA; }
-  }
-  const float* slopes = alibi_slopes_host ? d_slopes : nullptr;
-  if (int rc = sigattn_fwd(d[0], d[1], d[2], d[4], B, H, N, D, scale, bias, causal, slopes, dtype, stream)) return rc;
-  if (int rc = sigattn_bwd(d[0], d[1], d[2], d[3], d[5], d[6], d[7], B, H, N, D, scale, bias, causal, slopes, dtype,
-                           ws_bytes ? d_ws : nullptr, ws_bytes, stream))
-    return rc;
   void* out_host[4] = {o_host, dq_host, dk_host, dv_host};
-  for (int i = 0; i < 4; ++i) {
-    cudaError_t e = cudaMemcpyAsync(out_host[i], d[4 + i], bytes, cudaMemcpyDeviceToHost, st);
-    if (e != cudaSuccess) { t_last_cuda = e; return SIGATTN_ERR_CUDA; }
+  auto fail = [](cudaError_t e) { t_last_cuda = e; return SIGATTN_ERR_CUDA; };
+  cudaError_t e;
+
+  // The three internal streams start after everything already enqueued on the caller's stream.
+  if ((e = cudaEventRecord(pipe->start, caller)) != cudaSuccess) return fail(e);
+  if ((e = cudaStreamWaitEvent(pipe->in, pipe->start, 0)) != cudaSuccess) return fail(e);
+  if ((e = cudaStreamWaitEvent(pipe->compute, pipe->start, 0)) != cudaSuccess) return fail(e);
+  if ((e = cudaStreamWaitEvent(pipe->out, pipe->start, 0)) != cudaSuccess) return fail(e);
+  if (alibi_slopes_host) {
+    e = cudaMemcpyAsync(d_slopes, alibi_slopes_host, static_cast<size_t>(H) * sizeof(float), cudaMemcpyHostToDevice,
+                        pipe->in);
+    if (e != cudaSuccess) return fail(e);
   }
+  for (int c = 0; c < n_chunks; ++c) {
+    // chunk c covers `cb` batch entries x `ck.heads` heads starting at (b0, h0)
+    const bool whole = (ck.heads == H);
+    const int b0 = whole ? c * ck.batches : c / chunks_per_batch;
+    const int cb = whole ? (B - b0 < ck.batches ? B - b0 : ck.batches) : 1;
+    const int h0 = whole ? 0 : (c % chunks_per_batch) * ck.heads;
+    const size_t off = (static_cast<size_t>(b0) * H + h0) * head_bytes;
+    const size_t chunk_bytes = static_cast<size_t>(cb) * ck.heads * head_bytes;
+    const size_t chunk_ws = sigattn_bwd_workspace_bytes(cb, ck.heads, N, D, dtype);
+    const size_t ws_off = (dtype == SIGATTN_DTYPE_BF16) ? off / elem * sizeof(float) : 0;   // fp32 accumulator slab
+    for (int i = 0; i < 4; ++i) {
+      e = cudaMemcpyAsync(base + i * tensor + off, static_cast<const char*>(in_host[i]) + off, chunk_bytes,
+                          cudaMemcpyHostToDevice, pipe->in);
+      if (e != cudaSuccess) return fail(e);
+    }
+    cudaEvent_t in_done = pipe->in_done[c % kHostStepEvents], computed = pipe->computed[c % kHostStepEvents];
+    if ((e = cudaEventRecord(in_done, pipe->in)) != cudaSuccess) return fail(e);
+    if ((e = cudaStreamWaitEvent(pipe->compute, in_done, 0)) != cudaSuccess) return fail(e);
+    const float* slopes = alibi_slopes_host ? d_slopes + h0 : nullptr;
+    void* d[8];
+    for (int i = 0; i < 8; ++i) d[i] = base + i * tensor + off;
+    if (int rc = sigattn_fwd(d[0], d[1], d[2], d[4], cb, ck.heads, N, D, scale, bias, causal, slopes, dtype,
+                             pipe->compute))
+      return rc;
+    if (int rc = sigattn_bwd(d[0], d[1], d[2], d[3], d[5], d[6], d[7], cb, ck.heads, N, D, scale, bias, causal, slopes,
+                             dtype, chunk_ws ? d_ws + ws_off : nullptr, chunk_ws, pipe->compute))
+      return rc;
+    if ((e = cudaEventRecord(computed, pipe->compute)) != cudaSuccess) return fail(e);
+    if ((e = cudaStreamWaitEvent(pipe->out, computed, 0)) != cudaSuccess) return fail(e);
+    for (int i = 0; i < 4; ++i) {
+      e = cudaMemcpyAsync(static_cast<char*>(out_host[i]) + off, base + (4 + i) * tensor + off, chunk_bytes,
+                          cudaMemcpyDeviceToHost, pipe->out);
+      if (e != cudaSuccess) return fail(e);
+    }
+  }
+  // The last copies out follow the last kernels, which follow the last copies in.
+  if ((e = cudaEventRecord(pipe->done, pipe->out)) != cudaSuccess) return fail(e);
+  if ((e = cudaStreamWaitEvent(caller, pipe->done, 0)) != cudaSuccess) return fail(e);
   return SIGATTN_OK;
 }
 

@@ -167,23 +167,51 @@ def test_library_counts_its_launches():
     assert sa.sigattn_launch_count() - n0 == 3  # forward; backward main + dQ convert
 
 
-def test_step_from_host_buffers():
-    """sigattn_step_host: H2D copies, forward, backward, D2H copies in one call."""
+@pytest.mark.parametrize("B,H,N,D", [(2, 4, 333, 64),      # two chunks of one batch entry each
+                                      (1, 8, 1024, 128),    # two chunks of four heads: slopes at an offset
+                                      (3, 2, 64, 64)])      # small: per-batch chunks, ragged tiles
+def test_step_from_host_buffers(B, H, N, D):
+    """sigattn_step_host: H2D copies, forward, backward, D2H copies in one call, cut into
+    chunks of heads that run on the library's own streams."""
     import torch
     import paper_2409_04431_b200 as sa
-    B, H, N, D = 2, 4, 333, 64
     q, k, v, d_o = inputs.random_case(B, H, N, D, seed=21)
-    slopes = np.array([0.5, 0.25, 0.125, 0.0625], dtype=np.float32)
+    slopes = (0.5 ** np.arange(1, H + 1)).astype(np.float32)
     host_in = [torch.from_numpy(inputs.f32_to_bf16_bits(t).view(np.int16)).view(torch.bfloat16).pin_memory()
                for t in (q, k, v, d_o)]
     host_out = [torch.full_like(host_in[0], float("nan")).pin_memory() for _ in range(4)]
-    scale, bias = 0.125, -math.log(N)
-    sa.sigattn_step_host(*host_in, *host_out, scale, bias, True, torch.from_numpy(slopes))
+    scale, bias = 1.0 / math.sqrt(D), -math.log(N)
+    for _ in range(2):   # the second call reuses streams, events and (here) a fresh arena
+        sa.sigattn_step_host(*host_in, *host_out, scale, bias, True, torch.from_numpy(slopes))
     sa.sigattn_check()
     got = [t.float().numpy().astype(np.float64) for t in host_out]
     assert_close(got[0], oracle.sigattn_fwd(q, k, v, scale, bias, True, slopes), "O")
     for name, g, r in zip(("dQ", "dK", "dV"), got[1:], oracle.sigattn_bwd(q, k, v, d_o, scale, bias, True, slopes)):
         assert_close(g, r, name)
+
+
+def test_step_from_host_buffers_orders_with_caller_stream():
+    """Work enqueued on the caller's stream before the call is seen by it, and work enqueued
+    after it sees its results."""
+    import torch
+    import paper_2409_04431_b200 as sa
+    B, H, N, D = 1, 2, 256, 64
+    q, k, v, d_o = inputs.random_case(B, H, N, D, seed=5)
+    host_in = [torch.from_numpy(inputs.f32_to_bf16_bits(t).view(np.int16)).view(torch.bfloat16).pin_memory()
+               for t in (q, k, v, d_o)]
+    host_out = [torch.zeros_like(host_in[0]).pin_memory() for _ in range(4)]
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        arena = torch.empty(sa.sigattn_step_host_arena_bytes(B, H, N, D, sa.DTYPE_BF16), dtype=torch.uint8,
+                            device="cuda")
+        arena.fill_(0xFF)                      # must finish before the copies in overwrite the arena
+        sa.sigattn_step_host(*host_in, *host_out, 0.125, -5.0, False, None, arena=arena, stream=side)
+        o_dev = arena[4 * host_in[0].numel() * 2: 5 * host_in[0].numel() * 2].clone()   # O as left in the arena
+    side.synchronize()
+    sa.sigattn_check()
+    got = host_out[0].float().numpy().astype(np.float64)
+    assert_close(got, oracle.sigattn_fwd(q, k, v, 0.125, -5.0, False, None), "O")
+    assert torch.equal(o_dev.cpu().view(torch.bfloat16).view(B, H, N, D), host_out[0])
 
 
 # ---------------------------------------------------------------- full-size launches, sampled heads
