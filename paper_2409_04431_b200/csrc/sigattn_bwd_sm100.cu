@@ -5,13 +5,13 @@
 //     P^T  = sigmoid(scale S^T + b ...)     (registers -> bf16 over region A)
 //     dV_j += P^T dO_i                      (A operand from tensor memory)
 //     dP^T = V_j dO_i^T                     (region B)
-//     dS^T = P^T (1 - P^T) dP^T             (registers -> bf16 in shared memory)
-//     dK_j += dS^T Q_i
+//     dS^T = P^T (1 - P^T) dP^T             (registers -> bf16, over region B and in shared memory)
+//     dK_j += dS^T Q_i                      (A operand from tensor memory)
 //     dQ_i  = dS K_j                        (region B again, then fp32 reduce-add to HBM)
 //
 // Everything is kept transposed (keys on the 128 TMEM lanes, queries along columns) so
-// that P^T can feed the dV product straight from tensor memory and one shared-memory
-// copy of dS^T serves both dK (as a K-major A operand) and dQ (as an MN-major A operand).
+// that P^T and dS^T can feed the dV and dK products straight from tensor memory; only dQ
+// needs dS with queries as rows, and reads the shared-memory copy as an MN-major A operand.
 // No row statistic of any kind is read or written: dS is a point-wise function of S and
 // dP (Section 4 / Appendix F.1), and P is recomputed from Q and K alone.
 //
@@ -187,7 +187,6 @@ __device__ void bwd_mma_role(const BwdParams& p, uint32_t smem_base, uint32_t tm
   const uint64_t dDo_k = make_smem_desc_sw128(sDo, 16, 1024);               // dO_i, K-major (dP^T)
   const uint64_t dDo_mn = make_smem_desc_sw128(sDo, L::kPanelBytes, 1024);  // dO_i, MN-major (dV)
   const uint64_t dK_mn = make_smem_desc_sw128(sK, L::kPanelBytes, 1024);    // K_j, MN-major (dQ)
-  const uint64_t dDs_k = make_smem_desc_sw128(sDs, 16, 1024);               // dS^T, K-major (dK)
   const uint64_t dDs_mn = make_smem_desc_sw128(sDs, L::kPanelBytes, 1024);  // dS^T, MN-major (dQ)
   const uint64_t dQ_k[2] = {make_smem_desc_sw128(smem_base + L::kQOff, 16, 1024),
                             make_smem_desc_sw128(smem_base + L::kQOff + L::kTileBytes, 16, 1024)};
@@ -235,19 +234,21 @@ __device__ void bwd_mma_role(const BwdParams& p, uint32_t smem_base, uint32_t tm
         issue_kk(TM::kA, dK_k, dQ_k[nst]);
         umma_commit(smem_u32(&bars->s_full));
       }
-      // dQ_i = dS K_j first (its drain is on the critical path), then dK += dS^T Q_i
+      // dK += dS^T Q_i with dS^T read from region B of tensor memory (the activation groups
+      // leave a bf16 copy there, over the dP^T columns they have consumed), then dQ_i = dS K_j,
+      // which overwrites region B: MMAs of one thread execute in issue order.
       if (!mbar_wait(smem_u32(&bars->ds_ready), step_cnt & 1, cta_err, 57)) return;
       tc_fence_after_sync();
+#pragma unroll
+      for (int ks = 0; ks < kT / 16; ++ks) {
+        umma_ts(tmem + TM::kDk, tmem + TM::kB + (ks >> 2) * 64 + (ks & 3) * 8, desc_advance(dQ_mn[st], ks * 2048),
+                kIdescAcc, (it > 0 || ks > 0));
+      }
 #pragma unroll
       for (int ks = 0; ks < kT / 16; ++ks) {
         umma_ss(tmem + TM::kB, desc_advance(dDs_mn, ks * 2048), desc_advance(dK_mn, ks * 2048), kIdescDq, ks > 0);
       }
       umma_commit(smem_u32(&bars->dq_full));
-#pragma unroll
-      for (int ks = 0; ks < kT / 16; ++ks) {
-        umma_ss(tmem + TM::kDk, desc_advance(dDs_k, (ks >> 2) * L::kPanelBytes + (ks & 3) * 32),
-                desc_advance(dQ_mn[st], ks * 2048), kIdescAcc, (it > 0 || ks > 0));
-      }
       umma_commit(smem_u32(&bars->q_empty[st]));
       ++q_cnt;
       ++step_cnt;
@@ -364,18 +365,23 @@ __device__ void bwd_act_role(const BwdParams& p, const CUtensorMap* tmDk, const 
         uint32_t dp[16];
         tmem_ld16(tmem + TM::kB + lane_off + wg * 64 + c * 16, dp);
         tmem_wait_ld();
+        uint32_t ds[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const float* f = ((c < 2) ? pp0 : pp1) + (c & 1) * 16 + 2 * e;
+          ds[e] = pack_bf16x2(f[0] * __uint_as_float(dp[2 * e]), f[1] * __uint_as_float(dp[2 * e + 1]));
+        }
+        // one copy to shared memory (A operand of dQ, MN-major) ...
 #pragma unroll
         for (int g = 0; g < 2; ++g) {
-          uint4 val;
-          const float* f = ((c < 2) ? pp0 : pp1) + (c & 1) * 16 + g * 8;
-          val.x = pack_bf16x2(f[0] * __uint_as_float(dp[8 * g + 0]), f[1] * __uint_as_float(dp[8 * g + 1]));
-          val.y = pack_bf16x2(f[2] * __uint_as_float(dp[8 * g + 2]), f[3] * __uint_as_float(dp[8 * g + 3]));
-          val.z = pack_bf16x2(f[4] * __uint_as_float(dp[8 * g + 4]), f[5] * __uint_as_float(dp[8 * g + 5]));
-          val.w = pack_bf16x2(f[6] * __uint_as_float(dp[8 * g + 6]), f[7] * __uint_as_float(dp[8 * g + 7]));
           const int chunk = c * 2 + g;
-          *reinterpret_cast<uint4*>(ds_row + ((chunk ^ (tid & 7)) * 16)) = val;
+          *reinterpret_cast<uint4*>(ds_row + ((chunk ^ (tid & 7)) * 16)) =
+              make_uint4(ds[4 * g + 0], ds[4 * g + 1], ds[4 * g + 2], ds[4 * g + 3]);
         }
+        // ... and one to tensor memory (A operand of dK), over dP^T columns already consumed
+        tmem_st8(tmem + TM::kB + lane_off + wg * 64 + c * 8, ds);
       }
+      tmem_wait_st();
       tc_fence_before_sync();   // the dP^T reads above precede the dQ MMA that overwrites region B
       fence_proxy_async_smem();
       mbar_arrive(smem_u32(&bars->ds_ready));
