@@ -179,6 +179,7 @@ __device__ void fwd_mma_role(const FwdParams& p, uint32_t smem_base, uint32_t tm
   using L = FwdSmem<D>;
   constexpr uint32_t kIdescS = make_idesc_bf16(kBM, kBN, 0, 0);
   constexpr uint32_t kIdescPV = make_idesc_bf16(kBM, D, 0, 1);
+  const uint32_t leader = (threadIdx.x & 31) == 0;   // the lane that issues; all lanes run the loop
   uint32_t kv_cnt = 0;
   uint32_t it[2] = {0, 0};      // items seen per query tile
   uint32_t p_cnt[2] = {0, 0};   // P tiles consumed per query tile
@@ -193,7 +194,7 @@ __device__ void fwd_mma_role(const FwdParams& p, uint32_t smem_base, uint32_t tm
 #pragma unroll
     for (int ks = 0; ks < D / 16; ++ks) {
       const uint32_t off = (ks >> 2) * L::kPanelBytes + (ks & 3) * 32;
-      umma_ss(tmem + t * kBN, desc_advance(qd, off), desc_advance(kd, off), kIdescS, ks > 0);
+      umma_ss_warp(leader, tmem + t * kBN, desc_advance(qd, off), desc_advance(kd, off), kIdescS, ks > 0);
     }
   };
   // O_t (+)= P_t V : A = bf16 P in tensor memory (aliasing S_t), B = V, MN-major.
@@ -204,7 +205,7 @@ __device__ void fwd_mma_role(const FwdParams& p, uint32_t smem_base, uint32_t tm
       // column group c wrote its bf16 P over the first half of its own logits columns:
       // [c kCols, c kCols + kCols / 2), one k-step of 16 keys per 8 columns
       const uint32_t p_col = (ks / (kCols / 16)) * kCols + (ks % (kCols / 16)) * 8;
-      umma_ts(tmem + 2 * kBN + t * D, tmem + t * kBN + p_col, desc_advance(vd, ks * 2048), kIdescPV,
+      umma_ts_warp(leader, tmem + 2 * kBN + t * D, tmem + t * kBN + p_col, desc_advance(vd, ks * 2048), kIdescPV,
               (accumulate || ks > 0));
     }
   };
@@ -213,7 +214,7 @@ __device__ void fwd_mma_role(const FwdParams& p, uint32_t smem_base, uint32_t tm
     return mbar_wait(smem_u32(&bars->kv_full[stage]), phase, cta_err, 20);
   };
   auto kv_addr = [&](uint32_t cnt) { return smem_base + L::kKvOff + (cnt % L::kStages) * L::kTileBytes; };
-  auto kv_release = [&](uint32_t cnt) { umma_commit(smem_u32(&bars->kv_empty[cnt % L::kStages])); };
+  auto kv_release = [&](uint32_t cnt) { umma_commit_warp(leader, smem_u32(&bars->kv_empty[cnt % L::kStages])); };
 
   for (int round = 0, rounds = num_rounds(p.n_items); round < rounds; ++round) {
     const int item = snake_rank(round, p.n_items);
@@ -229,12 +230,12 @@ __device__ void fwd_mma_role(const FwdParams& p, uint32_t smem_base, uint32_t tm
     if (!kv_wait(k_cnt(0))) return;
     tc_fence_after_sync();
     issue_s(0, kv_addr(k_cnt(0)));
-    umma_commit(smem_u32(&bars->s_full[0]));
+    umma_commit_warp(leader, smem_u32(&bars->s_full[0]));
     if (w.n[1] > 0) {
       if (!mbar_wait(smem_u32(&bars->q_full[1]), it[1] & 1, cta_err, 22)) return;
       tc_fence_after_sync();
       issue_s(1, kv_addr(k_cnt(0)));
-      umma_commit(smem_u32(&bars->s_full[1]));
+      umma_commit_warp(leader, smem_u32(&bars->s_full[1]));
     }
     kv_release(k_cnt(0));
     // accumulators of the previous item must have been read out before the first PV overwrites them
@@ -249,25 +250,25 @@ __device__ void fwd_mma_role(const FwdParams& p, uint32_t smem_base, uint32_t tm
         ++p_cnt[0];
         tc_fence_after_sync();
         issue_pv(0, kv_addr(v_cnt(j)), j > 0);
-        if (j == w.n[0] - 1) umma_commit(smem_u32(&bars->o_full[0]));
+        if (j == w.n[0] - 1) umma_commit_warp(leader, smem_u32(&bars->o_full[0]));
       }
       if (more && !kv_wait(k_cnt(j + 1))) return;
       if (j + 1 < w.n[0]) {
         tc_fence_after_sync();
         issue_s(0, kv_addr(k_cnt(j + 1)));
-        umma_commit(smem_u32(&bars->s_full[0]));
+        umma_commit_warp(leader, smem_u32(&bars->s_full[0]));
       }
       if (j < w.n[1]) {
         if (!mbar_wait(smem_u32(&bars->p_full[1]), p_cnt[1] & 1, cta_err, 26)) return;
         ++p_cnt[1];
         tc_fence_after_sync();
         issue_pv(1, kv_addr(v_cnt(j)), j > 0);
-        if (j == w.n[1] - 1) umma_commit(smem_u32(&bars->o_full[1]));
+        if (j == w.n[1] - 1) umma_commit_warp(leader, smem_u32(&bars->o_full[1]));
       }
       kv_release(v_cnt(j));
       if (j + 1 < w.n[1]) {
         issue_s(1, kv_addr(k_cnt(j + 1)));
-        umma_commit(smem_u32(&bars->s_full[1]));
+        umma_commit_warp(leader, smem_u32(&bars->s_full[1]));
       }
       if (more) kv_release(k_cnt(j + 1));
     }
@@ -468,7 +469,7 @@ sigattn_fwd_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
     if ((threadIdx.x & 31) == 0) fwd_load_role<D, CAUSAL>(p, &tmQ, &tmK, &tmV, smem_base, &bars, &cta_err);
     __syncwarp();
   } else if (warp == kMmaWarp) {
-    if ((threadIdx.x & 31) == 0) fwd_mma_role<D, CAUSAL>(p, smem_base, tmem, &bars, &cta_err);
+    fwd_mma_role<D, CAUSAL>(p, smem_base, tmem, &bars, &cta_err);
     __syncwarp();
   } else {
     fwd_act_role<D, CAUSAL, ALIBI>(p, &tmO, smem, tmem, &bars, &cta_err);
