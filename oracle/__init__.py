@@ -11,5 +11,6 @@ from .sigattn_oracle import (  # noqa: F401
     attention_weights,
     sigattn_fwd,
     sigattn_bwd,
+    sigattn_bwd_dbias,
     sigattn_fwd_sequence_form,
 )

@@ -34,6 +34,12 @@ Readings of the paper taken here
     head's positive slope m_h times the distance |i - j| is subtracted from the scaled
     logit (not multiplied by scale); for causal calls only j <= i survives, which is
     the usual m_h * (i - j).
+  * The bias may differ per sequence and per head: the speech models use b = -log n with
+    n the length of each sample and ablate a learnable bias (Section 5.4, Appendix G.4),
+    and a learnable scalar b replaces LayerScale in Appendix G.2.2.  `bias` is therefore
+    a scalar or anything that broadcasts to [B, H]; it enters x_ij additively, so its
+    gradient is db[b, h] = sum_ij dS_ij (the chain rule through x = u + b; masked entries
+    carry dS = 0).  The paper prints no formula for db.
 
 Every function is pinned by tests that do not call back into this file's own
 formulae (closed forms, brute-force loops, finite differences, the paper's second
@@ -50,6 +56,7 @@ __all__ = [
     "attention_weights",
     "sigattn_fwd",
     "sigattn_bwd",
+    "sigattn_bwd_dbias",
     "sigattn_fwd_sequence_form",
 ]
 
@@ -114,6 +121,14 @@ def _slopes(alibi_slopes, num_heads):
     return s
 
 
+def _bias_per_head(bias, num_batch, num_heads):
+    """Scalar, [B], [B, 1], [1, H] or [B, H] bias -> float64 [B, H]."""
+    b = np.asarray(bias, dtype=np.float64)
+    if b.ndim == 1 and b.shape[0] == num_batch and num_batch != num_heads:
+        b = b[:, None]
+    return np.ascontiguousarray(np.broadcast_to(b, (num_batch, num_heads)))
+
+
 def _row_ranges(n, row_block):
     """Query rows are independent in the forward and enter dK, dV only through a sum
     over rows, so they may be visited in slabs to bound memory (an n x n float64 matrix
@@ -126,43 +141,63 @@ def sigattn_fwd(q, k, v, scale, bias, causal=False, alibi_slopes=None, row_block
     """O = sigmoid(scale * Q K^T + b [+ position bias]) [* causal mask] V  (Eq. 3).
 
     q, k, v: [B, H, N, D] arrays (any float dtype; converted to float64).
+    bias: scalar, or an array that broadcasts to [B, H] (one bias per sequence and head).
     Returns O as float64 [B, H, N, D].
     """
     q, k, v = _as_f64(q, k, v)
     B, H, N, D = q.shape
     slopes = _slopes(alibi_slopes, H)
+    bias_bh = _bias_per_head(bias, B, H)
     o = np.zeros((B, H, N, D), dtype=np.float64)
     for b in range(B):
         for h in range(H):
             for i0, i1 in _row_ranges(N, row_block):
-                p = attention_weights(q[b, h], k[b, h], scale, bias, causal, slopes[h], i0, i1)
+                p = attention_weights(q[b, h], k[b, h], scale, bias_bh[b, h], causal, slopes[h], i0, i1)
                 o[b, h, i0:i1] = p @ v[b, h]
     return o
 
 
-def sigattn_bwd(q, k, v, d_o, scale, bias, causal=False, alibi_slopes=None, row_block=None):
-    """Gradients of L = sum(O * dO) with respect to Q, K, V (sigmoid column of the
-    forward/backward table in Appendix F.1, with the 1/sqrt(d) factor; see header).
-
-    Returns (dQ, dK, dV), float64 [B, H, N, D] each.
-    """
+def _bwd_all(q, k, v, d_o, scale, bias, causal, alibi_slopes, row_block):
     q, k, v, d_o = _as_f64(q, k, v, d_o)
     B, H, N, D = q.shape
     slopes = _slopes(alibi_slopes, H)
+    bias_bh = _bias_per_head(bias, B, H)
     dq = np.zeros_like(q)
     dk = np.zeros_like(q)
     dv = np.zeros_like(q)
+    dbias = np.zeros((B, H), dtype=np.float64)
     for b in range(B):
         for h in range(H):
             for i0, i1 in _row_ranges(N, row_block):
-                p = attention_weights(q[b, h], k[b, h], scale, bias, causal, slopes[h], i0, i1)
+                p = attention_weights(q[b, h], k[b, h], scale, bias_bh[b, h], causal, slopes[h], i0, i1)
                 do_rows = d_o[b, h, i0:i1]
                 dv[b, h] += p.T @ do_rows
                 dp = do_rows @ v[b, h].T
                 ds = p * (1.0 - p) * dp
                 dq[b, h, i0:i1] = scale * (ds @ k[b, h])
                 dk[b, h] += scale * (ds.T @ q[b, h, i0:i1])
-    return dq, dk, dv
+                dbias[b, h] += ds.sum()
+    return dq, dk, dv, dbias
+
+
+def sigattn_bwd(q, k, v, d_o, scale, bias, causal=False, alibi_slopes=None, row_block=None):
+    """Gradients of L = sum(O * dO) with respect to Q, K, V (sigmoid column of the
+    forward/backward table in Appendix F.1, with the 1/sqrt(d) factor; see header).
+
+    bias: scalar, or an array that broadcasts to [B, H].
+    Returns (dQ, dK, dV), float64 [B, H, N, D] each.
+    """
+    return _bwd_all(q, k, v, d_o, scale, bias, causal, alibi_slopes, row_block)[:3]
+
+
+def sigattn_bwd_dbias(q, k, v, d_o, scale, bias, causal=False, alibi_slopes=None, row_block=None):
+    """Gradient of L = sum(O * dO) with respect to a bias held per (batch, head):
+    db[b, h] = sum_ij dS_ij with dS = P (1 - P) dP as in sigattn_bwd (see header).  A
+    bias shared by several heads or sequences gets the sum of their entries.
+
+    Returns float64 [B, H].
+    """
+    return _bwd_all(q, k, v, d_o, scale, bias, causal, alibi_slopes, row_block)[3]
 
 
 def sigattn_fwd_sequence_form(q, k, v, scale, n_bias):

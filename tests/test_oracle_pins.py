@@ -307,3 +307,79 @@ def test_backward_structure_properties():
     dq, dk, dv = g1
     p = scalar_sigmoid(scale * float(q[0, 0, -1] @ k[0, 0, -1]) + b)
     np.testing.assert_allclose(dv[0, 0, -1], p * d_o[0, 0, -1], rtol=1e-13)
+
+
+# ------------------------------------------------------- bias per (batch, head) and its gradient
+
+
+def test_bias_per_batch_and_head_equals_separate_scalar_calls():
+    """A [B, H] bias must act as if every (batch, head) were computed alone with its own
+    scalar bias; a [B] vector is one bias per sequence (b = -log n of each sample)."""
+    B, H, N, D = 3, 2, 5, 4
+    q, k, v, d_o = (rnd((B, H, N, D), s) for s in (60, 61, 62, 63))
+    bias = rnd((B, H), 64)
+    slopes = np.array([0.5, 0.25])
+    o = oracle.sigattn_fwd(q, k, v, 0.4, bias, True, slopes)
+    grads = oracle.sigattn_bwd(q, k, v, d_o, 0.4, bias, True, slopes)
+    for b in range(B):
+        for h in range(H):
+            sel = (slice(b, b + 1), slice(h, h + 1))
+            np.testing.assert_array_equal(
+                o[sel], oracle.sigattn_fwd(q[sel], k[sel], v[sel], 0.4, float(bias[b, h]), True, slopes[h:h + 1]))
+            one = oracle.sigattn_bwd(q[sel], k[sel], v[sel], d_o[sel], 0.4, float(bias[b, h]), True, slopes[h:h + 1])
+            for g, r in zip(grads, one):
+                np.testing.assert_array_equal(g[sel], r)
+    per_sample = -np.log(np.array([3.0, 4.0, 5.0]))
+    np.testing.assert_array_equal(oracle.sigattn_fwd(q, k, v, 0.4, per_sample, False),
+                                  oracle.sigattn_fwd(q, k, v, 0.4, np.repeat(per_sample[:, None], H, axis=1), False))
+    o_brute = np.concatenate([brute_forward(q[b:b + 1], k[b:b + 1], v[b:b + 1], 0.4, float(per_sample[b]), False, None)
+                              for b in range(B)])
+    np.testing.assert_allclose(oracle.sigattn_fwd(q, k, v, 0.4, per_sample, False), o_brute, rtol=1e-13, atol=1e-15)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("with_slopes", [False, True])
+def test_bias_gradient_finite_differences(causal, with_slopes):
+    """Central differences of L = sum(O * dO) with respect to each entry of a [B, H] bias."""
+    B, H, N, D = 2, 2, 6, 4
+    q, k, v, d_o = (rnd((B, H, N, D), s) for s in (70, 71, 72, 73))
+    slopes = np.array([0.5, 0.125]) if with_slopes else None
+    bias = -math.log(N) + 0.3 * rnd((B, H), 74)
+    scale = 1 / math.sqrt(D)
+    db = oracle.sigattn_bwd_dbias(q, k, v, d_o, scale, bias, causal, slopes)
+    assert db.shape == (B, H)
+    h = 1e-6
+    fd = np.zeros_like(bias)
+    for idx in np.ndindex(*bias.shape):
+        bp, bm = bias.copy(), bias.copy()
+        bp[idx] += h
+        bm[idx] -= h
+        fd[idx] = (loss(q, k, v, d_o, scale, bp, causal, slopes) - loss(q, k, v, d_o, scale, bm, causal, slopes)) / (2 * h)
+    assert np.linalg.norm(fd - db) / np.linalg.norm(fd) < 1e-7
+    # a scalar bias shared by everything gets the sum of the entries
+    shared = -math.log(N)
+    total = float(oracle.sigattn_bwd_dbias(q, k, v, d_o, scale, shared, causal, slopes).sum())
+    fd_shared = (loss(q, k, v, d_o, scale, shared + h, causal, slopes) - loss(q, k, v, d_o, scale, shared - h, causal, slopes)) / (2 * h)
+    assert abs(total - fd_shared) < 1e-7 * max(1.0, abs(fd_shared))
+
+
+def test_bias_gradient_single_token_closed_form_and_brute_force():
+    D = 5
+    q, k, v, d_o = (rnd((1, 1, 1, D), s) for s in (80, 81, 82, 83))
+    scale, b = 0.3, -0.4
+    p = scalar_sigmoid(scale * float(q[0, 0, 0] @ k[0, 0, 0]) + b)
+    expect = float(d_o[0, 0, 0] @ v[0, 0, 0]) * p * (1 - p)
+    np.testing.assert_allclose(oracle.sigattn_bwd_dbias(q, k, v, d_o, scale, b, True), [[expect]], rtol=1e-14)
+    # brute force over every (i, j) of a small causal problem with slopes
+    B, H, N, D = 1, 2, 5, 3
+    q, k, v, d_o = (rnd((B, H, N, D), s) for s in (84, 85, 86, 87))
+    slopes = np.array([0.25, 0.5])
+    bias = np.array([[-0.9, 0.2]])
+    ref = np.zeros((B, H))
+    for h in range(H):
+        for i in range(N):
+            for j in range(i + 1):
+                x = 0.7 * float(q[0, h, i] @ k[0, h, j]) + bias[0, h] - slopes[h] * (i - j)
+                pp = scalar_sigmoid(x)
+                ref[0, h] += pp * (1 - pp) * float(d_o[0, h, i] @ v[0, h, j])
+    np.testing.assert_allclose(oracle.sigattn_bwd_dbias(q, k, v, d_o, 0.7, bias, True, slopes), ref, rtol=1e-13)
