@@ -122,6 +122,31 @@ SIGATTN_API int sigattn_bwd_static_scratch(const void* q, const void* k, const v
 /* Largest B*H*N*D that sigattn_bwd_static_scratch accepts. */
 SIGATTN_API size_t sigattn_bwd_static_scratch_max_elements(void);
 
+/* sigattn_fwd with one bias per (batch, head) instead of one scalar: the speech models of
+ * Section 5.4 / Appendix G.4 use b = -log n with n the length of each sample, and a
+ * learnable bias is ablated there and in Appendix G.2.2.  `bias_bh` is a DEVICE pointer to
+ * B*H floats, row-major [B][H], 4-byte aligned, read while the kernel runs; entry [b][h]
+ * takes the place of `bias` for that sequence and head.  Everything else as sigattn_fwd. */
+SIGATTN_API int sigattn_fwd_bias_vec(const void* q, const void* k, const void* v, void* o,
+                         int B, int H, int N, int D,
+                         float scale, const float* bias_bh, int causal,
+                         const float* alibi_slopes, int dtype, void* stream);
+
+/* sigattn_bwd with the bias vector of sigattn_fwd_bias_vec, and optionally the gradient
+ * of L = sum(O * dO) with respect to it: if `dbias_bh` is not NULL it is a DEVICE pointer
+ * to B*H floats that receive db[b][h] = sum over (i, j) of dS_ij (dS = P (1 - P) dP; the
+ * bias enters every logit additively).  The paper prints no formula for db; a bias shared
+ * by heads or sequences gets the sum of their entries.  The array is cleared and then
+ * added into with fp32 atomics, so its last bits depend on the order of the additions.
+ * Everything else as sigattn_bwd. */
+SIGATTN_API int sigattn_bwd_bias_vec(const void* q, const void* k, const void* v, const void* d_o,
+                         void* dq, void* dk, void* dv,
+                         int B, int H, int N, int D,
+                         float scale, const float* bias_bh, int causal,
+                         const float* alibi_slopes, int dtype,
+                         float* dbias_bh,
+                         void* workspace, size_t workspace_bytes, void* stream);
+
 /* Bytes of scratch sigattn_bwd needs for this problem (0 for the fp32 debug path).
  * Returns 0 for invalid shapes as well; sigattn_bwd reports those. */
 SIGATTN_API size_t sigattn_bwd_workspace_bytes(int B, int H, int N, int D, int dtype);

@@ -25,6 +25,9 @@ _BINDING_NAMES = (
     "sigattn_bwd_static_scratch",
     "sigattn_bwd_static_scratch_max_elements",
     "sigattn_selftest_bounded_wait",
+    "sigattn_fwd_bias_vec",
+    "sigattn_bwd_bias_vec",
+    "lib",
 )
 
 __all__ = list(_BINDING_NAMES)

@@ -31,6 +31,13 @@ _lib.sigattn_bwd.restype = _c.c_int
 _lib.sigattn_bwd.argtypes = [_c.c_void_p] * 7 + [_c.c_int] * 4 + [_c.c_float, _c.c_float, _c.c_int,
                                                                     _c.c_void_p, _c.c_int, _c.c_void_p,
                                                                     _c.c_size_t, _c.c_void_p]
+_lib.sigattn_fwd_bias_vec.restype = _c.c_int
+_lib.sigattn_fwd_bias_vec.argtypes = [_c.c_void_p] * 4 + [_c.c_int] * 4 + [_c.c_float, _c.c_void_p, _c.c_int,
+                                                                             _c.c_void_p, _c.c_int, _c.c_void_p]
+_lib.sigattn_bwd_bias_vec.restype = _c.c_int
+_lib.sigattn_bwd_bias_vec.argtypes = [_c.c_void_p] * 7 + [_c.c_int] * 4 + [_c.c_float, _c.c_void_p, _c.c_int,
+                                                                             _c.c_void_p, _c.c_int, _c.c_void_p,
+                                                                             _c.c_void_p, _c.c_size_t, _c.c_void_p]
 _lib.sigattn_bwd_workspace_bytes.restype = _c.c_size_t
 _lib.sigattn_bwd_workspace_bytes.argtypes = [_c.c_int] * 5
 _lib.sigattn_step_host.restype = _c.c_int
@@ -64,7 +71,7 @@ EXPORTED = [
     "sigattn_strerror", "sigattn_last_cuda_error", "sigattn_version", "sigattn_launch_count",
     "sigattn_step_host", "sigattn_step_host_arena_bytes", "sigattn_bwd_set_timing_events",
     "sigattn_bwd_static_scratch", "sigattn_bwd_static_scratch_max_elements",
-    "sigattn_selftest_bounded_wait",
+    "sigattn_selftest_bounded_wait", "sigattn_fwd_bias_vec", "sigattn_bwd_bias_vec",
 ]
 
 
@@ -190,6 +197,62 @@ def sigattn_bwd(q, k, v, d_o, scale, bias, causal=False, alibi_slopes=None, work
     if rc != 0:
         raise SigattnError(rc)
     return dq, dk, dv
+
+
+def _check_bias_vec(bias_bh, q):
+    import torch
+    B, H = q.shape[0], q.shape[1]
+    if (not isinstance(bias_bh, torch.Tensor) or not bias_bh.is_cuda or bias_bh.dtype != torch.float32
+            or tuple(bias_bh.shape) != (B, H) or not bias_bh.is_contiguous() or bias_bh.device != q.device):
+        raise ValueError("bias_bh must be a contiguous float32 CUDA tensor of shape [B, H] on q's device")
+
+
+def sigattn_fwd_bias_vec(q, k, v, scale, bias_bh, causal=False, alibi_slopes=None, out=None, stream=None):
+    """sigattn_fwd with one bias per (batch, head): `bias_bh` is a float32 CUDA tensor [B, H]."""
+    import torch
+    _check_same([q, k, v], ["q", "k", "v"])
+    _check_bias_vec(bias_bh, q)
+    if out is None:
+        out = torch.empty_like(q)
+    else:
+        _check_same([q, out], ["q", "out"])
+    B, H, N, D = q.shape
+    with torch.cuda.device(q.device):
+        rc = _lib.sigattn_fwd_bias_vec(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, H, N, D, float(scale),
+                                       _ptr(bias_bh), int(bool(causal)), _ptr(alibi_slopes), _dtype_code(q),
+                                       _stream_ptr(stream))
+    if rc != 0:
+        raise SigattnError(rc)
+    return out
+
+
+def sigattn_bwd_bias_vec(q, k, v, d_o, scale, bias_bh, causal=False, alibi_slopes=None, want_dbias=True,
+                         workspace=None, out=None, stream=None):
+    """sigattn_bwd with the bias vector of sigattn_fwd_bias_vec.  Returns (dQ, dK, dV, dbias)
+    where dbias is a float32 CUDA tensor [B, H] holding sum dS per (batch, head), or None if
+    `want_dbias` is False."""
+    import torch
+    _check_same([q, k, v, d_o], ["q", "k", "v", "d_o"])
+    _check_bias_vec(bias_bh, q)
+    B, H, N, D = q.shape
+    code = _dtype_code(q)
+    if out is None:
+        dq, dk, dv = torch.empty_like(q), torch.empty_like(q), torch.empty_like(q)
+    else:
+        dq, dk, dv = out
+        _check_same([q, dq, dk, dv], ["q", "dq", "dk", "dv"])
+    dbias = torch.empty((B, H), dtype=torch.float32, device=q.device) if want_dbias else None
+    need = sigattn_bwd_workspace_bytes(B, H, N, D, code)
+    if workspace is None and need > 0:
+        workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    with torch.cuda.device(q.device):
+        rc = _lib.sigattn_bwd_bias_vec(_ptr(q), _ptr(k), _ptr(v), _ptr(d_o), _ptr(dq), _ptr(dk), _ptr(dv), B, H, N, D,
+                                       float(scale), _ptr(bias_bh), int(bool(causal)), _ptr(alibi_slopes), code,
+                                       _ptr(dbias), _ptr(workspace), ws_bytes, _stream_ptr(stream))
+    if rc != 0:
+        raise SigattnError(rc)
+    return dq, dk, dv, dbias
 
 
 def sigattn_step_host_arena_bytes(B, H, N, D, dtype_code) -> int:

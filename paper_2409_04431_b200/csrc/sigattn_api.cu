@@ -84,10 +84,11 @@ void account(unsigned long long launches, int rc, cudaError_t cuda_err) {
 
 }  // namespace sigattn
 
-extern "C" {
+namespace {
 
-int sigattn_fwd(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int D, float scale,
-                float bias, int causal, const float* alibi_slopes, int dtype, void* stream) {
+// Shared by the scalar-bias and the bias-vector entry points.
+int fwd_any(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int D, float scale, float bias,
+            const float* bias_vec, int causal, const float* alibi_slopes, int dtype, void* stream) {
   if (!q || !k || !v || !o) return SIGATTN_ERR_NULL;
   if (int rc = check_shape(B, H, N, D)) return rc;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return SIGATTN_ERR_ALIGN;
@@ -97,7 +98,7 @@ int sigattn_fwd(const void* q, const void* k, const void* v, void* o, int B, int
   int dev = 0;
   int* status = nullptr;
   if (int rc = device_setup(&dev, &status)) return rc;
-  sigattn::Problem p{B, H, N, D, scale, bias, causal, alibi_slopes};
+  sigattn::Problem p{B, H, N, D, scale, bias, causal, alibi_slopes, bias_vec, nullptr};
   unsigned long long launches = 0;
   cudaError_t ce = cudaSuccess;
   int rc;
@@ -113,9 +114,9 @@ int sigattn_fwd(const void* q, const void* k, const void* v, void* o, int B, int
   return rc;
 }
 
-int sigattn_bwd(const void* q, const void* k, const void* v, const void* d_o, void* dq, void* dk, void* dv, int B,
-                int H, int N, int D, float scale, float bias, int causal, const float* alibi_slopes, int dtype,
-                void* workspace, size_t workspace_bytes, void* stream) {
+int bwd_any(const void* q, const void* k, const void* v, const void* d_o, void* dq, void* dk, void* dv, int B, int H,
+            int N, int D, float scale, float bias, const float* bias_vec, float* dbias, int causal,
+            const float* alibi_slopes, int dtype, void* workspace, size_t workspace_bytes, void* stream) {
   if (!q || !k || !v || !d_o || !dq || !dk || !dv) return SIGATTN_ERR_NULL;
   if (int rc = check_shape(B, H, N, D)) return rc;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(d_o) || !aligned16(dq) || !aligned16(dk) ||
@@ -133,7 +134,7 @@ int sigattn_bwd(const void* q, const void* k, const void* v, const void* d_o, vo
   int dev = 0;
   int* status = nullptr;
   if (int rc = device_setup(&dev, &status)) return rc;
-  sigattn::Problem p{B, H, N, D, scale, bias, causal, alibi_slopes};
+  sigattn::Problem p{B, H, N, D, scale, bias, causal, alibi_slopes, bias_vec, dbias};
   unsigned long long launches = 0;
   cudaError_t ce = cudaSuccess;
   int rc;
@@ -149,6 +150,41 @@ int sigattn_bwd(const void* q, const void* k, const void* v, const void* d_o, vo
   g_launches.fetch_add(launches);
   if (rc == SIGATTN_ERR_CUDA) t_last_cuda = ce;
   return rc;
+}
+
+}  // namespace
+
+extern "C" {
+
+int sigattn_fwd(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int D, float scale,
+                float bias, int causal, const float* alibi_slopes, int dtype, void* stream) {
+  return fwd_any(q, k, v, o, B, H, N, D, scale, bias, nullptr, causal, alibi_slopes, dtype, stream);
+}
+
+int sigattn_fwd_bias_vec(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int D,
+                         float scale, const float* bias_bh, int causal, const float* alibi_slopes, int dtype,
+                         void* stream) {
+  if (!bias_bh) return SIGATTN_ERR_NULL;
+  if (reinterpret_cast<uintptr_t>(bias_bh) & 3u) return SIGATTN_ERR_ALIGN;
+  return fwd_any(q, k, v, o, B, H, N, D, scale, 0.0f, bias_bh, causal, alibi_slopes, dtype, stream);
+}
+
+int sigattn_bwd(const void* q, const void* k, const void* v, const void* d_o, void* dq, void* dk, void* dv, int B,
+                int H, int N, int D, float scale, float bias, int causal, const float* alibi_slopes, int dtype,
+                void* workspace, size_t workspace_bytes, void* stream) {
+  return bwd_any(q, k, v, d_o, dq, dk, dv, B, H, N, D, scale, bias, nullptr, nullptr, causal, alibi_slopes, dtype,
+                 workspace, workspace_bytes, stream);
+}
+
+int sigattn_bwd_bias_vec(const void* q, const void* k, const void* v, const void* d_o, void* dq, void* dk, void* dv,
+                         int B, int H, int N, int D, float scale, const float* bias_bh, int causal,
+                         const float* alibi_slopes, int dtype, float* dbias_bh, void* workspace,
+                         size_t workspace_bytes, void* stream) {
+  if (!bias_bh) return SIGATTN_ERR_NULL;
+  if ((reinterpret_cast<uintptr_t>(bias_bh) & 3u) || (reinterpret_cast<uintptr_t>(dbias_bh) & 3u))
+    return SIGATTN_ERR_ALIGN;
+  return bwd_any(q, k, v, d_o, dq, dk, dv, B, H, N, D, scale, 0.0f, bias_bh, dbias_bh, causal, alibi_slopes, dtype,
+                 workspace, workspace_bytes, stream);
 }
 
 int sigattn_bwd_set_timing_events(void* start_event, void* stop_event) {

@@ -71,6 +71,8 @@ struct BwdParams {
   int n_tiles;  // ceil(N / 128), for keys and for queries
   int n_items;
   float scale, scale_log2e, bias_log2e;
+  const float* bias_vec;   // one bias per (batch, head) instead of the scalar, or nullptr
+  float* dbias;            // receives sum dS per (batch, head), or nullptr
   const float* slopes;
   int* status;
 };
@@ -316,7 +318,7 @@ __device__ __forceinline__ void bwd_store_acc_rows(uint32_t t_acc, uint8_t* stag
   }
 }
 
-template <int D, bool CAUSAL, bool ALIBI>
+template <int D, bool CAUSAL, bool ALIBI, bool DBIAS>
 __device__ void bwd_act_role(const BwdParams& p, const CUtensorMap* tmDk, const CUtensorMap* tmDv, int wg,
                              uint8_t* smem, uint32_t tmem, BwdBarriers* bars, volatile int* cta_err) {
   using L = BwdSmem<D>;
@@ -331,6 +333,8 @@ __device__ void bwd_act_role(const BwdParams& p, const CUtensorMap* tmDk, const 
     const BwdItem w = decode_bwd_item<CAUSAL>(p, item);
     float slope_log2e = 0.0f;
     if (ALIBI) slope_log2e = p.slopes[w.bh % p.H] * kLog2eB;
+    const float bias_log2e = p.bias_vec ? __ldg(p.bias_vec + w.bh) * kLog2eB : p.bias_log2e;
+    float ds_sum = 0.0f;   // this thread's share of sum dS over the item (the bias gradient)
 
     for (int it = 0; it < w.n; ++it) {
       const int i = w.i_begin + it;
@@ -347,9 +351,9 @@ __device__ void bwd_act_role(const BwdParams& p, const CUtensorMap* tmDk, const 
         tmem_wait_ld();
         float(&ppc)[32] = (c == 0) ? pp0 : pp1;
         if (diag)
-          bwd_sigmoid_chunk<true, ALIBI>(s, pk, ppc, p.scale_log2e, p.bias_log2e, slope_log2e, col_rel, gc * 32);
+          bwd_sigmoid_chunk<true, ALIBI>(s, pk, ppc, p.scale_log2e, bias_log2e, slope_log2e, col_rel, gc * 32);
         else
-          bwd_sigmoid_chunk<false, ALIBI>(s, pk, ppc, p.scale_log2e, p.bias_log2e, slope_log2e, col_rel, gc * 32);
+          bwd_sigmoid_chunk<false, ALIBI>(s, pk, ppc, p.scale_log2e, bias_log2e, slope_log2e, col_rel, gc * 32);
         tmem_st16(tmem + TM::kA + lane_off + wg * 64 + c * 16, pk);
       }
       tmem_wait_st();
@@ -369,7 +373,9 @@ __device__ void bwd_act_role(const BwdParams& p, const CUtensorMap* tmDk, const 
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
           const float* f = ((c < 2) ? pp0 : pp1) + (c & 1) * 16 + 2 * e;
-          ds[e] = pack_bf16x2(f[0] * __uint_as_float(dp[2 * e]), f[1] * __uint_as_float(dp[2 * e + 1]));
+          const float ds0 = f[0] * __uint_as_float(dp[2 * e]), ds1 = f[1] * __uint_as_float(dp[2 * e + 1]);
+          if (DBIAS) ds_sum += ds0 + ds1;
+          ds[e] = pack_bf16x2(ds0, ds1);
         }
         // one copy to shared memory (A operand of dQ, MN-major) ...
 #pragma unroll
@@ -386,6 +392,12 @@ __device__ void bwd_act_role(const BwdParams& p, const CUtensorMap* tmDk, const 
       fence_proxy_async_smem();
       mbar_arrive(smem_u32(&bars->ds_ready));
       ++step_cnt;
+    }
+
+    if (DBIAS) {   // sum over the warp, one atomic per warp and item
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) ds_sum += __shfl_xor_sync(0xffffffffu, ds_sum, off);
+      if ((threadIdx.x & 31) == 0) atomicAdd(p.dbias + w.bh, ds_sum);
     }
 
     // epilogue: group 0 stores dV_j (staged in the V tile), group 1 stores scale * dK_j (K tile)
@@ -469,7 +481,7 @@ __device__ void bwd_drain_role(const BwdParams& p, const CUtensorMap* tmW, uint8
 
 // ------------------------------------------------------------------ kernels
 
-template <int D, bool CAUSAL, bool ALIBI>
+template <int D, bool CAUSAL, bool ALIBI, bool DBIAS>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 sigattn_bwd_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                         const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmDo,
@@ -529,7 +541,7 @@ sigattn_bwd_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
     if ((threadIdx.x & 31) == 0) bwd_mma_role<D, CAUSAL>(p, smem_base, tmem, &bars, &cta_err);
     __syncwarp();
   } else if (warp < 8) {
-    bwd_act_role<D, CAUSAL, ALIBI>(p, &tmDk, &tmDv, warp >> 2, smem, tmem, &bars, &cta_err);
+    bwd_act_role<D, CAUSAL, ALIBI, DBIAS>(p, &tmDk, &tmDv, warp >> 2, smem, tmem, &bars, &cta_err);
   } else {
     bwd_drain_role<D, CAUSAL>(p, &tmW, smem, tmem, &bars, &cta_err);
   }
@@ -556,10 +568,10 @@ sigattn_bwd_convert_dq_kernel(const float4* __restrict__ ws, uint2* __restrict__
   }
 }
 
-template <int D, bool CAUSAL, bool ALIBI>
+template <int D, bool CAUSAL, bool ALIBI, bool DBIAS>
 int launch_bwd_variant(const CUtensorMap* maps, const BwdParams& bp, int num_sms, cudaStream_t stream,
                        cudaError_t* cuda_err) {
-  auto kernel = sigattn_bwd_bf16_kernel<D, CAUSAL, ALIBI>;
+  auto kernel = sigattn_bwd_bf16_kernel<D, CAUSAL, ALIBI, DBIAS>;
   static bool configured = false;
   if (!configured) {
     *cuda_err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<D>::kDynBytes);
@@ -620,20 +632,30 @@ int launch_bwd_bf16(const void* q, const void* k, const void* v, const void* d_o
   bp.scale = p.scale;
   bp.scale_log2e = p.scale * kLog2eB;
   bp.bias_log2e = p.bias * kLog2eB;
+  bp.bias_vec = p.bias_vec;
+  bp.dbias = p.dbias;
   bp.slopes = p.slopes;
   bp.status = status;
 
   const size_t n_elems = static_cast<size_t>(BH) * p.N * p.D;
-  // step 1: clear the fp32 dQ accumulator
+  // step 1: clear the fp32 dQ accumulator (and the bias gradient, which the kernel adds into)
   *cuda_err = cudaMemsetAsync(workspace, 0, n_elems * sizeof(float), stream);
   if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
+  if (p.dbias != nullptr) {
+    *cuda_err = cudaMemsetAsync(p.dbias, 0, BH * sizeof(float), stream);
+    if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
+  }
 
   // step 2: main kernel
   const bool timed = (t_ev_start != nullptr && t_ev_stop != nullptr);
   if (timed) cudaEventRecord(t_ev_start, stream);
   int rc;
   const bool alibi = p.slopes != nullptr;
-#define SIGATTN_BWD_CASE(DD, CC, AA) rc = launch_bwd_variant<DD, CC, AA>(maps, bp, num_sms, stream, cuda_err)
+  // the bias gradient costs the activation groups a running sum (4-5 % of the kernel), so it
+  // is compiled in only where it is asked for
+#define SIGATTN_BWD_CASE(DD, CC, AA)                                                          \
+  rc = (p.dbias != nullptr) ? launch_bwd_variant<DD, CC, AA, true>(maps, bp, num_sms, stream, cuda_err) \
+                            : launch_bwd_variant<DD, CC, AA, false>(maps, bp, num_sms, stream, cuda_err)
   if (p.D == 128) {
     if (p.causal) { if (alibi) SIGATTN_BWD_CASE(128, true, true); else SIGATTN_BWD_CASE(128, true, false); }
     else          { if (alibi) SIGATTN_BWD_CASE(128, false, true); else SIGATTN_BWD_CASE(128, false, false); }

@@ -1,7 +1,8 @@
 // float32 debug path on CUDA cores: the definition evaluated with exact expf and a
 // true division, fp32 FMA accumulation, no tensor cores (TF32 would cost 1e-3 of
 // accuracy).  One thread block per query row (forward, dQ) or per key row (dK, dV);
-// nothing is shared between blocks, so every output is deterministic.
+// nothing is shared between blocks, so every tensor output is deterministic (the optional
+// bias gradient is a sum over all blocks of a head and is added with fp32 atomics).
 //
 // Forward: Eq. 3 / Algorithm 1.  Backward: the sigmoid column of the forward/backward
 // table in Appendix F.1 / Algorithm 2, with the factor scale = 1/sqrt(d) in dQ and dK.
@@ -28,10 +29,12 @@ __device__ __forceinline__ float dot_row(const float* __restrict__ a_smem, const
 // grid (N, B*H); block 128.  Thread t handles key j0 + t, then output column t.
 __global__ void fwd_fp32_kernel(const float* __restrict__ q, const float* __restrict__ k,
                                 const float* __restrict__ v, float* __restrict__ o, int H, int N, int D,
-                                float scale, float bias, int causal, const float* __restrict__ slopes) {
+                                float scale, float bias, int causal, const float* __restrict__ slopes,
+                                const float* __restrict__ bias_vec) {
   __shared__ float sq[128];
   __shared__ float sp[kThreads];
   const int i = blockIdx.x, bh = blockIdx.y, t = threadIdx.x;
+  if (bias_vec) bias = bias_vec[bh];
   const size_t base = static_cast<size_t>(bh) * N * D;
   const float slope = slopes ? slopes[bh % H] : 0.0f;
   if (t < D) sq[t] = q[base + static_cast<size_t>(i) * D + t];
@@ -61,11 +64,14 @@ __global__ void fwd_fp32_kernel(const float* __restrict__ q, const float* __rest
 __global__ void bwd_dq_fp32_kernel(const float* __restrict__ q, const float* __restrict__ k,
                                    const float* __restrict__ v, const float* __restrict__ d_o,
                                    float* __restrict__ dq, int H, int N, int D, float scale, float bias,
-                                   int causal, const float* __restrict__ slopes) {
+                                   int causal, const float* __restrict__ slopes,
+                                   const float* __restrict__ bias_vec, float* __restrict__ dbias) {
   __shared__ float sq[128];
   __shared__ float sdo[128];
   __shared__ float sds[kThreads];
   const int i = blockIdx.x, bh = blockIdx.y, t = threadIdx.x;
+  if (bias_vec) bias = bias_vec[bh];
+  float ds_sum = 0.0f;   // this thread's share of sum_j dS_ij
   const size_t base = static_cast<size_t>(bh) * N * D;
   const float slope = slopes ? slopes[bh % H] : 0.0f;
   if (t < D) {
@@ -85,6 +91,7 @@ __global__ void bwd_dq_fp32_kernel(const float* __restrict__ q, const float* __r
       ds = sigmoid_slope(x) * dp;
     }
     sds[t] = ds;
+    ds_sum += ds;
     __syncthreads();
     if (t < D) {
       const int cnt = min(kThreads, jend - j0);
@@ -93,18 +100,29 @@ __global__ void bwd_dq_fp32_kernel(const float* __restrict__ q, const float* __r
     __syncthreads();
   }
   if (t < D) dq[base + static_cast<size_t>(i) * D + t] = scale * acc;
+  if (dbias) {   // d(bias) of this head: sum of dS over the row, then over the rows (atomics)
+    sds[t] = ds_sum;
+    __syncthreads();
+    for (int half = kThreads / 2; half > 0; half >>= 1) {
+      if (t < half) sds[t] += sds[t + half];
+      __syncthreads();
+    }
+    if (t == 0) atomicAdd(dbias + bh, sds[0]);
+  }
 }
 
 // dV_j = sum_i P_ij dO_i ; dK_j = scale * sum_i dS_ij Q_i.  grid (N, B*H), one key row each.
 __global__ void bwd_dkdv_fp32_kernel(const float* __restrict__ q, const float* __restrict__ k,
                                      const float* __restrict__ v, const float* __restrict__ d_o,
                                      float* __restrict__ dk, float* __restrict__ dv, int H, int N, int D,
-                                     float scale, float bias, int causal, const float* __restrict__ slopes) {
+                                     float scale, float bias, int causal, const float* __restrict__ slopes,
+                                     const float* __restrict__ bias_vec) {
   __shared__ float sk[128];
   __shared__ float sv[128];
   __shared__ float sp[kThreads];
   __shared__ float sds[kThreads];
   const int j = blockIdx.x, bh = blockIdx.y, t = threadIdx.x;
+  if (bias_vec) bias = bias_vec[bh];
   const size_t base = static_cast<size_t>(bh) * N * D;
   const float slope = slopes ? slopes[bh % H] : 0.0f;
   if (t < D) {
@@ -148,7 +166,8 @@ __global__ void bwd_dkdv_fp32_kernel(const float* __restrict__ q, const float* _
 int launch_fwd_fp32(const float* q, const float* k, const float* v, float* o, const Problem& p,
                     cudaStream_t stream, unsigned long long* launches, cudaError_t* cuda_err) {
   dim3 grid(p.N, p.B * p.H);
-  fwd_fp32_kernel<<<grid, kThreads, 0, stream>>>(q, k, v, o, p.H, p.N, p.D, p.scale, p.bias, p.causal, p.slopes);
+  fwd_fp32_kernel<<<grid, kThreads, 0, stream>>>(q, k, v, o, p.H, p.N, p.D, p.scale, p.bias, p.causal, p.slopes,
+                                                 p.bias_vec);
   *launches += 1;
   *cuda_err = cudaGetLastError();
   return *cuda_err == cudaSuccess ? SIGATTN_OK : SIGATTN_ERR_CUDA;
@@ -158,10 +177,14 @@ int launch_bwd_fp32(const float* q, const float* k, const float* v, const float*
                     float* dv, const Problem& p, cudaStream_t stream, unsigned long long* launches,
                     cudaError_t* cuda_err) {
   dim3 grid(p.N, p.B * p.H);
+  if (p.dbias) {
+    *cuda_err = cudaMemsetAsync(p.dbias, 0, static_cast<size_t>(p.B) * p.H * sizeof(float), stream);
+    if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
+  }
   bwd_dq_fp32_kernel<<<grid, kThreads, 0, stream>>>(q, k, v, d_o, dq, p.H, p.N, p.D, p.scale, p.bias, p.causal,
-                                                    p.slopes);
+                                                    p.slopes, p.bias_vec, p.dbias);
   bwd_dkdv_fp32_kernel<<<grid, kThreads, 0, stream>>>(q, k, v, d_o, dk, dv, p.H, p.N, p.D, p.scale, p.bias,
-                                                      p.causal, p.slopes);
+                                                      p.causal, p.slopes, p.bias_vec);
   *launches += 2;
   *cuda_err = cudaGetLastError();
   return *cuda_err == cudaSuccess ? SIGATTN_OK : SIGATTN_ERR_CUDA;

@@ -87,6 +87,7 @@ struct FwdParams {
   int n_kv_total;  // ceil(N / 128)
   int n_items;
   float scale_log2e, bias_log2e;
+  const float* bias_vec;   // one bias per (batch, head) instead of the scalar, or nullptr
   const float* slopes;
   int* status;
 };
@@ -343,6 +344,7 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
     const Item w = decode_item<CAUSAL>(p, item);
     float slope_log2e = 0.0f;
     if (ALIBI) slope_log2e = p.slopes[w.bh % p.H] * kLog2e;
+    const float bias_log2e = p.bias_vec ? __ldg(p.bias_vec + w.bh) * kLog2e : p.bias_log2e;
 
     // Tile-steps are visited in the order (j, tile 0), (j, tile 1), (j + 1, tile 0), ...
     for (int j = 0; j < w.n_kv; ++j) {
@@ -362,7 +364,7 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
         tmem_wait_ld();
         uint32_t pk[kCols / 2];
         constexpr int kEmulateEvery = (D == 128) ? SIGATTN_FWD_EMULATE_D128 : SIGATTN_FWD_EMULATE_D64;
-        sigmoid_cols<ALIBI, kEmulateEvery>(sv, pk, p.scale_log2e, p.bias_log2e, slope_log2e, row_rel, g * kCols,
+        sigmoid_cols<ALIBI, kEmulateEvery>(sv, pk, p.scale_log2e, bias_log2e, slope_log2e, row_rel, g * kCols,
                                            diag);
         tmem_st_cols(tS, pk);
         tmem_wait_st();
@@ -529,6 +531,7 @@ int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const 
   fp.n_items = fp.n_pairs * fp.BH;
   fp.scale_log2e = p.scale * kLog2e;
   fp.bias_log2e = p.bias * kLog2e;
+  fp.bias_vec = p.bias_vec;
   fp.slopes = p.slopes;
   fp.status = status;
 

@@ -11,7 +11,9 @@ struct Problem {
   int B, H, N, D;
   float scale, bias;
   int causal;
-  const float* slopes;  // device pointer to H floats, or nullptr
+  const float* slopes;    // device pointer to H floats, or nullptr
+  const float* bias_vec;  // device pointer to B*H biases that replace `bias`, or nullptr
+  float* dbias;           // backward only: device pointer to B*H floats that receive sum dS, or nullptr
 };
 
 // Every launcher enqueues on `stream`, adds the number of kernels it launched to
