@@ -40,6 +40,12 @@ Readings of the paper taken here
     a scalar or anything that broadcasts to [B, H]; it enters x_ij additively, so its
     gradient is db[b, h] = sum_ij dS_ij (the chain rule through x = u + b; masked entries
     carry dS = 0).  The paper prints no formula for db.
+  * Keys and values may have fewer heads than the queries (multi-query and grouped-query
+    attention; the ablation of Section 5.1 uses multi-query attention): k, v are
+    [B, H_kv, N, D] with H a multiple of H_kv, query head h reads key/value head
+    h // (H / H_kv) (consecutive query heads share one), and dK, dV of a key/value head
+    are the sums over the query heads that read it.  The paper gives no layout; this is
+    the usual one.
 
 Every function is pinned by tests that do not call back into this file's own
 formulae (closed forms, brute-force loops, finite differences, the paper's second
@@ -129,6 +135,14 @@ def _bias_per_head(bias, num_batch, num_heads):
     return np.ascontiguousarray(np.broadcast_to(b, (num_batch, num_heads)))
 
 
+def _kv_group(num_heads, k):
+    """Query heads per key/value head."""
+    h_kv = k.shape[1]
+    if h_kv < 1 or num_heads % h_kv != 0:
+        raise ValueError("the number of query heads must be a multiple of the number of key/value heads")
+    return num_heads // h_kv
+
+
 def _row_ranges(n, row_block):
     """Query rows are independent in the forward and enter dK, dV only through a sum
     over rows, so they may be visited in slabs to bound memory (an n x n float64 matrix
@@ -140,42 +154,47 @@ def _row_ranges(n, row_block):
 def sigattn_fwd(q, k, v, scale, bias, causal=False, alibi_slopes=None, row_block=None):
     """O = sigmoid(scale * Q K^T + b [+ position bias]) [* causal mask] V  (Eq. 3).
 
-    q, k, v: [B, H, N, D] arrays (any float dtype; converted to float64).
+    q: [B, H, N, D]; k, v: [B, H_kv, N, D] with H a multiple of H_kv (any float dtype;
+    converted to float64).
     bias: scalar, or an array that broadcasts to [B, H] (one bias per sequence and head).
     Returns O as float64 [B, H, N, D].
     """
     q, k, v = _as_f64(q, k, v)
     B, H, N, D = q.shape
+    group = _kv_group(H, k)
     slopes = _slopes(alibi_slopes, H)
     bias_bh = _bias_per_head(bias, B, H)
     o = np.zeros((B, H, N, D), dtype=np.float64)
     for b in range(B):
         for h in range(H):
+            hk = h // group
             for i0, i1 in _row_ranges(N, row_block):
-                p = attention_weights(q[b, h], k[b, h], scale, bias_bh[b, h], causal, slopes[h], i0, i1)
-                o[b, h, i0:i1] = p @ v[b, h]
+                p = attention_weights(q[b, h], k[b, hk], scale, bias_bh[b, h], causal, slopes[h], i0, i1)
+                o[b, h, i0:i1] = p @ v[b, hk]
     return o
 
 
 def _bwd_all(q, k, v, d_o, scale, bias, causal, alibi_slopes, row_block):
     q, k, v, d_o = _as_f64(q, k, v, d_o)
     B, H, N, D = q.shape
+    group = _kv_group(H, k)
     slopes = _slopes(alibi_slopes, H)
     bias_bh = _bias_per_head(bias, B, H)
     dq = np.zeros_like(q)
-    dk = np.zeros_like(q)
-    dv = np.zeros_like(q)
+    dk = np.zeros_like(k)
+    dv = np.zeros_like(v)
     dbias = np.zeros((B, H), dtype=np.float64)
     for b in range(B):
         for h in range(H):
+            hk = h // group
             for i0, i1 in _row_ranges(N, row_block):
-                p = attention_weights(q[b, h], k[b, h], scale, bias_bh[b, h], causal, slopes[h], i0, i1)
+                p = attention_weights(q[b, h], k[b, hk], scale, bias_bh[b, h], causal, slopes[h], i0, i1)
                 do_rows = d_o[b, h, i0:i1]
-                dv[b, h] += p.T @ do_rows
-                dp = do_rows @ v[b, h].T
+                dv[b, hk] += p.T @ do_rows
+                dp = do_rows @ v[b, hk].T
                 ds = p * (1.0 - p) * dp
-                dq[b, h, i0:i1] = scale * (ds @ k[b, h])
-                dk[b, h] += scale * (ds.T @ q[b, h, i0:i1])
+                dq[b, h, i0:i1] = scale * (ds @ k[b, hk])
+                dk[b, hk] += scale * (ds.T @ q[b, h, i0:i1])
                 dbias[b, h] += ds.sum()
     return dq, dk, dv, dbias
 
@@ -184,8 +203,9 @@ def sigattn_bwd(q, k, v, d_o, scale, bias, causal=False, alibi_slopes=None, row_
     """Gradients of L = sum(O * dO) with respect to Q, K, V (sigmoid column of the
     forward/backward table in Appendix F.1, with the 1/sqrt(d) factor; see header).
 
-    bias: scalar, or an array that broadcasts to [B, H].
-    Returns (dQ, dK, dV), float64 [B, H, N, D] each.
+    bias: scalar, or an array that broadcasts to [B, H].  k, v may have fewer heads
+    than q (see header).
+    Returns (dQ, dK, dV), float64, shaped like q, k, v.
     """
     return _bwd_all(q, k, v, d_o, scale, bias, causal, alibi_slopes, row_block)[:3]
 

@@ -383,3 +383,38 @@ def test_bias_gradient_single_token_closed_form_and_brute_force():
                 pp = scalar_sigmoid(x)
                 ref[0, h] += pp * (1 - pp) * float(d_o[0, h, i] @ v[0, h, j])
     np.testing.assert_allclose(oracle.sigattn_bwd_dbias(q, k, v, d_o, 0.7, bias, True, slopes), ref, rtol=1e-13)
+
+
+# ------------------------------------------------------------- fewer key/value heads than query heads
+
+
+@pytest.mark.parametrize("h_kv", [1, 2])
+def test_grouped_kv_heads_forward_and_backward(h_kv):
+    """k, v with H_kv heads: the forward must equal the element-by-element definition on
+    keys/values repeated per query head, the gradients must match central differences of
+    L = sum(O * dO) taken on the SHARED k, v (so sums over the group are checked too)."""
+    B, H, N, D = 1, 4, 5, 3
+    G = H // h_kv
+    q, d_o = rnd((B, H, N, D), 90), rnd((B, H, N, D), 91)
+    k, v = rnd((B, h_kv, N, D), 92), rnd((B, h_kv, N, D), 93)
+    slopes = np.array([0.5, 0.25, 0.125, 0.0625])
+    scale, b = 0.6, -1.1
+    o = oracle.sigattn_fwd(q, k, v, scale, b, True, slopes)
+    np.testing.assert_allclose(o, brute_forward(q, np.repeat(k, G, axis=1), np.repeat(v, G, axis=1), scale, b, True, slopes),
+                               rtol=1e-13, atol=1e-15)
+    dq, dk, dv = oracle.sigattn_bwd(q, k, v, d_o, scale, b, True, slopes)
+    assert dk.shape == k.shape and dv.shape == v.shape
+    h = 1e-6
+    for name, x, g in (("q", q, dq), ("k", k, dk), ("v", v, dv)):
+        fd = np.zeros_like(x)
+        for idx in np.ndindex(*x.shape):
+            old = x[idx]
+            x[idx] = old + h
+            lp = loss(q, k, v, d_o, scale, b, True, slopes)
+            x[idx] = old - h
+            lm = loss(q, k, v, d_o, scale, b, True, slopes)
+            x[idx] = old
+            fd[idx] = (lp - lm) / (2 * h)
+        assert np.linalg.norm(fd - g) / np.linalg.norm(fd) < 1e-7, name
+    with pytest.raises(ValueError):
+        oracle.sigattn_fwd(q, rnd((B, 3, N, D), 94), rnd((B, 3, N, D), 95), scale, b)
