@@ -147,6 +147,31 @@ SIGATTN_API int sigattn_bwd_bias_vec(const void* q, const void* k, const void* v
                          float* dbias_bh,
                          void* workspace, size_t workspace_bytes, void* stream);
 
+/* Multi-query / grouped-query attention (the multi-query ablation of Section 5.1): k and v
+ * (and dk, dv) have H_kv heads, [B, H_kv, N, D], with H a multiple of H_kv; query head h
+ * reads key/value head h / (H / H_kv), i.e. consecutive query heads share one.  The paper
+ * gives no layout; this is the usual one.  q, o, d_o, dq stay [B, H, N, D].  `bias_bh` is
+ * NULL (the scalar `bias` is used) or a DEVICE pointer to B*H floats as in
+ * sigattn_fwd_bias_vec (then `bias` is ignored); slopes are per query head.  H_kv == H is
+ * plain multi-head attention.  H % H_kv != 0 or H_kv < 1: SIGATTN_ERR_SHAPE. */
+SIGATTN_API int sigattn_fwd_gqa(const void* q, const void* k, const void* v, void* o,
+                    int B, int H, int H_kv, int N, int D,
+                    float scale, float bias, const float* bias_bh, int causal,
+                    const float* alibi_slopes, int dtype, void* stream);
+
+/* Backward of sigattn_fwd_gqa: dk, dv are [B, H_kv, N, D] and hold the sums over the query
+ * heads that read each key/value head (accumulated on chip: a work item keeps dK_j, dV_j
+ * of one key/value head in tensor memory while it walks the query tiles of all its query
+ * heads).  `dbias_bh`: NULL or B*H floats as in sigattn_bwd_bias_vec.  The workspace is
+ * that of sigattn_bwd for (B, H, N, D). */
+SIGATTN_API int sigattn_bwd_gqa(const void* q, const void* k, const void* v, const void* d_o,
+                    void* dq, void* dk, void* dv,
+                    int B, int H, int H_kv, int N, int D,
+                    float scale, float bias, const float* bias_bh, int causal,
+                    const float* alibi_slopes, int dtype,
+                    float* dbias_bh,
+                    void* workspace, size_t workspace_bytes, void* stream);
+
 /* Bytes of scratch sigattn_bwd needs for this problem (0 for the fp32 debug path).
  * Returns 0 for invalid shapes as well; sigattn_bwd reports those. */
 SIGATTN_API size_t sigattn_bwd_workspace_bytes(int B, int H, int N, int D, int dtype);

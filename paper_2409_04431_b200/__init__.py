@@ -27,6 +27,8 @@ _BINDING_NAMES = (
     "sigattn_selftest_bounded_wait",
     "sigattn_fwd_bias_vec",
     "sigattn_bwd_bias_vec",
+    "sigattn_fwd_gqa",
+    "sigattn_bwd_gqa",
     "lib",
 )
 

@@ -87,10 +87,11 @@ void account(unsigned long long launches, int rc, cudaError_t cuda_err) {
 namespace {
 
 // Shared by the scalar-bias and the bias-vector entry points.
-int fwd_any(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int D, float scale, float bias,
-            const float* bias_vec, int causal, const float* alibi_slopes, int dtype, void* stream) {
+int fwd_any(const void* q, const void* k, const void* v, void* o, int B, int H, int H_kv, int N, int D, float scale,
+            float bias, const float* bias_vec, int causal, const float* alibi_slopes, int dtype, void* stream) {
   if (!q || !k || !v || !o) return SIGATTN_ERR_NULL;
   if (int rc = check_shape(B, H, N, D)) return rc;
+  if (H_kv < 1 || H % H_kv != 0) return SIGATTN_ERR_SHAPE;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return SIGATTN_ERR_ALIGN;
   if (alibi_slopes && (reinterpret_cast<uintptr_t>(alibi_slopes) & 3u)) return SIGATTN_ERR_ALIGN;
   if (dtype != SIGATTN_DTYPE_BF16 && dtype != SIGATTN_DTYPE_FP32) return SIGATTN_ERR_FLAG;
@@ -98,7 +99,7 @@ int fwd_any(const void* q, const void* k, const void* v, void* o, int B, int H, 
   int dev = 0;
   int* status = nullptr;
   if (int rc = device_setup(&dev, &status)) return rc;
-  sigattn::Problem p{B, H, N, D, scale, bias, causal, alibi_slopes, bias_vec, nullptr};
+  sigattn::Problem p{B, H, N, D, scale, bias, causal, alibi_slopes, bias_vec, nullptr, H_kv};
   unsigned long long launches = 0;
   cudaError_t ce = cudaSuccess;
   int rc;
@@ -115,10 +116,11 @@ int fwd_any(const void* q, const void* k, const void* v, void* o, int B, int H, 
 }
 
 int bwd_any(const void* q, const void* k, const void* v, const void* d_o, void* dq, void* dk, void* dv, int B, int H,
-            int N, int D, float scale, float bias, const float* bias_vec, float* dbias, int causal,
+            int H_kv, int N, int D, float scale, float bias, const float* bias_vec, float* dbias, int causal,
             const float* alibi_slopes, int dtype, void* workspace, size_t workspace_bytes, void* stream) {
   if (!q || !k || !v || !d_o || !dq || !dk || !dv) return SIGATTN_ERR_NULL;
   if (int rc = check_shape(B, H, N, D)) return rc;
+  if (H_kv < 1 || H % H_kv != 0) return SIGATTN_ERR_SHAPE;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(d_o) || !aligned16(dq) || !aligned16(dk) ||
       !aligned16(dv))
     return SIGATTN_ERR_ALIGN;
@@ -134,7 +136,7 @@ int bwd_any(const void* q, const void* k, const void* v, const void* d_o, void* 
   int dev = 0;
   int* status = nullptr;
   if (int rc = device_setup(&dev, &status)) return rc;
-  sigattn::Problem p{B, H, N, D, scale, bias, causal, alibi_slopes, bias_vec, dbias};
+  sigattn::Problem p{B, H, N, D, scale, bias, causal, alibi_slopes, bias_vec, dbias, H_kv};
   unsigned long long launches = 0;
   cudaError_t ce = cudaSuccess;
   int rc;
@@ -158,7 +160,7 @@ extern "C" {
 
 int sigattn_fwd(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int D, float scale,
                 float bias, int causal, const float* alibi_slopes, int dtype, void* stream) {
-  return fwd_any(q, k, v, o, B, H, N, D, scale, bias, nullptr, causal, alibi_slopes, dtype, stream);
+  return fwd_any(q, k, v, o, B, H, H, N, D, scale, bias, nullptr, causal, alibi_slopes, dtype, stream);
 }
 
 int sigattn_fwd_bias_vec(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int D,
@@ -166,13 +168,20 @@ int sigattn_fwd_bias_vec(const void* q, const void* k, const void* v, void* o, i
                          void* stream) {
   if (!bias_bh) return SIGATTN_ERR_NULL;
   if (reinterpret_cast<uintptr_t>(bias_bh) & 3u) return SIGATTN_ERR_ALIGN;
-  return fwd_any(q, k, v, o, B, H, N, D, scale, 0.0f, bias_bh, causal, alibi_slopes, dtype, stream);
+  return fwd_any(q, k, v, o, B, H, H, N, D, scale, 0.0f, bias_bh, causal, alibi_slopes, dtype, stream);
+}
+
+int sigattn_fwd_gqa(const void* q, const void* k, const void* v, void* o, int B, int H, int H_kv, int N, int D,
+                    float scale, float bias, const float* bias_bh, int causal, const float* alibi_slopes, int dtype,
+                    void* stream) {
+  if (bias_bh && (reinterpret_cast<uintptr_t>(bias_bh) & 3u)) return SIGATTN_ERR_ALIGN;
+  return fwd_any(q, k, v, o, B, H, H_kv, N, D, scale, bias, bias_bh, causal, alibi_slopes, dtype, stream);
 }
 
 int sigattn_bwd(const void* q, const void* k, const void* v, const void* d_o, void* dq, void* dk, void* dv, int B,
                 int H, int N, int D, float scale, float bias, int causal, const float* alibi_slopes, int dtype,
                 void* workspace, size_t workspace_bytes, void* stream) {
-  return bwd_any(q, k, v, d_o, dq, dk, dv, B, H, N, D, scale, bias, nullptr, nullptr, causal, alibi_slopes, dtype,
+  return bwd_any(q, k, v, d_o, dq, dk, dv, B, H, H, N, D, scale, bias, nullptr, nullptr, causal, alibi_slopes, dtype,
                  workspace, workspace_bytes, stream);
 }
 
@@ -183,8 +192,18 @@ int sigattn_bwd_bias_vec(const void* q, const void* k, const void* v, const void
   if (!bias_bh) return SIGATTN_ERR_NULL;
   if ((reinterpret_cast<uintptr_t>(bias_bh) & 3u) || (reinterpret_cast<uintptr_t>(dbias_bh) & 3u))
     return SIGATTN_ERR_ALIGN;
-  return bwd_any(q, k, v, d_o, dq, dk, dv, B, H, N, D, scale, 0.0f, bias_bh, dbias_bh, causal, alibi_slopes, dtype,
-                 workspace, workspace_bytes, stream);
+  return bwd_any(q, k, v, d_o, dq, dk, dv, B, H, H, N, D, scale, 0.0f, bias_bh, dbias_bh, causal, alibi_slopes,
+                 dtype, workspace, workspace_bytes, stream);
+}
+
+int sigattn_bwd_gqa(const void* q, const void* k, const void* v, const void* d_o, void* dq, void* dk, void* dv, int B,
+                    int H, int H_kv, int N, int D, float scale, float bias, const float* bias_bh, int causal,
+                    const float* alibi_slopes, int dtype, float* dbias_bh, void* workspace, size_t workspace_bytes,
+                    void* stream) {
+  if ((reinterpret_cast<uintptr_t>(bias_bh) & 3u) || (reinterpret_cast<uintptr_t>(dbias_bh) & 3u))
+    return SIGATTN_ERR_ALIGN;
+  return bwd_any(q, k, v, d_o, dq, dk, dv, B, H, H_kv, N, D, scale, bias, bias_bh, dbias_bh, causal, alibi_slopes,
+                 dtype, workspace, workspace_bytes, stream);
 }
 
 int sigattn_bwd_set_timing_events(void* start_event, void* stop_event) {

@@ -67,7 +67,8 @@ struct BwdBarriers {
 };
 
 struct BwdParams {
-  int BH, H, N;
+  int BH, H, N;    // BH counts (batch, key/value head) pairs: the work items are per key/value head
+  int H_kv, group; // heads of K, V and query heads per key/value head (H = H_kv * group)
   int n_tiles;  // ceil(N / 128), for keys and for queries
   int n_items;
   float scale, scale_log2e, bias_log2e;
@@ -78,7 +79,11 @@ struct BwdParams {
 };
 
 struct BwdItem {
-  int bh, j, i_begin, n;
+  int bh;       // (batch, key/value head) index: K_j, V_j, dK_j, dV_j
+  int bh_q0;    // first of the `group` query heads that read this key/value head
+  int j, i_begin;
+  int n;        // query tiles per query head
+  int steps;    // group * n, visited head by head
 };
 
 // Ranks are ordered by decreasing cost; rounds alternate direction over the CTAs so that
@@ -92,13 +97,17 @@ __device__ __forceinline__ int bwd_snake_rank(int round, int n_items) {
 
 __device__ __forceinline__ int bwd_num_rounds(int n_items) { return (n_items + gridDim.x - 1) / gridDim.x; }
 
-template <bool CAUSAL>
+// GROUPED = false compiles the one-head-per-group case (plain multi-head attention) without
+// the head loop; it is the benchmarked path.
+template <bool CAUSAL, bool GROUPED>
 __device__ __forceinline__ BwdItem decode_bwd_item(const BwdParams& p, int item) {
   BwdItem w;
   w.j = item / p.BH;  // ascending key tile = descending work when causal
   w.bh = item - w.j * p.BH;
+  w.bh_q0 = GROUPED ? (w.bh / p.H_kv) * p.H + (w.bh % p.H_kv) * p.group : w.bh;
   w.i_begin = CAUSAL ? w.j : 0;
   w.n = p.n_tiles - w.i_begin;
+  w.steps = GROUPED ? p.group * w.n : w.n;
   return w;
 }
 
@@ -113,7 +122,7 @@ struct BwdTmem {
 
 // ------------------------------------------------------------------ producer
 
-template <int D, bool CAUSAL>
+template <int D, bool CAUSAL, bool GROUPED>
 __device__ void bwd_load_role(const BwdParams& p, const CUtensorMap* tmQ, const CUtensorMap* tmK,
                               const CUtensorMap* tmV, const CUtensorMap* tmDo, uint32_t smem_base,
                               BwdBarriers* bars, volatile int* cta_err) {
@@ -143,9 +152,9 @@ __device__ void bwd_load_role(const BwdParams& p, const CUtensorMap* tmQ, const 
   for (int round = 0, rounds = bwd_num_rounds(p.n_items); round < rounds; ++round) {
     const int item = bwd_snake_rank(round, p.n_items);
     if (item < 0) continue;
-    const BwdItem w = decode_bwd_item<CAUSAL>(p, item);
-    if (!load_q(w.i_begin, w.bh)) return;
-    if (!load_do(w.i_begin, w.bh)) return;
+    const BwdItem w = decode_bwd_item<CAUSAL, GROUPED>(p, item);
+    if (!load_q(w.i_begin, w.bh_q0)) return;
+    if (!load_do(w.i_begin, w.bh_q0)) return;
     if (!mbar_wait(smem_u32(&bars->kv_empty), (item_cnt & 1) ^ 1, cta_err, 42)) return;
     {
       const uint32_t bar = smem_u32(&bars->kv_full);
@@ -154,16 +163,18 @@ __device__ void bwd_load_role(const BwdParams& p, const CUtensorMap* tmQ, const 
       load_tile(tmV, smem_base + L::kVOff, bar, w.j * kT, w.bh);
     }
     ++item_cnt;
-    for (int it = 1; it < w.n; ++it) {
-      if (!load_q(w.i_begin + it, w.bh)) return;
-      if (!load_do(w.i_begin + it, w.bh)) return;
+    for (int g = 0; g < (GROUPED ? p.group : 1); ++g) {
+      for (int it = (g == 0 ? 1 : 0); it < w.n; ++it) {
+        if (!load_q(w.i_begin + it, w.bh_q0 + g)) return;
+        if (!load_do(w.i_begin + it, w.bh_q0 + g)) return;
+      }
     }
   }
 }
 
 // ------------------------------------------------------------------ MMA issuer
 
-template <int D, bool CAUSAL>
+template <int D, bool CAUSAL, bool GROUPED>
 __device__ void bwd_mma_role(const BwdParams& p, uint32_t smem_base, uint32_t tmem, BwdBarriers* bars,
                              volatile int* cta_err) {
   using L = BwdSmem<D>;
@@ -198,7 +209,7 @@ __device__ void bwd_mma_role(const BwdParams& p, uint32_t smem_base, uint32_t tm
   for (int round = 0, rounds = bwd_num_rounds(p.n_items); round < rounds; ++round) {
     const int item = bwd_snake_rank(round, p.n_items);
     if (item < 0) continue;
-    const BwdItem w = decode_bwd_item<CAUSAL>(p, item);
+    const BwdItem w = decode_bwd_item<CAUSAL, GROUPED>(p, item);
     if (!mbar_wait(smem_u32(&bars->kv_full), item_cnt & 1, cta_err, 50)) return;
 
     // prologue: S^T(0), dP^T(0)
@@ -214,9 +225,9 @@ __device__ void bwd_mma_role(const BwdParams& p, uint32_t smem_base, uint32_t tm
       issue_kk(TM::kB, dV_k, dDo_k);
       umma_commit(smem_u32(&bars->dp_full));
     }
-    for (int it = 0; it < w.n; ++it) {
+    for (int it = 0; it < w.steps; ++it) {
       const uint32_t st = q_cnt & 1;
-      const bool more = (it + 1 < w.n);
+      const bool more = (it + 1 < w.steps);
       // dV += P^T dO_i
       if (!mbar_wait(smem_u32(&bars->p_ready), step_cnt & 1, cta_err, 54)) return;
       if (it == 0 && !mbar_wait(smem_u32(&bars->dkv_empty), (item_cnt & 1) ^ 1, cta_err, 55)) return;
@@ -318,7 +329,7 @@ __device__ __forceinline__ void bwd_store_acc_rows(uint32_t t_acc, uint8_t* stag
   }
 }
 
-template <int D, bool CAUSAL, bool ALIBI, bool DBIAS>
+template <int D, bool CAUSAL, bool ALIBI, bool DBIAS, bool GROUPED>
 __device__ void bwd_act_role(const BwdParams& p, const CUtensorMap* tmDk, const CUtensorMap* tmDv, int wg,
                              uint8_t* smem, uint32_t tmem, BwdBarriers* bars, volatile int* cta_err) {
   using L = BwdSmem<D>;
@@ -330,11 +341,13 @@ __device__ void bwd_act_role(const BwdParams& p, const CUtensorMap* tmDk, const 
   for (int round = 0, rounds = bwd_num_rounds(p.n_items); round < rounds; ++round) {
     const int item = bwd_snake_rank(round, p.n_items);
     if (item < 0) continue;
-    const BwdItem w = decode_bwd_item<CAUSAL>(p, item);
+    const BwdItem w = decode_bwd_item<CAUSAL, GROUPED>(p, item);
+    for (int g = 0; g < (GROUPED ? p.group : 1); ++g) {   // the query heads that read this key/value head
+    const int bh_q = w.bh_q0 + g;
     float slope_log2e = 0.0f;
-    if (ALIBI) slope_log2e = p.slopes[w.bh % p.H] * kLog2eB;
-    const float bias_log2e = p.bias_vec ? __ldg(p.bias_vec + w.bh) * kLog2eB : p.bias_log2e;
-    float ds_sum = 0.0f;   // this thread's share of sum dS over the item (the bias gradient)
+    if (ALIBI) slope_log2e = p.slopes[bh_q % p.H] * kLog2eB;
+    const float bias_log2e = p.bias_vec ? __ldg(p.bias_vec + bh_q) * kLog2eB : p.bias_log2e;
+    float ds_sum = 0.0f;   // this thread's share of sum dS over the head's tiles (the bias gradient)
 
     for (int it = 0; it < w.n; ++it) {
       const int i = w.i_begin + it;
@@ -394,11 +407,12 @@ __device__ void bwd_act_role(const BwdParams& p, const CUtensorMap* tmDk, const 
       ++step_cnt;
     }
 
-    if (DBIAS) {   // sum over the warp, one atomic per warp and item
+    if (DBIAS) {   // sum over the warp, one atomic per warp, item and query head
 #pragma unroll
       for (int off = 16; off > 0; off >>= 1) ds_sum += __shfl_xor_sync(0xffffffffu, ds_sum, off);
-      if ((threadIdx.x & 31) == 0) atomicAdd(p.dbias + w.bh, ds_sum);
+      if ((threadIdx.x & 31) == 0) atomicAdd(p.dbias + bh_q, ds_sum);
     }
+    }   // query heads
 
     // epilogue: group 0 stores dV_j (staged in the V tile), group 1 stores scale * dK_j (K tile)
     if (!mbar_wait(smem_u32(&bars->dkv_full), item_cnt & 1, cta_err, 64 + wg)) return;
@@ -425,7 +439,7 @@ __device__ void bwd_act_role(const BwdParams& p, const CUtensorMap* tmDk, const 
 
 // ------------------------------------------------------------------ dQ drain group
 
-template <int D, bool CAUSAL>
+template <int D, bool CAUSAL, bool GROUPED>
 __device__ void bwd_drain_role(const BwdParams& p, const CUtensorMap* tmW, uint8_t* smem, uint32_t tmem,
                                BwdBarriers* bars, volatile int* cta_err) {
   using L = BwdSmem<D>;
@@ -436,9 +450,10 @@ __device__ void bwd_drain_role(const BwdParams& p, const CUtensorMap* tmW, uint8
   for (int round = 0, rounds = bwd_num_rounds(p.n_items); round < rounds; ++round) {
     const int item = bwd_snake_rank(round, p.n_items);
     if (item < 0) continue;
-    const BwdItem w = decode_bwd_item<CAUSAL>(p, item);
-    for (int it = 0; it < w.n; ++it) {
-      const int row0 = (w.i_begin + it) * kT;
+    const BwdItem w = decode_bwd_item<CAUSAL, GROUPED>(p, item);
+    for (int s = 0; s < w.steps; ++s) {
+      const int g = GROUPED ? s / w.n : 0, it = s - g * w.n;   // query head within the group, query tile
+      const int row0 = (w.i_begin + it) * kT, bh_q = w.bh_q0 + g;
       if (!mbar_wait(smem_u32(&bars->dq_full), step_cnt & 1, cta_err, 70)) return;
       ++step_cnt;
       tc_fence_after_sync();
@@ -469,8 +484,8 @@ __device__ void bwd_drain_role(const BwdParams& p, const CUtensorMap* tmW, uint8
         fence_proxy_async_smem();
         named_barrier_sync<3, 128>();
         if (tid == 0) {
-          tma_reduce_add_3d(tmW, smem_u32(smem + L::kDqOff), r * 64, row0, w.bh);
-          tma_reduce_add_3d(tmW, smem_u32(smem + L::kDqOff + L::kPanelBytes), r * 64 + 32, row0, w.bh);
+          tma_reduce_add_3d(tmW, smem_u32(smem + L::kDqOff), r * 64, row0, bh_q);
+          tma_reduce_add_3d(tmW, smem_u32(smem + L::kDqOff + L::kPanelBytes), r * 64 + 32, row0, bh_q);
           tma_commit_group();
         }
       }
@@ -481,7 +496,7 @@ __device__ void bwd_drain_role(const BwdParams& p, const CUtensorMap* tmW, uint8
 
 // ------------------------------------------------------------------ kernels
 
-template <int D, bool CAUSAL, bool ALIBI, bool DBIAS>
+template <int D, bool CAUSAL, bool ALIBI, bool DBIAS, bool GROUPED>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 sigattn_bwd_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                         const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmDo,
@@ -535,15 +550,15 @@ sigattn_bwd_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
   const uint32_t tmem = tmem_base_slot;
 
   if (warp == kBwdLoadWarp) {
-    if ((threadIdx.x & 31) == 0) bwd_load_role<D, CAUSAL>(p, &tmQ, &tmK, &tmV, &tmDo, smem_base, &bars, &cta_err);
+    if ((threadIdx.x & 31) == 0) bwd_load_role<D, CAUSAL, GROUPED>(p, &tmQ, &tmK, &tmV, &tmDo, smem_base, &bars, &cta_err);
     __syncwarp();
   } else if (warp == kBwdMmaWarp) {
-    if ((threadIdx.x & 31) == 0) bwd_mma_role<D, CAUSAL>(p, smem_base, tmem, &bars, &cta_err);
+    if ((threadIdx.x & 31) == 0) bwd_mma_role<D, CAUSAL, GROUPED>(p, smem_base, tmem, &bars, &cta_err);
     __syncwarp();
   } else if (warp < 8) {
-    bwd_act_role<D, CAUSAL, ALIBI, DBIAS>(p, &tmDk, &tmDv, warp >> 2, smem, tmem, &bars, &cta_err);
+    bwd_act_role<D, CAUSAL, ALIBI, DBIAS, GROUPED>(p, &tmDk, &tmDv, warp >> 2, smem, tmem, &bars, &cta_err);
   } else {
-    bwd_drain_role<D, CAUSAL>(p, &tmW, smem, tmem, &bars, &cta_err);
+    bwd_drain_role<D, CAUSAL, GROUPED>(p, &tmW, smem, tmem, &bars, &cta_err);
   }
 
   tc_fence_before_sync();
@@ -568,10 +583,10 @@ sigattn_bwd_convert_dq_kernel(const float4* __restrict__ ws, uint2* __restrict__
   }
 }
 
-template <int D, bool CAUSAL, bool ALIBI, bool DBIAS>
+template <int D, bool CAUSAL, bool ALIBI, bool DBIAS, bool GROUPED>
 int launch_bwd_variant(const CUtensorMap* maps, const BwdParams& bp, int num_sms, cudaStream_t stream,
                        cudaError_t* cuda_err) {
-  auto kernel = sigattn_bwd_bf16_kernel<D, CAUSAL, ALIBI, DBIAS>;
+  auto kernel = sigattn_bwd_bf16_kernel<D, CAUSAL, ALIBI, DBIAS, GROUPED>;
   static bool configured = false;
   if (!configured) {
     *cuda_err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<D>::kDynBytes);
@@ -610,11 +625,13 @@ int launch_bwd_bf16(const void* q, const void* k, const void* v, const void* d_o
   *cuda_err = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
   if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
 
-  const uint64_t BH = static_cast<uint64_t>(p.B) * p.H;
+  const uint64_t BH = static_cast<uint64_t>(p.B) * p.H;             // query heads: Q, dO, the dQ accumulator
+  const uint64_t BH_kv = static_cast<uint64_t>(p.B) * p.kv_heads();  // K, V, dK, dV
   CUtensorMap maps[7];
   const void* ptrs[6] = {q, k, v, d_o, dk, dv};
   for (int i = 0; i < 6; ++i) {
-    if (make_map_3d(&maps[i], ptrs[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, BH, p.N, p.D, kT, 64) != 0) {
+    const uint64_t heads = (i == 0 || i == 3) ? BH : BH_kv;
+    if (make_map_3d(&maps[i], ptrs[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.N, p.D, kT, 64) != 0) {
       *cuda_err = cudaErrorInvalidValue;
       return SIGATTN_ERR_CUDA;
     }
@@ -624,8 +641,10 @@ int launch_bwd_bf16(const void* q, const void* k, const void* v, const void* d_o
     return SIGATTN_ERR_CUDA;
   }
   BwdParams bp;
-  bp.BH = static_cast<int>(BH);
+  bp.BH = static_cast<int>(BH_kv);
   bp.H = p.H;
+  bp.H_kv = p.kv_heads();
+  bp.group = p.H / p.kv_heads();
   bp.N = p.N;
   bp.n_tiles = (p.N + kT - 1) / kT;
   bp.n_items = bp.n_tiles * bp.BH;
@@ -653,9 +672,13 @@ int launch_bwd_bf16(const void* q, const void* k, const void* v, const void* d_o
   const bool alibi = p.slopes != nullptr;
   // the bias gradient costs the activation groups a running sum (4-5 % of the kernel), so it
   // is compiled in only where it is asked for
-#define SIGATTN_BWD_CASE(DD, CC, AA)                                                          \
-  rc = (p.dbias != nullptr) ? launch_bwd_variant<DD, CC, AA, true>(maps, bp, num_sms, stream, cuda_err) \
-                            : launch_bwd_variant<DD, CC, AA, false>(maps, bp, num_sms, stream, cuda_err)
+  // is compiled in only where it is asked for; likewise the loop over a group's query heads
+#define SIGATTN_BWD_CASE(DD, CC, AA)                                                                        \
+  rc = (bp.group > 1)                                                                                       \
+           ? ((p.dbias != nullptr) ? launch_bwd_variant<DD, CC, AA, true, true>(maps, bp, num_sms, stream, cuda_err)   \
+                                   : launch_bwd_variant<DD, CC, AA, false, true>(maps, bp, num_sms, stream, cuda_err)) \
+           : ((p.dbias != nullptr) ? launch_bwd_variant<DD, CC, AA, true, false>(maps, bp, num_sms, stream, cuda_err)  \
+                                   : launch_bwd_variant<DD, CC, AA, false, false>(maps, bp, num_sms, stream, cuda_err))
   if (p.D == 128) {
     if (p.causal) { if (alibi) SIGATTN_BWD_CASE(128, true, true); else SIGATTN_BWD_CASE(128, true, false); }
     else          { if (alibi) SIGATTN_BWD_CASE(128, false, true); else SIGATTN_BWD_CASE(128, false, false); }

@@ -30,12 +30,13 @@ __device__ __forceinline__ float dot_row(const float* __restrict__ a_smem, const
 __global__ void fwd_fp32_kernel(const float* __restrict__ q, const float* __restrict__ k,
                                 const float* __restrict__ v, float* __restrict__ o, int H, int N, int D,
                                 float scale, float bias, int causal, const float* __restrict__ slopes,
-                                const float* __restrict__ bias_vec) {
+                                const float* __restrict__ bias_vec, int H_kv) {
   __shared__ float sq[128];
   __shared__ float sp[kThreads];
   const int i = blockIdx.x, bh = blockIdx.y, t = threadIdx.x;
   if (bias_vec) bias = bias_vec[bh];
   const size_t base = static_cast<size_t>(bh) * N * D;
+  const size_t kv_base = static_cast<size_t>((bh / H) * H_kv + (bh % H) / (H / H_kv)) * N * D;
   const float slope = slopes ? slopes[bh % H] : 0.0f;
   if (t < D) sq[t] = q[base + static_cast<size_t>(i) * D + t];
   __syncthreads();
@@ -45,7 +46,7 @@ __global__ void fwd_fp32_kernel(const float* __restrict__ q, const float* __rest
     const int j = j0 + t;
     float p = 0.0f;
     if (j < jend) {
-      const float s = dot_row(sq, k + base + static_cast<size_t>(j) * D, D);
+      const float s = dot_row(sq, k + kv_base + static_cast<size_t>(j) * D, D);
       const float x = fmaf(scale, s, bias) - slope * fabsf(static_cast<float>(i - j));
       p = sigmoid_exact(x);
     }
@@ -53,7 +54,7 @@ __global__ void fwd_fp32_kernel(const float* __restrict__ q, const float* __rest
     __syncthreads();
     if (t < D) {
       const int cnt = min(kThreads, jend - j0);
-      for (int jj = 0; jj < cnt; ++jj) acc = fmaf(sp[jj], v[base + static_cast<size_t>(j0 + jj) * D + t], acc);
+      for (int jj = 0; jj < cnt; ++jj) acc = fmaf(sp[jj], v[kv_base + static_cast<size_t>(j0 + jj) * D + t], acc);
     }
     __syncthreads();
   }
@@ -65,12 +66,13 @@ __global__ void bwd_dq_fp32_kernel(const float* __restrict__ q, const float* __r
                                    const float* __restrict__ v, const float* __restrict__ d_o,
                                    float* __restrict__ dq, int H, int N, int D, float scale, float bias,
                                    int causal, const float* __restrict__ slopes,
-                                   const float* __restrict__ bias_vec, float* __restrict__ dbias) {
+                                   const float* __restrict__ bias_vec, float* __restrict__ dbias, int H_kv) {
   __shared__ float sq[128];
   __shared__ float sdo[128];
   __shared__ float sds[kThreads];
   const int i = blockIdx.x, bh = blockIdx.y, t = threadIdx.x;
   if (bias_vec) bias = bias_vec[bh];
+  const size_t kv_base = static_cast<size_t>((bh / H) * H_kv + (bh % H) / (H / H_kv)) * N * D;
   float ds_sum = 0.0f;   // this thread's share of sum_j dS_ij
   const size_t base = static_cast<size_t>(bh) * N * D;
   const float slope = slopes ? slopes[bh % H] : 0.0f;
@@ -85,9 +87,9 @@ __global__ void bwd_dq_fp32_kernel(const float* __restrict__ q, const float* __r
     const int j = j0 + t;
     float ds = 0.0f;
     if (j < jend) {
-      const float s = dot_row(sq, k + base + static_cast<size_t>(j) * D, D);
+      const float s = dot_row(sq, k + kv_base + static_cast<size_t>(j) * D, D);
       const float x = fmaf(scale, s, bias) - slope * fabsf(static_cast<float>(i - j));
-      const float dp = dot_row(sdo, v + base + static_cast<size_t>(j) * D, D);
+      const float dp = dot_row(sdo, v + kv_base + static_cast<size_t>(j) * D, D);
       ds = sigmoid_slope(x) * dp;
     }
     sds[t] = ds;
@@ -95,7 +97,7 @@ __global__ void bwd_dq_fp32_kernel(const float* __restrict__ q, const float* __r
     __syncthreads();
     if (t < D) {
       const int cnt = min(kThreads, jend - j0);
-      for (int jj = 0; jj < cnt; ++jj) acc = fmaf(sds[jj], k[base + static_cast<size_t>(j0 + jj) * D + t], acc);
+      for (int jj = 0; jj < cnt; ++jj) acc = fmaf(sds[jj], k[kv_base + static_cast<size_t>(j0 + jj) * D + t], acc);
     }
     __syncthreads();
   }
@@ -111,53 +113,59 @@ __global__ void bwd_dq_fp32_kernel(const float* __restrict__ q, const float* __r
   }
 }
 
-// dV_j = sum_i P_ij dO_i ; dK_j = scale * sum_i dS_ij Q_i.  grid (N, B*H), one key row each.
+// dV_j = sum_i P_ij dO_i ; dK_j = scale * sum_i dS_ij Q_i, summed over the query heads that read
+// this key/value head.  grid (N, B*H_kv), one key row each.
 __global__ void bwd_dkdv_fp32_kernel(const float* __restrict__ q, const float* __restrict__ k,
                                      const float* __restrict__ v, const float* __restrict__ d_o,
                                      float* __restrict__ dk, float* __restrict__ dv, int H, int N, int D,
-                                     float scale, float bias, int causal, const float* __restrict__ slopes,
-                                     const float* __restrict__ bias_vec) {
+                                     float scale, float bias_scalar, int causal, const float* __restrict__ slopes,
+                                     const float* __restrict__ bias_vec, int H_kv) {
   __shared__ float sk[128];
   __shared__ float sv[128];
   __shared__ float sp[kThreads];
   __shared__ float sds[kThreads];
-  const int j = blockIdx.x, bh = blockIdx.y, t = threadIdx.x;
-  if (bias_vec) bias = bias_vec[bh];
-  const size_t base = static_cast<size_t>(bh) * N * D;
-  const float slope = slopes ? slopes[bh % H] : 0.0f;
+  const int j = blockIdx.x, bh_kv = blockIdx.y, t = threadIdx.x;
+  const int group = H / H_kv;
+  const size_t kv_base = static_cast<size_t>(bh_kv) * N * D;
   if (t < D) {
-    sk[t] = k[base + static_cast<size_t>(j) * D + t];
-    sv[t] = v[base + static_cast<size_t>(j) * D + t];
+    sk[t] = k[kv_base + static_cast<size_t>(j) * D + t];
+    sv[t] = v[kv_base + static_cast<size_t>(j) * D + t];
   }
   __syncthreads();
   const int ibeg = causal ? j : 0;
   float acc_k = 0.0f, acc_v = 0.0f;
-  for (int i0 = ibeg; i0 < N; i0 += kThreads) {
-    const int i = i0 + t;
-    float p = 0.0f, ds = 0.0f;
-    if (i < N) {
-      const float s = dot_row(sk, q + base + static_cast<size_t>(i) * D, D);
-      const float x = fmaf(scale, s, bias) - slope * fabsf(static_cast<float>(i - j));
-      p = sigmoid_exact(x);
-      const float dp = dot_row(sv, d_o + base + static_cast<size_t>(i) * D, D);
-      ds = sigmoid_slope(x) * dp;
-    }
-    sp[t] = p;
-    sds[t] = ds;
-    __syncthreads();
-    if (t < D) {
-      const int cnt = min(kThreads, N - i0);
-      for (int ii = 0; ii < cnt; ++ii) {
-        const size_t row = base + static_cast<size_t>(i0 + ii) * D + t;
-        acc_v = fmaf(sp[ii], d_o[row], acc_v);
-        acc_k = fmaf(sds[ii], q[row], acc_k);
+  for (int g = 0; g < group; ++g) {
+    const int bh = (bh_kv / H_kv) * H + (bh_kv % H_kv) * group + g;   // query head
+    const size_t base = static_cast<size_t>(bh) * N * D;
+    const float slope = slopes ? slopes[bh % H] : 0.0f;
+    const float bias = bias_vec ? bias_vec[bh] : bias_scalar;
+    for (int i0 = ibeg; i0 < N; i0 += kThreads) {
+      const int i = i0 + t;
+      float p = 0.0f, ds = 0.0f;
+      if (i < N) {
+        const float s = dot_row(sk, q + base + static_cast<size_t>(i) * D, D);
+        const float x = fmaf(scale, s, bias) - slope * fabsf(static_cast<float>(i - j));
+        p = sigmoid_exact(x);
+        const float dp = dot_row(sv, d_o + base + static_cast<size_t>(i) * D, D);
+        ds = sigmoid_slope(x) * dp;
       }
+      sp[t] = p;
+      sds[t] = ds;
+      __syncthreads();
+      if (t < D) {
+        const int cnt = min(kThreads, N - i0);
+        for (int ii = 0; ii < cnt; ++ii) {
+          const size_t row = base + static_cast<size_t>(i0 + ii) * D + t;
+          acc_v = fmaf(sp[ii], d_o[row], acc_v);
+          acc_k = fmaf(sds[ii], q[row], acc_k);
+        }
+      }
+      __syncthreads();
     }
-    __syncthreads();
   }
   if (t < D) {
-    dv[base + static_cast<size_t>(j) * D + t] = acc_v;
-    dk[base + static_cast<size_t>(j) * D + t] = scale * acc_k;
+    dv[kv_base + static_cast<size_t>(j) * D + t] = acc_v;
+    dk[kv_base + static_cast<size_t>(j) * D + t] = scale * acc_k;
   }
 }
 
@@ -167,7 +175,7 @@ int launch_fwd_fp32(const float* q, const float* k, const float* v, float* o, co
                     cudaStream_t stream, unsigned long long* launches, cudaError_t* cuda_err) {
   dim3 grid(p.N, p.B * p.H);
   fwd_fp32_kernel<<<grid, kThreads, 0, stream>>>(q, k, v, o, p.H, p.N, p.D, p.scale, p.bias, p.causal, p.slopes,
-                                                 p.bias_vec);
+                                                 p.bias_vec, p.kv_heads());
   *launches += 1;
   *cuda_err = cudaGetLastError();
   return *cuda_err == cudaSuccess ? SIGATTN_OK : SIGATTN_ERR_CUDA;
@@ -182,9 +190,10 @@ int launch_bwd_fp32(const float* q, const float* k, const float* v, const float*
     if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
   }
   bwd_dq_fp32_kernel<<<grid, kThreads, 0, stream>>>(q, k, v, d_o, dq, p.H, p.N, p.D, p.scale, p.bias, p.causal,
-                                                    p.slopes, p.bias_vec, p.dbias);
-  bwd_dkdv_fp32_kernel<<<grid, kThreads, 0, stream>>>(q, k, v, d_o, dk, dv, p.H, p.N, p.D, p.scale, p.bias,
-                                                      p.causal, p.slopes, p.bias_vec);
+                                                    p.slopes, p.bias_vec, p.dbias, p.kv_heads());
+  dim3 grid_kv(p.N, p.B * p.kv_heads());
+  bwd_dkdv_fp32_kernel<<<grid_kv, kThreads, 0, stream>>>(q, k, v, d_o, dk, dv, p.H, p.N, p.D, p.scale, p.bias,
+                                                         p.causal, p.slopes, p.bias_vec, p.kv_heads());
   *launches += 2;
   *cuda_err = cudaGetLastError();
   return *cuda_err == cudaSuccess ? SIGATTN_OK : SIGATTN_ERR_CUDA;

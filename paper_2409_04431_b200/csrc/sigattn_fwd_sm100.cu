@@ -83,6 +83,7 @@ struct FwdBarriers {
 
 struct FwdParams {
   int BH, H, N;
+  int H_kv, group;  // heads of K, V and query heads per key/value head (H = H_kv * group)
   int n_pairs;     // ceil(N / 256)
   int n_kv_total;  // ceil(N / 128)
   int n_items;
@@ -137,6 +138,7 @@ __device__ void fwd_load_role(const FwdParams& p, const CUtensorMap* tmQ, const 
     const int item = snake_rank(round, p.n_items);
     if (item < 0) continue;
     const Item w = decode_item<CAUSAL>(p, item);
+    const int bh_kv = (w.bh / p.H) * p.H_kv + (w.bh % p.H) / p.group;   // the key/value head this query head reads
     auto load_q = [&](int t) -> bool {
       if (w.n[t] == 0) return true;
       if (!mbar_wait(smem_u32(&bars->q_empty[t]), (q_iter[t] & 1) ^ 1, cta_err, 10 + t)) return false;
@@ -158,7 +160,7 @@ __device__ void fwd_load_role(const FwdParams& p, const CUtensorMap* tmQ, const 
 #pragma unroll
       for (int pn = 0; pn < L::kPanels; ++pn)
         tma_load_3d(smem_base + L::kKvOff + stage * L::kTileBytes + pn * L::kPanelBytes, tm, bar, pn * 64, j * kBN,
-                    w.bh);
+                    bh_kv);
       ++kv_cnt;
       return true;
     };
@@ -513,11 +515,13 @@ int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const 
   if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
 
   const uint64_t BH = static_cast<uint64_t>(p.B) * p.H;
+  const uint64_t BH_kv = static_cast<uint64_t>(p.B) * p.kv_heads();
   CUtensorMap tmQ, tmK, tmV, tmO;
   const void* ptrs[4] = {q, k, v, o};
   CUtensorMap* maps[4] = {&tmQ, &tmK, &tmV, &tmO};
   for (int i = 0; i < 4; ++i) {
-    if (make_map_3d(maps[i], ptrs[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, BH, p.N, p.D, kBM, 64) != 0) {
+    const uint64_t heads = (i == 1 || i == 2) ? BH_kv : BH;
+    if (make_map_3d(maps[i], ptrs[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.N, p.D, kBM, 64) != 0) {
       *cuda_err = cudaErrorInvalidValue;
       return SIGATTN_ERR_CUDA;
     }
@@ -525,6 +529,8 @@ int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const 
   FwdParams fp;
   fp.BH = static_cast<int>(BH);
   fp.H = p.H;
+  fp.H_kv = p.kv_heads();
+  fp.group = p.H / p.kv_heads();
   fp.N = p.N;
   fp.n_pairs = (p.N + 2 * kBM - 1) / (2 * kBM);
   fp.n_kv_total = (p.N + kBN - 1) / kBN;

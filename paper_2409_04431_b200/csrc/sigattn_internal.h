@@ -14,6 +14,8 @@ struct Problem {
   const float* slopes;    // device pointer to H floats, or nullptr
   const float* bias_vec;  // device pointer to B*H biases that replace `bias`, or nullptr
   float* dbias;           // backward only: device pointer to B*H floats that receive sum dS, or nullptr
+  int H_kv;               // heads of k, v (H is a multiple of it; query head h reads head h / (H / H_kv)); 0 = H
+  int kv_heads() const { return H_kv > 0 ? H_kv : H; }
 };
 
 // Every launcher enqueues on `stream`, adds the number of kernels it launched to
