@@ -418,3 +418,15 @@ def test_grouped_kv_heads_forward_and_backward(h_kv):
         assert np.linalg.norm(fd - g) / np.linalg.norm(fd) < 1e-7, name
     with pytest.raises(ValueError):
         oracle.sigattn_fwd(q, rnd((B, 3, N, D), 94), rnd((B, 3, N, D), 95), scale, b)
+
+
+def test_temperature_gradient_is_a_reduction_of_q_and_dq():
+    """sigma(e^t [Q K^T / sqrt(d)] + b) V (Appendix G.2.2): with scale' = scale e^t passed as
+    the scale, dL/dt = sum_i <Q_i, dQ_i>, because dQ_i = scale' sum_j dS_ij K_j."""
+    B, H, N, D = 1, 2, 6, 4
+    q, k, v, d_o = (rnd((B, H, N, D), s) for s in (100, 101, 102, 103))
+    scale, b, t = 0.5, -1.3, 0.4
+    dq, _, _ = oracle.sigattn_bwd(q, k, v, d_o, scale * math.exp(t), b, True)
+    h = 1e-6
+    fd = (loss(q, k, v, d_o, scale * math.exp(t + h), b, True, None) - loss(q, k, v, d_o, scale * math.exp(t - h), b, True, None)) / (2 * h)
+    assert abs(float(np.sum(q * dq)) - fd) < 1e-7 * max(1.0, abs(fd))
