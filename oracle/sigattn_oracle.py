@@ -46,6 +46,13 @@ Readings of the paper taken here
     h // (H / H_kv) (consecutive query heads share one), and dK, dV of a key/value head
     are the sums over the query heads that read it.  The paper gives no layout; this is
     the usual one.
+  * The paper defines self-attention (as many queries as keys).  Generation with a cache
+    of earlier keys and values, where its inference gains are measured (Appendix F.3), has
+    N_q queries against N_k >= N_q keys: q is [B, H, N_q, D], k and v are [B, H_kv, N_k, D],
+    and the queries are the LAST N_q positions, i.e. query i sits at position
+    i + N_k - N_q for the causal mask (keys j <= i + N_k - N_q are kept) and for the
+    position bias.  N_q = N_k is the paper's case.  Without a causal mask and without
+    slopes the positions play no role and any N_q, N_k are allowed (cross-attention).
 
 Every function is pinned by tests that do not call back into this file's own
 formulae (closed forms, brute-force loops, finite differences, the paper's second
@@ -82,35 +89,41 @@ def sigmoid(x):
     return out
 
 
-def causal_mask(n: int, i0: int = 0, i1: int | None = None):
+def causal_mask(n: int, i0: int = 0, i1: int | None = None, n_q: int | None = None):
     """Rows i0..i1-1 of the n x n lower-triangular 0/1 matrix, diagonal included
-    (the matrix M printed for n = 3 in Appendix G's normalisation ablation)."""
-    i1 = n if i1 is None else i1
-    i = np.arange(i0, i1)[:, None]
+    (the matrix M printed for n = 3 in Appendix G's normalisation ablation).
+
+    With n_q query rows against n keys (n_q != n) query i sits at position i + n - n_q
+    (see the module header), so the row keeps keys j <= i + n - n_q."""
+    n_q = n if n_q is None else n_q
+    i1 = n_q if i1 is None else i1
+    i = np.arange(i0, i1)[:, None] + (n - n_q)
     j = np.arange(n)[None, :]
     return (j <= i).astype(np.float64)
 
 
-def position_bias(n: int, slope: float, i0: int = 0, i1: int | None = None):
+def position_bias(n: int, slope: float, i0: int = 0, i1: int | None = None, n_q: int | None = None):
     """Additive linear position bias -slope * |i - j| for rows i0..i1-1 (Appendix F.4
-    names ALiBi; see the module header for the reading)."""
-    i1 = n if i1 is None else i1
-    i = np.arange(i0, i1, dtype=np.float64)[:, None]
+    names ALiBi; see the module header for the reading); with n_q != n query rows the
+    distance is taken from the query's position i + n - n_q."""
+    n_q = n if n_q is None else n_q
+    i1 = n_q if i1 is None else i1
+    i = np.arange(i0, i1, dtype=np.float64)[:, None] + float(n - n_q)
     j = np.arange(n, dtype=np.float64)[None, :]
     return -float(slope) * np.abs(i - j)
 
 
 def attention_weights(q, k, scale, bias, causal, slope=0.0, i0=0, i1=None):
     """P for query rows i0..i1-1 of one head: sigmoid(scale * q k^T + b + position
-    bias), times the causal mask.  q, k: [n, d] float64."""
-    n = q.shape[0]
-    i1 = n if i1 is None else i1
+    bias), times the causal mask.  q: [n_q, d], k: [n, d] float64."""
+    n_q, n = q.shape[0], k.shape[0]
+    i1 = n_q if i1 is None else i1
     x = scale * (q[i0:i1] @ k.T) + bias
     if slope != 0.0:
-        x = x + position_bias(n, slope, i0, i1)
+        x = x + position_bias(n, slope, i0, i1, n_q)
     p = sigmoid(x)
     if causal:
-        p = p * causal_mask(n, i0, i1)
+        p = p * causal_mask(n, i0, i1, n_q)
     return p
 
 
@@ -160,7 +173,7 @@ def sigattn_fwd(q, k, v, scale, bias, causal=False, alibi_slopes=None, row_block
     Returns O as float64 [B, H, N, D].
     """
     q, k, v = _as_f64(q, k, v)
-    B, H, N, D = q.shape
+    B, H, N, D = q.shape          # N counts query rows; k, v may hold more (or fewer) rows
     group = _kv_group(H, k)
     slopes = _slopes(alibi_slopes, H)
     bias_bh = _bias_per_head(bias, B, H)

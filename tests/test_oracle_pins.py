@@ -430,3 +430,62 @@ def test_temperature_gradient_is_a_reduction_of_q_and_dq():
     h = 1e-6
     fd = (loss(q, k, v, d_o, scale * math.exp(t + h), b, True, None) - loss(q, k, v, d_o, scale * math.exp(t - h), b, True, None)) / (2 * h)
     assert abs(float(np.sum(q * dq)) - fd) < 1e-7 * max(1.0, abs(fd))
+
+
+# ------------------------------------------------------------------ N_q queries against N_k keys
+
+
+def test_queries_at_the_end_of_a_longer_key_sequence():
+    """Decoding with a cache: the last N_q rows of square causal attention over N_k
+    positions must equal rectangular attention of those N_q queries against all N_k keys,
+    forward and backward (dK, dV of the rectangular call see only those queries)."""
+    B, H, NK, NQ, D = 1, 2, 7, 3, 4
+    q_full, k, v, do_full = (rnd((B, H, NK, D), s) for s in (110, 111, 112, 113))
+    slopes = np.array([0.5, 0.125])
+    scale, b = 0.5, -0.7
+    q, d_o = q_full[:, :, NK - NQ:], do_full[:, :, NK - NQ:]
+    o_sq = oracle.sigattn_fwd(q_full, k, v, scale, b, True, slopes)
+    o = oracle.sigattn_fwd(q, k, v, scale, b, True, slopes)
+    assert o.shape == (B, H, NQ, D)
+    np.testing.assert_allclose(o, o_sq[:, :, NK - NQ:], rtol=1e-14, atol=1e-16)
+    do_masked = np.zeros_like(do_full)
+    do_masked[:, :, NK - NQ:] = d_o
+    dq_sq, dk_sq, dv_sq = oracle.sigattn_bwd(q_full, k, v, do_masked, scale, b, True, slopes)
+    dq, dk, dv = oracle.sigattn_bwd(q, k, v, d_o, scale, b, True, slopes)
+    np.testing.assert_allclose(dq, dq_sq[:, :, NK - NQ:], rtol=1e-13, atol=1e-16)
+    np.testing.assert_allclose(dk, dk_sq, rtol=1e-13, atol=1e-16)
+    np.testing.assert_allclose(dv, dv_sq, rtol=1e-13, atol=1e-16)
+    # one query against the whole cache, element by element
+    o1 = oracle.sigattn_fwd(q[:, :, -1:], k, v, scale, b, True, slopes)
+    for h in range(H):
+        ref = np.zeros(D)
+        for j in range(NK):
+            x = scale * float(q[0, h, -1] @ k[0, h, j]) + b - slopes[h] * (NK - 1 - j)
+            ref += scalar_sigmoid(x) * v[0, h, j]
+        np.testing.assert_allclose(o1[0, h, 0], ref, rtol=1e-13)
+
+
+def test_cross_attention_without_mask_brute_force():
+    B, H, NQ, NK, D = 1, 1, 5, 3, 2
+    q, d_o = rnd((B, H, NQ, D), 120), rnd((B, H, NQ, D), 121)
+    k, v = rnd((B, H, NK, D), 122), rnd((B, H, NK, D), 123)
+    scale, b = 0.8, -0.2
+    o = oracle.sigattn_fwd(q, k, v, scale, b, False)
+    ref = np.zeros_like(o)
+    for i in range(NQ):
+        for j in range(NK):
+            ref[0, 0, i] += scalar_sigmoid(scale * float(q[0, 0, i] @ k[0, 0, j]) + b) * v[0, 0, j]
+    np.testing.assert_allclose(o, ref, rtol=1e-13)
+    dq, dk, dv = oracle.sigattn_bwd(q, k, v, d_o, scale, b, False)
+    h = 1e-6
+    for name, x, g in (("q", q, dq), ("k", k, dk), ("v", v, dv)):
+        fd = np.zeros_like(x)
+        for idx in np.ndindex(*x.shape):
+            old = x[idx]
+            x[idx] = old + h
+            lp = loss(q, k, v, d_o, scale, b, False, None)
+            x[idx] = old - h
+            lm = loss(q, k, v, d_o, scale, b, False, None)
+            x[idx] = old
+            fd[idx] = (lp - lm) / (2 * h)
+        assert np.linalg.norm(fd - g) / np.linalg.norm(fd) < 1e-7, name
