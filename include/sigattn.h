@@ -172,6 +172,28 @@ SIGATTN_API int sigattn_bwd_gqa(const void* q, const void* k, const void* v, con
                     float* dbias_bh,
                     void* workspace, size_t workspace_bytes, void* stream);
 
+/* N_q queries against N_k keys and values: q, o (d_o, dq) are [B, H, N_q, D], k, v (dk, dv)
+ * are [B, H_kv, N_k, D].  The paper defines self-attention (N_q = N_k); generation with a
+ * cache of earlier keys and values, where its inference gains are measured (Appendix F.3),
+ * has the queries at the LAST N_q positions: query i sits at position i + N_k - N_q for the
+ * causal mask (keys j <= i + N_k - N_q are kept) and for the ALiBi distance.  With causal = 1,
+ * N_k >= N_q is required (SIGATTN_ERR_SHAPE otherwise); without a mask any N_q, N_k >= 1 are
+ * allowed (cross-attention).  H_kv, bias_bh as in sigattn_fwd_gqa.  N_q = N_k and H_kv = H
+ * is sigattn_fwd. */
+SIGATTN_API int sigattn_fwd_nk(const void* q, const void* k, const void* v, void* o,
+                   int B, int H, int H_kv, int N_q, int N_k, int D,
+                   float scale, float bias, const float* bias_bh, int causal,
+                   const float* alibi_slopes, int dtype, void* stream);
+
+/* Backward of sigattn_fwd_nk.  The workspace is that of sigattn_bwd for (B, H, N_q, D). */
+SIGATTN_API int sigattn_bwd_nk(const void* q, const void* k, const void* v, const void* d_o,
+                   void* dq, void* dk, void* dv,
+                   int B, int H, int H_kv, int N_q, int N_k, int D,
+                   float scale, float bias, const float* bias_bh, int causal,
+                   const float* alibi_slopes, int dtype,
+                   float* dbias_bh,
+                   void* workspace, size_t workspace_bytes, void* stream);
+
 /* Bytes of scratch sigattn_bwd needs for this problem (0 for the fp32 debug path).
  * Returns 0 for invalid shapes as well; sigattn_bwd reports those. */
 SIGATTN_API size_t sigattn_bwd_workspace_bytes(int B, int H, int N, int D, int dtype);

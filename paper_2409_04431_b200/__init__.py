@@ -29,6 +29,8 @@ _BINDING_NAMES = (
     "sigattn_bwd_bias_vec",
     "sigattn_fwd_gqa",
     "sigattn_bwd_gqa",
+    "sigattn_fwd_nk",
+    "sigattn_bwd_nk",
     "lib",
 )
 

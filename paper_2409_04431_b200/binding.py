@@ -45,6 +45,13 @@ _lib.sigattn_bwd_gqa.restype = _c.c_int
 _lib.sigattn_bwd_gqa.argtypes = [_c.c_void_p] * 7 + [_c.c_int] * 5 + [_c.c_float, _c.c_float, _c.c_void_p, _c.c_int,
                                                                         _c.c_void_p, _c.c_int, _c.c_void_p,
                                                                         _c.c_void_p, _c.c_size_t, _c.c_void_p]
+_lib.sigattn_fwd_nk.restype = _c.c_int
+_lib.sigattn_fwd_nk.argtypes = [_c.c_void_p] * 4 + [_c.c_int] * 6 + [_c.c_float, _c.c_float, _c.c_void_p, _c.c_int,
+                                                                       _c.c_void_p, _c.c_int, _c.c_void_p]
+_lib.sigattn_bwd_nk.restype = _c.c_int
+_lib.sigattn_bwd_nk.argtypes = [_c.c_void_p] * 7 + [_c.c_int] * 6 + [_c.c_float, _c.c_float, _c.c_void_p, _c.c_int,
+                                                                       _c.c_void_p, _c.c_int, _c.c_void_p,
+                                                                       _c.c_void_p, _c.c_size_t, _c.c_void_p]
 _lib.sigattn_bwd_workspace_bytes.restype = _c.c_size_t
 _lib.sigattn_bwd_workspace_bytes.argtypes = [_c.c_int] * 5
 _lib.sigattn_step_host.restype = _c.c_int
@@ -79,7 +86,7 @@ EXPORTED = [
     "sigattn_step_host", "sigattn_step_host_arena_bytes", "sigattn_bwd_set_timing_events",
     "sigattn_bwd_static_scratch", "sigattn_bwd_static_scratch_max_elements",
     "sigattn_selftest_bounded_wait", "sigattn_fwd_bias_vec", "sigattn_bwd_bias_vec",
-    "sigattn_fwd_gqa", "sigattn_bwd_gqa",
+    "sigattn_fwd_gqa", "sigattn_bwd_gqa", "sigattn_fwd_nk", "sigattn_bwd_nk",
 ]
 
 
@@ -317,6 +324,65 @@ def sigattn_bwd_gqa(q, k, v, d_o, scale, bias, causal=False, alibi_slopes=None, 
                                   float(scale), 0.0 if vec else float(bias), _ptr(bias) if vec else None,
                                   int(bool(causal)), _ptr(alibi_slopes), code, _ptr(dbias), _ptr(workspace), ws_bytes,
                                   _stream_ptr(stream))
+    if rc != 0:
+        raise SigattnError(rc)
+    return dq, dk, dv, dbias
+
+
+def _check_nk(q, k, v):
+    import torch
+    for t, n in ((q, "q"), (k, "k"), (v, "v")):
+        if not isinstance(t, torch.Tensor) or not t.is_cuda or t.dim() != 4 or not t.is_contiguous():
+            raise ValueError(f"{n} must be a contiguous 4-D CUDA tensor")
+    B, H, N_q, D = q.shape
+    if k.shape != v.shape or k.shape[0] != B or k.shape[3] != D or k.dtype != q.dtype or v.dtype != q.dtype \
+            or k.device != q.device or v.device != q.device:
+        raise ValueError("k, v must be [B, H_kv, N_k, D] with q's B, D, dtype and device")
+    return B, H, k.shape[1], N_q, k.shape[2], D
+
+
+def sigattn_fwd_nk(q, k, v, scale, bias, causal=False, alibi_slopes=None, out=None, stream=None):
+    """N_q queries against N_k keys: q [B, H, N_q, D], k, v [B, H_kv, N_k, D]; the queries are
+    the last N_q positions (causal needs N_k >= N_q).  `bias`: float or float32 CUDA [B, H]."""
+    import torch
+    B, H, H_kv, N_q, N_k, D = _check_nk(q, k, v)
+    if out is None:
+        out = torch.empty_like(q)
+    else:
+        _check_same([q, out], ["q", "out"])
+    vec = isinstance(bias, torch.Tensor)
+    if vec:
+        _check_bias_vec(bias, q)
+    with torch.cuda.device(q.device):
+        rc = _lib.sigattn_fwd_nk(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, H, H_kv, N_q, N_k, D, float(scale),
+                                 0.0 if vec else float(bias), _ptr(bias) if vec else None, int(bool(causal)),
+                                 _ptr(alibi_slopes), _dtype_code(q), _stream_ptr(stream))
+    if rc != 0:
+        raise SigattnError(rc)
+    return out
+
+
+def sigattn_bwd_nk(q, k, v, d_o, scale, bias, causal=False, alibi_slopes=None, want_dbias=False, workspace=None,
+                   stream=None):
+    """Backward of sigattn_fwd_nk.  Returns (dQ like q, dK like k, dV like v, dbias [B, H] or None)."""
+    import torch
+    B, H, H_kv, N_q, N_k, D = _check_nk(q, k, v)
+    _check_same([q, d_o], ["q", "d_o"])
+    code = _dtype_code(q)
+    dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+    vec = isinstance(bias, torch.Tensor)
+    if vec:
+        _check_bias_vec(bias, q)
+    dbias = torch.empty((B, H), dtype=torch.float32, device=q.device) if want_dbias else None
+    need = sigattn_bwd_workspace_bytes(B, H, N_q, D, code)
+    if workspace is None and need > 0:
+        workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    with torch.cuda.device(q.device):
+        rc = _lib.sigattn_bwd_nk(_ptr(q), _ptr(k), _ptr(v), _ptr(d_o), _ptr(dq), _ptr(dk), _ptr(dv), B, H, H_kv, N_q, N_k,
+                                 D, float(scale), 0.0 if vec else float(bias), _ptr(bias) if vec else None,
+                                 int(bool(causal)), _ptr(alibi_slopes), code, _ptr(dbias), _ptr(workspace), ws_bytes,
+                                 _stream_ptr(stream))
     if rc != 0:
         raise SigattnError(rc)
     return dq, dk, dv, dbias

@@ -87,11 +87,21 @@ void account(unsigned long long launches, int rc, cudaError_t cuda_err) {
 namespace {
 
 // Shared by the scalar-bias and the bias-vector entry points.
-int fwd_any(const void* q, const void* k, const void* v, void* o, int B, int H, int H_kv, int N, int D, float scale,
-            float bias, const float* bias_vec, int causal, const float* alibi_slopes, int dtype, void* stream) {
-  if (!q || !k || !v || !o) return SIGATTN_ERR_NULL;
+// N counts query rows, N_k key/value rows; a causal mask needs N_k >= N (the queries are the last
+// N positions, so every query then sees at least one key).
+int check_lengths(int B, int H, int H_kv, int N, int N_k, int D, int causal) {
   if (int rc = check_shape(B, H, N, D)) return rc;
   if (H_kv < 1 || H % H_kv != 0) return SIGATTN_ERR_SHAPE;
+  if (int rc = check_shape(B, H_kv, N_k, D)) return rc;
+  if (causal == 1 && N_k < N) return SIGATTN_ERR_SHAPE;
+  return SIGATTN_OK;
+}
+
+int fwd_any(const void* q, const void* k, const void* v, void* o, int B, int H, int H_kv, int N, int N_k, int D,
+            float scale, float bias, const float* bias_vec, int causal, const float* alibi_slopes, int dtype,
+            void* stream) {
+  if (!q || !k || !v || !o) return SIGATTN_ERR_NULL;
+  if (int rc = check_lengths(B, H, H_kv, N, N_k, D, causal)) return rc;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return SIGATTN_ERR_ALIGN;
   if (alibi_slopes && (reinterpret_cast<uintptr_t>(alibi_slopes) & 3u)) return SIGATTN_ERR_ALIGN;
   if (dtype != SIGATTN_DTYPE_BF16 && dtype != SIGATTN_DTYPE_FP32) return SIGATTN_ERR_FLAG;
@@ -99,7 +109,7 @@ int fwd_any(const void* q, const void* k, const void* v, void* o, int B, int H, 
   int dev = 0;
   int* status = nullptr;
   if (int rc = device_setup(&dev, &status)) return rc;
-  sigattn::Problem p{B, H, N, D, scale, bias, causal, alibi_slopes, bias_vec, nullptr, H_kv};
+  sigattn::Problem p{B, H, N, D, scale, bias, causal, alibi_slopes, bias_vec, nullptr, H_kv, N_k};
   unsigned long long launches = 0;
   cudaError_t ce = cudaSuccess;
   int rc;
@@ -116,11 +126,10 @@ int fwd_any(const void* q, const void* k, const void* v, void* o, int B, int H, 
 }
 
 int bwd_any(const void* q, const void* k, const void* v, const void* d_o, void* dq, void* dk, void* dv, int B, int H,
-            int H_kv, int N, int D, float scale, float bias, const float* bias_vec, float* dbias, int causal,
+            int H_kv, int N, int N_k, int D, float scale, float bias, const float* bias_vec, float* dbias, int causal,
             const float* alibi_slopes, int dtype, void* workspace, size_t workspace_bytes, void* stream) {
   if (!q || !k || !v || !d_o || !dq || !dk || !dv) return SIGATTN_ERR_NULL;
-  if (int rc = check_shape(B, H, N, D)) return rc;
-  if (H_kv < 1 || H % H_kv != 0) return SIGATTN_ERR_SHAPE;
+  if (int rc = check_lengths(B, H, H_kv, N, N_k, D, causal)) return rc;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(d_o) || !aligned16(dq) || !aligned16(dk) ||
       !aligned16(dv))
     return SIGATTN_ERR_ALIGN;
@@ -136,7 +145,7 @@ int bwd_any(const void* q, const void* k, const void* v, const void* d_o, void* 
   int dev = 0;
   int* status = nullptr;
   if (int rc = device_setup(&dev, &status)) return rc;
-  sigattn::Problem p{B, H, N, D, scale, bias, causal, alibi_slopes, bias_vec, dbias, H_kv};
+  sigattn::Problem p{B, H, N, D, scale, bias, causal, alibi_slopes, bias_vec, dbias, H_kv, N_k};
   unsigned long long launches = 0;
   cudaError_t ce = cudaSuccess;
   int rc;
@@ -160,7 +169,7 @@ extern "C" {
 
 int sigattn_fwd(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int D, float scale,
                 float bias, int causal, const float* alibi_slopes, int dtype, void* stream) {
-  return fwd_any(q, k, v, o, B, H, H, N, D, scale, bias, nullptr, causal, alibi_slopes, dtype, stream);
+  return fwd_any(q, k, v, o, B, H, H, N, N, D, scale, bias, nullptr, causal, alibi_slopes, dtype, stream);
 }
 
 int sigattn_fwd_bias_vec(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int D,
@@ -168,20 +177,20 @@ int sigattn_fwd_bias_vec(const void* q, const void* k, const void* v, void* o, i
                          void* stream) {
   if (!bias_bh) return SIGATTN_ERR_NULL;
   if (reinterpret_cast<uintptr_t>(bias_bh) & 3u) return SIGATTN_ERR_ALIGN;
-  return fwd_any(q, k, v, o, B, H, H, N, D, scale, 0.0f, bias_bh, causal, alibi_slopes, dtype, stream);
+  return fwd_any(q, k, v, o, B, H, H, N, N, D, scale, 0.0f, bias_bh, causal, alibi_slopes, dtype, stream);
 }
 
 int sigattn_fwd_gqa(const void* q, const void* k, const void* v, void* o, int B, int H, int H_kv, int N, int D,
                     float scale, float bias, const float* bias_bh, int causal, const float* alibi_slopes, int dtype,
                     void* stream) {
   if (bias_bh && (reinterpret_cast<uintptr_t>(bias_bh) & 3u)) return SIGATTN_ERR_ALIGN;
-  return fwd_any(q, k, v, o, B, H, H_kv, N, D, scale, bias, bias_bh, causal, alibi_slopes, dtype, stream);
+  return fwd_any(q, k, v, o, B, H, H_kv, N, N, D, scale, bias, bias_bh, causal, alibi_slopes, dtype, stream);
 }
 
 int sigattn_bwd(const void* q, const void* k, const void* v, const void* d_o, void* dq, void* dk, void* dv, int B,
                 int H, int N, int D, float scale, float bias, int causal, const float* alibi_slopes, int dtype,
                 void* workspace, size_t workspace_bytes, void* stream) {
-  return bwd_any(q, k, v, d_o, dq, dk, dv, B, H, H, N, D, scale, bias, nullptr, nullptr, causal, alibi_slopes, dtype,
+  return bwd_any(q, k, v, d_o, dq, dk, dv, B, H, H, N, N, D, scale, bias, nullptr, nullptr, causal, alibi_slopes, dtype,
                  workspace, workspace_bytes, stream);
 }
 
@@ -192,7 +201,7 @@ int sigattn_bwd_bias_vec(const void* q, const void* k, const void* v, const void
   if (!bias_bh) return SIGATTN_ERR_NULL;
   if ((reinterpret_cast<uintptr_t>(bias_bh) & 3u) || (reinterpret_cast<uintptr_t>(dbias_bh) & 3u))
     return SIGATTN_ERR_ALIGN;
-  return bwd_any(q, k, v, d_o, dq, dk, dv, B, H, H, N, D, scale, 0.0f, bias_bh, dbias_bh, causal, alibi_slopes,
+  return bwd_any(q, k, v, d_o, dq, dk, dv, B, H, H, N, N, D, scale, 0.0f, bias_bh, dbias_bh, causal, alibi_slopes,
                  dtype, workspace, workspace_bytes, stream);
 }
 
@@ -202,8 +211,25 @@ int sigattn_bwd_gqa(const void* q, const void* k, const void* v, const void* d_o
                     void* stream) {
   if ((reinterpret_cast<uintptr_t>(bias_bh) & 3u) || (reinterpret_cast<uintptr_t>(dbias_bh) & 3u))
     return SIGATTN_ERR_ALIGN;
-  return bwd_any(q, k, v, d_o, dq, dk, dv, B, H, H_kv, N, D, scale, bias, bias_bh, dbias_bh, causal, alibi_slopes,
+  return bwd_any(q, k, v, d_o, dq, dk, dv, B, H, H_kv, N, N, D, scale, bias, bias_bh, dbias_bh, causal, alibi_slopes,
                  dtype, workspace, workspace_bytes, stream);
+}
+
+int sigattn_fwd_nk(const void* q, const void* k, const void* v, void* o, int B, int H, int H_kv, int N_q, int N_k,
+                   int D, float scale, float bias, const float* bias_bh, int causal, const float* alibi_slopes,
+                   int dtype, void* stream) {
+  if (bias_bh && (reinterpret_cast<uintptr_t>(bias_bh) & 3u)) return SIGATTN_ERR_ALIGN;
+  return fwd_any(q, k, v, o, B, H, H_kv, N_q, N_k, D, scale, bias, bias_bh, causal, alibi_slopes, dtype, stream);
+}
+
+int sigattn_bwd_nk(const void* q, const void* k, const void* v, const void* d_o, void* dq, void* dk, void* dv, int B,
+                   int H, int H_kv, int N_q, int N_k, int D, float scale, float bias, const float* bias_bh, int causal,
+                   const float* alibi_slopes, int dtype, float* dbias_bh, void* workspace, size_t workspace_bytes,
+                   void* stream) {
+  if ((reinterpret_cast<uintptr_t>(bias_bh) & 3u) || (reinterpret_cast<uintptr_t>(dbias_bh) & 3u))
+    return SIGATTN_ERR_ALIGN;
+  return bwd_any(q, k, v, d_o, dq, dk, dv, B, H, H_kv, N_q, N_k, D, scale, bias, bias_bh, dbias_bh, causal,
+                 alibi_slopes, dtype, workspace, workspace_bytes, stream);
 }
 
 int sigattn_bwd_set_timing_events(void* start_event, void* stop_event) {

@@ -69,7 +69,9 @@ struct BwdBarriers {
 struct BwdParams {
   int BH, H, N;    // BH counts (batch, key/value head) pairs: the work items are per key/value head
   int H_kv, group; // heads of K, V and query heads per key/value head (H = H_kv * group)
-  int n_tiles;  // ceil(N / 128), for keys and for queries
+  int n_tiles;    // query tiles: ceil(N / 128), N = rows of Q
+  int n_tiles_k;  // key tiles: ceil(rows of K / 128)
+  int pos0;       // position of query row 0: rows of K, V minus N (0 for self-attention)
   int n_items;
   float scale, scale_log2e, bias_log2e;
   const float* bias_vec;   // one bias per (batch, head) instead of the scalar, or nullptr
@@ -105,7 +107,8 @@ __device__ __forceinline__ BwdItem decode_bwd_item(const BwdParams& p, int item)
   w.j = item / p.BH;  // ascending key tile = descending work when causal
   w.bh = item - w.j * p.BH;
   w.bh_q0 = GROUPED ? (w.bh / p.H_kv) * p.H + (w.bh % p.H_kv) * p.group : w.bh;
-  w.i_begin = CAUSAL ? w.j : 0;
+  // causal: the first query tile whose last row, at position 128 i + 127 + pos0, reaches key 128 j
+  w.i_begin = CAUSAL ? max(0, (w.j * kT - p.pos0) / kT) : 0;
   w.n = p.n_tiles - w.i_begin;
   w.steps = GROUPED ? p.group * w.n : w.n;
   return w;
@@ -351,8 +354,11 @@ __device__ void bwd_act_role(const BwdParams& p, const CUtensorMap* tmDk, const 
 
     for (int it = 0; it < w.n; ++it) {
       const int i = w.i_begin + it;
-      const float col_rel = static_cast<float>((w.j - i) * kT + tid);  // key index minus first query of the tile
-      const bool diag = CAUSAL && (it == 0);
+      // this thread's key index minus the position of the tile's first query
+      const float col_rel = static_cast<float>((w.j - i) * kT + tid - p.pos0);
+      // the mask cuts through the tile unless even its first query sits at or after the last key:
+      // the first tile of the loop, and with pos0 not a multiple of 128 also the second
+      const bool diag = CAUSAL && (i * kT + p.pos0 < w.j * kT + kT - 1);
       float pp0[32], pp1[32];
       if (!mbar_wait(smem_u32(&bars->s_full), step_cnt & 1, cta_err, 60 + wg)) return;
       tc_fence_after_sync();
@@ -631,7 +637,8 @@ int launch_bwd_bf16(const void* q, const void* k, const void* v, const void* d_o
   const void* ptrs[6] = {q, k, v, d_o, dk, dv};
   for (int i = 0; i < 6; ++i) {
     const uint64_t heads = (i == 0 || i == 3) ? BH : BH_kv;
-    if (make_map_3d(&maps[i], ptrs[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.N, p.D, kT, 64) != 0) {
+    const uint64_t rows = (i == 0 || i == 3) ? p.N : p.key_rows();
+    if (make_map_3d(&maps[i], ptrs[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, rows, p.D, kT, 64) != 0) {
       *cuda_err = cudaErrorInvalidValue;
       return SIGATTN_ERR_CUDA;
     }
@@ -647,7 +654,9 @@ int launch_bwd_bf16(const void* q, const void* k, const void* v, const void* d_o
   bp.group = p.H / p.kv_heads();
   bp.N = p.N;
   bp.n_tiles = (p.N + kT - 1) / kT;
-  bp.n_items = bp.n_tiles * bp.BH;
+  bp.n_tiles_k = (p.key_rows() + kT - 1) / kT;
+  bp.pos0 = p.key_rows() - p.N;
+  bp.n_items = bp.n_tiles_k * bp.BH;
   bp.scale = p.scale;
   bp.scale_log2e = p.scale * kLog2eB;
   bp.bias_log2e = p.bias * kLog2eB;

@@ -4,6 +4,9 @@
 // nothing is shared between blocks, so every tensor output is deterministic (the optional
 // bias gradient is a sum over all blocks of a head and is added with fp32 atomics).
 //
+// N counts query rows, N_k key/value rows; the queries sit at the last N positions, so query
+// i has position i + off with off = N_k - N (0 for self-attention).
+//
 // Forward: Eq. 3 / Algorithm 1.  Backward: the sigmoid column of the forward/backward
 // table in Appendix F.1 / Algorithm 2, with the factor scale = 1/sqrt(d) in dQ and dK.
 #include "sigattn_internal.h"
@@ -30,24 +33,25 @@ __device__ __forceinline__ float dot_row(const float* __restrict__ a_smem, const
 __global__ void fwd_fp32_kernel(const float* __restrict__ q, const float* __restrict__ k,
                                 const float* __restrict__ v, float* __restrict__ o, int H, int N, int D,
                                 float scale, float bias, int causal, const float* __restrict__ slopes,
-                                const float* __restrict__ bias_vec, int H_kv) {
+                                const float* __restrict__ bias_vec, int H_kv, int N_k) {
   __shared__ float sq[128];
   __shared__ float sp[kThreads];
+  const int off = N_k - N;
   const int i = blockIdx.x, bh = blockIdx.y, t = threadIdx.x;
   if (bias_vec) bias = bias_vec[bh];
   const size_t base = static_cast<size_t>(bh) * N * D;
-  const size_t kv_base = static_cast<size_t>((bh / H) * H_kv + (bh % H) / (H / H_kv)) * N * D;
+  const size_t kv_base = static_cast<size_t>((bh / H) * H_kv + (bh % H) / (H / H_kv)) * N_k * D;
   const float slope = slopes ? slopes[bh % H] : 0.0f;
   if (t < D) sq[t] = q[base + static_cast<size_t>(i) * D + t];
   __syncthreads();
-  const int jend = causal ? i + 1 : N;
+  const int jend = causal ? min(N_k, i + off + 1) : N_k;
   float acc = 0.0f;
   for (int j0 = 0; j0 < jend; j0 += kThreads) {
     const int j = j0 + t;
     float p = 0.0f;
     if (j < jend) {
       const float s = dot_row(sq, k + kv_base + static_cast<size_t>(j) * D, D);
-      const float x = fmaf(scale, s, bias) - slope * fabsf(static_cast<float>(i - j));
+      const float x = fmaf(scale, s, bias) - slope * fabsf(static_cast<float>(i + off - j));
       p = sigmoid_exact(x);
     }
     sp[t] = p;
@@ -66,13 +70,15 @@ __global__ void bwd_dq_fp32_kernel(const float* __restrict__ q, const float* __r
                                    const float* __restrict__ v, const float* __restrict__ d_o,
                                    float* __restrict__ dq, int H, int N, int D, float scale, float bias,
                                    int causal, const float* __restrict__ slopes,
-                                   const float* __restrict__ bias_vec, float* __restrict__ dbias, int H_kv) {
+                                   const float* __restrict__ bias_vec, float* __restrict__ dbias, int H_kv,
+                                   int N_k) {
+  const int off = N_k - N;
   __shared__ float sq[128];
   __shared__ float sdo[128];
   __shared__ float sds[kThreads];
   const int i = blockIdx.x, bh = blockIdx.y, t = threadIdx.x;
   if (bias_vec) bias = bias_vec[bh];
-  const size_t kv_base = static_cast<size_t>((bh / H) * H_kv + (bh % H) / (H / H_kv)) * N * D;
+  const size_t kv_base = static_cast<size_t>((bh / H) * H_kv + (bh % H) / (H / H_kv)) * N_k * D;
   float ds_sum = 0.0f;   // this thread's share of sum_j dS_ij
   const size_t base = static_cast<size_t>(bh) * N * D;
   const float slope = slopes ? slopes[bh % H] : 0.0f;
@@ -81,14 +87,14 @@ __global__ void bwd_dq_fp32_kernel(const float* __restrict__ q, const float* __r
     sdo[t] = d_o[base + static_cast<size_t>(i) * D + t];
   }
   __syncthreads();
-  const int jend = causal ? i + 1 : N;
+  const int jend = causal ? min(N_k, i + off + 1) : N_k;
   float acc = 0.0f;
   for (int j0 = 0; j0 < jend; j0 += kThreads) {
     const int j = j0 + t;
     float ds = 0.0f;
     if (j < jend) {
       const float s = dot_row(sq, k + kv_base + static_cast<size_t>(j) * D, D);
-      const float x = fmaf(scale, s, bias) - slope * fabsf(static_cast<float>(i - j));
+      const float x = fmaf(scale, s, bias) - slope * fabsf(static_cast<float>(i + off - j));
       const float dp = dot_row(sdo, v + kv_base + static_cast<size_t>(j) * D, D);
       ds = sigmoid_slope(x) * dp;
     }
@@ -119,20 +125,21 @@ __global__ void bwd_dkdv_fp32_kernel(const float* __restrict__ q, const float* _
                                      const float* __restrict__ v, const float* __restrict__ d_o,
                                      float* __restrict__ dk, float* __restrict__ dv, int H, int N, int D,
                                      float scale, float bias_scalar, int causal, const float* __restrict__ slopes,
-                                     const float* __restrict__ bias_vec, int H_kv) {
+                                     const float* __restrict__ bias_vec, int H_kv, int N_k) {
+  const int off = N_k - N;
   __shared__ float sk[128];
   __shared__ float sv[128];
   __shared__ float sp[kThreads];
   __shared__ float sds[kThreads];
   const int j = blockIdx.x, bh_kv = blockIdx.y, t = threadIdx.x;
   const int group = H / H_kv;
-  const size_t kv_base = static_cast<size_t>(bh_kv) * N * D;
+  const size_t kv_base = static_cast<size_t>(bh_kv) * N_k * D;
   if (t < D) {
     sk[t] = k[kv_base + static_cast<size_t>(j) * D + t];
     sv[t] = v[kv_base + static_cast<size_t>(j) * D + t];
   }
   __syncthreads();
-  const int ibeg = causal ? j : 0;
+  const int ibeg = causal ? max(0, j - off) : 0;
   float acc_k = 0.0f, acc_v = 0.0f;
   for (int g = 0; g < group; ++g) {
     const int bh = (bh_kv / H_kv) * H + (bh_kv % H_kv) * group + g;   // query head
@@ -144,7 +151,7 @@ __global__ void bwd_dkdv_fp32_kernel(const float* __restrict__ q, const float* _
       float p = 0.0f, ds = 0.0f;
       if (i < N) {
         const float s = dot_row(sk, q + base + static_cast<size_t>(i) * D, D);
-        const float x = fmaf(scale, s, bias) - slope * fabsf(static_cast<float>(i - j));
+        const float x = fmaf(scale, s, bias) - slope * fabsf(static_cast<float>(i + off - j));
         p = sigmoid_exact(x);
         const float dp = dot_row(sv, d_o + base + static_cast<size_t>(i) * D, D);
         ds = sigmoid_slope(x) * dp;
@@ -175,7 +182,7 @@ int launch_fwd_fp32(const float* q, const float* k, const float* v, float* o, co
                     cudaStream_t stream, unsigned long long* launches, cudaError_t* cuda_err) {
   dim3 grid(p.N, p.B * p.H);
   fwd_fp32_kernel<<<grid, kThreads, 0, stream>>>(q, k, v, o, p.H, p.N, p.D, p.scale, p.bias, p.causal, p.slopes,
-                                                 p.bias_vec, p.kv_heads());
+                                                 p.bias_vec, p.kv_heads(), p.key_rows());
   *launches += 1;
   *cuda_err = cudaGetLastError();
   return *cuda_err == cudaSuccess ? SIGATTN_OK : SIGATTN_ERR_CUDA;
@@ -190,10 +197,10 @@ int launch_bwd_fp32(const float* q, const float* k, const float* v, const float*
     if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
   }
   bwd_dq_fp32_kernel<<<grid, kThreads, 0, stream>>>(q, k, v, d_o, dq, p.H, p.N, p.D, p.scale, p.bias, p.causal,
-                                                    p.slopes, p.bias_vec, p.dbias, p.kv_heads());
-  dim3 grid_kv(p.N, p.B * p.kv_heads());
+                                                    p.slopes, p.bias_vec, p.dbias, p.kv_heads(), p.key_rows());
+  dim3 grid_kv(p.key_rows(), p.B * p.kv_heads());
   bwd_dkdv_fp32_kernel<<<grid_kv, kThreads, 0, stream>>>(q, k, v, d_o, dk, dv, p.H, p.N, p.D, p.scale, p.bias,
-                                                         p.causal, p.slopes, p.bias_vec, p.kv_heads());
+                                                         p.causal, p.slopes, p.bias_vec, p.kv_heads(), p.key_rows());
   *launches += 2;
   *cuda_err = cudaGetLastError();
   return *cuda_err == cudaSuccess ? SIGATTN_OK : SIGATTN_ERR_CUDA;

@@ -82,7 +82,8 @@ struct FwdBarriers {
 };
 
 struct FwdParams {
-  int BH, H, N;
+  int BH, H, N;     // N counts query rows
+  int pos0;         // position of query row 0: rows of K, V minus N (0 for self-attention)
   int H_kv, group;  // heads of K, V and query heads per key/value head (H = H_kv * group)
   int n_pairs;     // ceil(N / 256)
   int n_kv_total;  // ceil(N / 128)
@@ -120,7 +121,8 @@ __device__ __forceinline__ Item decode_item(const FwdParams& p, int item) {
 #pragma unroll
   for (int t = 0; t < 2; ++t) {
     const int r = w.row0 + t * kBM;
-    w.n[t] = (r >= p.N) ? 0 : (CAUSAL ? min(p.n_kv_total, r / kBN + 1) : p.n_kv_total);
+    // causal: the tile's last row, at position r + 127 + pos0, sees keys up to that position
+    w.n[t] = (r >= p.N) ? 0 : (CAUSAL ? min(p.n_kv_total, (r + kBM - 1 + p.pos0) / kBN + 1) : p.n_kv_total);
   }
   w.n_kv = max(w.n[0], w.n[1]);
   return w;
@@ -357,8 +359,11 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
         if (!mbar_wait(smem_u32(&bars->s_full[t]), cnt & 1, cta_err, 30 + t)) return;
         ++cnt;
         tc_fence_after_sync();
-        const float row_rel = static_cast<float>(w.row0 + t * kBM + tid - j * kBN);
-        const bool diag = CAUSAL && (j == w.n[t] - 1);
+        // position of this thread's query relative to the first key of the tile
+        const float row_rel = static_cast<float>(w.row0 + t * kBM + tid + p.pos0 - j * kBN);
+        // the mask cuts through every key tile that reaches beyond the position of the tile's
+        // first row: the last one, and with pos0 not a multiple of 128 also the one before
+        const bool diag = CAUSAL && ((j + 1) * kBN - 1 > w.row0 + t * kBM + p.pos0);
         // bf16 P goes back over the first half of the columns this thread has just read
         const uint32_t tS = tmem + t * kBN + lane_off + g * kCols;
         uint32_t sv[kCols];
@@ -521,7 +526,8 @@ int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const 
   CUtensorMap* maps[4] = {&tmQ, &tmK, &tmV, &tmO};
   for (int i = 0; i < 4; ++i) {
     const uint64_t heads = (i == 1 || i == 2) ? BH_kv : BH;
-    if (make_map_3d(maps[i], ptrs[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, p.N, p.D, kBM, 64) != 0) {
+    const uint64_t rows = (i == 1 || i == 2) ? p.key_rows() : p.N;
+    if (make_map_3d(maps[i], ptrs[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, rows, p.D, kBM, 64) != 0) {
       *cuda_err = cudaErrorInvalidValue;
       return SIGATTN_ERR_CUDA;
     }
@@ -532,8 +538,9 @@ int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const 
   fp.H_kv = p.kv_heads();
   fp.group = p.H / p.kv_heads();
   fp.N = p.N;
+  fp.pos0 = p.key_rows() - p.N;
   fp.n_pairs = (p.N + 2 * kBM - 1) / (2 * kBM);
-  fp.n_kv_total = (p.N + kBN - 1) / kBN;
+  fp.n_kv_total = (p.key_rows() + kBN - 1) / kBN;
   fp.n_items = fp.n_pairs * fp.BH;
   fp.scale_log2e = p.scale * kLog2e;
   fp.bias_log2e = p.bias * kLog2e;

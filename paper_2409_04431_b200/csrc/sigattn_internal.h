@@ -16,6 +16,8 @@ struct Problem {
   float* dbias;           // backward only: device pointer to B*H floats that receive sum dS, or nullptr
   int H_kv;               // heads of k, v (H is a multiple of it; query head h reads head h / (H / H_kv)); 0 = H
   int kv_heads() const { return H_kv > 0 ? H_kv : H; }
+  int N_k;                // rows of k, v (N counts the rows of q); 0 = N.  The queries sit at the last N positions.
+  int key_rows() const { return N_k > 0 ? N_k : N; }
 };
 
 // Every launcher enqueues on `stream`, adds the number of kernels it launched to
