@@ -85,6 +85,12 @@ struct FwdParams {
   int BH, H, N;     // N counts query rows
   int pos0;         // position of query row 0: rows of K, V minus N (0 for self-attention)
   int H_kv, group;  // heads of K, V and query heads per key/value head (H = H_kv * group)
+  // Packed grouped heads (few queries per head, e.g. decoding): the rows of all `pack_group`
+  // query heads of one key/value head form ONE sequence of pack_group * pack_rows rows, row r
+  // belonging to head r / pack_rows, query r % pack_rows, so that K and V are streamed once per
+  // group instead of once per query head.  Then BH counts (batch, key/value head) pairs, N is
+  // pack_group * pack_rows and H = H_kv, group = 1 for the producer.  0 = not packed.
+  int pack_rows, pack_group;
   int n_pairs;     // ceil(N / 256)
   int n_kv_total;  // ceil(N / 128)
   int n_items;
@@ -122,7 +128,9 @@ __device__ __forceinline__ Item decode_item(const FwdParams& p, int item) {
   for (int t = 0; t < 2; ++t) {
     const int r = w.row0 + t * kBM;
     // causal: the tile's last row, at position r + 127 + pos0, sees keys up to that position
-    w.n[t] = (r >= p.N) ? 0 : (CAUSAL ? min(p.n_kv_total, (r + kBM - 1 + p.pos0) / kBN + 1) : p.n_kv_total);
+    // (packed rows: every tile holds last queries of some head, so every key tile is visited)
+    w.n[t] = (r >= p.N) ? 0
+             : ((CAUSAL && p.pack_rows == 0) ? min(p.n_kv_total, (r + kBM - 1 + p.pos0) / kBN + 1) : p.n_kv_total);
   }
   w.n_kv = max(w.n[0], w.n[1]);
   return w;
@@ -333,7 +341,7 @@ __device__ __forceinline__ void sigmoid_cols(const uint32_t (&s)[kCols], uint32_
 // of the tile.  While the groups evaluate one tile, the tensor pipe runs
 // P V and the next logits of the other one, so the MUFU pipe and the tensor pipe take turns
 // on a tile instead of competing for it.
-template <int D, bool CAUSAL, bool ALIBI>
+template <int D, bool CAUSAL, bool ALIBI, bool PACKED>
 __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t* smem, uint32_t tmem,
                              FwdBarriers* bars, volatile int* cta_err) {
   using L = FwdSmem<D>;
@@ -346,9 +354,22 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
     const int item = snake_rank(round, p.n_items);
     if (item < 0) continue;
     const Item w = decode_item<CAUSAL>(p, item);
-    float slope_log2e = 0.0f;
-    if (ALIBI) slope_log2e = p.slopes[w.bh % p.H] * kLog2e;
-    const float bias_log2e = p.bias_vec ? __ldg(p.bias_vec + w.bh) * kLog2e : p.bias_log2e;
+    // Per item, or with packed heads per row (one value for each of the two tiles): slope, bias
+    // and the position of this thread's query row.
+    float slope_t[2] = {0.0f, 0.0f}, bias_t[2], pos_t[2];
+#pragma unroll
+    for (int t = 0; t < 2; ++t) {
+      const int r = w.row0 + t * kBM + tid;
+      int head = w.bh, i = r;   // query head (index into [B][H]) and query index within the head
+      if (PACKED) {
+        const int g_head = min(r / p.pack_rows, p.pack_group - 1);   // rows past the end only fill the tile
+        i = r - g_head * p.pack_rows;
+        head = w.bh * p.pack_group + g_head;                        // (b * H_kv + h_kv) * group + g = b * H + h
+      }
+      if (ALIBI) slope_t[t] = p.slopes[head % (PACKED ? p.H * p.pack_group : p.H)] * kLog2e;
+      bias_t[t] = p.bias_vec ? __ldg(p.bias_vec + head) * kLog2e : p.bias_log2e;
+      pos_t[t] = static_cast<float>(i + p.pos0);
+    }
 
     // Tile-steps are visited in the order (j, tile 0), (j, tile 1), (j + 1, tile 0), ...
     for (int j = 0; j < w.n_kv; ++j) {
@@ -360,10 +381,11 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
         ++cnt;
         tc_fence_after_sync();
         // position of this thread's query relative to the first key of the tile
-        const float row_rel = static_cast<float>(w.row0 + t * kBM + tid + p.pos0 - j * kBN);
+        const float row_rel = pos_t[t] - static_cast<float>(j * kBN);
         // the mask cuts through every key tile that reaches beyond the position of the tile's
         // first row: the last one, and with pos0 not a multiple of 128 also the one before
-        const bool diag = CAUSAL && ((j + 1) * kBN - 1 > w.row0 + t * kBM + p.pos0);
+        // (packed rows: a tile may hold a head's first query, at position pos0)
+        const bool diag = CAUSAL && ((j + 1) * kBN - 1 > (PACKED ? 0 : w.row0 + t * kBM) + p.pos0);
         // bf16 P goes back over the first half of the columns this thread has just read
         const uint32_t tS = tmem + t * kBN + lane_off + g * kCols;
         uint32_t sv[kCols];
@@ -371,7 +393,7 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
         tmem_wait_ld();
         uint32_t pk[kCols / 2];
         constexpr int kEmulateEvery = (D == 128) ? SIGATTN_FWD_EMULATE_D128 : SIGATTN_FWD_EMULATE_D64;
-        sigmoid_cols<ALIBI, kEmulateEvery>(sv, pk, p.scale_log2e, bias_log2e, slope_log2e, row_rel, g * kCols,
+        sigmoid_cols<ALIBI, kEmulateEvery>(sv, pk, p.scale_log2e, bias_t[t], slope_t[t], row_rel, g * kCols,
                                            diag);
         tmem_st_cols(tS, pk);
         tmem_wait_st();
@@ -428,7 +450,7 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
 
 // ------------------------------------------------------------------ kernel
 
-template <int D, bool CAUSAL, bool ALIBI>
+template <int D, bool CAUSAL, bool ALIBI, bool PACKED>
 __global__ void __launch_bounds__(kFwdThreads, 1)
 sigattn_fwd_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                         const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
@@ -481,7 +503,7 @@ sigattn_fwd_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
     fwd_mma_role<D, CAUSAL>(p, smem_base, tmem, &bars, &cta_err);
     __syncwarp();
   } else {
-    fwd_act_role<D, CAUSAL, ALIBI>(p, &tmO, smem, tmem, &bars, &cta_err);
+    fwd_act_role<D, CAUSAL, ALIBI, PACKED>(p, &tmO, smem, tmem, &bars, &cta_err);
   }
 
   tc_fence_before_sync();
@@ -493,10 +515,10 @@ sigattn_fwd_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
   if (warp == kMmaWarp) tmem_dealloc(tmem, 512);
 }
 
-template <int D, bool CAUSAL, bool ALIBI>
+template <int D, bool CAUSAL, bool ALIBI, bool PACKED>
 int launch_fwd_variant(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtensorMap& tmO,
                        const FwdParams& fp, int num_sms, cudaStream_t stream, cudaError_t* cuda_err) {
-  auto kernel = sigattn_fwd_bf16_kernel<D, CAUSAL, ALIBI>;
+  auto kernel = sigattn_fwd_bf16_kernel<D, CAUSAL, ALIBI, PACKED>;
   static bool configured = false;
   if (!configured) {
     *cuda_err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdSmem<D>::kDynBytes);
@@ -521,25 +543,33 @@ int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const 
 
   const uint64_t BH = static_cast<uint64_t>(p.B) * p.H;
   const uint64_t BH_kv = static_cast<uint64_t>(p.B) * p.kv_heads();
+  const int group = p.H / p.kv_heads();
+  // Few queries per head and several query heads per key/value head (decoding with grouped
+  // heads): pack the group's rows into one sequence so that K and V are streamed once per group.
+  const bool packed = group > 1 && static_cast<long long>(p.N) * group <= 2 * kBM;
+  const uint64_t q_heads = packed ? BH_kv : BH;
+  const uint64_t q_rows = packed ? static_cast<uint64_t>(p.N) * group : p.N;
   CUtensorMap tmQ, tmK, tmV, tmO;
   const void* ptrs[4] = {q, k, v, o};
   CUtensorMap* maps[4] = {&tmQ, &tmK, &tmV, &tmO};
   for (int i = 0; i < 4; ++i) {
-    const uint64_t heads = (i == 1 || i == 2) ? BH_kv : BH;
-    const uint64_t rows = (i == 1 || i == 2) ? p.key_rows() : p.N;
-    if (make_map_3d(maps[i], ptrs[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads, rows, p.D, kBM, 64) != 0) {
+    const bool kv = (i == 1 || i == 2);
+    if (make_map_3d(maps[i], ptrs[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, kv ? BH_kv : q_heads,
+                    kv ? p.key_rows() : q_rows, p.D, kBM, 64) != 0) {
       *cuda_err = cudaErrorInvalidValue;
       return SIGATTN_ERR_CUDA;
     }
   }
   FwdParams fp;
-  fp.BH = static_cast<int>(BH);
-  fp.H = p.H;
+  fp.BH = static_cast<int>(q_heads);
+  fp.H = packed ? p.kv_heads() : p.H;
   fp.H_kv = p.kv_heads();
-  fp.group = p.H / p.kv_heads();
-  fp.N = p.N;
+  fp.group = packed ? 1 : group;
+  fp.pack_rows = packed ? p.N : 0;
+  fp.pack_group = packed ? group : 1;
+  fp.N = static_cast<int>(q_rows);
   fp.pos0 = p.key_rows() - p.N;
-  fp.n_pairs = (p.N + 2 * kBM - 1) / (2 * kBM);
+  fp.n_pairs = (fp.N + 2 * kBM - 1) / (2 * kBM);
   fp.n_kv_total = (p.key_rows() + kBN - 1) / kBN;
   fp.n_items = fp.n_pairs * fp.BH;
   fp.scale_log2e = p.scale * kLog2e;
@@ -550,8 +580,9 @@ int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const 
 
   int rc;
   const bool alibi = p.slopes != nullptr;
-#define SIGATTN_FWD_CASE(DD, CC, AA) \
-  rc = launch_fwd_variant<DD, CC, AA>(tmQ, tmK, tmV, tmO, fp, num_sms, stream, cuda_err)
+#define SIGATTN_FWD_CASE(DD, CC, AA)                                                                       \
+  rc = packed ? launch_fwd_variant<DD, CC, AA, true>(tmQ, tmK, tmV, tmO, fp, num_sms, stream, cuda_err)    \
+              : launch_fwd_variant<DD, CC, AA, false>(tmQ, tmK, tmV, tmO, fp, num_sms, stream, cuda_err)
   if (p.D == 128) {
     if (p.causal) { if (alibi) SIGATTN_FWD_CASE(128, true, true); else SIGATTN_FWD_CASE(128, true, false); }
     else          { if (alibi) SIGATTN_FWD_CASE(128, false, true); else SIGATTN_FWD_CASE(128, false, false); }

@@ -49,6 +49,41 @@ def test_nk_bf16(B, H, H_kv, N_q, N_k, D, causal, with_slopes):
     assert rel_fro(db.cpu().numpy().astype(np.float64), ref_db) < BF16_REL_FRO
 
 
+@pytest.mark.parametrize("B,H,H_kv,N_q,N_k,D,causal,with_slopes", [
+    (2, 8, 2, 1, 1000, 128, True, False),     # decoding with grouped heads: 4 rows per key/value head
+    (1, 8, 1, 3, 500, 64, True, True),        # multi-query, 24 packed rows, slopes per query head
+    (1, 4, 1, 64, 300, 128, True, False),     # 256 packed rows: both tiles of one item
+    (1, 4, 1, 65, 300, 128, True, False),     # 260 rows: one too many, the unpacked path
+    (1, 6, 3, 20, 100, 64, False, True),      # packed, no mask, position bias
+])
+def test_nk_grouped_heads_packed_forward(B, H, H_kv, N_q, N_k, D, causal, with_slopes):
+    """With few queries per head the forward packs the query heads of a key/value head into
+    the rows of one tile; each packed row keeps its own head's slope and bias and its own
+    position."""
+    import torch
+    import paper_2409_04431_b200 as sa
+    q, k, v, _ = _case(B, H, H_kv, N_q, N_k, D, 91)
+    slopes = (0.5 ** np.arange(1, H + 1)).astype(np.float32) if with_slopes else None
+    bias = (-math.log(N_k) + 0.3 * np.random.default_rng(92).standard_normal((B, H))).astype(np.float32)
+    tq, tk, tv = (to_device(t, "bf16") for t in (q, k, v))
+    sl = None if slopes is None else torch.from_numpy(slopes).cuda()
+    scale = 1.0 / math.sqrt(D)
+    o = sa.sigattn_fwd_nk(tq, tk, tv, scale, torch.from_numpy(bias).cuda(), causal, sl)
+    sa.sigattn_check()
+    ref = oracle.sigattn_fwd(q, k, v, scale, bias.astype(np.float64), causal, slopes)
+    g = to_host(o)
+    assert np.isfinite(g).all()
+    assert rel_fro(g, ref) < BF16_REL_FRO, rel_fro(g, ref)
+    assert max_abs(g, ref) < 2e-2 * max(1.0, float(np.abs(ref).max()))
+    # every head on its own (one head per group is never packed) gives the same rows
+    for h in range(H):
+        hk = h // (H // H_kv)
+        one = sa.sigattn_fwd_nk(tq[:, h:h + 1].contiguous(), tk[:, hk:hk + 1].contiguous(), tv[:, hk:hk + 1].contiguous(),
+                                scale, torch.from_numpy(bias[:, h:h + 1].copy()).cuda(), causal,
+                                None if sl is None else sl[h:h + 1].contiguous())
+        assert torch.equal(one, o[:, h:h + 1])
+
+
 def test_nk_fp32_debug_path():
     import paper_2409_04431_b200 as sa
     B, H, H_kv, N_q, N_k, D = 1, 4, 2, 37, 150, 64
