@@ -53,6 +53,13 @@ Readings of the paper taken here
     i + N_k - N_q for the causal mask (keys j <= i + N_k - N_q are kept) and for the
     position bias.  N_q = N_k is the paper's case.  Without a causal mask and without
     slopes the positions play no role and any N_q, N_k are allowed (cross-attention).
+  * Keys and values split into contiguous shards (over devices, or over thread blocks):
+    sigmoid attention has no row normalisation, so O is the plain sum over shards of the
+    attention of all queries against one shard, dQ likewise, and dK, dV of a shard need only
+    that shard (the distributed setting the paper leaves open in its Limitations).  A shard
+    call must place the queries relative to ITS first key: `pos0` is the position of query
+    row 0 minus the position of the shard's first key (default N_k - N_q as above) and may
+    be negative; a query that lies before every key of the shard gets weight 0 everywhere.
 
 Every function is pinned by tests that do not call back into this file's own
 formulae (closed forms, brute-force loops, finite differences, the paper's second
@@ -89,41 +96,49 @@ def sigmoid(x):
     return out
 
 
-def causal_mask(n: int, i0: int = 0, i1: int | None = None, n_q: int | None = None):
+def _query_offset(n, n_q, pos0):
+    """Position of query row 0 relative to key 0: given, or n - n_q (queries at the end)."""
+    n_q = n if n_q is None else n_q
+    return n_q, (n - n_q if pos0 is None else int(pos0))
+
+
+def causal_mask(n: int, i0: int = 0, i1: int | None = None, n_q: int | None = None, pos0: int | None = None):
     """Rows i0..i1-1 of the n x n lower-triangular 0/1 matrix, diagonal included
     (the matrix M printed for n = 3 in Appendix G's normalisation ablation).
 
-    With n_q query rows against n keys (n_q != n) query i sits at position i + n - n_q
-    (see the module header), so the row keeps keys j <= i + n - n_q."""
-    n_q = n if n_q is None else n_q
+    With n_q query rows against n keys query i sits at position i + pos0 relative to key
+    0 (pos0 = n - n_q unless given; see the module header), so the row keeps keys
+    j <= i + pos0; a row whose position lies before key 0 keeps none."""
+    n_q, off = _query_offset(n, n_q, pos0)
     i1 = n_q if i1 is None else i1
-    i = np.arange(i0, i1)[:, None] + (n - n_q)
+    i = np.arange(i0, i1)[:, None] + off
     j = np.arange(n)[None, :]
     return (j <= i).astype(np.float64)
 
 
-def position_bias(n: int, slope: float, i0: int = 0, i1: int | None = None, n_q: int | None = None):
+def position_bias(n: int, slope: float, i0: int = 0, i1: int | None = None, n_q: int | None = None,
+                  pos0: int | None = None):
     """Additive linear position bias -slope * |i - j| for rows i0..i1-1 (Appendix F.4
-    names ALiBi; see the module header for the reading); with n_q != n query rows the
-    distance is taken from the query's position i + n - n_q."""
-    n_q = n if n_q is None else n_q
+    names ALiBi; see the module header for the reading); the distance is taken from the
+    query's position i + pos0 (pos0 = n - n_q unless given)."""
+    n_q, off = _query_offset(n, n_q, pos0)
     i1 = n_q if i1 is None else i1
-    i = np.arange(i0, i1, dtype=np.float64)[:, None] + float(n - n_q)
+    i = np.arange(i0, i1, dtype=np.float64)[:, None] + float(off)
     j = np.arange(n, dtype=np.float64)[None, :]
     return -float(slope) * np.abs(i - j)
 
 
-def attention_weights(q, k, scale, bias, causal, slope=0.0, i0=0, i1=None):
+def attention_weights(q, k, scale, bias, causal, slope=0.0, i0=0, i1=None, pos0=None):
     """P for query rows i0..i1-1 of one head: sigmoid(scale * q k^T + b + position
     bias), times the causal mask.  q: [n_q, d], k: [n, d] float64."""
     n_q, n = q.shape[0], k.shape[0]
     i1 = n_q if i1 is None else i1
     x = scale * (q[i0:i1] @ k.T) + bias
     if slope != 0.0:
-        x = x + position_bias(n, slope, i0, i1, n_q)
+        x = x + position_bias(n, slope, i0, i1, n_q, pos0)
     p = sigmoid(x)
     if causal:
-        p = p * causal_mask(n, i0, i1, n_q)
+        p = p * causal_mask(n, i0, i1, n_q, pos0)
     return p
 
 
@@ -164,12 +179,13 @@ def _row_ranges(n, row_block):
     return [(a, min(n, a + step)) for a in range(0, n, step)]
 
 
-def sigattn_fwd(q, k, v, scale, bias, causal=False, alibi_slopes=None, row_block=None):
+def sigattn_fwd(q, k, v, scale, bias, causal=False, alibi_slopes=None, row_block=None, pos0=None):
     """O = sigmoid(scale * Q K^T + b [+ position bias]) [* causal mask] V  (Eq. 3).
 
     q: [B, H, N, D]; k, v: [B, H_kv, N, D] with H a multiple of H_kv (any float dtype;
     converted to float64).
     bias: scalar, or an array that broadcasts to [B, H] (one bias per sequence and head).
+    pos0: position of query row 0 relative to key row 0 (default: rows of k minus rows of q).
     Returns O as float64 [B, H, N, D].
     """
     q, k, v = _as_f64(q, k, v)
@@ -182,12 +198,12 @@ def sigattn_fwd(q, k, v, scale, bias, causal=False, alibi_slopes=None, row_block
         for h in range(H):
             hk = h // group
             for i0, i1 in _row_ranges(N, row_block):
-                p = attention_weights(q[b, h], k[b, hk], scale, bias_bh[b, h], causal, slopes[h], i0, i1)
+                p = attention_weights(q[b, h], k[b, hk], scale, bias_bh[b, h], causal, slopes[h], i0, i1, pos0)
                 o[b, h, i0:i1] = p @ v[b, hk]
     return o
 
 
-def _bwd_all(q, k, v, d_o, scale, bias, causal, alibi_slopes, row_block):
+def _bwd_all(q, k, v, d_o, scale, bias, causal, alibi_slopes, row_block, pos0=None):
     q, k, v, d_o = _as_f64(q, k, v, d_o)
     B, H, N, D = q.shape
     group = _kv_group(H, k)
@@ -201,7 +217,7 @@ def _bwd_all(q, k, v, d_o, scale, bias, causal, alibi_slopes, row_block):
         for h in range(H):
             hk = h // group
             for i0, i1 in _row_ranges(N, row_block):
-                p = attention_weights(q[b, h], k[b, hk], scale, bias_bh[b, h], causal, slopes[h], i0, i1)
+                p = attention_weights(q[b, h], k[b, hk], scale, bias_bh[b, h], causal, slopes[h], i0, i1, pos0)
                 do_rows = d_o[b, h, i0:i1]
                 dv[b, hk] += p.T @ do_rows
                 dp = do_rows @ v[b, hk].T
@@ -212,7 +228,7 @@ def _bwd_all(q, k, v, d_o, scale, bias, causal, alibi_slopes, row_block):
     return dq, dk, dv, dbias
 
 
-def sigattn_bwd(q, k, v, d_o, scale, bias, causal=False, alibi_slopes=None, row_block=None):
+def sigattn_bwd(q, k, v, d_o, scale, bias, causal=False, alibi_slopes=None, row_block=None, pos0=None):
     """Gradients of L = sum(O * dO) with respect to Q, K, V (sigmoid column of the
     forward/backward table in Appendix F.1, with the 1/sqrt(d) factor; see header).
 
@@ -220,17 +236,17 @@ def sigattn_bwd(q, k, v, d_o, scale, bias, causal=False, alibi_slopes=None, row_
     than q (see header).
     Returns (dQ, dK, dV), float64, shaped like q, k, v.
     """
-    return _bwd_all(q, k, v, d_o, scale, bias, causal, alibi_slopes, row_block)[:3]
+    return _bwd_all(q, k, v, d_o, scale, bias, causal, alibi_slopes, row_block, pos0)[:3]
 
 
-def sigattn_bwd_dbias(q, k, v, d_o, scale, bias, causal=False, alibi_slopes=None, row_block=None):
+def sigattn_bwd_dbias(q, k, v, d_o, scale, bias, causal=False, alibi_slopes=None, row_block=None, pos0=None):
     """Gradient of L = sum(O * dO) with respect to a bias held per (batch, head):
     db[b, h] = sum_ij dS_ij with dS = P (1 - P) dP as in sigattn_bwd (see header).  A
     bias shared by several heads or sequences gets the sum of their entries.
 
     Returns float64 [B, H].
     """
-    return _bwd_all(q, k, v, d_o, scale, bias, causal, alibi_slopes, row_block)[3]
+    return _bwd_all(q, k, v, d_o, scale, bias, causal, alibi_slopes, row_block, pos0)[3]
 
 
 def sigattn_fwd_sequence_form(q, k, v, scale, n_bias):

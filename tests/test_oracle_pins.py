@@ -489,3 +489,43 @@ def test_cross_attention_without_mask_brute_force():
             x[idx] = old
             fd[idx] = (lp - lm) / (2 * h)
         assert np.linalg.norm(fd - g) / np.linalg.norm(fd) < 1e-7, name
+
+
+# ------------------------------------------------------------------------- key/value shards
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_key_value_shards_sum_to_the_whole(causal):
+    """O and dQ are plain sums over contiguous key/value shards, dK and dV of a shard need
+    only that shard; each shard call places the queries relative to its own first key.  One
+    shard (entirely after some queries) is also checked element by element."""
+    B, H, N, D = 1, 2, 9, 3
+    q, k, v, d_o = (rnd((B, H, N, D), s) for s in (130, 131, 132, 133))
+    slopes = np.array([0.5, 0.125])
+    scale, b = 0.6, -0.8
+    o = oracle.sigattn_fwd(q, k, v, scale, b, causal, slopes)
+    dq, dk, dv = oracle.sigattn_bwd(q, k, v, d_o, scale, b, causal, slopes)
+    bounds = [0, 2, 5, 9]
+    o_sum, dq_sum = np.zeros_like(o), np.zeros_like(dq)
+    for lo, hi in zip(bounds[:-1], bounds[1:]):
+        ks, vs = k[:, :, lo:hi], v[:, :, lo:hi]
+        o_sum += oracle.sigattn_fwd(q, ks, vs, scale, b, causal, slopes, pos0=-lo)
+        g = oracle.sigattn_bwd(q, ks, vs, d_o, scale, b, causal, slopes, pos0=-lo)
+        dq_sum += g[0]
+        np.testing.assert_allclose(g[1], dk[:, :, lo:hi], rtol=1e-12, atol=1e-15)
+        np.testing.assert_allclose(g[2], dv[:, :, lo:hi], rtol=1e-12, atol=1e-15)
+    np.testing.assert_allclose(o_sum, o, rtol=1e-12, atol=1e-15)
+    np.testing.assert_allclose(dq_sum, dq, rtol=1e-12, atol=1e-15)
+    lo, hi = 5, 9   # the last shard: queries 0..4 lie before all of its keys when causal
+    part = oracle.sigattn_fwd(q, k[:, :, lo:hi], v[:, :, lo:hi], scale, b, causal, slopes, pos0=-lo)
+    ref = np.zeros_like(part)
+    for h in range(H):
+        for i in range(N):
+            for j in range(lo, hi):
+                if causal and j > i:
+                    continue
+                x = scale * float(q[0, h, i] @ k[0, h, j]) + b - slopes[h] * abs(i - j)
+                ref[0, h, i] += scalar_sigmoid(x) * v[0, h, j]
+    np.testing.assert_allclose(part, ref, rtol=1e-13, atol=1e-16)
+    if causal:
+        assert np.all(part[:, :, :lo] == 0.0)
