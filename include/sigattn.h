@@ -194,6 +194,30 @@ SIGATTN_API int sigattn_bwd_nk(const void* q, const void* k, const void* v, cons
                    float* dbias_bh,
                    void* workspace, size_t workspace_bytes, void* stream);
 
+/* One contiguous shard of keys and values (over devices, or over callers that split a long
+ * sequence).  Sigmoid attention has no row normalisation (Section 4), so O is the plain
+ * sum over shards of the attention of all queries against one shard, dQ likewise, and
+ * dK, dV of a shard need only that shard: the distributed setting the paper leaves open in
+ * its Limitations needs one sum per tensor and no log-sum-exp.  These are sigattn_fwd_nk /
+ * sigattn_bwd_nk with the position of the queries stated instead of implied: `pos0` is the
+ * position of query row 0 minus the position of the shard's first key (any value in
+ * +-2^30; N_k - N_q reproduces sigattn_fwd_nk).  Query i keeps keys j <= i + pos0 when
+ * causal = 1 and measures the ALiBi distance from i + pos0; a query that lies before every
+ * key of the shard gets an all-zero row of O (and contributes nothing to the gradients).
+ * The caller adds the summands (e.g. one all-reduce). */
+SIGATTN_API int sigattn_fwd_shard(const void* q, const void* k, const void* v, void* o,
+                      int B, int H, int H_kv, int N_q, int N_k, int D,
+                      float scale, float bias, const float* bias_bh, int causal, int pos0,
+                      const float* alibi_slopes, int dtype, void* stream);
+
+SIGATTN_API int sigattn_bwd_shard(const void* q, const void* k, const void* v, const void* d_o,
+                      void* dq, void* dk, void* dv,
+                      int B, int H, int H_kv, int N_q, int N_k, int D,
+                      float scale, float bias, const float* bias_bh, int causal, int pos0,
+                      const float* alibi_slopes, int dtype,
+                      float* dbias_bh,
+                      void* workspace, size_t workspace_bytes, void* stream);
+
 /* Bytes of scratch sigattn_bwd needs for this problem (0 for the fp32 debug path).
  * Returns 0 for invalid shapes as well; sigattn_bwd reports those. */
 SIGATTN_API size_t sigattn_bwd_workspace_bytes(int B, int H, int N, int D, int dtype);

@@ -31,6 +31,8 @@ _BINDING_NAMES = (
     "sigattn_bwd_gqa",
     "sigattn_fwd_nk",
     "sigattn_bwd_nk",
+    "sigattn_fwd_shard",
+    "sigattn_bwd_shard",
     "lib",
 )
 

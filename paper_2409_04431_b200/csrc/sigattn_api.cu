@@ -89,19 +89,22 @@ namespace {
 // Shared by the scalar-bias and the bias-vector entry points.
 // N counts query rows, N_k key/value rows; a causal mask needs N_k >= N (the queries are the last
 // N positions, so every query then sees at least one key).
-int check_lengths(int B, int H, int H_kv, int N, int N_k, int D, int causal) {
+// With pos0_given the caller states where the queries sit relative to key 0 (any value within
+// +-2^30; a query before every key then gets zeros), so the N_k >= N rule does not apply.
+int check_lengths(int B, int H, int H_kv, int N, int N_k, int D, int causal, int pos0_given, int pos0) {
   if (int rc = check_shape(B, H, N, D)) return rc;
   if (H_kv < 1 || H % H_kv != 0) return SIGATTN_ERR_SHAPE;
   if (int rc = check_shape(B, H_kv, N_k, D)) return rc;
-  if (causal == 1 && N_k < N) return SIGATTN_ERR_SHAPE;
+  if (!pos0_given && causal == 1 && N_k < N) return SIGATTN_ERR_SHAPE;
+  if (pos0_given && (pos0 > (1 << 30) || pos0 < -(1 << 30))) return SIGATTN_ERR_SHAPE;
   return SIGATTN_OK;
 }
 
 int fwd_any(const void* q, const void* k, const void* v, void* o, int B, int H, int H_kv, int N, int N_k, int D,
             float scale, float bias, const float* bias_vec, int causal, const float* alibi_slopes, int dtype,
-            void* stream) {
+            void* stream, int pos0_given = 0, int pos0 = 0) {
   if (!q || !k || !v || !o) return SIGATTN_ERR_NULL;
-  if (int rc = check_lengths(B, H, H_kv, N, N_k, D, causal)) return rc;
+  if (int rc = check_lengths(B, H, H_kv, N, N_k, D, causal, pos0_given, pos0)) return rc;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return SIGATTN_ERR_ALIGN;
   if (alibi_slopes && (reinterpret_cast<uintptr_t>(alibi_slopes) & 3u)) return SIGATTN_ERR_ALIGN;
   if (dtype != SIGATTN_DTYPE_BF16 && dtype != SIGATTN_DTYPE_FP32) return SIGATTN_ERR_FLAG;
@@ -109,7 +112,7 @@ int fwd_any(const void* q, const void* k, const void* v, void* o, int B, int H, 
   int dev = 0;
   int* status = nullptr;
   if (int rc = device_setup(&dev, &status)) return rc;
-  sigattn::Problem p{B, H, N, D, scale, bias, causal, alibi_slopes, bias_vec, nullptr, H_kv, N_k};
+  sigattn::Problem p{B, H, N, D, scale, bias, causal, alibi_slopes, bias_vec, nullptr, H_kv, N_k, pos0_given, pos0};
   unsigned long long launches = 0;
   cudaError_t ce = cudaSuccess;
   int rc;
@@ -127,9 +130,10 @@ int fwd_any(const void* q, const void* k, const void* v, void* o, int B, int H, 
 
 int bwd_any(const void* q, const void* k, const void* v, const void* d_o, void* dq, void* dk, void* dv, int B, int H,
             int H_kv, int N, int N_k, int D, float scale, float bias, const float* bias_vec, float* dbias, int causal,
-            const float* alibi_slopes, int dtype, void* workspace, size_t workspace_bytes, void* stream) {
+            const float* alibi_slopes, int dtype, void* workspace, size_t workspace_bytes, void* stream,
+            int pos0_given = 0, int pos0 = 0) {
   if (!q || !k || !v || !d_o || !dq || !dk || !dv) return SIGATTN_ERR_NULL;
-  if (int rc = check_lengths(B, H, H_kv, N, N_k, D, causal)) return rc;
+  if (int rc = check_lengths(B, H, H_kv, N, N_k, D, causal, pos0_given, pos0)) return rc;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(d_o) || !aligned16(dq) || !aligned16(dk) ||
       !aligned16(dv))
     return SIGATTN_ERR_ALIGN;
@@ -145,7 +149,7 @@ int bwd_any(const void* q, const void* k, const void* v, const void* d_o, void* 
   int dev = 0;
   int* status = nullptr;
   if (int rc = device_setup(&dev, &status)) return rc;
-  sigattn::Problem p{B, H, N, D, scale, bias, causal, alibi_slopes, bias_vec, dbias, H_kv, N_k};
+  sigattn::Problem p{B, H, N, D, scale, bias, causal, alibi_slopes, bias_vec, dbias, H_kv, N_k, pos0_given, pos0};
   unsigned long long launches = 0;
   cudaError_t ce = cudaSuccess;
   int rc;
@@ -230,6 +234,24 @@ int sigattn_bwd_nk(const void* q, const void* k, const void* v, const void* d_o,
     return SIGATTN_ERR_ALIGN;
   return bwd_any(q, k, v, d_o, dq, dk, dv, B, H, H_kv, N_q, N_k, D, scale, bias, bias_bh, dbias_bh, causal,
                  alibi_slopes, dtype, workspace, workspace_bytes, stream);
+}
+
+int sigattn_fwd_shard(const void* q, const void* k, const void* v, void* o, int B, int H, int H_kv, int N_q, int N_k,
+                      int D, float scale, float bias, const float* bias_bh, int causal, int pos0,
+                      const float* alibi_slopes, int dtype, void* stream) {
+  if (bias_bh && (reinterpret_cast<uintptr_t>(bias_bh) & 3u)) return SIGATTN_ERR_ALIGN;
+  return fwd_any(q, k, v, o, B, H, H_kv, N_q, N_k, D, scale, bias, bias_bh, causal, alibi_slopes, dtype, stream, 1,
+                 pos0);
+}
+
+int sigattn_bwd_shard(const void* q, const void* k, const void* v, const void* d_o, void* dq, void* dk, void* dv,
+                      int B, int H, int H_kv, int N_q, int N_k, int D, float scale, float bias, const float* bias_bh,
+                      int causal, int pos0, const float* alibi_slopes, int dtype, float* dbias_bh, void* workspace,
+                      size_t workspace_bytes, void* stream) {
+  if ((reinterpret_cast<uintptr_t>(bias_bh) & 3u) || (reinterpret_cast<uintptr_t>(dbias_bh) & 3u))
+    return SIGATTN_ERR_ALIGN;
+  return bwd_any(q, k, v, d_o, dq, dk, dv, B, H, H_kv, N_q, N_k, D, scale, bias, bias_bh, dbias_bh, causal,
+                 alibi_slopes, dtype, workspace, workspace_bytes, stream, 1, pos0);
 }
 
 int sigattn_bwd_set_timing_events(void* start_event, void* stop_event) {

@@ -71,7 +71,7 @@ struct BwdParams {
   int H_kv, group; // heads of K, V and query heads per key/value head (H = H_kv * group)
   int n_tiles;    // query tiles: ceil(N / 128), N = rows of Q
   int n_tiles_k;  // key tiles: ceil(rows of K / 128)
-  int pos0;       // position of query row 0: rows of K, V minus N (0 for self-attention)
+  int pos0;       // position of query row 0 relative to key row 0 (see FwdParams of the forward)
   int n_items;
   float scale, scale_log2e, bias_log2e;
   const float* bias_vec;   // one bias per (batch, head) instead of the scalar, or nullptr
@@ -108,7 +108,8 @@ __device__ __forceinline__ BwdItem decode_bwd_item(const BwdParams& p, int item)
   w.bh = item - w.j * p.BH;
   w.bh_q0 = GROUPED ? (w.bh / p.H_kv) * p.H + (w.bh % p.H_kv) * p.group : w.bh;
   // causal: the first query tile whose last row, at position 128 i + 127 + pos0, reaches key 128 j
-  w.i_begin = CAUSAL ? max(0, (w.j * kT - p.pos0) / kT) : 0;
+  // (a key tile that lies after every query still visits the last query tile, fully masked: zeros)
+  w.i_begin = CAUSAL ? min(p.n_tiles - 1, max(0, (w.j * kT - p.pos0) / kT)) : 0;
   w.n = p.n_tiles - w.i_begin;
   w.steps = GROUPED ? p.group * w.n : w.n;
   return w;
@@ -655,7 +656,7 @@ int launch_bwd_bf16(const void* q, const void* k, const void* v, const void* d_o
   bp.N = p.N;
   bp.n_tiles = (p.N + kT - 1) / kT;
   bp.n_tiles_k = (p.key_rows() + kT - 1) / kT;
-  bp.pos0 = p.key_rows() - p.N;
+  bp.pos0 = p.query_pos0();
   bp.n_items = bp.n_tiles_k * bp.BH;
   bp.scale = p.scale;
   bp.scale_log2e = p.scale * kLog2eB;

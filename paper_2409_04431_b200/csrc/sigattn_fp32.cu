@@ -4,8 +4,9 @@
 // nothing is shared between blocks, so every tensor output is deterministic (the optional
 // bias gradient is a sum over all blocks of a head and is added with fp32 atomics).
 //
-// N counts query rows, N_k key/value rows; the queries sit at the last N positions, so query
-// i has position i + off with off = N_k - N (0 for self-attention).
+// N counts query rows, N_k key/value rows; query i has position i + off relative to key 0
+// (off = N_k - N when the queries are the last N positions, 0 for self-attention; any value,
+// also negative, for a shard of keys and values).
 //
 // Forward: Eq. 3 / Algorithm 1.  Backward: the sigmoid column of the forward/backward
 // table in Appendix F.1 / Algorithm 2, with the factor scale = 1/sqrt(d) in dQ and dK.
@@ -33,10 +34,9 @@ __device__ __forceinline__ float dot_row(const float* __restrict__ a_smem, const
 __global__ void fwd_fp32_kernel(const float* __restrict__ q, const float* __restrict__ k,
                                 const float* __restrict__ v, float* __restrict__ o, int H, int N, int D,
                                 float scale, float bias, int causal, const float* __restrict__ slopes,
-                                const float* __restrict__ bias_vec, int H_kv, int N_k) {
+                                const float* __restrict__ bias_vec, int H_kv, int N_k, int off) {
   __shared__ float sq[128];
   __shared__ float sp[kThreads];
-  const int off = N_k - N;
   const int i = blockIdx.x, bh = blockIdx.y, t = threadIdx.x;
   if (bias_vec) bias = bias_vec[bh];
   const size_t base = static_cast<size_t>(bh) * N * D;
@@ -44,7 +44,7 @@ __global__ void fwd_fp32_kernel(const float* __restrict__ q, const float* __rest
   const float slope = slopes ? slopes[bh % H] : 0.0f;
   if (t < D) sq[t] = q[base + static_cast<size_t>(i) * D + t];
   __syncthreads();
-  const int jend = causal ? min(N_k, i + off + 1) : N_k;
+  const int jend = causal ? max(0, min(N_k, i + off + 1)) : N_k;
   float acc = 0.0f;
   for (int j0 = 0; j0 < jend; j0 += kThreads) {
     const int j = j0 + t;
@@ -71,8 +71,7 @@ __global__ void bwd_dq_fp32_kernel(const float* __restrict__ q, const float* __r
                                    float* __restrict__ dq, int H, int N, int D, float scale, float bias,
                                    int causal, const float* __restrict__ slopes,
                                    const float* __restrict__ bias_vec, float* __restrict__ dbias, int H_kv,
-                                   int N_k) {
-  const int off = N_k - N;
+                                   int N_k, int off) {
   __shared__ float sq[128];
   __shared__ float sdo[128];
   __shared__ float sds[kThreads];
@@ -87,7 +86,7 @@ __global__ void bwd_dq_fp32_kernel(const float* __restrict__ q, const float* __r
     sdo[t] = d_o[base + static_cast<size_t>(i) * D + t];
   }
   __syncthreads();
-  const int jend = causal ? min(N_k, i + off + 1) : N_k;
+  const int jend = causal ? max(0, min(N_k, i + off + 1)) : N_k;
   float acc = 0.0f;
   for (int j0 = 0; j0 < jend; j0 += kThreads) {
     const int j = j0 + t;
@@ -125,8 +124,7 @@ __global__ void bwd_dkdv_fp32_kernel(const float* __restrict__ q, const float* _
                                      const float* __restrict__ v, const float* __restrict__ d_o,
                                      float* __restrict__ dk, float* __restrict__ dv, int H, int N, int D,
                                      float scale, float bias_scalar, int causal, const float* __restrict__ slopes,
-                                     const float* __restrict__ bias_vec, int H_kv, int N_k) {
-  const int off = N_k - N;
+                                     const float* __restrict__ bias_vec, int H_kv, int N_k, int off) {
   __shared__ float sk[128];
   __shared__ float sv[128];
   __shared__ float sp[kThreads];
@@ -182,7 +180,7 @@ int launch_fwd_fp32(const float* q, const float* k, const float* v, float* o, co
                     cudaStream_t stream, unsigned long long* launches, cudaError_t* cuda_err) {
   dim3 grid(p.N, p.B * p.H);
   fwd_fp32_kernel<<<grid, kThreads, 0, stream>>>(q, k, v, o, p.H, p.N, p.D, p.scale, p.bias, p.causal, p.slopes,
-                                                 p.bias_vec, p.kv_heads(), p.key_rows());
+                                                 p.bias_vec, p.kv_heads(), p.key_rows(), p.query_pos0());
   *launches += 1;
   *cuda_err = cudaGetLastError();
   return *cuda_err == cudaSuccess ? SIGATTN_OK : SIGATTN_ERR_CUDA;
@@ -197,10 +195,11 @@ int launch_bwd_fp32(const float* q, const float* k, const float* v, const float*
     if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
   }
   bwd_dq_fp32_kernel<<<grid, kThreads, 0, stream>>>(q, k, v, d_o, dq, p.H, p.N, p.D, p.scale, p.bias, p.causal,
-                                                    p.slopes, p.bias_vec, p.dbias, p.kv_heads(), p.key_rows());
+                                                    p.slopes, p.bias_vec, p.dbias, p.kv_heads(), p.key_rows(), p.query_pos0());
   dim3 grid_kv(p.key_rows(), p.B * p.kv_heads());
   bwd_dkdv_fp32_kernel<<<grid_kv, kThreads, 0, stream>>>(q, k, v, d_o, dk, dv, p.H, p.N, p.D, p.scale, p.bias,
-                                                         p.causal, p.slopes, p.bias_vec, p.kv_heads(), p.key_rows());
+                                                         p.causal, p.slopes, p.bias_vec, p.kv_heads(), p.key_rows(),
+                                                         p.query_pos0());
   *launches += 2;
   *cuda_err = cudaGetLastError();
   return *cuda_err == cudaSuccess ? SIGATTN_OK : SIGATTN_ERR_CUDA;

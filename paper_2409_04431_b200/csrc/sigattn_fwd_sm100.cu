@@ -83,7 +83,8 @@ struct FwdBarriers {
 
 struct FwdParams {
   int BH, H, N;     // N counts query rows
-  int pos0;         // position of query row 0: rows of K, V minus N (0 for self-attention)
+  int pos0;         // position of query row 0 relative to key row 0: rows of K, V minus N when the
+                    // queries are the last positions (0 for self-attention); any value for a shard
   int H_kv, group;  // heads of K, V and query heads per key/value head (H = H_kv * group)
   // Packed grouped heads (few queries per head, e.g. decoding): the rows of all `pack_group`
   // query heads of one key/value head form ONE sequence of pack_group * pack_rows rows, row r
@@ -130,7 +131,10 @@ __device__ __forceinline__ Item decode_item(const FwdParams& p, int item) {
     // causal: the tile's last row, at position r + 127 + pos0, sees keys up to that position
     // (packed rows: every tile holds last queries of some head, so every key tile is visited)
     w.n[t] = (r >= p.N) ? 0
-             : ((CAUSAL && p.pack_rows == 0) ? min(p.n_kv_total, (r + kBM - 1 + p.pos0) / kBN + 1) : p.n_kv_total);
+             : ((CAUSAL && p.pack_rows == 0)
+                    // (a tile that lies before every key still visits one key tile, fully masked: zeros)
+                    ? ((r + kBM - 1 + p.pos0 < 0) ? 1 : min(p.n_kv_total, (r + kBM - 1 + p.pos0) / kBN + 1))
+                    : p.n_kv_total);
   }
   w.n_kv = max(w.n[0], w.n[1]);
   return w;
@@ -568,7 +572,7 @@ int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const 
   fp.pack_rows = packed ? p.N : 0;
   fp.pack_group = packed ? group : 1;
   fp.N = static_cast<int>(q_rows);
-  fp.pos0 = p.key_rows() - p.N;
+  fp.pos0 = p.query_pos0();
   fp.n_pairs = (fp.N + 2 * kBM - 1) / (2 * kBM);
   fp.n_kv_total = (p.key_rows() + kBN - 1) / kBN;
   fp.n_items = fp.n_pairs * fp.BH;

@@ -18,6 +18,9 @@ struct Problem {
   int kv_heads() const { return H_kv > 0 ? H_kv : H; }
   int N_k;                // rows of k, v (N counts the rows of q); 0 = N.  The queries sit at the last N positions.
   int key_rows() const { return N_k > 0 ? N_k : N; }
+  int pos0_given;         // 1: `pos0` is the position of query row 0 relative to key row 0 (key/value shards)
+  int pos0;               //    0: the queries are the last N positions, pos0 = key_rows() - N
+  int query_pos0() const { return pos0_given ? pos0 : key_rows() - N; }
 };
 
 // Every launcher enqueues on `stream`, adds the number of kernels it launched to

@@ -5,6 +5,13 @@ The attention path has no exchange step: (batch, head) pairs are independent, so
 independent shards (each rank its own batch, drawn from its own seed) and the only
 communication is the timing reduction below.  Kept free of CUDA so that it can be tested with
 the gloo backend on CPU.
+
+The second half shards ONE long sequence's keys and values over the ranks (long context):
+sigmoid attention has no row normalisation (Section 4), so the attention of all queries
+against one contiguous key/value shard is a plain summand of O, and of dQ; ranks exchange one
+sum (all-reduce) and no log-sum-exp.  The per-shard computation is the library's
+sigattn_fwd_shard / sigattn_bwd_shard; it is passed in, so the exchange logic can be run on
+CPU with any stand-in.
 """
 from __future__ import annotations
 
@@ -41,3 +48,45 @@ def whole_job_tflops(flops_per_rank_step: float, steps: int, world: int, total_m
     """Weak scaling: every rank does `flops_per_rank_step` per step; the job's throughput is
     all ranks' work over the slowest rank's device time."""
     return world * flops_per_rank_step * steps / (total_ms_max * 1e-3) / 1e12
+
+
+def kv_shard_range(n_keys: int, world: int, rank: int) -> range:
+    """Contiguous block of key/value rows held by `rank`; the first `n_keys % world` ranks
+    hold one row more."""
+    return shard_heads(n_keys, world, rank)
+
+
+def kv_sharded_fwd(attend, q, k_shard, v_shard, key_start: int, query_start: int = 0, group=None):
+    """O of all queries `q` against the whole key/value sequence, of which this rank holds
+    rows [key_start, key_start + k_shard.shape[2]).
+
+    attend(q, k_shard, v_shard, pos0) -> this rank's summand of O, where pos0 is the position
+    of query row 0 relative to the shard's first key (binding.sigattn_fwd_shard with the
+    remaining arguments bound).  `query_start`: position of query row 0 in the sequence.
+    The summands are added in float32 with one all-reduce over `group`; the result has
+    q's dtype.  Without a process group the local summand is returned (one rank)."""
+    import torch
+    import torch.distributed as dist
+
+    part = attend(q, k_shard, v_shard, query_start - key_start)
+    if not (dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1):
+        return part
+    acc = part.to(torch.float32)
+    dist.all_reduce(acc, op=dist.ReduceOp.SUM, group=group)
+    return acc.to(part.dtype)
+
+
+def kv_sharded_bwd(attend_bwd, q, k_shard, v_shard, d_o, key_start: int, query_start: int = 0, group=None):
+    """(dQ, dK_shard, dV_shard): dQ is summed over the ranks like O; dK and dV of a shard
+    need only that shard's keys and values and stay local.
+
+    attend_bwd(q, k_shard, v_shard, d_o, pos0) -> (dq summand, dk_shard, dv_shard)."""
+    import torch
+    import torch.distributed as dist
+
+    dq, dk, dv = attend_bwd(q, k_shard, v_shard, d_o, query_start - key_start)[:3]
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1:
+        acc = dq.to(torch.float32)
+        dist.all_reduce(acc, op=dist.ReduceOp.SUM, group=group)
+        dq = acc.to(dq.dtype)
+    return dq, dk, dv

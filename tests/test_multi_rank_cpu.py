@@ -66,3 +66,65 @@ def test_sharding_rules():
     assert one == pytest.approx(100.0)
     # without a process group the reduction is the identity
     assert sharding.max_over_ranks([1.0, 2.0]) == [1.0, 2.0]
+
+
+def _kv_worker(rank, world, port, out_dir):
+    """Each rank holds one contiguous key/value shard of the same sequence; the per-shard
+    computation is the float64 oracle standing in for the CUDA entry points."""
+    import torch
+    import torch.distributed as dist
+    import oracle
+    from paper_2409_04431_b200 import sharding
+
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        B, H, N, D = 1, 2, 11, 4
+        rng = np.random.default_rng(5)                      # the same sequence on every rank
+        q, k, v, d_o = (rng.standard_normal((B, H, N, D)) for _ in range(4))
+        slopes = np.array([0.5, 0.25])
+        scale, bias = 0.5, -1.0
+        rows = sharding.kv_shard_range(N, world, rank)
+        ks, vs = k[:, :, rows.start:rows.stop], v[:, :, rows.start:rows.stop]
+
+        def attend(a, b, c, pos0):
+            return torch.from_numpy(oracle.sigattn_fwd(a.numpy(), b.numpy(), c.numpy(), scale, bias, True, slopes, pos0=pos0))
+
+        def attend_bwd(a, b, c, d, pos0):
+            return tuple(torch.from_numpy(g) for g in
+                         oracle.sigattn_bwd(a.numpy(), b.numpy(), c.numpy(), d.numpy(), scale, bias, True, slopes, pos0=pos0))
+
+        tq, tks, tvs, tdo = (torch.from_numpy(np.ascontiguousarray(t)) for t in (q, ks, vs, d_o))
+        o = sharding.kv_sharded_fwd(attend, tq, tks, tvs, rows.start)
+        dq, dk, dv = sharding.kv_sharded_bwd(attend_bwd, tq, tks, tvs, tdo, rows.start)
+        np.savez(os.path.join(out_dir, f"kv{rank}.npz"), o=o.numpy(), dq=dq.numpy(), dk=dk.numpy(), dv=dv.numpy(),
+                 lo=rows.start, hi=rows.stop)
+        dist.barrier()
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_gloo_ranks_sum_key_value_shards(tmp_path):
+    """O and dQ after the all-reduce equal the attention against the whole sequence on every
+    rank; dK, dV of each rank are the slices of the whole gradient."""
+    import torch.multiprocessing as mp
+    import oracle
+    world, port = 2, _free_port()
+    mp.spawn(_kv_worker, args=(world, port, str(tmp_path)), nprocs=world, join=True)
+    rng = np.random.default_rng(5)
+    q, k, v, d_o = (rng.standard_normal((1, 2, 11, 4)) for _ in range(4))
+    slopes = np.array([0.5, 0.25])
+    ref_o = oracle.sigattn_fwd(q, k, v, 0.5, -1.0, True, slopes)
+    ref_dq, ref_dk, ref_dv = oracle.sigattn_bwd(q, k, v, d_o, 0.5, -1.0, True, slopes)
+    covered = []
+    for rank in range(world):
+        r = np.load(tmp_path / f"kv{rank}.npz")
+        # the exchange adds in float32
+        np.testing.assert_allclose(r["o"], ref_o, rtol=1e-5, atol=1e-6)
+        np.testing.assert_allclose(r["dq"], ref_dq, rtol=1e-5, atol=1e-6)
+        lo, hi = int(r["lo"]), int(r["hi"])
+        np.testing.assert_allclose(r["dk"], ref_dk[:, :, lo:hi], rtol=1e-12, atol=1e-14)
+        np.testing.assert_allclose(r["dv"], ref_dv[:, :, lo:hi], rtol=1e-12, atol=1e-14)
+        covered += list(range(lo, hi))
+    assert covered == list(range(11))
