@@ -61,6 +61,13 @@ Readings of the paper taken here
     row 0 minus the position of the shard's first key (default N_k - N_q as above) and may
     be negative; a query that lies before every key of the shard gets weight 0 everywhere.
 
+  * Batches of sequences of different lengths, padded to a common N (the speech batches of
+    Section 5.4): with `seqlens[b] = n_b <= N`, keys j >= n_b get weight 0 like masked keys,
+    query rows i >= n_b produce all-zero rows of O and take no part in any gradient (their
+    dQ rows are zero, dK and dV do not see them).  The paper does not print this; it is the
+    usual padding mask, and it makes the call equal to separate calls on the unpadded
+    sequences.  Only for N_q = N_k.
+
 Every function is pinned by tests that do not call back into this file's own
 formulae (closed forms, brute-force loops, finite differences, the paper's second
 form of the forward, the printed n = 3 mask): there is no "parity unpinned" part.
@@ -128,9 +135,10 @@ def position_bias(n: int, slope: float, i0: int = 0, i1: int | None = None, n_q:
     return -float(slope) * np.abs(i - j)
 
 
-def attention_weights(q, k, scale, bias, causal, slope=0.0, i0=0, i1=None, pos0=None):
+def attention_weights(q, k, scale, bias, causal, slope=0.0, i0=0, i1=None, pos0=None, seqlen=None):
     """P for query rows i0..i1-1 of one head: sigmoid(scale * q k^T + b + position
-    bias), times the causal mask.  q: [n_q, d], k: [n, d] float64."""
+    bias), times the causal mask and, with `seqlen`, times the padding mask (rows and
+    columns >= seqlen are 0).  q: [n_q, d], k: [n, d] float64."""
     n_q, n = q.shape[0], k.shape[0]
     i1 = n_q if i1 is None else i1
     x = scale * (q[i0:i1] @ k.T) + bias
@@ -139,6 +147,10 @@ def attention_weights(q, k, scale, bias, causal, slope=0.0, i0=0, i1=None, pos0=
     p = sigmoid(x)
     if causal:
         p = p * causal_mask(n, i0, i1, n_q, pos0)
+    if seqlen is not None:
+        valid_rows = (np.arange(i0, i1) < int(seqlen)).astype(np.float64)[:, None]
+        valid_cols = (np.arange(n) < int(seqlen)).astype(np.float64)[None, :]
+        p = p * valid_rows * valid_cols
     return p
 
 
@@ -171,6 +183,17 @@ def _kv_group(num_heads, k):
     return num_heads // h_kv
 
 
+def _seqlens(seqlens, num_batch, n_q, n_k):
+    if seqlens is None:
+        return [None] * num_batch
+    if n_q != n_k:
+        raise ValueError("seqlens need as many query rows as key rows")
+    s = np.asarray(seqlens).reshape(-1)
+    if s.shape[0] != num_batch or np.any(s < 0) or np.any(s > n_q):
+        raise ValueError("seqlens must hold one length in [0, N] per batch entry")
+    return [int(x) for x in s]
+
+
 def _row_ranges(n, row_block):
     """Query rows are independent in the forward and enter dK, dV only through a sum
     over rows, so they may be visited in slabs to bound memory (an n x n float64 matrix
@@ -179,7 +202,7 @@ def _row_ranges(n, row_block):
     return [(a, min(n, a + step)) for a in range(0, n, step)]
 
 
-def sigattn_fwd(q, k, v, scale, bias, causal=False, alibi_slopes=None, row_block=None, pos0=None):
+def sigattn_fwd(q, k, v, scale, bias, causal=False, alibi_slopes=None, row_block=None, pos0=None, seqlens=None):
     """O = sigmoid(scale * Q K^T + b [+ position bias]) [* causal mask] V  (Eq. 3).
 
     q: [B, H, N, D]; k, v: [B, H_kv, N, D] with H a multiple of H_kv (any float dtype;
@@ -193,22 +216,25 @@ def sigattn_fwd(q, k, v, scale, bias, causal=False, alibi_slopes=None, row_block
     group = _kv_group(H, k)
     slopes = _slopes(alibi_slopes, H)
     bias_bh = _bias_per_head(bias, B, H)
+    lens = _seqlens(seqlens, B, N, k.shape[2])
     o = np.zeros((B, H, N, D), dtype=np.float64)
     for b in range(B):
         for h in range(H):
             hk = h // group
             for i0, i1 in _row_ranges(N, row_block):
-                p = attention_weights(q[b, h], k[b, hk], scale, bias_bh[b, h], causal, slopes[h], i0, i1, pos0)
+                p = attention_weights(q[b, h], k[b, hk], scale, bias_bh[b, h], causal, slopes[h], i0, i1, pos0,
+                                      lens[b])
                 o[b, h, i0:i1] = p @ v[b, hk]
     return o
 
 
-def _bwd_all(q, k, v, d_o, scale, bias, causal, alibi_slopes, row_block, pos0=None):
+def _bwd_all(q, k, v, d_o, scale, bias, causal, alibi_slopes, row_block, pos0=None, seqlens=None):
     q, k, v, d_o = _as_f64(q, k, v, d_o)
     B, H, N, D = q.shape
     group = _kv_group(H, k)
     slopes = _slopes(alibi_slopes, H)
     bias_bh = _bias_per_head(bias, B, H)
+    lens = _seqlens(seqlens, B, N, k.shape[2])
     dq = np.zeros_like(q)
     dk = np.zeros_like(k)
     dv = np.zeros_like(v)
@@ -217,7 +243,8 @@ def _bwd_all(q, k, v, d_o, scale, bias, causal, alibi_slopes, row_block, pos0=No
         for h in range(H):
             hk = h // group
             for i0, i1 in _row_ranges(N, row_block):
-                p = attention_weights(q[b, h], k[b, hk], scale, bias_bh[b, h], causal, slopes[h], i0, i1, pos0)
+                p = attention_weights(q[b, h], k[b, hk], scale, bias_bh[b, h], causal, slopes[h], i0, i1, pos0,
+                                      lens[b])
                 do_rows = d_o[b, h, i0:i1]
                 dv[b, hk] += p.T @ do_rows
                 dp = do_rows @ v[b, hk].T
@@ -228,7 +255,8 @@ def _bwd_all(q, k, v, d_o, scale, bias, causal, alibi_slopes, row_block, pos0=No
     return dq, dk, dv, dbias
 
 
-def sigattn_bwd(q, k, v, d_o, scale, bias, causal=False, alibi_slopes=None, row_block=None, pos0=None):
+def sigattn_bwd(q, k, v, d_o, scale, bias, causal=False, alibi_slopes=None, row_block=None, pos0=None,
+                seqlens=None):
     """Gradients of L = sum(O * dO) with respect to Q, K, V (sigmoid column of the
     forward/backward table in Appendix F.1, with the 1/sqrt(d) factor; see header).
 
@@ -236,17 +264,18 @@ def sigattn_bwd(q, k, v, d_o, scale, bias, causal=False, alibi_slopes=None, row_
     than q (see header).
     Returns (dQ, dK, dV), float64, shaped like q, k, v.
     """
-    return _bwd_all(q, k, v, d_o, scale, bias, causal, alibi_slopes, row_block, pos0)[:3]
+    return _bwd_all(q, k, v, d_o, scale, bias, causal, alibi_slopes, row_block, pos0, seqlens)[:3]
 
 
-def sigattn_bwd_dbias(q, k, v, d_o, scale, bias, causal=False, alibi_slopes=None, row_block=None, pos0=None):
+def sigattn_bwd_dbias(q, k, v, d_o, scale, bias, causal=False, alibi_slopes=None, row_block=None, pos0=None,
+                      seqlens=None):
     """Gradient of L = sum(O * dO) with respect to a bias held per (batch, head):
     db[b, h] = sum_ij dS_ij with dS = P (1 - P) dP as in sigattn_bwd (see header).  A
     bias shared by several heads or sequences gets the sum of their entries.
 
     Returns float64 [B, H].
     """
-    return _bwd_all(q, k, v, d_o, scale, bias, causal, alibi_slopes, row_block, pos0)[3]
+    return _bwd_all(q, k, v, d_o, scale, bias, causal, alibi_slopes, row_block, pos0, seqlens)[3]
 
 
 def sigattn_fwd_sequence_form(q, k, v, scale, n_bias):

@@ -529,3 +529,41 @@ def test_key_value_shards_sum_to_the_whole(causal):
     np.testing.assert_allclose(part, ref, rtol=1e-13, atol=1e-16)
     if causal:
         assert np.all(part[:, :, :lo] == 0.0)
+
+
+# ----------------------------------------------------------------------- padded batches
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_padded_batch_equals_separate_unpadded_calls(causal):
+    """seqlens: the valid part of every output equals the call on the unpadded sequence
+    alone, whatever the padding holds; the padded part is exactly zero."""
+    B, H, N, D = 3, 2, 7, 3
+    q, k, v, d_o = (rnd((B, H, N, D), s) for s in (140, 141, 142, 143))
+    lens = [7, 4, 1]
+    slopes = np.array([0.5, 0.25])
+    scale = 0.7
+    bias = -np.log(np.array(lens, dtype=np.float64))     # b = -log n of each sample
+    o = oracle.sigattn_fwd(q, k, v, scale, bias, causal, slopes, seqlens=lens)
+    dq, dk, dv = oracle.sigattn_bwd(q, k, v, d_o, scale, bias, causal, slopes, seqlens=lens)
+    db = oracle.sigattn_bwd_dbias(q, k, v, d_o, scale, bias, causal, slopes, seqlens=lens)
+    for b, n in enumerate(lens):
+        sel = (slice(b, b + 1), slice(None), slice(0, n))
+        args = (q[sel], k[sel], v[sel])
+        np.testing.assert_allclose(o[sel], oracle.sigattn_fwd(*args, scale, float(bias[b]), causal, slopes), rtol=1e-14, atol=1e-16)
+        one = oracle.sigattn_bwd(*args, d_o[sel], scale, float(bias[b]), causal, slopes)
+        for g, r in zip((dq, dk, dv), one):
+            np.testing.assert_allclose(g[sel], r, rtol=1e-13, atol=1e-16)
+        np.testing.assert_allclose(db[b], oracle.sigattn_bwd_dbias(*args, d_o[sel], scale, float(bias[b]), causal, slopes)[0], rtol=1e-13)
+        for g in (o, dq, dk, dv):
+            assert np.all(g[b, :, n:] == 0.0)
+    # the padding must not matter
+    q2, k2, v2, do2 = q.copy(), k.copy(), v.copy(), d_o.copy()
+    for b, n in enumerate(lens):
+        for t in (q2, k2, v2, do2):
+            t[b, :, n:] = 1e3
+    np.testing.assert_array_equal(oracle.sigattn_fwd(q2, k2, v2, scale, bias, causal, slopes, seqlens=lens), o)
+    for g, r in zip(oracle.sigattn_bwd(q2, k2, v2, do2, scale, bias, causal, slopes, seqlens=lens), (dq, dk, dv)):
+        np.testing.assert_array_equal(g, r)
+    with pytest.raises(ValueError):
+        oracle.sigattn_fwd(q, k, v, scale, -1.0, causal, seqlens=[7, 8, 1])
