@@ -218,6 +218,30 @@ SIGATTN_API int sigattn_bwd_shard(const void* q, const void* k, const void* v, c
                       float* dbias_bh,
                       void* workspace, size_t workspace_bytes, void* stream);
 
+/* Padded batches of sequences of different lengths (the speech batches of Section 5.4, with
+ * b = -log n_b per sample through `bias_bh`): `seqlens` is a DEVICE pointer to B int32, 4-byte
+ * aligned, read while the kernels run; entry b is the number n_b of rows of batch entry b that
+ * count (values outside [0, N] are clamped).  Keys j >= n_b get weight 0; query rows i >= n_b
+ * give all-zero rows of O and take no part in any gradient (their dq rows are zero, dk and dv
+ * do not see them; dk, dv rows >= n_b are zero).  What the padding holds does not matter.  The
+ * paper does not print this; it is the usual padding mask and makes the call equal to separate
+ * calls on the unpadded sequences.  q, k, v share N.  Other arguments as in sigattn_fwd_gqa /
+ * sigattn_bwd_gqa. */
+SIGATTN_API int sigattn_fwd_varlen(const void* q, const void* k, const void* v, void* o,
+                       int B, int H, int H_kv, int N, int D,
+                       float scale, float bias, const float* bias_bh, int causal,
+                       const int* seqlens,
+                       const float* alibi_slopes, int dtype, void* stream);
+
+SIGATTN_API int sigattn_bwd_varlen(const void* q, const void* k, const void* v, const void* d_o,
+                       void* dq, void* dk, void* dv,
+                       int B, int H, int H_kv, int N, int D,
+                       float scale, float bias, const float* bias_bh, int causal,
+                       const int* seqlens,
+                       const float* alibi_slopes, int dtype,
+                       float* dbias_bh,
+                       void* workspace, size_t workspace_bytes, void* stream);
+
 /* Bytes of scratch sigattn_bwd needs for this problem (0 for the fp32 debug path).
  * Returns 0 for invalid shapes as well; sigattn_bwd reports those. */
 SIGATTN_API size_t sigattn_bwd_workspace_bytes(int B, int H, int N, int D, int dtype);

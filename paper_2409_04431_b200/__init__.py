@@ -33,6 +33,8 @@ _BINDING_NAMES = (
     "sigattn_bwd_nk",
     "sigattn_fwd_shard",
     "sigattn_bwd_shard",
+    "sigattn_fwd_varlen",
+    "sigattn_bwd_varlen",
     "lib",
 )
 

@@ -59,6 +59,13 @@ _lib.sigattn_bwd_shard.restype = _c.c_int
 _lib.sigattn_bwd_shard.argtypes = [_c.c_void_p] * 7 + [_c.c_int] * 6 + [_c.c_float, _c.c_float, _c.c_void_p, _c.c_int,
                                                                           _c.c_int, _c.c_void_p, _c.c_int, _c.c_void_p,
                                                                           _c.c_void_p, _c.c_size_t, _c.c_void_p]
+_lib.sigattn_fwd_varlen.restype = _c.c_int
+_lib.sigattn_fwd_varlen.argtypes = [_c.c_void_p] * 4 + [_c.c_int] * 5 + [_c.c_float, _c.c_float, _c.c_void_p, _c.c_int,
+                                                                           _c.c_void_p, _c.c_void_p, _c.c_int, _c.c_void_p]
+_lib.sigattn_bwd_varlen.restype = _c.c_int
+_lib.sigattn_bwd_varlen.argtypes = [_c.c_void_p] * 7 + [_c.c_int] * 5 + [_c.c_float, _c.c_float, _c.c_void_p, _c.c_int,
+                                                                           _c.c_void_p, _c.c_void_p, _c.c_int, _c.c_void_p,
+                                                                           _c.c_void_p, _c.c_size_t, _c.c_void_p]
 _lib.sigattn_bwd_workspace_bytes.restype = _c.c_size_t
 _lib.sigattn_bwd_workspace_bytes.argtypes = [_c.c_int] * 5
 _lib.sigattn_step_host.restype = _c.c_int
@@ -94,7 +101,7 @@ EXPORTED = [
     "sigattn_bwd_static_scratch", "sigattn_bwd_static_scratch_max_elements",
     "sigattn_selftest_bounded_wait", "sigattn_fwd_bias_vec", "sigattn_bwd_bias_vec",
     "sigattn_fwd_gqa", "sigattn_bwd_gqa", "sigattn_fwd_nk", "sigattn_bwd_nk",
-    "sigattn_fwd_shard", "sigattn_bwd_shard",
+    "sigattn_fwd_shard", "sigattn_bwd_shard", "sigattn_fwd_varlen", "sigattn_bwd_varlen",
 ]
 
 
@@ -439,6 +446,62 @@ def sigattn_bwd_shard(q, k, v, d_o, scale, bias, pos0, causal=False, alibi_slope
                                     N_k, D, float(scale), 0.0 if vec else float(bias), _ptr(bias) if vec else None,
                                     int(bool(causal)), int(pos0), _ptr(alibi_slopes), code, _ptr(dbias),
                                     _ptr(workspace), ws_bytes, _stream_ptr(stream))
+    if rc != 0:
+        raise SigattnError(rc)
+    return dq, dk, dv, dbias
+
+
+def _check_seqlens(seqlens, q):
+    import torch
+    if (not isinstance(seqlens, torch.Tensor) or not seqlens.is_cuda or seqlens.dtype != torch.int32
+            or tuple(seqlens.shape) != (q.shape[0],) or not seqlens.is_contiguous() or seqlens.device != q.device):
+        raise ValueError("seqlens must be a contiguous int32 CUDA tensor of shape [B] on q's device")
+
+
+def sigattn_fwd_varlen(q, k, v, scale, bias, seqlens, causal=False, alibi_slopes=None, out=None, stream=None):
+    """Padded batch: `seqlens` (int32 CUDA [B]) gives the rows of each batch entry that count.
+    `bias`: float or float32 CUDA [B, H] (e.g. -log of each length)."""
+    import torch
+    B, H, H_kv, N, D = _check_gqa(q, k, v)
+    _check_seqlens(seqlens, q)
+    if out is None:
+        out = torch.empty_like(q)
+    else:
+        _check_same([q, out], ["q", "out"])
+    vec = isinstance(bias, torch.Tensor)
+    if vec:
+        _check_bias_vec(bias, q)
+    with torch.cuda.device(q.device):
+        rc = _lib.sigattn_fwd_varlen(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, H, H_kv, N, D, float(scale),
+                                     0.0 if vec else float(bias), _ptr(bias) if vec else None, int(bool(causal)),
+                                     _ptr(seqlens), _ptr(alibi_slopes), _dtype_code(q), _stream_ptr(stream))
+    if rc != 0:
+        raise SigattnError(rc)
+    return out
+
+
+def sigattn_bwd_varlen(q, k, v, d_o, scale, bias, seqlens, causal=False, alibi_slopes=None, want_dbias=False,
+                       workspace=None, stream=None):
+    """Backward of sigattn_fwd_varlen: (dQ, dK, dV, dbias or None); padded rows come out zero."""
+    import torch
+    B, H, H_kv, N, D = _check_gqa(q, k, v)
+    _check_same([q, d_o], ["q", "d_o"])
+    _check_seqlens(seqlens, q)
+    code = _dtype_code(q)
+    dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+    vec = isinstance(bias, torch.Tensor)
+    if vec:
+        _check_bias_vec(bias, q)
+    dbias = torch.empty((B, H), dtype=torch.float32, device=q.device) if want_dbias else None
+    need = sigattn_bwd_workspace_bytes(B, H, N, D, code)
+    if workspace is None and need > 0:
+        workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    with torch.cuda.device(q.device):
+        rc = _lib.sigattn_bwd_varlen(_ptr(q), _ptr(k), _ptr(v), _ptr(d_o), _ptr(dq), _ptr(dk), _ptr(dv), B, H, H_kv, N, D,
+                                     float(scale), 0.0 if vec else float(bias), _ptr(bias) if vec else None,
+                                     int(bool(causal)), _ptr(seqlens), _ptr(alibi_slopes), code, _ptr(dbias),
+                                     _ptr(workspace), ws_bytes, _stream_ptr(stream))
     if rc != 0:
         raise SigattnError(rc)
     return dq, dk, dv, dbias

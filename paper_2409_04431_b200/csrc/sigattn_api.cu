@@ -102,7 +102,7 @@ int check_lengths(int B, int H, int H_kv, int N, int N_k, int D, int causal, int
 
 int fwd_any(const void* q, const void* k, const void* v, void* o, int B, int H, int H_kv, int N, int N_k, int D,
             float scale, float bias, const float* bias_vec, int causal, const float* alibi_slopes, int dtype,
-            void* stream, int pos0_given = 0, int pos0 = 0) {
+            void* stream, int pos0_given = 0, int pos0 = 0, const int* seqlens = nullptr) {
   if (!q || !k || !v || !o) return SIGATTN_ERR_NULL;
   if (int rc = check_lengths(B, H, H_kv, N, N_k, D, causal, pos0_given, pos0)) return rc;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return SIGATTN_ERR_ALIGN;
@@ -112,7 +112,8 @@ int fwd_any(const void* q, const void* k, const void* v, void* o, int B, int H, 
   int dev = 0;
   int* status = nullptr;
   if (int rc = device_setup(&dev, &status)) return rc;
-  sigattn::Problem p{B, H, N, D, scale, bias, causal, alibi_slopes, bias_vec, nullptr, H_kv, N_k, pos0_given, pos0};
+  sigattn::Problem p{B, H, N, D, scale, bias, causal, alibi_slopes, bias_vec, nullptr, H_kv, N_k, pos0_given, pos0,
+                     seqlens};
   unsigned long long launches = 0;
   cudaError_t ce = cudaSuccess;
   int rc;
@@ -131,7 +132,7 @@ int fwd_any(const void* q, const void* k, const void* v, void* o, int B, int H, 
 int bwd_any(const void* q, const void* k, const void* v, const void* d_o, void* dq, void* dk, void* dv, int B, int H,
             int H_kv, int N, int N_k, int D, float scale, float bias, const float* bias_vec, float* dbias, int causal,
             const float* alibi_slopes, int dtype, void* workspace, size_t workspace_bytes, void* stream,
-            int pos0_given = 0, int pos0 = 0) {
+            int pos0_given = 0, int pos0 = 0, const int* seqlens = nullptr) {
   if (!q || !k || !v || !d_o || !dq || !dk || !dv) return SIGATTN_ERR_NULL;
   if (int rc = check_lengths(B, H, H_kv, N, N_k, D, causal, pos0_given, pos0)) return rc;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(d_o) || !aligned16(dq) || !aligned16(dk) ||
@@ -149,7 +150,8 @@ int bwd_any(const void* q, const void* k, const void* v, const void* d_o, void* 
   int dev = 0;
   int* status = nullptr;
   if (int rc = device_setup(&dev, &status)) return rc;
-  sigattn::Problem p{B, H, N, D, scale, bias, causal, alibi_slopes, bias_vec, dbias, H_kv, N_k, pos0_given, pos0};
+  sigattn::Problem p{B, H, N, D, scale, bias, causal, alibi_slopes, bias_vec, dbias, H_kv, N_k, pos0_given, pos0,
+                     seqlens};
   unsigned long long launches = 0;
   cudaError_t ce = cudaSuccess;
   int rc;
@@ -252,6 +254,28 @@ int sigattn_bwd_shard(const void* q, const void* k, const void* v, const void* d
     return SIGATTN_ERR_ALIGN;
   return bwd_any(q, k, v, d_o, dq, dk, dv, B, H, H_kv, N_q, N_k, D, scale, bias, bias_bh, dbias_bh, causal,
                  alibi_slopes, dtype, workspace, workspace_bytes, stream, 1, pos0);
+}
+
+int sigattn_fwd_varlen(const void* q, const void* k, const void* v, void* o, int B, int H, int H_kv, int N, int D,
+                       float scale, float bias, const float* bias_bh, int causal, const int* seqlens,
+                       const float* alibi_slopes, int dtype, void* stream) {
+  if (!seqlens) return SIGATTN_ERR_NULL;
+  if ((reinterpret_cast<uintptr_t>(seqlens) & 3u) || (reinterpret_cast<uintptr_t>(bias_bh) & 3u))
+    return SIGATTN_ERR_ALIGN;
+  return fwd_any(q, k, v, o, B, H, H_kv, N, N, D, scale, bias, bias_bh, causal, alibi_slopes, dtype, stream, 0, 0,
+                 seqlens);
+}
+
+int sigattn_bwd_varlen(const void* q, const void* k, const void* v, const void* d_o, void* dq, void* dk, void* dv,
+                       int B, int H, int H_kv, int N, int D, float scale, float bias, const float* bias_bh, int causal,
+                       const int* seqlens, const float* alibi_slopes, int dtype, float* dbias_bh, void* workspace,
+                       size_t workspace_bytes, void* stream) {
+  if (!seqlens) return SIGATTN_ERR_NULL;
+  if ((reinterpret_cast<uintptr_t>(seqlens) & 3u) || (reinterpret_cast<uintptr_t>(bias_bh) & 3u) ||
+      (reinterpret_cast<uintptr_t>(dbias_bh) & 3u))
+    return SIGATTN_ERR_ALIGN;
+  return bwd_any(q, k, v, d_o, dq, dk, dv, B, H, H_kv, N, N, D, scale, bias, bias_bh, dbias_bh, causal, alibi_slopes,
+                 dtype, workspace, workspace_bytes, stream, 0, 0, seqlens);
 }
 
 int sigattn_bwd_set_timing_events(void* start_event, void* stop_event) {

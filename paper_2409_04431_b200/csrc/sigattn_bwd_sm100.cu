@@ -72,6 +72,7 @@ struct BwdParams {
   int n_tiles;    // query tiles: ceil(N / 128), N = rows of Q
   int n_tiles_k;  // key tiles: ceil(rows of K / 128)
   int pos0;       // position of query row 0 relative to key row 0 (see FwdParams of the forward)
+  const int* seqlens;   // padded batch: valid length per batch entry (keys and queries), or nullptr
   int n_items;
   float scale, scale_log2e, bias_log2e;
   const float* bias_vec;   // one bias per (batch, head) instead of the scalar, or nullptr
@@ -86,6 +87,7 @@ struct BwdItem {
   int j, i_begin;
   int n;        // query tiles per query head
   int steps;    // group * n, visited head by head
+  int n_valid;  // rows of this sequence that count (N unless the batch is padded)
 };
 
 // Ranks are ordered by decreasing cost; rounds alternate direction over the CTAs so that
@@ -99,8 +101,9 @@ __device__ __forceinline__ int bwd_snake_rank(int round, int n_items) {
 
 __device__ __forceinline__ int bwd_num_rounds(int n_items) { return (n_items + gridDim.x - 1) / gridDim.x; }
 
-// GROUPED = false compiles the one-head-per-group case (plain multi-head attention) without
-// the head loop; it is the benchmarked path.
+// GROUPED = false compiles the plain case (one query head per key/value head, no padded batch)
+// without the head loop and without the per-sequence lengths; it is the benchmarked path.
+// GROUPED = true serves both grouped heads and padded batches.
 template <bool CAUSAL, bool GROUPED>
 __device__ __forceinline__ BwdItem decode_bwd_item(const BwdParams& p, int item) {
   BwdItem w;
@@ -108,9 +111,15 @@ __device__ __forceinline__ BwdItem decode_bwd_item(const BwdParams& p, int item)
   w.bh = item - w.j * p.BH;
   w.bh_q0 = GROUPED ? (w.bh / p.H_kv) * p.H + (w.bh % p.H_kv) * p.group : w.bh;
   // causal: the first query tile whose last row, at position 128 i + 127 + pos0, reaches key 128 j
+  // padded batch: query tiles past the sequence's end are not visited at all
+  const bool padded = GROUPED && p.seqlens != nullptr;
+  w.n_valid = padded ? max(0, min(p.N, __ldg(p.seqlens + w.bh / p.H_kv))) : p.N;
+  const int n_tiles_q = padded ? max(1, (w.n_valid + kT - 1) / kT) : p.n_tiles;
   // (a key tile that lies after every query still visits the last query tile, fully masked: zeros)
-  w.i_begin = CAUSAL ? min(p.n_tiles - 1, max(0, (w.j * kT - p.pos0) / kT)) : 0;
-  w.n = p.n_tiles - w.i_begin;
+  w.i_begin = CAUSAL ? min(n_tiles_q - 1, max(0, (w.j * kT - p.pos0) / kT)) : 0;
+  // a key tile wholly past the sequence's end needs one (fully masked) query tile to write its zeros
+  if (padded && w.j * kT >= w.n_valid) w.i_begin = n_tiles_q - 1;
+  w.n = n_tiles_q - w.i_begin;
   w.steps = GROUPED ? p.group * w.n : w.n;
   return w;
 }
@@ -288,10 +297,11 @@ __device__ void bwd_mma_role(const BwdParams& p, uint32_t smem_base, uint32_t tm
 // 32 logits (transposed tile: this thread's key against 32 queries) -> P as bf16x2 for
 // the dV product and P (1 - P) in fp32 for dS.
 //   a = log2(e) * (scale * s + b - slope * |i - j|);  u = 2^a;  P = u / (1 + u);  1 - P = 1 / (1 + u)
-template <bool DIAG, bool ALIBI>
+// MASK: 0 no element masked, 1 causal only (queries before mask_lo), 2 both ends (padded batch)
+template <int MASK, bool ALIBI>
 __device__ __forceinline__ void bwd_sigmoid_chunk(const uint32_t (&s)[32], uint32_t (&p_out)[16], float (&pp)[32],
                                                   float scale_log2e, float bias_log2e, float slope_log2e,
-                                                  float col_rel, int q_base) {
+                                                  float col_rel, int q_base, float mask_lo, float mask_hi) {
   float a[32];
 #pragma unroll
   for (int e = 0; e < 32; ++e) {
@@ -301,10 +311,19 @@ __device__ __forceinline__ void bwd_sigmoid_chunk(const uint32_t (&s)[32], uint3
   }
   float pr[32];
   sigmoid_block<32, true, 0>(a, pr, pp);
-  if (DIAG) {
+  if (MASK == 1) {
 #pragma unroll
     for (int e = 0; e < 32; ++e)
-      if (static_cast<float>(q_base + e) < col_rel) { pr[e] = 0.0f; pp[e] = 0.0f; }  // query before key
+      if (static_cast<float>(q_base + e) < mask_lo) { pr[e] = 0.0f; pp[e] = 0.0f; }  // query before key
+  }
+  if (MASK == 2) {
+#pragma unroll
+    for (int e = 0; e < 32; ++e)
+      // query before key (causal), or, in a padded batch, past the end of the sequence
+      if (static_cast<float>(q_base + e) < mask_lo || static_cast<float>(q_base + e) >= mask_hi) {
+        pr[e] = 0.0f;
+        pp[e] = 0.0f;
+      }
   }
 #pragma unroll
   for (int e = 0; e < 16; ++e) p_out[e] = pack_bf16x2(pr[2 * e], pr[2 * e + 1]);
@@ -359,7 +378,14 @@ __device__ void bwd_act_role(const BwdParams& p, const CUtensorMap* tmDk, const 
       const float col_rel = static_cast<float>((w.j - i) * kT + tid - p.pos0);
       // the mask cuts through the tile unless even its first query sits at or after the last key:
       // the first tile of the loop, and with pos0 not a multiple of 128 also the second
-      const bool diag = CAUSAL && (i * kT + p.pos0 < w.j * kT + kT - 1);
+      bool diag = CAUSAL && (i * kT + p.pos0 < w.j * kT + kT - 1);
+      // queries [mask_lo, mask_hi) of the tile keep their weight for this thread's key
+      float mask_lo = CAUSAL ? col_rel : -1.0f, mask_hi = 1.0e9f;
+      if (GROUPED && p.seqlens != nullptr) {
+        mask_hi = static_cast<float>(w.n_valid - i * kT);
+        if (w.j * kT + tid >= w.n_valid) mask_hi = -1.0f;   // a key past the end: the whole row
+        diag = diag || (w.j + 1) * kT > w.n_valid || (i + 1) * kT > w.n_valid;
+      }
       float pp0[32], pp1[32];
       if (!mbar_wait(smem_u32(&bars->s_full), step_cnt & 1, cta_err, 60 + wg)) return;
       tc_fence_after_sync();
@@ -370,10 +396,15 @@ __device__ void bwd_act_role(const BwdParams& p, const CUtensorMap* tmDk, const 
         tmem_ld32(tmem + TM::kA + lane_off + gc * 32, s);
         tmem_wait_ld();
         float(&ppc)[32] = (c == 0) ? pp0 : pp1;
-        if (diag)
-          bwd_sigmoid_chunk<true, ALIBI>(s, pk, ppc, p.scale_log2e, bias_log2e, slope_log2e, col_rel, gc * 32);
+        if (GROUPED && diag)
+          bwd_sigmoid_chunk<2, ALIBI>(s, pk, ppc, p.scale_log2e, bias_log2e, slope_log2e, col_rel, gc * 32, mask_lo,
+                                      mask_hi);
+        else if (CAUSAL && diag)
+          bwd_sigmoid_chunk<1, ALIBI>(s, pk, ppc, p.scale_log2e, bias_log2e, slope_log2e, col_rel, gc * 32, col_rel,
+                                      0.0f);
         else
-          bwd_sigmoid_chunk<false, ALIBI>(s, pk, ppc, p.scale_log2e, bias_log2e, slope_log2e, col_rel, gc * 32);
+          bwd_sigmoid_chunk<0, ALIBI>(s, pk, ppc, p.scale_log2e, bias_log2e, slope_log2e, col_rel, gc * 32, 0.0f,
+                                      0.0f);
         tmem_st16(tmem + TM::kA + lane_off + wg * 64 + c * 16, pk);
       }
       tmem_wait_st();
@@ -664,6 +695,7 @@ int launch_bwd_bf16(const void* q, const void* k, const void* v, const void* d_o
   bp.bias_vec = p.bias_vec;
   bp.dbias = p.dbias;
   bp.slopes = p.slopes;
+  bp.seqlens = p.seqlens;
   bp.status = status;
 
   const size_t n_elems = static_cast<size_t>(BH) * p.N * p.D;
@@ -684,7 +716,7 @@ int launch_bwd_bf16(const void* q, const void* k, const void* v, const void* d_o
   // is compiled in only where it is asked for
   // is compiled in only where it is asked for; likewise the loop over a group's query heads
 #define SIGATTN_BWD_CASE(DD, CC, AA)                                                                        \
-  rc = (bp.group > 1)                                                                                       \
+  rc = (bp.group > 1 || bp.seqlens != nullptr)                                                              \
            ? ((p.dbias != nullptr) ? launch_bwd_variant<DD, CC, AA, true, true>(maps, bp, num_sms, stream, cuda_err)   \
                                    : launch_bwd_variant<DD, CC, AA, false, true>(maps, bp, num_sms, stream, cuda_err)) \
            : ((p.dbias != nullptr) ? launch_bwd_variant<DD, CC, AA, true, false>(maps, bp, num_sms, stream, cuda_err)  \

@@ -34,7 +34,8 @@ __device__ __forceinline__ float dot_row(const float* __restrict__ a_smem, const
 __global__ void fwd_fp32_kernel(const float* __restrict__ q, const float* __restrict__ k,
                                 const float* __restrict__ v, float* __restrict__ o, int H, int N, int D,
                                 float scale, float bias, int causal, const float* __restrict__ slopes,
-                                const float* __restrict__ bias_vec, int H_kv, int N_k, int off) {
+                                const float* __restrict__ bias_vec, int H_kv, int N_k, int off,
+                                const int* __restrict__ seqlens) {
   __shared__ float sq[128];
   __shared__ float sp[kThreads];
   const int i = blockIdx.x, bh = blockIdx.y, t = threadIdx.x;
@@ -44,7 +45,9 @@ __global__ void fwd_fp32_kernel(const float* __restrict__ q, const float* __rest
   const float slope = slopes ? slopes[bh % H] : 0.0f;
   if (t < D) sq[t] = q[base + static_cast<size_t>(i) * D + t];
   __syncthreads();
-  const int jend = causal ? max(0, min(N_k, i + off + 1)) : N_k;
+  // padded batch: keys past the sequence's length carry no weight, rows past it are zero
+  const int n_valid = seqlens ? max(0, min(N, seqlens[bh / H])) : N_k;
+  const int jend = (i >= n_valid && seqlens) ? 0 : min(n_valid, causal ? max(0, min(N_k, i + off + 1)) : N_k);
   float acc = 0.0f;
   for (int j0 = 0; j0 < jend; j0 += kThreads) {
     const int j = j0 + t;
@@ -71,7 +74,7 @@ __global__ void bwd_dq_fp32_kernel(const float* __restrict__ q, const float* __r
                                    float* __restrict__ dq, int H, int N, int D, float scale, float bias,
                                    int causal, const float* __restrict__ slopes,
                                    const float* __restrict__ bias_vec, float* __restrict__ dbias, int H_kv,
-                                   int N_k, int off) {
+                                   int N_k, int off, const int* __restrict__ seqlens) {
   __shared__ float sq[128];
   __shared__ float sdo[128];
   __shared__ float sds[kThreads];
@@ -86,7 +89,8 @@ __global__ void bwd_dq_fp32_kernel(const float* __restrict__ q, const float* __r
     sdo[t] = d_o[base + static_cast<size_t>(i) * D + t];
   }
   __syncthreads();
-  const int jend = causal ? max(0, min(N_k, i + off + 1)) : N_k;
+  const int n_valid = seqlens ? max(0, min(N, seqlens[bh / H])) : N_k;
+  const int jend = (i >= n_valid && seqlens) ? 0 : min(n_valid, causal ? max(0, min(N_k, i + off + 1)) : N_k);
   float acc = 0.0f;
   for (int j0 = 0; j0 < jend; j0 += kThreads) {
     const int j = j0 + t;
@@ -124,7 +128,8 @@ __global__ void bwd_dkdv_fp32_kernel(const float* __restrict__ q, const float* _
                                      const float* __restrict__ v, const float* __restrict__ d_o,
                                      float* __restrict__ dk, float* __restrict__ dv, int H, int N, int D,
                                      float scale, float bias_scalar, int causal, const float* __restrict__ slopes,
-                                     const float* __restrict__ bias_vec, int H_kv, int N_k, int off) {
+                                     const float* __restrict__ bias_vec, int H_kv, int N_k, int off,
+                                     const int* __restrict__ seqlens) {
   __shared__ float sk[128];
   __shared__ float sv[128];
   __shared__ float sp[kThreads];
@@ -137,17 +142,20 @@ __global__ void bwd_dkdv_fp32_kernel(const float* __restrict__ q, const float* _
     sv[t] = v[kv_base + static_cast<size_t>(j) * D + t];
   }
   __syncthreads();
-  const int ibeg = causal ? max(0, j - off) : 0;
+  // padded batch: a key past the sequence's length gets zero gradients, queries past it do not count
+  const int n_valid = seqlens ? max(0, min(N, seqlens[bh_kv / H_kv])) : N;
+  const int ibeg = (seqlens && j >= n_valid) ? N : (causal ? max(0, j - off) : 0);
+  const int iend = n_valid;
   float acc_k = 0.0f, acc_v = 0.0f;
   for (int g = 0; g < group; ++g) {
     const int bh = (bh_kv / H_kv) * H + (bh_kv % H_kv) * group + g;   // query head
     const size_t base = static_cast<size_t>(bh) * N * D;
     const float slope = slopes ? slopes[bh % H] : 0.0f;
     const float bias = bias_vec ? bias_vec[bh] : bias_scalar;
-    for (int i0 = ibeg; i0 < N; i0 += kThreads) {
+    for (int i0 = ibeg; i0 < iend; i0 += kThreads) {
       const int i = i0 + t;
       float p = 0.0f, ds = 0.0f;
-      if (i < N) {
+      if (i < iend) {
         const float s = dot_row(sk, q + base + static_cast<size_t>(i) * D, D);
         const float x = fmaf(scale, s, bias) - slope * fabsf(static_cast<float>(i + off - j));
         p = sigmoid_exact(x);
@@ -158,7 +166,7 @@ __global__ void bwd_dkdv_fp32_kernel(const float* __restrict__ q, const float* _
       sds[t] = ds;
       __syncthreads();
       if (t < D) {
-        const int cnt = min(kThreads, N - i0);
+        const int cnt = min(kThreads, iend - i0);
         for (int ii = 0; ii < cnt; ++ii) {
           const size_t row = base + static_cast<size_t>(i0 + ii) * D + t;
           acc_v = fmaf(sp[ii], d_o[row], acc_v);
@@ -180,7 +188,7 @@ int launch_fwd_fp32(const float* q, const float* k, const float* v, float* o, co
                     cudaStream_t stream, unsigned long long* launches, cudaError_t* cuda_err) {
   dim3 grid(p.N, p.B * p.H);
   fwd_fp32_kernel<<<grid, kThreads, 0, stream>>>(q, k, v, o, p.H, p.N, p.D, p.scale, p.bias, p.causal, p.slopes,
-                                                 p.bias_vec, p.kv_heads(), p.key_rows(), p.query_pos0());
+                                                 p.bias_vec, p.kv_heads(), p.key_rows(), p.query_pos0(), p.seqlens);
   *launches += 1;
   *cuda_err = cudaGetLastError();
   return *cuda_err == cudaSuccess ? SIGATTN_OK : SIGATTN_ERR_CUDA;
@@ -195,11 +203,12 @@ int launch_bwd_fp32(const float* q, const float* k, const float* v, const float*
     if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
   }
   bwd_dq_fp32_kernel<<<grid, kThreads, 0, stream>>>(q, k, v, d_o, dq, p.H, p.N, p.D, p.scale, p.bias, p.causal,
-                                                    p.slopes, p.bias_vec, p.dbias, p.kv_heads(), p.key_rows(), p.query_pos0());
+                                                    p.slopes, p.bias_vec, p.dbias, p.kv_heads(), p.key_rows(), p.query_pos0(),
+                                                    p.seqlens);
   dim3 grid_kv(p.key_rows(), p.B * p.kv_heads());
   bwd_dkdv_fp32_kernel<<<grid_kv, kThreads, 0, stream>>>(q, k, v, d_o, dk, dv, p.H, p.N, p.D, p.scale, p.bias,
                                                          p.causal, p.slopes, p.bias_vec, p.kv_heads(), p.key_rows(),
-                                                         p.query_pos0());
+                                                         p.query_pos0(), p.seqlens);
   *launches += 2;
   *cuda_err = cudaGetLastError();
   return *cuda_err == cudaSuccess ? SIGATTN_OK : SIGATTN_ERR_CUDA;

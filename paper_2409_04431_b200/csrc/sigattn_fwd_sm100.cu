@@ -92,6 +92,7 @@ struct FwdParams {
   // group instead of once per query head.  Then BH counts (batch, key/value head) pairs, N is
   // pack_group * pack_rows and H = H_kv, group = 1 for the producer.  0 = not packed.
   int pack_rows, pack_group;
+  const int* seqlens;   // padded batch: valid length per batch entry (keys and queries), or nullptr
   int n_pairs;     // ceil(N / 256)
   int n_kv_total;  // ceil(N / 128)
   int n_items;
@@ -103,6 +104,7 @@ struct FwdParams {
 
 struct Item {
   int bh, row0, n_kv, n[2];
+  int n_valid;   // rows of this sequence that count (N unless the batch is padded)
 };
 
 // Work items are ranked by decreasing cost (causal: later query tiles see more keys).
@@ -125,6 +127,8 @@ __device__ __forceinline__ Item decode_item(const FwdParams& p, int item) {
   w.bh = item - rank * p.BH;
   const int pair = CAUSAL ? (p.n_pairs - 1 - rank) : rank;
   w.row0 = pair * 2 * kBM;
+  w.n_valid = p.seqlens ? max(0, min(p.N, __ldg(p.seqlens + w.bh / p.H))) : p.N;
+  const int n_kv_valid = p.seqlens ? max(1, (w.n_valid + kBN - 1) / kBN) : p.n_kv_total;
 #pragma unroll
   for (int t = 0; t < 2; ++t) {
     const int r = w.row0 + t * kBM;
@@ -133,8 +137,10 @@ __device__ __forceinline__ Item decode_item(const FwdParams& p, int item) {
     w.n[t] = (r >= p.N) ? 0
              : ((CAUSAL && p.pack_rows == 0)
                     // (a tile that lies before every key still visits one key tile, fully masked: zeros)
-                    ? ((r + kBM - 1 + p.pos0 < 0) ? 1 : min(p.n_kv_total, (r + kBM - 1 + p.pos0) / kBN + 1))
-                    : p.n_kv_total);
+                    ? ((r + kBM - 1 + p.pos0 < 0) ? 1 : min(n_kv_valid, (r + kBM - 1 + p.pos0) / kBN + 1))
+                    : n_kv_valid);
+    // (a tile of a padded batch that lies past the sequence's end visits one key tile, fully masked)
+    if (p.seqlens && r < p.N && r >= w.n_valid) w.n[t] = 1;
   }
   w.n_kv = max(w.n[0], w.n[1]);
   return w;
@@ -318,7 +324,7 @@ __device__ __forceinline__ void tmem_st_cols(uint32_t addr, uint32_t (&v)[N]) {
 template <bool ALIBI, int EMULATE_EVERY>
 __device__ __forceinline__ void sigmoid_cols(const uint32_t (&s)[kCols], uint32_t (&out)[kCols / 2],
                                              float scale_log2e, float bias_log2e, float slope_log2e, float row_rel,
-                                             int col_base, bool causal_diag) {
+                                             int col_base, bool masked, float mask_limit) {
   float a[kCols];
 #pragma unroll
   for (int i = 0; i < kCols; ++i) {
@@ -331,10 +337,10 @@ __device__ __forceinline__ void sigmoid_cols(const uint32_t (&s)[kCols], uint32_
   }
   float pr[kCols];
   sigmoid_block<kCols, false, EMULATE_EVERY>(a, pr, nullptr);
-  if (causal_diag) {  // keys after the query get weight 0 (only on the diagonal tile)
+  if (masked) {  // keys after the query (and, in a padded batch, past the sequence's end) get weight 0
 #pragma unroll
     for (int i = 0; i < kCols; ++i)
-      if (static_cast<float>(col_base + i) > row_rel) pr[i] = 0.0f;
+      if (static_cast<float>(col_base + i) > mask_limit) pr[i] = 0.0f;
   }
 #pragma unroll
   for (int i = 0; i < kCols / 2; ++i) out[i] = pack_bf16x2(pr[2 * i], pr[2 * i + 1]);
@@ -345,10 +351,12 @@ __device__ __forceinline__ void sigmoid_cols(const uint32_t (&s)[kCols], uint32_
 // of the tile.  While the groups evaluate one tile, the tensor pipe runs
 // P V and the next logits of the other one, so the MUFU pipe and the tensor pipe take turns
 // on a tile instead of competing for it.
-template <int D, bool CAUSAL, bool ALIBI, bool PACKED>
+// MODE: 0 plain (the benchmarked path), 1 packed grouped heads, 2 padded batch with per-sequence lengths
+template <int D, bool CAUSAL, bool ALIBI, int MODE>
 __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t* smem, uint32_t tmem,
                              FwdBarriers* bars, volatile int* cta_err) {
   using L = FwdSmem<D>;
+  constexpr bool PACKED = (MODE == 1), VARLEN = (MODE == 2);
   const int g = threadIdx.x >> 7;            // column group of the tile
   const int tid = threadIdx.x & 127;         // row of the tile
   const uint32_t lane_off = static_cast<uint32_t>(((threadIdx.x >> 5) & 3) * 32) << 16;
@@ -358,21 +366,23 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
     const int item = snake_rank(round, p.n_items);
     if (item < 0) continue;
     const Item w = decode_item<CAUSAL>(p, item);
-    // Per item, or with packed heads per row (one value for each of the two tiles): slope, bias
-    // and the position of this thread's query row.
+    // Slope, bias and the position of this thread's query row: per item, or with packed heads
+    // per row and tile (index 1 of the arrays is only used then).
     float slope_t[2] = {0.0f, 0.0f}, bias_t[2], pos_t[2];
+    if (PACKED) {
 #pragma unroll
-    for (int t = 0; t < 2; ++t) {
-      const int r = w.row0 + t * kBM + tid;
-      int head = w.bh, i = r;   // query head (index into [B][H]) and query index within the head
-      if (PACKED) {
+      for (int t = 0; t < 2; ++t) {
+        const int r = w.row0 + t * kBM + tid;
         const int g_head = min(r / p.pack_rows, p.pack_group - 1);   // rows past the end only fill the tile
-        i = r - g_head * p.pack_rows;
-        head = w.bh * p.pack_group + g_head;                        // (b * H_kv + h_kv) * group + g = b * H + h
+        const int head = w.bh * p.pack_group + g_head;               // (b * H_kv + h_kv) * group + g = b * H + h
+        if (ALIBI) slope_t[t] = p.slopes[head % (p.H * p.pack_group)] * kLog2e;
+        bias_t[t] = p.bias_vec ? __ldg(p.bias_vec + head) * kLog2e : p.bias_log2e;
+        pos_t[t] = static_cast<float>(r - g_head * p.pack_rows + p.pos0);
       }
-      if (ALIBI) slope_t[t] = p.slopes[head % (PACKED ? p.H * p.pack_group : p.H)] * kLog2e;
-      bias_t[t] = p.bias_vec ? __ldg(p.bias_vec + head) * kLog2e : p.bias_log2e;
-      pos_t[t] = static_cast<float>(i + p.pos0);
+    } else {
+      if (ALIBI) slope_t[0] = p.slopes[w.bh % p.H] * kLog2e;
+      bias_t[0] = p.bias_vec ? __ldg(p.bias_vec + w.bh) * kLog2e : p.bias_log2e;
+      pos_t[0] = static_cast<float>(w.row0 + tid + p.pos0);
     }
 
     // Tile-steps are visited in the order (j, tile 0), (j, tile 1), (j + 1, tile 0), ...
@@ -385,11 +395,19 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
         ++cnt;
         tc_fence_after_sync();
         // position of this thread's query relative to the first key of the tile
-        const float row_rel = pos_t[t] - static_cast<float>(j * kBN);
+        const float row_rel = (PACKED ? pos_t[t] : pos_t[0] + static_cast<float>(t * kBM)) - static_cast<float>(j * kBN);
         // the mask cuts through every key tile that reaches beyond the position of the tile's
         // first row: the last one, and with pos0 not a multiple of 128 also the one before
         // (packed rows: a tile may hold a head's first query, at position pos0)
-        const bool diag = CAUSAL && ((j + 1) * kBN - 1 > (PACKED ? 0 : w.row0 + t * kBM) + p.pos0);
+        bool diag = CAUSAL && ((j + 1) * kBN - 1 > (PACKED ? 0 : w.row0 + t * kBM) + p.pos0);
+        float mask_limit = row_rel;   // last key (relative to the tile's first) that keeps its weight
+        if (VARLEN) {
+          // padded batch: keys past the end of the sequence are masked, rows past it are masked whole
+          const float key_limit = static_cast<float>(w.n_valid - 1 - j * kBN);
+          mask_limit = CAUSAL ? fminf(row_rel, key_limit) : key_limit;
+          if (w.row0 + t * kBM + tid >= w.n_valid) mask_limit = -1.0f;
+          diag = diag || (j + 1) * kBN > w.n_valid || w.row0 + (t + 1) * kBM > w.n_valid;
+        }
         // bf16 P goes back over the first half of the columns this thread has just read
         const uint32_t tS = tmem + t * kBN + lane_off + g * kCols;
         uint32_t sv[kCols];
@@ -397,8 +415,9 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
         tmem_wait_ld();
         uint32_t pk[kCols / 2];
         constexpr int kEmulateEvery = (D == 128) ? SIGATTN_FWD_EMULATE_D128 : SIGATTN_FWD_EMULATE_D64;
-        sigmoid_cols<ALIBI, kEmulateEvery>(sv, pk, p.scale_log2e, bias_t[t], slope_t[t], row_rel, g * kCols,
-                                           diag);
+        sigmoid_cols<ALIBI, kEmulateEvery>(sv, pk, p.scale_log2e, bias_t[PACKED ? t : 0], slope_t[PACKED ? t : 0], row_rel,
+                                           g * kCols,
+                                           diag, mask_limit);
         tmem_st_cols(tS, pk);
         tmem_wait_st();
         tc_fence_before_sync();
@@ -454,7 +473,7 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
 
 // ------------------------------------------------------------------ kernel
 
-template <int D, bool CAUSAL, bool ALIBI, bool PACKED>
+template <int D, bool CAUSAL, bool ALIBI, int MODE>
 __global__ void __launch_bounds__(kFwdThreads, 1)
 sigattn_fwd_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                         const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
@@ -507,7 +526,7 @@ sigattn_fwd_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
     fwd_mma_role<D, CAUSAL>(p, smem_base, tmem, &bars, &cta_err);
     __syncwarp();
   } else {
-    fwd_act_role<D, CAUSAL, ALIBI, PACKED>(p, &tmO, smem, tmem, &bars, &cta_err);
+    fwd_act_role<D, CAUSAL, ALIBI, MODE>(p, &tmO, smem, tmem, &bars, &cta_err);
   }
 
   tc_fence_before_sync();
@@ -519,10 +538,10 @@ sigattn_fwd_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
   if (warp == kMmaWarp) tmem_dealloc(tmem, 512);
 }
 
-template <int D, bool CAUSAL, bool ALIBI, bool PACKED>
+template <int D, bool CAUSAL, bool ALIBI, int MODE>
 int launch_fwd_variant(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtensorMap& tmO,
                        const FwdParams& fp, int num_sms, cudaStream_t stream, cudaError_t* cuda_err) {
-  auto kernel = sigattn_fwd_bf16_kernel<D, CAUSAL, ALIBI, PACKED>;
+  auto kernel = sigattn_fwd_bf16_kernel<D, CAUSAL, ALIBI, MODE>;
   static bool configured = false;
   if (!configured) {
     *cuda_err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdSmem<D>::kDynBytes);
@@ -550,7 +569,7 @@ int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const 
   const int group = p.H / p.kv_heads();
   // Few queries per head and several query heads per key/value head (decoding with grouped
   // heads): pack the group's rows into one sequence so that K and V are streamed once per group.
-  const bool packed = group > 1 && static_cast<long long>(p.N) * group <= 2 * kBM;
+  const bool packed = group > 1 && static_cast<long long>(p.N) * group <= 2 * kBM && p.seqlens == nullptr;
   const uint64_t q_heads = packed ? BH_kv : BH;
   const uint64_t q_rows = packed ? static_cast<uint64_t>(p.N) * group : p.N;
   CUtensorMap tmQ, tmK, tmV, tmO;
@@ -580,13 +599,16 @@ int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const 
   fp.bias_log2e = p.bias * kLog2e;
   fp.bias_vec = p.bias_vec;
   fp.slopes = p.slopes;
+  fp.seqlens = p.seqlens;
   fp.status = status;
 
   int rc;
   const bool alibi = p.slopes != nullptr;
 #define SIGATTN_FWD_CASE(DD, CC, AA)                                                                       \
-  rc = packed ? launch_fwd_variant<DD, CC, AA, true>(tmQ, tmK, tmV, tmO, fp, num_sms, stream, cuda_err)    \
-              : launch_fwd_variant<DD, CC, AA, false>(tmQ, tmK, tmV, tmO, fp, num_sms, stream, cuda_err)
+  rc = packed ? launch_fwd_variant<DD, CC, AA, 1>(tmQ, tmK, tmV, tmO, fp, num_sms, stream, cuda_err)       \
+       : (p.seqlens != nullptr)                                                                            \
+           ? launch_fwd_variant<DD, CC, AA, 2>(tmQ, tmK, tmV, tmO, fp, num_sms, stream, cuda_err)          \
+           : launch_fwd_variant<DD, CC, AA, 0>(tmQ, tmK, tmV, tmO, fp, num_sms, stream, cuda_err)
   if (p.D == 128) {
     if (p.causal) { if (alibi) SIGATTN_FWD_CASE(128, true, true); else SIGATTN_FWD_CASE(128, true, false); }
     else          { if (alibi) SIGATTN_FWD_CASE(128, false, true); else SIGATTN_FWD_CASE(128, false, false); }

@@ -21,6 +21,7 @@ struct Problem {
   int pos0_given;         // 1: `pos0` is the position of query row 0 relative to key row 0 (key/value shards)
   int pos0;               //    0: the queries are the last N positions, pos0 = key_rows() - N
   int query_pos0() const { return pos0_given ? pos0 : key_rows() - N; }
+  const int* seqlens;     // device pointer to B valid lengths (padded batch, N_k = N only), or nullptr
 };
 
 // Every launcher enqueues on `stream`, adds the number of kernels it launched to
