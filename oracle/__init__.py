@@ -13,4 +13,5 @@ from .sigattn_oracle import (  # noqa: F401
     sigattn_bwd,
     sigattn_bwd_dbias,
     sigattn_fwd_sequence_form,
+    seqlen_norm,
 )

@@ -67,6 +67,17 @@ Readings of the paper taken here
     dQ rows are zero, dK and dV do not see them).  The paper does not print this; it is the
     usual padding mask, and it makes the call equal to separate calls on the unpadded
     sequences.  Only for N_q = N_k.
+  * Sequence-length normalisation (the ablation in Appendix G that compares b = -log n with
+    the scaling n^-alpha sigma(Q K^T / sqrt(d)) V): every row of O is multiplied by one
+    factor r_i.  Without a mask r_i = n^-alpha for all rows.  For the causal form the paper
+    prints an n = 3 matrix whose rows read 1, 0.5^-alpha, 0.33^-alpha under the label
+    n^-alpha; taken literally 0.5^-alpha = 2^alpha would grow with the row, against the
+    label and against the purpose (dividing by the number of keys a row sees), so it is read
+    as r_i = (i + 1)^-alpha = (1 / (i + 1))^alpha, i + 1 being the number of keys row i keeps.
+    With N_q != N_k the count is pos_i + 1 with pos_i the query's position.  The factor does
+    not depend on Q, K, V, so the backward is the plain one with dO replaced by r_i dO_i; a
+    bias and slopes may be combined with it.  `row_scale` takes any vector of N_q factors,
+    `seqlen_norm` builds the paper's.
 
 Every function is pinned by tests that do not call back into this file's own
 formulae (closed forms, brute-force loops, finite differences, the paper's second
@@ -85,6 +96,7 @@ __all__ = [
     "sigattn_bwd",
     "sigattn_bwd_dbias",
     "sigattn_fwd_sequence_form",
+    "seqlen_norm",
 ]
 
 
@@ -194,6 +206,31 @@ def _seqlens(seqlens, num_batch, n_q, n_k):
     return [int(x) for x in s]
 
 
+def seqlen_norm(n_q, alpha, causal, n_k=None, pos0=None):
+    """Row factors of the sequence-length normalisation (Appendix G, ablation of n^-alpha
+    against the bias; see the header for the reading of the causal form): without a mask
+    n_k^-alpha for every row, causal (pos_i + 1)^-alpha with pos_i = i + pos0 the query's
+    position, i.e. one over the number of keys the row keeps, to the power alpha.  A row
+    that keeps no key (position before key 0) gets factor 0.  Returns float64 [n_q]."""
+    n_k = n_q if n_k is None else n_k
+    _, off = _query_offset(n_k, n_q, pos0)
+    if not causal:
+        return np.full(n_q, float(n_k) ** (-float(alpha)), dtype=np.float64)
+    count = np.arange(n_q, dtype=np.float64) + float(off) + 1.0
+    r = np.zeros(n_q, dtype=np.float64)
+    r[count >= 1.0] = count[count >= 1.0] ** (-float(alpha))
+    return r
+
+
+def _row_scale(row_scale, n_q):
+    if row_scale is None:
+        return np.ones(n_q, dtype=np.float64)
+    r = np.asarray(row_scale, dtype=np.float64).reshape(-1)
+    if r.shape[0] != n_q:
+        raise ValueError("row_scale must hold one factor per query row")
+    return r
+
+
 def _row_ranges(n, row_block):
     """Query rows are independent in the forward and enter dK, dV only through a sum
     over rows, so they may be visited in slabs to bound memory (an n x n float64 matrix
@@ -202,13 +239,15 @@ def _row_ranges(n, row_block):
     return [(a, min(n, a + step)) for a in range(0, n, step)]
 
 
-def sigattn_fwd(q, k, v, scale, bias, causal=False, alibi_slopes=None, row_block=None, pos0=None, seqlens=None):
+def sigattn_fwd(q, k, v, scale, bias, causal=False, alibi_slopes=None, row_block=None, pos0=None, seqlens=None,
+                row_scale=None):
     """O = sigmoid(scale * Q K^T + b [+ position bias]) [* causal mask] V  (Eq. 3).
 
     q: [B, H, N, D]; k, v: [B, H_kv, N, D] with H a multiple of H_kv (any float dtype;
     converted to float64).
     bias: scalar, or an array that broadcasts to [B, H] (one bias per sequence and head).
     pos0: position of query row 0 relative to key row 0 (default: rows of k minus rows of q).
+    row_scale: one factor per query row (sequence-length normalisation), or None.
     Returns O as float64 [B, H, N, D].
     """
     q, k, v = _as_f64(q, k, v)
@@ -217,6 +256,7 @@ def sigattn_fwd(q, k, v, scale, bias, causal=False, alibi_slopes=None, row_block
     slopes = _slopes(alibi_slopes, H)
     bias_bh = _bias_per_head(bias, B, H)
     lens = _seqlens(seqlens, B, N, k.shape[2])
+    r = _row_scale(row_scale, N)
     o = np.zeros((B, H, N, D), dtype=np.float64)
     for b in range(B):
         for h in range(H):
@@ -224,17 +264,18 @@ def sigattn_fwd(q, k, v, scale, bias, causal=False, alibi_slopes=None, row_block
             for i0, i1 in _row_ranges(N, row_block):
                 p = attention_weights(q[b, h], k[b, hk], scale, bias_bh[b, h], causal, slopes[h], i0, i1, pos0,
                                       lens[b])
-                o[b, h, i0:i1] = p @ v[b, hk]
+                o[b, h, i0:i1] = r[i0:i1, None] * (p @ v[b, hk])
     return o
 
 
-def _bwd_all(q, k, v, d_o, scale, bias, causal, alibi_slopes, row_block, pos0=None, seqlens=None):
+def _bwd_all(q, k, v, d_o, scale, bias, causal, alibi_slopes, row_block, pos0=None, seqlens=None, row_scale=None):
     q, k, v, d_o = _as_f64(q, k, v, d_o)
     B, H, N, D = q.shape
     group = _kv_group(H, k)
     slopes = _slopes(alibi_slopes, H)
     bias_bh = _bias_per_head(bias, B, H)
     lens = _seqlens(seqlens, B, N, k.shape[2])
+    r = _row_scale(row_scale, N)
     dq = np.zeros_like(q)
     dk = np.zeros_like(k)
     dv = np.zeros_like(v)
@@ -245,7 +286,7 @@ def _bwd_all(q, k, v, d_o, scale, bias, causal, alibi_slopes, row_block, pos0=No
             for i0, i1 in _row_ranges(N, row_block):
                 p = attention_weights(q[b, h], k[b, hk], scale, bias_bh[b, h], causal, slopes[h], i0, i1, pos0,
                                       lens[b])
-                do_rows = d_o[b, h, i0:i1]
+                do_rows = r[i0:i1, None] * d_o[b, h, i0:i1]   # O = r (P V): the factor passes to dO
                 dv[b, hk] += p.T @ do_rows
                 dp = do_rows @ v[b, hk].T
                 ds = p * (1.0 - p) * dp
@@ -256,7 +297,7 @@ def _bwd_all(q, k, v, d_o, scale, bias, causal, alibi_slopes, row_block, pos0=No
 
 
 def sigattn_bwd(q, k, v, d_o, scale, bias, causal=False, alibi_slopes=None, row_block=None, pos0=None,
-                seqlens=None):
+                seqlens=None, row_scale=None):
     """Gradients of L = sum(O * dO) with respect to Q, K, V (sigmoid column of the
     forward/backward table in Appendix F.1, with the 1/sqrt(d) factor; see header).
 
@@ -264,18 +305,18 @@ def sigattn_bwd(q, k, v, d_o, scale, bias, causal=False, alibi_slopes=None, row_
     than q (see header).
     Returns (dQ, dK, dV), float64, shaped like q, k, v.
     """
-    return _bwd_all(q, k, v, d_o, scale, bias, causal, alibi_slopes, row_block, pos0, seqlens)[:3]
+    return _bwd_all(q, k, v, d_o, scale, bias, causal, alibi_slopes, row_block, pos0, seqlens, row_scale)[:3]
 
 
 def sigattn_bwd_dbias(q, k, v, d_o, scale, bias, causal=False, alibi_slopes=None, row_block=None, pos0=None,
-                      seqlens=None):
+                      seqlens=None, row_scale=None):
     """Gradient of L = sum(O * dO) with respect to a bias held per (batch, head):
     db[b, h] = sum_ij dS_ij with dS = P (1 - P) dP as in sigattn_bwd (see header).  A
     bias shared by several heads or sequences gets the sum of their entries.
 
     Returns float64 [B, H].
     """
-    return _bwd_all(q, k, v, d_o, scale, bias, causal, alibi_slopes, row_block, pos0, seqlens)[3]
+    return _bwd_all(q, k, v, d_o, scale, bias, causal, alibi_slopes, row_block, pos0, seqlens, row_scale)[3]
 
 
 def sigattn_fwd_sequence_form(q, k, v, scale, n_bias):

@@ -567,3 +567,83 @@ def test_padded_batch_equals_separate_unpadded_calls(causal):
         np.testing.assert_array_equal(g, r)
     with pytest.raises(ValueError):
         oracle.sigattn_fwd(q, k, v, scale, -1.0, causal, seqlens=[7, 8, 1])
+
+
+# ------------------------------------------------------- sequence-length normalisation
+
+
+@pytest.mark.parametrize("alpha", [1.0, 0.5])
+def test_seqlen_norm_matches_printed_n3_bases(alpha):
+    """The causal row factors are the printed bases 1, 0.5, 0.33 raised to alpha (0.33 is
+    1/3 to two places); without a mask every row gets n^-alpha."""
+    bases = np.loadtxt(os.path.join(GOLDEN, "seqlen_norm_n3.txt"))
+    r = oracle.seqlen_norm(3, alpha, True)
+    np.testing.assert_allclose(r, bases ** alpha, rtol=1.1e-2)
+    assert r[0] == 1.0 and r[1] == 0.5 ** alpha
+    assert np.all(np.diff(r) < 0)          # more keys, smaller factor
+    np.testing.assert_allclose(oracle.seqlen_norm(3, alpha, False), np.full(3, 3.0 ** -alpha), rtol=1e-15)
+    # queries at the end of a longer key sequence count the keys they see
+    np.testing.assert_allclose(oracle.seqlen_norm(2, alpha, True, n_k=5), np.array([4.0, 5.0]) ** -alpha, rtol=1e-15)
+    assert oracle.seqlen_norm(3, alpha, True, n_k=4, pos0=-2)[:2].tolist() == [0.0, 0.0]
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_seqlen_norm_q_zero_closed_form(causal):
+    """Q = 0, b = 0: every kept weight is 1/2.  With alpha = 1 row i of O is half the mean
+    of the values it sees (a running mean when causal); with alpha = 1/2 half the sum over
+    sqrt(count)."""
+    B, H, N, D = 2, 2, 9, 3
+    q = np.zeros((B, H, N, D))
+    k, v = rnd((B, H, N, D), 150), rnd((B, H, N, D), 151)
+    count = np.arange(1, N + 1, dtype=np.float64) if causal else np.full(N, float(N))
+    sums = np.cumsum(v, axis=2) if causal else np.repeat(v.sum(axis=2, keepdims=True), N, axis=2)
+    for alpha in (1.0, 0.5):
+        o = oracle.sigattn_fwd(q, k, v, 0.3, 0.0, causal, row_scale=oracle.seqlen_norm(N, alpha, causal))
+        np.testing.assert_allclose(o, 0.5 * sums / (count ** alpha)[None, None, :, None], rtol=1e-13, atol=1e-15)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_row_scale_brute_force_and_finite_differences(causal):
+    """Any vector of row factors: forward by explicit loops; gradients of L = sum(O * dO)
+    with respect to Q, K, V and a per-(batch, head) bias by central differences."""
+    B, H, N, D = 1, 2, 5, 3
+    q, k, v, d_o = (rnd((B, H, N, D), s) for s in (160, 161, 162, 163))
+    slopes = np.array([0.5, 0.125])
+    scale = 0.6
+    bias = np.array([[-0.7, 0.2]])
+    r = np.array([1.0, 0.7, 0.1, 2.0, 0.0]) if not causal else oracle.seqlen_norm(N, 0.5, True)
+    o = oracle.sigattn_fwd(q, k, v, scale, bias, causal, slopes, row_scale=r)
+    ref = np.zeros_like(o)
+    for h in range(H):
+        for i in range(N):
+            for j in range(N):
+                if causal and j > i:
+                    continue
+                x = scale * float(q[0, h, i] @ k[0, h, j]) + bias[0, h] - slopes[h] * abs(i - j)
+                ref[0, h, i] += r[i] * scalar_sigmoid(x) * v[0, h, j]
+    np.testing.assert_allclose(o, ref, rtol=1e-13, atol=1e-16)
+
+    def f():
+        return float(np.sum(oracle.sigattn_fwd(q, k, v, scale, bias, causal, slopes, row_scale=r) * d_o))
+
+    dq, dk, dv = oracle.sigattn_bwd(q, k, v, d_o, scale, bias, causal, slopes, row_scale=r)
+    db = oracle.sigattn_bwd_dbias(q, k, v, d_o, scale, bias, causal, slopes, row_scale=r)
+    step = 1e-6
+    for name, x, g in (("q", q, dq), ("k", k, dk), ("v", v, dv), ("bias", bias, db)):
+        fd = np.zeros_like(x)
+        it = np.nditer(x, flags=["multi_index"])
+        for _ in it:
+            idx = it.multi_index
+            old = x[idx]
+            x[idx] = old + step
+            lp = f()
+            x[idx] = old - step
+            lm = f()
+            x[idx] = old
+            fd[idx] = (lp - lm) / (2 * step)
+        err = np.linalg.norm(fd - g) / np.linalg.norm(fd)
+        assert err < 1e-7, (name, err)
+    # the factor must reach dV as well as dQ, dK: dropping it from any of them is far off
+    plain = oracle.sigattn_bwd(q, k, v, d_o, scale, bias, causal, slopes)
+    for g, pl in zip((dq, dk, dv), plain):
+        assert np.linalg.norm(g - pl) / np.linalg.norm(g) > 0.05
