@@ -242,6 +242,41 @@ SIGATTN_API int sigattn_bwd_varlen(const void* q, const void* k, const void* v, 
                        float* dbias_bh,
                        void* workspace, size_t workspace_bytes, void* stream);
 
+/* Sequence-length normalisation (Appendix G, the ablation that compares the bias b = -log n with
+ * the scaling n^-alpha sigma(Q K^T / sqrt(d)) V and its causal form, the equation labelled
+ * "ar_seq_len_normalization"): O_i = r_i sum_j P_ij V_j with one factor r_i per query row, shared by
+ * all batch entries and heads.  The factor does not depend on Q, K, V, so the backward is the plain
+ * one with dO_i replaced by r_i dO_i (dV = (r P)^T dO, dS = P (1 - P) (r dP)); db, if asked for,
+ * is the sum of that dS.  The bf16 backward forms r_i dO_i in one extra pass (rounded to bf16,
+ * held in the dq buffer until dq itself is written at the end of the call).
+ *
+ * row_scale: DEVICE pointer to N_q floats, 4-byte aligned, read only.  sigattn_seqlen_norm fills
+ *   such a vector with the paper's factors: N_k^-alpha for every row without a mask; with the
+ *   causal mask (pos_i + 1)^-alpha, pos_i = i + N_k - N_q being the query's position and
+ *   pos_i + 1 the number of keys the row keeps (the printed n = 3 example reads 1, 0.5, 0.33 as
+ *   bases; its exponent is taken as +alpha on these bases, i.e. -alpha on the counts 1, 2, 3).
+ *   Any other vector of factors may be passed as well.
+ * Other arguments as in sigattn_fwd_nk / sigattn_bwd_nk (bias_bh and dbias_bh as in
+ * sigattn_fwd_gqa / sigattn_bwd_gqa).  Errors as there; row_scale == NULL is SIGATTN_ERR_NULL. */
+SIGATTN_API int sigattn_fwd_rowscale(const void* q, const void* k, const void* v, void* o,
+                         int B, int H, int H_kv, int N_q, int N_k, int D,
+                         float scale, float bias, const float* bias_bh, int causal,
+                         const float* row_scale,
+                         const float* alibi_slopes, int dtype, void* stream);
+
+SIGATTN_API int sigattn_bwd_rowscale(const void* q, const void* k, const void* v, const void* d_o,
+                         void* dq, void* dk, void* dv,
+                         int B, int H, int H_kv, int N_q, int N_k, int D,
+                         float scale, float bias, const float* bias_bh, int causal,
+                         const float* row_scale,
+                         const float* alibi_slopes, int dtype,
+                         float* dbias_bh,
+                         void* workspace, size_t workspace_bytes, void* stream);
+
+/* Writes the paper's N_q factors (see above) to the DEVICE vector row_scale, asynchronously on
+ * `stream`.  causal = 1 needs N_k >= N_q. */
+SIGATTN_API int sigattn_seqlen_norm(float* row_scale, int N_q, int N_k, float alpha, int causal, void* stream);
+
 /* Bytes of scratch sigattn_bwd needs for this problem (0 for the fp32 debug path).
  * Returns 0 for invalid shapes as well; sigattn_bwd reports those. */
 SIGATTN_API size_t sigattn_bwd_workspace_bytes(int B, int H, int N, int D, int dtype);

@@ -35,6 +35,9 @@ _BINDING_NAMES = (
     "sigattn_bwd_shard",
     "sigattn_fwd_varlen",
     "sigattn_bwd_varlen",
+    "sigattn_fwd_rowscale",
+    "sigattn_bwd_rowscale",
+    "sigattn_seqlen_norm",
     "lib",
 )
 

@@ -66,6 +66,15 @@ _lib.sigattn_bwd_varlen.restype = _c.c_int
 _lib.sigattn_bwd_varlen.argtypes = [_c.c_void_p] * 7 + [_c.c_int] * 5 + [_c.c_float, _c.c_float, _c.c_void_p, _c.c_int,
                                                                            _c.c_void_p, _c.c_void_p, _c.c_int, _c.c_void_p,
                                                                            _c.c_void_p, _c.c_size_t, _c.c_void_p]
+_lib.sigattn_fwd_rowscale.restype = _c.c_int
+_lib.sigattn_fwd_rowscale.argtypes = [_c.c_void_p] * 4 + [_c.c_int] * 6 + [_c.c_float, _c.c_float, _c.c_void_p, _c.c_int,
+                                                                             _c.c_void_p, _c.c_void_p, _c.c_int, _c.c_void_p]
+_lib.sigattn_bwd_rowscale.restype = _c.c_int
+_lib.sigattn_bwd_rowscale.argtypes = [_c.c_void_p] * 7 + [_c.c_int] * 6 + [_c.c_float, _c.c_float, _c.c_void_p, _c.c_int,
+                                                                             _c.c_void_p, _c.c_void_p, _c.c_int, _c.c_void_p,
+                                                                             _c.c_void_p, _c.c_size_t, _c.c_void_p]
+_lib.sigattn_seqlen_norm.restype = _c.c_int
+_lib.sigattn_seqlen_norm.argtypes = [_c.c_void_p, _c.c_int, _c.c_int, _c.c_float, _c.c_int, _c.c_void_p]
 _lib.sigattn_bwd_workspace_bytes.restype = _c.c_size_t
 _lib.sigattn_bwd_workspace_bytes.argtypes = [_c.c_int] * 5
 _lib.sigattn_step_host.restype = _c.c_int
@@ -102,6 +111,7 @@ EXPORTED = [
     "sigattn_selftest_bounded_wait", "sigattn_fwd_bias_vec", "sigattn_bwd_bias_vec",
     "sigattn_fwd_gqa", "sigattn_bwd_gqa", "sigattn_fwd_nk", "sigattn_bwd_nk",
     "sigattn_fwd_shard", "sigattn_bwd_shard", "sigattn_fwd_varlen", "sigattn_bwd_varlen",
+    "sigattn_fwd_rowscale", "sigattn_bwd_rowscale", "sigattn_seqlen_norm",
 ]
 
 
@@ -502,6 +512,77 @@ def sigattn_bwd_varlen(q, k, v, d_o, scale, bias, seqlens, causal=False, alibi_s
                                      float(scale), 0.0 if vec else float(bias), _ptr(bias) if vec else None,
                                      int(bool(causal)), _ptr(seqlens), _ptr(alibi_slopes), code, _ptr(dbias),
                                      _ptr(workspace), ws_bytes, _stream_ptr(stream))
+    if rc != 0:
+        raise SigattnError(rc)
+    return dq, dk, dv, dbias
+
+
+def _check_row_scale(row_scale, q):
+    import torch
+    if (not isinstance(row_scale, torch.Tensor) or not row_scale.is_cuda or row_scale.dtype != torch.float32
+            or tuple(row_scale.shape) != (q.shape[2],) or not row_scale.is_contiguous()
+            or row_scale.device != q.device):
+        raise ValueError("row_scale must be a contiguous float32 CUDA tensor of shape [N_q] on q's device")
+
+
+def sigattn_seqlen_norm(n_q, n_k, alpha, causal, device, stream=None):
+    """The paper's row factors of the sequence-length normalisation as a float32 CUDA [n_q]:
+    n_k^-alpha without a mask, (position + 1)^-alpha with the causal mask."""
+    import torch
+    out = torch.empty(int(n_q), dtype=torch.float32, device=device)
+    with torch.cuda.device(out.device):
+        rc = _lib.sigattn_seqlen_norm(_ptr(out), int(n_q), int(n_k), float(alpha), int(bool(causal)),
+                                      _stream_ptr(stream))
+    if rc != 0:
+        raise SigattnError(rc)
+    return out
+
+
+def sigattn_fwd_rowscale(q, k, v, scale, bias, row_scale, causal=False, alibi_slopes=None, out=None, stream=None):
+    """O_i = row_scale[i] * sum_j P_ij V_j (sequence-length normalisation); q [B, H, N_q, D], k, v
+    [B, H_kv, N_k, D]; `bias`: float or float32 CUDA [B, H]."""
+    import torch
+    B, H, H_kv, N_q, N_k, D = _check_nk(q, k, v)
+    _check_row_scale(row_scale, q)
+    if out is None:
+        out = torch.empty_like(q)
+    else:
+        _check_same([q, out], ["q", "out"])
+    vec = isinstance(bias, torch.Tensor)
+    if vec:
+        _check_bias_vec(bias, q)
+    with torch.cuda.device(q.device):
+        rc = _lib.sigattn_fwd_rowscale(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, H, H_kv, N_q, N_k, D, float(scale),
+                                       0.0 if vec else float(bias), _ptr(bias) if vec else None, int(bool(causal)),
+                                       _ptr(row_scale), _ptr(alibi_slopes), _dtype_code(q), _stream_ptr(stream))
+    if rc != 0:
+        raise SigattnError(rc)
+    return out
+
+
+def sigattn_bwd_rowscale(q, k, v, d_o, scale, bias, row_scale, causal=False, alibi_slopes=None, want_dbias=False,
+                         workspace=None, stream=None):
+    """Backward of sigattn_fwd_rowscale: (dQ, dK, dV, dbias or None)."""
+    import torch
+    B, H, H_kv, N_q, N_k, D = _check_nk(q, k, v)
+    _check_same([q, d_o], ["q", "d_o"])
+    _check_row_scale(row_scale, q)
+    code = _dtype_code(q)
+    dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+    vec = isinstance(bias, torch.Tensor)
+    if vec:
+        _check_bias_vec(bias, q)
+    dbias = torch.empty((B, H), dtype=torch.float32, device=q.device) if want_dbias else None
+    need = sigattn_bwd_workspace_bytes(B, H, N_q, D, code)
+    if workspace is None and need > 0:
+        workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    with torch.cuda.device(q.device):
+        rc = _lib.sigattn_bwd_rowscale(_ptr(q), _ptr(k), _ptr(v), _ptr(d_o), _ptr(dq), _ptr(dk), _ptr(dv), B, H, H_kv,
+                                       N_q, N_k, D, float(scale), 0.0 if vec else float(bias),
+                                       _ptr(bias) if vec else None, int(bool(causal)), _ptr(row_scale),
+                                       _ptr(alibi_slopes), code, _ptr(dbias), _ptr(workspace), ws_bytes,
+                                       _stream_ptr(stream))
     if rc != 0:
         raise SigattnError(rc)
     return dq, dk, dv, dbias

@@ -102,7 +102,8 @@ int check_lengths(int B, int H, int H_kv, int N, int N_k, int D, int causal, int
 
 int fwd_any(const void* q, const void* k, const void* v, void* o, int B, int H, int H_kv, int N, int N_k, int D,
             float scale, float bias, const float* bias_vec, int causal, const float* alibi_slopes, int dtype,
-            void* stream, int pos0_given = 0, int pos0 = 0, const int* seqlens = nullptr) {
+            void* stream, int pos0_given = 0, int pos0 = 0, const int* seqlens = nullptr,
+            const float* row_scale = nullptr) {
   if (!q || !k || !v || !o) return SIGATTN_ERR_NULL;
   if (int rc = check_lengths(B, H, H_kv, N, N_k, D, causal, pos0_given, pos0)) return rc;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return SIGATTN_ERR_ALIGN;
@@ -113,7 +114,7 @@ int fwd_any(const void* q, const void* k, const void* v, void* o, int B, int H, 
   int* status = nullptr;
   if (int rc = device_setup(&dev, &status)) return rc;
   sigattn::Problem p{B, H, N, D, scale, bias, causal, alibi_slopes, bias_vec, nullptr, H_kv, N_k, pos0_given, pos0,
-                     seqlens};
+                     seqlens, row_scale};
   unsigned long long launches = 0;
   cudaError_t ce = cudaSuccess;
   int rc;
@@ -132,7 +133,7 @@ int fwd_any(const void* q, const void* k, const void* v, void* o, int B, int H, 
 int bwd_any(const void* q, const void* k, const void* v, const void* d_o, void* dq, void* dk, void* dv, int B, int H,
             int H_kv, int N, int N_k, int D, float scale, float bias, const float* bias_vec, float* dbias, int causal,
             const float* alibi_slopes, int dtype, void* workspace, size_t workspace_bytes, void* stream,
-            int pos0_given = 0, int pos0 = 0, const int* seqlens = nullptr) {
+            int pos0_given = 0, int pos0 = 0, const int* seqlens = nullptr, const float* row_scale = nullptr) {
   if (!q || !k || !v || !d_o || !dq || !dk || !dv) return SIGATTN_ERR_NULL;
   if (int rc = check_lengths(B, H, H_kv, N, N_k, D, causal, pos0_given, pos0)) return rc;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(d_o) || !aligned16(dq) || !aligned16(dk) ||
@@ -151,7 +152,7 @@ int bwd_any(const void* q, const void* k, const void* v, const void* d_o, void* 
   int* status = nullptr;
   if (int rc = device_setup(&dev, &status)) return rc;
   sigattn::Problem p{B, H, N, D, scale, bias, causal, alibi_slopes, bias_vec, dbias, H_kv, N_k, pos0_given, pos0,
-                     seqlens};
+                     seqlens, row_scale};
   unsigned long long launches = 0;
   cudaError_t ce = cudaSuccess;
   int rc;
@@ -494,5 +495,44 @@ const char* sigattn_last_cuda_error(void) { return cudaGetErrorString(t_last_cud
 int sigattn_version(void) { return 100; }
 
 unsigned long long sigattn_launch_count(void) { return g_launches.load(); }
+
+int sigattn_fwd_rowscale(const void* q, const void* k, const void* v, void* o, int B, int H, int H_kv, int N_q,
+                         int N_k, int D, float scale, float bias, const float* bias_bh, int causal,
+                         const float* row_scale, const float* alibi_slopes, int dtype, void* stream) {
+  if (!row_scale) return SIGATTN_ERR_NULL;
+  if ((reinterpret_cast<uintptr_t>(row_scale) & 3u) || (reinterpret_cast<uintptr_t>(bias_bh) & 3u))
+    return SIGATTN_ERR_ALIGN;
+  return fwd_any(q, k, v, o, B, H, H_kv, N_q, N_k, D, scale, bias, bias_bh, causal, alibi_slopes, dtype, stream, 0, 0,
+                 nullptr, row_scale);
+}
+
+int sigattn_bwd_rowscale(const void* q, const void* k, const void* v, const void* d_o, void* dq, void* dk, void* dv,
+                         int B, int H, int H_kv, int N_q, int N_k, int D, float scale, float bias,
+                         const float* bias_bh, int causal, const float* row_scale, const float* alibi_slopes,
+                         int dtype, float* dbias_bh, void* workspace, size_t workspace_bytes, void* stream) {
+  if (!row_scale) return SIGATTN_ERR_NULL;
+  if ((reinterpret_cast<uintptr_t>(row_scale) & 3u) || (reinterpret_cast<uintptr_t>(bias_bh) & 3u) ||
+      (reinterpret_cast<uintptr_t>(dbias_bh) & 3u))
+    return SIGATTN_ERR_ALIGN;
+  return bwd_any(q, k, v, d_o, dq, dk, dv, B, H, H_kv, N_q, N_k, D, scale, bias, bias_bh, dbias_bh, causal,
+                 alibi_slopes, dtype, workspace, workspace_bytes, stream, 0, 0, nullptr, row_scale);
+}
+
+int sigattn_seqlen_norm(float* row_scale, int N_q, int N_k, float alpha, int causal, void* stream) {
+  if (!row_scale) return SIGATTN_ERR_NULL;
+  if (reinterpret_cast<uintptr_t>(row_scale) & 3u) return SIGATTN_ERR_ALIGN;
+  if (N_q < 1 || N_k < 1 || (causal == 1 && N_k < N_q)) return SIGATTN_ERR_SHAPE;
+  if (causal != 0 && causal != 1) return SIGATTN_ERR_FLAG;
+  int dev = 0;
+  int* status = nullptr;
+  if (int rc = device_setup(&dev, &status)) return rc;
+  unsigned long long launches = 0;
+  cudaError_t ce = cudaSuccess;
+  const int rc = sigattn::launch_seqlen_norm(row_scale, N_q, N_k, N_k - N_q, causal, alpha,
+                                             static_cast<cudaStream_t>(stream), &launches, &ce);
+  g_launches.fetch_add(launches);
+  if (rc == SIGATTN_ERR_CUDA) t_last_cuda = ce;
+  return rc;
+}
 
 }  // extern "C"

@@ -621,6 +621,24 @@ sigattn_bwd_convert_dq_kernel(const float4* __restrict__ ws, uint2* __restrict__
   }
 }
 
+// Sequence-length normalisation, O = r (P V) with one factor per query row: the whole backward
+// is the plain one on r_i dO_i.  This pass writes bf16(r_i dO_i) for every row ([B*H, N, D]
+// row-major, 8 elements per thread); the main kernel then reads it in place of dO.
+__device__ __forceinline__ uint32_t scale_bf16x2(uint32_t x, float r) {
+  return pack_bf16x2(r * __uint_as_float(x << 16), r * __uint_as_float(x & 0xffff0000u));
+}
+
+__global__ void __launch_bounds__(256)
+sigattn_bwd_scale_rows_kernel(const uint4* __restrict__ d_o, const float* __restrict__ row_scale,
+                              uint4* __restrict__ out, size_t n_vec8, int N, int vec_per_row) {
+  const size_t stride = static_cast<size_t>(gridDim.x) * blockDim.x;
+  for (size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < n_vec8; i += stride) {
+    const float r = __ldg(row_scale + static_cast<int>((i / vec_per_row) % N));
+    const uint4 x = d_o[i];
+    out[i] = make_uint4(scale_bf16x2(x.x, r), scale_bf16x2(x.y, r), scale_bf16x2(x.z, r), scale_bf16x2(x.w, r));
+  }
+}
+
 template <int D, bool CAUSAL, bool ALIBI, bool DBIAS, bool GROUPED>
 int launch_bwd_variant(const CUtensorMap* maps, const BwdParams& bp, int num_sms, cudaStream_t stream,
                        cudaError_t* cuda_err) {
@@ -666,7 +684,9 @@ int launch_bwd_bf16(const void* q, const void* k, const void* v, const void* d_o
   const uint64_t BH = static_cast<uint64_t>(p.B) * p.H;             // query heads: Q, dO, the dQ accumulator
   const uint64_t BH_kv = static_cast<uint64_t>(p.B) * p.kv_heads();  // K, V, dK, dV
   CUtensorMap maps[7];
-  const void* ptrs[6] = {q, k, v, d_o, dk, dv};
+  // with factors per query row the main kernel reads r dO, staged in the dq buffer: nothing
+  // writes dq before the conversion step at the end, which reads only the workspace
+  const void* ptrs[6] = {q, k, v, p.row_scale != nullptr ? dq : d_o, dk, dv};
   for (int i = 0; i < 6; ++i) {
     const uint64_t heads = (i == 0 || i == 3) ? BH : BH_kv;
     const uint64_t rows = (i == 0 || i == 3) ? p.N : p.key_rows();
@@ -707,14 +727,24 @@ int launch_bwd_bf16(const void* q, const void* k, const void* v, const void* d_o
     if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
   }
 
+  if (p.row_scale != nullptr) {
+    const size_t n_vec8 = n_elems / 8;
+    const size_t want = n_vec8 / 256 + 1, cap = static_cast<size_t>(num_sms) * 8;
+    sigattn_bwd_scale_rows_kernel<<<static_cast<int>(want < cap ? want : cap), 256, 0, stream>>>(
+        static_cast<const uint4*>(d_o), p.row_scale, static_cast<uint4*>(dq), n_vec8, p.N, p.D / 8);
+    *cuda_err = cudaGetLastError();
+    if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
+    *launches += 1;
+  }
+
   // step 2: main kernel
   const bool timed = (t_ev_start != nullptr && t_ev_stop != nullptr);
   if (timed) cudaEventRecord(t_ev_start, stream);
   int rc;
   const bool alibi = p.slopes != nullptr;
   // the bias gradient costs the activation groups a running sum (4-5 % of the kernel), so it
-  // is compiled in only where it is asked for
   // is compiled in only where it is asked for; likewise the loop over a group's query heads
+  // and the per-sequence lengths
 #define SIGATTN_BWD_CASE(DD, CC, AA)                                                                        \
   rc = (bp.group > 1 || bp.seqlens != nullptr)                                                              \
            ? ((p.dbias != nullptr) ? launch_bwd_variant<DD, CC, AA, true, true>(maps, bp, num_sms, stream, cuda_err)   \

@@ -35,7 +35,7 @@ __global__ void fwd_fp32_kernel(const float* __restrict__ q, const float* __rest
                                 const float* __restrict__ v, float* __restrict__ o, int H, int N, int D,
                                 float scale, float bias, int causal, const float* __restrict__ slopes,
                                 const float* __restrict__ bias_vec, int H_kv, int N_k, int off,
-                                const int* __restrict__ seqlens) {
+                                const int* __restrict__ seqlens, const float* __restrict__ row_scale) {
   __shared__ float sq[128];
   __shared__ float sp[kThreads];
   const int i = blockIdx.x, bh = blockIdx.y, t = threadIdx.x;
@@ -65,7 +65,7 @@ __global__ void fwd_fp32_kernel(const float* __restrict__ q, const float* __rest
     }
     __syncthreads();
   }
-  if (t < D) o[base + static_cast<size_t>(i) * D + t] = acc;
+  if (t < D) o[base + static_cast<size_t>(i) * D + t] = row_scale ? row_scale[i] * acc : acc;
 }
 
 // dQ_i = scale * sum_j dS_ij K_j.  grid (N, B*H).
@@ -74,7 +74,8 @@ __global__ void bwd_dq_fp32_kernel(const float* __restrict__ q, const float* __r
                                    float* __restrict__ dq, int H, int N, int D, float scale, float bias,
                                    int causal, const float* __restrict__ slopes,
                                    const float* __restrict__ bias_vec, float* __restrict__ dbias, int H_kv,
-                                   int N_k, int off, const int* __restrict__ seqlens) {
+                                   int N_k, int off, const int* __restrict__ seqlens,
+                                   const float* __restrict__ row_scale) {
   __shared__ float sq[128];
   __shared__ float sdo[128];
   __shared__ float sds[kThreads];
@@ -86,7 +87,8 @@ __global__ void bwd_dq_fp32_kernel(const float* __restrict__ q, const float* __r
   const float slope = slopes ? slopes[bh % H] : 0.0f;
   if (t < D) {
     sq[t] = q[base + static_cast<size_t>(i) * D + t];
-    sdo[t] = d_o[base + static_cast<size_t>(i) * D + t];
+    // O = r (P V): the row's factor passes to dO
+    sdo[t] = d_o[base + static_cast<size_t>(i) * D + t] * (row_scale ? row_scale[i] : 1.0f);
   }
   __syncthreads();
   const int n_valid = seqlens ? max(0, min(N, seqlens[bh / H])) : N_k;
@@ -129,7 +131,7 @@ __global__ void bwd_dkdv_fp32_kernel(const float* __restrict__ q, const float* _
                                      float* __restrict__ dk, float* __restrict__ dv, int H, int N, int D,
                                      float scale, float bias_scalar, int causal, const float* __restrict__ slopes,
                                      const float* __restrict__ bias_vec, int H_kv, int N_k, int off,
-                                     const int* __restrict__ seqlens) {
+                                     const int* __restrict__ seqlens, const float* __restrict__ row_scale) {
   __shared__ float sk[128];
   __shared__ float sv[128];
   __shared__ float sp[kThreads];
@@ -158,9 +160,10 @@ __global__ void bwd_dkdv_fp32_kernel(const float* __restrict__ q, const float* _
       if (i < iend) {
         const float s = dot_row(sk, q + base + static_cast<size_t>(i) * D, D);
         const float x = fmaf(scale, s, bias) - slope * fabsf(static_cast<float>(i + off - j));
-        p = sigmoid_exact(x);
+        const float r = row_scale ? row_scale[i] : 1.0f;   // O = r (P V): both products see r dO
+        p = r * sigmoid_exact(x);
         const float dp = dot_row(sv, d_o + base + static_cast<size_t>(i) * D, D);
-        ds = sigmoid_slope(x) * dp;
+        ds = r * sigmoid_slope(x) * dp;
       }
       sp[t] = p;
       sds[t] = ds;
@@ -182,13 +185,31 @@ __global__ void bwd_dkdv_fp32_kernel(const float* __restrict__ q, const float* _
   }
 }
 
+// Row factors of the sequence-length normalisation: n_k^-alpha without a mask, else
+// (pos + 1)^-alpha with pos = i + pos0 the query's position (0 for a row that keeps no key).
+__global__ void seqlen_norm_kernel(float* __restrict__ out, int N, int N_k, int pos0, int causal, float alpha) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= N) return;
+  const float count = causal ? static_cast<float>(i + pos0 + 1) : static_cast<float>(N_k);
+  out[i] = count >= 1.0f ? powf(count, -alpha) : 0.0f;
+}
+
 }  // namespace
+
+int launch_seqlen_norm(float* out, int N, int N_k, int pos0, int causal, float alpha, cudaStream_t stream,
+                       unsigned long long* launches, cudaError_t* cuda_err) {
+  seqlen_norm_kernel<<<(N + 255) / 256, 256, 0, stream>>>(out, N, N_k, pos0, causal, alpha);
+  *launches += 1;
+  *cuda_err = cudaGetLastError();
+  return *cuda_err == cudaSuccess ? SIGATTN_OK : SIGATTN_ERR_CUDA;
+}
 
 int launch_fwd_fp32(const float* q, const float* k, const float* v, float* o, const Problem& p,
                     cudaStream_t stream, unsigned long long* launches, cudaError_t* cuda_err) {
   dim3 grid(p.N, p.B * p.H);
   fwd_fp32_kernel<<<grid, kThreads, 0, stream>>>(q, k, v, o, p.H, p.N, p.D, p.scale, p.bias, p.causal, p.slopes,
-                                                 p.bias_vec, p.kv_heads(), p.key_rows(), p.query_pos0(), p.seqlens);
+                                                 p.bias_vec, p.kv_heads(), p.key_rows(), p.query_pos0(), p.seqlens,
+                                                 p.row_scale);
   *launches += 1;
   *cuda_err = cudaGetLastError();
   return *cuda_err == cudaSuccess ? SIGATTN_OK : SIGATTN_ERR_CUDA;
@@ -204,11 +225,11 @@ int launch_bwd_fp32(const float* q, const float* k, const float* v, const float*
   }
   bwd_dq_fp32_kernel<<<grid, kThreads, 0, stream>>>(q, k, v, d_o, dq, p.H, p.N, p.D, p.scale, p.bias, p.causal,
                                                     p.slopes, p.bias_vec, p.dbias, p.kv_heads(), p.key_rows(), p.query_pos0(),
-                                                    p.seqlens);
+                                                    p.seqlens, p.row_scale);
   dim3 grid_kv(p.key_rows(), p.B * p.kv_heads());
   bwd_dkdv_fp32_kernel<<<grid_kv, kThreads, 0, stream>>>(q, k, v, d_o, dk, dv, p.H, p.N, p.D, p.scale, p.bias,
                                                          p.causal, p.slopes, p.bias_vec, p.kv_heads(), p.key_rows(),
-                                                         p.query_pos0(), p.seqlens);
+                                                         p.query_pos0(), p.seqlens, p.row_scale);
   *launches += 2;
   *cuda_err = cudaGetLastError();
   return *cuda_err == cudaSuccess ? SIGATTN_OK : SIGATTN_ERR_CUDA;

@@ -93,6 +93,7 @@ struct FwdParams {
   // pack_group * pack_rows and H = H_kv, group = 1 for the producer.  0 = not packed.
   int pack_rows, pack_group;
   const int* seqlens;   // padded batch: valid length per batch entry (keys and queries), or nullptr
+  const float* row_scale;   // one factor per query row applied to O, or nullptr
   int n_pairs;     // ceil(N / 256)
   int n_kv_total;  // ceil(N / 128)
   int n_items;
@@ -351,12 +352,14 @@ __device__ __forceinline__ void sigmoid_cols(const uint32_t (&s)[kCols], uint32_
 // of the tile.  While the groups evaluate one tile, the tensor pipe runs
 // P V and the next logits of the other one, so the MUFU pipe and the tensor pipe take turns
 // on a tile instead of competing for it.
-// MODE: 0 plain (the benchmarked path), 1 packed grouped heads, 2 padded batch with per-sequence lengths
+// MODE: 0 plain (the benchmarked path), 1 packed grouped heads, 2 general: padded batch with
+// per-sequence lengths and / or one output factor per query row, each asked for at run time
 template <int D, bool CAUSAL, bool ALIBI, int MODE>
 __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t* smem, uint32_t tmem,
                              FwdBarriers* bars, volatile int* cta_err) {
   using L = FwdSmem<D>;
-  constexpr bool PACKED = (MODE == 1), VARLEN = (MODE == 2);
+  constexpr bool PACKED = (MODE == 1), GENERAL = (MODE == 2);
+  const bool varlen = GENERAL && p.seqlens != nullptr;
   const int g = threadIdx.x >> 7;            // column group of the tile
   const int tid = threadIdx.x & 127;         // row of the tile
   const uint32_t lane_off = static_cast<uint32_t>(((threadIdx.x >> 5) & 3) * 32) << 16;
@@ -401,7 +404,7 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
         // (packed rows: a tile may hold a head's first query, at position pos0)
         bool diag = CAUSAL && ((j + 1) * kBN - 1 > (PACKED ? 0 : w.row0 + t * kBM) + p.pos0);
         float mask_limit = row_rel;   // last key (relative to the tile's first) that keeps its weight
-        if (VARLEN) {
+        if (varlen) {
           // padded batch: keys past the end of the sequence are masked, rows past it are masked whole
           const float key_limit = static_cast<float>(w.n_valid - 1 - j * kBN);
           mask_limit = CAUSAL ? fminf(row_rel, key_limit) : key_limit;
@@ -440,6 +443,13 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
       uint32_t o[kECols];
       tmem_ld_cols(tO, o);
       tmem_wait_ld();
+      if (GENERAL && p.row_scale != nullptr) {
+        // sequence-length normalisation: one factor per query row (rows past the end are not stored)
+        const int row = w.row0 + t * kBM + tid;
+        const float r = row < p.N ? __ldg(p.row_scale + row) : 0.0f;
+#pragma unroll
+        for (int e = 0; e < kECols; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * r);
+      }
       {
         const int col = g * kECols;           // first of this thread's columns
         uint8_t* row_ptr = stage + (col >> 6) * L::kPanelBytes + tid * 128;
@@ -569,7 +579,8 @@ int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const 
   const int group = p.H / p.kv_heads();
   // Few queries per head and several query heads per key/value head (decoding with grouped
   // heads): pack the group's rows into one sequence so that K and V are streamed once per group.
-  const bool packed = group > 1 && static_cast<long long>(p.N) * group <= 2 * kBM && p.seqlens == nullptr;
+  const bool packed = group > 1 && static_cast<long long>(p.N) * group <= 2 * kBM && p.seqlens == nullptr &&
+                      p.row_scale == nullptr;
   const uint64_t q_heads = packed ? BH_kv : BH;
   const uint64_t q_rows = packed ? static_cast<uint64_t>(p.N) * group : p.N;
   CUtensorMap tmQ, tmK, tmV, tmO;
@@ -600,13 +611,14 @@ int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const 
   fp.bias_vec = p.bias_vec;
   fp.slopes = p.slopes;
   fp.seqlens = p.seqlens;
+  fp.row_scale = p.row_scale;
   fp.status = status;
 
   int rc;
   const bool alibi = p.slopes != nullptr;
 #define SIGATTN_FWD_CASE(DD, CC, AA)                                                                       \
   rc = packed ? launch_fwd_variant<DD, CC, AA, 1>(tmQ, tmK, tmV, tmO, fp, num_sms, stream, cuda_err)       \
-       : (p.seqlens != nullptr)                                                                            \
+       : (p.seqlens != nullptr || p.row_scale != nullptr)                                                  \
            ? launch_fwd_variant<DD, CC, AA, 2>(tmQ, tmK, tmV, tmO, fp, num_sms, stream, cuda_err)          \
            : launch_fwd_variant<DD, CC, AA, 0>(tmQ, tmK, tmV, tmO, fp, num_sms, stream, cuda_err)
   if (p.D == 128) {

@@ -22,6 +22,7 @@ struct Problem {
   int pos0;               //    0: the queries are the last N positions, pos0 = key_rows() - N
   int query_pos0() const { return pos0_given ? pos0 : key_rows() - N; }
   const int* seqlens;     // device pointer to B valid lengths (padded batch, N_k = N only), or nullptr
+  const float* row_scale; // device pointer to N factors, one per query row, applied to O, or nullptr
 };
 
 // Every launcher enqueues on `stream`, adds the number of kernels it launched to
@@ -42,6 +43,9 @@ int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const 
 int launch_bwd_bf16(const void* q, const void* k, const void* v, const void* d_o, void* dq, void* dk, void* dv,
                     const Problem& p, void* workspace, int* status, cudaStream_t stream,
                     unsigned long long* launches, cudaError_t* cuda_err);
+
+int launch_seqlen_norm(float* out, int N, int N_k, int pos0, int causal, float alpha, cudaStream_t stream,
+                       unsigned long long* launches, cudaError_t* cuda_err);
 
 size_t bwd_bf16_workspace_bytes(int B, int H, int N, int D);
 
