@@ -277,6 +277,28 @@ SIGATTN_API int sigattn_bwd_rowscale(const void* q, const void* k, const void* v
  * `stream`.  causal = 1 needs N_k >= N_q. */
 SIGATTN_API int sigattn_seqlen_norm(float* row_scale, int N_q, int N_k, float alpha, int causal, void* stream);
 
+/* Forward for generation with a cache of keys and values (where the paper measures its
+ * inference gains, Appendix F.3): the same operation, arguments and result as sigattn_fwd_nk,
+ * plus a scratch buffer that lets the library split the keys of one head over several thread
+ * blocks when B * H_kv alone cannot fill the GPU.  Sigmoid attention has no row normalisation
+ * (Section 4), so the partial outputs of the splits are plain fp32 sums - no running maximum, no
+ * log-sum-exp to merge; they are added with fp32 atomics (the last bits of O may differ from run
+ * to run) and converted to bf16 by a second small kernel.  The split is used when the queries of
+ * a key/value head fit one pair of tiles (N_q * H / H_kv <= 256) and it shortens the run; otherwise
+ * the call is sigattn_fwd_nk and leaves the workspace untouched.
+ * workspace: DEVICE scratch of at least sigattn_fwd_decode_workspace_bytes(...) bytes, 256-byte
+ * aligned, owned by the caller; two calls that share it must not overlap on the device.  Errors
+ * as sigattn_fwd_nk, plus SIGATTN_ERR_WORKSPACE. */
+SIGATTN_API int sigattn_fwd_decode(const void* q, const void* k, const void* v, void* o,
+                       int B, int H, int H_kv, int N_q, int N_k, int D,
+                       float scale, float bias, const float* bias_bh, int causal,
+                       const float* alibi_slopes, int dtype,
+                       void* workspace, size_t workspace_bytes, void* stream);
+
+/* Bytes of scratch sigattn_fwd_decode needs: B * H * N_q * D floats (0 for the fp32 debug path
+ * and for invalid shapes). */
+SIGATTN_API size_t sigattn_fwd_decode_workspace_bytes(int B, int H, int N_q, int D, int dtype);
+
 /* Bytes of scratch sigattn_bwd needs for this problem (0 for the fp32 debug path).
  * Returns 0 for invalid shapes as well; sigattn_bwd reports those. */
 SIGATTN_API size_t sigattn_bwd_workspace_bytes(int B, int H, int N, int D, int dtype);

@@ -38,6 +38,8 @@ _BINDING_NAMES = (
     "sigattn_fwd_rowscale",
     "sigattn_bwd_rowscale",
     "sigattn_seqlen_norm",
+    "sigattn_fwd_decode",
+    "sigattn_fwd_decode_workspace_bytes",
     "lib",
 )
 

@@ -73,6 +73,12 @@ _lib.sigattn_bwd_rowscale.restype = _c.c_int
 _lib.sigattn_bwd_rowscale.argtypes = [_c.c_void_p] * 7 + [_c.c_int] * 6 + [_c.c_float, _c.c_float, _c.c_void_p, _c.c_int,
                                                                              _c.c_void_p, _c.c_void_p, _c.c_int, _c.c_void_p,
                                                                              _c.c_void_p, _c.c_size_t, _c.c_void_p]
+_lib.sigattn_fwd_decode.restype = _c.c_int
+_lib.sigattn_fwd_decode.argtypes = [_c.c_void_p] * 4 + [_c.c_int] * 6 + [_c.c_float, _c.c_float, _c.c_void_p, _c.c_int,
+                                                                           _c.c_void_p, _c.c_int, _c.c_void_p, _c.c_size_t,
+                                                                           _c.c_void_p]
+_lib.sigattn_fwd_decode_workspace_bytes.restype = _c.c_size_t
+_lib.sigattn_fwd_decode_workspace_bytes.argtypes = [_c.c_int] * 5
 _lib.sigattn_seqlen_norm.restype = _c.c_int
 _lib.sigattn_seqlen_norm.argtypes = [_c.c_void_p, _c.c_int, _c.c_int, _c.c_float, _c.c_int, _c.c_void_p]
 _lib.sigattn_bwd_workspace_bytes.restype = _c.c_size_t
@@ -112,6 +118,7 @@ EXPORTED = [
     "sigattn_fwd_gqa", "sigattn_bwd_gqa", "sigattn_fwd_nk", "sigattn_bwd_nk",
     "sigattn_fwd_shard", "sigattn_bwd_shard", "sigattn_fwd_varlen", "sigattn_bwd_varlen",
     "sigattn_fwd_rowscale", "sigattn_bwd_rowscale", "sigattn_seqlen_norm",
+    "sigattn_fwd_decode", "sigattn_fwd_decode_workspace_bytes",
 ]
 
 
@@ -515,6 +522,36 @@ def sigattn_bwd_varlen(q, k, v, d_o, scale, bias, seqlens, causal=False, alibi_s
     if rc != 0:
         raise SigattnError(rc)
     return dq, dk, dv, dbias
+
+
+def sigattn_fwd_decode_workspace_bytes(B, H, N_q, D, dtype_code) -> int:
+    return int(_lib.sigattn_fwd_decode_workspace_bytes(B, H, N_q, D, dtype_code))
+
+
+def sigattn_fwd_decode(q, k, v, scale, bias, causal=False, alibi_slopes=None, workspace=None, out=None, stream=None):
+    """sigattn_fwd_nk with a scratch buffer that lets the keys of one head be split over several
+    thread blocks (generation with a cache: few queries, long key sequences)."""
+    import torch
+    B, H, H_kv, N_q, N_k, D = _check_nk(q, k, v)
+    if out is None:
+        out = torch.empty_like(q)
+    else:
+        _check_same([q, out], ["q", "out"])
+    vec = isinstance(bias, torch.Tensor)
+    if vec:
+        _check_bias_vec(bias, q)
+    code = _dtype_code(q)
+    need = sigattn_fwd_decode_workspace_bytes(B, H, N_q, D, code)
+    if workspace is None and need > 0:
+        workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    with torch.cuda.device(q.device):
+        rc = _lib.sigattn_fwd_decode(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, H, H_kv, N_q, N_k, D, float(scale),
+                                     0.0 if vec else float(bias), _ptr(bias) if vec else None, int(bool(causal)),
+                                     _ptr(alibi_slopes), code, _ptr(workspace), ws_bytes, _stream_ptr(stream))
+    if rc != 0:
+        raise SigattnError(rc)
+    return out
 
 
 def _check_row_scale(row_scale, q):

@@ -103,7 +103,7 @@ int check_lengths(int B, int H, int H_kv, int N, int N_k, int D, int causal, int
 int fwd_any(const void* q, const void* k, const void* v, void* o, int B, int H, int H_kv, int N, int N_k, int D,
             float scale, float bias, const float* bias_vec, int causal, const float* alibi_slopes, int dtype,
             void* stream, int pos0_given = 0, int pos0 = 0, const int* seqlens = nullptr,
-            const float* row_scale = nullptr) {
+            const float* row_scale = nullptr, float* split_ws = nullptr) {
   if (!q || !k || !v || !o) return SIGATTN_ERR_NULL;
   if (int rc = check_lengths(B, H, H_kv, N, N_k, D, causal, pos0_given, pos0)) return rc;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return SIGATTN_ERR_ALIGN;
@@ -114,7 +114,7 @@ int fwd_any(const void* q, const void* k, const void* v, void* o, int B, int H, 
   int* status = nullptr;
   if (int rc = device_setup(&dev, &status)) return rc;
   sigattn::Problem p{B, H, N, D, scale, bias, causal, alibi_slopes, bias_vec, nullptr, H_kv, N_k, pos0_given, pos0,
-                     seqlens, row_scale};
+                     seqlens, row_scale, split_ws};
   unsigned long long launches = 0;
   cudaError_t ce = cudaSuccess;
   int rc;
@@ -516,6 +516,26 @@ int sigattn_bwd_rowscale(const void* q, const void* k, const void* v, const void
     return SIGATTN_ERR_ALIGN;
   return bwd_any(q, k, v, d_o, dq, dk, dv, B, H, H_kv, N_q, N_k, D, scale, bias, bias_bh, dbias_bh, causal,
                  alibi_slopes, dtype, workspace, workspace_bytes, stream, 0, 0, nullptr, row_scale);
+}
+
+size_t sigattn_fwd_decode_workspace_bytes(int B, int H, int N_q, int D, int dtype) {
+  if (check_shape(B, H, N_q, D) != SIGATTN_OK) return 0;
+  if (dtype != SIGATTN_DTYPE_BF16) return 0;
+  return static_cast<size_t>(B) * H * N_q * D * sizeof(float);
+}
+
+int sigattn_fwd_decode(const void* q, const void* k, const void* v, void* o, int B, int H, int H_kv, int N_q, int N_k,
+                       int D, float scale, float bias, const float* bias_bh, int causal, const float* alibi_slopes,
+                       int dtype, void* workspace, size_t workspace_bytes, void* stream) {
+  if (reinterpret_cast<uintptr_t>(bias_bh) & 3u) return SIGATTN_ERR_ALIGN;
+  const size_t need = sigattn_fwd_decode_workspace_bytes(B, H, N_q, D, dtype);
+  if (need > 0) {
+    if (!workspace) return SIGATTN_ERR_NULL;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255u) return SIGATTN_ERR_ALIGN;
+    if (workspace_bytes < need) return SIGATTN_ERR_WORKSPACE;
+  }
+  return fwd_any(q, k, v, o, B, H, H_kv, N_q, N_k, D, scale, bias, bias_bh, causal, alibi_slopes, dtype, stream, 0, 0,
+                 nullptr, nullptr, need > 0 ? static_cast<float*>(workspace) : nullptr);
 }
 
 int sigattn_seqlen_norm(float* row_scale, int N_q, int N_k, float alpha, int causal, void* stream) {

@@ -96,6 +96,12 @@ struct FwdParams {
   const float* row_scale;   // one factor per query row applied to O, or nullptr
   int n_pairs;     // ceil(N / 256)
   int n_kv_total;  // ceil(N / 128)
+  // Keys split over several work items (packed mode only; decoding has too few (batch, head)
+  // pairs to fill the GPU): split s of a (head, pair) visits key tiles [s, s + 1) * tiles_per_split
+  // and adds its partial O, in fp32, into split_ws [BH, N, D]; there is no row normalisation, so
+  // the partial results simply add up.  n_splits = 1: off.
+  int n_splits, tiles_per_split;
+  float* split_ws;
   int n_items;
   float scale_log2e, bias_log2e;
   const float* bias_vec;   // one bias per (batch, head) instead of the scalar, or nullptr
@@ -105,6 +111,7 @@ struct FwdParams {
 
 struct Item {
   int bh, row0, n_kv, n[2];
+  int j0;        // first key tile of the item (0 unless the keys are split)
   int n_valid;   // rows of this sequence that count (N unless the batch is padded)
 };
 
@@ -124,8 +131,10 @@ __device__ __forceinline__ int num_rounds(int n_items) { return (n_items + gridD
 template <bool CAUSAL>
 __device__ __forceinline__ Item decode_item(const FwdParams& p, int item) {
   Item w;
-  const int rank = item / p.BH;
+  int rank = item / p.BH;
   w.bh = item - rank * p.BH;
+  const int split = rank / p.n_pairs;   // 0 unless the keys are split
+  rank -= split * p.n_pairs;
   const int pair = CAUSAL ? (p.n_pairs - 1 - rank) : rank;
   w.row0 = pair * 2 * kBM;
   w.n_valid = p.seqlens ? max(0, min(p.N, __ldg(p.seqlens + w.bh / p.H))) : p.N;
@@ -142,6 +151,13 @@ __device__ __forceinline__ Item decode_item(const FwdParams& p, int item) {
                     : n_kv_valid);
     // (a tile of a padded batch that lies past the sequence's end visits one key tile, fully masked)
     if (p.seqlens && r < p.N && r >= w.n_valid) w.n[t] = 1;
+  }
+  w.j0 = 0;
+  if (p.n_splits > 1) {   // packed mode: every valid tile visits all key tiles; this item takes its share
+    w.j0 = split * p.tiles_per_split;
+    const int n = min(p.tiles_per_split, p.n_kv_total - w.j0);
+#pragma unroll
+    for (int t = 0; t < 2; ++t) w.n[t] = w.n[t] > 0 ? n : 0;
   }
   w.n_kv = max(w.n[0], w.n[1]);
   return w;
@@ -180,8 +196,8 @@ __device__ void fwd_load_role(const FwdParams& p, const CUtensorMap* tmQ, const 
       mbar_arrive_expect_tx(bar, L::kTileBytes);
 #pragma unroll
       for (int pn = 0; pn < L::kPanels; ++pn)
-        tma_load_3d(smem_base + L::kKvOff + stage * L::kTileBytes + pn * L::kPanelBytes, tm, bar, pn * 64, j * kBN,
-                    bh_kv);
+        tma_load_3d(smem_base + L::kKvOff + stage * L::kTileBytes + pn * L::kPanelBytes, tm, bar, pn * 64,
+                    (w.j0 + j) * kBN, bh_kv);
       ++kv_cnt;
       return true;
     };
@@ -397,12 +413,13 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
         if (!mbar_wait(smem_u32(&bars->s_full[t]), cnt & 1, cta_err, 30 + t)) return;
         ++cnt;
         tc_fence_after_sync();
+        const int jk = PACKED ? w.j0 + j : j;   // key tile within the sequence (the keys may be split)
         // position of this thread's query relative to the first key of the tile
-        const float row_rel = (PACKED ? pos_t[t] : pos_t[0] + static_cast<float>(t * kBM)) - static_cast<float>(j * kBN);
+        const float row_rel = (PACKED ? pos_t[t] : pos_t[0] + static_cast<float>(t * kBM)) - static_cast<float>(jk * kBN);
         // the mask cuts through every key tile that reaches beyond the position of the tile's
         // first row: the last one, and with pos0 not a multiple of 128 also the one before
         // (packed rows: a tile may hold a head's first query, at position pos0)
-        bool diag = CAUSAL && ((j + 1) * kBN - 1 > (PACKED ? 0 : w.row0 + t * kBM) + p.pos0);
+        bool diag = CAUSAL && ((jk + 1) * kBN - 1 > (PACKED ? 0 : w.row0 + t * kBM) + p.pos0);
         float mask_limit = row_rel;   // last key (relative to the tile's first) that keeps its weight
         if (varlen) {
           // padded batch: keys past the end of the sequence are masked, rows past it are masked whole
@@ -443,6 +460,20 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
       uint32_t o[kECols];
       tmem_ld_cols(tO, o);
       tmem_wait_ld();
+      if (PACKED && p.n_splits > 1) {
+        // split keys: add this item's partial rows into the fp32 buffer (few rows: plain atomics);
+        // a later pass converts the sums to bf16.  The Q buffer is not needed for staging.
+        const int row = w.row0 + t * kBM + tid;
+        if (row < p.N) {
+          float* dst = p.split_ws + (static_cast<size_t>(w.bh) * p.N + row) * D + g * kECols;
+#pragma unroll
+          for (int e = 0; e < kECols; ++e) atomicAdd(dst + e, __uint_as_float(o[e]));
+        }
+        tc_fence_before_sync();
+        mbar_arrive(smem_u32(&bars->o_empty[t]));
+        if (threadIdx.x == 0) mbar_arrive(smem_u32(&bars->q_empty[t]));   // all logits MMAs of the item are done
+        continue;
+      }
       if (GENERAL && p.row_scale != nullptr) {
         // sequence-length normalisation: one factor per query row (rows past the end are not stored)
         const int row = w.row0 + t * kBM + tid;
@@ -548,6 +579,33 @@ sigattn_fwd_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
   if (warp == kMmaWarp) tmem_dealloc(tmem, 512);
 }
 
+// O (bf16) = the fp32 sums of the key splits: the pass that follows a split forward.
+__global__ void __launch_bounds__(256)
+sigattn_fwd_convert_o_kernel(const float4* __restrict__ ws, uint2* __restrict__ o, size_t n_vec4) {
+  const size_t stride = static_cast<size_t>(gridDim.x) * blockDim.x;
+  for (size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < n_vec4; i += stride) {
+    const float4 v = ws[i];
+    o[i] = make_uint2(pack_bf16x2(v.x, v.y), pack_bf16x2(v.z, v.w));
+  }
+}
+
+// Number of key splits for a problem with `base_items` work items of `n_kv` key tiles each:
+// the count that minimises rounds of the persistent grid times tiles per item (plus about two
+// tiles' worth of per-item start-up and epilogue), each split keeping at least two key tiles.
+int choose_key_splits(int base_items, int n_kv, int num_sms) {
+  int best = 1;
+  long long best_cost = -1;
+  for (int s = 1; s <= 64 && 2 * s <= n_kv + 1; ++s) {
+    const int per = (n_kv + s - 1) / s;
+    const int used = (n_kv + per - 1) / per;   // splits that are not empty
+    if (used != s) continue;
+    const long long rounds = (static_cast<long long>(base_items) * s + num_sms - 1) / num_sms;
+    const long long cost = rounds * (per + 2);
+    if (best_cost < 0 || cost < best_cost) { best = s; best_cost = cost; }
+  }
+  return best;
+}
+
 template <int D, bool CAUSAL, bool ALIBI, int MODE>
 int launch_fwd_variant(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtensorMap& tmO,
                        const FwdParams& fp, int num_sms, cudaStream_t stream, cudaError_t* cuda_err) {
@@ -579,8 +637,12 @@ int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const 
   const int group = p.H / p.kv_heads();
   // Few queries per head and several query heads per key/value head (decoding with grouped
   // heads): pack the group's rows into one sequence so that K and V are streamed once per group.
-  const bool packed = group > 1 && static_cast<long long>(p.N) * group <= 2 * kBM && p.seqlens == nullptr &&
-                      p.row_scale == nullptr;
+  const bool small = static_cast<long long>(p.N) * group <= 2 * kBM && p.seqlens == nullptr && p.row_scale == nullptr;
+  // With a scratch buffer for fp32 partial sums, the keys of one head may also be split over
+  // several work items (decoding: too few (batch, head) pairs for 148 SMs otherwise).
+  const int n_kv_tiles = (p.key_rows() + kBN - 1) / kBN;
+  const int n_splits = (small && p.split_ws != nullptr) ? choose_key_splits(static_cast<int>(BH_kv), n_kv_tiles, num_sms) : 1;
+  const bool packed = small && (group > 1 || n_splits > 1);
   const uint64_t q_heads = packed ? BH_kv : BH;
   const uint64_t q_rows = packed ? static_cast<uint64_t>(p.N) * group : p.N;
   CUtensorMap tmQ, tmK, tmV, tmO;
@@ -605,7 +667,10 @@ int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const 
   fp.pos0 = p.query_pos0();
   fp.n_pairs = (fp.N + 2 * kBM - 1) / (2 * kBM);
   fp.n_kv_total = (p.key_rows() + kBN - 1) / kBN;
-  fp.n_items = fp.n_pairs * fp.BH;
+  fp.n_splits = n_splits;
+  fp.tiles_per_split = (fp.n_kv_total + n_splits - 1) / n_splits;
+  fp.split_ws = p.split_ws;
+  fp.n_items = fp.n_pairs * fp.BH * n_splits;
   fp.scale_log2e = p.scale * kLog2e;
   fp.bias_log2e = p.bias * kLog2e;
   fp.bias_vec = p.bias_vec;
@@ -613,6 +678,12 @@ int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const 
   fp.seqlens = p.seqlens;
   fp.row_scale = p.row_scale;
   fp.status = status;
+
+  const size_t n_elems = static_cast<size_t>(BH) * p.N * p.D;
+  if (n_splits > 1) {
+    *cuda_err = cudaMemsetAsync(p.split_ws, 0, n_elems * sizeof(float), stream);
+    if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
+  }
 
   int rc;
   const bool alibi = p.slopes != nullptr;
@@ -629,8 +700,18 @@ int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const 
     else          { if (alibi) SIGATTN_FWD_CASE(64, false, true); else SIGATTN_FWD_CASE(64, false, false); }
   }
 #undef SIGATTN_FWD_CASE
-  if (rc == SIGATTN_OK) *launches += 1;
-  return rc;
+  if (rc != SIGATTN_OK) return rc;
+  *launches += 1;
+  if (n_splits > 1) {
+    const size_t n_vec4 = n_elems / 4;
+    const size_t want = n_vec4 / 256 + 1, cap = static_cast<size_t>(num_sms) * 8;
+    sigattn_fwd_convert_o_kernel<<<static_cast<int>(want < cap ? want : cap), 256, 0, stream>>>(
+        static_cast<const float4*>(static_cast<const void*>(p.split_ws)), static_cast<uint2*>(o), n_vec4);
+    *cuda_err = cudaGetLastError();
+    if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
+    *launches += 1;
+  }
+  return SIGATTN_OK;
 }
 
 }  // namespace sigattn

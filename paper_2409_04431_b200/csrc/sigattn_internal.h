@@ -23,6 +23,8 @@ struct Problem {
   int query_pos0() const { return pos0_given ? pos0 : key_rows() - N; }
   const int* seqlens;     // device pointer to B valid lengths (padded batch, N_k = N only), or nullptr
   const float* row_scale; // device pointer to N factors, one per query row, applied to O, or nullptr
+  float* split_ws;        // forward only: device scratch of B*H*N*D floats that allows splitting the keys of a
+                          // head over several thread blocks when there are few queries (decoding), or nullptr
 };
 
 // Every launcher enqueues on `stream`, adds the number of kernels it launched to
