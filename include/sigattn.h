@@ -218,6 +218,39 @@ SIGATTN_API int sigattn_bwd_shard(const void* q, const void* k, const void* v, c
                       float* dbias_bh,
                       void* workspace, size_t workspace_bytes, void* stream);
 
+/* The same shard calls with the sum fused into the kernels: instead of writing its summand the
+ * call ADDS it, in fp32, into an accumulator that the caller owns, so that shards running on
+ * different GPUs can add straight into the memory of the GPU that owns the query rows (a peer
+ * mapping of its accumulator) and no separate all-reduce or reduce-scatter pass is needed.
+ * bf16 only (dtype 1 returns SIGATTN_ERR_FLAG).
+ *
+ * sigattn_fwd_shard_acc: o_acc, DEVICE pointer to B*H*N_q*D floats [B, H, N_q, D], 16-byte
+ *   aligned, receives += P V of this shard; the forward's epilogue issues vector reductions
+ *   (red.global.add) per row, nothing else touches it.  No O is written.
+ * sigattn_bwd_shard_acc: dq_acc, DEVICE pointer to B*H*N_q*D floats, 256-byte aligned, receives
+ *   += dS K of this shard WITHOUT the factor `scale` (TMA reduce-add tiles, as in sigattn_bwd);
+ *   dk, dv of the shard are written as in sigattn_bwd_shard; no dq is written.
+ * The accumulators must be zero before the first shard adds (the caller clears them) and all
+ * shards must have finished (stream or cross-GPU synchronisation, the caller's) before
+ * sigattn_acc_to_bf16 turns them into the result: out = bf16(mul * acc), mul = 1 for O and
+ * `scale` for dQ; n = number of elements, a multiple of 4; acc and out 16-byte aligned.
+ * Accumulators in another GPU's memory are reached with plain reductions and TMA reduce
+ * operations only (no multicast load is ever issued on them).  The order of the additions is
+ * not fixed, so the last bits of the sums may differ from run to run. */
+SIGATTN_API int sigattn_fwd_shard_acc(const void* q, const void* k, const void* v, float* o_acc,
+                          int B, int H, int H_kv, int N_q, int N_k, int D,
+                          float scale, float bias, const float* bias_bh, int causal, int pos0,
+                          const float* alibi_slopes, int dtype, void* stream);
+
+SIGATTN_API int sigattn_bwd_shard_acc(const void* q, const void* k, const void* v, const void* d_o,
+                          float* dq_acc, void* dk, void* dv,
+                          int B, int H, int H_kv, int N_q, int N_k, int D,
+                          float scale, float bias, const float* bias_bh, int causal, int pos0,
+                          const float* alibi_slopes, int dtype,
+                          float* dbias_bh, void* stream);
+
+SIGATTN_API int sigattn_acc_to_bf16(const float* acc, void* out, size_t n, float mul, void* stream);
+
 /* Padded batches of sequences of different lengths (the speech batches of Section 5.4, with
  * b = -log n_b per sample through `bias_bh`): `seqlens` is a DEVICE pointer to B int32, 4-byte
  * aligned, read while the kernels run; entry b is the number n_b of rows of batch entry b that

@@ -39,6 +39,9 @@ _BINDING_NAMES = (
     "sigattn_bwd_rowscale",
     "sigattn_seqlen_norm",
     "sigattn_fwd_decode",
+    "sigattn_fwd_shard_acc",
+    "sigattn_bwd_shard_acc",
+    "sigattn_acc_to_bf16",
     "sigattn_fwd_decode_workspace_bytes",
     "lib",
 )

@@ -73,6 +73,16 @@ _lib.sigattn_bwd_rowscale.restype = _c.c_int
 _lib.sigattn_bwd_rowscale.argtypes = [_c.c_void_p] * 7 + [_c.c_int] * 6 + [_c.c_float, _c.c_float, _c.c_void_p, _c.c_int,
                                                                              _c.c_void_p, _c.c_void_p, _c.c_int, _c.c_void_p,
                                                                              _c.c_void_p, _c.c_size_t, _c.c_void_p]
+_lib.sigattn_fwd_shard_acc.restype = _c.c_int
+_lib.sigattn_fwd_shard_acc.argtypes = [_c.c_void_p] * 4 + [_c.c_int] * 6 + [_c.c_float, _c.c_float, _c.c_void_p,
+                                                                              _c.c_int, _c.c_int, _c.c_void_p, _c.c_int,
+                                                                              _c.c_void_p]
+_lib.sigattn_bwd_shard_acc.restype = _c.c_int
+_lib.sigattn_bwd_shard_acc.argtypes = [_c.c_void_p] * 7 + [_c.c_int] * 6 + [_c.c_float, _c.c_float, _c.c_void_p,
+                                                                              _c.c_int, _c.c_int, _c.c_void_p, _c.c_int,
+                                                                              _c.c_void_p, _c.c_void_p]
+_lib.sigattn_acc_to_bf16.restype = _c.c_int
+_lib.sigattn_acc_to_bf16.argtypes = [_c.c_void_p, _c.c_void_p, _c.c_size_t, _c.c_float, _c.c_void_p]
 _lib.sigattn_fwd_decode.restype = _c.c_int
 _lib.sigattn_fwd_decode.argtypes = [_c.c_void_p] * 4 + [_c.c_int] * 6 + [_c.c_float, _c.c_float, _c.c_void_p, _c.c_int,
                                                                            _c.c_void_p, _c.c_int, _c.c_void_p, _c.c_size_t,
@@ -119,6 +129,7 @@ EXPORTED = [
     "sigattn_fwd_shard", "sigattn_bwd_shard", "sigattn_fwd_varlen", "sigattn_bwd_varlen",
     "sigattn_fwd_rowscale", "sigattn_bwd_rowscale", "sigattn_seqlen_norm",
     "sigattn_fwd_decode", "sigattn_fwd_decode_workspace_bytes",
+    "sigattn_fwd_shard_acc", "sigattn_bwd_shard_acc", "sigattn_acc_to_bf16",
 ]
 
 
@@ -522,6 +533,64 @@ def sigattn_bwd_varlen(q, k, v, d_o, scale, bias, seqlens, causal=False, alibi_s
     if rc != 0:
         raise SigattnError(rc)
     return dq, dk, dv, dbias
+
+
+def sigattn_fwd_shard_acc(q, k, v, o_acc, scale, bias, pos0, causal=False, alibi_slopes=None, stream=None):
+    """Adds this key/value shard's summand of O, in fp32, into `o_acc`: a float32 CUDA tensor shaped
+    like q, or an integer device address (e.g. a peer mapping of another GPU's accumulator)."""
+    import torch
+    B, H, H_kv, N_q, N_k, D = _check_nk(q, k, v)
+    if isinstance(o_acc, torch.Tensor) and (o_acc.dtype != torch.float32 or o_acc.shape != q.shape
+                                            or not o_acc.is_contiguous() or not o_acc.is_cuda):
+        raise ValueError("o_acc must be a contiguous float32 CUDA tensor shaped like q")
+    vec = isinstance(bias, torch.Tensor)
+    if vec:
+        _check_bias_vec(bias, q)
+    with torch.cuda.device(q.device):
+        rc = _lib.sigattn_fwd_shard_acc(_ptr(q), _ptr(k), _ptr(v), _ptr(o_acc), B, H, H_kv, N_q, N_k, D, float(scale),
+                                        0.0 if vec else float(bias), _ptr(bias) if vec else None, int(bool(causal)),
+                                        int(pos0), _ptr(alibi_slopes), _dtype_code(q), _stream_ptr(stream))
+    if rc != 0:
+        raise SigattnError(rc)
+
+
+def sigattn_bwd_shard_acc(q, k, v, d_o, dq_acc, scale, bias, pos0, causal=False, alibi_slopes=None, want_dbias=False,
+                          stream=None):
+    """Adds this shard's summand of dQ (without the factor `scale`) into `dq_acc` (float32 CUDA tensor
+    shaped like q, or an integer device address) and returns (dK, dV, dbias or None) of the shard."""
+    import torch
+    B, H, H_kv, N_q, N_k, D = _check_nk(q, k, v)
+    _check_same([q, d_o], ["q", "d_o"])
+    if isinstance(dq_acc, torch.Tensor) and (dq_acc.dtype != torch.float32 or dq_acc.shape != q.shape
+                                             or not dq_acc.is_contiguous() or not dq_acc.is_cuda):
+        raise ValueError("dq_acc must be a contiguous float32 CUDA tensor shaped like q")
+    vec = isinstance(bias, torch.Tensor)
+    if vec:
+        _check_bias_vec(bias, q)
+    dk, dv = torch.empty_like(k), torch.empty_like(v)
+    dbias = torch.empty((B, H), dtype=torch.float32, device=q.device) if want_dbias else None
+    with torch.cuda.device(q.device):
+        rc = _lib.sigattn_bwd_shard_acc(_ptr(q), _ptr(k), _ptr(v), _ptr(d_o), _ptr(dq_acc), _ptr(dk), _ptr(dv), B, H,
+                                        H_kv, N_q, N_k, D, float(scale), 0.0 if vec else float(bias),
+                                        _ptr(bias) if vec else None, int(bool(causal)), int(pos0), _ptr(alibi_slopes),
+                                        _dtype_code(q), _ptr(dbias), _stream_ptr(stream))
+    if rc != 0:
+        raise SigattnError(rc)
+    return dk, dv, dbias
+
+
+def sigattn_acc_to_bf16(acc, mul=1.0, out=None, stream=None):
+    """bf16(mul * acc) for a float32 accumulator filled by the *_shard_acc calls."""
+    import torch
+    if not isinstance(acc, torch.Tensor) or acc.dtype != torch.float32 or not acc.is_cuda or not acc.is_contiguous():
+        raise ValueError("acc must be a contiguous float32 CUDA tensor")
+    if out is None:
+        out = torch.empty(acc.shape, dtype=torch.bfloat16, device=acc.device)
+    with torch.cuda.device(acc.device):
+        rc = _lib.sigattn_acc_to_bf16(_ptr(acc), _ptr(out), acc.numel(), float(mul), _stream_ptr(stream))
+    if rc != 0:
+        raise SigattnError(rc)
+    return out
 
 
 def sigattn_fwd_decode_workspace_bytes(B, H, N_q, D, dtype_code) -> int:

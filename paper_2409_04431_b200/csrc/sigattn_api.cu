@@ -103,18 +103,19 @@ int check_lengths(int B, int H, int H_kv, int N, int N_k, int D, int causal, int
 int fwd_any(const void* q, const void* k, const void* v, void* o, int B, int H, int H_kv, int N, int N_k, int D,
             float scale, float bias, const float* bias_vec, int causal, const float* alibi_slopes, int dtype,
             void* stream, int pos0_given = 0, int pos0 = 0, const int* seqlens = nullptr,
-            const float* row_scale = nullptr, float* split_ws = nullptr) {
-  if (!q || !k || !v || !o) return SIGATTN_ERR_NULL;
+            const float* row_scale = nullptr, float* split_ws = nullptr, int acc_only = 0) {
+  if (!q || !k || !v || (!o && !acc_only)) return SIGATTN_ERR_NULL;
   if (int rc = check_lengths(B, H, H_kv, N, N_k, D, causal, pos0_given, pos0)) return rc;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return SIGATTN_ERR_ALIGN;
   if (alibi_slopes && (reinterpret_cast<uintptr_t>(alibi_slopes) & 3u)) return SIGATTN_ERR_ALIGN;
   if (dtype != SIGATTN_DTYPE_BF16 && dtype != SIGATTN_DTYPE_FP32) return SIGATTN_ERR_FLAG;
+  if (acc_only && dtype != SIGATTN_DTYPE_BF16) return SIGATTN_ERR_FLAG;
   if (causal != 0 && causal != 1) return SIGATTN_ERR_FLAG;
   int dev = 0;
   int* status = nullptr;
   if (int rc = device_setup(&dev, &status)) return rc;
   sigattn::Problem p{B, H, N, D, scale, bias, causal, alibi_slopes, bias_vec, nullptr, H_kv, N_k, pos0_given, pos0,
-                     seqlens, row_scale, split_ws};
+                     seqlens, row_scale, split_ws, acc_only};
   unsigned long long launches = 0;
   cudaError_t ce = cudaSuccess;
   int rc;
@@ -133,8 +134,10 @@ int fwd_any(const void* q, const void* k, const void* v, void* o, int B, int H, 
 int bwd_any(const void* q, const void* k, const void* v, const void* d_o, void* dq, void* dk, void* dv, int B, int H,
             int H_kv, int N, int N_k, int D, float scale, float bias, const float* bias_vec, float* dbias, int causal,
             const float* alibi_slopes, int dtype, void* workspace, size_t workspace_bytes, void* stream,
-            int pos0_given = 0, int pos0 = 0, const int* seqlens = nullptr, const float* row_scale = nullptr) {
-  if (!q || !k || !v || !d_o || !dq || !dk || !dv) return SIGATTN_ERR_NULL;
+            int pos0_given = 0, int pos0 = 0, const int* seqlens = nullptr, const float* row_scale = nullptr,
+            int acc_only = 0) {
+  if (!q || !k || !v || !d_o || (!dq && !acc_only) || !dk || !dv) return SIGATTN_ERR_NULL;
+  if (acc_only && dtype != SIGATTN_DTYPE_BF16) return SIGATTN_ERR_FLAG;
   if (int rc = check_lengths(B, H, H_kv, N, N_k, D, causal, pos0_given, pos0)) return rc;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(d_o) || !aligned16(dq) || !aligned16(dk) ||
       !aligned16(dv))
@@ -152,7 +155,7 @@ int bwd_any(const void* q, const void* k, const void* v, const void* d_o, void* 
   int* status = nullptr;
   if (int rc = device_setup(&dev, &status)) return rc;
   sigattn::Problem p{B, H, N, D, scale, bias, causal, alibi_slopes, bias_vec, dbias, H_kv, N_k, pos0_given, pos0,
-                     seqlens, row_scale};
+                     seqlens, row_scale, nullptr, acc_only};
   unsigned long long launches = 0;
   cudaError_t ce = cudaSuccess;
   int rc;
@@ -516,6 +519,42 @@ int sigattn_bwd_rowscale(const void* q, const void* k, const void* v, const void
     return SIGATTN_ERR_ALIGN;
   return bwd_any(q, k, v, d_o, dq, dk, dv, B, H, H_kv, N_q, N_k, D, scale, bias, bias_bh, dbias_bh, causal,
                  alibi_slopes, dtype, workspace, workspace_bytes, stream, 0, 0, nullptr, row_scale);
+}
+
+int sigattn_fwd_shard_acc(const void* q, const void* k, const void* v, float* o_acc, int B, int H, int H_kv, int N_q,
+                          int N_k, int D, float scale, float bias, const float* bias_bh, int causal, int pos0,
+                          const float* alibi_slopes, int dtype, void* stream) {
+  if (!o_acc) return SIGATTN_ERR_NULL;
+  if ((reinterpret_cast<uintptr_t>(o_acc) & 15u) || (reinterpret_cast<uintptr_t>(bias_bh) & 3u)) return SIGATTN_ERR_ALIGN;
+  return fwd_any(q, k, v, nullptr, B, H, H_kv, N_q, N_k, D, scale, bias, bias_bh, causal, alibi_slopes, dtype, stream,
+                 1, pos0, nullptr, nullptr, o_acc, 1);
+}
+
+int sigattn_bwd_shard_acc(const void* q, const void* k, const void* v, const void* d_o, float* dq_acc, void* dk,
+                          void* dv, int B, int H, int H_kv, int N_q, int N_k, int D, float scale, float bias,
+                          const float* bias_bh, int causal, int pos0, const float* alibi_slopes, int dtype,
+                          float* dbias_bh, void* stream) {
+  if (!dq_acc) return SIGATTN_ERR_NULL;
+  if ((reinterpret_cast<uintptr_t>(bias_bh) & 3u) || (reinterpret_cast<uintptr_t>(dbias_bh) & 3u))
+    return SIGATTN_ERR_ALIGN;
+  return bwd_any(q, k, v, d_o, nullptr, dk, dv, B, H, H_kv, N_q, N_k, D, scale, bias, bias_bh, dbias_bh, causal,
+                 alibi_slopes, dtype, dq_acc, sigattn_bwd_workspace_bytes(B, H, N_q, D, dtype), stream, 1, pos0, nullptr,
+                 nullptr, 1);
+}
+
+int sigattn_acc_to_bf16(const float* acc, void* out, size_t n, float mul, void* stream) {
+  if (!acc || !out) return SIGATTN_ERR_NULL;
+  if (!aligned16(acc) || !aligned16(out)) return SIGATTN_ERR_ALIGN;
+  if (n == 0 || n % 4 != 0) return SIGATTN_ERR_SHAPE;
+  int dev = 0;
+  int* status = nullptr;
+  if (int rc = device_setup(&dev, &status)) return rc;
+  unsigned long long launches = 0;
+  cudaError_t ce = cudaSuccess;
+  const int rc = sigattn::launch_acc_to_bf16(acc, out, n, mul, static_cast<cudaStream_t>(stream), &launches, &ce);
+  g_launches.fetch_add(launches);
+  if (rc == SIGATTN_ERR_CUDA) t_last_cuda = ce;
+  return rc;
 }
 
 size_t sigattn_fwd_decode_workspace_bytes(int B, int H, int N_q, int D, int dtype) {

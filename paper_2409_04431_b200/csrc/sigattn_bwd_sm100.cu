@@ -668,6 +668,23 @@ void set_bwd_timing_events(cudaEvent_t start, cudaEvent_t stop) {
   t_ev_stop = stop;
 }
 
+int launch_acc_to_bf16(const float* acc, void* out, size_t n, float mul, cudaStream_t stream,
+                       unsigned long long* launches, cudaError_t* cuda_err) {
+  int dev = 0, num_sms = 0;
+  *cuda_err = cudaGetDevice(&dev);
+  if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
+  *cuda_err = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
+  if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
+  const size_t n_vec4 = n / 4;
+  const size_t want = n_vec4 / 256 + 1, cap = static_cast<size_t>(num_sms) * 8;
+  sigattn_bwd_convert_dq_kernel<<<static_cast<int>(want < cap ? want : cap), 256, 0, stream>>>(
+      reinterpret_cast<const float4*>(acc), static_cast<uint2*>(out), n_vec4, mul);
+  *cuda_err = cudaGetLastError();
+  if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
+  *launches += 1;
+  return SIGATTN_OK;
+}
+
 size_t bwd_bf16_workspace_bytes(int B, int H, int N, int D) {
   return static_cast<size_t>(B) * H * N * D * sizeof(float);
 }
@@ -719,9 +736,12 @@ int launch_bwd_bf16(const void* q, const void* k, const void* v, const void* d_o
   bp.status = status;
 
   const size_t n_elems = static_cast<size_t>(BH) * p.N * p.D;
-  // step 1: clear the fp32 dQ accumulator (and the bias gradient, which the kernel adds into)
-  *cuda_err = cudaMemsetAsync(workspace, 0, n_elems * sizeof(float), stream);
-  if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
+  // step 1: clear the fp32 dQ accumulator (and the bias gradient, which the kernel adds into);
+  // with acc_only the accumulator is the caller's running sum over key/value shards: not cleared
+  if (!p.acc_only) {
+    *cuda_err = cudaMemsetAsync(workspace, 0, n_elems * sizeof(float), stream);
+    if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
+  }
   if (p.dbias != nullptr) {
     *cuda_err = cudaMemsetAsync(p.dbias, 0, BH * sizeof(float), stream);
     if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
@@ -762,6 +782,8 @@ int launch_bwd_bf16(const void* q, const void* k, const void* v, const void* d_o
   if (rc != SIGATTN_OK) return rc;
   if (timed) cudaEventRecord(t_ev_stop, stream);
   *launches += 1;
+
+  if (p.acc_only) return SIGATTN_OK;   // the owner of the accumulator converts once every shard has added
 
   // step 3: dQ = scale * accumulator, as bf16
   const size_t n_vec4 = n_elems / 4;  // D is a multiple of 64

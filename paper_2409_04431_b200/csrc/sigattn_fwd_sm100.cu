@@ -460,26 +460,30 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
       uint32_t o[kECols];
       tmem_ld_cols(tO, o);
       tmem_wait_ld();
-      if (PACKED && p.n_splits > 1) {
-        // split keys: add this item's partial rows into the fp32 buffer (few rows: plain atomics);
-        // a later pass converts the sums to bf16.  The Q buffer is not needed for staging.
-        const int row = w.row0 + t * kBM + tid;
-        if (row < p.N) {
-          float* dst = p.split_ws + (static_cast<size_t>(w.bh) * p.N + row) * D + g * kECols;
-#pragma unroll
-          for (int e = 0; e < kECols; ++e) atomicAdd(dst + e, __uint_as_float(o[e]));
-        }
-        tc_fence_before_sync();
-        mbar_arrive(smem_u32(&bars->o_empty[t]));
-        if (threadIdx.x == 0) mbar_arrive(smem_u32(&bars->q_empty[t]));   // all logits MMAs of the item are done
-        continue;
-      }
       if (GENERAL && p.row_scale != nullptr) {
         // sequence-length normalisation: one factor per query row (rows past the end are not stored)
         const int row = w.row0 + t * kBM + tid;
         const float r = row < p.N ? __ldg(p.row_scale + row) : 0.0f;
 #pragma unroll
         for (int e = 0; e < kECols; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * r);
+      }
+      if ((PACKED || GENERAL) && p.split_ws != nullptr) {
+        // Partial result (split keys, or one shard of the keys): add this item's rows, in fp32,
+        // into the accumulator - local scratch or another GPU's memory, plain vector reductions
+        // either way.  Whoever owns the accumulator converts the sums to bf16 afterwards.  The Q
+        // buffer is not needed for staging.
+        const int row = w.row0 + t * kBM + tid;
+        if (row < p.N) {
+          float* dst = p.split_ws + (static_cast<size_t>(w.bh) * p.N + row) * D + g * kECols;
+#pragma unroll
+          for (int e = 0; e < kECols; e += 4)
+            red_add_v4_f32(dst + e, __uint_as_float(o[e]), __uint_as_float(o[e + 1]), __uint_as_float(o[e + 2]),
+                           __uint_as_float(o[e + 3]));
+        }
+        tc_fence_before_sync();
+        mbar_arrive(smem_u32(&bars->o_empty[t]));
+        if (threadIdx.x == 0) mbar_arrive(smem_u32(&bars->q_empty[t]));   // all logits MMAs of the item are done
+        continue;
       }
       {
         const int col = g * kECols;           // first of this thread's columns
@@ -643,10 +647,14 @@ int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const 
   const int n_kv_tiles = (p.key_rows() + kBN - 1) / kBN;
   const int n_splits = (small && p.split_ws != nullptr) ? choose_key_splits(static_cast<int>(BH_kv), n_kv_tiles, num_sms) : 1;
   const bool packed = small && (group > 1 || n_splits > 1);
+  // acc_only: the caller owns an fp32 accumulator that this call adds its (partial) O into; nothing
+  // is cleared, nothing converted, `o` is not written.  Otherwise the accumulator is only used as
+  // scratch when the keys are split.
+  const bool accumulate = p.split_ws != nullptr && (p.acc_only != 0 || n_splits > 1);
   const uint64_t q_heads = packed ? BH_kv : BH;
   const uint64_t q_rows = packed ? static_cast<uint64_t>(p.N) * group : p.N;
   CUtensorMap tmQ, tmK, tmV, tmO;
-  const void* ptrs[4] = {q, k, v, o};
+  const void* ptrs[4] = {q, k, v, (p.acc_only && o == nullptr) ? q : o};   // accumulate only: O is never stored
   CUtensorMap* maps[4] = {&tmQ, &tmK, &tmV, &tmO};
   for (int i = 0; i < 4; ++i) {
     const bool kv = (i == 1 || i == 2);
@@ -669,7 +677,7 @@ int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const 
   fp.n_kv_total = (p.key_rows() + kBN - 1) / kBN;
   fp.n_splits = n_splits;
   fp.tiles_per_split = (fp.n_kv_total + n_splits - 1) / n_splits;
-  fp.split_ws = p.split_ws;
+  fp.split_ws = accumulate ? p.split_ws : nullptr;
   fp.n_items = fp.n_pairs * fp.BH * n_splits;
   fp.scale_log2e = p.scale * kLog2e;
   fp.bias_log2e = p.bias * kLog2e;
@@ -680,7 +688,7 @@ int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const 
   fp.status = status;
 
   const size_t n_elems = static_cast<size_t>(BH) * p.N * p.D;
-  if (n_splits > 1) {
+  if (accumulate && !p.acc_only) {
     *cuda_err = cudaMemsetAsync(p.split_ws, 0, n_elems * sizeof(float), stream);
     if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
   }
@@ -689,7 +697,7 @@ int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const 
   const bool alibi = p.slopes != nullptr;
 #define SIGATTN_FWD_CASE(DD, CC, AA)                                                                       \
   rc = packed ? launch_fwd_variant<DD, CC, AA, 1>(tmQ, tmK, tmV, tmO, fp, num_sms, stream, cuda_err)       \
-       : (p.seqlens != nullptr || p.row_scale != nullptr)                                                  \
+       : (p.seqlens != nullptr || p.row_scale != nullptr || accumulate)                                    \
            ? launch_fwd_variant<DD, CC, AA, 2>(tmQ, tmK, tmV, tmO, fp, num_sms, stream, cuda_err)          \
            : launch_fwd_variant<DD, CC, AA, 0>(tmQ, tmK, tmV, tmO, fp, num_sms, stream, cuda_err)
   if (p.D == 128) {
@@ -702,7 +710,7 @@ int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const 
 #undef SIGATTN_FWD_CASE
   if (rc != SIGATTN_OK) return rc;
   *launches += 1;
-  if (n_splits > 1) {
+  if (accumulate && !p.acc_only) {
     const size_t n_vec4 = n_elems / 4;
     const size_t want = n_vec4 / 256 + 1, cap = static_cast<size_t>(num_sms) * 8;
     sigattn_fwd_convert_o_kernel<<<static_cast<int>(want < cap ? want : cap), 256, 0, stream>>>(

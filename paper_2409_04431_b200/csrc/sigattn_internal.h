@@ -25,6 +25,9 @@ struct Problem {
   const float* row_scale; // device pointer to N factors, one per query row, applied to O, or nullptr
   float* split_ws;        // forward only: device scratch of B*H*N*D floats that allows splitting the keys of a
                           // head over several thread blocks when there are few queries (decoding), or nullptr
+  int acc_only;           // 1: accumulate and stop.  Forward: add the partial O, fp32, into split_ws (never cleared,
+                          // never converted; o is not written).  Backward: add the partial dQ into the workspace
+                          // (not cleared) and leave dq unwritten.  For key/value shards whose results are summed.
 };
 
 // Every launcher enqueues on `stream`, adds the number of kernels it launched to
@@ -47,6 +50,10 @@ int launch_bwd_bf16(const void* q, const void* k, const void* v, const void* d_o
                     unsigned long long* launches, cudaError_t* cuda_err);
 
 int launch_seqlen_norm(float* out, int N, int N_k, int pos0, int causal, float alpha, cudaStream_t stream,
+                       unsigned long long* launches, cudaError_t* cuda_err);
+
+// out (bf16, n elements, n a multiple of 4) = mul * acc (fp32).
+int launch_acc_to_bf16(const float* acc, void* out, size_t n, float mul, cudaStream_t stream,
                        unsigned long long* launches, cudaError_t* cuda_err);
 
 size_t bwd_bf16_workspace_bytes(int B, int H, int N, int D);

@@ -84,6 +84,11 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   return mbar_wait_limit(bar, parity, cta_error, where, kWaitLimitCycles);
 }
 
+// Four consecutive floats added to global memory (16-byte aligned), no return value.
+__device__ __forceinline__ void red_add_v4_f32(float* dst, float a, float b, float c, float d) {
+  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+
 // ------------------------------------------------------------------ proxies and fences
 
 __device__ __forceinline__ void fence_proxy_async_smem() {

@@ -90,3 +90,32 @@ def kv_sharded_bwd(attend_bwd, q, k_shard, v_shard, d_o, key_start: int, query_s
         dist.all_reduce(acc, op=dist.ReduceOp.SUM, group=group)
         dq = acc.to(dq.dtype)
     return dq, dk, dv
+
+
+def kv_sharded_fwd_acc(attend_acc, q_slices, query_starts, k_shard, v_shard, key_start: int, accumulators):
+    """The sum over shards fused into the kernels: this rank adds its shard's summand of O for the
+    query rows of every owner straight into that owner's float32 accumulator (on several GPUs a
+    peer mapping of it), so no all-reduce follows.
+
+    q_slices[r], query_starts[r]: the query rows rank r owns and the position of their first row;
+    accumulators[r]: rank r's accumulator for those rows (tensor or device address), zero before
+    the first shard adds.  attend_acc(q, k_shard, v_shard, acc, pos0) is
+    binding.sigattn_fwd_shard_acc with the remaining arguments bound.  Every owner converts its
+    accumulator (binding.sigattn_acc_to_bf16) once all ranks have added."""
+    for q_r, start, acc in zip(q_slices, query_starts, accumulators):
+        attend_acc(q_r, k_shard, v_shard, acc, start - key_start)
+
+
+def kv_sharded_bwd_acc(attend_bwd_acc, q_slices, d_o_slices, query_starts, k_shard, v_shard, key_start: int,
+                       accumulators):
+    """Backward counterpart: dQ summands go into the owners' accumulators; dK and dV of this
+    rank's shard are the sums over the owners' query rows and stay local (float32 here, since
+    several calls contribute).
+
+    attend_bwd_acc(q, k_shard, v_shard, d_o, dq_acc, pos0) -> (dk_shard, dv_shard, ...)."""
+    dk = dv = None
+    for q_r, do_r, start, acc in zip(q_slices, d_o_slices, query_starts, accumulators):
+        g = attend_bwd_acc(q_r, k_shard, v_shard, do_r, acc, start - key_start)
+        dk = g[0].float() if dk is None else dk + g[0].float()
+        dv = g[1].float() if dv is None else dv + g[1].float()
+    return dk, dv

@@ -128,3 +128,45 @@ def test_two_gloo_ranks_sum_key_value_shards(tmp_path):
         np.testing.assert_allclose(r["dv"], ref_dv[:, :, lo:hi], rtol=1e-12, atol=1e-14)
         covered += list(range(lo, hi))
     assert covered == list(range(11))
+
+
+def test_fused_shard_sum_host_logic_with_shared_accumulators():
+    """kv_sharded_fwd_acc / kv_sharded_bwd_acc: every rank adds, for every owner of query rows,
+    into that owner's accumulator with the right position offset.  Three ranks are played in turn
+    in one process (the accumulators stand for peer-mapped memory), the oracle is the local call."""
+    import torch
+    import oracle
+    from paper_2409_04431_b200 import sharding
+    world, B, H, N, D = 3, 1, 2, 13, 4
+    rng = np.random.default_rng(9)
+    q, k, v, d_o = (rng.standard_normal((B, H, N, D)) for _ in range(4))
+    slopes = np.array([0.5, 0.25])
+    scale, bias = 0.5, -1.0
+
+    def attend_acc(a, b, c, acc, pos0):
+        acc += torch.from_numpy(oracle.sigattn_fwd(a.numpy(), b.numpy(), c.numpy(), scale, bias, True, slopes, pos0=pos0))
+
+    def attend_bwd_acc(a, b, c, d, acc, pos0):
+        dq, dk, dv = oracle.sigattn_bwd(a.numpy(), b.numpy(), c.numpy(), d.numpy(), scale, bias, True, slopes, pos0=pos0)
+        acc += torch.from_numpy(dq)
+        return torch.from_numpy(dk), torch.from_numpy(dv)
+
+    owners = [sharding.kv_shard_range(N, world, r) for r in range(world)]
+    cut = lambda t, r: torch.from_numpy(np.ascontiguousarray(t[:, :, r.start:r.stop]))
+    q_sl, do_sl = [cut(q, r) for r in owners], [cut(d_o, r) for r in owners]
+    starts = [r.start for r in owners]
+    o_acc = [torch.zeros_like(t) for t in q_sl]
+    dq_acc = [torch.zeros_like(t) for t in q_sl]
+    dk, dv = np.zeros_like(k), np.zeros_like(v)
+    for rank in range(world):
+        rows = sharding.kv_shard_range(N, world, rank)
+        sharding.kv_sharded_fwd_acc(attend_acc, q_sl, starts, cut(k, rows), cut(v, rows), rows.start, o_acc)
+        g = sharding.kv_sharded_bwd_acc(attend_bwd_acc, q_sl, do_sl, starts, cut(k, rows), cut(v, rows), rows.start,
+                                        dq_acc)
+        dk[:, :, rows.start:rows.stop], dv[:, :, rows.start:rows.stop] = g[0].numpy(), g[1].numpy()
+    ref_o = oracle.sigattn_fwd(q, k, v, scale, bias, True, slopes)
+    ref = oracle.sigattn_bwd(q, k, v, d_o, scale, bias, True, slopes)
+    np.testing.assert_allclose(torch.cat(o_acc, dim=2).numpy(), ref_o, rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(torch.cat(dq_acc, dim=2).numpy(), ref[0], rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(dk, ref[1], rtol=1e-6, atol=1e-7)      # the helper sums dK, dV in float32
+    np.testing.assert_allclose(dv, ref[2], rtol=1e-6, atol=1e-7)
