@@ -39,7 +39,7 @@ L2_FLUSH_BYTES = 256 << 20
 
 # DRAM bytes per launch of the dominant kernel (backward main kernel) from the committed
 # ncu capture, per workload; see profiles/.  None where no capture exists.
-NCU_TRAFFIC_BYTES = {"c4": 441.39e6 + 219.32e6}  # profiles/sigattn_bwd_bf16_kernel_c4.md
+NCU_TRAFFIC_BYTES = {"c4": 429.68e6 + 212.91e6}  # profiles/sigattn_bwd_bf16_kernel_c4.md
 
 
 def load_peaks():
