@@ -58,3 +58,26 @@ def test_decode_many_queries_is_the_plain_path_and_workspace_is_checked():
     with pytest.raises(sa.SigattnError) as e:
         sa.sigattn_fwd_decode(tq, tk, tv, scale, -2.0, True, workspace=ws[:-256])
     assert e.value.code == -5
+
+
+@pytest.mark.parametrize("B,H,H_kv,N_k", [
+    (8, 32, 32, 16384),      # the measured plain-head decode case
+    (1, 32, 8, 131072),      # the measured long-cache grouped-head case (8 work items unsplit)
+])
+def test_decode_full_size_cases(B, H, H_kv, N_k):
+    """The decode cases whose times are reported, checked in full against the oracle (one query
+    per head keeps the float64 reference cheap)."""
+    import torch
+    import paper_2409_04431_b200 as sa
+    D = 128
+    q, _, _, _ = inputs.random_case(B, H, 1, D, 191)
+    _, k, v, _ = inputs.random_case(B, H_kv, N_k, D, 192)
+    tq, tk, tv = (to_device(t, "bf16") for t in (q, k, v))
+    scale, bias = 1.0 / math.sqrt(D), -math.log(N_k)
+    o = sa.sigattn_fwd_decode(tq, tk, tv, scale, bias, True)
+    sa.sigattn_check()
+    ref = oracle.sigattn_fwd(q, k, v, scale, bias, True)
+    g = to_host(o)
+    assert np.isfinite(g).all()
+    assert rel_fro(g, ref) < BF16_REL_FRO, rel_fro(g, ref)
+    assert max_abs(g, ref) < 2e-2 * max(1.0, float(np.abs(ref).max()))
