@@ -67,6 +67,14 @@ Readings of the paper taken here
     dQ rows are zero, dK and dV do not see them).  The paper does not print this; it is the
     usual padding mask, and it makes the call equal to separate calls on the unpadded
     sequences.  Only for N_q = N_k.
+  * The same batches stored without padding, one after the other along the row axis (B = 1,
+    T = sum of the lengths rows): `cu_seqlens` holds the S + 1 row offsets 0 = c_0 <= c_1 <= ...
+    <= c_S = T, sequence s owns rows [c_s, c_{s+1}) of q, k and v.  The definition is the one
+    mask the layout implies: the weight of (query i, key j) is kept only if both rows belong to
+    the same sequence (a block-diagonal mask times, if asked for, the causal mask; positions are
+    counted within the sequence, which leaves i - j unchanged), and `bias` may then be an array
+    that broadcasts to [S, H], one bias per sequence and head (b = -log n_s).  That this equals
+    separate calls on the S sequences is what the tests check.
   * Sequence-length normalisation (the ablation in Appendix G that compares b = -log n with
     the scaling n^-alpha sigma(Q K^T / sqrt(d)) V): every row of O is multiplied by one
     factor r_i.  Without a mask r_i = n^-alpha for all rows.  For the causal form the paper
@@ -231,6 +239,17 @@ def _row_scale(row_scale, n_q):
     return r
 
 
+def _cu_seqlens(cu_seqlens, num_batch, n_q, n_k):
+    """Row offsets of a packed batch -> (offsets, sequence index of every row)."""
+    c = np.asarray(cu_seqlens).reshape(-1).astype(np.int64)
+    if num_batch != 1 or n_q != n_k:
+        raise ValueError("a packed batch has B = 1 and as many query rows as key rows")
+    if c.shape[0] < 2 or c[0] != 0 or c[-1] != n_q or np.any(np.diff(c) < 0):
+        raise ValueError("cu_seqlens must rise from 0 to the number of rows")
+    seq_of_row = np.searchsorted(c, np.arange(n_q), side="right") - 1
+    return c, seq_of_row
+
+
 def _row_ranges(n, row_block):
     """Query rows are independent in the forward and enter dK, dV only through a sum
     over rows, so they may be visited in slabs to bound memory (an n x n float64 matrix
@@ -240,7 +259,7 @@ def _row_ranges(n, row_block):
 
 
 def sigattn_fwd(q, k, v, scale, bias, causal=False, alibi_slopes=None, row_block=None, pos0=None, seqlens=None,
-                row_scale=None):
+                row_scale=None, cu_seqlens=None):
     """O = sigmoid(scale * Q K^T + b [+ position bias]) [* causal mask] V  (Eq. 3).
 
     q: [B, H, N, D]; k, v: [B, H_kv, N, D] with H a multiple of H_kv (any float dtype;
@@ -248,10 +267,13 @@ def sigattn_fwd(q, k, v, scale, bias, causal=False, alibi_slopes=None, row_block
     bias: scalar, or an array that broadcasts to [B, H] (one bias per sequence and head).
     pos0: position of query row 0 relative to key row 0 (default: rows of k minus rows of q).
     row_scale: one factor per query row (sequence-length normalisation), or None.
+    cu_seqlens: row offsets of a packed batch (B = 1; see header), or None.
     Returns O as float64 [B, H, N, D].
     """
     q, k, v = _as_f64(q, k, v)
     B, H, N, D = q.shape          # N counts query rows; k, v may hold more (or fewer) rows
+    if cu_seqlens is not None:
+        return _packed_all(q, k, v, None, scale, bias, causal, alibi_slopes, cu_seqlens)[0]
     group = _kv_group(H, k)
     slopes = _slopes(alibi_slopes, H)
     bias_bh = _bias_per_head(bias, B, H)
@@ -268,8 +290,46 @@ def sigattn_fwd(q, k, v, scale, bias, causal=False, alibi_slopes=None, row_block
     return o
 
 
-def _bwd_all(q, k, v, d_o, scale, bias, causal, alibi_slopes, row_block, pos0=None, seqlens=None, row_scale=None):
+def _packed_all(q, k, v, d_o, scale, bias, causal, alibi_slopes, cu_seqlens):
+    """Packed batch (see header): block-diagonal mask over the T x T weights of each head, one
+    bias per (sequence, head).  Returns (O, dQ, dK, dV, dbias[S, H]); gradients are None without d_o."""
+    B, H, T, D = q.shape
+    group = _kv_group(H, k)
+    slopes = _slopes(alibi_slopes, H)
+    c, seq = _cu_seqlens(cu_seqlens, B, T, k.shape[2])
+    S = c.shape[0] - 1
+    bias_sh = _bias_per_head(bias, S, H)
+    same = (seq[:, None] == seq[None, :]).astype(np.float64)       # both rows in one sequence
+    o = np.zeros_like(q)
+    dq, dk, dv = np.zeros_like(q), np.zeros_like(k), np.zeros_like(v)
+    dbias = np.zeros((S, H), dtype=np.float64)
+    for h in range(H):
+        hk = h // group
+        x = scale * (q[0, h] @ k[0, hk].T) + bias_sh[seq, h][:, None]
+        if slopes[h] != 0.0:
+            x = x + position_bias(T, slopes[h])
+        p = sigmoid(x) * same
+        if causal:
+            p = p * causal_mask(T)
+        o[0, h] = p @ v[0, hk]
+        if d_o is None:
+            continue
+        dv[0, hk] += p.T @ d_o[0, h]
+        dp = d_o[0, h] @ v[0, hk].T
+        ds = p * (1.0 - p) * dp
+        dq[0, h] = scale * (ds @ k[0, hk])
+        dk[0, hk] += scale * (ds.T @ q[0, h])
+        np.add.at(dbias[:, h], seq, ds.sum(axis=1))
+    if d_o is None:
+        return o, None, None, None, None
+    return o, dq, dk, dv, dbias
+
+
+def _bwd_all(q, k, v, d_o, scale, bias, causal, alibi_slopes, row_block, pos0=None, seqlens=None, row_scale=None,
+             cu_seqlens=None):
     q, k, v, d_o = _as_f64(q, k, v, d_o)
+    if cu_seqlens is not None:
+        return _packed_all(q, k, v, d_o, scale, bias, causal, alibi_slopes, cu_seqlens)[1:]
     B, H, N, D = q.shape
     group = _kv_group(H, k)
     slopes = _slopes(alibi_slopes, H)
@@ -297,7 +357,7 @@ def _bwd_all(q, k, v, d_o, scale, bias, causal, alibi_slopes, row_block, pos0=No
 
 
 def sigattn_bwd(q, k, v, d_o, scale, bias, causal=False, alibi_slopes=None, row_block=None, pos0=None,
-                seqlens=None, row_scale=None):
+                seqlens=None, row_scale=None, cu_seqlens=None):
     """Gradients of L = sum(O * dO) with respect to Q, K, V (sigmoid column of the
     forward/backward table in Appendix F.1, with the 1/sqrt(d) factor; see header).
 
@@ -305,18 +365,20 @@ def sigattn_bwd(q, k, v, d_o, scale, bias, causal=False, alibi_slopes=None, row_
     than q (see header).
     Returns (dQ, dK, dV), float64, shaped like q, k, v.
     """
-    return _bwd_all(q, k, v, d_o, scale, bias, causal, alibi_slopes, row_block, pos0, seqlens, row_scale)[:3]
+    return _bwd_all(q, k, v, d_o, scale, bias, causal, alibi_slopes, row_block, pos0, seqlens, row_scale,
+                    cu_seqlens)[:3]
 
 
 def sigattn_bwd_dbias(q, k, v, d_o, scale, bias, causal=False, alibi_slopes=None, row_block=None, pos0=None,
-                      seqlens=None, row_scale=None):
+                      seqlens=None, row_scale=None, cu_seqlens=None):
     """Gradient of L = sum(O * dO) with respect to a bias held per (batch, head):
     db[b, h] = sum_ij dS_ij with dS = P (1 - P) dP as in sigattn_bwd (see header).  A
     bias shared by several heads or sequences gets the sum of their entries.
 
-    Returns float64 [B, H].
+    Returns float64 [B, H] ([S, H], one row per sequence, for a packed batch).
     """
-    return _bwd_all(q, k, v, d_o, scale, bias, causal, alibi_slopes, row_block, pos0, seqlens, row_scale)[3]
+    return _bwd_all(q, k, v, d_o, scale, bias, causal, alibi_slopes, row_block, pos0, seqlens, row_scale,
+                    cu_seqlens)[3]
 
 
 def sigattn_fwd_sequence_form(q, k, v, scale, n_bias):

@@ -647,3 +647,58 @@ def test_row_scale_brute_force_and_finite_differences(causal):
     plain = oracle.sigattn_bwd(q, k, v, d_o, scale, bias, causal, slopes)
     for g, pl in zip((dq, dk, dv), plain):
         assert np.linalg.norm(g - pl) / np.linalg.norm(g) > 0.05
+
+
+# ------------------------------------------------------------------------ packed batches
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_packed_batch_equals_separate_calls(causal):
+    """cu_seqlens: sequences stored one after the other; every output equals the call on
+    that sequence alone (with its own bias), including an empty sequence in the middle."""
+    H, D = 2, 3
+    lens = [4, 0, 7, 1]
+    cu = np.concatenate([[0], np.cumsum(lens)])
+    T = int(cu[-1])
+    q, k, v, d_o = (rnd((1, H, T, D), s) for s in (170, 171, 172, 173))
+    slopes = np.array([0.5, 0.25])
+    scale = 0.7
+    bias = np.array([[-1.0, -0.5], [9.0, 9.0], [-2.0, 0.3], [0.0, -3.0]])   # per (sequence, head)
+    o = oracle.sigattn_fwd(q, k, v, scale, bias, causal, slopes, cu_seqlens=cu)
+    dq, dk, dv = oracle.sigattn_bwd(q, k, v, d_o, scale, bias, causal, slopes, cu_seqlens=cu)
+    db = oracle.sigattn_bwd_dbias(q, k, v, d_o, scale, bias, causal, slopes, cu_seqlens=cu)
+    assert db.shape == (4, H) and np.all(db[1] == 0.0)
+    for s, n in enumerate(lens):
+        if n == 0:
+            continue
+        sel = (slice(None), slice(None), slice(int(cu[s]), int(cu[s + 1])))
+        b = bias[s][None, :]
+        np.testing.assert_allclose(o[sel], oracle.sigattn_fwd(q[sel], k[sel], v[sel], scale, b, causal, slopes),
+                                   rtol=1e-13, atol=1e-16)
+        one = oracle.sigattn_bwd(q[sel], k[sel], v[sel], d_o[sel], scale, b, causal, slopes)
+        for g, r in zip((dq, dk, dv), one):
+            np.testing.assert_allclose(g[sel], r, rtol=1e-12, atol=1e-15)
+        np.testing.assert_allclose(db[s], oracle.sigattn_bwd_dbias(q[sel], k[sel], v[sel], d_o[sel], scale, b, causal, slopes)[0],
+                                   rtol=1e-12)
+    # one sequence is the plain call
+    np.testing.assert_allclose(oracle.sigattn_fwd(q, k, v, scale, -1.0, causal, slopes, cu_seqlens=[0, T]),
+                               oracle.sigattn_fwd(q, k, v, scale, -1.0, causal, slopes), rtol=1e-14)
+    with pytest.raises(ValueError):
+        oracle.sigattn_fwd(q, k, v, scale, -1.0, causal, cu_seqlens=[0, 5, 3, T])
+
+
+def test_packed_batch_brute_force_with_shared_kv_heads():
+    """Explicit loops over the packed layout with one key/value head for two query heads."""
+    H, D = 2, 2
+    cu = [0, 3, 5]
+    q, d_o = rnd((1, H, 5, D), 180), rnd((1, H, 5, D), 183)
+    k, v = rnd((1, 1, 5, D), 181), rnd((1, 1, 5, D), 182)
+    scale, bias = 0.9, np.array([[-0.4, 0.1], [0.6, -1.1]])
+    o = oracle.sigattn_fwd(q, k, v, scale, bias, True, cu_seqlens=cu)
+    ref = np.zeros_like(o)
+    for h in range(H):
+        for s in range(2):
+            for i in range(cu[s], cu[s + 1]):
+                for j in range(cu[s], i + 1):
+                    ref[0, h, i] += scalar_sigmoid(scale * float(q[0, h, i] @ k[0, 0, j]) + bias[s, h]) * v[0, 0, j]
+    np.testing.assert_allclose(o, ref, rtol=1e-13, atol=1e-16)
