@@ -275,6 +275,34 @@ SIGATTN_API int sigattn_bwd_varlen(const void* q, const void* k, const void* v, 
                        float* dbias_bh,
                        void* workspace, size_t workspace_bytes, void* stream);
 
+/* The same batches stored WITHOUT padding, one sequence after the other along the row axis:
+ * q, o are [1, H, T, D], k, v are [1, H_kv, T, D] with T the sum of the lengths, and
+ * `cu_seqlens` is a DEVICE pointer to n_seqs + 1 int32 row offsets 0 = c_0 <= c_1 <= ... <=
+ * c_{n_seqs} = T (4-byte aligned, read while the kernels run; the caller guarantees that they
+ * rise from 0 to T - they are not checked on the device).  Sequence s owns rows [c_s, c_{s+1});
+ * the weight of (query i, key j) is kept only if both rows belong to the same sequence (a
+ * block-diagonal mask, times the causal mask if asked for; ALiBi distances are i - j as ever),
+ * so the call equals n_seqs separate calls.  Empty sequences are allowed.  `bias_sh` is NULL
+ * (scalar `bias`) or a DEVICE pointer to n_seqs * H floats, one bias per (sequence, head), e.g.
+ * b = -log n_s; `dbias_sh`, if not NULL, receives the matching n_seqs * H gradients.  Tiles are
+ * 128 rows whatever the lengths: a tile that spans several short sequences computes all its
+ * 128 x 128 logits and masks the foreign ones, so many sequences much shorter than 128 rows cost
+ * as much as 128-row ones.  The workspace is that of sigattn_bwd for (1, H, T, D). */
+SIGATTN_API int sigattn_fwd_ragged(const void* q, const void* k, const void* v, void* o,
+                       int H, int H_kv, int T, int D,
+                       const int* cu_seqlens, int n_seqs,
+                       float scale, float bias, const float* bias_sh, int causal,
+                       const float* alibi_slopes, int dtype, void* stream);
+
+SIGATTN_API int sigattn_bwd_ragged(const void* q, const void* k, const void* v, const void* d_o,
+                       void* dq, void* dk, void* dv,
+                       int H, int H_kv, int T, int D,
+                       const int* cu_seqlens, int n_seqs,
+                       float scale, float bias, const float* bias_sh, int causal,
+                       const float* alibi_slopes, int dtype,
+                       float* dbias_sh,
+                       void* workspace, size_t workspace_bytes, void* stream);
+
 /* Sequence-length normalisation (Appendix G, the ablation that compares the bias b = -log n with
  * the scaling n^-alpha sigma(Q K^T / sqrt(d)) V and its causal form, the equation labelled
  * "ar_seq_len_normalization"): O_i = r_i sum_j P_ij V_j with one factor r_i per query row, shared by

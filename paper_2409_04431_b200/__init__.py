@@ -42,6 +42,8 @@ _BINDING_NAMES = (
     "sigattn_fwd_shard_acc",
     "sigattn_bwd_shard_acc",
     "sigattn_acc_to_bf16",
+    "sigattn_fwd_ragged",
+    "sigattn_bwd_ragged",
     "sigattn_fwd_decode_workspace_bytes",
     "lib",
 )

@@ -73,6 +73,14 @@ _lib.sigattn_bwd_rowscale.restype = _c.c_int
 _lib.sigattn_bwd_rowscale.argtypes = [_c.c_void_p] * 7 + [_c.c_int] * 6 + [_c.c_float, _c.c_float, _c.c_void_p, _c.c_int,
                                                                              _c.c_void_p, _c.c_void_p, _c.c_int, _c.c_void_p,
                                                                              _c.c_void_p, _c.c_size_t, _c.c_void_p]
+_lib.sigattn_fwd_ragged.restype = _c.c_int
+_lib.sigattn_fwd_ragged.argtypes = [_c.c_void_p] * 4 + [_c.c_int] * 4 + [_c.c_void_p, _c.c_int, _c.c_float, _c.c_float,
+                                                                           _c.c_void_p, _c.c_int, _c.c_void_p, _c.c_int,
+                                                                           _c.c_void_p]
+_lib.sigattn_bwd_ragged.restype = _c.c_int
+_lib.sigattn_bwd_ragged.argtypes = [_c.c_void_p] * 7 + [_c.c_int] * 4 + [_c.c_void_p, _c.c_int, _c.c_float, _c.c_float,
+                                                                           _c.c_void_p, _c.c_int, _c.c_void_p, _c.c_int,
+                                                                           _c.c_void_p, _c.c_void_p, _c.c_size_t, _c.c_void_p]
 _lib.sigattn_fwd_shard_acc.restype = _c.c_int
 _lib.sigattn_fwd_shard_acc.argtypes = [_c.c_void_p] * 4 + [_c.c_int] * 6 + [_c.c_float, _c.c_float, _c.c_void_p,
                                                                               _c.c_int, _c.c_int, _c.c_void_p, _c.c_int,
@@ -130,6 +138,7 @@ EXPORTED = [
     "sigattn_fwd_rowscale", "sigattn_bwd_rowscale", "sigattn_seqlen_norm",
     "sigattn_fwd_decode", "sigattn_fwd_decode_workspace_bytes",
     "sigattn_fwd_shard_acc", "sigattn_bwd_shard_acc", "sigattn_acc_to_bf16",
+    "sigattn_fwd_ragged", "sigattn_bwd_ragged",
 ]
 
 
@@ -530,6 +539,65 @@ def sigattn_bwd_varlen(q, k, v, d_o, scale, bias, seqlens, causal=False, alibi_s
                                      float(scale), 0.0 if vec else float(bias), _ptr(bias) if vec else None,
                                      int(bool(causal)), _ptr(seqlens), _ptr(alibi_slopes), code, _ptr(dbias),
                                      _ptr(workspace), ws_bytes, _stream_ptr(stream))
+    if rc != 0:
+        raise SigattnError(rc)
+    return dq, dk, dv, dbias
+
+
+def _check_ragged(q, k, v, cu_seqlens, bias):
+    import torch
+    B, H, H_kv, T, D = _check_gqa(q, k, v)
+    if B != 1:
+        raise ValueError("a batch without padding has B = 1: q [1, H, T, D], k, v [1, H_kv, T, D]")
+    if (not isinstance(cu_seqlens, torch.Tensor) or not cu_seqlens.is_cuda or cu_seqlens.dtype != torch.int32
+            or cu_seqlens.dim() != 1 or cu_seqlens.numel() < 2 or not cu_seqlens.is_contiguous()
+            or cu_seqlens.device != q.device):
+        raise ValueError("cu_seqlens must be a contiguous int32 CUDA tensor of n_seqs + 1 row offsets on q's device")
+    n_seqs = cu_seqlens.numel() - 1
+    vec = isinstance(bias, torch.Tensor)
+    if vec and (not bias.is_cuda or bias.dtype != torch.float32 or tuple(bias.shape) != (n_seqs, H)
+                or not bias.is_contiguous() or bias.device != q.device):
+        raise ValueError("bias must be a float or a contiguous float32 CUDA tensor [n_seqs, H] on q's device")
+    return H, H_kv, T, D, n_seqs, vec
+
+
+def sigattn_fwd_ragged(q, k, v, cu_seqlens, scale, bias, causal=False, alibi_slopes=None, out=None, stream=None):
+    """Batch stored without padding: q [1, H, T, D], k, v [1, H_kv, T, D]; `cu_seqlens` int32 CUDA
+    [n_seqs + 1] row offsets (rising from 0 to T; the caller's responsibility); `bias`: float or
+    float32 CUDA [n_seqs, H]."""
+    import torch
+    H, H_kv, T, D, n_seqs, vec = _check_ragged(q, k, v, cu_seqlens, bias)
+    if out is None:
+        out = torch.empty_like(q)
+    else:
+        _check_same([q, out], ["q", "out"])
+    with torch.cuda.device(q.device):
+        rc = _lib.sigattn_fwd_ragged(_ptr(q), _ptr(k), _ptr(v), _ptr(out), H, H_kv, T, D, _ptr(cu_seqlens), n_seqs,
+                                     float(scale), 0.0 if vec else float(bias), _ptr(bias) if vec else None,
+                                     int(bool(causal)), _ptr(alibi_slopes), _dtype_code(q), _stream_ptr(stream))
+    if rc != 0:
+        raise SigattnError(rc)
+    return out
+
+
+def sigattn_bwd_ragged(q, k, v, d_o, cu_seqlens, scale, bias, causal=False, alibi_slopes=None, want_dbias=False,
+                       workspace=None, stream=None):
+    """Backward of sigattn_fwd_ragged: (dQ, dK, dV, dbias [n_seqs, H] or None)."""
+    import torch
+    H, H_kv, T, D, n_seqs, vec = _check_ragged(q, k, v, cu_seqlens, bias)
+    _check_same([q, d_o], ["q", "d_o"])
+    code = _dtype_code(q)
+    dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+    dbias = torch.empty((n_seqs, H), dtype=torch.float32, device=q.device) if want_dbias else None
+    need = sigattn_bwd_workspace_bytes(1, H, T, D, code)
+    if workspace is None and need > 0:
+        workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    with torch.cuda.device(q.device):
+        rc = _lib.sigattn_bwd_ragged(_ptr(q), _ptr(k), _ptr(v), _ptr(d_o), _ptr(dq), _ptr(dk), _ptr(dv), H, H_kv, T, D,
+                                     _ptr(cu_seqlens), n_seqs, float(scale), 0.0 if vec else float(bias),
+                                     _ptr(bias) if vec else None, int(bool(causal)), _ptr(alibi_slopes), code,
+                                     _ptr(dbias), _ptr(workspace), ws_bytes, _stream_ptr(stream))
     if rc != 0:
         raise SigattnError(rc)
     return dq, dk, dv, dbias

@@ -103,7 +103,8 @@ int check_lengths(int B, int H, int H_kv, int N, int N_k, int D, int causal, int
 int fwd_any(const void* q, const void* k, const void* v, void* o, int B, int H, int H_kv, int N, int N_k, int D,
             float scale, float bias, const float* bias_vec, int causal, const float* alibi_slopes, int dtype,
             void* stream, int pos0_given = 0, int pos0 = 0, const int* seqlens = nullptr,
-            const float* row_scale = nullptr, float* split_ws = nullptr, int acc_only = 0) {
+            const float* row_scale = nullptr, float* split_ws = nullptr, int acc_only = 0,
+            const int* cu_seqlens = nullptr, int n_seqs = 0) {
   if (!q || !k || !v || (!o && !acc_only)) return SIGATTN_ERR_NULL;
   if (int rc = check_lengths(B, H, H_kv, N, N_k, D, causal, pos0_given, pos0)) return rc;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return SIGATTN_ERR_ALIGN;
@@ -115,7 +116,7 @@ int fwd_any(const void* q, const void* k, const void* v, void* o, int B, int H, 
   int* status = nullptr;
   if (int rc = device_setup(&dev, &status)) return rc;
   sigattn::Problem p{B, H, N, D, scale, bias, causal, alibi_slopes, bias_vec, nullptr, H_kv, N_k, pos0_given, pos0,
-                     seqlens, row_scale, split_ws, acc_only};
+                     seqlens, row_scale, split_ws, acc_only, cu_seqlens, n_seqs};
   unsigned long long launches = 0;
   cudaError_t ce = cudaSuccess;
   int rc;
@@ -135,7 +136,7 @@ int bwd_any(const void* q, const void* k, const void* v, const void* d_o, void* 
             int H_kv, int N, int N_k, int D, float scale, float bias, const float* bias_vec, float* dbias, int causal,
             const float* alibi_slopes, int dtype, void* workspace, size_t workspace_bytes, void* stream,
             int pos0_given = 0, int pos0 = 0, const int* seqlens = nullptr, const float* row_scale = nullptr,
-            int acc_only = 0) {
+            int acc_only = 0, const int* cu_seqlens = nullptr, int n_seqs = 0) {
   if (!q || !k || !v || !d_o || (!dq && !acc_only) || !dk || !dv) return SIGATTN_ERR_NULL;
   if (acc_only && dtype != SIGATTN_DTYPE_BF16) return SIGATTN_ERR_FLAG;
   if (int rc = check_lengths(B, H, H_kv, N, N_k, D, causal, pos0_given, pos0)) return rc;
@@ -155,7 +156,7 @@ int bwd_any(const void* q, const void* k, const void* v, const void* d_o, void* 
   int* status = nullptr;
   if (int rc = device_setup(&dev, &status)) return rc;
   sigattn::Problem p{B, H, N, D, scale, bias, causal, alibi_slopes, bias_vec, dbias, H_kv, N_k, pos0_given, pos0,
-                     seqlens, row_scale, nullptr, acc_only};
+                     seqlens, row_scale, nullptr, acc_only, cu_seqlens, n_seqs};
   unsigned long long launches = 0;
   cudaError_t ce = cudaSuccess;
   int rc;
@@ -555,6 +556,30 @@ int sigattn_acc_to_bf16(const float* acc, void* out, size_t n, float mul, void* 
   g_launches.fetch_add(launches);
   if (rc == SIGATTN_ERR_CUDA) t_last_cuda = ce;
   return rc;
+}
+
+int sigattn_fwd_ragged(const void* q, const void* k, const void* v, void* o, int H, int H_kv, int T, int D,
+                       const int* cu_seqlens, int n_seqs, float scale, float bias, const float* bias_sh, int causal,
+                       const float* alibi_slopes, int dtype, void* stream) {
+  if (!cu_seqlens) return SIGATTN_ERR_NULL;
+  if (n_seqs < 1) return SIGATTN_ERR_SHAPE;
+  if ((reinterpret_cast<uintptr_t>(cu_seqlens) & 3u) || (reinterpret_cast<uintptr_t>(bias_sh) & 3u))
+    return SIGATTN_ERR_ALIGN;
+  return fwd_any(q, k, v, o, 1, H, H_kv, T, T, D, scale, bias, bias_sh, causal, alibi_slopes, dtype, stream, 0, 0,
+                 nullptr, nullptr, nullptr, 0, cu_seqlens, n_seqs);
+}
+
+int sigattn_bwd_ragged(const void* q, const void* k, const void* v, const void* d_o, void* dq, void* dk, void* dv,
+                       int H, int H_kv, int T, int D, const int* cu_seqlens, int n_seqs, float scale, float bias,
+                       const float* bias_sh, int causal, const float* alibi_slopes, int dtype, float* dbias_sh,
+                       void* workspace, size_t workspace_bytes, void* stream) {
+  if (!cu_seqlens) return SIGATTN_ERR_NULL;
+  if (n_seqs < 1) return SIGATTN_ERR_SHAPE;
+  if ((reinterpret_cast<uintptr_t>(cu_seqlens) & 3u) || (reinterpret_cast<uintptr_t>(bias_sh) & 3u) ||
+      (reinterpret_cast<uintptr_t>(dbias_sh) & 3u))
+    return SIGATTN_ERR_ALIGN;
+  return bwd_any(q, k, v, d_o, dq, dk, dv, 1, H, H_kv, T, T, D, scale, bias, bias_sh, dbias_sh, causal, alibi_slopes,
+                 dtype, workspace, workspace_bytes, stream, 0, 0, nullptr, nullptr, 0, cu_seqlens, n_seqs);
 }
 
 size_t sigattn_fwd_decode_workspace_bytes(int B, int H, int N_q, int D, int dtype) {

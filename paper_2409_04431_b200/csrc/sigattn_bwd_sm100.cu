@@ -73,6 +73,10 @@ struct BwdParams {
   int n_tiles_k;  // key tiles: ceil(rows of K / 128)
   int pos0;       // position of query row 0 relative to key row 0 (see FwdParams of the forward)
   const int* seqlens;   // padded batch: valid length per batch entry (keys and queries), or nullptr
+  // batch stored without padding (B = 1): sequence s owns rows [cu_seqlens[s], cu_seqlens[s + 1]);
+  // bias_vec and dbias then hold one entry per (sequence, head)
+  const int* cu_seqlens;
+  int n_seqs;
   int n_items;
   float scale, scale_log2e, bias_log2e;
   const float* bias_vec;   // one bias per (batch, head) instead of the scalar, or nullptr
@@ -104,6 +108,16 @@ __device__ __forceinline__ int bwd_num_rounds(int n_items) { return (n_items + g
 // GROUPED = false compiles the plain case (one query head per key/value head, no padded batch)
 // without the head loop and without the per-sequence lengths; it is the benchmarked path.
 // GROUPED = true serves both grouped heads and padded batches.
+// Sequence that owns `row` in a batch stored without padding: the largest s with cu[s] <= row.
+__device__ __forceinline__ int bwd_seq_of_row(const int* __restrict__ cu, int n_seqs, int row) {
+  int lo = 0, hi = n_seqs;   // cu[lo] <= row < cu[hi]
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (__ldg(cu + mid) <= row) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
 template <bool CAUSAL, bool GROUPED>
 __device__ __forceinline__ BwdItem decode_bwd_item(const BwdParams& p, int item) {
   BwdItem w;
@@ -120,6 +134,15 @@ __device__ __forceinline__ BwdItem decode_bwd_item(const BwdParams& p, int item)
   // a key tile wholly past the sequence's end needs one (fully masked) query tile to write its zeros
   if (padded && w.j * kT >= w.n_valid) w.i_begin = n_tiles_q - 1;
   w.n = n_tiles_q - w.i_begin;
+  if (GROUPED && p.cu_seqlens != nullptr) {
+    // batch without padding: the queries that see this key tile run from the start of its first
+    // key's sequence (causal: from the first key itself) to the end of its last key's sequence
+    const int k_first = w.j * kT, k_last = min(p.N, k_first + kT) - 1;
+    const int q_lo = CAUSAL ? k_first : __ldg(p.cu_seqlens + bwd_seq_of_row(p.cu_seqlens, p.n_seqs, k_first));
+    const int q_hi = __ldg(p.cu_seqlens + bwd_seq_of_row(p.cu_seqlens, p.n_seqs, k_last) + 1);
+    w.i_begin = q_lo / kT;
+    w.n = (q_hi + kT - 1) / kT - w.i_begin;
+  }
   w.steps = GROUPED ? p.group * w.n : w.n;
   return w;
 }
@@ -369,8 +392,22 @@ __device__ void bwd_act_role(const BwdParams& p, const CUtensorMap* tmDk, const 
     const int bh_q = w.bh_q0 + g;
     float slope_log2e = 0.0f;
     if (ALIBI) slope_log2e = p.slopes[bh_q % p.H] * kLog2eB;
-    const float bias_log2e = p.bias_vec ? __ldg(p.bias_vec + bh_q) * kLog2eB : p.bias_log2e;
+    float bias_log2e = p.bias_vec ? __ldg(p.bias_vec + bh_q) * kLog2eB : p.bias_log2e;
     float ds_sum = 0.0f;   // this thread's share of sum dS over the head's tiles (the bias gradient)
+    // batch without padding: the queries [q_lo, q_hi) that see this thread's key (its own sequence,
+    // from the key itself on when causal), and the sequence's bias
+    const bool ragged = GROUPED && p.cu_seqlens != nullptr;
+    int q_lo = 0, q_hi = 0, seq = 0;
+    if (ragged) {
+      const int kr = w.j * kT + tid;
+      bias_log2e = p.bias_log2e;
+      if (kr < p.N) {
+        seq = bwd_seq_of_row(p.cu_seqlens, p.n_seqs, kr);
+        q_lo = CAUSAL ? kr : __ldg(p.cu_seqlens + seq);
+        q_hi = __ldg(p.cu_seqlens + seq + 1);
+        if (p.bias_vec) bias_log2e = __ldg(p.bias_vec + seq * p.H + bh_q) * kLog2eB;
+      }
+    }
 
     for (int it = 0; it < w.n; ++it) {
       const int i = w.i_begin + it;
@@ -385,6 +422,11 @@ __device__ void bwd_act_role(const BwdParams& p, const CUtensorMap* tmDk, const 
         mask_hi = static_cast<float>(w.n_valid - i * kT);
         if (w.j * kT + tid >= w.n_valid) mask_hi = -1.0f;   // a key past the end: the whole row
         diag = diag || (w.j + 1) * kT > w.n_valid || (i + 1) * kT > w.n_valid;
+      }
+      if (ragged) {
+        mask_lo = static_cast<float>(q_lo - i * kT);
+        mask_hi = static_cast<float>(q_hi - i * kT);
+        diag = i * kT < q_lo || (i + 1) * kT > q_hi;   // the tile is not wholly inside this key's queries
       }
       float pp0[32], pp1[32];
       if (!mbar_wait(smem_u32(&bars->s_full), step_cnt & 1, cta_err, 60 + wg)) return;
@@ -445,7 +487,9 @@ __device__ void bwd_act_role(const BwdParams& p, const CUtensorMap* tmDk, const 
       ++step_cnt;
     }
 
-    if (DBIAS) {   // sum over the warp, one atomic per warp, item and query head
+    if (DBIAS && ragged) {   // keys of one warp may belong to different sequences: one atomic per key
+      if (q_hi > q_lo) atomicAdd(p.dbias + seq * p.H + bh_q, ds_sum);
+    } else if (DBIAS) {   // sum over the warp, one atomic per warp, item and query head
 #pragma unroll
       for (int off = 16; off > 0; off >>= 1) ds_sum += __shfl_xor_sync(0xffffffffu, ds_sum, off);
       if ((threadIdx.x & 31) == 0) atomicAdd(p.dbias + bh_q, ds_sum);
@@ -733,6 +777,8 @@ int launch_bwd_bf16(const void* q, const void* k, const void* v, const void* d_o
   bp.dbias = p.dbias;
   bp.slopes = p.slopes;
   bp.seqlens = p.seqlens;
+  bp.cu_seqlens = p.cu_seqlens;
+  bp.n_seqs = p.n_seqs;
   bp.status = status;
 
   const size_t n_elems = static_cast<size_t>(BH) * p.N * p.D;
@@ -743,7 +789,8 @@ int launch_bwd_bf16(const void* q, const void* k, const void* v, const void* d_o
     if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
   }
   if (p.dbias != nullptr) {
-    *cuda_err = cudaMemsetAsync(p.dbias, 0, BH * sizeof(float), stream);
+    const size_t n_bias = p.cu_seqlens != nullptr ? static_cast<size_t>(p.n_seqs) * p.H : BH;
+    *cuda_err = cudaMemsetAsync(p.dbias, 0, n_bias * sizeof(float), stream);
     if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
   }
 
@@ -766,7 +813,7 @@ int launch_bwd_bf16(const void* q, const void* k, const void* v, const void* d_o
   // is compiled in only where it is asked for; likewise the loop over a group's query heads
   // and the per-sequence lengths
 #define SIGATTN_BWD_CASE(DD, CC, AA)                                                                        \
-  rc = (bp.group > 1 || bp.seqlens != nullptr)                                                              \
+  rc = (bp.group > 1 || bp.seqlens != nullptr || bp.cu_seqlens != nullptr)                                  \
            ? ((p.dbias != nullptr) ? launch_bwd_variant<DD, CC, AA, true, true>(maps, bp, num_sms, stream, cuda_err)   \
                                    : launch_bwd_variant<DD, CC, AA, false, true>(maps, bp, num_sms, stream, cuda_err)) \
            : ((p.dbias != nullptr) ? launch_bwd_variant<DD, CC, AA, true, false>(maps, bp, num_sms, stream, cuda_err)  \

@@ -30,16 +30,28 @@ __device__ __forceinline__ float dot_row(const float* __restrict__ a_smem, const
   return s;
 }
 
+// Batch stored without padding: the sequence that owns `row` (largest s with cu[s] <= row).
+__device__ __forceinline__ int seq_of_row_fp32(const int* __restrict__ cu, int n_seqs, int row) {
+  int lo = 0, hi = n_seqs;
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (cu[mid] <= row) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
 // grid (N, B*H); block 128.  Thread t handles key j0 + t, then output column t.
 __global__ void fwd_fp32_kernel(const float* __restrict__ q, const float* __restrict__ k,
                                 const float* __restrict__ v, float* __restrict__ o, int H, int N, int D,
                                 float scale, float bias, int causal, const float* __restrict__ slopes,
                                 const float* __restrict__ bias_vec, int H_kv, int N_k, int off,
-                                const int* __restrict__ seqlens, const float* __restrict__ row_scale) {
+                                const int* __restrict__ seqlens, const float* __restrict__ row_scale,
+                                const int* __restrict__ cu, int n_seqs) {
   __shared__ float sq[128];
   __shared__ float sp[kThreads];
   const int i = blockIdx.x, bh = blockIdx.y, t = threadIdx.x;
-  if (bias_vec) bias = bias_vec[bh];
+  const int sq_id = cu ? seq_of_row_fp32(cu, n_seqs, i) : 0;
+  if (bias_vec) bias = bias_vec[cu ? sq_id * H + bh : bh];
   const size_t base = static_cast<size_t>(bh) * N * D;
   const size_t kv_base = static_cast<size_t>((bh / H) * H_kv + (bh % H) / (H / H_kv)) * N_k * D;
   const float slope = slopes ? slopes[bh % H] : 0.0f;
@@ -47,9 +59,11 @@ __global__ void fwd_fp32_kernel(const float* __restrict__ q, const float* __rest
   __syncthreads();
   // padded batch: keys past the sequence's length carry no weight, rows past it are zero
   const int n_valid = seqlens ? max(0, min(N, seqlens[bh / H])) : N_k;
-  const int jend = (i >= n_valid && seqlens) ? 0 : min(n_valid, causal ? max(0, min(N_k, i + off + 1)) : N_k);
+  int jend = (i >= n_valid && seqlens) ? 0 : min(n_valid, causal ? max(0, min(N_k, i + off + 1)) : N_k);
+  const int jbeg = cu ? cu[sq_id] : 0;          // batch without padding: keys of the row's own sequence only
+  if (cu) jend = min(jend, cu[sq_id + 1]);
   float acc = 0.0f;
-  for (int j0 = 0; j0 < jend; j0 += kThreads) {
+  for (int j0 = jbeg; j0 < jend; j0 += kThreads) {
     const int j = j0 + t;
     float p = 0.0f;
     if (j < jend) {
@@ -75,12 +89,13 @@ __global__ void bwd_dq_fp32_kernel(const float* __restrict__ q, const float* __r
                                    int causal, const float* __restrict__ slopes,
                                    const float* __restrict__ bias_vec, float* __restrict__ dbias, int H_kv,
                                    int N_k, int off, const int* __restrict__ seqlens,
-                                   const float* __restrict__ row_scale) {
+                                   const float* __restrict__ row_scale, const int* __restrict__ cu, int n_seqs) {
   __shared__ float sq[128];
   __shared__ float sdo[128];
   __shared__ float sds[kThreads];
   const int i = blockIdx.x, bh = blockIdx.y, t = threadIdx.x;
-  if (bias_vec) bias = bias_vec[bh];
+  const int sq_id = cu ? seq_of_row_fp32(cu, n_seqs, i) : 0;
+  if (bias_vec) bias = bias_vec[cu ? sq_id * H + bh : bh];
   const size_t kv_base = static_cast<size_t>((bh / H) * H_kv + (bh % H) / (H / H_kv)) * N_k * D;
   float ds_sum = 0.0f;   // this thread's share of sum_j dS_ij
   const size_t base = static_cast<size_t>(bh) * N * D;
@@ -92,9 +107,11 @@ __global__ void bwd_dq_fp32_kernel(const float* __restrict__ q, const float* __r
   }
   __syncthreads();
   const int n_valid = seqlens ? max(0, min(N, seqlens[bh / H])) : N_k;
-  const int jend = (i >= n_valid && seqlens) ? 0 : min(n_valid, causal ? max(0, min(N_k, i + off + 1)) : N_k);
+  int jend = (i >= n_valid && seqlens) ? 0 : min(n_valid, causal ? max(0, min(N_k, i + off + 1)) : N_k);
+  const int jbeg = cu ? cu[sq_id] : 0;
+  if (cu) jend = min(jend, cu[sq_id + 1]);
   float acc = 0.0f;
-  for (int j0 = 0; j0 < jend; j0 += kThreads) {
+  for (int j0 = jbeg; j0 < jend; j0 += kThreads) {
     const int j = j0 + t;
     float ds = 0.0f;
     if (j < jend) {
@@ -120,7 +137,7 @@ __global__ void bwd_dq_fp32_kernel(const float* __restrict__ q, const float* __r
       if (t < half) sds[t] += sds[t + half];
       __syncthreads();
     }
-    if (t == 0) atomicAdd(dbias + bh, sds[0]);
+    if (t == 0) atomicAdd(dbias + (cu ? sq_id * H + bh : bh), sds[0]);
   }
 }
 
@@ -131,7 +148,8 @@ __global__ void bwd_dkdv_fp32_kernel(const float* __restrict__ q, const float* _
                                      float* __restrict__ dk, float* __restrict__ dv, int H, int N, int D,
                                      float scale, float bias_scalar, int causal, const float* __restrict__ slopes,
                                      const float* __restrict__ bias_vec, int H_kv, int N_k, int off,
-                                     const int* __restrict__ seqlens, const float* __restrict__ row_scale) {
+                                     const int* __restrict__ seqlens, const float* __restrict__ row_scale,
+                                     const int* __restrict__ cu, int n_seqs) {
   __shared__ float sk[128];
   __shared__ float sv[128];
   __shared__ float sp[kThreads];
@@ -146,14 +164,19 @@ __global__ void bwd_dkdv_fp32_kernel(const float* __restrict__ q, const float* _
   __syncthreads();
   // padded batch: a key past the sequence's length gets zero gradients, queries past it do not count
   const int n_valid = seqlens ? max(0, min(N, seqlens[bh_kv / H_kv])) : N;
-  const int ibeg = (seqlens && j >= n_valid) ? N : (causal ? max(0, j - off) : 0);
-  const int iend = n_valid;
+  int ibeg = (seqlens && j >= n_valid) ? N : (causal ? max(0, j - off) : 0);
+  int iend = n_valid;
+  const int sq_id = cu ? seq_of_row_fp32(cu, n_seqs, j) : 0;
+  if (cu) {   // batch without padding: queries of the key's own sequence only
+    ibeg = max(ibeg, cu[sq_id]);
+    iend = cu[sq_id + 1];
+  }
   float acc_k = 0.0f, acc_v = 0.0f;
   for (int g = 0; g < group; ++g) {
     const int bh = (bh_kv / H_kv) * H + (bh_kv % H_kv) * group + g;   // query head
     const size_t base = static_cast<size_t>(bh) * N * D;
     const float slope = slopes ? slopes[bh % H] : 0.0f;
-    const float bias = bias_vec ? bias_vec[bh] : bias_scalar;
+    const float bias = bias_vec ? bias_vec[cu ? sq_id * H + bh : bh] : bias_scalar;
     for (int i0 = ibeg; i0 < iend; i0 += kThreads) {
       const int i = i0 + t;
       float p = 0.0f, ds = 0.0f;
@@ -209,7 +232,7 @@ int launch_fwd_fp32(const float* q, const float* k, const float* v, float* o, co
   dim3 grid(p.N, p.B * p.H);
   fwd_fp32_kernel<<<grid, kThreads, 0, stream>>>(q, k, v, o, p.H, p.N, p.D, p.scale, p.bias, p.causal, p.slopes,
                                                  p.bias_vec, p.kv_heads(), p.key_rows(), p.query_pos0(), p.seqlens,
-                                                 p.row_scale);
+                                                 p.row_scale, p.cu_seqlens, p.n_seqs);
   *launches += 1;
   *cuda_err = cudaGetLastError();
   return *cuda_err == cudaSuccess ? SIGATTN_OK : SIGATTN_ERR_CUDA;
@@ -220,16 +243,18 @@ int launch_bwd_fp32(const float* q, const float* k, const float* v, const float*
                     cudaError_t* cuda_err) {
   dim3 grid(p.N, p.B * p.H);
   if (p.dbias) {
-    *cuda_err = cudaMemsetAsync(p.dbias, 0, static_cast<size_t>(p.B) * p.H * sizeof(float), stream);
+    const size_t n_bias = p.cu_seqlens ? static_cast<size_t>(p.n_seqs) * p.H : static_cast<size_t>(p.B) * p.H;
+    *cuda_err = cudaMemsetAsync(p.dbias, 0, n_bias * sizeof(float), stream);
     if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
   }
   bwd_dq_fp32_kernel<<<grid, kThreads, 0, stream>>>(q, k, v, d_o, dq, p.H, p.N, p.D, p.scale, p.bias, p.causal,
                                                     p.slopes, p.bias_vec, p.dbias, p.kv_heads(), p.key_rows(), p.query_pos0(),
-                                                    p.seqlens, p.row_scale);
+                                                    p.seqlens, p.row_scale, p.cu_seqlens, p.n_seqs);
   dim3 grid_kv(p.key_rows(), p.B * p.kv_heads());
   bwd_dkdv_fp32_kernel<<<grid_kv, kThreads, 0, stream>>>(q, k, v, d_o, dk, dv, p.H, p.N, p.D, p.scale, p.bias,
                                                          p.causal, p.slopes, p.bias_vec, p.kv_heads(), p.key_rows(),
-                                                         p.query_pos0(), p.seqlens, p.row_scale);
+                                                         p.query_pos0(), p.seqlens, p.row_scale, p.cu_seqlens,
+                                                         p.n_seqs);
   *launches += 2;
   *cuda_err = cudaGetLastError();
   return *cuda_err == cudaSuccess ? SIGATTN_OK : SIGATTN_ERR_CUDA;

@@ -94,6 +94,10 @@ struct FwdParams {
   int pack_rows, pack_group;
   const int* seqlens;   // padded batch: valid length per batch entry (keys and queries), or nullptr
   const float* row_scale;   // one factor per query row applied to O, or nullptr
+  // Batch stored without padding (B = 1): sequence s owns rows [cu_seqlens[s], cu_seqlens[s + 1]) of
+  // Q, K and V and attends only within them; bias_vec then holds one bias per (sequence, head).
+  const int* cu_seqlens;    // n_seqs + 1 row offsets, or nullptr
+  int n_seqs;
   int n_pairs;     // ceil(N / 256)
   int n_kv_total;  // ceil(N / 128)
   // Keys split over several work items (packed mode only; decoding has too few (batch, head)
@@ -128,6 +132,17 @@ __device__ __forceinline__ int snake_rank(int round, int n_items) {
 
 __device__ __forceinline__ int num_rounds(int n_items) { return (n_items + gridDim.x - 1) / gridDim.x; }
 
+// Sequence that owns `row` in a batch stored without padding: the largest s with cu[s] <= row
+// (0 <= row < cu[n_seqs]; empty sequences own no row).
+__device__ __forceinline__ int seq_of_row(const int* __restrict__ cu, int n_seqs, int row) {
+  int lo = 0, hi = n_seqs;   // cu[lo] <= row < cu[hi]
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (__ldg(cu + mid) <= row) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
 template <bool CAUSAL>
 __device__ __forceinline__ Item decode_item(const FwdParams& p, int item) {
   Item w;
@@ -153,6 +168,21 @@ __device__ __forceinline__ Item decode_item(const FwdParams& p, int item) {
     if (p.seqlens && r < p.N && r >= w.n_valid) w.n[t] = 1;
   }
   w.j0 = 0;
+  if (p.cu_seqlens != nullptr) {
+    // Batch without padding: a tile's rows see keys from the start of its first row's sequence to
+    // the end of its last row's sequence (causal: to its last row).  Both tiles of the item walk
+    // the same key tiles, starting where tile 0's keys start; what lies outside a row's own
+    // sequence is masked row by row.
+    w.j0 = __ldg(p.cu_seqlens + seq_of_row(p.cu_seqlens, p.n_seqs, w.row0)) / kBN;
+#pragma unroll
+    for (int t = 0; t < 2; ++t) {
+      const int r_first = w.row0 + t * kBM;
+      if (r_first >= p.N) { w.n[t] = 0; continue; }
+      const int r_last = min(p.N, r_first + kBM) - 1;
+      const int key_end = CAUSAL ? r_last + 1 : __ldg(p.cu_seqlens + seq_of_row(p.cu_seqlens, p.n_seqs, r_last) + 1);
+      w.n[t] = (key_end + kBN - 1) / kBN - w.j0;
+    }
+  }
   if (p.n_splits > 1) {   // packed mode: every valid tile visits all key tiles; this item takes its share
     w.j0 = split * p.tiles_per_split;
     const int n = min(p.tiles_per_split, p.n_kv_total - w.j0);
@@ -338,10 +368,10 @@ __device__ __forceinline__ void tmem_st_cols(uint32_t addr, uint32_t (&v)[N]) {
 
 // kCols logits of one row (32-column TMEM loads) -> kCols / 2 packed bf16x2 sigmoid values.
 //   a = s * scale_log2e + c0   (c0 carries the bias and, with ALiBi, the position term)
-template <bool ALIBI, int EMULATE_EVERY>
+template <bool ALIBI, int EMULATE_EVERY, bool TWO_SIDED = false>
 __device__ __forceinline__ void sigmoid_cols(const uint32_t (&s)[kCols], uint32_t (&out)[kCols / 2],
                                              float scale_log2e, float bias_log2e, float slope_log2e, float row_rel,
-                                             int col_base, bool masked, float mask_limit) {
+                                             int col_base, bool masked, float mask_limit, float mask_first = 0.0f) {
   float a[kCols];
 #pragma unroll
   for (int i = 0; i < kCols; ++i) {
@@ -357,7 +387,9 @@ __device__ __forceinline__ void sigmoid_cols(const uint32_t (&s)[kCols], uint32_
   if (masked) {  // keys after the query (and, in a padded batch, past the sequence's end) get weight 0
 #pragma unroll
     for (int i = 0; i < kCols; ++i)
-      if (static_cast<float>(col_base + i) > mask_limit) pr[i] = 0.0f;
+      if (static_cast<float>(col_base + i) > mask_limit ||
+          (TWO_SIDED && static_cast<float>(col_base + i) < mask_first))   // keys before the row's own sequence
+        pr[i] = 0.0f;
   }
 #pragma unroll
   for (int i = 0; i < kCols / 2; ++i) out[i] = pack_bf16x2(pr[2 * i], pr[2 * i + 1]);
@@ -376,6 +408,7 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
   using L = FwdSmem<D>;
   constexpr bool PACKED = (MODE == 1), GENERAL = (MODE == 2);
   const bool varlen = GENERAL && p.seqlens != nullptr;
+  const bool ragged = GENERAL && p.cu_seqlens != nullptr;
   const int g = threadIdx.x >> 7;            // column group of the tile
   const int tid = threadIdx.x & 127;         // row of the tile
   const uint32_t lane_off = static_cast<uint32_t>(((threadIdx.x >> 5) & 3) * 32) << 16;
@@ -403,6 +436,22 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
       bias_t[0] = p.bias_vec ? __ldg(p.bias_vec + w.bh) * kLog2e : p.bias_log2e;
       pos_t[0] = static_cast<float>(w.row0 + tid + p.pos0);
     }
+    // Batch without padding: the keys [key_lo, key_hi) this thread's row may see in each tile (its own
+    // sequence, cut at the row itself when causal) and the bias of its sequence and head.
+    int key_lo[2] = {0, 0}, key_hi[2] = {0, 0};
+    if (ragged) {
+#pragma unroll
+      for (int t = 0; t < 2; ++t) {
+        const int r = w.row0 + t * kBM + tid;
+        bias_t[t] = p.bias_log2e;
+        if (r < p.N) {
+          const int sq = seq_of_row(p.cu_seqlens, p.n_seqs, r);
+          key_lo[t] = __ldg(p.cu_seqlens + sq);
+          key_hi[t] = CAUSAL ? r + 1 : __ldg(p.cu_seqlens + sq + 1);
+          if (p.bias_vec) bias_t[t] = __ldg(p.bias_vec + sq * p.H + w.bh) * kLog2e;
+        }
+      }
+    }
 
     // Tile-steps are visited in the order (j, tile 0), (j, tile 1), (j + 1, tile 0), ...
     for (int j = 0; j < w.n_kv; ++j) {
@@ -413,7 +462,7 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
         if (!mbar_wait(smem_u32(&bars->s_full[t]), cnt & 1, cta_err, 30 + t)) return;
         ++cnt;
         tc_fence_after_sync();
-        const int jk = PACKED ? w.j0 + j : j;   // key tile within the sequence (the keys may be split)
+        const int jk = (PACKED || GENERAL) ? w.j0 + j : j;   // key tile (split keys, unpadded batches: items start later)
         // position of this thread's query relative to the first key of the tile
         const float row_rel = (PACKED ? pos_t[t] : pos_t[0] + static_cast<float>(t * kBM)) - static_cast<float>(jk * kBN);
         // the mask cuts through every key tile that reaches beyond the position of the tile's
@@ -435,9 +484,16 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
         tmem_wait_ld();
         uint32_t pk[kCols / 2];
         constexpr int kEmulateEvery = (D == 128) ? SIGATTN_FWD_EMULATE_D128 : SIGATTN_FWD_EMULATE_D64;
-        sigmoid_cols<ALIBI, kEmulateEvery>(sv, pk, p.scale_log2e, bias_t[PACKED ? t : 0], slope_t[PACKED ? t : 0], row_rel,
-                                           g * kCols,
-                                           diag, mask_limit);
+        if (ragged) {
+          const int key0 = jk * kBN;
+          const bool cut = key0 < key_lo[t] || key0 + kBN > key_hi[t];   // not wholly inside the row's range
+          sigmoid_cols<ALIBI, kEmulateEvery, true>(sv, pk, p.scale_log2e, bias_t[t], slope_t[0], row_rel, g * kCols, cut,
+                                                   static_cast<float>(key_hi[t] - 1 - key0),
+                                                   static_cast<float>(key_lo[t] - key0));
+        } else {
+          sigmoid_cols<ALIBI, kEmulateEvery>(sv, pk, p.scale_log2e, bias_t[PACKED ? t : 0], slope_t[PACKED ? t : 0],
+                                             row_rel, g * kCols, diag, mask_limit);
+        }
         tmem_st_cols(tS, pk);
         tmem_wait_st();
         tc_fence_before_sync();
@@ -641,7 +697,8 @@ int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const 
   const int group = p.H / p.kv_heads();
   // Few queries per head and several query heads per key/value head (decoding with grouped
   // heads): pack the group's rows into one sequence so that K and V are streamed once per group.
-  const bool small = static_cast<long long>(p.N) * group <= 2 * kBM && p.seqlens == nullptr && p.row_scale == nullptr;
+  const bool small = static_cast<long long>(p.N) * group <= 2 * kBM && p.seqlens == nullptr &&
+                     p.row_scale == nullptr && p.cu_seqlens == nullptr;
   // With a scratch buffer for fp32 partial sums, the keys of one head may also be split over
   // several work items (decoding: too few (batch, head) pairs for 148 SMs otherwise).
   const int n_kv_tiles = (p.key_rows() + kBN - 1) / kBN;
@@ -685,6 +742,8 @@ int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const 
   fp.slopes = p.slopes;
   fp.seqlens = p.seqlens;
   fp.row_scale = p.row_scale;
+  fp.cu_seqlens = p.cu_seqlens;
+  fp.n_seqs = p.n_seqs;
   fp.status = status;
 
   const size_t n_elems = static_cast<size_t>(BH) * p.N * p.D;
@@ -697,7 +756,7 @@ int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const 
   const bool alibi = p.slopes != nullptr;
 #define SIGATTN_FWD_CASE(DD, CC, AA)                                                                       \
   rc = packed ? launch_fwd_variant<DD, CC, AA, 1>(tmQ, tmK, tmV, tmO, fp, num_sms, stream, cuda_err)       \
-       : (p.seqlens != nullptr || p.row_scale != nullptr || accumulate)                                    \
+       : (p.seqlens != nullptr || p.row_scale != nullptr || p.cu_seqlens != nullptr || accumulate)         \
            ? launch_fwd_variant<DD, CC, AA, 2>(tmQ, tmK, tmV, tmO, fp, num_sms, stream, cuda_err)          \
            : launch_fwd_variant<DD, CC, AA, 0>(tmQ, tmK, tmV, tmO, fp, num_sms, stream, cuda_err)
   if (p.D == 128) {

@@ -28,6 +28,8 @@ struct Problem {
   int acc_only;           // 1: accumulate and stop.  Forward: add the partial O, fp32, into split_ws (never cleared,
                           // never converted; o is not written).  Backward: add the partial dQ into the workspace
                           // (not cleared) and leave dq unwritten.  For key/value shards whose results are summed.
+  const int* cu_seqlens;  // batch stored without padding (B = 1): device pointer to n_seqs + 1 row offsets, or nullptr;
+  int n_seqs;             // bias_vec and dbias then hold one entry per (sequence, head)
 };
 
 // Every launcher enqueues on `stream`, adds the number of kernels it launched to
