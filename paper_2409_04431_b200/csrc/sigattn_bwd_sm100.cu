@@ -107,7 +107,7 @@ __device__ __forceinline__ int bwd_num_rounds(int n_items) { return (n_items + g
 
 // GROUPED = false compiles the plain case (one query head per key/value head, no padded batch)
 // without the head loop and without the per-sequence lengths; it is the benchmarked path.
-// GROUPED = true serves both grouped heads and padded batches.
+// GROUPED = true serves grouped heads, padded batches and batches stored without padding.
 // Sequence that owns `row` in a batch stored without padding: the largest s with cu[s] <= row.
 __device__ __forceinline__ int bwd_seq_of_row(const int* __restrict__ cu, int n_seqs, int row) {
   int lo = 0, hi = n_seqs;   // cu[lo] <= row < cu[hi]
@@ -375,11 +375,13 @@ __device__ __forceinline__ void bwd_store_acc_rows(uint32_t t_acc, uint8_t* stag
   }
 }
 
-template <int D, bool CAUSAL, bool ALIBI, bool DBIAS, bool GROUPED>
+// KIND: 0 plain, 1 general (grouped heads, padded batch), 2 general plus a batch stored without padding
+template <int D, bool CAUSAL, bool ALIBI, bool DBIAS, int KIND>
 __device__ void bwd_act_role(const BwdParams& p, const CUtensorMap* tmDk, const CUtensorMap* tmDv, int wg,
                              uint8_t* smem, uint32_t tmem, BwdBarriers* bars, volatile int* cta_err) {
   using L = BwdSmem<D>;
   using TM = BwdTmem<D>;
+  constexpr bool GROUPED = KIND >= 1;
   const int tid = threadIdx.x & 127;  // key row within the tile
   const uint32_t lane_off = static_cast<uint32_t>(((threadIdx.x >> 5) & 3) * 32) << 16;
   uint32_t step_cnt = 0, item_cnt = 0;
@@ -396,7 +398,7 @@ __device__ void bwd_act_role(const BwdParams& p, const CUtensorMap* tmDk, const 
     float ds_sum = 0.0f;   // this thread's share of sum dS over the head's tiles (the bias gradient)
     // batch without padding: the queries [q_lo, q_hi) that see this thread's key (its own sequence,
     // from the key itself on when causal), and the sequence's bias
-    const bool ragged = GROUPED && p.cu_seqlens != nullptr;
+    constexpr bool ragged = (KIND == 2);
     int q_lo = 0, q_hi = 0, seq = 0;
     if (ragged) {
       const int kr = w.j * kT + tid;
@@ -578,12 +580,13 @@ __device__ void bwd_drain_role(const BwdParams& p, const CUtensorMap* tmW, uint8
 
 // ------------------------------------------------------------------ kernels
 
-template <int D, bool CAUSAL, bool ALIBI, bool DBIAS, bool GROUPED>
+template <int D, bool CAUSAL, bool ALIBI, bool DBIAS, int KIND>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 sigattn_bwd_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                         const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmDo,
                         const __grid_constant__ CUtensorMap tmDk, const __grid_constant__ CUtensorMap tmDv,
                         const __grid_constant__ CUtensorMap tmW, const BwdParams p) {
+  constexpr bool GROUPED = KIND >= 1;
   extern __shared__ uint8_t smem_raw[];
   __shared__ BwdBarriers bars;
   __shared__ uint32_t tmem_base_slot;
@@ -638,7 +641,7 @@ sigattn_bwd_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
     if ((threadIdx.x & 31) == 0) bwd_mma_role<D, CAUSAL, GROUPED>(p, smem_base, tmem, &bars, &cta_err);
     __syncwarp();
   } else if (warp < 8) {
-    bwd_act_role<D, CAUSAL, ALIBI, DBIAS, GROUPED>(p, &tmDk, &tmDv, warp >> 2, smem, tmem, &bars, &cta_err);
+    bwd_act_role<D, CAUSAL, ALIBI, DBIAS, KIND>(p, &tmDk, &tmDv, warp >> 2, smem, tmem, &bars, &cta_err);
   } else {
     bwd_drain_role<D, CAUSAL, GROUPED>(p, &tmW, smem, tmem, &bars, &cta_err);
   }
@@ -683,10 +686,10 @@ sigattn_bwd_scale_rows_kernel(const uint4* __restrict__ d_o, const float* __rest
   }
 }
 
-template <int D, bool CAUSAL, bool ALIBI, bool DBIAS, bool GROUPED>
+template <int D, bool CAUSAL, bool ALIBI, bool DBIAS, int KIND>
 int launch_bwd_variant(const CUtensorMap* maps, const BwdParams& bp, int num_sms, cudaStream_t stream,
                        cudaError_t* cuda_err) {
-  auto kernel = sigattn_bwd_bf16_kernel<D, CAUSAL, ALIBI, DBIAS, GROUPED>;
+  auto kernel = sigattn_bwd_bf16_kernel<D, CAUSAL, ALIBI, DBIAS, KIND>;
   static bool configured = false;
   if (!configured) {
     *cuda_err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<D>::kDynBytes);
@@ -810,14 +813,15 @@ int launch_bwd_bf16(const void* q, const void* k, const void* v, const void* d_o
   int rc;
   const bool alibi = p.slopes != nullptr;
   // the bias gradient costs the activation groups a running sum (4-5 % of the kernel), so it
-  // is compiled in only where it is asked for; likewise the loop over a group's query heads
-  // and the per-sequence lengths
-#define SIGATTN_BWD_CASE(DD, CC, AA)                                                                        \
-  rc = (bp.group > 1 || bp.seqlens != nullptr || bp.cu_seqlens != nullptr)                                  \
-           ? ((p.dbias != nullptr) ? launch_bwd_variant<DD, CC, AA, true, true>(maps, bp, num_sms, stream, cuda_err)   \
-                                   : launch_bwd_variant<DD, CC, AA, false, true>(maps, bp, num_sms, stream, cuda_err)) \
-           : ((p.dbias != nullptr) ? launch_bwd_variant<DD, CC, AA, true, false>(maps, bp, num_sms, stream, cuda_err)  \
-                                   : launch_bwd_variant<DD, CC, AA, false, false>(maps, bp, num_sms, stream, cuda_err))
+  // is compiled in only where it is asked for; likewise the loop over a group's query heads and
+  // the per-sequence lengths (kind 1) and the lookups of a batch without padding (kind 2)
+#define SIGATTN_BWD_KIND(DD, CC, AA, KK)                                                                   \
+  ((p.dbias != nullptr) ? launch_bwd_variant<DD, CC, AA, true, KK>(maps, bp, num_sms, stream, cuda_err)    \
+                        : launch_bwd_variant<DD, CC, AA, false, KK>(maps, bp, num_sms, stream, cuda_err))
+#define SIGATTN_BWD_CASE(DD, CC, AA)                                                                       \
+  rc = (bp.cu_seqlens != nullptr)                  ? SIGATTN_BWD_KIND(DD, CC, AA, 2)                        \
+       : (bp.group > 1 || bp.seqlens != nullptr)   ? SIGATTN_BWD_KIND(DD, CC, AA, 1)                        \
+                                                   : SIGATTN_BWD_KIND(DD, CC, AA, 0)
   if (p.D == 128) {
     if (p.causal) { if (alibi) SIGATTN_BWD_CASE(128, true, true); else SIGATTN_BWD_CASE(128, true, false); }
     else          { if (alibi) SIGATTN_BWD_CASE(128, false, true); else SIGATTN_BWD_CASE(128, false, false); }
@@ -826,6 +830,7 @@ int launch_bwd_bf16(const void* q, const void* k, const void* v, const void* d_o
     else          { if (alibi) SIGATTN_BWD_CASE(64, false, true); else SIGATTN_BWD_CASE(64, false, false); }
   }
 #undef SIGATTN_BWD_CASE
+#undef SIGATTN_BWD_KIND
   if (rc != SIGATTN_OK) return rc;
   if (timed) cudaEventRecord(t_ev_stop, stream);
   *launches += 1;

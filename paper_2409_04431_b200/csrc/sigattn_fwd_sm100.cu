@@ -401,14 +401,15 @@ __device__ __forceinline__ void sigmoid_cols(const uint32_t (&s)[kCols], uint32_
 // P V and the next logits of the other one, so the MUFU pipe and the tensor pipe take turns
 // on a tile instead of competing for it.
 // MODE: 0 plain (the benchmarked path), 1 packed grouped heads, 2 general: padded batch with
-// per-sequence lengths and / or one output factor per query row, each asked for at run time
+// per-sequence lengths, one output factor per query row, accumulation into an fp32 buffer, each
+// asked for at run time; 3 = 2 plus a batch stored without padding (row offsets per sequence)
 template <int D, bool CAUSAL, bool ALIBI, int MODE>
 __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t* smem, uint32_t tmem,
                              FwdBarriers* bars, volatile int* cta_err) {
   using L = FwdSmem<D>;
-  constexpr bool PACKED = (MODE == 1), GENERAL = (MODE == 2);
+  constexpr bool PACKED = (MODE == 1), GENERAL = (MODE >= 2);
   const bool varlen = GENERAL && p.seqlens != nullptr;
-  const bool ragged = GENERAL && p.cu_seqlens != nullptr;
+  constexpr bool ragged = (MODE == 3);
   const int g = threadIdx.x >> 7;            // column group of the tile
   const int tid = threadIdx.x & 127;         // row of the tile
   const uint32_t lane_off = static_cast<uint32_t>(((threadIdx.x >> 5) & 3) * 32) << 16;
@@ -756,7 +757,9 @@ int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const 
   const bool alibi = p.slopes != nullptr;
 #define SIGATTN_FWD_CASE(DD, CC, AA)                                                                       \
   rc = packed ? launch_fwd_variant<DD, CC, AA, 1>(tmQ, tmK, tmV, tmO, fp, num_sms, stream, cuda_err)       \
-       : (p.seqlens != nullptr || p.row_scale != nullptr || p.cu_seqlens != nullptr || accumulate)         \
+       : (p.cu_seqlens != nullptr)                                                                         \
+           ? launch_fwd_variant<DD, CC, AA, 3>(tmQ, tmK, tmV, tmO, fp, num_sms, stream, cuda_err)          \
+       : (p.seqlens != nullptr || p.row_scale != nullptr || accumulate)                                    \
            ? launch_fwd_variant<DD, CC, AA, 2>(tmQ, tmK, tmV, tmO, fp, num_sms, stream, cuda_err)          \
            : launch_fwd_variant<DD, CC, AA, 0>(tmQ, tmK, tmV, tmO, fp, num_sms, stream, cuda_err)
   if (p.D == 128) {
