@@ -140,8 +140,9 @@ __device__ __forceinline__ BwdItem decode_bwd_item(const BwdParams& p, int item)
     const int k_first = w.j * kT, k_last = min(p.N, k_first + kT) - 1;
     const int q_lo = CAUSAL ? k_first : __ldg(p.cu_seqlens + bwd_seq_of_row(p.cu_seqlens, p.n_seqs, k_first));
     const int q_hi = __ldg(p.cu_seqlens + bwd_seq_of_row(p.cu_seqlens, p.n_seqs, k_last) + 1);
-    w.i_begin = q_lo / kT;
-    w.n = (q_hi + kT - 1) / kT - w.i_begin;
+    // (offsets that do not rise from 0 to N give wrong results, but the clamps keep every loop bounded)
+    w.i_begin = max(0, min(p.n_tiles - 1, q_lo / kT));
+    w.n = max(1, min(p.n_tiles, (q_hi + kT - 1) / kT) - w.i_begin);
   }
   w.steps = GROUPED ? p.group * w.n : w.n;
   return w;

@@ -173,14 +173,15 @@ __device__ __forceinline__ Item decode_item(const FwdParams& p, int item) {
     // the end of its last row's sequence (causal: to its last row).  Both tiles of the item walk
     // the same key tiles, starting where tile 0's keys start; what lies outside a row's own
     // sequence is masked row by row.
-    w.j0 = __ldg(p.cu_seqlens + seq_of_row(p.cu_seqlens, p.n_seqs, w.row0)) / kBN;
+    // (offsets that do not rise from 0 to N give wrong results, but the clamps keep every loop bounded)
+    w.j0 = max(0, min(p.n_kv_total - 1, __ldg(p.cu_seqlens + seq_of_row(p.cu_seqlens, p.n_seqs, w.row0)) / kBN));
 #pragma unroll
     for (int t = 0; t < 2; ++t) {
       const int r_first = w.row0 + t * kBM;
       if (r_first >= p.N) { w.n[t] = 0; continue; }
       const int r_last = min(p.N, r_first + kBM) - 1;
       const int key_end = CAUSAL ? r_last + 1 : __ldg(p.cu_seqlens + seq_of_row(p.cu_seqlens, p.n_seqs, r_last) + 1);
-      w.n[t] = (key_end + kBN - 1) / kBN - w.j0;
+      w.n[t] = max(1, min(p.n_kv_total, (key_end + kBN - 1) / kBN) - w.j0);
     }
   }
   if (p.n_splits > 1) {   // packed mode: every valid tile visits all key tiles; this item takes its share
