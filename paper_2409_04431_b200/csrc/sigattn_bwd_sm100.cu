@@ -24,6 +24,8 @@
 // Warp roles (448 threads): warps 0-7 two activation groups (query columns 0-63 and
 // 64-127 of the tile; every thread owns one key row), warps 8-11 dQ drain group,
 // warp 12 TMA producer, warp 13 MMA issuer.
+#include <atomic>
+
 #include "sigattn_internal.h"
 #include "sigattn_activation.cuh"
 #include "sm100_primitives.cuh"
@@ -64,6 +66,10 @@ struct BwdBarriers {
   uint64_t p_ready, ds_ready;
   uint64_t dq_full, dq_empty;
   uint64_t dkv_full, dkv_empty;
+  // dynamic schedule (batches without padding): the TMA thread draws the next work item from a
+  // global counter and hands it to the other roles through this two-slot ring
+  uint64_t sched_full[2], sched_empty[2];
+  int sched_item[2];
 };
 
 struct BwdParams {
@@ -77,6 +83,7 @@ struct BwdParams {
   // bias_vec and dbias then hold one entry per (sequence, head)
   const int* cu_seqlens;
   int n_seqs;
+  int* sched_counter;   // dynamic schedule: next work item to hand out (zero at launch), or nullptr
   int n_items;
   float scale, scale_log2e, bias_log2e;
   const float* bias_vec;   // one bias per (batch, head) instead of the scalar, or nullptr
@@ -104,6 +111,31 @@ __device__ __forceinline__ int bwd_snake_rank(int round, int n_items) {
 }
 
 __device__ __forceinline__ int bwd_num_rounds(int n_items) { return (n_items + gridDim.x - 1) / gridDim.x; }
+
+// Dynamic schedule for batches without padding, where an item's cost follows the position of its
+// key tile inside its own sequence and the static order above no longer sorts by cost: the CTAs
+// draw items from a global counter in key-tile order (every sequence hands out its expensive key
+// tiles first).  One thread per CTA draws; the MMA thread, the activation groups and the drain
+// group read the item from a two-slot ring.  false: a bounded wait expired; *item < 0: none left.
+constexpr int kBwdSchedConsumers = 1 + 256 + 128;
+__device__ __forceinline__ bool bwd_sched_draw(const BwdParams& p, BwdBarriers* bars, int round, int* item,
+                                               volatile int* cta_err) {
+  const uint32_t slot = round & 1, phase = (round >> 1) & 1;
+  if (!mbar_wait(smem_u32(&bars->sched_empty[slot]), phase ^ 1, cta_err, 70)) return false;
+  int it = atomicAdd(p.sched_counter, 1);
+  if (it >= p.n_items) it = -1;
+  *reinterpret_cast<volatile int*>(&bars->sched_item[slot]) = it;
+  mbar_arrive(smem_u32(&bars->sched_full[slot]));
+  *item = it;
+  return true;
+}
+__device__ __forceinline__ bool bwd_sched_take(BwdBarriers* bars, int round, int* item, volatile int* cta_err) {
+  const uint32_t slot = round & 1, phase = (round >> 1) & 1;
+  if (!mbar_wait(smem_u32(&bars->sched_full[slot]), phase, cta_err, 71)) return false;
+  *item = *reinterpret_cast<volatile int*>(&bars->sched_item[slot]);
+  mbar_arrive(smem_u32(&bars->sched_empty[slot]));
+  return true;
+}
 
 // GROUPED = false compiles the plain case (one query head per key/value head, no padded batch)
 // without the head loop and without the per-sequence lengths; it is the benchmarked path.
@@ -159,7 +191,7 @@ struct BwdTmem {
 
 // ------------------------------------------------------------------ producer
 
-template <int D, bool CAUSAL, bool GROUPED>
+template <int D, bool CAUSAL, bool GROUPED, bool DYNAMIC>
 __device__ void bwd_load_role(const BwdParams& p, const CUtensorMap* tmQ, const CUtensorMap* tmK,
                               const CUtensorMap* tmV, const CUtensorMap* tmDo, uint32_t smem_base,
                               BwdBarriers* bars, volatile int* cta_err) {
@@ -186,9 +218,15 @@ __device__ void bwd_load_role(const BwdParams& p, const CUtensorMap* tmQ, const 
     ++do_cnt;
     return true;
   };
-  for (int round = 0, rounds = bwd_num_rounds(p.n_items); round < rounds; ++round) {
-    const int item = bwd_snake_rank(round, p.n_items);
-    if (item < 0) continue;
+  for (int round = 0, rounds = bwd_num_rounds(p.n_items); DYNAMIC || round < rounds; ++round) {
+    int item;
+    if (DYNAMIC) {
+      if (!bwd_sched_draw(p, bars, round, &item, cta_err)) return;
+      if (item < 0) break;
+    } else {
+      item = bwd_snake_rank(round, p.n_items);
+      if (item < 0) continue;
+    }
     const BwdItem w = decode_bwd_item<CAUSAL, GROUPED>(p, item);
     if (!load_q(w.i_begin, w.bh_q0)) return;
     if (!load_do(w.i_begin, w.bh_q0)) return;
@@ -211,7 +249,7 @@ __device__ void bwd_load_role(const BwdParams& p, const CUtensorMap* tmQ, const 
 
 // ------------------------------------------------------------------ MMA issuer
 
-template <int D, bool CAUSAL, bool GROUPED>
+template <int D, bool CAUSAL, bool GROUPED, bool DYNAMIC>
 __device__ void bwd_mma_role(const BwdParams& p, uint32_t smem_base, uint32_t tmem, BwdBarriers* bars,
                              volatile int* cta_err) {
   using L = BwdSmem<D>;
@@ -243,9 +281,15 @@ __device__ void bwd_mma_role(const BwdParams& p, uint32_t smem_base, uint32_t tm
   const uint64_t dQ_mn[2] = {make_smem_desc_sw128(smem_base + L::kQOff, L::kPanelBytes, 1024),
                              make_smem_desc_sw128(smem_base + L::kQOff + L::kTileBytes, L::kPanelBytes, 1024)};
 
-  for (int round = 0, rounds = bwd_num_rounds(p.n_items); round < rounds; ++round) {
-    const int item = bwd_snake_rank(round, p.n_items);
-    if (item < 0) continue;
+  for (int round = 0, rounds = bwd_num_rounds(p.n_items); DYNAMIC || round < rounds; ++round) {
+    int item;
+    if (DYNAMIC) {
+      if (!bwd_sched_take(bars, round, &item, cta_err)) return;
+      if (item < 0) break;
+    } else {
+      item = bwd_snake_rank(round, p.n_items);
+      if (item < 0) continue;
+    }
     const BwdItem w = decode_bwd_item<CAUSAL, GROUPED>(p, item);
     if (!mbar_wait(smem_u32(&bars->kv_full), item_cnt & 1, cta_err, 50)) return;
 
@@ -382,14 +426,20 @@ __device__ void bwd_act_role(const BwdParams& p, const CUtensorMap* tmDk, const 
                              uint8_t* smem, uint32_t tmem, BwdBarriers* bars, volatile int* cta_err) {
   using L = BwdSmem<D>;
   using TM = BwdTmem<D>;
-  constexpr bool GROUPED = KIND >= 1;
+  constexpr bool GROUPED = KIND >= 1, DYNAMIC = KIND == 2;
   const int tid = threadIdx.x & 127;  // key row within the tile
   const uint32_t lane_off = static_cast<uint32_t>(((threadIdx.x >> 5) & 3) * 32) << 16;
   uint32_t step_cnt = 0, item_cnt = 0;
 
-  for (int round = 0, rounds = bwd_num_rounds(p.n_items); round < rounds; ++round) {
-    const int item = bwd_snake_rank(round, p.n_items);
-    if (item < 0) continue;
+  for (int round = 0, rounds = bwd_num_rounds(p.n_items); DYNAMIC || round < rounds; ++round) {
+    int item;
+    if (DYNAMIC) {
+      if (!bwd_sched_take(bars, round, &item, cta_err)) return;
+      if (item < 0) break;
+    } else {
+      item = bwd_snake_rank(round, p.n_items);
+      if (item < 0) continue;
+    }
     const BwdItem w = decode_bwd_item<CAUSAL, GROUPED>(p, item);
     for (int g = 0; g < (GROUPED ? p.group : 1); ++g) {   // the query heads that read this key/value head
     const int bh_q = w.bh_q0 + g;
@@ -524,7 +574,7 @@ __device__ void bwd_act_role(const BwdParams& p, const CUtensorMap* tmDk, const 
 
 // ------------------------------------------------------------------ dQ drain group
 
-template <int D, bool CAUSAL, bool GROUPED>
+template <int D, bool CAUSAL, bool GROUPED, bool DYNAMIC>
 __device__ void bwd_drain_role(const BwdParams& p, const CUtensorMap* tmW, uint8_t* smem, uint32_t tmem,
                                BwdBarriers* bars, volatile int* cta_err) {
   using L = BwdSmem<D>;
@@ -532,9 +582,15 @@ __device__ void bwd_drain_role(const BwdParams& p, const CUtensorMap* tmW, uint8
   const int tid = threadIdx.x & 127;  // query row within the tile
   const uint32_t lane_off = static_cast<uint32_t>(((threadIdx.x >> 5) & 3) * 32) << 16;
   uint32_t step_cnt = 0;
-  for (int round = 0, rounds = bwd_num_rounds(p.n_items); round < rounds; ++round) {
-    const int item = bwd_snake_rank(round, p.n_items);
-    if (item < 0) continue;
+  for (int round = 0, rounds = bwd_num_rounds(p.n_items); DYNAMIC || round < rounds; ++round) {
+    int item;
+    if (DYNAMIC) {
+      if (!bwd_sched_take(bars, round, &item, cta_err)) return;
+      if (item < 0) break;
+    } else {
+      item = bwd_snake_rank(round, p.n_items);
+      if (item < 0) continue;
+    }
     const BwdItem w = decode_bwd_item<CAUSAL, GROUPED>(p, item);
     for (int s = 0; s < w.steps; ++s) {
       const int g = GROUPED ? s / w.n : 0, it = s - g * w.n;   // query head within the group, query tile
@@ -615,6 +671,10 @@ sigattn_bwd_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
     mbar_init(smem_u32(&bars.dq_empty), 128);
     mbar_init(smem_u32(&bars.dkv_full), 1);
     mbar_init(smem_u32(&bars.dkv_empty), 256);
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(smem_u32(&bars.sched_full[s]), 1);
+      mbar_init(smem_u32(&bars.sched_empty[s]), kBwdSchedConsumers);
+    }
     fence_mbar_init();
   }
   if (warp == kBwdLoadWarp && elect_one()) {
@@ -636,15 +696,15 @@ sigattn_bwd_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
   const uint32_t tmem = tmem_base_slot;
 
   if (warp == kBwdLoadWarp) {
-    if ((threadIdx.x & 31) == 0) bwd_load_role<D, CAUSAL, GROUPED>(p, &tmQ, &tmK, &tmV, &tmDo, smem_base, &bars, &cta_err);
+    if ((threadIdx.x & 31) == 0) bwd_load_role<D, CAUSAL, GROUPED, KIND == 2>(p, &tmQ, &tmK, &tmV, &tmDo, smem_base, &bars, &cta_err);
     __syncwarp();
   } else if (warp == kBwdMmaWarp) {
-    if ((threadIdx.x & 31) == 0) bwd_mma_role<D, CAUSAL, GROUPED>(p, smem_base, tmem, &bars, &cta_err);
+    if ((threadIdx.x & 31) == 0) bwd_mma_role<D, CAUSAL, GROUPED, KIND == 2>(p, smem_base, tmem, &bars, &cta_err);
     __syncwarp();
   } else if (warp < 8) {
     bwd_act_role<D, CAUSAL, ALIBI, DBIAS, KIND>(p, &tmDk, &tmDv, warp >> 2, smem, tmem, &bars, &cta_err);
   } else {
-    bwd_drain_role<D, CAUSAL, GROUPED>(p, &tmW, smem, tmem, &bars, &cta_err);
+    bwd_drain_role<D, CAUSAL, GROUPED, KIND == 2>(p, &tmW, smem, tmem, &bars, &cta_err);
   }
 
   tc_fence_before_sync();
@@ -686,6 +746,10 @@ sigattn_bwd_scale_rows_kernel(const uint4* __restrict__ d_o, const float* __rest
     out[i] = make_uint4(scale_bf16x2(x.x, r), scale_bf16x2(x.y, r), scale_bf16x2(x.z, r), scale_bf16x2(x.w, r));
   }
 }
+
+// Work-item counters of the dynamic schedule: one per launch in flight, handed out round robin.
+constexpr int kBwdSchedSlots = 64;
+__device__ int g_bwd_sched_counters[kBwdSchedSlots];
 
 template <int D, bool CAUSAL, bool ALIBI, bool DBIAS, int KIND>
 int launch_bwd_variant(const CUtensorMap* maps, const BwdParams& bp, int num_sms, cudaStream_t stream,
@@ -783,6 +847,7 @@ int launch_bwd_bf16(const void* q, const void* k, const void* v, const void* d_o
   bp.seqlens = p.seqlens;
   bp.cu_seqlens = p.cu_seqlens;
   bp.n_seqs = p.n_seqs;
+  bp.sched_counter = nullptr;
   bp.status = status;
 
   const size_t n_elems = static_cast<size_t>(BH) * p.N * p.D;
@@ -798,6 +863,15 @@ int launch_bwd_bf16(const void* q, const void* k, const void* v, const void* d_o
     if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
   }
 
+  if (p.cu_seqlens != nullptr) {
+    static std::atomic<unsigned> next_slot{0};
+    int* counters = nullptr;
+    *cuda_err = cudaGetSymbolAddress(reinterpret_cast<void**>(&counters), g_bwd_sched_counters);
+    if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
+    bp.sched_counter = counters + next_slot.fetch_add(1) % kBwdSchedSlots;
+    *cuda_err = cudaMemsetAsync(bp.sched_counter, 0, sizeof(int), stream);
+    if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
+  }
   if (p.row_scale != nullptr) {
     const size_t n_vec8 = n_elems / 8;
     const size_t want = n_vec8 / 256 + 1, cap = static_cast<size_t>(num_sms) * 8;

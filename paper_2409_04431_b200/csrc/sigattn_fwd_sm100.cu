@@ -25,6 +25,8 @@
 // Activation: P = u / (1 + u) with u = 2^(log2(e) x), one MUFU op per element in the
 // common case; see sigattn_activation.cuh for the evaluation and for why the paper's
 // tanh form is not used.
+#include <atomic>
+
 #include "sigattn_internal.h"
 #include "sigattn_activation.cuh"
 #include "sm100_primitives.cuh"
@@ -79,6 +81,10 @@ struct FwdBarriers {
   uint64_t s_full[2], p_full[2];
   uint64_t o_full[2], o_empty[2];
   uint64_t kv_full[8], kv_empty[8];
+  // dynamic schedule (batches without padding): the TMA thread draws the next work item from a
+  // global counter and hands it to the other roles through this two-slot ring
+  uint64_t sched_full[2], sched_empty[2];
+  int sched_item[2];
 };
 
 struct FwdParams {
@@ -98,6 +104,7 @@ struct FwdParams {
   // Q, K and V and attends only within them; bias_vec then holds one bias per (sequence, head).
   const int* cu_seqlens;    // n_seqs + 1 row offsets, or nullptr
   int n_seqs;
+  int* sched_counter;       // dynamic schedule: next work item to hand out (zero at launch), or nullptr
   int n_pairs;     // ceil(N / 256)
   int n_kv_total;  // ceil(N / 128)
   // Keys split over several work items (packed mode only; decoding has too few (batch, head)
@@ -131,6 +138,33 @@ __device__ __forceinline__ int snake_rank(int round, int n_items) {
 }
 
 __device__ __forceinline__ int num_rounds(int n_items) { return (n_items + gridDim.x - 1) / gridDim.x; }
+
+// Dynamic schedule.  The static snake order balances the CTAs only if the items' costs fall with
+// their rank; in a batch without padding the cost of a causal item follows its position inside its
+// own sequence, a sawtooth over the rows.  There the CTAs draw items from a global counter instead,
+// in row order from the last row down (every sequence then hands out its expensive items first,
+// and the cheap starts of the first sequences come last).  One thread per CTA draws; the other
+// roles read the item from a two-slot ring in shared memory.  Returns false when a bounded wait
+// expired; *item < 0 means no items are left.
+constexpr int kSchedConsumers = 32 + kActThreads;   // the MMA warp and the activation threads
+__device__ __forceinline__ bool sched_draw(const FwdParams& p, FwdBarriers* bars, int round, int* item,
+                                           volatile int* cta_err) {
+  const uint32_t slot = round & 1, phase = (round >> 1) & 1;
+  if (!mbar_wait(smem_u32(&bars->sched_empty[slot]), phase ^ 1, cta_err, 40)) return false;
+  int it = atomicAdd(p.sched_counter, 1);
+  if (it >= p.n_items) it = -1;
+  *reinterpret_cast<volatile int*>(&bars->sched_item[slot]) = it;
+  mbar_arrive(smem_u32(&bars->sched_full[slot]));
+  *item = it;
+  return true;
+}
+__device__ __forceinline__ bool sched_take(FwdBarriers* bars, int round, int* item, volatile int* cta_err) {
+  const uint32_t slot = round & 1, phase = (round >> 1) & 1;
+  if (!mbar_wait(smem_u32(&bars->sched_full[slot]), phase, cta_err, 41)) return false;
+  *item = *reinterpret_cast<volatile int*>(&bars->sched_item[slot]);
+  mbar_arrive(smem_u32(&bars->sched_empty[slot]));
+  return true;
+}
 
 // Sequence that owns `row` in a batch stored without padding: the largest s with cu[s] <= row
 // (0 <= row < cu[n_seqs]; empty sequences own no row).
@@ -196,15 +230,21 @@ __device__ __forceinline__ Item decode_item(const FwdParams& p, int item) {
 
 // ------------------------------------------------------------------ producer
 
-template <int D, bool CAUSAL>
+template <int D, bool CAUSAL, bool DYNAMIC>
 __device__ void fwd_load_role(const FwdParams& p, const CUtensorMap* tmQ, const CUtensorMap* tmK,
                               const CUtensorMap* tmV, uint32_t smem_base, FwdBarriers* bars, volatile int* cta_err) {
   using L = FwdSmem<D>;
   uint32_t kv_cnt = 0;
   uint32_t q_iter[2] = {0, 0};
-  for (int round = 0, rounds = num_rounds(p.n_items); round < rounds; ++round) {
-    const int item = snake_rank(round, p.n_items);
-    if (item < 0) continue;
+  for (int round = 0, rounds = num_rounds(p.n_items); DYNAMIC || round < rounds; ++round) {
+    int item;
+    if (DYNAMIC) {
+      if (!sched_draw(p, bars, round, &item, cta_err)) return;
+      if (item < 0) break;
+    } else {
+      item = snake_rank(round, p.n_items);
+      if (item < 0) continue;
+    }
     const Item w = decode_item<CAUSAL>(p, item);
     const int bh_kv = (w.bh / p.H) * p.H_kv + (w.bh % p.H) / p.group;   // the key/value head this query head reads
     auto load_q = [&](int t) -> bool {
@@ -244,7 +284,7 @@ __device__ void fwd_load_role(const FwdParams& p, const CUtensorMap* tmQ, const 
 
 // ------------------------------------------------------------------ MMA issuer
 
-template <int D, bool CAUSAL>
+template <int D, bool CAUSAL, bool DYNAMIC>
 __device__ void fwd_mma_role(const FwdParams& p, uint32_t smem_base, uint32_t tmem, FwdBarriers* bars,
                              volatile int* cta_err) {
   using L = FwdSmem<D>;
@@ -287,9 +327,15 @@ __device__ void fwd_mma_role(const FwdParams& p, uint32_t smem_base, uint32_t tm
   auto kv_addr = [&](uint32_t cnt) { return smem_base + L::kKvOff + (cnt % L::kStages) * L::kTileBytes; };
   auto kv_release = [&](uint32_t cnt) { umma_commit_warp(leader, smem_u32(&bars->kv_empty[cnt % L::kStages])); };
 
-  for (int round = 0, rounds = num_rounds(p.n_items); round < rounds; ++round) {
-    const int item = snake_rank(round, p.n_items);
-    if (item < 0) continue;
+  for (int round = 0, rounds = num_rounds(p.n_items); DYNAMIC || round < rounds; ++round) {
+    int item;
+    if (DYNAMIC) {
+      if (!sched_take(bars, round, &item, cta_err)) return;
+      if (item < 0) break;
+    } else {
+      item = snake_rank(round, p.n_items);
+      if (item < 0) continue;
+    }
     const Item w = decode_item<CAUSAL>(p, item);
     // ring positions: K_j at kv_cnt + 2 j (j > 0: 2 j), V_j right after K_j ... order K0 V0 K1 V1 ...
     const uint32_t base_cnt = kv_cnt;
@@ -416,9 +462,16 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
   const uint32_t lane_off = static_cast<uint32_t>(((threadIdx.x >> 5) & 3) * 32) << 16;
   uint32_t s_cnt0 = 0, s_cnt1 = 0, it[2] = {0, 0};
 
-  for (int round = 0, rounds = num_rounds(p.n_items); round < rounds; ++round) {
-    const int item = snake_rank(round, p.n_items);
-    if (item < 0) continue;
+  constexpr bool DYNAMIC = (MODE == 3);
+  for (int round = 0, rounds = num_rounds(p.n_items); DYNAMIC || round < rounds; ++round) {
+    int item;
+    if (DYNAMIC) {
+      if (!sched_take(bars, round, &item, cta_err)) return;
+      if (item < 0) break;
+    } else {
+      item = snake_rank(round, p.n_items);
+      if (item < 0) continue;
+    }
     const Item w = decode_item<CAUSAL>(p, item);
     // Slope, bias and the position of this thread's query row: per item, or with packed heads
     // per row and tile (index 1 of the arrays is only used then).
@@ -605,6 +658,10 @@ sigattn_fwd_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
       mbar_init(smem_u32(&bars.kv_full[s]), 1);
       mbar_init(smem_u32(&bars.kv_empty[s]), 1);
     }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(smem_u32(&bars.sched_full[s]), 1);
+      mbar_init(smem_u32(&bars.sched_empty[s]), kSchedConsumers);
+    }
     fence_mbar_init();
   }
   if (warp == kLoadWarp && elect_one()) {
@@ -623,10 +680,10 @@ sigattn_fwd_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
   const uint32_t tmem = tmem_base_slot;
 
   if (warp == kLoadWarp) {
-    if ((threadIdx.x & 31) == 0) fwd_load_role<D, CAUSAL>(p, &tmQ, &tmK, &tmV, smem_base, &bars, &cta_err);
+    if ((threadIdx.x & 31) == 0) fwd_load_role<D, CAUSAL, MODE == 3>(p, &tmQ, &tmK, &tmV, smem_base, &bars, &cta_err);
     __syncwarp();
   } else if (warp == kMmaWarp) {
-    fwd_mma_role<D, CAUSAL>(p, smem_base, tmem, &bars, &cta_err);
+    fwd_mma_role<D, CAUSAL, MODE == 3>(p, smem_base, tmem, &bars, &cta_err);
     __syncwarp();
   } else {
     fwd_act_role<D, CAUSAL, ALIBI, MODE>(p, &tmO, smem, tmem, &bars, &cta_err);
@@ -667,6 +724,11 @@ int choose_key_splits(int base_items, int n_kv, int num_sms) {
   }
   return best;
 }
+
+// Work-item counters of the dynamic schedule: one per launch in flight, handed out round robin
+// (64 launches may overlap on different streams before two of them share a counter).
+constexpr int kSchedSlots = 64;
+__device__ int g_fwd_sched_counters[kSchedSlots];
 
 template <int D, bool CAUSAL, bool ALIBI, int MODE>
 int launch_fwd_variant(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtensorMap& tmO,
@@ -748,6 +810,16 @@ int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const 
   fp.n_seqs = p.n_seqs;
   fp.status = status;
 
+  fp.sched_counter = nullptr;
+  if (p.cu_seqlens != nullptr) {
+    static std::atomic<unsigned> next_slot{0};
+    int* counters = nullptr;
+    *cuda_err = cudaGetSymbolAddress(reinterpret_cast<void**>(&counters), g_fwd_sched_counters);
+    if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
+    fp.sched_counter = counters + next_slot.fetch_add(1) % kSchedSlots;
+    *cuda_err = cudaMemsetAsync(fp.sched_counter, 0, sizeof(int), stream);
+    if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
+  }
   const size_t n_elems = static_cast<size_t>(BH) * p.N * p.D;
   if (accumulate && !p.acc_only) {
     *cuda_err = cudaMemsetAsync(p.split_ws, 0, n_elems * sizeof(float), stream);
