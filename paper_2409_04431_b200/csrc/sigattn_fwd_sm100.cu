@@ -140,10 +140,11 @@ __device__ __forceinline__ int snake_rank(int round, int n_items) {
 __device__ __forceinline__ int num_rounds(int n_items) { return (n_items + gridDim.x - 1) / gridDim.x; }
 
 // Dynamic schedule.  The static snake order balances the CTAs only if the items' costs fall with
-// their rank; in a batch without padding the cost of a causal item follows its position inside its
-// own sequence, a sawtooth over the rows.  There the CTAs draw items from a global counter instead,
-// in row order from the last row down (every sequence then hands out its expensive items first,
-// and the cheap starts of the first sequences come last).  One thread per CTA draws; the other
+// their rank.  In a padded batch the cost of an item also depends on the length of its sequence,
+// and in a batch without padding the cost of a causal item follows its position inside its own
+// sequence, a sawtooth over the rows.  The general instantiations therefore draw their items from
+// a global counter instead, in row order from the last row down (every sequence then hands out
+// its expensive items first, and the cheap starts come last).  One thread per CTA draws; the other
 // roles read the item from a two-slot ring in shared memory.  Returns false when a bounded wait
 // expired; *item < 0 means no items are left.
 constexpr int kSchedConsumers = 32 + kActThreads;   // the MMA warp and the activation threads
@@ -462,7 +463,7 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
   const uint32_t lane_off = static_cast<uint32_t>(((threadIdx.x >> 5) & 3) * 32) << 16;
   uint32_t s_cnt0 = 0, s_cnt1 = 0, it[2] = {0, 0};
 
-  constexpr bool DYNAMIC = (MODE == 3);
+  constexpr bool DYNAMIC = (MODE >= 2);
   for (int round = 0, rounds = num_rounds(p.n_items); DYNAMIC || round < rounds; ++round) {
     int item;
     if (DYNAMIC) {
@@ -680,10 +681,10 @@ sigattn_fwd_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
   const uint32_t tmem = tmem_base_slot;
 
   if (warp == kLoadWarp) {
-    if ((threadIdx.x & 31) == 0) fwd_load_role<D, CAUSAL, MODE == 3>(p, &tmQ, &tmK, &tmV, smem_base, &bars, &cta_err);
+    if ((threadIdx.x & 31) == 0) fwd_load_role<D, CAUSAL, MODE >= 2>(p, &tmQ, &tmK, &tmV, smem_base, &bars, &cta_err);
     __syncwarp();
   } else if (warp == kMmaWarp) {
-    fwd_mma_role<D, CAUSAL, MODE == 3>(p, smem_base, tmem, &bars, &cta_err);
+    fwd_mma_role<D, CAUSAL, MODE >= 2>(p, smem_base, tmem, &bars, &cta_err);
     __syncwarp();
   } else {
     fwd_act_role<D, CAUSAL, ALIBI, MODE>(p, &tmO, smem, tmem, &bars, &cta_err);
@@ -811,7 +812,8 @@ int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const 
   fp.status = status;
 
   fp.sched_counter = nullptr;
-  if (p.cu_seqlens != nullptr) {
+  const bool general = !packed && (p.cu_seqlens != nullptr || p.seqlens != nullptr || p.row_scale != nullptr || accumulate);
+  if (general) {   // the general instantiations draw their work items from a counter
     static std::atomic<unsigned> next_slot{0};
     int* counters = nullptr;
     *cuda_err = cudaGetSymbolAddress(reinterpret_cast<void**>(&counters), g_fwd_sched_counters);
@@ -832,7 +834,7 @@ int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const 
   rc = packed ? launch_fwd_variant<DD, CC, AA, 1>(tmQ, tmK, tmV, tmO, fp, num_sms, stream, cuda_err)       \
        : (p.cu_seqlens != nullptr)                                                                         \
            ? launch_fwd_variant<DD, CC, AA, 3>(tmQ, tmK, tmV, tmO, fp, num_sms, stream, cuda_err)          \
-       : (p.seqlens != nullptr || p.row_scale != nullptr || accumulate)                                    \
+       : general                                                                                           \
            ? launch_fwd_variant<DD, CC, AA, 2>(tmQ, tmK, tmV, tmO, fp, num_sms, stream, cuda_err)          \
            : launch_fwd_variant<DD, CC, AA, 0>(tmQ, tmK, tmV, tmO, fp, num_sms, stream, cuda_err)
   if (p.D == 128) {
