@@ -58,6 +58,19 @@ def host_cores() -> int:
         return os.cpu_count() or 1
 
 
+def blas_threads_all_cores():
+    """Let numpy's BLAS use every host core of this process (torchrun exports OMP_NUM_THREADS=1 to
+    its ranks, which would otherwise time the oracle on one core) and return the thread count in use."""
+    try:
+        from threadpoolctl import threadpool_info, threadpool_limits
+        threadpool_limits(limits=host_cores(), user_api="blas")
+        counts = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(counts) if counts else 1
+    except Exception:  # noqa: BLE001 - without threadpoolctl the environment decides
+        env = os.environ.get("OMP_NUM_THREADS")
+        return int(env) if env and env.isdigit() else host_cores()
+
+
 # ----------------------------------------------------------------------------- oracle legs
 
 
@@ -66,6 +79,7 @@ def oracle_sample(cfg, budget_s: float = 20.0):
     one batch element, as many as fit the time budget (at least one)."""
     import oracle  # test infrastructure; used here for the CPU baseline only
 
+    threads = blas_threads_all_cores()
     q, k, v, d_o = inputs.make_inputs(cfg, heads=1, batch=1)
     slopes = cfg.slopes()
     sl = None if slopes is None else slopes[:1]
@@ -87,7 +101,7 @@ def oracle_sample(cfg, budget_s: float = 20.0):
     return {
         "value": flops_head * done / total / 1e12,
         "unit": UNIT,
-        "cores": host_cores(),
+        "cores": threads,
         "kind": "oracle",
         "sample": f"{done} of {cfg.B * cfg.H} (batch, head) pairs of {cfg.name}, fwd+bwd, float64 numpy, "
                   f"{total:.1f} s wall",
