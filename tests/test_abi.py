@@ -124,3 +124,50 @@ def test_bf16_rounding_is_round_to_nearest_even():
         np.testing.assert_array_equal(back, t)
     except ImportError:
         pass
+
+
+def test_argument_validation_of_the_widened_entry_points(lib):
+    """Error codes of the wider entry points, also returned before any device work."""
+    import ctypes as c
+    buf = np.zeros(8192, dtype=np.uint8)
+    p = (buf.ctypes.data + 255) & ~255
+    vp, i, f32 = c.c_void_p, c.c_int, c.c_float
+
+    def sig(fn, types):
+        fn.restype, fn.argtypes = c.c_int, types
+        return fn
+
+    gqa = sig(lib.sigattn_fwd_gqa, [vp] * 4 + [i] * 5 + [f32, f32, vp, i, vp, i, vp])
+    assert gqa(p, p, p, p, 1, 6, 4, 4, 64, 0.125, 0.0, None, 0, None, 0, None) == -2      # H not a multiple of H_kv
+    assert gqa(p, p, p, p, 1, 6, 0, 4, 64, 0.125, 0.0, None, 0, None, 0, None) == -2
+    assert gqa(p, p, p, p, 1, 6, 3, 4, 64, 0.125, 0.0, p + 2, 0, None, 0, None) == -3     # bias vector alignment
+    nk = sig(lib.sigattn_fwd_nk, [vp] * 4 + [i] * 6 + [f32, f32, vp, i, vp, i, vp])
+    assert nk(p, p, p, p, 1, 2, 2, 8, 4, 64, 0.125, 0.0, None, 1, None, 0, None) == -2    # causal needs N_k >= N_q
+    assert nk(p, p, None, p, 1, 2, 2, 4, 8, 64, 0.125, 0.0, None, 1, None, 0, None) == -1
+    shard = sig(lib.sigattn_fwd_shard, [vp] * 4 + [i] * 6 + [f32, f32, vp, i, i, vp, i, vp])
+    assert shard(p, p, p, p, 1, 2, 2, 4, 8, 64, 0.125, 0.0, None, 1, (1 << 30) + 1, None, 0, None) == -2   # pos0 out of range
+    varlen = sig(lib.sigattn_fwd_varlen, [vp] * 4 + [i] * 5 + [f32, f32, vp, i, vp, vp, i, vp])
+    assert varlen(p, p, p, p, 1, 2, 2, 4, 64, 0.125, 0.0, None, 0, None, None, 0, None) == -1             # no lengths
+    assert varlen(p, p, p, p, 1, 2, 2, 4, 64, 0.125, 0.0, None, 0, p + 2, None, 0, None) == -3
+    ragged = sig(lib.sigattn_fwd_ragged, [vp] * 4 + [i] * 4 + [vp, i, f32, f32, vp, i, vp, i, vp])
+    assert ragged(p, p, p, p, 2, 2, 4, 64, None, 1, 0.125, 0.0, None, 0, None, 0, None) == -1
+    assert ragged(p, p, p, p, 2, 2, 4, 64, p, 0, 0.125, 0.0, None, 0, None, 0, None) == -2                # no sequences
+    rows = sig(lib.sigattn_fwd_rowscale, [vp] * 4 + [i] * 6 + [f32, f32, vp, i, vp, vp, i, vp])
+    assert rows(p, p, p, p, 1, 2, 2, 4, 4, 64, 0.125, 0.0, None, 0, None, None, 0, None) == -1            # no factors
+    norm = sig(lib.sigattn_seqlen_norm, [vp, i, i, f32, i, vp])
+    assert norm(None, 4, 4, 0.5, 1, None) == -1
+    assert norm(p, 8, 4, 0.5, 1, None) == -2                                                              # causal needs N_k >= N_q
+    assert norm(p, 4, 4, 0.5, 3, None) == -4
+    dec = sig(lib.sigattn_fwd_decode, [vp] * 4 + [i] * 6 + [f32, f32, vp, i, vp, i, vp, c.c_size_t, vp])
+    assert dec(p, p, p, p, 1, 2, 2, 1, 8, 64, 0.125, 0.0, None, 1, None, 0, None, 0, None) == -1          # workspace missing
+    assert dec(p, p, p, p, 1, 2, 2, 1, 8, 64, 0.125, 0.0, None, 1, None, 0, p, 16, None) == -5
+    lib.sigattn_fwd_decode_workspace_bytes.restype = c.c_size_t
+    lib.sigattn_fwd_decode_workspace_bytes.argtypes = [i] * 5
+    assert lib.sigattn_fwd_decode_workspace_bytes(2, 4, 3, 128, 0) == 2 * 4 * 3 * 128 * 4
+    assert lib.sigattn_fwd_decode_workspace_bytes(2, 4, 3, 128, 1) == 0
+    acc = sig(lib.sigattn_fwd_shard_acc, [vp] * 4 + [i] * 6 + [f32, f32, vp, i, i, vp, i, vp])
+    assert acc(p, p, p, None, 1, 2, 2, 4, 8, 64, 0.125, 0.0, None, 1, 0, None, 0, None) == -1             # no accumulator
+    assert acc(p, p, p, p, 1, 2, 2, 4, 8, 64, 0.125, 0.0, None, 1, 0, None, 1, None) == -4                # bf16 only
+    conv = sig(lib.sigattn_acc_to_bf16, [vp, vp, c.c_size_t, f32, vp])
+    assert conv(p, None, 8, 1.0, None) == -1
+    assert conv(p, p, 6, 1.0, None) == -2                                                                 # n not a multiple of 4
