@@ -56,3 +56,64 @@ def test_random_case(case):
     if c["bias_vec"]:
         ref_db = oracle.sigattn_bwd_dbias(q, k, v, d_o, scale, b64, c["causal"], slopes)
         assert rel_fro(db.cpu().numpy().astype(np.float64), ref_db) < BF16_REL_FRO, c
+
+
+@pytest.mark.parametrize("case", range(10))
+def test_random_batches_of_different_lengths(case):
+    """The same random batch of sequences through the padded entry points and through the ones
+    without padding, both against the oracle."""
+    import torch
+    import paper_2409_04431_b200 as sa
+    rng = np.random.default_rng(2000 + case)
+    D = int(rng.choice([64, 128]))
+    H_kv = int(rng.integers(1, 3))
+    H = H_kv * int(rng.integers(1, 3))
+    n_seqs = int(rng.integers(1, 7))
+    lens = [int(x) for x in rng.integers(0 if n_seqs > 1 else 1, 330, size=n_seqs)]
+    if sum(lens) == 0:
+        lens[0] = 5
+    causal = bool(rng.integers(0, 2))
+    slopes = (0.5 ** np.arange(1, H + 1)).astype(np.float32) if rng.integers(0, 2) else None
+    sl = None if slopes is None else torch.from_numpy(slopes).cuda()
+    scale = 1.0 / math.sqrt(D)
+    bias = (-np.log(np.maximum(np.array(lens, dtype=np.float64), 1.0))[:, None] + 0.2 * rng.standard_normal((n_seqs, H))).astype(np.float32)
+    tb = torch.from_numpy(bias).cuda()
+    b64 = bias.astype(np.float64)
+    tag = dict(case=case, D=D, H=H, H_kv=H_kv, lens=lens, causal=causal, slopes=slopes is not None)
+
+    def check(outs, refs, ref_db, db):
+        for name, g, r in zip(("O", "dQ", "dK", "dV"), outs, refs):
+            g = to_host(g)
+            assert np.isfinite(g).all(), (name, tag)
+            assert rel_fro(g, r) < BF16_REL_FRO, (name, rel_fro(g, r), tag)
+            assert max_abs(g, r) < 2e-2 * max(1.0, float(np.abs(r).max())), (name, tag)
+        assert rel_fro(db.cpu().numpy().astype(np.float64), ref_db) < BF16_REL_FRO, tag
+
+    # without padding
+    T = sum(lens)
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    q, _, _, d_o = inputs.random_case(1, H, T, D, 500 + case)
+    _, k, v, _ = inputs.random_case(1, H_kv, T, D, 600 + case)
+    tq, tk, tv, tdo = (to_device(t, "bf16") for t in (q, k, v, d_o))
+    tcu = torch.from_numpy(cu).cuda()
+    o = sa.sigattn_fwd_ragged(tq, tk, tv, tcu, scale, tb, causal, sl)
+    dq, dk, dv, db = sa.sigattn_bwd_ragged(tq, tk, tv, tdo, tcu, scale, tb, causal, sl, want_dbias=True)
+    sa.sigattn_check()
+    check((o, dq, dk, dv),
+          (oracle.sigattn_fwd(q, k, v, scale, b64, causal, slopes, cu_seqlens=cu),) + tuple(
+              oracle.sigattn_bwd(q, k, v, d_o, scale, b64, causal, slopes, cu_seqlens=cu)),
+          oracle.sigattn_bwd_dbias(q, k, v, d_o, scale, b64, causal, slopes, cu_seqlens=cu), db)
+
+    # padded to the longest sequence (rounded up a little so that some padding always exists)
+    N = max(lens) + int(rng.integers(1, 40))
+    qp, _, _, dop = inputs.random_case(n_seqs, H, N, D, 700 + case)
+    _, kp, vp, _ = inputs.random_case(n_seqs, H_kv, N, D, 800 + case)
+    tq, tk, tv, tdo = (to_device(t, "bf16") for t in (qp, kp, vp, dop))
+    tl = torch.tensor(lens, dtype=torch.int32, device="cuda")
+    o = sa.sigattn_fwd_varlen(tq, tk, tv, scale, tb, tl, causal, sl)
+    dq, dk, dv, db = sa.sigattn_bwd_varlen(tq, tk, tv, tdo, scale, tb, tl, causal, sl, want_dbias=True)
+    sa.sigattn_check()
+    check((o, dq, dk, dv),
+          (oracle.sigattn_fwd(qp, kp, vp, scale, b64, causal, slopes, seqlens=lens),) + tuple(
+              oracle.sigattn_bwd(qp, kp, vp, dop, scale, b64, causal, slopes, seqlens=lens)),
+          oracle.sigattn_bwd_dbias(qp, kp, vp, dop, scale, b64, causal, slopes, seqlens=lens), db)
