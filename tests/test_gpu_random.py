@@ -117,3 +117,45 @@ def test_random_batches_of_different_lengths(case):
           (oracle.sigattn_fwd(qp, kp, vp, scale, b64, causal, slopes, seqlens=lens),) + tuple(
               oracle.sigattn_bwd(qp, kp, vp, dop, scale, b64, causal, slopes, seqlens=lens)),
           oracle.sigattn_bwd_dbias(qp, kp, vp, dop, scale, b64, causal, slopes, seqlens=lens), db)
+
+
+@pytest.mark.parametrize("case", range(8))
+def test_random_decode_and_row_factors(case):
+    """Random cache-decoding shapes through the split-key forward, and random row factors through
+    forward and backward."""
+    import torch
+    import paper_2409_04431_b200 as sa
+    rng = np.random.default_rng(3000 + case)
+    D = int(rng.choice([64, 128]))
+    H_kv = int(rng.integers(1, 4))
+    H = H_kv * int(rng.integers(1, 5))
+    B = int(rng.integers(1, 3))
+    N_q = int(rng.integers(1, 9))
+    N_k = int(rng.integers(max(N_q, 130), 5000))
+    causal = bool(rng.integers(0, 2))
+    slopes = (0.5 ** np.arange(1, H + 1)).astype(np.float32) if rng.integers(0, 2) else None
+    sl = None if slopes is None else torch.from_numpy(slopes).cuda()
+    scale, bias = 1.0 / math.sqrt(D), -math.log(N_k)
+    tag = dict(case=case, B=B, H=H, H_kv=H_kv, N_q=N_q, N_k=N_k, D=D, causal=causal, slopes=slopes is not None)
+    q, _, _, d_o = inputs.random_case(B, H, N_q, D, 900 + case)
+    _, k, v, _ = inputs.random_case(B, H_kv, N_k, D, 950 + case)
+    tq, tk, tv, tdo = (to_device(t, "bf16") for t in (q, k, v, d_o))
+    o = sa.sigattn_fwd_decode(tq, tk, tv, scale, bias, causal, sl)
+    sa.sigattn_check()
+    ref = oracle.sigattn_fwd(q, k, v, scale, bias, causal, slopes)
+    g = to_host(o)
+    assert rel_fro(g, ref) < BF16_REL_FRO, (rel_fro(g, ref), tag)
+    assert max_abs(g, ref) < 2e-2 * max(1.0, float(np.abs(ref).max())), tag
+
+    r = rng.uniform(0.05, 1.5, size=N_q).astype(np.float32)
+    tr = torch.from_numpy(r).cuda()
+    o = sa.sigattn_fwd_rowscale(tq, tk, tv, scale, bias, tr, causal, sl)
+    dq, dk, dv, _ = sa.sigattn_bwd_rowscale(tq, tk, tv, tdo, scale, bias, tr, causal, sl)
+    sa.sigattn_check()
+    r64 = r.astype(np.float64)
+    refs = (oracle.sigattn_fwd(q, k, v, scale, bias, causal, slopes, row_scale=r64),) + tuple(
+        oracle.sigattn_bwd(q, k, v, d_o, scale, bias, causal, slopes, row_scale=r64))
+    for name, g, rf in zip(("O", "dQ", "dK", "dV"), (o, dq, dk, dv), refs):
+        g = to_host(g)
+        assert rel_fro(g, rf) < BF16_REL_FRO, (name, rel_fro(g, rf), tag)
+        assert max_abs(g, rf) < 2e-2 * max(1.0, float(np.abs(rf).max())), (name, tag)
