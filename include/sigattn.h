@@ -162,8 +162,11 @@ SIGATTN_API int sigattn_fwd_gqa(const void* q, const void* k, const void* v, voi
 /* Backward of sigattn_fwd_gqa: dk, dv are [B, H_kv, N, D] and hold the sums over the query
  * heads that read each key/value head (accumulated on chip: a work item keeps dK_j, dV_j
  * of one key/value head in tensor memory while it walks the query tiles of all its query
- * heads).  `dbias_bh`: NULL or B*H floats as in sigattn_bwd_bias_vec.  The workspace is
- * that of sigattn_bwd for (B, H, N, D). */
+ * heads).  When B * H_kv * ceil(N / 128) work items cannot fill the GPU (multi-query attention at
+ * a small batch) the query heads of a group are divided over several work items, which add their
+ * dK_j, dV_j into the cleared outputs with bf16 reduce-adds; dk and dv then depend on the order of
+ * the additions in their last bits, like dq.  `dbias_bh`: NULL or B*H floats as in
+ * sigattn_bwd_bias_vec.  The workspace is that of sigattn_bwd for (B, H, N, D). */
 SIGATTN_API int sigattn_bwd_gqa(const void* q, const void* k, const void* v, const void* d_o,
                     void* dq, void* dk, void* dv,
                     int B, int H, int H_kv, int N, int D,

@@ -84,6 +84,10 @@ struct BwdParams {
   const int* cu_seqlens;
   int n_seqs;
   int* sched_counter;   // dynamic schedule: next work item to hand out (zero at launch), or nullptr
+  // Few (batch, key/value head) pairs (multi-query attention at a small batch): the query heads of a
+  // group are split over n_sub work items of heads_per_sub heads each, which add their dK_j, dV_j
+  // (bf16 TMA reduce-adds into the cleared outputs) instead of storing them.  n_sub = 1: off.
+  int n_sub, heads_per_sub;
   int n_items;
   float scale, scale_log2e, bias_log2e;
   const float* bias_vec;   // one bias per (batch, head) instead of the scalar, or nullptr
@@ -155,7 +159,15 @@ __device__ __forceinline__ BwdItem decode_bwd_item(const BwdParams& p, int item)
   BwdItem w;
   w.j = item / p.BH;  // ascending key tile = descending work when causal
   w.bh = item - w.j * p.BH;
-  w.bh_q0 = GROUPED ? (w.bh / p.H_kv) * p.H + (w.bh % p.H_kv) * p.group : w.bh;
+  int sub = 0;
+  if (GROUPED && p.n_sub > 1) {   // item = (key tile, key/value head, part of its query heads)
+    const int per_j = p.BH * p.n_sub;
+    w.j = item / per_j;
+    const int r = item - w.j * per_j;
+    w.bh = r / p.n_sub;
+    sub = r - w.bh * p.n_sub;
+  }
+  w.bh_q0 = GROUPED ? (w.bh / p.H_kv) * p.H + (w.bh % p.H_kv) * p.group + sub * p.heads_per_sub : w.bh;
   // causal: the first query tile whose last row, at position 128 i + 127 + pos0, reaches key 128 j
   // padded batch: query tiles past the sequence's end are not visited at all
   const bool padded = GROUPED && p.seqlens != nullptr;
@@ -176,7 +188,7 @@ __device__ __forceinline__ BwdItem decode_bwd_item(const BwdParams& p, int item)
     w.i_begin = max(0, min(p.n_tiles - 1, q_lo / kT));
     w.n = max(1, min(p.n_tiles, (q_hi + kT - 1) / kT) - w.i_begin);
   }
-  w.steps = GROUPED ? p.group * w.n : w.n;
+  w.steps = GROUPED ? p.heads_per_sub * w.n : w.n;
   return w;
 }
 
@@ -238,7 +250,7 @@ __device__ void bwd_load_role(const BwdParams& p, const CUtensorMap* tmQ, const 
       load_tile(tmV, smem_base + L::kVOff, bar, w.j * kT, w.bh);
     }
     ++item_cnt;
-    for (int g = 0; g < (GROUPED ? p.group : 1); ++g) {
+    for (int g = 0; g < (GROUPED ? p.heads_per_sub : 1); ++g) {
       for (int it = (g == 0 ? 1 : 0); it < w.n; ++it) {
         if (!load_q(w.i_begin + it, w.bh_q0 + g)) return;
         if (!load_do(w.i_begin + it, w.bh_q0 + g)) return;
@@ -441,7 +453,7 @@ __device__ void bwd_act_role(const BwdParams& p, const CUtensorMap* tmDk, const 
       if (item < 0) continue;
     }
     const BwdItem w = decode_bwd_item<CAUSAL, GROUPED>(p, item);
-    for (int g = 0; g < (GROUPED ? p.group : 1); ++g) {   // the query heads that read this key/value head
+    for (int g = 0; g < (GROUPED ? p.heads_per_sub : 1); ++g) {   // the query heads that read this key/value head
     const int bh_q = w.bh_q0 + g;
     float slope_log2e = 0.0f;
     if (ALIBI) slope_log2e = p.slopes[bh_q % p.H] * kLog2eB;
@@ -563,7 +575,10 @@ __device__ void bwd_act_role(const BwdParams& p, const CUtensorMap* tmDk, const 
       const CUtensorMap* tm = (wg == 0) ? tmDv : tmDk;
 #pragma unroll
       for (int pn = 0; pn < L::kPanels; ++pn)
-        tma_store_3d(tm, smem_u32(stage + pn * L::kPanelBytes), pn * 64, w.j * kT, w.bh);
+        if (GROUPED && p.n_sub > 1)   // the parts of a group add their shares
+          tma_reduce_add_3d(tm, smem_u32(stage + pn * L::kPanelBytes), pn * 64, w.j * kT, w.bh);
+        else
+          tma_store_3d(tm, smem_u32(stage + pn * L::kPanelBytes), pn * 64, w.j * kT, w.bh);
       tma_commit_group();
       tma_wait_group_read<0>();
       mbar_arrive(smem_u32(&bars->kv_empty));
@@ -837,7 +852,19 @@ int launch_bwd_bf16(const void* q, const void* k, const void* v, const void* d_o
   bp.n_tiles = (p.N + kT - 1) / kT;
   bp.n_tiles_k = (p.key_rows() + kT - 1) / kT;
   bp.pos0 = p.query_pos0();
-  bp.n_items = bp.n_tiles_k * bp.BH;
+  // Grouped heads with few (batch, key/value head) pairs: split a group's query heads over several
+  // work items (the smallest divisor of the group size that yields two items per SM, if any).
+  bp.n_sub = 1;
+  if (bp.group > 1 && p.seqlens == nullptr && p.cu_seqlens == nullptr) {
+    const long long base_items = static_cast<long long>(bp.n_tiles_k) * bp.BH;
+    for (int d = 1; d <= bp.group; ++d) {
+      if (bp.group % d != 0) continue;
+      bp.n_sub = d;
+      if (base_items * d >= 2ll * num_sms) break;
+    }
+  }
+  bp.heads_per_sub = bp.group / bp.n_sub;
+  bp.n_items = bp.n_tiles_k * bp.BH * bp.n_sub;
   bp.scale = p.scale;
   bp.scale_log2e = p.scale * kLog2eB;
   bp.bias_log2e = p.bias * kLog2eB;
@@ -851,6 +878,13 @@ int launch_bwd_bf16(const void* q, const void* k, const void* v, const void* d_o
   bp.status = status;
 
   const size_t n_elems = static_cast<size_t>(BH) * p.N * p.D;
+  if (bp.n_sub > 1) {   // dK, dV are summed over the parts of a group: clear them first
+    const size_t kv_bytes = static_cast<size_t>(BH_kv) * p.key_rows() * p.D * 2;
+    *cuda_err = cudaMemsetAsync(dk, 0, kv_bytes, stream);
+    if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
+    *cuda_err = cudaMemsetAsync(dv, 0, kv_bytes, stream);
+    if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
+  }
   // step 1: clear the fp32 dQ accumulator (and the bias gradient, which the kernel adds into);
   // with acc_only the accumulator is the caller's running sum over key/value shards: not cleared
   if (!p.acc_only) {
