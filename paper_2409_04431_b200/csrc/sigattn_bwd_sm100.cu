@@ -857,7 +857,9 @@ int launch_bwd_bf16(const void* q, const void* k, const void* v, const void* d_o
   bp.n_sub = 1;
   if (bp.group > 1 && p.seqlens == nullptr && p.cu_seqlens == nullptr) {
     const long long base_items = static_cast<long long>(bp.n_tiles_k) * bp.BH;
-    for (int d = 1; d <= bp.group; ++d) {
+    // at most four parts: every part adds one bf16 rounding to dK, dV (sixteen parts measured a
+    // relative error of 5.5e-3, four stay near 3e-3)
+    for (int d = 1; d <= bp.group && d <= 4; ++d) {
       if (bp.group % d != 0) continue;
       bp.n_sub = d;
       if (base_items * d >= 2ll * num_sms) break;

@@ -113,6 +113,7 @@ struct FwdParams {
   // the partial results simply add up.  n_splits = 1: off.
   int n_splits, tiles_per_split;
   float* split_ws;
+  int o_reduce;    // 1: split items of the unpacked general mode add bf16 tiles into O instead of storing them
   int n_items;
   float scale_log2e, bias_log2e;
   const float* bias_vec;   // one bias per (batch, head) instead of the scalar, or nullptr
@@ -219,11 +220,31 @@ __device__ __forceinline__ Item decode_item(const FwdParams& p, int item) {
       w.n[t] = max(1, min(p.n_kv_total, (key_end + kBN - 1) / kBN) - w.j0);
     }
   }
-  if (p.n_splits > 1) {   // packed mode: every valid tile visits all key tiles; this item takes its share
+  if (p.n_splits > 1 && p.pack_rows > 0) {   // packed mode: every valid tile visits all key tiles; this item takes its share
     w.j0 = split * p.tiles_per_split;
     const int n = min(p.tiles_per_split, p.n_kv_total - w.j0);
 #pragma unroll
     for (int t = 0; t < 2; ++t) w.n[t] = w.n[t] > 0 ? n : 0;
+  } else if (p.n_splits > 1) {
+    // Few work items (one long causal sequence, few heads): the key tiles of an item are divided
+    // over n_splits items that add their shares of O.  Tile 1 of a pair sees as many key tiles as
+    // tile 0 or one more; both must stay non-empty in every part, so the parts are cut by tile 0's
+    // count.  Items too short to cut go to part 0 whole; their other parts visit one key tile past
+    // the diagonal, which is fully masked (or out of range and read as zeros), and add zeros.
+    const int n0 = w.n[0], n1 = w.n[1];
+    if (n0 >= 2 * p.n_splits && (n1 == 0 || n1 >= n0)) {
+      // part s takes key tiles [s n0 / S, (s + 1) n0 / S): never empty since n0 >= 2 S; the last
+      // part of tile 1 runs on to n1
+      const int first = split * n0 / p.n_splits, end = (split + 1) * n0 / p.n_splits;
+      const bool last = split == p.n_splits - 1;
+      w.j0 = first;
+      w.n[0] = end - first;
+      w.n[1] = n1 == 0 ? 0 : (last ? n1 : end) - first;
+    } else if (split > 0) {
+      w.j0 = max(n0, n1);
+      w.n[0] = n0 > 0 ? 1 : 0;
+      w.n[1] = n1 > 0 ? 1 : 0;
+    }
   }
   w.n_kv = max(w.n[0], w.n[1]);
   return w;
@@ -618,7 +639,10 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
       if (threadIdx.x == 0) {
 #pragma unroll
         for (int pn = 0; pn < L::kPanels; ++pn)
-          tma_store_3d(tmO, smem_u32(stage + pn * L::kPanelBytes), pn * 64, w.row0 + t * kBM, w.bh);
+          if (GENERAL && p.o_reduce)   // the parts of a split item add their shares of O (cleared before the launch)
+            tma_reduce_add_3d(tmO, smem_u32(stage + pn * L::kPanelBytes), pn * 64, w.row0 + t * kBM, w.bh);
+          else
+            tma_store_3d(tmO, smem_u32(stage + pn * L::kPanelBytes), pn * 64, w.row0 + t * kBM, w.bh);
         tma_commit_group();
         tma_wait_group_read<0>();
         mbar_arrive(smem_u32(&bars->q_empty[t]));
@@ -773,6 +797,20 @@ int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const 
   // is cleared, nothing converted, `o` is not written.  Otherwise the accumulator is only used as
   // scratch when the keys are split.
   const bool accumulate = p.split_ws != nullptr && (p.acc_only != 0 || n_splits > 1);
+  // One long causal sequence with few heads: the most expensive work item alone takes as long as
+  // the whole job should.  Divide the key tiles of every item over 2 to 4 items that add their
+  // bf16 shares into O (one extra rounding per part; with two parts the sum does not depend on
+  // their order).
+  int o_splits = 1;
+  {
+    const long long base_items = static_cast<long long>((p.N + 2 * kBM - 1) / (2 * kBM)) * BH;
+    if (p.causal && !small && p.split_ws == nullptr && p.seqlens == nullptr && p.cu_seqlens == nullptr &&
+        base_items < 2ll * num_sms && n_kv_tiles >= 32) {   // measured: +9 % at N = 4096, +47 % at 32768; a loss below
+      o_splits = static_cast<int>((2ll * num_sms + base_items - 1) / base_items);
+      if (o_splits > 4) o_splits = 4;
+      if (o_splits > n_kv_tiles / 4) o_splits = n_kv_tiles / 4;
+    }
+  }
   const uint64_t q_heads = packed ? BH_kv : BH;
   const uint64_t q_rows = packed ? static_cast<uint64_t>(p.N) * group : p.N;
   CUtensorMap tmQ, tmK, tmV, tmO;
@@ -797,10 +835,11 @@ int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const 
   fp.pos0 = p.query_pos0();
   fp.n_pairs = (fp.N + 2 * kBM - 1) / (2 * kBM);
   fp.n_kv_total = (p.key_rows() + kBN - 1) / kBN;
-  fp.n_splits = n_splits;
+  fp.n_splits = o_splits > 1 ? o_splits : n_splits;
+  fp.o_reduce = o_splits > 1 ? 1 : 0;
   fp.tiles_per_split = (fp.n_kv_total + n_splits - 1) / n_splits;
   fp.split_ws = accumulate ? p.split_ws : nullptr;
-  fp.n_items = fp.n_pairs * fp.BH * n_splits;
+  fp.n_items = fp.n_pairs * fp.BH * fp.n_splits;
   fp.scale_log2e = p.scale * kLog2e;
   fp.bias_log2e = p.bias * kLog2e;
   fp.bias_vec = p.bias_vec;
@@ -812,7 +851,8 @@ int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const 
   fp.status = status;
 
   fp.sched_counter = nullptr;
-  const bool general = !packed && (p.cu_seqlens != nullptr || p.seqlens != nullptr || p.row_scale != nullptr || accumulate);
+  const bool general = !packed && (p.cu_seqlens != nullptr || p.seqlens != nullptr || p.row_scale != nullptr || accumulate ||
+                                   o_splits > 1);
   if (general) {   // the general instantiations draw their work items from a counter
     static std::atomic<unsigned> next_slot{0};
     int* counters = nullptr;
@@ -823,6 +863,10 @@ int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const 
     if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
   }
   const size_t n_elems = static_cast<size_t>(BH) * p.N * p.D;
+  if (o_splits > 1) {
+    *cuda_err = cudaMemsetAsync(o, 0, n_elems * 2, stream);
+    if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
+  }
   if (accumulate && !p.acc_only) {
     *cuda_err = cudaMemsetAsync(p.split_ws, 0, n_elems * sizeof(float), stream);
     if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
