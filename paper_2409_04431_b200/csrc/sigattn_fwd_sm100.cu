@@ -810,6 +810,12 @@ int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const 
       if (o_splits > 4) o_splits = 4;
       if (o_splits > n_kv_tiles / 4) o_splits = n_kv_tiles / 4;
     }
+    // without a mask all items cost the same; dividing them pays only while the parts still fit one round
+    if (!p.causal && !small && p.split_ws == nullptr && p.seqlens == nullptr && p.cu_seqlens == nullptr &&
+        2 * base_items <= num_sms && n_kv_tiles >= 32) {
+      o_splits = static_cast<int>(num_sms / base_items);
+      if (o_splits > 4) o_splits = 4;
+    }
   }
   const uint64_t q_heads = packed ? BH_kv : BH;
   const uint64_t q_rows = packed ? static_cast<uint64_t>(p.N) * group : p.N;

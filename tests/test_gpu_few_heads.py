@@ -13,6 +13,20 @@ from parity_util import BF16_REL_FRO, max_abs, rel_fro, to_device, to_host
 pytestmark = pytest.mark.gpu
 
 
+def test_forward_without_mask_few_items():
+    """No mask, 34 work items of 33 key tiles each: divided four ways so that they fill the GPU."""
+    import paper_2409_04431_b200 as sa
+    B, H, N, D = 1, 2, 4224, 64
+    q, k, v, _ = inputs.random_case(B, H, N, D, 251)
+    tq, tk, tv = (to_device(t, "bf16") for t in (q, k, v))
+    scale, bias = 1.0 / math.sqrt(D), -math.log(N)
+    o = sa.sigattn_fwd(tq, tk, tv, scale, bias, False)
+    sa.sigattn_check()
+    ref = oracle.sigattn_fwd(q, k, v, scale, bias, False)
+    assert rel_fro(to_host(o), ref) < BF16_REL_FRO
+    assert max_abs(to_host(o), ref) < 2e-2 * max(1.0, float(np.abs(ref).max()))
+
+
 @pytest.mark.parametrize("B,H,N,D,with_slopes", [
     (1, 2, 4224, 128, False),     # 33 key tiles, 34 work items: four parts per item
     (1, 3, 4300, 64, True),       # ragged tail, ALiBi
