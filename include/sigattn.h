@@ -73,10 +73,9 @@ extern "C" {
 #define SIGATTN_DTYPE_FP32 1
 
 /* Forward (Eq. 3; Algorithm 1).  q, k, v: inputs; o: output; all [B, H, N, D].
- * O is bit-reproducible from run to run, except for calls with so few (batch, head) pairs that
- * the library divides the keys of a work item over several thread blocks (N >= 4096 and fewer than
- * two work items per SM with the causal mask, at most half an item per SM without): their bf16
- * shares are added in arrival order. */
+ * O is bit-reproducible from run to run.  (Calls with so few (batch, head) pairs that they cannot
+ * fill the GPU divide the keys of a work item over two thread blocks that add their bf16 shares
+ * into the cleared O; the sum of two shares does not depend on their order.) */
 SIGATTN_API int sigattn_fwd(const void* q, const void* k, const void* v, void* o,
                 int B, int H, int N, int D,
                 float scale, float bias, int causal,

@@ -798,24 +798,26 @@ int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const 
   // scratch when the keys are split.
   const bool accumulate = p.split_ws != nullptr && (p.acc_only != 0 || n_splits > 1);
   // One long causal sequence with few heads: the most expensive work item alone takes as long as
-  // the whole job should.  Divide the key tiles of every item over 2 to 4 items that add their
-  // bf16 shares into O (one extra rounding per part; with two parts the sum does not depend on
-  // their order).
+  // the whole job should.  Divide the key tiles of every item over two items that add their
+  // bf16 shares into O (one extra rounding; the sum of two parts does not depend on their order).
   int o_splits = 1;
-  {
+  if (!small && p.split_ws == nullptr && p.seqlens == nullptr && p.cu_seqlens == nullptr) {
     const long long base_items = static_cast<long long>((p.N + 2 * kBM - 1) / (2 * kBM)) * BH;
-    if (p.causal && !small && p.split_ws == nullptr && p.seqlens == nullptr && p.cu_seqlens == nullptr &&
-        base_items < 2ll * num_sms && n_kv_tiles >= 32) {   // measured: +9 % at N = 4096, +47 % at 32768; a loss below
-      o_splits = static_cast<int>((2ll * num_sms + base_items - 1) / base_items);
-      if (o_splits > 4) o_splits = 4;
-      if (o_splits > n_kv_tiles / 4) o_splits = n_kv_tiles / 4;
+    int by_mask = 1, by_round = 1;
+    if (p.causal && base_items < 2ll * num_sms && n_kv_tiles >= 32) {   // measured: +9 % at N = 4096, +47 % at 32768; a loss below
+      by_mask = static_cast<int>((2ll * num_sms + base_items - 1) / base_items);
+      if (by_mask > n_kv_tiles / 4) by_mask = n_kv_tiles / 4;
     }
-    // without a mask all items cost the same; dividing them pays only while the parts still fit one round
-    if (!p.causal && !small && p.split_ws == nullptr && p.seqlens == nullptr && p.cu_seqlens == nullptr &&
-        2 * base_items <= num_sms && n_kv_tiles >= 32) {
-      o_splits = static_cast<int>(num_sms / base_items);
-      if (o_splits > 4) o_splits = 4;
+    // whatever the mask: while all parts still fit one round of the grid, dividing the items only
+    // shortens the longest one (B1 H1 N2048 has 8 items, the last of them 16 key tiles long)
+    if (2 * base_items <= num_sms && n_kv_tiles >= 4) {
+      by_round = static_cast<int>(num_sms / base_items);
+      if (by_round > n_kv_tiles / 2) by_round = n_kv_tiles / 2;
     }
+    o_splits = by_mask > by_round ? by_mask : by_round;
+    // two parts at most: 0 + a + b does not depend on which part arrives first, so O stays
+    // bit-reproducible; three or four parts measured 5-10 % faster still but would give that up
+    if (o_splits > 2) o_splits = 2;
   }
   const uint64_t q_heads = packed ? BH_kv : BH;
   const uint64_t q_rows = packed ? static_cast<uint64_t>(p.N) * group : p.N;

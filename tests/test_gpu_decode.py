@@ -53,7 +53,9 @@ def test_decode_many_queries_is_the_plain_path_and_workspace_is_checked():
     scale = 1.0 / math.sqrt(D)
     ws = torch.full((sa.sigattn_fwd_decode_workspace_bytes(B, H, N_q, D, 0),), 7, dtype=torch.uint8, device="cuda")
     o = sa.sigattn_fwd_decode(tq, tk, tv, scale, -2.0, True, workspace=ws)
-    assert torch.equal(o, sa.sigattn_fwd_nk(tq, tk, tv, scale, -2.0, True))
+    # the same kernels either way; the call without scratch may divide its few work items over the keys
+    # and add bf16 shares, so the two agree to single roundings
+    assert rel_fro(to_host(o), to_host(sa.sigattn_fwd_nk(tq, tk, tv, scale, -2.0, True)).astype(np.float64)) < 4e-3
     assert bool((ws == 7).all())                          # more than one pair of query tiles: no split, no scratch use
     with pytest.raises(sa.SigattnError) as e:
         sa.sigattn_fwd_decode(tq, tk, tv, scale, -2.0, True, workspace=ws[:-256])

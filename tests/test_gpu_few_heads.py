@@ -14,7 +14,7 @@ pytestmark = pytest.mark.gpu
 
 
 def test_forward_without_mask_few_items():
-    """No mask, 34 work items of 33 key tiles each: divided four ways so that they fill the GPU."""
+    """No mask, 34 work items of 33 key tiles each: divided in two."""
     import paper_2409_04431_b200 as sa
     B, H, N, D = 1, 2, 4224, 64
     q, k, v, _ = inputs.random_case(B, H, N, D, 251)
@@ -28,7 +28,7 @@ def test_forward_without_mask_few_items():
 
 
 @pytest.mark.parametrize("B,H,N,D,with_slopes", [
-    (1, 2, 4224, 128, False),     # 33 key tiles, 34 work items: four parts per item
+    (1, 2, 4224, 128, False),     # 33 key tiles, 34 work items: two parts per item
     (1, 3, 4300, 64, True),       # ragged tail, ALiBi
     (2, 8, 4100, 128, False),     # 272 items: two parts, the short items are not cut
     (1, 24, 4100, 64, False),     # 408 items: enough, no split (same entry point, other path)
@@ -49,8 +49,7 @@ def test_forward_with_split_key_tiles(B, H, N, D, with_slopes):
     assert rel_fro(g, ref) < BF16_REL_FRO, rel_fro(g, ref)
     assert max_abs(g, ref) < 2e-2 * max(1.0, float(np.abs(ref).max()))
     o2 = sa.sigattn_fwd(tq, tk, tv, scale, bias, True, sl)
-    # parts may add in another order: single bf16 roundings differ, nothing more
-    assert rel_fro(to_host(o2), g.astype(np.float64)) < 4e-3
+    assert torch.equal(o2, o)       # two parts: their sum does not depend on the order of arrival
 
 
 def test_forward_split_with_query_offset_and_row_factors():
