@@ -30,7 +30,7 @@ def test_forward_without_mask_few_items():
 @pytest.mark.parametrize("B,H,N,D,with_slopes", [
     (1, 2, 4224, 128, False),     # 33 key tiles, 34 work items: two parts per item
     (1, 3, 4300, 64, True),       # ragged tail, ALiBi
-    (2, 8, 4100, 128, False),     # 272 items: two parts, the short items are not cut
+    (2, 4, 4100, 128, False),     # 136 items: two parts, the short items are not cut
     (1, 24, 4100, 64, False),     # 408 items: enough, no split (same entry point, other path)
 ])
 def test_forward_with_split_key_tiles(B, H, N, D, with_slopes):
