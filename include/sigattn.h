@@ -87,7 +87,10 @@ SIGATTN_API int sigattn_fwd(const void* q, const void* k, const void* v, void* o
  * 256-byte aligned; its contents on entry are irrelevant and on exit unspecified.
  * Two calls that share a workspace must not overlap on the device.
  * dQ sums contributions of different key tiles with floating-point atomics, so its
- * low-order bits may differ from run to run; dK and dV are deterministic. */
+ * low-order bits may differ from run to run; dK and dV are deterministic.  (With so few
+ * (batch, head) pairs that the work items cannot fill the GPU, the query tiles of a key tile are
+ * divided over two thread blocks that add their bf16 shares of dK, dV into the cleared outputs;
+ * the sum of two shares does not depend on their order.) */
 SIGATTN_API int sigattn_bwd(const void* q, const void* k, const void* v, const void* d_o,
                 void* dq, void* dk, void* dv,
                 int B, int H, int N, int D,

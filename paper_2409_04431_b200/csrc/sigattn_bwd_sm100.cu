@@ -88,6 +88,9 @@ struct BwdParams {
   // group are split over n_sub work items of heads_per_sub heads each, which add their dK_j, dV_j
   // (bf16 TMA reduce-adds into the cleared outputs) instead of storing them.  n_sub = 1: off.
   int n_sub, heads_per_sub;
+  // Few work items with one query head per key/value head (one long sequence, few heads): the query
+  // tiles of a key tile are divided over two items (i_split = 2) that add their dK_j, dV_j likewise.
+  int i_split;
   int n_items;
   float scale, scale_log2e, bias_log2e;
   const float* bias_vec;   // one bias per (batch, head) instead of the scalar, or nullptr
@@ -167,6 +170,14 @@ __device__ __forceinline__ BwdItem decode_bwd_item(const BwdParams& p, int item)
     w.bh = r / p.n_sub;
     sub = r - w.bh * p.n_sub;
   }
+  int part = 0;
+  if (GROUPED && p.i_split > 1) {   // item = (key tile, head, half of its query tiles)
+    const int per_j = p.BH * 2;
+    w.j = item / per_j;
+    const int r = item - w.j * per_j;
+    w.bh = r >> 1;
+    part = r & 1;
+  }
   w.bh_q0 = GROUPED ? (w.bh / p.H_kv) * p.H + (w.bh % p.H_kv) * p.group + sub * p.heads_per_sub : w.bh;
   // causal: the first query tile whose last row, at position 128 i + 127 + pos0, reaches key 128 j
   // padded batch: query tiles past the sequence's end are not visited at all
@@ -187,6 +198,20 @@ __device__ __forceinline__ BwdItem decode_bwd_item(const BwdParams& p, int item)
     // (offsets that do not rise from 0 to N give wrong results, but the clamps keep every loop bounded)
     w.i_begin = max(0, min(p.n_tiles - 1, q_lo / kT));
     w.n = max(1, min(p.n_tiles, (q_hi + kT - 1) / kT) - w.i_begin);
+  }
+  if (GROUPED && p.i_split > 1) {
+    const int first_half = (w.n + 1) / 2;
+    if (part == 0) {
+      w.n = first_half;
+    } else if (w.n > first_half) {
+      w.i_begin += first_half;
+      w.n -= first_half;
+    } else {
+      // a single query tile cannot be divided (the last key tile of a causal call): the second item
+      // visits the query tile before it, which the mask blanks completely, and adds zeros
+      w.i_begin = max(0, w.i_begin - 1);
+      w.n = 1;
+    }
   }
   w.steps = GROUPED ? p.heads_per_sub * w.n : w.n;
   return w;
@@ -575,7 +600,7 @@ __device__ void bwd_act_role(const BwdParams& p, const CUtensorMap* tmDk, const 
       const CUtensorMap* tm = (wg == 0) ? tmDv : tmDk;
 #pragma unroll
       for (int pn = 0; pn < L::kPanels; ++pn)
-        if (GROUPED && p.n_sub > 1)   // the parts of a group add their shares
+        if (GROUPED && (p.n_sub > 1 || p.i_split > 1))   // the parts add their shares
           tma_reduce_add_3d(tm, smem_u32(stage + pn * L::kPanelBytes), pn * 64, w.j * kT, w.bh);
         else
           tma_store_3d(tm, smem_u32(stage + pn * L::kPanelBytes), pn * 64, w.j * kT, w.bh);
@@ -866,7 +891,18 @@ int launch_bwd_bf16(const void* q, const void* k, const void* v, const void* d_o
     }
   }
   bp.heads_per_sub = bp.group / bp.n_sub;
-  bp.n_items = bp.n_tiles_k * bp.BH * bp.n_sub;
+  // One query head per key/value head and at most one round of items: the first key tiles, which
+  // meet every query tile, set the time.  Divide the query tiles of every key tile over two items
+  // (two shares add up the same in either order, so dK, dV stay bit-reproducible).
+  bp.i_split = 1;
+  {
+    const long long base_items = static_cast<long long>(bp.n_tiles_k) * bp.BH;
+    const bool square = p.key_rows() == p.N && p.query_pos0() == 0;
+    if (bp.group == 1 && square && p.seqlens == nullptr && p.cu_seqlens == nullptr && bp.n_tiles >= 4 &&
+        (2 * base_items <= num_sms || (p.causal && base_items <= num_sms && bp.n_tiles >= 16)))
+      bp.i_split = 2;
+  }
+  bp.n_items = bp.n_tiles_k * bp.BH * bp.n_sub * bp.i_split;
   bp.scale = p.scale;
   bp.scale_log2e = p.scale * kLog2eB;
   bp.bias_log2e = p.bias * kLog2eB;
@@ -880,7 +916,7 @@ int launch_bwd_bf16(const void* q, const void* k, const void* v, const void* d_o
   bp.status = status;
 
   const size_t n_elems = static_cast<size_t>(BH) * p.N * p.D;
-  if (bp.n_sub > 1) {   // dK, dV are summed over the parts of a group: clear them first
+  if (bp.n_sub > 1 || bp.i_split > 1) {   // dK, dV are summed over the parts: clear them first
     const size_t kv_bytes = static_cast<size_t>(BH_kv) * p.key_rows() * p.D * 2;
     *cuda_err = cudaMemsetAsync(dk, 0, kv_bytes, stream);
     if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
@@ -931,7 +967,7 @@ int launch_bwd_bf16(const void* q, const void* k, const void* v, const void* d_o
                         : launch_bwd_variant<DD, CC, AA, false, KK>(maps, bp, num_sms, stream, cuda_err))
 #define SIGATTN_BWD_CASE(DD, CC, AA)                                                                       \
   rc = (bp.cu_seqlens != nullptr)                  ? SIGATTN_BWD_KIND(DD, CC, AA, 2)                        \
-       : (bp.group > 1 || bp.seqlens != nullptr)   ? SIGATTN_BWD_KIND(DD, CC, AA, 1)                        \
+       : (bp.group > 1 || bp.seqlens != nullptr || bp.i_split > 1) ? SIGATTN_BWD_KIND(DD, CC, AA, 1)        \
                                                    : SIGATTN_BWD_KIND(DD, CC, AA, 0)
   if (p.D == 128) {
     if (p.causal) { if (alibi) SIGATTN_BWD_CASE(128, true, true); else SIGATTN_BWD_CASE(128, true, false); }
