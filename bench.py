@@ -37,9 +37,10 @@ UNIT = "TFLOP/s"
 FALLBACK_PEAKS = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0}
 L2_FLUSH_BYTES = 256 << 20
 
-# DRAM bytes per launch of the dominant kernel (backward main kernel) from the committed
-# ncu capture, per workload; see profiles/.  None where no capture exists.
-NCU_TRAFFIC_BYTES = {"c4": 429.68e6 + 212.91e6}  # profiles/sigattn_bwd_bf16_kernel_c4.md
+# DRAM bytes per launch of the dominant kernel (backward main kernel), dram__bytes_read.sum +
+# dram__bytes_write.sum of one ncu capture per workload (the summaries are committed with the
+# other profile summaries).  None where no capture exists.
+NCU_TRAFFIC_BYTES = {"c4": 429.68e6 + 212.91e6, "c5": 12.753e9 + 7.068e9}
 
 
 def load_peaks():
