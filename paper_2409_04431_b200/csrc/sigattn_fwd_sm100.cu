@@ -72,7 +72,12 @@ struct FwdSmem {
   static constexpr int kStages = (D == 128) ? 4 : 8;
   static constexpr int kQOff = 0;
   static constexpr int kKvOff = 2 * kTileBytes;
-  static constexpr int kTotal = kKvOff + kStages * kTileBytes;
+  // At D = 64 there is room for a staging buffer of O of its own: the Q buffer is then free as soon
+  // as the item's last logits are computed, and the next item's Q load runs under the last activation,
+  // the last P V and the epilogue.  At D = 128 O is staged in the Q buffer (shared memory is full).
+  static constexpr bool kOStaged = (D == 64);
+  static constexpr int kOOff = kKvOff + kStages * kTileBytes;
+  static constexpr int kTotal = kOOff + (kOStaged ? 2 * kTileBytes : 0);
   static constexpr int kDynBytes = kTotal + 1024;  // slack to align the base to 1024 B
 };
 
@@ -370,11 +375,13 @@ __device__ void fwd_mma_role(const FwdParams& p, uint32_t smem_base, uint32_t tm
     tc_fence_after_sync();
     issue_s(0, kv_addr(k_cnt(0)));
     umma_commit_warp(leader, smem_u32(&bars->s_full[0]));
+    if (L::kOStaged && w.n[0] == 1) umma_commit_warp(leader, smem_u32(&bars->q_empty[0]));   // Q_0 no longer needed
     if (w.n[1] > 0) {
       if (!mbar_wait(smem_u32(&bars->q_full[1]), it[1] & 1, cta_err, 22)) return;
       tc_fence_after_sync();
       issue_s(1, kv_addr(k_cnt(0)));
       umma_commit_warp(leader, smem_u32(&bars->s_full[1]));
+      if (L::kOStaged && w.n[1] == 1) umma_commit_warp(leader, smem_u32(&bars->q_empty[1]));
     }
     kv_release(k_cnt(0));
     // accumulators of the previous item must have been read out before the first PV overwrites them
@@ -396,6 +403,7 @@ __device__ void fwd_mma_role(const FwdParams& p, uint32_t smem_base, uint32_t tm
         tc_fence_after_sync();
         issue_s(0, kv_addr(k_cnt(j + 1)));
         umma_commit_warp(leader, smem_u32(&bars->s_full[0]));
+        if (L::kOStaged && j + 2 == w.n[0]) umma_commit_warp(leader, smem_u32(&bars->q_empty[0]));
       }
       if (j < w.n[1]) {
         if (!mbar_wait(smem_u32(&bars->p_full[1]), p_cnt[1] & 1, cta_err, 26)) return;
@@ -408,6 +416,7 @@ __device__ void fwd_mma_role(const FwdParams& p, uint32_t smem_base, uint32_t tm
       if (j + 1 < w.n[1]) {
         issue_s(1, kv_addr(k_cnt(j + 1)));
         umma_commit_warp(leader, smem_u32(&bars->s_full[1]));
+        if (L::kOStaged && j + 2 == w.n[1]) umma_commit_warp(leader, smem_u32(&bars->q_empty[1]));
       }
       if (more) kv_release(k_cnt(j + 1));
     }
@@ -578,8 +587,8 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
       }
     }
 
-    // epilogue: O_t (fp32, tensor memory) -> bf16 -> swizzled shared memory (the Q_t buffer,
-    // free once every logits MMA of the item is done) -> TMA store.  Each column group
+    // epilogue: O_t (fp32, tensor memory) -> bf16 -> swizzled shared memory (at D = 128 the Q_t
+    // buffer, free once every logits MMA of the item is done; at D = 64 a buffer of its own) -> TMA store.  Each column group
     // converts its share of the D columns.
 #pragma unroll
     for (int t = 0; t < 2; ++t) {
@@ -587,7 +596,7 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
       if (!mbar_wait(smem_u32(&bars->o_full[t]), it[t] & 1, cta_err, 32 + t)) return;
       ++it[t];
       tc_fence_after_sync();
-      uint8_t* stage = smem + L::kQOff + t * L::kTileBytes;
+      uint8_t* stage = smem + (L::kOStaged ? L::kOOff : L::kQOff) + t * L::kTileBytes;
       constexpr int kECols = D / kGroups;   // accumulator columns per thread
       const uint32_t tO = tmem + 2 * kBN + t * D + lane_off + g * kECols;
       uint32_t o[kECols];
@@ -615,7 +624,7 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
         }
         tc_fence_before_sync();
         mbar_arrive(smem_u32(&bars->o_empty[t]));
-        if (threadIdx.x == 0) mbar_arrive(smem_u32(&bars->q_empty[t]));   // all logits MMAs of the item are done
+        if (!L::kOStaged && threadIdx.x == 0) mbar_arrive(smem_u32(&bars->q_empty[t]));   // all logits MMAs of the item are done
         continue;
       }
       {
@@ -644,8 +653,8 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
           else
             tma_store_3d(tmO, smem_u32(stage + pn * L::kPanelBytes), pn * 64, w.row0 + t * kBM, w.bh);
         tma_commit_group();
-        tma_wait_group_read<0>();
-        mbar_arrive(smem_u32(&bars->q_empty[t]));
+        tma_wait_group_read<0>();   // (with a staging buffer of its own: before the next item's rows are written there)
+        if (!L::kOStaged) mbar_arrive(smem_u32(&bars->q_empty[t]));
       }
     }
   }
