@@ -55,9 +55,13 @@ constexpr float kLog2e = 1.4426950408889634f;
 // Share of the forward's exponentials evaluated on the FMA pipe (every m-th, 0 = none).
 // At D = 128 the shorter instruction stream wins (emulating every 4th measured -6 %); at
 // D = 64, where a tile step has half the tensor work per exponential, unloading the MUFU
-// pipe gains 1-2 %.
+// pipe gains 1-3 % with a causal mask (N = 2048 and 8192) and loses 3-5 % without one
+// (N = 2048 and 8100), so only the causal instantiations do it.
 #ifndef SIGATTN_FWD_EMULATE_D64
 #define SIGATTN_FWD_EMULATE_D64 8
+#endif
+#ifndef SIGATTN_FWD_EMULATE_D64_UNMASKED
+#define SIGATTN_FWD_EMULATE_D64_UNMASKED 0
 #endif
 #ifndef SIGATTN_FWD_EMULATE_D128
 #define SIGATTN_FWD_EMULATE_D128 0
@@ -569,7 +573,8 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
         tmem_ld_cols(tS, sv);
         tmem_wait_ld();
         uint32_t pk[kCols / 2];
-        constexpr int kEmulateEvery = (D == 128) ? SIGATTN_FWD_EMULATE_D128 : SIGATTN_FWD_EMULATE_D64;
+        constexpr int kEmulateEvery = (D == 128) ? SIGATTN_FWD_EMULATE_D128
+                                      : CAUSAL ? SIGATTN_FWD_EMULATE_D64 : SIGATTN_FWD_EMULATE_D64_UNMASKED;
         if (ragged) {
           const int key0 = jk * kBN;
           const bool cut = key0 < key_lo[t] || key0 + kBN > key_hi[t];   // not wholly inside the row's range
