@@ -40,7 +40,7 @@ L2_FLUSH_BYTES = 256 << 20
 # DRAM bytes per launch of the dominant kernel (backward main kernel), dram__bytes_read.sum +
 # dram__bytes_write.sum of one ncu capture per workload (the summaries are committed with the
 # other profile summaries).  None where no capture exists.
-NCU_TRAFFIC_BYTES = {"c4": 429.68e6 + 212.91e6, "c5": 12.753e9 + 7.068e9}
+NCU_TRAFFIC_BYTES = {"c3": 546.96e6 + 297.38e6, "c4": 429.68e6 + 212.91e6, "c5": 12.753e9 + 7.068e9}
 
 
 def load_peaks():
