@@ -795,11 +795,17 @@ template <int D, bool CAUSAL, bool ALIBI, bool DBIAS, int KIND>
 int launch_bwd_variant(const CUtensorMap* maps, const BwdParams& bp, int num_sms, cudaStream_t stream,
                        cudaError_t* cuda_err) {
   auto kernel = sigattn_bwd_bf16_kernel<D, CAUSAL, ALIBI, DBIAS, KIND>;
-  static bool configured = false;
-  if (!configured) {
+  // The shared-memory opt-in is a per-device attribute of the kernel: one bit per device ordinal
+  // (a process may drive several GPUs); ordinals past 63 simply set it on every launch.
+  static std::atomic<unsigned long long> configured{0};
+  int dev = 0;
+  *cuda_err = cudaGetDevice(&dev);
+  if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
+  const unsigned long long bit = (dev >= 0 && dev < 64) ? (1ull << dev) : 0ull;
+  if ((configured.load(std::memory_order_relaxed) & bit) == 0) {
     *cuda_err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<D>::kDynBytes);
     if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
-    configured = true;
+    configured.fetch_or(bit, std::memory_order_relaxed);
   }
   const int grid = bp.n_items < num_sms ? bp.n_items : num_sms;
   kernel<<<grid, kBwdThreads, BwdSmem<D>::kDynBytes, stream>>>(maps[0], maps[1], maps[2], maps[3], maps[4], maps[5],
