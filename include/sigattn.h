@@ -42,6 +42,16 @@
  *   -8 a bounded device-side wait expired in an earlier launch (reported by sigattn_check)
  *   -9 problem too large for sigattn_bwd_static_scratch's built-in scratch
  * Arguments are validated before anything is enqueued.
+ *
+ * Launches in flight.  Some launches hand their work items out dynamically from a device
+ * counter owned by the library: the padded-batch, unpadded-batch, row-factor and accumulating
+ * entry points, sigattn_fwd_decode, and the plain calls when a problem has so few work items
+ * that the library divides them (fewer (batch, head, tile) items than about one per SM).  The
+ * library holds 1024 such counters per kernel family and hands them out round robin, so at
+ * most 1024 of these launches may be in flight at once in one process (over all streams);
+ * beyond that two launches would share a counter and skip or repeat items.  A kernel that
+ * sees its counter advance further than one launch can advance it records a device-side
+ * error, which sigattn_check reports as -8.
  */
 #ifndef SIGATTN_H_
 #define SIGATTN_H_

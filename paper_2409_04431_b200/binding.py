@@ -182,6 +182,43 @@ def _dtype_code(t) -> int:
     raise TypeError(f"sigattn supports bfloat16 and float32 tensors, got {t.dtype}")
 
 
+def _slopes_ptr(alibi_slopes, q):
+    """Device pointer of the per-head slopes after checking what the kernels rely on: float32, on q's
+    device, contiguous, one slope per query head.  Anything else would make a kernel read a host
+    address or past the end of the tensor, so it is refused here, before any launch."""
+    if alibi_slopes is None:
+        return None
+    import torch
+    H = q.shape[1]
+    if (not isinstance(alibi_slopes, torch.Tensor) or not alibi_slopes.is_cuda or alibi_slopes.device != q.device
+            or alibi_slopes.dtype != torch.float32 or not alibi_slopes.is_contiguous() or alibi_slopes.numel() != H):
+        raise ValueError(f"alibi_slopes must be a contiguous float32 CUDA tensor of {H} slopes (one per query head) "
+                         "on q's device")
+    return alibi_slopes.data_ptr()
+
+
+def _host_slopes_ptr(alibi_slopes, H):
+    """Host pointer of the per-head slopes for sigattn_step_host, which copies them to the device itself."""
+    if alibi_slopes is None:
+        return None
+    import torch
+    if (not isinstance(alibi_slopes, torch.Tensor) or alibi_slopes.is_cuda or alibi_slopes.dtype != torch.float32
+            or not alibi_slopes.is_contiguous() or alibi_slopes.numel() != H):
+        raise ValueError(f"sigattn_step_host takes alibi_slopes as a contiguous float32 CPU tensor of {H} slopes")
+    return alibi_slopes.data_ptr()
+
+
+def _ws_ptr(workspace, q):
+    """Device pointer of a caller-supplied scratch tensor: uint8, on q's device, contiguous."""
+    if workspace is None:
+        return None
+    import torch
+    if (not isinstance(workspace, torch.Tensor) or not workspace.is_cuda or workspace.device != q.device
+            or workspace.dtype != torch.uint8 or not workspace.is_contiguous()):
+        raise ValueError("workspace must be a contiguous uint8 CUDA tensor on q's device")
+    return workspace.data_ptr()
+
+
 def _check_same(ts, names):
     import torch
     ref = ts[0]
@@ -234,7 +271,7 @@ def sigattn_fwd(q, k, v, scale, bias, causal=False, alibi_slopes=None, out=None,
     B, H, N, D = q.shape
     with torch.cuda.device(q.device):
         rc = _lib.sigattn_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, H, N, D, float(scale), float(bias),
-                              int(bool(causal)), _ptr(alibi_slopes), _dtype_code(q), _stream_ptr(stream))
+                              int(bool(causal)), _slopes_ptr(alibi_slopes, q), _dtype_code(q), _stream_ptr(stream))
     if rc != 0:
         raise SigattnError(rc)
     return out
@@ -259,8 +296,8 @@ def sigattn_bwd(q, k, v, d_o, scale, bias, causal=False, alibi_slopes=None, work
     ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     with torch.cuda.device(q.device):
         rc = _lib.sigattn_bwd(_ptr(q), _ptr(k), _ptr(v), _ptr(d_o), _ptr(dq), _ptr(dk), _ptr(dv), B, H, N, D,
-                              float(scale), float(bias), int(bool(causal)), _ptr(alibi_slopes), code,
-                              _ptr(workspace), ws_bytes, _stream_ptr(stream))
+                              float(scale), float(bias), int(bool(causal)), _slopes_ptr(alibi_slopes, q), code,
+                              _ws_ptr(workspace, q), ws_bytes, _stream_ptr(stream))
     if rc != 0:
         raise SigattnError(rc)
     return dq, dk, dv
@@ -286,7 +323,7 @@ def sigattn_fwd_bias_vec(q, k, v, scale, bias_bh, causal=False, alibi_slopes=Non
     B, H, N, D = q.shape
     with torch.cuda.device(q.device):
         rc = _lib.sigattn_fwd_bias_vec(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, H, N, D, float(scale),
-                                       _ptr(bias_bh), int(bool(causal)), _ptr(alibi_slopes), _dtype_code(q),
+                                       _ptr(bias_bh), int(bool(causal)), _slopes_ptr(alibi_slopes, q), _dtype_code(q),
                                        _stream_ptr(stream))
     if rc != 0:
         raise SigattnError(rc)
@@ -315,8 +352,8 @@ def sigattn_bwd_bias_vec(q, k, v, d_o, scale, bias_bh, causal=False, alibi_slope
     ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     with torch.cuda.device(q.device):
         rc = _lib.sigattn_bwd_bias_vec(_ptr(q), _ptr(k), _ptr(v), _ptr(d_o), _ptr(dq), _ptr(dk), _ptr(dv), B, H, N, D,
-                                       float(scale), _ptr(bias_bh), int(bool(causal)), _ptr(alibi_slopes), code,
-                                       _ptr(dbias), _ptr(workspace), ws_bytes, _stream_ptr(stream))
+                                       float(scale), _ptr(bias_bh), int(bool(causal)), _slopes_ptr(alibi_slopes, q), code,
+                                       _ptr(dbias), _ws_ptr(workspace, q), ws_bytes, _stream_ptr(stream))
     if rc != 0:
         raise SigattnError(rc)
     return dq, dk, dv, dbias
@@ -349,7 +386,7 @@ def sigattn_fwd_gqa(q, k, v, scale, bias, causal=False, alibi_slopes=None, out=N
     with torch.cuda.device(q.device):
         rc = _lib.sigattn_fwd_gqa(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, H, H_kv, N, D, float(scale),
                                   0.0 if vec else float(bias), _ptr(bias) if vec else None, int(bool(causal)),
-                                  _ptr(alibi_slopes), _dtype_code(q), _stream_ptr(stream))
+                                  _slopes_ptr(alibi_slopes, q), _dtype_code(q), _stream_ptr(stream))
     if rc != 0:
         raise SigattnError(rc)
     return out
@@ -374,7 +411,7 @@ def sigattn_bwd_gqa(q, k, v, d_o, scale, bias, causal=False, alibi_slopes=None, 
     with torch.cuda.device(q.device):
         rc = _lib.sigattn_bwd_gqa(_ptr(q), _ptr(k), _ptr(v), _ptr(d_o), _ptr(dq), _ptr(dk), _ptr(dv), B, H, H_kv, N, D,
                                   float(scale), 0.0 if vec else float(bias), _ptr(bias) if vec else None,
-                                  int(bool(causal)), _ptr(alibi_slopes), code, _ptr(dbias), _ptr(workspace), ws_bytes,
+                                  int(bool(causal)), _slopes_ptr(alibi_slopes, q), code, _ptr(dbias), _ws_ptr(workspace, q), ws_bytes,
                                   _stream_ptr(stream))
     if rc != 0:
         raise SigattnError(rc)
@@ -408,7 +445,7 @@ def sigattn_fwd_nk(q, k, v, scale, bias, causal=False, alibi_slopes=None, out=No
     with torch.cuda.device(q.device):
         rc = _lib.sigattn_fwd_nk(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, H, H_kv, N_q, N_k, D, float(scale),
                                  0.0 if vec else float(bias), _ptr(bias) if vec else None, int(bool(causal)),
-                                 _ptr(alibi_slopes), _dtype_code(q), _stream_ptr(stream))
+                                 _slopes_ptr(alibi_slopes, q), _dtype_code(q), _stream_ptr(stream))
     if rc != 0:
         raise SigattnError(rc)
     return out
@@ -433,7 +470,7 @@ def sigattn_bwd_nk(q, k, v, d_o, scale, bias, causal=False, alibi_slopes=None, w
     with torch.cuda.device(q.device):
         rc = _lib.sigattn_bwd_nk(_ptr(q), _ptr(k), _ptr(v), _ptr(d_o), _ptr(dq), _ptr(dk), _ptr(dv), B, H, H_kv, N_q, N_k,
                                  D, float(scale), 0.0 if vec else float(bias), _ptr(bias) if vec else None,
-                                 int(bool(causal)), _ptr(alibi_slopes), code, _ptr(dbias), _ptr(workspace), ws_bytes,
+                                 int(bool(causal)), _slopes_ptr(alibi_slopes, q), code, _ptr(dbias), _ws_ptr(workspace, q), ws_bytes,
                                  _stream_ptr(stream))
     if rc != 0:
         raise SigattnError(rc)
@@ -456,7 +493,7 @@ def sigattn_fwd_shard(q, k, v, scale, bias, pos0, causal=False, alibi_slopes=Non
     with torch.cuda.device(q.device):
         rc = _lib.sigattn_fwd_shard(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, H, H_kv, N_q, N_k, D, float(scale),
                                     0.0 if vec else float(bias), _ptr(bias) if vec else None, int(bool(causal)),
-                                    int(pos0), _ptr(alibi_slopes), _dtype_code(q), _stream_ptr(stream))
+                                    int(pos0), _slopes_ptr(alibi_slopes, q), _dtype_code(q), _stream_ptr(stream))
     if rc != 0:
         raise SigattnError(rc)
     return out
@@ -481,8 +518,8 @@ def sigattn_bwd_shard(q, k, v, d_o, scale, bias, pos0, causal=False, alibi_slope
     with torch.cuda.device(q.device):
         rc = _lib.sigattn_bwd_shard(_ptr(q), _ptr(k), _ptr(v), _ptr(d_o), _ptr(dq), _ptr(dk), _ptr(dv), B, H, H_kv, N_q,
                                     N_k, D, float(scale), 0.0 if vec else float(bias), _ptr(bias) if vec else None,
-                                    int(bool(causal)), int(pos0), _ptr(alibi_slopes), code, _ptr(dbias),
-                                    _ptr(workspace), ws_bytes, _stream_ptr(stream))
+                                    int(bool(causal)), int(pos0), _slopes_ptr(alibi_slopes, q), code, _ptr(dbias),
+                                    _ws_ptr(workspace, q), ws_bytes, _stream_ptr(stream))
     if rc != 0:
         raise SigattnError(rc)
     return dq, dk, dv, dbias
@@ -511,7 +548,7 @@ def sigattn_fwd_varlen(q, k, v, scale, bias, seqlens, causal=False, alibi_slopes
     with torch.cuda.device(q.device):
         rc = _lib.sigattn_fwd_varlen(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, H, H_kv, N, D, float(scale),
                                      0.0 if vec else float(bias), _ptr(bias) if vec else None, int(bool(causal)),
-                                     _ptr(seqlens), _ptr(alibi_slopes), _dtype_code(q), _stream_ptr(stream))
+                                     _ptr(seqlens), _slopes_ptr(alibi_slopes, q), _dtype_code(q), _stream_ptr(stream))
     if rc != 0:
         raise SigattnError(rc)
     return out
@@ -537,8 +574,8 @@ def sigattn_bwd_varlen(q, k, v, d_o, scale, bias, seqlens, causal=False, alibi_s
     with torch.cuda.device(q.device):
         rc = _lib.sigattn_bwd_varlen(_ptr(q), _ptr(k), _ptr(v), _ptr(d_o), _ptr(dq), _ptr(dk), _ptr(dv), B, H, H_kv, N, D,
                                      float(scale), 0.0 if vec else float(bias), _ptr(bias) if vec else None,
-                                     int(bool(causal)), _ptr(seqlens), _ptr(alibi_slopes), code, _ptr(dbias),
-                                     _ptr(workspace), ws_bytes, _stream_ptr(stream))
+                                     int(bool(causal)), _ptr(seqlens), _slopes_ptr(alibi_slopes, q), code, _ptr(dbias),
+                                     _ws_ptr(workspace, q), ws_bytes, _stream_ptr(stream))
     if rc != 0:
         raise SigattnError(rc)
     return dq, dk, dv, dbias
@@ -574,7 +611,7 @@ def sigattn_fwd_ragged(q, k, v, cu_seqlens, scale, bias, causal=False, alibi_slo
     with torch.cuda.device(q.device):
         rc = _lib.sigattn_fwd_ragged(_ptr(q), _ptr(k), _ptr(v), _ptr(out), H, H_kv, T, D, _ptr(cu_seqlens), n_seqs,
                                      float(scale), 0.0 if vec else float(bias), _ptr(bias) if vec else None,
-                                     int(bool(causal)), _ptr(alibi_slopes), _dtype_code(q), _stream_ptr(stream))
+                                     int(bool(causal)), _slopes_ptr(alibi_slopes, q), _dtype_code(q), _stream_ptr(stream))
     if rc != 0:
         raise SigattnError(rc)
     return out
@@ -596,8 +633,8 @@ def sigattn_bwd_ragged(q, k, v, d_o, cu_seqlens, scale, bias, causal=False, alib
     with torch.cuda.device(q.device):
         rc = _lib.sigattn_bwd_ragged(_ptr(q), _ptr(k), _ptr(v), _ptr(d_o), _ptr(dq), _ptr(dk), _ptr(dv), H, H_kv, T, D,
                                      _ptr(cu_seqlens), n_seqs, float(scale), 0.0 if vec else float(bias),
-                                     _ptr(bias) if vec else None, int(bool(causal)), _ptr(alibi_slopes), code,
-                                     _ptr(dbias), _ptr(workspace), ws_bytes, _stream_ptr(stream))
+                                     _ptr(bias) if vec else None, int(bool(causal)), _slopes_ptr(alibi_slopes, q), code,
+                                     _ptr(dbias), _ws_ptr(workspace, q), ws_bytes, _stream_ptr(stream))
     if rc != 0:
         raise SigattnError(rc)
     return dq, dk, dv, dbias
@@ -617,7 +654,7 @@ def sigattn_fwd_shard_acc(q, k, v, o_acc, scale, bias, pos0, causal=False, alibi
     with torch.cuda.device(q.device):
         rc = _lib.sigattn_fwd_shard_acc(_ptr(q), _ptr(k), _ptr(v), _ptr(o_acc), B, H, H_kv, N_q, N_k, D, float(scale),
                                         0.0 if vec else float(bias), _ptr(bias) if vec else None, int(bool(causal)),
-                                        int(pos0), _ptr(alibi_slopes), _dtype_code(q), _stream_ptr(stream))
+                                        int(pos0), _slopes_ptr(alibi_slopes, q), _dtype_code(q), _stream_ptr(stream))
     if rc != 0:
         raise SigattnError(rc)
 
@@ -640,7 +677,7 @@ def sigattn_bwd_shard_acc(q, k, v, d_o, dq_acc, scale, bias, pos0, causal=False,
     with torch.cuda.device(q.device):
         rc = _lib.sigattn_bwd_shard_acc(_ptr(q), _ptr(k), _ptr(v), _ptr(d_o), _ptr(dq_acc), _ptr(dk), _ptr(dv), B, H,
                                         H_kv, N_q, N_k, D, float(scale), 0.0 if vec else float(bias),
-                                        _ptr(bias) if vec else None, int(bool(causal)), int(pos0), _ptr(alibi_slopes),
+                                        _ptr(bias) if vec else None, int(bool(causal)), int(pos0), _slopes_ptr(alibi_slopes, q),
                                         _dtype_code(q), _ptr(dbias), _stream_ptr(stream))
     if rc != 0:
         raise SigattnError(rc)
@@ -685,7 +722,7 @@ def sigattn_fwd_decode(q, k, v, scale, bias, causal=False, alibi_slopes=None, wo
     with torch.cuda.device(q.device):
         rc = _lib.sigattn_fwd_decode(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, H, H_kv, N_q, N_k, D, float(scale),
                                      0.0 if vec else float(bias), _ptr(bias) if vec else None, int(bool(causal)),
-                                     _ptr(alibi_slopes), code, _ptr(workspace), ws_bytes, _stream_ptr(stream))
+                                     _slopes_ptr(alibi_slopes, q), code, _ws_ptr(workspace, q), ws_bytes, _stream_ptr(stream))
     if rc != 0:
         raise SigattnError(rc)
     return out
@@ -728,7 +765,7 @@ def sigattn_fwd_rowscale(q, k, v, scale, bias, row_scale, causal=False, alibi_sl
     with torch.cuda.device(q.device):
         rc = _lib.sigattn_fwd_rowscale(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, H, H_kv, N_q, N_k, D, float(scale),
                                        0.0 if vec else float(bias), _ptr(bias) if vec else None, int(bool(causal)),
-                                       _ptr(row_scale), _ptr(alibi_slopes), _dtype_code(q), _stream_ptr(stream))
+                                       _ptr(row_scale), _slopes_ptr(alibi_slopes, q), _dtype_code(q), _stream_ptr(stream))
     if rc != 0:
         raise SigattnError(rc)
     return out
@@ -755,7 +792,7 @@ def sigattn_bwd_rowscale(q, k, v, d_o, scale, bias, row_scale, causal=False, ali
         rc = _lib.sigattn_bwd_rowscale(_ptr(q), _ptr(k), _ptr(v), _ptr(d_o), _ptr(dq), _ptr(dk), _ptr(dv), B, H, H_kv,
                                        N_q, N_k, D, float(scale), 0.0 if vec else float(bias),
                                        _ptr(bias) if vec else None, int(bool(causal)), _ptr(row_scale),
-                                       _ptr(alibi_slopes), code, _ptr(dbias), _ptr(workspace), ws_bytes,
+                                       _slopes_ptr(alibi_slopes, q), code, _ptr(dbias), _ws_ptr(workspace, q), ws_bytes,
                                        _stream_ptr(stream))
     if rc != 0:
         raise SigattnError(rc)
@@ -785,7 +822,7 @@ def sigattn_step_host(q, k, v, d_o, o, dq, dk, dv, scale, bias, causal=False, al
         arena = torch.empty(need, dtype=torch.uint8, device="cuda")
     with torch.cuda.device(arena.device):
         rc = _lib.sigattn_step_host(*[_ptr(t) for t in ts], B, H, N, D, float(scale), float(bias),
-                                    int(bool(causal)), _ptr(alibi_slopes), code, _ptr(arena),
+                                    int(bool(causal)), _host_slopes_ptr(alibi_slopes, H), code, _ptr(arena),
                                     arena.numel(), _stream_ptr(stream))
     if rc != 0:
         raise SigattnError(rc)
@@ -821,7 +858,7 @@ def sigattn_bwd_static_scratch(q, k, v, d_o, scale, bias, causal=False, alibi_sl
     with torch.cuda.device(q.device):
         rc = _lib.sigattn_bwd_static_scratch(_ptr(q), _ptr(k), _ptr(v), _ptr(d_o), _ptr(dq), _ptr(dk), _ptr(dv),
                                              B, H, N, D, float(scale), float(bias), int(bool(causal)),
-                                             _ptr(alibi_slopes), _dtype_code(q), _stream_ptr(stream))
+                                             _slopes_ptr(alibi_slopes, q), _dtype_code(q), _stream_ptr(stream))
     if rc != 0:
         raise SigattnError(rc)
     return dq, dk, dv

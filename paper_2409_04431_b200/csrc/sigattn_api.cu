@@ -16,6 +16,7 @@ std::atomic<unsigned long long> g_launches{0};
 thread_local cudaError_t t_last_cuda = cudaSuccess;
 
 constexpr int kMaxDevices = 64;
+std::mutex g_setup_mutex;                    // guards the two per-device tables below
 int* g_status_ptr[kMaxDevices] = {nullptr};
 int g_arch_ok[kMaxDevices] = {0};  // 0 unknown, 1 sm_100, -1 other
 
@@ -43,6 +44,9 @@ int device_setup(int* dev_out, int** status_out) {
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) { t_last_cuda = e; return SIGATTN_ERR_CUDA; }
   if (dev < 0 || dev >= kMaxDevices) return SIGATTN_ERR_ARCH;
+  // Host threads may make their first call on a device together: the tables are filled and read
+  // under one lock, so no reader sees the architecture flag without the status pointer.
+  std::lock_guard<std::mutex> lock(g_setup_mutex);
   if (g_arch_ok[dev] == 0) {
     int major = 0;
     e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
@@ -54,6 +58,7 @@ int device_setup(int* dev_out, int** status_out) {
     g_arch_ok[dev] = (major == 10) ? 1 : -1;
   }
   if (g_arch_ok[dev] != 1) return SIGATTN_ERR_ARCH;
+  if (g_status_ptr[dev] == nullptr) return SIGATTN_ERR_CUDA;   // never launch a kernel that would report to address 0
   *dev_out = dev;
   *status_out = g_status_ptr[dev];
   return SIGATTN_OK;

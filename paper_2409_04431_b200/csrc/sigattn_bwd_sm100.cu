@@ -130,6 +130,10 @@ __device__ __forceinline__ bool bwd_sched_draw(const BwdParams& p, BwdBarriers* 
   const uint32_t slot = round & 1, phase = (round >> 1) & 1;
   if (!mbar_wait(smem_u32(&bars->sched_empty[slot]), phase ^ 1, cta_err, 70)) return false;
   int it = atomicAdd(p.sched_counter, 1);
+  // every thread block draws until its first value >= n_items, so one launch draws n_items + gridDim.x
+  // values in all; a larger value means another launch in flight shares the counter (more launches
+  // overlapping than the library has counters): report it instead of silently skipping or repeating items
+  if (it >= p.n_items + static_cast<int>(gridDim.x)) *cta_err = 76;
   if (it >= p.n_items) it = -1;
   *reinterpret_cast<volatile int*>(&bars->sched_item[slot]) = it;
   mbar_arrive(smem_u32(&bars->sched_full[slot]));
@@ -788,7 +792,7 @@ sigattn_bwd_scale_rows_kernel(const uint4* __restrict__ d_o, const float* __rest
 }
 
 // Work-item counters of the dynamic schedule: one per launch in flight, handed out round robin.
-constexpr int kBwdSchedSlots = 64;
+constexpr int kBwdSchedSlots = 1024;
 __device__ int g_bwd_sched_counters[kBwdSchedSlots];
 
 template <int D, bool CAUSAL, bool ALIBI, bool DBIAS, int KIND>

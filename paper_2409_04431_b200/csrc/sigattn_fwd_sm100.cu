@@ -163,6 +163,10 @@ __device__ __forceinline__ bool sched_draw(const FwdParams& p, FwdBarriers* bars
   const uint32_t slot = round & 1, phase = (round >> 1) & 1;
   if (!mbar_wait(smem_u32(&bars->sched_empty[slot]), phase ^ 1, cta_err, 40)) return false;
   int it = atomicAdd(p.sched_counter, 1);
+  // every thread block draws until its first value >= n_items, so one launch draws n_items + gridDim.x
+  // values in all; a larger value means another launch in flight shares the counter (more launches
+  // overlapping than the library has counters): report it instead of silently skipping or repeating items
+  if (it >= p.n_items + static_cast<int>(gridDim.x)) *cta_err = 46;
   if (it >= p.n_items) it = -1;
   *reinterpret_cast<volatile int*>(&bars->sched_item[slot]) = it;
   mbar_arrive(smem_u32(&bars->sched_full[slot]));
@@ -765,8 +769,9 @@ int choose_key_splits(int base_items, int n_kv, int num_sms) {
 }
 
 // Work-item counters of the dynamic schedule: one per launch in flight, handed out round robin
-// (64 launches may overlap on different streams before two of them share a counter).
-constexpr int kSchedSlots = 64;
+// (1024 launches may overlap on different streams before two of them share a counter; a kernel that
+// sees its counter run past what one launch can draw sets the device status word).
+constexpr int kSchedSlots = 1024;
 __device__ int g_fwd_sched_counters[kSchedSlots];
 
 template <int D, bool CAUSAL, bool ALIBI, int MODE>

@@ -171,3 +171,25 @@ def test_argument_validation_of_the_widened_entry_points(lib):
     conv = sig(lib.sigattn_acc_to_bf16, [vp, vp, c.c_size_t, f32, vp])
     assert conv(p, None, 8, 1.0, None) == -1
     assert conv(p, p, 6, 1.0, None) == -2                                                                 # n not a multiple of 4
+
+
+def test_binding_refuses_slopes_and_workspaces_the_kernels_could_not_read():
+    """The Python wrappers check slopes (float32, CUDA, q's device, one per head) and scratch tensors
+    (uint8, CUDA, q's device) before any launch: a CPU, float64 or short tensor would make a kernel read
+    a host address or past the end, which on a GPU is a fault, not an exception."""
+    import torch
+    from paper_2409_04431_b200 import binding
+    q = torch.zeros(1, 4, 8, 64)
+    for bad in (torch.ones(4), torch.ones(4, dtype=torch.float64), torch.ones(3), [0.5] * 4, np.ones(4, np.float32)):
+        with pytest.raises(ValueError):
+            binding._slopes_ptr(bad, q)       # not on a GPU (and wrong dtype, length or type)
+    assert binding._slopes_ptr(None, q) is None
+    with pytest.raises(ValueError):
+        binding._ws_ptr(torch.zeros(64, dtype=torch.uint8), q)   # host memory
+    assert binding._ws_ptr(None, q) is None
+    # sigattn_step_host is the one entry point that takes the slopes from the host
+    ok = torch.ones(4)
+    assert binding._host_slopes_ptr(ok, 4) == ok.data_ptr()
+    for bad in (torch.ones(4, dtype=torch.float64), torch.ones(5), torch.ones(8)[::2]):
+        with pytest.raises(ValueError):
+            binding._host_slopes_ptr(bad, 4)

@@ -247,12 +247,14 @@ def test_config3_full_launch_sampled_heads():
     _full_size_sampled("c3", [(0, 0), (3, 7), (7, 15)])
 
 
-def test_config4_full_launch_sampled_heads():
-    _full_size_sampled("c4", [(0, 0), (1, 15)])
+def test_config4_full_launch_every_head():
+    """The launch the benchmark times, compared on all 32 (batch, head) pairs: the persistent
+    schedule hands heads to thread blocks by rank, so no head stands in for its neighbours."""
+    _full_size_sampled("c4", [(b, h) for b in range(2) for h in range(16)])
 
 
-def test_config5_full_launch_sampled_head():
-    _full_size_sampled("c5", [(0, 31)])
+def test_config5_full_launch_heads_spread_over_the_schedule():
+    _full_size_sampled("c5", [(0, 0), (0, 10), (0, 21), (0, 31)])
 
 
 def test_non_default_stream_and_back_to_back_calls():
@@ -292,6 +294,24 @@ def test_device_side_argument_errors():
     assert lib.sigattn_fwd(p + 2, p, p, p, 1, 1, 128, 64, 0.125, 0.0, 0, None, 0, None) == -3
     assert lib.sigattn_bwd(p, p, p, p, p, p, p, 1, 1, 128, 64, 0.125, 0.0, 0, None, 0, ws.data_ptr(), 1024, None) == -5
     assert lib.sigattn_bwd(p, p, p, p, p, p, p, 1, 1, 128, 64, 0.125, 0.0, 0, None, 0, ws.data_ptr() + 64, 1 << 19, None) == -3
+    assert sa.sigattn_launch_count() == n0
+    sa.sigattn_check()
+
+
+def test_wrappers_refuse_host_slopes_and_host_workspace():
+    """A CPU slopes tensor, a short one, or a CPU workspace is an error in Python, not a device fault."""
+    import torch
+    import paper_2409_04431_b200 as sa
+    q, k, v, d_o = inputs.random_case(1, 2, 130, 64, seed=2)
+    tq, tk, tv, tdo = (to_device(t, "bf16") for t in (q, k, v, d_o))
+    n0 = sa.sigattn_launch_count()
+    for bad in (torch.ones(2), torch.ones(3, device="cuda"), torch.ones(2, device="cuda", dtype=torch.float64)):
+        with pytest.raises(ValueError):
+            sa.sigattn_fwd(tq, tk, tv, 0.125, -4.0, True, bad)
+        with pytest.raises(ValueError):
+            sa.sigattn_bwd(tq, tk, tv, tdo, 0.125, -4.0, True, bad)
+    with pytest.raises(ValueError):
+        sa.sigattn_bwd(tq, tk, tv, tdo, 0.125, -4.0, True, None, workspace=torch.zeros(1 << 20, dtype=torch.uint8))
     assert sa.sigattn_launch_count() == n0
     sa.sigattn_check()
 

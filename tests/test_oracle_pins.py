@@ -687,18 +687,70 @@ def test_packed_batch_equals_separate_calls(causal):
         oracle.sigattn_fwd(q, k, v, scale, -1.0, causal, cu_seqlens=[0, 5, 3, T])
 
 
-def test_packed_batch_brute_force_with_shared_kv_heads():
-    """Explicit loops over the packed layout with one key/value head for two query heads."""
+@pytest.mark.parametrize("causal", [True, False])
+def test_packed_batch_brute_force_with_shared_kv_heads(causal):
+    """Explicit loops over the packed layout with one key/value head for two query heads:
+    forward, and every gradient of L = sum(O * dO) written out entry by entry (dK and dV of
+    the shared head are sums over both query heads, db is per (sequence, head))."""
     H, D = 2, 2
     cu = [0, 3, 5]
     q, d_o = rnd((1, H, 5, D), 180), rnd((1, H, 5, D), 183)
     k, v = rnd((1, 1, 5, D), 181), rnd((1, 1, 5, D), 182)
     scale, bias = 0.9, np.array([[-0.4, 0.1], [0.6, -1.1]])
-    o = oracle.sigattn_fwd(q, k, v, scale, bias, True, cu_seqlens=cu)
+    slopes = np.array([0.3, 0.0])
+    o = oracle.sigattn_fwd(q, k, v, scale, bias, causal, slopes, cu_seqlens=cu)
+    dq, dk, dv = oracle.sigattn_bwd(q, k, v, d_o, scale, bias, causal, slopes, cu_seqlens=cu)
+    db = oracle.sigattn_bwd_dbias(q, k, v, d_o, scale, bias, causal, slopes, cu_seqlens=cu)
     ref = np.zeros_like(o)
+    rdq, rdk, rdv, rdb = np.zeros_like(q), np.zeros_like(k), np.zeros_like(v), np.zeros((2, H))
     for h in range(H):
         for s in range(2):
             for i in range(cu[s], cu[s + 1]):
-                for j in range(cu[s], i + 1):
-                    ref[0, h, i] += scalar_sigmoid(scale * float(q[0, h, i] @ k[0, 0, j]) + bias[s, h]) * v[0, 0, j]
+                for j in range(cu[s], (i + 1) if causal else cu[s + 1]):
+                    x = scale * float(q[0, h, i] @ k[0, 0, j]) + bias[s, h] - slopes[h] * abs(i - j)
+                    pw = scalar_sigmoid(x)
+                    ref[0, h, i] += pw * v[0, 0, j]
+                    g = pw * (1.0 - pw) * float(d_o[0, h, i] @ v[0, 0, j])   # dL/dx_ij
+                    rdv[0, 0, j] += pw * d_o[0, h, i]
+                    rdq[0, h, i] += scale * g * k[0, 0, j]
+                    rdk[0, 0, j] += scale * g * q[0, h, i]
+                    rdb[s, h] += g
     np.testing.assert_allclose(o, ref, rtol=1e-13, atol=1e-16)
+    for got, want in ((dq, rdq), (dk, rdk), (dv, rdv), (db, rdb)):
+        np.testing.assert_allclose(got, want, rtol=1e-12, atol=1e-15)
+
+
+@pytest.mark.parametrize("causal", [True, False])
+def test_packed_batch_shared_kv_heads_finite_differences(causal):
+    """Central differences of L = sum(O * dO) with respect to every entry of q, of the shared k
+    and v, and of the per-(sequence, head) bias, for a packed batch with H_kv < H (two groups of
+    two query heads, an empty sequence in the middle)."""
+    H, H_kv, D = 4, 2, 3
+    cu = [0, 2, 2, 6]
+    T = cu[-1]
+    q, d_o = rnd((1, H, T, D), 190), rnd((1, H, T, D), 193)
+    k, v = rnd((1, H_kv, T, D), 191), rnd((1, H_kv, T, D), 192)
+    bias = rnd((3, H), 194)
+    slopes = np.array([0.5, 0.25, 0.0, 0.125])
+    scale = 0.6
+
+    def L(bq, bk, bv, bb):
+        return float(np.sum(oracle.sigattn_fwd(bq, bk, bv, scale, bb, causal, slopes, cu_seqlens=cu) * d_o))
+
+    dq, dk, dv = oracle.sigattn_bwd(q, k, v, d_o, scale, bias, causal, slopes, cu_seqlens=cu)
+    db = oracle.sigattn_bwd_dbias(q, k, v, d_o, scale, bias, causal, slopes, cu_seqlens=cu)
+    assert np.all(db[1] == 0.0)
+    h = 1e-6
+    args = [q.copy(), k.copy(), v.copy(), bias.copy()]
+    for which, g in enumerate((dq, dk, dv, db)):
+        fd = np.zeros_like(g)
+        x = args[which]
+        for idx in np.ndindex(*x.shape):
+            old = x[idx]
+            x[idx] = old + h
+            lp = L(*args)
+            x[idx] = old - h
+            lm = L(*args)
+            x[idx] = old
+            fd[idx] = (lp - lm) / (2 * h)
+        assert np.linalg.norm(fd - g) / np.linalg.norm(fd) < 1e-7, which

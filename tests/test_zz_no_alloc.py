@@ -1,14 +1,17 @@
 """sigattn_bwd_static_scratch: the backward for callers that cannot allocate device memory
 (allocator callbacks, real-time loops, plugins whose host forbids allocation after start-up):
 they have no workspace to give sigattn_bwd, so the library keeps the fp32 dQ accumulator in a
-fixed built-in array.  The entry point must give the same gradients as sigattn_bwd, also
-on a second call that finds the array dirty from the first, and must refuse problems that do
-not fit the array.  This file is named to be collected last."""
+fixed built-in array.  The entry point must give the same gradients as sigattn_bwd (and meet
+the float64 oracle at the usual tolerance), also on a second call that finds the array dirty
+from the first, must refuse problems that do not fit the array, and must leave the amount of
+free device memory and the caching allocator's counters exactly as it found them.  This file
+is named to be collected last."""
 import math
 
 import numpy as np
 import pytest
 
+import oracle
 from paper_2409_04431_b200 import inputs
 from parity_util import BF16_MAX_ABS, BF16_REL_FRO, max_abs, rel_fro, to_device, to_host
 
@@ -44,10 +47,25 @@ def test_static_scratch_backward_matches_workspace_backward_twice_in_a_row():
         tq, tk, tv, tdo = (to_device(t, "bf16") for t in (q, k, v, d_o))
         scale, bias = 1 / math.sqrt(D), -math.log(N)
         ref = sa.sigattn_bwd(tq, tk, tv, tdo, scale, bias, causal, sl)
+        ref64 = oracle.sigattn_bwd(q, k, v, d_o, scale, bias, causal, None if sl is None else sl.cpu().numpy())
         out = tuple(torch.full_like(tq, float("nan")) for _ in range(3))
         for call in range(2):
+            # the promise in the name: with the outputs preallocated, the call takes no device memory,
+            # neither from the driver (free bytes) nor from torch's caching allocator (its counters)
+            torch.cuda.synchronize()
+            free0 = torch.cuda.mem_get_info()[0]
+            stats0 = torch.cuda.memory_stats()
             got = sa.sigattn_bwd_static_scratch(tq, tk, tv, tdo, scale, bias, causal, sl, out=out)
             sa.sigattn_check()
+            stats1 = torch.cuda.memory_stats()
+            if call > 0:   # (the very first call on a device may load the module that holds the array)
+                assert torch.cuda.mem_get_info()[0] == free0, "free device memory changed across the call"
+            for key in ("allocation.all.allocated", "segment.all.allocated", "allocated_bytes.all.allocated"):
+                assert stats1[key] == stats0[key], f"caching allocator counter {key} moved"
+            for name, g, r in zip(("dQ", "dK", "dV"), got, ref64):
+                g64 = to_host(g)
+                assert max_abs(g64, r) <= BF16_MAX_ABS, f"{name} call {call} vs oracle"
+                assert rel_fro(g64, r) <= BF16_REL_FRO, f"{name} call {call} vs oracle"
             for name, g, r in zip(("dQ", "dK", "dV"), got, ref):
                 g64, r64 = to_host(g), to_host(r)
                 assert np.all(np.isfinite(g64)), f"{name} call {call}: non-finite"
