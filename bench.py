@@ -37,10 +37,20 @@ UNIT = "TFLOP/s"
 FALLBACK_PEAKS = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0}
 L2_FLUSH_BYTES = 256 << 20
 
-# DRAM bytes per launch of the dominant kernel (backward main kernel), dram__bytes_read.sum +
-# dram__bytes_write.sum of one ncu capture per workload (the summaries are committed with the
-# other profile summaries).  None where no capture exists.
-NCU_TRAFFIC_BYTES = {"c3": 546.96e6 + 297.38e6, "c4": 429.68e6 + 212.91e6, "c5": 12.753e9 + 7.068e9}
+# DRAM bytes per launch of each kernel (dram__bytes_read.sum + dram__bytes_write.sum of one ncu
+# capture per kernel and workload) are kept in a small data file next to the profile summaries
+# they come from, so that a refreshed capture updates the bench line without touching this file.
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "ncu_dram_traffic.json")
+
+
+def ncu_traffic(kernel: str, workload: str):
+    """Measured DRAM bytes per launch of `kernel` ("fwd" or "bwd_main") on `workload`, or None."""
+    try:
+        with open(TRAFFIC_FILE) as f:
+            entry = json.load(f)["kernels"][kernel][workload]
+        return float(entry["dram_bytes_read"]) + float(entry["dram_bytes_write"])
+    except (OSError, KeyError, ValueError, TypeError):
+        return None
 
 
 def load_peaks():
@@ -138,6 +148,15 @@ def run_reference(args, cfg):
     print(json.dumps(line), flush=True)
 
 
+def algorithmic_bytes(cfg):
+    """Compulsory HBM bytes of one forward and of one backward: every [B, H, N, D] tensor once
+    (forward: Q, K, V in, O out; backward: Q, K, V, dO in, dQ, dK, dV out) plus the three passes
+    (clear, accumulate, convert) over the fp32 dQ accumulator."""
+    t = cfg.B * cfg.H * cfg.N * cfg.D
+    e = 2 if cfg.dtype == "bf16" else 4
+    return 4 * t * e, 7 * t * e + 3 * t * 4
+
+
 def workload_config(cfg, n_gpus):
     return {
         "workload": f"{cfg.name}: B={cfg.B} H={cfg.H} N={cfg.N} D={cfg.D} {cfg.dtype} "
@@ -213,6 +232,82 @@ def physical_gpu_index(local_index: int) -> int:
 
 
 # ----------------------------------------------------------------------------- our arm
+
+
+def time_side_workload(sa, torch, dev, cfg, steps, flush, peaks, bias=None, sampler_index=None):
+    """Forward and backward of one further configuration, timed like the headline one: seeded host
+    inputs copied to the device, >= 3 warm-up steps, L2 flushed before every timed step, CUDA events
+    around each pass, clocks sampled while it runs.  Returns the per-pass figures for the bench line."""
+    code = 0 if cfg.dtype == "bf16" else 1
+    bias = cfg.bias if bias is None else bias
+    host = inputs.make_inputs(cfg)
+    q, k, v, d_o = (torch.from_numpy(inputs.f32_to_bf16_bits(x).view(np.int16)).view(torch.bfloat16).to(dev)
+                    for x in host)
+    del host
+    o = torch.empty_like(q)
+    grads = tuple(torch.empty_like(q) for _ in range(3))
+    sl = cfg.slopes()
+    slopes = None if sl is None else torch.from_numpy(sl).to(dev)
+    ws = torch.empty(max(1, sa.sigattn_bwd_workspace_bytes(cfg.B, cfg.H, cfg.N, cfg.D, code)), dtype=torch.uint8,
+                     device=dev)
+    ev = lambda: torch.cuda.Event(enable_timing=True)  # noqa: E731
+    k0, k1 = ev(), ev()
+    k0.record(); k1.record()
+    torch.cuda.synchronize()
+    for _ in range(3):
+        sa.sigattn_fwd(q, k, v, cfg.scale, bias, cfg.causal, slopes, out=o)
+        sa.sigattn_bwd(q, k, v, d_o, cfg.scale, bias, cfg.causal, slopes, workspace=ws, out=grads)
+    sa.sigattn_check()
+    sampler = ClockSampler(sampler_index) if sampler_index is not None else None
+    e0, e1, e2 = [ev() for _ in range(steps)], [ev() for _ in range(steps)], [ev() for _ in range(steps)]
+    torch.cuda.synchronize()
+    launches0 = sa.sigattn_launch_count()
+    if sampler:
+        sampler.start()
+    kern = []
+    for s in range(steps):
+        flush.zero_()
+        e0[s].record()
+        sa.sigattn_fwd(q, k, v, cfg.scale, bias, cfg.causal, slopes, out=o)
+        e1[s].record()
+        timed = s % 4 == 0
+        if timed:
+            sa.sigattn_bwd_set_timing_events(k0, k1)
+        sa.sigattn_bwd(q, k, v, d_o, cfg.scale, bias, cfg.causal, slopes, workspace=ws, out=grads)
+        if timed:
+            sa.sigattn_bwd_set_timing_events(None, None)
+        e2[s].record()
+        if timed:
+            torch.cuda.synchronize()
+            kern.append(k0.elapsed_time(k1))
+    torch.cuda.synchronize()
+    if sampler:
+        sampler.stop_flag.set()
+        sampler.join()
+    sa.sigattn_check()
+    launches = sa.sigattn_launch_count() - launches0
+    t_fwd = float(np.median([e0[s].elapsed_time(e1[s]) for s in range(steps)]))
+    t_bwd = float(np.median([e1[s].elapsed_time(e2[s]) for s in range(steps)]))
+    t_kern = float(np.median(kern))
+    peak, hbm = peaks["bf16_tflops"], peaks["hbm_gbs"]
+    bytes_fwd, bytes_bwd = algorithmic_bytes(cfg)
+    f_fwd, f_bwd = cfg.flops_fwd(), cfg.flops_bwd()
+    out = {
+        "workload": workload_config(cfg, 1)["workload"] if bias == cfg.bias else
+                    workload_config(cfg, 1)["workload"].replace("b=-ln(N)", f"b={bias:g}"),
+        "steps": steps, "timing": "median of per-step CUDA-event times, L2 flushed before every step",
+        "fwd": {"ms": t_fwd, "tflops": f_fwd / t_fwd / 1e9, "frac_of_peak": f_fwd / t_fwd / 1e9 / peak,
+                "hbm_gbs": bytes_fwd / t_fwd / 1e6, "frac_of_hbm_peak": bytes_fwd / t_fwd / 1e6 / hbm},
+        "bwd": {"ms": t_bwd, "tflops": f_bwd / t_bwd / 1e9, "frac_of_peak": f_bwd / t_bwd / 1e9 / peak,
+                "hbm_gbs": bytes_bwd / t_bwd / 1e6, "frac_of_hbm_peak": bytes_bwd / t_bwd / 1e6 / hbm,
+                "main_kernel_ms": t_kern, "main_kernel_tflops": f_bwd / t_kern / 1e9,
+                "main_kernel_frac_of_peak": f_bwd / t_kern / 1e9 / peak},
+        "gpu_launches": int(launches),
+    }
+    if sampler:
+        out["clocks"] = sampler.summary()
+    return out
+
 
 
 def run_ours(args, cfg):
@@ -361,7 +456,16 @@ def run_ours(args, cfg):
                 "peak_source": f"{peak_src} bf16_tflops (burst)", "peak_sustained": peak_sus,
                 "frac_of_sustained_peak": kern_tf / peak_sus, "avg_launch_ms": t_kern,
                 "algorithmic_flops_per_launch": f_bwd,
-                "traffic": NCU_TRAFFIC_BYTES.get(cfg.name),
+                "traffic": ncu_traffic("bwd_main", cfg.name),
+            },
+            # the forward is one launch of one kernel, so its CUDA-event time is the kernel's
+            "roofline_fwd": {
+                "kernel": "sigattn_fwd_bf16_kernel (the forward is this one launch)",
+                "bound": "tensor", "achieved": fwd_tf, "peak": peak, "unit": "TFLOP/s", "frac": fwd_tf / peak,
+                "peak_source": f"{peak_src} bf16_tflops (burst)", "peak_sustained": peak_sus,
+                "frac_of_sustained_peak": fwd_tf / peak_sus, "avg_launch_ms": t_fwd / steps,
+                "algorithmic_flops_per_launch": f_fwd,
+                "traffic": ncu_traffic("fwd", cfg.name),
             },
             "e2e": {"value": world * (f_fwd + f_bwd) / (t_e2e * 1e-3) / 1e12, "unit": UNIT,
                     "ms_per_step": t_e2e, "h2d_bytes_per_step": 4 * tensor_bytes, "d2h_bytes_per_step": 4 * tensor_bytes},
@@ -369,6 +473,25 @@ def run_ours(args, cfg):
             "clocks": sampler.summary(),
             "wall_s_timed_region": wall,
         }
+        if world == 1 and not args.no_side_workloads:
+            # the other bf16 configurations and the exact (two-MUFU) activation path, same timing rules;
+            # reported beside the headline, never folded into `value`
+            del q, k, v, d_o, o, grads, ws, arena
+            torch.cuda.empty_cache()
+            side = {}
+            idx = physical_gpu_index(local)
+            for name in ("c2", "c3", "c5"):
+                if name == cfg.name:
+                    continue
+                c = inputs.CONFIGS[name]
+                side[name] = time_side_workload(sa, torch, dev, c, 30 if name == "c5" else 100, flush, peaks,
+                                                sampler_index=idx)
+                for kern in ("fwd", "bwd_main"):
+                    side[name][kern.split("_")[0]]["ncu_dram_bytes_per_launch"] = ncu_traffic(kern, name)
+            # every logit block on the exact path: same shape as the headline, bias 0 instead of -ln N
+            side[cfg.name + "_exact_path"] = time_side_workload(sa, torch, dev, cfg, 50, flush, peaks, bias=0.0,
+                                                                sampler_index=idx)
+            line["workloads"] = side
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"], _ = oracle_sample(cfg, budget_s=args.cpu_budget)
         print(json.dumps(line), flush=True)
@@ -385,6 +508,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c4", choices=sorted(inputs.CONFIGS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-side-workloads", action="store_true",
+                    help="skip the c2/c3/c5 and exact-path figures that follow the headline measurement")
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     args = ap.parse_args()
     cfg = inputs.CONFIGS[args.workload]
