@@ -163,6 +163,26 @@ SIGATTN_API int sigattn_bwd_bias_vec(const void* q, const void* k, const void* v
                          float* dbias_bh,
                          void* workspace, size_t workspace_bytes, void* stream);
 
+/* sigattn_bwd with the gradient of a learnable temperature.  The paper's temperature variant
+ * (footnote to the list of variants in Section 5; the LayerScale-free ablation of Appendix G.2.2)
+ * computes sigmoid(e^t * Q K^T / sqrt(d) + b) V with a learnable scalar t.  The forward needs no
+ * entry point of its own: pass scale * e^t as `scale`.  This backward does the same and also
+ * returns dL/dt for L = sum(O * dO): with x_ij = scale' q_i k_j + b, dL/dt = sum_ij dS_ij * scale'
+ * q_i k_j = sum_i <Q_i, dQ_i> (the paper prints no formula), one value per (batch, head) in
+ * `dtemp_bh`, a DEVICE pointer to B*H floats, row-major [B][H]; a temperature shared by heads or
+ * sequences gets the sum of their entries.  On the bf16 path the sum is taken in the pass that
+ * converts the fp32 dQ accumulator (from the unrounded dQ, with fp32 atomics per block, so its last
+ * bits depend on the order); on the fp32 path a separate reduction runs after the gradients.
+ * `bias_bh` (NULL: use the scalar `bias`) and `dbias_bh` (NULL: no bias gradient) as in
+ * sigattn_bwd_bias_vec.  Everything else as sigattn_bwd. */
+SIGATTN_API int sigattn_bwd_dtemp(const void* q, const void* k, const void* v, const void* d_o,
+                      void* dq, void* dk, void* dv,
+                      int B, int H, int N, int D,
+                      float scale, float bias, const float* bias_bh, int causal,
+                      const float* alibi_slopes, int dtype,
+                      float* dbias_bh, float* dtemp_bh,
+                      void* workspace, size_t workspace_bytes, void* stream);
+
 /* Multi-query / grouped-query attention (the multi-query ablation of Section 5.1): k and v
  * (and dk, dv) have H_kv heads, [B, H_kv, N, D], with H a multiple of H_kv; query head h
  * reads key/value head h / (H / H_kv), i.e. consecutive query heads share one.  The paper

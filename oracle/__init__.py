@@ -12,6 +12,7 @@ from .sigattn_oracle import (  # noqa: F401
     sigattn_fwd,
     sigattn_bwd,
     sigattn_bwd_dbias,
+    sigattn_bwd_dtemp,
     sigattn_fwd_sequence_form,
     seqlen_norm,
 )

@@ -381,6 +381,28 @@ def sigattn_bwd_dbias(q, k, v, d_o, scale, bias, causal=False, alibi_slopes=None
                     cu_seqlens)[3]
 
 
+def sigattn_bwd_dtemp(q, k, v, d_o, scale, bias, causal=False, alibi_slopes=None):
+    """Gradient of L = sum(O * dO) with respect to a temperature t that multiplies the scaled logit,
+    x_ij = e^t * scale * <q_i, k_j> + b (the learnable temperature of Section 5 / Appendix G.2.2),
+    taken at t = 0: the caller passes scale * e^t as `scale`.  dx_ij/dt = scale <q_i, k_j>, so
+    dt[b, h] = sum_ij dS_ij * scale * <q_i, k_j> with dS = P (1 - P) dP as in sigattn_bwd; the position
+    bias does not depend on t.  Written from the logits, not from dQ.  Plain [B, H, N, D] shapes only.
+
+    Returns float64 [B, H].
+    """
+    q, k, v, d_o = _as_f64(q, k, v, d_o)
+    B, H, N, D = q.shape
+    slopes = _slopes(alibi_slopes, H)
+    bias_bh = _bias_per_head(bias, B, H)
+    dt = np.zeros((B, H), dtype=np.float64)
+    for b in range(B):
+        for h in range(H):
+            p = attention_weights(q[b, h], k[b, h], scale, bias_bh[b, h], causal, slopes[h])
+            ds = p * (1.0 - p) * (d_o[b, h] @ v[b, h].T)
+            dt[b, h] = np.sum(ds * (scale * (q[b, h] @ k[b, h].T)))
+    return dt
+
+
 def sigattn_fwd_sequence_form(q, k, v, scale, n_bias):
     """Second form of the forward, valid at b = -log(n_bias), non-causal, no position
     bias (Eq. 4): y_i = sum_j exp(s_ij) / (exp(s_ij) + n_bias) v_j with s the scaled

@@ -27,6 +27,7 @@ _BINDING_NAMES = (
     "sigattn_selftest_bounded_wait",
     "sigattn_fwd_bias_vec",
     "sigattn_bwd_bias_vec",
+    "sigattn_bwd_dtemp",
     "sigattn_fwd_gqa",
     "sigattn_bwd_gqa",
     "sigattn_fwd_nk",

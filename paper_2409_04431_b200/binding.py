@@ -38,6 +38,10 @@ _lib.sigattn_bwd_bias_vec.restype = _c.c_int
 _lib.sigattn_bwd_bias_vec.argtypes = [_c.c_void_p] * 7 + [_c.c_int] * 4 + [_c.c_float, _c.c_void_p, _c.c_int,
                                                                              _c.c_void_p, _c.c_int, _c.c_void_p,
                                                                              _c.c_void_p, _c.c_size_t, _c.c_void_p]
+_lib.sigattn_bwd_dtemp.restype = _c.c_int
+_lib.sigattn_bwd_dtemp.argtypes = [_c.c_void_p] * 7 + [_c.c_int] * 4 + [_c.c_float, _c.c_float, _c.c_void_p, _c.c_int,
+                                                                          _c.c_void_p, _c.c_int, _c.c_void_p, _c.c_void_p,
+                                                                          _c.c_void_p, _c.c_size_t, _c.c_void_p]
 _lib.sigattn_fwd_gqa.restype = _c.c_int
 _lib.sigattn_fwd_gqa.argtypes = [_c.c_void_p] * 4 + [_c.c_int] * 5 + [_c.c_float, _c.c_float, _c.c_void_p, _c.c_int,
                                                                         _c.c_void_p, _c.c_int, _c.c_void_p]
@@ -132,7 +136,7 @@ EXPORTED = [
     "sigattn_strerror", "sigattn_last_cuda_error", "sigattn_version", "sigattn_launch_count",
     "sigattn_step_host", "sigattn_step_host_arena_bytes", "sigattn_bwd_set_timing_events",
     "sigattn_bwd_static_scratch", "sigattn_bwd_static_scratch_max_elements",
-    "sigattn_selftest_bounded_wait", "sigattn_fwd_bias_vec", "sigattn_bwd_bias_vec",
+    "sigattn_selftest_bounded_wait", "sigattn_fwd_bias_vec", "sigattn_bwd_bias_vec", "sigattn_bwd_dtemp",
     "sigattn_fwd_gqa", "sigattn_bwd_gqa", "sigattn_fwd_nk", "sigattn_bwd_nk",
     "sigattn_fwd_shard", "sigattn_bwd_shard", "sigattn_fwd_varlen", "sigattn_bwd_varlen",
     "sigattn_fwd_rowscale", "sigattn_bwd_rowscale", "sigattn_seqlen_norm",
@@ -357,6 +361,41 @@ def sigattn_bwd_bias_vec(q, k, v, d_o, scale, bias_bh, causal=False, alibi_slope
     if rc != 0:
         raise SigattnError(rc)
     return dq, dk, dv, dbias
+
+
+def sigattn_bwd_dtemp(q, k, v, d_o, scale, bias, causal=False, alibi_slopes=None, want_dbias=False, workspace=None,
+                      out=None, stream=None):
+    """sigattn_bwd plus the gradient of a learnable temperature t in sigmoid(e^t * scale * Q K^T + b):
+    pass scale * e^t as `scale`.  `bias`: a float, or a float32 CUDA tensor [B, H].  Returns
+    (dQ, dK, dV, dtemp, dbias): dtemp is a float32 CUDA tensor [B, H] with sum_i <Q_i, dQ_i> per
+    (batch, head) (sum it for a temperature shared by all heads); dbias as in sigattn_bwd_bias_vec, or
+    None unless `want_dbias`."""
+    import torch
+    _check_same([q, k, v, d_o], ["q", "k", "v", "d_o"])
+    vec = isinstance(bias, torch.Tensor)
+    if vec:
+        _check_bias_vec(bias, q)
+    B, H, N, D = q.shape
+    code = _dtype_code(q)
+    if out is None:
+        dq, dk, dv = torch.empty_like(q), torch.empty_like(q), torch.empty_like(q)
+    else:
+        dq, dk, dv = out
+        _check_same([q, dq, dk, dv], ["q", "dq", "dk", "dv"])
+    dtemp = torch.empty((B, H), dtype=torch.float32, device=q.device)
+    dbias = torch.empty((B, H), dtype=torch.float32, device=q.device) if want_dbias else None
+    need = sigattn_bwd_workspace_bytes(B, H, N, D, code)
+    if workspace is None and need > 0:
+        workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    with torch.cuda.device(q.device):
+        rc = _lib.sigattn_bwd_dtemp(_ptr(q), _ptr(k), _ptr(v), _ptr(d_o), _ptr(dq), _ptr(dk), _ptr(dv), B, H, N, D,
+                                    float(scale), 0.0 if vec else float(bias), _ptr(bias) if vec else None,
+                                    int(bool(causal)), _slopes_ptr(alibi_slopes, q), code, _ptr(dbias), _ptr(dtemp),
+                                    _ws_ptr(workspace, q), ws_bytes, _stream_ptr(stream))
+    if rc != 0:
+        raise SigattnError(rc)
+    return dq, dk, dv, dtemp, dbias
 
 
 def _check_gqa(q, k, v):

@@ -141,8 +141,9 @@ int bwd_any(const void* q, const void* k, const void* v, const void* d_o, void* 
             int H_kv, int N, int N_k, int D, float scale, float bias, const float* bias_vec, float* dbias, int causal,
             const float* alibi_slopes, int dtype, void* workspace, size_t workspace_bytes, void* stream,
             int pos0_given = 0, int pos0 = 0, const int* seqlens = nullptr, const float* row_scale = nullptr,
-            int acc_only = 0, const int* cu_seqlens = nullptr, int n_seqs = 0) {
+            int acc_only = 0, const int* cu_seqlens = nullptr, int n_seqs = 0, float* dtemp = nullptr) {
   if (!q || !k || !v || !d_o || (!dq && !acc_only) || !dk || !dv) return SIGATTN_ERR_NULL;
+  if (dtemp && (reinterpret_cast<uintptr_t>(dtemp) & 3u)) return SIGATTN_ERR_ALIGN;
   if (acc_only && dtype != SIGATTN_DTYPE_BF16) return SIGATTN_ERR_FLAG;
   if (int rc = check_lengths(B, H, H_kv, N, N_k, D, causal, pos0_given, pos0)) return rc;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(d_o) || !aligned16(dq) || !aligned16(dk) ||
@@ -161,7 +162,7 @@ int bwd_any(const void* q, const void* k, const void* v, const void* d_o, void* 
   int* status = nullptr;
   if (int rc = device_setup(&dev, &status)) return rc;
   sigattn::Problem p{B, H, N, D, scale, bias, causal, alibi_slopes, bias_vec, dbias, H_kv, N_k, pos0_given, pos0,
-                     seqlens, row_scale, nullptr, acc_only, cu_seqlens, n_seqs};
+                     seqlens, row_scale, nullptr, acc_only, cu_seqlens, n_seqs, dtemp};
   unsigned long long launches = 0;
   cudaError_t ce = cudaSuccess;
   int rc;
@@ -208,6 +209,17 @@ int sigattn_bwd(const void* q, const void* k, const void* v, const void* d_o, vo
                 void* workspace, size_t workspace_bytes, void* stream) {
   return bwd_any(q, k, v, d_o, dq, dk, dv, B, H, H, N, N, D, scale, bias, nullptr, nullptr, causal, alibi_slopes, dtype,
                  workspace, workspace_bytes, stream);
+}
+
+int sigattn_bwd_dtemp(const void* q, const void* k, const void* v, const void* d_o, void* dq, void* dk, void* dv, int B,
+                      int H, int N, int D, float scale, float bias, const float* bias_bh, int causal,
+                      const float* alibi_slopes, int dtype, float* dbias_bh, float* dtemp_bh, void* workspace,
+                      size_t workspace_bytes, void* stream) {
+  if (!dtemp_bh) return SIGATTN_ERR_NULL;
+  if (bias_bh && (reinterpret_cast<uintptr_t>(bias_bh) & 3u)) return SIGATTN_ERR_ALIGN;
+  if (dbias_bh && (reinterpret_cast<uintptr_t>(dbias_bh) & 3u)) return SIGATTN_ERR_ALIGN;
+  return bwd_any(q, k, v, d_o, dq, dk, dv, B, H, H, N, N, D, scale, bias, bias_bh, dbias_bh, causal, alibi_slopes,
+                 dtype, workspace, workspace_bytes, stream, 0, 0, nullptr, nullptr, 0, nullptr, 0, dtemp_bh);
 }
 
 int sigattn_bwd_bias_vec(const void* q, const void* k, const void* v, const void* d_o, void* dq, void* dk, void* dv,

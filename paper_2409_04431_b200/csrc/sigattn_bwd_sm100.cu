@@ -773,6 +773,40 @@ sigattn_bwd_convert_dq_kernel(const float4* __restrict__ ws, uint2* __restrict__
   }
 }
 
+// The same conversion with the temperature gradient on the side.  With the logits e^t * scale * q k + b
+// (the learnable temperature of Section 5 and Appendix G.2.2; the caller passes scale * e^t as the
+// scale), dL/dt = sum_ij dS_ij * scale' q_i k_j = sum_i <q_i, dQ_i>, because dQ_i = scale' sum_j dS_ij k_j:
+// a reduction of what this pass streams anyway.  grid = (blocks per head, B*H); every block reduces its
+// slice of one head and adds it to dtemp[b*H + h] (fp32 atomics: the last bits depend on the order).
+__global__ void __launch_bounds__(256)
+sigattn_bwd_convert_dq_dtemp_kernel(const float4* __restrict__ ws, const uint2* __restrict__ q, uint2* __restrict__ dq,
+                                    size_t vec4_per_head, float scale, float* __restrict__ dtemp) {
+  const size_t base = static_cast<size_t>(blockIdx.y) * vec4_per_head;
+  const size_t stride = static_cast<size_t>(gridDim.x) * blockDim.x;
+  float sum = 0.0f;
+  for (size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < vec4_per_head; i += stride) {
+    const float4 v = ws[base + i];
+    const uint2 qq = q[base + i];
+    const float g0 = scale * v.x, g1 = scale * v.y, g2 = scale * v.z, g3 = scale * v.w;
+    dq[base + i] = make_uint2(pack_bf16x2(g0, g1), pack_bf16x2(g2, g3));
+    sum = fmaf(g0, __uint_as_float(qq.x << 16), sum);
+    sum = fmaf(g1, __uint_as_float(qq.x & 0xffff0000u), sum);
+    sum = fmaf(g2, __uint_as_float(qq.y << 16), sum);
+    sum = fmaf(g3, __uint_as_float(qq.y & 0xffff0000u), sum);
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+  __shared__ float warp_sums[8];
+  if ((threadIdx.x & 31) == 0) warp_sums[threadIdx.x >> 5] = sum;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float total = 0.0f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) total += warp_sums[w];
+    atomicAdd(dtemp + blockIdx.y, total);
+  }
+}
+
 // Sequence-length normalisation, O = r (P V) with one factor per query row: the whole backward
 // is the plain one on r_i dO_i.  This pass writes bf16(r_i dO_i) for every row ([B*H, N, D]
 // row-major, 8 elements per thread); the main kernel then reads it in place of dO.
@@ -994,8 +1028,22 @@ int launch_bwd_bf16(const void* q, const void* k, const void* v, const void* d_o
 
   if (p.acc_only) return SIGATTN_OK;   // the owner of the accumulator converts once every shard has added
 
-  // step 3: dQ = scale * accumulator, as bf16
+  // step 3: dQ = scale * accumulator, as bf16 (and, on request, the temperature gradient from the same pass)
   const size_t n_vec4 = n_elems / 4;  // D is a multiple of 64
+  if (p.dtemp != nullptr) {
+    *cuda_err = cudaMemsetAsync(p.dtemp, 0, BH * sizeof(float), stream);
+    if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
+    const size_t per_head = static_cast<size_t>(p.N) * p.D / 4;
+    const size_t want = per_head / 256 + 1, cap = (static_cast<size_t>(num_sms) * 8 + BH - 1) / BH;
+    dim3 grid(static_cast<unsigned>(want < cap ? want : (cap < 1 ? 1 : cap)), static_cast<unsigned>(BH));
+    sigattn_bwd_convert_dq_dtemp_kernel<<<grid, 256, 0, stream>>>(static_cast<const float4*>(workspace),
+                                                                  static_cast<const uint2*>(q), static_cast<uint2*>(dq),
+                                                                  per_head, p.scale, p.dtemp);
+    *cuda_err = cudaGetLastError();
+    if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
+    *launches += 1;
+    return SIGATTN_OK;
+  }
   const int blocks = static_cast<int>(n_vec4 / 256 + 1 < static_cast<size_t>(num_sms) * 8 ? n_vec4 / 256 + 1
                                                                                             : static_cast<size_t>(num_sms) * 8);
   sigattn_bwd_convert_dq_kernel<<<blocks, 256, 0, stream>>>(static_cast<const float4*>(workspace),

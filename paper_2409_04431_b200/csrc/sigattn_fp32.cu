@@ -238,6 +238,22 @@ int launch_fwd_fp32(const float* q, const float* k, const float* v, float* o, co
   return *cuda_err == cudaSuccess ? SIGATTN_OK : SIGATTN_ERR_CUDA;
 }
 
+// dtemp[b*H + h] = sum_i <q_i, dq_i> (see the bf16 conversion kernel): one block per (batch, head).
+__global__ void __launch_bounds__(256)
+dtemp_fp32_kernel(const float* __restrict__ q, const float* __restrict__ dq, size_t per_head, float* __restrict__ dtemp) {
+  const size_t base = static_cast<size_t>(blockIdx.x) * per_head;
+  double sum = 0.0;
+  for (size_t i = threadIdx.x; i < per_head; i += blockDim.x) sum += static_cast<double>(q[base + i]) * dq[base + i];
+  __shared__ double part[256];
+  part[threadIdx.x] = sum;
+  __syncthreads();
+  for (int off = 128; off > 0; off >>= 1) {
+    if (static_cast<int>(threadIdx.x) < off) part[threadIdx.x] += part[threadIdx.x + off];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) dtemp[blockIdx.x] = static_cast<float>(part[0]);
+}
+
 int launch_bwd_fp32(const float* q, const float* k, const float* v, const float* d_o, float* dq, float* dk,
                     float* dv, const Problem& p, cudaStream_t stream, unsigned long long* launches,
                     cudaError_t* cuda_err) {
@@ -256,6 +272,10 @@ int launch_bwd_fp32(const float* q, const float* k, const float* v, const float*
                                                          p.query_pos0(), p.seqlens, p.row_scale, p.cu_seqlens,
                                                          p.n_seqs);
   *launches += 2;
+  if (p.dtemp != nullptr) {
+    dtemp_fp32_kernel<<<p.B * p.H, 256, 0, stream>>>(q, dq, static_cast<size_t>(p.N) * p.D, p.dtemp);
+    *launches += 1;
+  }
   *cuda_err = cudaGetLastError();
   return *cuda_err == cudaSuccess ? SIGATTN_OK : SIGATTN_ERR_CUDA;
 }

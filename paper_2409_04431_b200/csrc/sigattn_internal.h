@@ -30,6 +30,8 @@ struct Problem {
                           // (not cleared) and leave dq unwritten.  For key/value shards whose results are summed.
   const int* cu_seqlens;  // batch stored without padding (B = 1): device pointer to n_seqs + 1 row offsets, or nullptr;
   int n_seqs;             // bias_vec and dbias then hold one entry per (sequence, head)
+  float* dtemp;           // backward only: device pointer to B*H floats that receive sum_i <Q_i, dQ_i>, the gradient
+                          // with respect to a temperature t that multiplies the scale as e^t (at t = 0), or nullptr
 };
 
 // Every launcher enqueues on `stream`, adds the number of kernels it launched to

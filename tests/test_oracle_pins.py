@@ -432,6 +432,40 @@ def test_temperature_gradient_is_a_reduction_of_q_and_dq():
     assert abs(float(np.sum(q * dq)) - fd) < 1e-7 * max(1.0, abs(fd))
 
 
+@pytest.mark.parametrize("causal,with_slopes", [(False, False), (True, False), (True, True)])
+def test_temperature_gradient_finite_differences_and_closed_forms(causal, with_slopes):
+    """oracle.sigattn_bwd_dtemp, written from the logits, against (a) central differences in t of
+    L(scale * e^t), one head at a time so that every [b, h] entry is pinned on its own, (b) the
+    reduction sum_i <Q_i, dQ_i> of the independently pinned dQ, (c) the N = 1 closed form."""
+    B, H, N, D = 2, 3, 6, 4
+    q, k, v, d_o = (rnd((B, H, N, D), s) for s in (110, 111, 112, 113))
+    slopes = np.array([0.5, 0.25, 0.125]) if with_slopes else None
+    bias = rnd((B, H), 114)
+    scale, t, hstep = 0.5, 0.3, 1e-6
+    s_t = scale * math.exp(t)
+    dt = oracle.sigattn_bwd_dtemp(q, k, v, d_o, s_t, bias, causal, slopes)
+    assert dt.shape == (B, H)
+    for b in range(B):
+        for h in range(H):
+            sel = (slice(b, b + 1), slice(h, h + 1))
+            sl = None if slopes is None else slopes[h:h + 1]
+
+            def L(tt):
+                o = oracle.sigattn_fwd(q[sel], k[sel], v[sel], scale * math.exp(tt), bias[b, h], causal, sl)
+                return float(np.sum(o * d_o[sel]))
+            fd = (L(t + hstep) - L(t - hstep)) / (2 * hstep)
+            assert abs(dt[b, h] - fd) < 1e-7 * max(1.0, abs(fd)), (b, h)
+    dq, _, _ = oracle.sigattn_bwd(q, k, v, d_o, s_t, bias, causal, slopes)
+    np.testing.assert_allclose(dt, np.sum(q * dq, axis=(2, 3)), rtol=1e-11, atol=1e-14)
+    # N = 1: x = s_t q.k + b, dL/dt = P (1 - P) (dO.v) s_t q.k
+    q1, k1, v1, g1 = (rnd((1, 1, 1, D), s) for s in (115, 116, 117, 118))
+    x = s_t * float(q1[0, 0, 0] @ k1[0, 0, 0]) - 0.7
+    pw = scalar_sigmoid(x)
+    want = pw * (1 - pw) * float(g1[0, 0, 0] @ v1[0, 0, 0]) * s_t * float(q1[0, 0, 0] @ k1[0, 0, 0])
+    got = oracle.sigattn_bwd_dtemp(q1, k1, v1, g1, s_t, -0.7, causal)
+    assert abs(got[0, 0] - want) < 1e-14 * max(1.0, abs(want))
+
+
 # ------------------------------------------------------------------ N_q queries against N_k keys
 
 
