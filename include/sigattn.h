@@ -290,6 +290,30 @@ SIGATTN_API int sigattn_bwd_shard_acc(const void* q, const void* k, const void* 
 
 SIGATTN_API int sigattn_acc_to_bf16(const float* acc, void* out, size_t n, float mul, void* stream);
 
+/* Peer mappings for the accumulating shard calls above (the distributed setting the paper's
+ * Limitations, Appendix A, leave open; no counterpart in its algorithms).  One process per GPU:
+ * the rank that owns a block of query rows keeps the fp32 accumulators for them in its own device
+ * memory, exports them once, and every other rank opens the export and passes the mapped address as
+ * `o_acc` / `dq_acc`.  All three calls are host-side set-up, not stream operations.
+ *
+ * sigattn_peer_export: `dev_ptr` is a device pointer of the calling process (any offset inside a
+ *   cudaMalloc'd allocation, e.g. a framework tensor); `handle` is HOST memory of
+ *   SIGATTN_PEER_HANDLE_BYTES bytes that receives an opaque handle for the allocation that contains
+ *   it, `*offset` the byte offset of dev_ptr inside that allocation.  Both travel to the other
+ *   processes by any host channel.  The memory must stay allocated while any process has it open.
+ * sigattn_peer_open: in ANOTHER process (CUDA cannot open a handle in the process that made it, nor
+ *   twice in one process: keep one export per allocation), with the GPU that will run the shard calls
+ *   current: maps the allocation and returns the device address that corresponds to dev_ptr in
+ *   `*mapped`.  Peer access between the two GPUs is enabled as a side effect if they differ.
+ * sigattn_peer_close: unmaps; `mapped` and `offset` as returned / given to sigattn_peer_open.
+ * Ordering is the caller's: the owner clears its accumulators before anyone adds, and converts them
+ * (sigattn_acc_to_bf16) only after every rank has finished its adding kernels (each rank synchronises
+ * its stream, then all ranks meet at a host barrier).  Errors: SIGATTN_ERR_NULL, SIGATTN_ERR_CUDA. */
+#define SIGATTN_PEER_HANDLE_BYTES 64
+SIGATTN_API int sigattn_peer_export(const void* dev_ptr, void* handle, size_t* offset);
+SIGATTN_API int sigattn_peer_open(const void* handle, size_t offset, void** mapped);
+SIGATTN_API int sigattn_peer_close(void* mapped, size_t offset);
+
 /* Padded batches of sequences of different lengths (the speech batches of Section 5.4, with
  * b = -log n_b per sample through `bias_bh`): `seqlens` is a DEVICE pointer to B int32, 4-byte
  * aligned, read while the kernels run; entry b is the number n_b of rows of batch entry b that

@@ -43,6 +43,9 @@ _BINDING_NAMES = (
     "sigattn_fwd_shard_acc",
     "sigattn_bwd_shard_acc",
     "sigattn_acc_to_bf16",
+    "sigattn_peer_export",
+    "sigattn_peer_open",
+    "sigattn_peer_close",
     "sigattn_fwd_ragged",
     "sigattn_bwd_ragged",
     "sigattn_fwd_decode_workspace_bytes",

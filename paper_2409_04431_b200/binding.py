@@ -42,6 +42,12 @@ _lib.sigattn_bwd_dtemp.restype = _c.c_int
 _lib.sigattn_bwd_dtemp.argtypes = [_c.c_void_p] * 7 + [_c.c_int] * 4 + [_c.c_float, _c.c_float, _c.c_void_p, _c.c_int,
                                                                           _c.c_void_p, _c.c_int, _c.c_void_p, _c.c_void_p,
                                                                           _c.c_void_p, _c.c_size_t, _c.c_void_p]
+_lib.sigattn_peer_export.restype = _c.c_int
+_lib.sigattn_peer_export.argtypes = [_c.c_void_p, _c.c_void_p, _c.POINTER(_c.c_size_t)]
+_lib.sigattn_peer_open.restype = _c.c_int
+_lib.sigattn_peer_open.argtypes = [_c.c_void_p, _c.c_size_t, _c.POINTER(_c.c_void_p)]
+_lib.sigattn_peer_close.restype = _c.c_int
+_lib.sigattn_peer_close.argtypes = [_c.c_void_p, _c.c_size_t]
 _lib.sigattn_fwd_gqa.restype = _c.c_int
 _lib.sigattn_fwd_gqa.argtypes = [_c.c_void_p] * 4 + [_c.c_int] * 5 + [_c.c_float, _c.c_float, _c.c_void_p, _c.c_int,
                                                                         _c.c_void_p, _c.c_int, _c.c_void_p]
@@ -137,6 +143,7 @@ EXPORTED = [
     "sigattn_step_host", "sigattn_step_host_arena_bytes", "sigattn_bwd_set_timing_events",
     "sigattn_bwd_static_scratch", "sigattn_bwd_static_scratch_max_elements",
     "sigattn_selftest_bounded_wait", "sigattn_fwd_bias_vec", "sigattn_bwd_bias_vec", "sigattn_bwd_dtemp",
+    "sigattn_peer_export", "sigattn_peer_open", "sigattn_peer_close",
     "sigattn_fwd_gqa", "sigattn_bwd_gqa", "sigattn_fwd_nk", "sigattn_bwd_nk",
     "sigattn_fwd_shard", "sigattn_bwd_shard", "sigattn_fwd_varlen", "sigattn_bwd_varlen",
     "sigattn_fwd_rowscale", "sigattn_bwd_rowscale", "sigattn_seqlen_norm",
@@ -901,6 +908,40 @@ def sigattn_bwd_static_scratch(q, k, v, d_o, scale, bias, causal=False, alibi_sl
     if rc != 0:
         raise SigattnError(rc)
     return dq, dk, dv
+
+
+PEER_HANDLE_BYTES = 64
+
+
+def sigattn_peer_export(t):
+    """Handle for the allocation that holds CUDA tensor `t` plus the offset of t's first byte in it:
+    (bytes, int), to be sent to the other processes over any host channel (see sigattn_peer_open)."""
+    buf = _c.create_string_buffer(PEER_HANDLE_BYTES)
+    off = _c.c_size_t(0)
+    with __import__("torch").cuda.device(t.device):
+        rc = _lib.sigattn_peer_export(_ptr(t), buf, _c.byref(off))
+    if rc != 0:
+        raise SigattnError(rc)
+    return bytes(buf.raw), int(off.value)
+
+
+def sigattn_peer_open(handle: bytes, offset: int, device=None) -> int:
+    """Map another process's exported allocation on `device` (default: the current one) and return
+    the device address that corresponds to the exported tensor's first byte.  Pass it where the shard
+    calls take an accumulator; close it with sigattn_peer_close(address, offset)."""
+    import torch
+    out = _c.c_void_p(0)
+    with torch.cuda.device(torch.cuda.current_device() if device is None else device):
+        rc = _lib.sigattn_peer_open(handle, int(offset), _c.byref(out))
+    if rc != 0:
+        raise SigattnError(rc)
+    return int(out.value)
+
+
+def sigattn_peer_close(address: int, offset: int) -> None:
+    rc = _lib.sigattn_peer_close(_c.c_void_p(address), int(offset))
+    if rc != 0:
+        raise SigattnError(rc)
 
 
 def sigattn_selftest_bounded_wait(limit_us: int = 2000, stream=None) -> None:

@@ -119,3 +119,59 @@ def kv_sharded_bwd_acc(attend_bwd_acc, q_slices, d_o_slices, query_starts, k_sha
         dk = g[0].float() if dk is None else dk + g[0].float()
         dv = g[1].float() if dv is None else dv + g[1].float()
     return dk, dv
+
+
+class PeerAccumulators:
+    """The fp32 accumulators of all ranks of `group` as this rank can address them: its own tensor,
+    and a peer mapping (an integer device address) of every other rank's.
+
+    Every rank passes the float32 CUDA tensor it owns (zeroed by the caller; any shape, e.g. the O and dQ
+    accumulators of its query rows stacked in one allocation - CUDA can map an allocation only once per
+    process, so give each rank ONE tensor).  The constructor is collective over `group` (any backend that
+    can gather Python objects; the handles are 64 bytes): it exports the local tensor
+    (binding.sigattn_peer_export), gathers all exports and opens the others (binding.sigattn_peer_open) on
+    this rank's current device.  `address(r, byte_offset)` is what the accumulating shard calls take
+    for owner r; `all_added()` orders the conversion after every rank's additions; `close()` unmaps.
+    One process per GPU; on one GPU two processes may share it (the kernels never wait on each other)."""
+
+    def __init__(self, local, group=None):
+        import torch
+        import torch.distributed as dist
+        from . import binding
+
+        if not (isinstance(local, torch.Tensor) and local.is_cuda and local.dtype == torch.float32
+                and local.is_contiguous()):
+            raise ValueError("the local accumulator must be a contiguous float32 CUDA tensor")
+        self.group, self.local = group, local
+        self.rank = dist.get_rank(group) if dist.is_initialized() else 0
+        self.world = dist.get_world_size(group) if dist.is_initialized() else 1
+        self._binding = binding
+        self._opened = {}
+        if self.world == 1:
+            return
+        handle, offset = binding.sigattn_peer_export(local)
+        exports = [None] * self.world
+        dist.all_gather_object(exports, (handle, offset), group=group)
+        for r, (h, off) in enumerate(exports):
+            if r != self.rank:
+                self._opened[r] = (binding.sigattn_peer_open(h, off, local.device), off)
+
+    def address(self, owner: int, byte_offset: int = 0) -> int:
+        """Device address, valid on this rank, of byte `byte_offset` of owner's accumulator tensor."""
+        if owner == self.rank:
+            return self.local.data_ptr() + byte_offset
+        return self._opened[owner][0] + byte_offset
+
+    def all_added(self, stream=None):
+        """Every rank calls this after enqueuing its additions: when it returns on a rank, the adding
+        kernels of ALL ranks have finished, and the rank may convert its own accumulator."""
+        import torch
+        import torch.distributed as dist
+        (torch.cuda.current_stream(self.local.device) if stream is None else stream).synchronize()
+        if self.world > 1:
+            dist.barrier(group=self.group)
+
+    def close(self):
+        for address, off in self._opened.values():
+            self._binding.sigattn_peer_close(address, off)
+        self._opened = {}
