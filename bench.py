@@ -500,18 +500,127 @@ def run_ours(args, cfg):
         dist.destroy_process_group()
 
 
+def run_kvshard(args):
+    """Strong scaling of ONE long causal sequence whose keys and values are sharded over the ranks
+    (workload: the c5 shape; every rank holds all queries and its own contiguous shard of K, V and owns
+    the same range of query rows).  Two arms per step, forward + backward each:
+      unfused  local shard call, then one NCCL all-reduce of the fp32 summands of O and of dQ;
+      fused    the kernels add into the owners' fp32 accumulators through peer mappings, owners convert.
+    Sigmoid attention has no row normalisation, so the summands simply add (no log-sum-exp exchange).
+    One JSON line from rank 0; times are the slowest rank's (CUDA events around each arm)."""
+    import torch
+    import torch.distributed as dist
+
+    import paper_2409_04431_b200 as sa
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+    cfg = inputs.CONFIGS["c5"]
+    B, H, N, D = cfg.B, cfg.H, cfg.N, cfg.D
+    g = torch.Generator(device=dev).manual_seed(20240904)      # the same tensors on every rank
+    q, k, v, d_o = (((torch.randn(B, H, N, D, device=dev, generator=g) * cfg.std).to(torch.bfloat16)) for _ in range(4))
+    owners = [sharding.kv_shard_range(N, world, r) for r in range(world)]
+    mine = owners[rank]
+    ks, vs = k[:, :, mine.start:mine.stop].contiguous(), v[:, :, mine.start:mine.stop].contiguous()
+    q_sl = [q[:, :, r.start:r.stop].contiguous() for r in owners]
+    do_sl = [d_o[:, :, r.start:r.stop].contiguous() for r in owners]
+    starts = [r.start for r in owners]
+    n_own = mine.stop - mine.start
+    acc = torch.zeros((2, B, H, n_own, D), dtype=torch.float32, device=dev)
+    peers = sharding.PeerAccumulators(acc)
+    half = [B * H * (r.stop - r.start) * D * 4 for r in owners]
+    o_addr = [peers.address(r, 0) for r in range(world)]
+    dq_addr = [peers.address(r, half[r]) for r in range(world)]
+    dk, dv = torch.empty_like(ks), torch.empty_like(vs)
+    ws = torch.empty(sa.sigattn_bwd_workspace_bytes(B, H, N, D, 0), dtype=torch.uint8, device=dev)
+    steps, warm = max(1, args.steps), max(3, args.warmup)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def unfused():
+        o = sa.sigattn_fwd_shard(q, ks, vs, cfg.scale, cfg.bias, -mine.start, True).float()
+        dq, gk, gv, _ = sa.sigattn_bwd_shard(q, ks, vs, d_o, cfg.scale, cfg.bias, -mine.start, True, workspace=ws)
+        dq = dq.float()
+        if world > 1:
+            dist.all_reduce(o)
+            dist.all_reduce(dq)
+        return o.to(torch.bfloat16), dq.to(torch.bfloat16), gk, gv
+
+    def fused():
+        acc.zero_()
+        barrier()                                       # every accumulator is clear before anyone adds
+        sharding.kv_sharded_fwd_acc(
+            lambda a, b, c, dst, pos0: sa.sigattn_fwd_shard_acc(a, b, c, dst, cfg.scale, cfg.bias, pos0, True),
+            q_sl, starts, ks, vs, mine.start, o_addr)
+        sharding.kv_sharded_bwd_acc(
+            lambda a, b, c, d, dst, gk, gv, pos0: sa.sigattn_bwd_shard_acc_kv(a, b, c, d, dst, gk, gv, cfg.scale,
+                                                                            cfg.bias, pos0, True),
+            q_sl, do_sl, starts, ks, vs, mine.start, dq_addr, dk, dv)
+        peers.all_added()
+        return sa.sigattn_acc_to_bf16(acc[0]), sa.sigattn_acc_to_bf16(acc[1], cfg.scale), dk, dv
+
+    times = {}
+    for name, fn in (("unfused", unfused), ("fused", fused)):
+        for _ in range(warm):
+            fn()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        barrier()
+        sa.sigattn_check()
+        times[name] = sharding.max_over_ranks([e0.elapsed_time(e1) / steps], device=dev)[0]
+    peers.close()
+    if rank == 0:
+        flops = cfg.flops_fwd() + cfg.flops_bwd()
+        line = {
+            "metric": METRIC, "value": flops / (times["fused"] * 1e-3) / 1e12, "unit": UNIT, "n_gpus": world,
+            "steps": steps, "warmup": warm, "ms_per_step": times["fused"], "higher_is_better": True,
+            "scaling": "strong", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"kvshard: one causal sequence B={B} H={H} N={N} D={D} bf16, keys and values in "
+                                   f"{world} contiguous shards, one fwd+bwd per step", "gpus": world,
+                       "cache": "inputs of 0.5 GB per tensor (larger than L2), no flush"},
+            "fused": {"ms_per_step": times["fused"], "tflops": flops / (times["fused"] * 1e-3) / 1e12,
+                      "how": "kernels add into the owners' fp32 accumulators through peer mappings; host barrier "
+                             "before the owners convert (inside the timed step)"},
+            "unfused": {"ms_per_step": times["unfused"], "tflops": flops / (times["unfused"] * 1e-3) / 1e12,
+                        "how": "local shard kernels, then NCCL all-reduce of the fp32 summands of O and dQ"},
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c4", choices=sorted(inputs.CONFIGS))
+    ap.add_argument("--workload", default="c4", choices=sorted(inputs.CONFIGS) + ["kvshard"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-side-workloads", action="store_true",
                     help="skip the c2/c3/c5 and exact-path figures that follow the headline measurement")
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     args = ap.parse_args()
+    if args.workload == "kvshard":
+        if args.impl == "reference":
+            print(json.dumps({"impl": "reference", "unavailable": "the kvshard workload has no CPU arm; use --workload c5"}))
+            return
+        run_kvshard(args)
+        return
     cfg = inputs.CONFIGS[args.workload]
     if args.impl == "reference":
         run_reference(args, cfg)

@@ -288,6 +288,19 @@ SIGATTN_API int sigattn_bwd_shard_acc(const void* q, const void* k, const void* 
                           const float* alibi_slopes, int dtype,
                           float* dbias_bh, void* stream);
 
+/* sigattn_bwd_shard_acc that also ADDS this call's dK, dV of the shard (bf16 TMA reduce-adds) into
+ * `dk`, `dv` instead of writing them: a rank that holds one key/value shard and the query rows of
+ * several owners calls it once per owner and finds the sums over the owners in dk, dv, with no
+ * arithmetic outside the library.  The caller clears dk and dv before the first call; every call adds
+ * one bf16-rounded summand, so the result carries one rounding per owner and its last bits depend on
+ * the order in which the tiles arrive. */
+SIGATTN_API int sigattn_bwd_shard_acc_kv(const void* q, const void* k, const void* v, const void* d_o,
+                             float* dq_acc, void* dk, void* dv,
+                             int B, int H, int H_kv, int N_q, int N_k, int D,
+                             float scale, float bias, const float* bias_bh, int causal, int pos0,
+                             const float* alibi_slopes, int dtype,
+                             float* dbias_bh, void* stream);
+
 SIGATTN_API int sigattn_acc_to_bf16(const float* acc, void* out, size_t n, float mul, void* stream);
 
 /* Peer mappings for the accumulating shard calls above (the distributed setting the paper's

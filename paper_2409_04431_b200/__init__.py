@@ -42,6 +42,7 @@ _BINDING_NAMES = (
     "sigattn_fwd_decode",
     "sigattn_fwd_shard_acc",
     "sigattn_bwd_shard_acc",
+    "sigattn_bwd_shard_acc_kv",
     "sigattn_acc_to_bf16",
     "sigattn_peer_export",
     "sigattn_peer_open",

@@ -42,6 +42,10 @@ _lib.sigattn_bwd_dtemp.restype = _c.c_int
 _lib.sigattn_bwd_dtemp.argtypes = [_c.c_void_p] * 7 + [_c.c_int] * 4 + [_c.c_float, _c.c_float, _c.c_void_p, _c.c_int,
                                                                           _c.c_void_p, _c.c_int, _c.c_void_p, _c.c_void_p,
                                                                           _c.c_void_p, _c.c_size_t, _c.c_void_p]
+_lib.sigattn_bwd_shard_acc_kv.restype = _c.c_int
+_lib.sigattn_bwd_shard_acc_kv.argtypes = [_c.c_void_p] * 7 + [_c.c_int] * 6 + [_c.c_float, _c.c_float, _c.c_void_p,
+                                                                                 _c.c_int, _c.c_int, _c.c_void_p, _c.c_int,
+                                                                                 _c.c_void_p, _c.c_void_p]
 _lib.sigattn_peer_export.restype = _c.c_int
 _lib.sigattn_peer_export.argtypes = [_c.c_void_p, _c.c_void_p, _c.POINTER(_c.c_size_t)]
 _lib.sigattn_peer_open.restype = _c.c_int
@@ -143,7 +147,7 @@ EXPORTED = [
     "sigattn_step_host", "sigattn_step_host_arena_bytes", "sigattn_bwd_set_timing_events",
     "sigattn_bwd_static_scratch", "sigattn_bwd_static_scratch_max_elements",
     "sigattn_selftest_bounded_wait", "sigattn_fwd_bias_vec", "sigattn_bwd_bias_vec", "sigattn_bwd_dtemp",
-    "sigattn_peer_export", "sigattn_peer_open", "sigattn_peer_close",
+    "sigattn_peer_export", "sigattn_peer_open", "sigattn_peer_close", "sigattn_bwd_shard_acc_kv",
     "sigattn_fwd_gqa", "sigattn_bwd_gqa", "sigattn_fwd_nk", "sigattn_bwd_nk",
     "sigattn_fwd_shard", "sigattn_bwd_shard", "sigattn_fwd_varlen", "sigattn_bwd_varlen",
     "sigattn_fwd_rowscale", "sigattn_bwd_rowscale", "sigattn_seqlen_norm",
@@ -728,6 +732,32 @@ def sigattn_bwd_shard_acc(q, k, v, d_o, dq_acc, scale, bias, pos0, causal=False,
     if rc != 0:
         raise SigattnError(rc)
     return dk, dv, dbias
+
+
+def sigattn_bwd_shard_acc_kv(q, k, v, d_o, dq_acc, dk, dv, scale, bias, pos0, causal=False, alibi_slopes=None,
+                             want_dbias=False, stream=None):
+    """sigattn_bwd_shard_acc that ADDS the shard's dK, dV into the given bf16 tensors `dk`, `dv` (shaped
+    like k, v; cleared by the caller before the first call) instead of returning new ones: the sum over
+    several calls (one per owner of query rows) forms inside the library.  Returns dbias or None."""
+    import torch
+    B, H, H_kv, N_q, N_k, D = _check_nk(q, k, v)
+    _check_same([q, d_o], ["q", "d_o"])
+    _check_same([k, dk, dv], ["k", "dk", "dv"])
+    if isinstance(dq_acc, torch.Tensor) and (dq_acc.dtype != torch.float32 or dq_acc.shape != q.shape
+                                             or not dq_acc.is_contiguous() or not dq_acc.is_cuda):
+        raise ValueError("dq_acc must be a contiguous float32 CUDA tensor shaped like q")
+    vec = isinstance(bias, torch.Tensor)
+    if vec:
+        _check_bias_vec(bias, q)
+    dbias = torch.empty((B, H), dtype=torch.float32, device=q.device) if want_dbias else None
+    with torch.cuda.device(q.device):
+        rc = _lib.sigattn_bwd_shard_acc_kv(_ptr(q), _ptr(k), _ptr(v), _ptr(d_o), _ptr(dq_acc), _ptr(dk), _ptr(dv), B,
+                                           H, H_kv, N_q, N_k, D, float(scale), 0.0 if vec else float(bias),
+                                           _ptr(bias) if vec else None, int(bool(causal)), int(pos0),
+                                           _slopes_ptr(alibi_slopes, q), _dtype_code(q), _ptr(dbias), _stream_ptr(stream))
+    if rc != 0:
+        raise SigattnError(rc)
+    return dbias
 
 
 def sigattn_acc_to_bf16(acc, mul=1.0, out=None, stream=None):

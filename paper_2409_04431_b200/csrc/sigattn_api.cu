@@ -560,6 +560,18 @@ int sigattn_bwd_shard_acc(const void* q, const void* k, const void* v, const voi
                  nullptr, 1);
 }
 
+int sigattn_bwd_shard_acc_kv(const void* q, const void* k, const void* v, const void* d_o, float* dq_acc, void* dk,
+                             void* dv, int B, int H, int H_kv, int N_q, int N_k, int D, float scale, float bias,
+                             const float* bias_bh, int causal, int pos0, const float* alibi_slopes, int dtype,
+                             float* dbias_bh, void* stream) {
+  if (!dq_acc) return SIGATTN_ERR_NULL;
+  if ((reinterpret_cast<uintptr_t>(bias_bh) & 3u) || (reinterpret_cast<uintptr_t>(dbias_bh) & 3u))
+    return SIGATTN_ERR_ALIGN;
+  return bwd_any(q, k, v, d_o, nullptr, dk, dv, B, H, H_kv, N_q, N_k, D, scale, bias, bias_bh, dbias_bh, causal,
+                 alibi_slopes, dtype, dq_acc, sigattn_bwd_workspace_bytes(B, H, N_q, D, dtype), stream, 1, pos0, nullptr,
+                 nullptr, 2);
+}
+
 int sigattn_acc_to_bf16(const float* acc, void* out, size_t n, float mul, void* stream) {
   if (!acc || !out) return SIGATTN_ERR_NULL;
   if (!aligned16(acc) || !aligned16(out)) return SIGATTN_ERR_ALIGN;

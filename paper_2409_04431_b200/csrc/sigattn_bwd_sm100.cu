@@ -91,6 +91,7 @@ struct BwdParams {
   // Few work items with one query head per key/value head (one long sequence, few heads): the query
   // tiles of a key tile are divided over two items (i_split = 2) that add their dK_j, dV_j likewise.
   int i_split;
+  int dkv_add;   // 1: dK_j, dV_j are added (bf16 TMA reduce-adds) into outputs the caller cleared: several calls sum up
   int n_items;
   float scale, scale_log2e, bias_log2e;
   const float* bias_vec;   // one bias per (batch, head) instead of the scalar, or nullptr
@@ -604,7 +605,7 @@ __device__ void bwd_act_role(const BwdParams& p, const CUtensorMap* tmDk, const 
       const CUtensorMap* tm = (wg == 0) ? tmDv : tmDk;
 #pragma unroll
       for (int pn = 0; pn < L::kPanels; ++pn)
-        if (GROUPED && (p.n_sub > 1 || p.i_split > 1))   // the parts add their shares
+        if (GROUPED && (p.n_sub > 1 || p.i_split > 1 || p.dkv_add))   // the parts (or successive calls) add their shares
           tma_reduce_add_3d(tm, smem_u32(stage + pn * L::kPanelBytes), pn * 64, w.j * kT, w.bh);
         else
           tma_store_3d(tm, smem_u32(stage + pn * L::kPanelBytes), pn * 64, w.j * kT, w.bh);
@@ -946,6 +947,7 @@ int launch_bwd_bf16(const void* q, const void* k, const void* v, const void* d_o
         (2 * base_items <= num_sms || (p.causal && base_items <= num_sms && bp.n_tiles >= 16)))
       bp.i_split = 2;
   }
+  bp.dkv_add = p.acc_only == 2 ? 1 : 0;
   bp.n_items = bp.n_tiles_k * bp.BH * bp.n_sub * bp.i_split;
   bp.scale = p.scale;
   bp.scale_log2e = p.scale * kLog2eB;
@@ -960,7 +962,7 @@ int launch_bwd_bf16(const void* q, const void* k, const void* v, const void* d_o
   bp.status = status;
 
   const size_t n_elems = static_cast<size_t>(BH) * p.N * p.D;
-  if (bp.n_sub > 1 || bp.i_split > 1) {   // dK, dV are summed over the parts: clear them first
+  if ((bp.n_sub > 1 || bp.i_split > 1) && !bp.dkv_add) {   // dK, dV are summed over the parts: clear them first
     const size_t kv_bytes = static_cast<size_t>(BH_kv) * p.key_rows() * p.D * 2;
     *cuda_err = cudaMemsetAsync(dk, 0, kv_bytes, stream);
     if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
@@ -1011,7 +1013,7 @@ int launch_bwd_bf16(const void* q, const void* k, const void* v, const void* d_o
                         : launch_bwd_variant<DD, CC, AA, false, KK>(maps, bp, num_sms, stream, cuda_err))
 #define SIGATTN_BWD_CASE(DD, CC, AA)                                                                       \
   rc = (bp.cu_seqlens != nullptr)                  ? SIGATTN_BWD_KIND(DD, CC, AA, 2)                        \
-       : (bp.group > 1 || bp.seqlens != nullptr || bp.i_split > 1) ? SIGATTN_BWD_KIND(DD, CC, AA, 1)        \
+       : (bp.group > 1 || bp.seqlens != nullptr || bp.i_split > 1 || bp.dkv_add) ? SIGATTN_BWD_KIND(DD, CC, AA, 1) \
                                                    : SIGATTN_BWD_KIND(DD, CC, AA, 0)
   if (p.D == 128) {
     if (p.causal) { if (alibi) SIGATTN_BWD_CASE(128, true, true); else SIGATTN_BWD_CASE(128, true, false); }

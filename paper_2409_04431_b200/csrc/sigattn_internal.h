@@ -25,9 +25,10 @@ struct Problem {
   const float* row_scale; // device pointer to N factors, one per query row, applied to O, or nullptr
   float* split_ws;        // forward only: device scratch of B*H*N*D floats that allows splitting the keys of a
                           // head over several thread blocks when there are few queries (decoding), or nullptr
-  int acc_only;           // 1: accumulate and stop.  Forward: add the partial O, fp32, into split_ws (never cleared,
+  int acc_only;           // 1 (or 2): accumulate and stop.  Forward: add the partial O, fp32, into split_ws (never cleared,
                           // never converted; o is not written).  Backward: add the partial dQ into the workspace
                           // (not cleared) and leave dq unwritten.  For key/value shards whose results are summed.
+                          // 2: the backward also ADDS dK, dV (bf16) into outputs the caller cleared.
   const int* cu_seqlens;  // batch stored without padding (B = 1): device pointer to n_seqs + 1 row offsets, or nullptr;
   int n_seqs;             // bias_vec and dbias then hold one entry per (sequence, head)
   float* dtemp;           // backward only: device pointer to B*H floats that receive sum_i <Q_i, dQ_i>, the gradient

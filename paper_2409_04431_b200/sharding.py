@@ -106,18 +106,18 @@ def kv_sharded_fwd_acc(attend_acc, q_slices, query_starts, k_shard, v_shard, key
         attend_acc(q_r, k_shard, v_shard, acc, start - key_start)
 
 
-def kv_sharded_bwd_acc(attend_bwd_acc, q_slices, d_o_slices, query_starts, k_shard, v_shard, key_start: int,
-                       accumulators):
-    """Backward counterpart: dQ summands go into the owners' accumulators; dK and dV of this
-    rank's shard are the sums over the owners' query rows and stay local (float32 here, since
-    several calls contribute).
+def kv_sharded_bwd_acc(attend_bwd_acc_kv, q_slices, d_o_slices, query_starts, k_shard, v_shard, key_start: int,
+                       accumulators, dk, dv):
+    """Backward counterpart: dQ summands go into the owners' accumulators; dK and dV of this rank's
+    shard are sums over the owners' query rows and stay local.  Those sums form inside the library
+    too: `dk`, `dv` (shaped like the shard) are cleared here and every call adds its summand into them.
 
-    attend_bwd_acc(q, k_shard, v_shard, d_o, dq_acc, pos0) -> (dk_shard, dv_shard, ...)."""
-    dk = dv = None
+    attend_bwd_acc_kv(q, k_shard, v_shard, d_o, dq_acc, dk, dv, pos0) is
+    binding.sigattn_bwd_shard_acc_kv with the remaining arguments bound."""
+    dk.zero_()
+    dv.zero_()
     for q_r, do_r, start, acc in zip(q_slices, d_o_slices, query_starts, accumulators):
-        g = attend_bwd_acc(q_r, k_shard, v_shard, do_r, acc, start - key_start)
-        dk = g[0].float() if dk is None else dk + g[0].float()
-        dv = g[1].float() if dv is None else dv + g[1].float()
+        attend_bwd_acc_kv(q_r, k_shard, v_shard, do_r, acc, dk, dv, start - key_start)
     return dk, dv
 
 

@@ -56,14 +56,16 @@ def _worker(rank, world, port, out_dir):
             lambda a, b, c, dst, pos0: sa.sigattn_fwd_shard_acc(a, b, c, dst, SCALE, BIAS, pos0, True, sl),
             q_sl, [r.start for r in owners], ks, vs, mine.start, o_addr)
         dk, dv = sharding.kv_sharded_bwd_acc(
-            lambda a, b, c, d, dst, pos0: sa.sigattn_bwd_shard_acc(a, b, c, d, dst, SCALE, BIAS, pos0, True, sl),
-            q_sl, do_sl, [r.start for r in owners], ks, vs, mine.start, dq_addr)
+            lambda a, b, c, d, dst, gk, gv, pos0: sa.sigattn_bwd_shard_acc_kv(a, b, c, d, dst, gk, gv, SCALE, BIAS, pos0,
+                                                                            True, sl),
+            q_sl, do_sl, [r.start for r in owners], ks, vs, mine.start, dq_addr, torch.empty_like(ks),
+            torch.empty_like(vs))
         peers.all_added()
         o = sa.sigattn_acc_to_bf16(acc[0])
         dq = sa.sigattn_acc_to_bf16(acc[1], SCALE)
         sa.sigattn_check()
         np.savez(os.path.join(out_dir, f"peer{rank}.npz"), o=o.float().cpu().numpy(), dq=dq.float().cpu().numpy(),
-                 dk=dk.cpu().numpy(), dv=dv.cpu().numpy(), lo=mine.start, hi=mine.stop)
+                 dk=dk.float().cpu().numpy(), dv=dv.float().cpu().numpy(), lo=mine.start, hi=mine.stop)
         dist.barrier()                                  # nobody unmaps while another rank still reads
         peers.close()
     finally:

@@ -146,10 +146,11 @@ def test_fused_shard_sum_host_logic_with_shared_accumulators():
     def attend_acc(a, b, c, acc, pos0):
         acc += torch.from_numpy(oracle.sigattn_fwd(a.numpy(), b.numpy(), c.numpy(), scale, bias, True, slopes, pos0=pos0))
 
-    def attend_bwd_acc(a, b, c, d, acc, pos0):
+    def attend_bwd_acc(a, b, c, d, acc, dk_sum, dv_sum, pos0):
         dq, dk, dv = oracle.sigattn_bwd(a.numpy(), b.numpy(), c.numpy(), d.numpy(), scale, bias, True, slopes, pos0=pos0)
         acc += torch.from_numpy(dq)
-        return torch.from_numpy(dk), torch.from_numpy(dv)
+        dk_sum += torch.from_numpy(dk)
+        dv_sum += torch.from_numpy(dv)
 
     owners = [sharding.kv_shard_range(N, world, r) for r in range(world)]
     cut = lambda t, r: torch.from_numpy(np.ascontiguousarray(t[:, :, r.start:r.stop]))
@@ -161,12 +162,13 @@ def test_fused_shard_sum_host_logic_with_shared_accumulators():
     for rank in range(world):
         rows = sharding.kv_shard_range(N, world, rank)
         sharding.kv_sharded_fwd_acc(attend_acc, q_sl, starts, cut(k, rows), cut(v, rows), rows.start, o_acc)
-        g = sharding.kv_sharded_bwd_acc(attend_bwd_acc, q_sl, do_sl, starts, cut(k, rows), cut(v, rows), rows.start,
-                                        dq_acc)
+        ks, vs = cut(k, rows), cut(v, rows)
+        g = sharding.kv_sharded_bwd_acc(attend_bwd_acc, q_sl, do_sl, starts, ks, vs, rows.start, dq_acc,
+                                        torch.full_like(ks, 7.0), torch.full_like(vs, 7.0))   # (cleared by the helper)
         dk[:, :, rows.start:rows.stop], dv[:, :, rows.start:rows.stop] = g[0].numpy(), g[1].numpy()
     ref_o = oracle.sigattn_fwd(q, k, v, scale, bias, True, slopes)
     ref = oracle.sigattn_bwd(q, k, v, d_o, scale, bias, True, slopes)
     np.testing.assert_allclose(torch.cat(o_acc, dim=2).numpy(), ref_o, rtol=1e-12, atol=1e-14)
     np.testing.assert_allclose(torch.cat(dq_acc, dim=2).numpy(), ref[0], rtol=1e-12, atol=1e-14)
-    np.testing.assert_allclose(dk, ref[1], rtol=1e-6, atol=1e-7)      # the helper sums dK, dV in float32
-    np.testing.assert_allclose(dv, ref[2], rtol=1e-6, atol=1e-7)
+    np.testing.assert_allclose(dk, ref[1], rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(dv, ref[2], rtol=1e-12, atol=1e-14)
