@@ -379,6 +379,13 @@ SIGATTN_API int sigattn_bwd_ragged(const void* q, const void* k, const void* v, 
                        float* dbias_sh,
                        void* workspace, size_t workspace_bytes, void* stream);
 
+/* The ragged calls read `cu_seqlens` on the device and trust it (offsets that do not rise from 0 to T
+ * give wrong results, never out-of-range accesses).  A caller that still holds the offsets on the HOST
+ * can have them checked before the launch: `host_cu_seqlens` is a host pointer to n_seqs + 1 int32;
+ * returns 0 if they start at 0, never decrease and end at T, SIGATTN_ERR_SHAPE otherwise.  No device
+ * work.  No counterpart in the paper. */
+SIGATTN_API int sigattn_check_cu_seqlens(const int* host_cu_seqlens, int n_seqs, int T);
+
 /* Sequence-length normalisation (Appendix G, the ablation that compares the bias b = -log n with
  * the scaling n^-alpha sigma(Q K^T / sqrt(d)) V and its causal form, the equation labelled
  * "ar_seq_len_normalization"): O_i = r_i sum_j P_ij V_j with one factor r_i per query row, shared by

@@ -49,6 +49,7 @@ _BINDING_NAMES = (
     "sigattn_peer_close",
     "sigattn_fwd_ragged",
     "sigattn_bwd_ragged",
+    "sigattn_check_cu_seqlens",
     "sigattn_fwd_decode_workspace_bytes",
     "lib",
 )

@@ -46,6 +46,8 @@ _lib.sigattn_bwd_shard_acc_kv.restype = _c.c_int
 _lib.sigattn_bwd_shard_acc_kv.argtypes = [_c.c_void_p] * 7 + [_c.c_int] * 6 + [_c.c_float, _c.c_float, _c.c_void_p,
                                                                                  _c.c_int, _c.c_int, _c.c_void_p, _c.c_int,
                                                                                  _c.c_void_p, _c.c_void_p]
+_lib.sigattn_check_cu_seqlens.restype = _c.c_int
+_lib.sigattn_check_cu_seqlens.argtypes = [_c.c_void_p, _c.c_int, _c.c_int]
 _lib.sigattn_peer_export.restype = _c.c_int
 _lib.sigattn_peer_export.argtypes = [_c.c_void_p, _c.c_void_p, _c.POINTER(_c.c_size_t)]
 _lib.sigattn_peer_open.restype = _c.c_int
@@ -147,7 +149,7 @@ EXPORTED = [
     "sigattn_step_host", "sigattn_step_host_arena_bytes", "sigattn_bwd_set_timing_events",
     "sigattn_bwd_static_scratch", "sigattn_bwd_static_scratch_max_elements",
     "sigattn_selftest_bounded_wait", "sigattn_fwd_bias_vec", "sigattn_bwd_bias_vec", "sigattn_bwd_dtemp",
-    "sigattn_peer_export", "sigattn_peer_open", "sigattn_peer_close", "sigattn_bwd_shard_acc_kv",
+    "sigattn_peer_export", "sigattn_peer_open", "sigattn_peer_close", "sigattn_bwd_shard_acc_kv", "sigattn_check_cu_seqlens",
     "sigattn_fwd_gqa", "sigattn_bwd_gqa", "sigattn_fwd_nk", "sigattn_bwd_nk",
     "sigattn_fwd_shard", "sigattn_bwd_shard", "sigattn_fwd_varlen", "sigattn_bwd_varlen",
     "sigattn_fwd_rowscale", "sigattn_bwd_rowscale", "sigattn_seqlen_norm",
@@ -938,6 +940,19 @@ def sigattn_bwd_static_scratch(q, k, v, d_o, scale, bias, causal=False, alibi_sl
     if rc != 0:
         raise SigattnError(rc)
     return dq, dk, dv
+
+
+def sigattn_check_cu_seqlens(cu_seqlens_host, T: int) -> None:
+    """Raise SigattnError(-2) unless the HOST int32 tensor `cu_seqlens_host` (n_seqs + 1 offsets) starts at 0,
+    never decreases and ends at T.  The ragged kernels trust the device copy; this is the check a caller
+    can run on its host copy before launching."""
+    import torch
+    if (not isinstance(cu_seqlens_host, torch.Tensor) or cu_seqlens_host.is_cuda or cu_seqlens_host.dtype != torch.int32
+            or not cu_seqlens_host.is_contiguous() or cu_seqlens_host.numel() < 2):
+        raise ValueError("cu_seqlens_host must be a contiguous int32 CPU tensor of n_seqs + 1 offsets")
+    rc = _lib.sigattn_check_cu_seqlens(cu_seqlens_host.data_ptr(), cu_seqlens_host.numel() - 1, int(T))
+    if rc != 0:
+        raise SigattnError(rc)
 
 
 PEER_HANDLE_BYTES = 64

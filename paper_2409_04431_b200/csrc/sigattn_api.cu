@@ -572,6 +572,15 @@ int sigattn_bwd_shard_acc_kv(const void* q, const void* k, const void* v, const 
                  nullptr, 2);
 }
 
+int sigattn_check_cu_seqlens(const int* host_cu_seqlens, int n_seqs, int T) {
+  if (!host_cu_seqlens) return SIGATTN_ERR_NULL;
+  if (n_seqs < 1 || T < 1) return SIGATTN_ERR_SHAPE;
+  if (host_cu_seqlens[0] != 0 || host_cu_seqlens[n_seqs] != T) return SIGATTN_ERR_SHAPE;
+  for (int s = 0; s < n_seqs; ++s)
+    if (host_cu_seqlens[s + 1] < host_cu_seqlens[s]) return SIGATTN_ERR_SHAPE;
+  return SIGATTN_OK;
+}
+
 int sigattn_acc_to_bf16(const float* acc, void* out, size_t n, float mul, void* stream) {
   if (!acc || !out) return SIGATTN_ERR_NULL;
   if (!aligned16(acc) || !aligned16(out)) return SIGATTN_ERR_ALIGN;

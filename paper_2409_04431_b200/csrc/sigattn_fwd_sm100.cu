@@ -514,7 +514,8 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
     const Item w = decode_item<CAUSAL>(p, item);
     // Slope, bias and the position of this thread's query row: per item, or with packed heads
     // per row and tile (index 1 of the arrays is only used then).
-    float slope_t[2] = {0.0f, 0.0f}, bias_t[2], pos_t[2];
+    float slope_t[2] = {0.0f, 0.0f}, bias_t[2];
+    int pos_t[2];   // positions stay integers: shards of very long sequences put them beyond 2^24
     if (PACKED) {
 #pragma unroll
       for (int t = 0; t < 2; ++t) {
@@ -523,12 +524,12 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
         const int head = w.bh * p.pack_group + g_head;               // (b * H_kv + h_kv) * group + g = b * H + h
         if (ALIBI) slope_t[t] = p.slopes[head % (p.H * p.pack_group)] * kLog2e;
         bias_t[t] = p.bias_vec ? __ldg(p.bias_vec + head) * kLog2e : p.bias_log2e;
-        pos_t[t] = static_cast<float>(r - g_head * p.pack_rows + p.pos0);
+        pos_t[t] = r - g_head * p.pack_rows + p.pos0;
       }
     } else {
       if (ALIBI) slope_t[0] = p.slopes[w.bh % p.H] * kLog2e;
       bias_t[0] = p.bias_vec ? __ldg(p.bias_vec + w.bh) * kLog2e : p.bias_log2e;
-      pos_t[0] = static_cast<float>(w.row0 + tid + p.pos0);
+      pos_t[0] = w.row0 + tid + p.pos0;
     }
     // Batch without padding: the keys [key_lo, key_hi) this thread's row may see in each tile (its own
     // sequence, cut at the row itself when causal) and the bias of its sequence and head.
@@ -558,7 +559,8 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
         tc_fence_after_sync();
         const int jk = (PACKED || GENERAL) ? w.j0 + j : j;   // key tile (split keys, unpadded batches: items start later)
         // position of this thread's query relative to the first key of the tile
-        const float row_rel = (PACKED ? pos_t[t] : pos_t[0] + static_cast<float>(t * kBM)) - static_cast<float>(jk * kBN);
+        // (formed in integers; only the small tile-relative difference is converted)
+        const float row_rel = static_cast<float>((PACKED ? pos_t[t] : pos_t[0] + t * kBM) - jk * kBN);
         // the mask cuts through every key tile that reaches beyond the position of the tile's
         // first row: the last one, and with pos0 not a multiple of 128 also the one before
         // (packed rows: a tile may hold a head's first query, at position pos0)

@@ -193,3 +193,19 @@ def test_binding_refuses_slopes_and_workspaces_the_kernels_could_not_read():
     for bad in (torch.ones(4, dtype=torch.float64), torch.ones(5), torch.ones(8)[::2]):
         with pytest.raises(ValueError):
             binding._host_slopes_ptr(bad, 4)
+
+
+def test_host_side_check_of_row_offsets(lib):
+    import ctypes as c
+    lib.sigattn_check_cu_seqlens.restype, lib.sigattn_check_cu_seqlens.argtypes = c.c_int, [c.c_void_p, c.c_int, c.c_int]
+    ok = np.array([0, 3, 3, 10], dtype=np.int32)
+    assert lib.sigattn_check_cu_seqlens(ok.ctypes.data, 3, 10) == 0
+    assert lib.sigattn_check_cu_seqlens(ok.ctypes.data, 3, 11) == -2                      # does not end at T
+    assert lib.sigattn_check_cu_seqlens(np.array([1, 3, 10], np.int32).ctypes.data, 2, 10) == -2   # does not start at 0
+    assert lib.sigattn_check_cu_seqlens(np.array([0, 7, 5, 10], np.int32).ctypes.data, 3, 10) == -2   # decreases
+    assert lib.sigattn_check_cu_seqlens(None, 3, 10) == -1
+    import torch
+    from paper_2409_04431_b200 import binding
+    binding.sigattn_check_cu_seqlens(torch.tensor([0, 4, 9], dtype=torch.int32), 9)
+    with pytest.raises(binding.SigattnError):
+        binding.sigattn_check_cu_seqlens(torch.tensor([0, 9, 4, 9], dtype=torch.int32), 9)
