@@ -50,9 +50,11 @@ struct BwdSmem {
   static constexpr int kTileBytes = kPanels * kPanelBytes;  // a K, V, Q or dO tile
   static constexpr int kKOff = 0;
   static constexpr int kVOff = kTileBytes;
-  static constexpr int kQOff = 2 * kTileBytes;              // two stages
-  static constexpr int kDoOff = 4 * kTileBytes;             // one stage
-  static constexpr int kDsOff = 5 * kTileBytes;             // dS^T, 128 x 128 bf16 = two panels
+  // Q stages: two at D = 128 (shared memory is full); three at D = 64, where S^T runs two steps ahead
+  static constexpr int kQStages = (D == 64) ? 3 : 2;
+  static constexpr int kQOff = 2 * kTileBytes;
+  static constexpr int kDoOff = (2 + kQStages) * kTileBytes;   // one stage
+  static constexpr int kDsOff = (3 + kQStages) * kTileBytes;   // dS^T, 128 x 128 bf16 = two panels
   static constexpr int kDqOff = kDsOff + 2 * kPanelBytes;   // two fp32 staging boxes of 128 x 32
   static constexpr int kTotal = kDqOff + 2 * kPanelBytes;
   static constexpr int kDynBytes = kTotal + 1024;
@@ -60,11 +62,13 @@ struct BwdSmem {
 
 struct BwdBarriers {
   uint64_t kv_full, kv_empty;
-  uint64_t q_full[2], q_empty[2];
+  uint64_t q_full[3], q_empty[3];
   uint64_t do_full, do_empty;
-  uint64_t s_full, dp_full;
-  uint64_t p_ready, ds_ready;
-  uint64_t dq_full, dq_empty;
+  // s_full, p_ready, dq_full, dq_empty: one per region of tensor memory that holds S^T / P^T (see BwdTmem);
+  // a region's barriers flip once per use of that region
+  uint64_t s_full[2], dp_full;
+  uint64_t p_ready[2], ds_ready;
+  uint64_t dq_full[2], dq_empty[2];
   uint64_t dkv_full, dkv_empty;
   // dynamic schedule (batches without padding): the TMA thread draws the next work item from a
   // global counter and hands it to the other roles through this two-slot ring
@@ -222,13 +226,25 @@ __device__ __forceinline__ BwdItem decode_bwd_item(const BwdParams& p, int item)
   return w;
 }
 
-// TMEM column map (fp32 columns): region A = S^T / P^T, region B = dP^T / dQ.
+// TMEM column map (fp32 columns).
+// D = 128: region A = S^T / P^T, region B = dP^T / dS^T / dQ, then dV and dK: 4 x 128 columns, tensor memory
+// is full.  S^T(i+1) has to wait for dV(i), which reads P^T(i) from A, and dP^T(i+1) for the drain of dQ(i).
+// D = 64: dV and dK take 64 columns each and 128 are left over.  They make a second region A: steps
+// alternate between A0 and A1, S^T runs two steps ahead of the activation, and dQ(i) is written over the
+// first 64 columns of the step's own region A (its P^T has been consumed by dV(i), which the same thread
+// issued earlier) so that region B is free for dP^T(i+1) at once.  S^T(i+2) waits for the drain of dQ(i).
 template <int D>
 struct BwdTmem {
-  static constexpr uint32_t kA = 0;
+  static constexpr bool kTwoA = (D == 64);
   static constexpr uint32_t kB = 128;
   static constexpr uint32_t kDv = 256;
   static constexpr uint32_t kDk = 256 + D;
+  // region A of (global) step `step`, its index, and how often that region has been used before
+  __device__ static __forceinline__ uint32_t a_col(uint32_t step) { return (kTwoA && (step & 1)) ? 384u : 0u; }
+  __device__ static __forceinline__ uint32_t r_index(uint32_t step) { return kTwoA ? (step & 1) : 0u; }
+  __device__ static __forceinline__ uint32_t r_use(uint32_t step) { return kTwoA ? (step >> 1) : step; }
+  // where dQ of that step is accumulated
+  __device__ static __forceinline__ uint32_t dq_col(uint32_t step) { return kTwoA ? a_col(step) : kB; }
 };
 
 // ------------------------------------------------------------------ producer
@@ -244,7 +260,7 @@ __device__ void bwd_load_role(const BwdParams& p, const CUtensorMap* tmQ, const 
     for (int pn = 0; pn < L::kPanels; ++pn) tma_load_3d(dst + pn * L::kPanelBytes, tm, bar, pn * 64, row, bh);
   };
   auto load_q = [&](int i, int bh) -> bool {
-    const uint32_t st = q_cnt & 1, ph = (q_cnt >> 1) & 1;
+    const uint32_t st = q_cnt % L::kQStages, ph = (q_cnt / L::kQStages) & 1;
     if (!mbar_wait(smem_u32(&bars->q_empty[st]), ph ^ 1, cta_err, 40)) return false;
     const uint32_t bar = smem_u32(&bars->q_full[st]);
     mbar_arrive_expect_tx(bar, L::kTileBytes);
@@ -280,11 +296,19 @@ __device__ void bwd_load_role(const BwdParams& p, const CUtensorMap* tmQ, const 
       load_tile(tmV, smem_base + L::kVOff, bar, w.j * kT, w.bh);
     }
     ++item_cnt;
-    for (int g = 0; g < (GROUPED ? p.heads_per_sub : 1); ++g) {
-      for (int it = (g == 0 ? 1 : 0); it < w.n; ++it) {
-        if (!load_q(w.i_begin + it, w.bh_q0 + g)) return;
-        if (!load_do(w.i_begin + it, w.bh_q0 + g)) return;
-      }
+    // The remaining steps, head by head.  With two regions A (D = 64) S^T runs a step further ahead than
+    // dP^T, so Q stays one tile ahead of dO: dO(s) can only be loaded after dV(s-1), and S^T(s+1) is issued
+    // before that product's inputs exist.
+    constexpr int lead = BwdTmem<D>::kTwoA ? 1 : 0;
+    auto load_step = [&](int s, bool is_q) -> bool {
+      const int g = GROUPED ? s / w.n : 0;
+      const int i = w.i_begin + (s - g * w.n), bh = w.bh_q0 + g;
+      return is_q ? load_q(i, bh) : load_do(i, bh);
+    };
+    for (int q_next = 1, do_next = 1; do_next < w.steps; ++do_next) {
+      for (; q_next < w.steps && q_next <= do_next + lead; ++q_next)
+        if (!load_step(q_next, true)) return;
+      if (!load_step(do_next, false)) return;
     }
   }
 }
@@ -318,10 +342,37 @@ __device__ void bwd_mma_role(const BwdParams& p, uint32_t smem_base, uint32_t tm
   const uint64_t dDo_mn = make_smem_desc_sw128(sDo, L::kPanelBytes, 1024);  // dO_i, MN-major (dV)
   const uint64_t dK_mn = make_smem_desc_sw128(sK, L::kPanelBytes, 1024);    // K_j, MN-major (dQ)
   const uint64_t dDs_mn = make_smem_desc_sw128(sDs, L::kPanelBytes, 1024);  // dS^T, MN-major (dQ)
-  const uint64_t dQ_k[2] = {make_smem_desc_sw128(smem_base + L::kQOff, 16, 1024),
-                            make_smem_desc_sw128(smem_base + L::kQOff + L::kTileBytes, 16, 1024)};
-  const uint64_t dQ_mn[2] = {make_smem_desc_sw128(smem_base + L::kQOff, L::kPanelBytes, 1024),
-                             make_smem_desc_sw128(smem_base + L::kQOff + L::kTileBytes, L::kPanelBytes, 1024)};
+  uint64_t dQ_k[L::kQStages], dQ_mn[L::kQStages];
+#pragma unroll
+  for (int st = 0; st < L::kQStages; ++st) {
+    dQ_k[st] = make_smem_desc_sw128(smem_base + L::kQOff + st * L::kTileBytes, 16, 1024);                 // S^T
+    dQ_mn[st] = make_smem_desc_sw128(smem_base + L::kQOff + st * L::kTileBytes, L::kPanelBytes, 1024);    // dK
+  }
+  auto q_stage = [](uint32_t cnt) -> uint32_t { return cnt % L::kQStages; };
+  auto q_phase = [](uint32_t cnt) -> uint32_t { return (cnt / L::kQStages) & 1; };
+  // S^T of global step `step` from the Q tile with running number `qn`.  D = 64: the step's region A last
+  // held dQ of two steps earlier, which the drain group must have read.
+  auto issue_s = [&](uint32_t step, uint32_t qn, int where) -> bool {
+    if (!mbar_wait(smem_u32(&bars->q_full[q_stage(qn)]), q_phase(qn), cta_err, where)) return false;
+    if (TM::kTwoA &&
+        !mbar_wait(smem_u32(&bars->dq_empty[TM::r_index(step)]), (TM::r_use(step) & 1) ^ 1, cta_err, where + 20))
+      return false;
+    tc_fence_after_sync();
+    issue_kk(TM::a_col(step), dK_k, dQ_k[q_stage(qn)]);
+    umma_commit(smem_u32(&bars->s_full[TM::r_index(step)]));
+    return true;
+  };
+  // dP^T of global step `step`.  D = 128: region B last held dQ of the step before.
+  auto issue_dp = [&](uint32_t step, int where) -> bool {
+    if (!mbar_wait(smem_u32(&bars->do_full), do_cnt & 1, cta_err, where)) return false;
+    if (!TM::kTwoA &&
+        !mbar_wait(smem_u32(&bars->dq_empty[0]), (step & 1) ^ 1, cta_err, where + 20))
+      return false;
+    tc_fence_after_sync();
+    issue_kk(TM::kB, dV_k, dDo_k);
+    umma_commit(smem_u32(&bars->dp_full));
+    return true;
+  };
 
   for (int round = 0, rounds = bwd_num_rounds(p.n_items); DYNAMIC || round < rounds; ++round) {
     int item;
@@ -335,44 +386,30 @@ __device__ void bwd_mma_role(const BwdParams& p, uint32_t smem_base, uint32_t tm
     const BwdItem w = decode_bwd_item<CAUSAL, GROUPED>(p, item);
     if (!mbar_wait(smem_u32(&bars->kv_full), item_cnt & 1, cta_err, 50)) return;
 
-    // prologue: S^T(0), dP^T(0)
-    {
-      const uint32_t st = q_cnt & 1, ph = (q_cnt >> 1) & 1;
-      if (!mbar_wait(smem_u32(&bars->q_full[st]), ph, cta_err, 51)) return;
-      tc_fence_after_sync();
-      issue_kk(TM::kA, dK_k, dQ_k[st]);
-      umma_commit(smem_u32(&bars->s_full));
-      if (!mbar_wait(smem_u32(&bars->do_full), do_cnt & 1, cta_err, 52)) return;
-      if (!mbar_wait(smem_u32(&bars->dq_empty), (step_cnt & 1) ^ 1, cta_err, 53)) return;
-      tc_fence_after_sync();
-      issue_kk(TM::kB, dV_k, dDo_k);
-      umma_commit(smem_u32(&bars->dp_full));
-    }
+    // prologue: S^T(0), dP^T(0) and, with two regions A, S^T(1)
+    if (!issue_s(step_cnt, q_cnt, 51)) return;
+    if (!issue_dp(step_cnt, 52)) return;
+    if (TM::kTwoA && w.steps > 1 && !issue_s(step_cnt + 1, q_cnt + 1, 53)) return;
+
     for (int it = 0; it < w.steps; ++it) {
-      const uint32_t st = q_cnt & 1;
-      const bool more = (it + 1 < w.steps);
+      const uint32_t st = q_stage(q_cnt), reg = TM::r_index(step_cnt);
       // dV += P^T dO_i
-      if (!mbar_wait(smem_u32(&bars->p_ready), step_cnt & 1, cta_err, 54)) return;
+      if (!mbar_wait(smem_u32(&bars->p_ready[reg]), TM::r_use(step_cnt) & 1, cta_err, 54)) return;
       if (it == 0 && !mbar_wait(smem_u32(&bars->dkv_empty), (item_cnt & 1) ^ 1, cta_err, 55)) return;
       tc_fence_after_sync();
 #pragma unroll
       for (int ks = 0; ks < kT / 16; ++ks) {
-        umma_ts(tmem + TM::kDv, tmem + TM::kA + (ks >> 2) * 64 + (ks & 3) * 8, desc_advance(dDo_mn, ks * 2048),
-                kIdescAcc, (it > 0 || ks > 0));
+        umma_ts(tmem + TM::kDv, tmem + TM::a_col(step_cnt) + (ks >> 2) * 64 + (ks & 3) * 8,
+                desc_advance(dDo_mn, ks * 2048), kIdescAcc, (it > 0 || ks > 0));
       }
       umma_commit(smem_u32(&bars->do_empty));
       ++do_cnt;
-      // S^T of the next query tile
-      if (more) {
-        const uint32_t nst = (q_cnt + 1) & 1, nph = ((q_cnt + 1) >> 1) & 1;
-        if (!mbar_wait(smem_u32(&bars->q_full[nst]), nph, cta_err, 56)) return;
-        tc_fence_after_sync();
-        issue_kk(TM::kA, dK_k, dQ_k[nst]);
-        umma_commit(smem_u32(&bars->s_full));
-      }
+      // one region A: S^T of the next query tile goes where P^T was
+      if (!TM::kTwoA && it + 1 < w.steps && !issue_s(step_cnt + 1, q_cnt + 1, 56)) return;
       // dK += dS^T Q_i with dS^T read from region B of tensor memory (the activation groups
       // leave a bf16 copy there, over the dP^T columns they have consumed), then dQ_i = dS K_j,
-      // which overwrites region B: MMAs of one thread execute in issue order.
+      // which overwrites region B (D = 128) or the head of the step's region A (D = 64): MMAs of
+      // one thread execute in issue order.
       if (!mbar_wait(smem_u32(&bars->ds_ready), step_cnt & 1, cta_err, 57)) return;
       tc_fence_after_sync();
 #pragma unroll
@@ -382,20 +419,16 @@ __device__ void bwd_mma_role(const BwdParams& p, uint32_t smem_base, uint32_t tm
       }
 #pragma unroll
       for (int ks = 0; ks < kT / 16; ++ks) {
-        umma_ss(tmem + TM::kB, desc_advance(dDs_mn, ks * 2048), desc_advance(dK_mn, ks * 2048), kIdescDq, ks > 0);
+        umma_ss(tmem + TM::dq_col(step_cnt), desc_advance(dDs_mn, ks * 2048), desc_advance(dK_mn, ks * 2048),
+                kIdescDq, ks > 0);
       }
-      umma_commit(smem_u32(&bars->dq_full));
+      umma_commit(smem_u32(&bars->dq_full[reg]));
       umma_commit(smem_u32(&bars->q_empty[st]));
+      // dP^T of the next query tile, then (two regions A) S^T of the one after it
+      if (it + 1 < w.steps && !issue_dp(step_cnt + 1, 58)) return;
+      if (TM::kTwoA && it + 2 < w.steps && !issue_s(step_cnt + 2, q_cnt + 2, 59)) return;
       ++q_cnt;
       ++step_cnt;
-      // dP^T of the next query tile (region B must have been drained of dQ_i first)
-      if (more) {
-        if (!mbar_wait(smem_u32(&bars->do_full), do_cnt & 1, cta_err, 58)) return;
-        if (!mbar_wait(smem_u32(&bars->dq_empty), (step_cnt & 1) ^ 1, cta_err, 59)) return;
-        tc_fence_after_sync();
-        issue_kk(TM::kB, dV_k, dDo_k);
-        umma_commit(smem_u32(&bars->dp_full));
-      }
     }
     umma_commit(smem_u32(&bars->dkv_full));
     ++item_cnt;
@@ -524,13 +557,14 @@ __device__ void bwd_act_role(const BwdParams& p, const CUtensorMap* tmDk, const 
         diag = i * kT < q_lo || (i + 1) * kT > q_hi;   // the tile is not wholly inside this key's queries
       }
       float pp0[32], pp1[32];
-      if (!mbar_wait(smem_u32(&bars->s_full), step_cnt & 1, cta_err, 60 + wg)) return;
+      if (!mbar_wait(smem_u32(&bars->s_full[TM::r_index(step_cnt)]), TM::r_use(step_cnt) & 1, cta_err, 60 + wg))
+        return;
       tc_fence_after_sync();
 #pragma unroll
       for (int c = 0; c < 2; ++c) {
         const int gc = wg * 2 + c;  // 32-query chunk of the tile
         uint32_t s[32], pk[16];
-        tmem_ld32(tmem + TM::kA + lane_off + gc * 32, s);
+        tmem_ld32(tmem + TM::a_col(step_cnt) + lane_off + gc * 32, s);
         tmem_wait_ld();
         float(&ppc)[32] = (c == 0) ? pp0 : pp1;
         if (GROUPED && diag)
@@ -542,11 +576,11 @@ __device__ void bwd_act_role(const BwdParams& p, const CUtensorMap* tmDk, const 
         else
           bwd_sigmoid_chunk<0, ALIBI>(s, pk, ppc, p.scale_log2e, bias_log2e, slope_log2e, col_rel, gc * 32, 0.0f,
                                       0.0f);
-        tmem_st16(tmem + TM::kA + lane_off + wg * 64 + c * 16, pk);
+        tmem_st16(tmem + TM::a_col(step_cnt) + lane_off + wg * 64 + c * 16, pk);
       }
       tmem_wait_st();
       tc_fence_before_sync();
-      mbar_arrive(smem_u32(&bars->p_ready));
+      mbar_arrive(smem_u32(&bars->p_ready[TM::r_index(step_cnt)]));
 
       // dS^T = P (1 - P) dP^T -> bf16 -> shared memory [key][query], 128-byte swizzle
       if (!mbar_wait(smem_u32(&bars->dp_full), step_cnt & 1, cta_err, 62 + wg)) return;
@@ -640,7 +674,8 @@ __device__ void bwd_drain_role(const BwdParams& p, const CUtensorMap* tmW, uint8
     for (int s = 0; s < w.steps; ++s) {
       const int g = GROUPED ? s / w.n : 0, it = s - g * w.n;   // query head within the group, query tile
       const int row0 = (w.i_begin + it) * kT, bh_q = w.bh_q0 + g;
-      if (!mbar_wait(smem_u32(&bars->dq_full), step_cnt & 1, cta_err, 70)) return;
+      const uint32_t reg = TM::r_index(step_cnt), dq_col = TM::dq_col(step_cnt);
+      if (!mbar_wait(smem_u32(&bars->dq_full[reg]), TM::r_use(step_cnt) & 1, cta_err, 70)) return;
       ++step_cnt;
       tc_fence_after_sync();
       // 64 columns per round: both staging boxes are filled from registers, so region B is
@@ -648,12 +683,12 @@ __device__ void bwd_drain_role(const BwdParams& p, const CUtensorMap* tmW, uint8
 #pragma unroll 1
       for (int r = 0; r < D / 64; ++r) {
         uint32_t o0[32], o1[32];
-        tmem_ld32(tmem + TM::kB + lane_off + r * 64, o0);
-        tmem_ld32(tmem + TM::kB + lane_off + r * 64 + 32, o1);
+        tmem_ld32(tmem + dq_col + lane_off + r * 64, o0);
+        tmem_ld32(tmem + dq_col + lane_off + r * 64 + 32, o1);
         tmem_wait_ld();
         if (r == D / 64 - 1) {
           tc_fence_before_sync();
-          mbar_arrive(smem_u32(&bars->dq_empty));
+          mbar_arrive(smem_u32(&bars->dq_empty[reg]));
         }
         // both staging boxes must have been read by the reduce-adds issued earlier
         if (tid == 0) tma_wait_group_read<0>();
@@ -702,18 +737,20 @@ sigattn_bwd_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
     cta_err = 0;
     mbar_init(smem_u32(&bars.kv_full), 1);
     mbar_init(smem_u32(&bars.kv_empty), 2);
-    for (int s = 0; s < 2; ++s) {
+    for (int s = 0; s < 3; ++s) {
       mbar_init(smem_u32(&bars.q_full[s]), 1);
       mbar_init(smem_u32(&bars.q_empty[s]), 1);
     }
     mbar_init(smem_u32(&bars.do_full), 1);
     mbar_init(smem_u32(&bars.do_empty), 1);
-    mbar_init(smem_u32(&bars.s_full), 1);
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(smem_u32(&bars.s_full[s]), 1);
+      mbar_init(smem_u32(&bars.p_ready[s]), 256);
+      mbar_init(smem_u32(&bars.dq_full[s]), 1);
+      mbar_init(smem_u32(&bars.dq_empty[s]), 128);
+    }
     mbar_init(smem_u32(&bars.dp_full), 1);
-    mbar_init(smem_u32(&bars.p_ready), 256);
     mbar_init(smem_u32(&bars.ds_ready), 256);
-    mbar_init(smem_u32(&bars.dq_full), 1);
-    mbar_init(smem_u32(&bars.dq_empty), 128);
     mbar_init(smem_u32(&bars.dkv_full), 1);
     mbar_init(smem_u32(&bars.dkv_empty), 256);
     for (int s = 0; s < 2; ++s) {
