@@ -267,6 +267,10 @@ def time_side_workload(sa, torch, dev, cfg, steps, flush, peaks, bias=None, samp
     kern = []
     for s in range(steps):
         flush.zero_()
+        # A short spin on the device (it touches no memory) lets the host enqueue the whole step before the
+        # device reaches it: the smallest configuration runs 0.03 ms per pass, less than the host needs to
+        # issue one, and the events would otherwise time the host.
+        torch.cuda._sleep(200_000)
         e0[s].record()
         sa.sigattn_fwd(q, k, v, cfg.scale, bias, cfg.causal, slopes, out=o)
         e1[s].record()
@@ -295,7 +299,8 @@ def time_side_workload(sa, torch, dev, cfg, steps, flush, peaks, bias=None, samp
     out = {
         "workload": workload_config(cfg, 1)["workload"] if bias == cfg.bias else
                     workload_config(cfg, 1)["workload"].replace("b=-ln(N)", f"b={bias:g}"),
-        "steps": steps, "timing": "median of per-step CUDA-event times, L2 flushed before every step",
+        "steps": steps, "timing": "median of per-step CUDA-event times, L2 flushed before every step, step enqueued "
+                                  "behind a 0.1 ms device-side spin so that host launch time is not counted",
         "fwd": {"ms": t_fwd, "tflops": f_fwd / t_fwd / 1e9, "frac_of_peak": f_fwd / t_fwd / 1e9 / peak,
                 "hbm_gbs": bytes_fwd / t_fwd / 1e6, "frac_of_hbm_peak": bytes_fwd / t_fwd / 1e6 / hbm},
         "bwd": {"ms": t_bwd, "tflops": f_bwd / t_bwd / 1e9, "frac_of_peak": f_bwd / t_bwd / 1e9 / peak,

@@ -7,9 +7,15 @@
 //                u^3 <= 2^-12 for a <= -4, below bf16 resolution), and P (1 - P) = P - P^2;
 //                one exponential per element; where the MUFU pipe is the bound (forward at
 //                D = 64) a fixed share of them is evaluated on the FMA pipe (ex2_emulated).
-//   exact path   e = 2^-a,  r = 1 / (1 + e),  P = r,  P (1 - P) = r e r  (two MUFU ops),
-//                taken if any logit of the block has a > -4.  At b = -log n almost no block
-//                needs it.
+//   exact path   e = 2^-a,  r = 1 / (1 + e),  P = r,  P (1 - P) = r e r, taken if any logit of
+//                the block has a > -4.  In the forward the reciprocal is formed on the FMA and ALU
+//                pipes (an integer first guess and two Newton steps, see rcp_newton), so this path
+//                also costs one MUFU op per element there (measured: +13 % on the ViT shape, +9 % at
+//                b = 0); the backward, whose activation is not MUFU-bound, keeps the MUFU reciprocal
+//                (the Newton form measured 3-8 % slower there).  At b = -log n with normalised q, k almost no
+//                block needs it; with unnormalised inputs of unit variance at n = 197 (the ViT
+//                shape) about one thread in five does, and since the threads of a warp decide
+//                one by one, most warps then run both paths.
 //
 // The paper evaluates sigmoid as 0.5 (1 + tanh(x / 2)) with the hardware tanh (Section 4).
 // On B200 tanh.approx.f32 followed by 0.5 + 0.5 t loses P's relative accuracy for x << 0
@@ -79,13 +85,23 @@ __device__ __forceinline__ void sigmoid_common(const float (&a)[N], float (&pr)[
   }
 }
 
+// 1 / y for 1 <= y < 2^126 without the MUFU pipe: the bit pattern of y subtracted from a constant
+// gives a first guess within 5 %, and two Newton steps r <- r (2 - y r) bring the relative error to
+// 7e-6 (checked over [1, 2) times every power of two used; the error pattern repeats per binade).
+__device__ __forceinline__ float rcp_newton(float y) {
+  float r = __int_as_float(0x7EF311C7 - __float_as_int(y));
+  r = r * fmaf(-y, r, 2.0f);
+  r = r * fmaf(-y, r, 2.0f);
+  return r;
+}
+
 // Exact path: r = 1 / (1 + 2^-a) = P, and 1 - P = 2^-a r (no subtraction from a rounded P).
 template <int N, bool WITH_SLOPE>
 __device__ __forceinline__ void sigmoid_exact(const float (&a)[N], float (&pr)[N], float* pp) {
 #pragma unroll
   for (int i = 0; i < N; ++i) {
     const float e = sm100::ex2_approx(fminf(-a[i], 120.0f));
-    const float r = sm100::rcp_approx(1.0f + e);
+    const float r = WITH_SLOPE ? sm100::rcp_approx(1.0f + e) : rcp_newton(1.0f + e);
     pr[i] = r;
     if (WITH_SLOPE) pp[i] = r * (e * r);
   }
