@@ -441,15 +441,19 @@ __device__ void bwd_mma_role(const BwdParams& p, uint32_t smem_base, uint32_t tm
 // the dV product and P (1 - P) in fp32 for dS.
 //   a = log2(e) * (scale * s + b - slope * |i - j|);  u = 2^a;  P = u / (1 + u);  1 - P = 1 / (1 + u)
 // MASK: 0 no element masked, 1 causal only (queries before mask_lo), 2 both ends (padded batch)
-template <int MASK, bool ALIBI>
+// CAUSAL: a query that keeps its weight sits at or after the key, so the position term is linear in the
+// query index: one FMA per logit from a per-call constant (a masked query is blanked afterwards).
+template <int MASK, bool ALIBI, bool CAUSAL>
 __device__ __forceinline__ void bwd_sigmoid_chunk(const uint32_t (&s)[32], uint32_t (&p_out)[16], float (&pp)[32],
                                                   float scale_log2e, float bias_log2e, float slope_log2e,
                                                   float col_rel, int q_base, float mask_lo, float mask_hi) {
   float a[32];
+  const float c_first = fmaf(-slope_log2e, static_cast<float>(q_base) - col_rel, bias_log2e);   // query q_base
 #pragma unroll
   for (int e = 0; e < 32; ++e) {
     float c0 = bias_log2e;
-    if (ALIBI) c0 = fmaf(-slope_log2e, fabsf(static_cast<float>(q_base + e) - col_rel), bias_log2e);
+    if (ALIBI && CAUSAL) c0 = fmaf(-slope_log2e, static_cast<float>(e), c_first);
+    else if (ALIBI) c0 = fmaf(-slope_log2e, fabsf(static_cast<float>(q_base + e) - col_rel), bias_log2e);
     a[e] = fmaf(__uint_as_float(s[e]), scale_log2e, c0);
   }
   float pr[32];
@@ -568,13 +572,13 @@ __device__ void bwd_act_role(const BwdParams& p, const CUtensorMap* tmDk, const 
         tmem_wait_ld();
         float(&ppc)[32] = (c == 0) ? pp0 : pp1;
         if (GROUPED && diag)
-          bwd_sigmoid_chunk<2, ALIBI>(s, pk, ppc, p.scale_log2e, bias_log2e, slope_log2e, col_rel, gc * 32, mask_lo,
+          bwd_sigmoid_chunk<2, ALIBI, CAUSAL>(s, pk, ppc, p.scale_log2e, bias_log2e, slope_log2e, col_rel, gc * 32, mask_lo,
                                       mask_hi);
         else if (CAUSAL && diag)
-          bwd_sigmoid_chunk<1, ALIBI>(s, pk, ppc, p.scale_log2e, bias_log2e, slope_log2e, col_rel, gc * 32, col_rel,
+          bwd_sigmoid_chunk<1, ALIBI, CAUSAL>(s, pk, ppc, p.scale_log2e, bias_log2e, slope_log2e, col_rel, gc * 32, col_rel,
                                       0.0f);
         else
-          bwd_sigmoid_chunk<0, ALIBI>(s, pk, ppc, p.scale_log2e, bias_log2e, slope_log2e, col_rel, gc * 32, 0.0f,
+          bwd_sigmoid_chunk<0, ALIBI, CAUSAL>(s, pk, ppc, p.scale_log2e, bias_log2e, slope_log2e, col_rel, gc * 32, 0.0f,
                                       0.0f);
         tmem_st16(tmem + TM::a_col(step_cnt) + lane_off + wg * 64 + c * 16, pk);
       }

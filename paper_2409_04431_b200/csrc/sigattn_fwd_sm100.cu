@@ -454,15 +454,21 @@ __device__ __forceinline__ void tmem_st_cols(uint32_t addr, uint32_t (&v)[N]) {
 
 // kCols logits of one row (32-column TMEM loads) -> kCols / 2 packed bf16x2 sigmoid values.
 //   a = s * scale_log2e + c0   (c0 carries the bias and, with ALiBi, the position term)
-template <bool ALIBI, int EMULATE_EVERY, bool TWO_SIDED = false>
+// CAUSAL: every key that keeps its weight sits at or before the query, so |i - j| = i - j there and the
+// position term is linear in the column: one FMA per logit from a per-call constant instead of a
+// difference and an FMA with |.| (what a masked key gets instead is blanked afterwards).
+template <bool ALIBI, bool CAUSAL, int EMULATE_EVERY, bool TWO_SIDED = false>
 __device__ __forceinline__ void sigmoid_cols(const uint32_t (&s)[kCols], uint32_t (&out)[kCols / 2],
                                              float scale_log2e, float bias_log2e, float slope_log2e, float row_rel,
                                              int col_base, bool masked, float mask_limit, float mask_first = 0.0f) {
   float a[kCols];
+  const float c_first = fmaf(-slope_log2e, row_rel - static_cast<float>(col_base), bias_log2e);   // column col_base
 #pragma unroll
   for (int i = 0; i < kCols; ++i) {
     float c0 = bias_log2e;
-    if (ALIBI) {
+    if (ALIBI && CAUSAL) {
+      c0 = fmaf(slope_log2e, static_cast<float>(i), c_first);
+    } else if (ALIBI) {
       const float dist = row_rel - static_cast<float>(col_base + i);
       c0 = fmaf(-slope_log2e, fabsf(dist), bias_log2e);
     }
@@ -584,11 +590,11 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
         if (ragged) {
           const int key0 = jk * kBN;
           const bool cut = key0 < key_lo[t] || key0 + kBN > key_hi[t];   // not wholly inside the row's range
-          sigmoid_cols<ALIBI, kEmulateEvery, true>(sv, pk, p.scale_log2e, bias_t[t], slope_t[0], row_rel, g * kCols, cut,
+          sigmoid_cols<ALIBI, CAUSAL, kEmulateEvery, true>(sv, pk, p.scale_log2e, bias_t[t], slope_t[0], row_rel, g * kCols, cut,
                                                    static_cast<float>(key_hi[t] - 1 - key0),
                                                    static_cast<float>(key_lo[t] - key0));
         } else {
-          sigmoid_cols<ALIBI, kEmulateEvery>(sv, pk, p.scale_log2e, bias_t[PACKED ? t : 0], slope_t[PACKED ? t : 0],
+          sigmoid_cols<ALIBI, CAUSAL, kEmulateEvery>(sv, pk, p.scale_log2e, bias_t[PACKED ? t : 0], slope_t[PACKED ? t : 0],
                                              row_rel, g * kCols, diag, mask_limit);
         }
         tmem_st_cols(tS, pk);
