@@ -479,7 +479,7 @@ def run_ours(args, cfg):
             "wall_s_timed_region": wall,
         }
         if world == 1 and not args.no_side_workloads:
-            # the other bf16 configurations and the exact (two-MUFU) activation path, same timing rules;
+            # the other bf16 configurations and the exact activation path (b = 0), same timing rules;
             # reported beside the headline, never folded into `value`
             del q, k, v, d_o, o, grads, ws, arena
             torch.cuda.empty_cache()
