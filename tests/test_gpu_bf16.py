@@ -119,6 +119,17 @@ def test_bias_extremes(bias, causal):
     compare(q, k, v, d_o, 0.125, bias, causal, None)
 
 
+@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("std", [2.0, 6.0])
+def test_wide_logits_through_the_exact_path(D, std):
+    """Logits of standard deviation std^2 (4 and 36): every block holds arguments on both sides of the
+    common path's limit, far into both tails and beyond the exponent clamp, so the exact path's
+    reciprocal (FMA-pipe Newton steps in the forward, MUFU in the backward) is exercised over its range."""
+    q, k, v, d_o = inputs.random_case(1, 2, 300, D, seed=4242 + D, std=std)
+    compare(q, k, v, d_o, 1 / math.sqrt(D), -math.log(300), False, None)
+    compare(q, k, v, d_o, 1 / math.sqrt(D), 0.0, True, np.array([0.25, 0.0078125], dtype=np.float32))
+
+
 def test_saturated_weights():
     """b = +30: P = 1 everywhere; O and dV are (prefix) sums, dQ = dK = 0 to working precision."""
     q, k, v, d_o = inputs.random_case(1, 2, 200, 128, seed=98)
