@@ -9,7 +9,7 @@ import sys
 PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libsigattn.so")
-SOURCES = ["sigattn_api.cu", "sigattn_fp32.cu", "sigattn_fwd_sm100.cu", "sigattn_bwd_sm100.cu",
+SOURCES = ["sigattn_api.cu", "sigattn_fp32.cu", "sigattn_fwd_sm100.cu", "sigattn_fwd_single_sm100.cu", "sigattn_bwd_sm100.cu",
            "sigattn_static_scratch.cu", "sigattn_peer.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a",

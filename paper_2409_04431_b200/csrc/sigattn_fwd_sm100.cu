@@ -40,17 +40,31 @@ using namespace sm100;
 
 constexpr int kBM = 128;        // query rows per tile (= TMEM lanes)
 constexpr int kBN = 128;        // keys per tile
+// This file is compiled in two shapes.  The default is the one described above (two query tiles per work
+// item, sixteen activation warps, one thread block per SM).  With SIGATTN_FWD_TILES = 1 a work item is a
+// single query tile, there are eight activation warps, and two thread blocks share an SM (256 columns of
+// tensor memory and under half of the shared memory each): the tile's own steps run one after the other
+// (logits, activation, P V), and the overlap of tensor and MUFU work comes from the other thread block,
+// which also hides a work item's start and end.  That shape serves short sequences (see the launcher).
+#ifndef SIGATTN_FWD_TILES
+#define SIGATTN_FWD_TILES 2
+#endif
+constexpr int kTiles = SIGATTN_FWD_TILES;
+static_assert(kTiles == 1 || kTiles == 2, "query tiles per work item");
 #ifndef SIGATTN_FWD_ACT_WARPS
-#define SIGATTN_FWD_ACT_WARPS 16
+#define SIGATTN_FWD_ACT_WARPS (SIGATTN_FWD_TILES == 2 ? 16 : 8)
 #endif
 constexpr int kActWarps = SIGATTN_FWD_ACT_WARPS;   // 8 or 16
 constexpr int kActThreads = 32 * kActWarps;
 constexpr int kGroups = kActWarps / 4;             // column groups of a tile
 constexpr int kCols = kBN / kGroups;               // key columns per activation thread
+constexpr int kRun = kCols > 32 ? 32 : kCols;      // of which it holds this many in registers at a time
 constexpr int kFwdThreads = kActThreads + 64;
 constexpr int kLoadWarp = kActWarps;
 constexpr int kMmaWarp = kActWarps + 1;
 constexpr float kLog2e = 1.4426950408889634f;
+constexpr uint32_t kTmemCols = 256 * kTiles;       // per tile: 128 columns of logits / P, up to 128 of O
+constexpr int kCtasPerSm = (kTiles == 1) ? 2 : 1;
 
 // Share of the forward's exponentials evaluated on the FMA pipe (every m-th, 0 = none).
 // At D = 128 the shorter instruction stream wins (emulating every 4th measured -6 %); at
@@ -73,15 +87,16 @@ struct FwdSmem {
   static constexpr int kPanels = D / 64;
   static constexpr int kPanelBytes = kBM * 128;           // 128 rows x 128 B
   static constexpr int kTileBytes = kPanels * kPanelBytes;  // one Q, K or V tile
-  static constexpr int kStages = (D == 128) ? 4 : 8;
+  // K/V ring; the single-tile shape must fit two thread blocks into an SM's shared memory
+  static constexpr int kStages = (kTiles == 2) ? ((D == 128) ? 4 : 8) : ((D == 128) ? 2 : 4);
   static constexpr int kQOff = 0;
-  static constexpr int kKvOff = 2 * kTileBytes;
+  static constexpr int kKvOff = kTiles * kTileBytes;
   // At D = 64 there is room for a staging buffer of O of its own: the Q buffer is then free as soon
   // as the item's last logits are computed, and the next item's Q load runs under the last activation,
   // the last P V and the epilogue.  At D = 128 O is staged in the Q buffer (shared memory is full).
   static constexpr bool kOStaged = (D == 64);
   static constexpr int kOOff = kKvOff + kStages * kTileBytes;
-  static constexpr int kTotal = kOOff + (kOStaged ? 2 * kTileBytes : 0);
+  static constexpr int kTotal = kOOff + (kOStaged ? kTiles * kTileBytes : 0);
   static constexpr int kDynBytes = kTotal + 1024;  // slack to align the base to 1024 B
 };
 
@@ -114,7 +129,7 @@ struct FwdParams {
   const int* cu_seqlens;    // n_seqs + 1 row offsets, or nullptr
   int n_seqs;
   int* sched_counter;       // dynamic schedule: next work item to hand out (zero at launch), or nullptr
-  int n_pairs;     // ceil(N / 256)
+  int n_pairs;     // work items per head: ceil(N / (128 kTiles))
   int n_kv_total;  // ceil(N / 128)
   // Keys split over several work items (packed mode only; decoding has too few (batch, head)
   // pairs to fill the GPU): split s of a (head, pair) visits key tiles [s, s + 1) * tiles_per_split
@@ -200,7 +215,7 @@ __device__ __forceinline__ Item decode_item(const FwdParams& p, int item) {
   const int split = rank / p.n_pairs;   // 0 unless the keys are split
   rank -= split * p.n_pairs;
   const int pair = CAUSAL ? (p.n_pairs - 1 - rank) : rank;
-  w.row0 = pair * 2 * kBM;
+  w.row0 = pair * kTiles * kBM;
   w.n_valid = p.seqlens ? max(0, min(p.N, __ldg(p.seqlens + w.bh / p.H))) : p.N;
   const int n_kv_valid = p.seqlens ? max(1, (w.n_valid + kBN - 1) / kBN) : p.n_kv_total;
 #pragma unroll
@@ -208,7 +223,7 @@ __device__ __forceinline__ Item decode_item(const FwdParams& p, int item) {
     const int r = w.row0 + t * kBM;
     // causal: the tile's last row, at position r + 127 + pos0, sees keys up to that position
     // (packed rows: every tile holds last queries of some head, so every key tile is visited)
-    w.n[t] = (r >= p.N) ? 0
+    w.n[t] = (t >= kTiles || r >= p.N) ? 0
              : ((CAUSAL && p.pack_rows == 0)
                     // (a tile that lies before every key still visits one key tile, fully masked: zeros)
                     ? ((r + kBM - 1 + p.pos0 < 0) ? 1 : min(n_kv_valid, (r + kBM - 1 + p.pos0) / kBN + 1))
@@ -227,7 +242,7 @@ __device__ __forceinline__ Item decode_item(const FwdParams& p, int item) {
 #pragma unroll
     for (int t = 0; t < 2; ++t) {
       const int r_first = w.row0 + t * kBM;
-      if (r_first >= p.N) { w.n[t] = 0; continue; }
+      if (t >= kTiles || r_first >= p.N) { w.n[t] = 0; continue; }
       const int r_last = min(p.N, r_first + kBM) - 1;
       const int key_end = CAUSAL ? r_last + 1 : __ldg(p.cu_seqlens + seq_of_row(p.cu_seqlens, p.n_seqs, r_last) + 1);
       w.n[t] = max(1, min(p.n_kv_total, (key_end + kBN - 1) / kBN) - w.j0);
@@ -351,7 +366,7 @@ __device__ void fwd_mma_role(const FwdParams& p, uint32_t smem_base, uint32_t tm
       // column group c wrote its bf16 P over the first half of its own logits columns:
       // [c kCols, c kCols + kCols / 2), one k-step of 16 keys per 8 columns
       const uint32_t p_col = (ks / (kCols / 16)) * kCols + (ks % (kCols / 16)) * 8;
-      umma_ts_warp(leader, tmem + 2 * kBN + t * D, tmem + t * kBN + p_col, desc_advance(vd, ks * 2048), kIdescPV,
+      umma_ts_warp(leader, tmem + kTiles * kBN + t * D, tmem + t * kBN + p_col, desc_advance(vd, ks * 2048), kIdescPV,
               (accumulate || ks > 0));
     }
   };
@@ -452,19 +467,19 @@ __device__ __forceinline__ void tmem_st_cols(uint32_t addr, uint32_t (&v)[N]) {
   if constexpr (N == 16) tmem_st16(addr, v); else tmem_st32(addr, v);
 }
 
-// kCols logits of one row (32-column TMEM loads) -> kCols / 2 packed bf16x2 sigmoid values.
+// NC logits of one row -> NC / 2 packed bf16x2 sigmoid values.
 //   a = s * scale_log2e + c0   (c0 carries the bias and, with ALiBi, the position term)
 // CAUSAL: every key that keeps its weight sits at or before the query, so |i - j| = i - j there and the
 // position term is linear in the column: one FMA per logit from a per-call constant instead of a
 // difference and an FMA with |.| (what a masked key gets instead is blanked afterwards).
-template <bool ALIBI, bool CAUSAL, int EMULATE_EVERY, bool TWO_SIDED = false>
-__device__ __forceinline__ void sigmoid_cols(const uint32_t (&s)[kCols], uint32_t (&out)[kCols / 2],
+template <int NC, bool ALIBI, bool CAUSAL, int EMULATE_EVERY, bool TWO_SIDED = false>
+__device__ __forceinline__ void sigmoid_cols(const uint32_t (&s)[NC], uint32_t (&out)[NC / 2],
                                              float scale_log2e, float bias_log2e, float slope_log2e, float row_rel,
                                              int col_base, bool masked, float mask_limit, float mask_first = 0.0f) {
-  float a[kCols];
+  float a[NC];
   const float c_first = fmaf(-slope_log2e, row_rel - static_cast<float>(col_base), bias_log2e);   // column col_base
 #pragma unroll
-  for (int i = 0; i < kCols; ++i) {
+  for (int i = 0; i < NC; ++i) {
     float c0 = bias_log2e;
     if (ALIBI && CAUSAL) {
       c0 = fmaf(slope_log2e, static_cast<float>(i), c_first);
@@ -474,17 +489,17 @@ __device__ __forceinline__ void sigmoid_cols(const uint32_t (&s)[kCols], uint32_
     }
     a[i] = fmaf(__uint_as_float(s[i]), scale_log2e, c0);
   }
-  float pr[kCols];
-  sigmoid_block<kCols, false, EMULATE_EVERY>(a, pr, nullptr);
+  float pr[NC];
+  sigmoid_block<NC, false, EMULATE_EVERY>(a, pr, nullptr);
   if (masked) {  // keys after the query (and, in a padded batch, past the sequence's end) get weight 0
 #pragma unroll
-    for (int i = 0; i < kCols; ++i)
+    for (int i = 0; i < NC; ++i)
       if (static_cast<float>(col_base + i) > mask_limit ||
           (TWO_SIDED && static_cast<float>(col_base + i) < mask_first))   // keys before the row's own sequence
         pr[i] = 0.0f;
   }
 #pragma unroll
-  for (int i = 0; i < kCols / 2; ++i) out[i] = pack_bf16x2(pr[2 * i], pr[2 * i + 1]);
+  for (int i = 0; i < NC / 2; ++i) out[i] = pack_bf16x2(pr[2 * i], pr[2 * i + 1]);
 }
 
 // All activation threads work on the same query tile at a time, alternating between the
@@ -524,7 +539,7 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
     int pos_t[2];   // positions stay integers: shards of very long sequences put them beyond 2^24
     if (PACKED) {
 #pragma unroll
-      for (int t = 0; t < 2; ++t) {
+      for (int t = 0; t < kTiles; ++t) {
         const int r = w.row0 + t * kBM + tid;
         const int g_head = min(r / p.pack_rows, p.pack_group - 1);   // rows past the end only fill the tile
         const int head = w.bh * p.pack_group + g_head;               // (b * H_kv + h_kv) * group + g = b * H + h
@@ -542,7 +557,7 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
     int key_lo[2] = {0, 0}, key_hi[2] = {0, 0};
     if (ragged) {
 #pragma unroll
-      for (int t = 0; t < 2; ++t) {
+      for (int t = 0; t < kTiles; ++t) {
         const int r = w.row0 + t * kBM + tid;
         bias_t[t] = p.bias_log2e;
         if (r < p.N) {
@@ -557,7 +572,7 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
     // Tile-steps are visited in the order (j, tile 0), (j, tile 1), (j + 1, tile 0), ...
     for (int j = 0; j < w.n_kv; ++j) {
 #pragma unroll
-      for (int t = 0; t < 2; ++t) {
+      for (int t = 0; t < kTiles; ++t) {
         if (j >= w.n[t]) continue;
         uint32_t& cnt = t ? s_cnt1 : s_cnt0;
         if (!mbar_wait(smem_u32(&bars->s_full[t]), cnt & 1, cta_err, 30 + t)) return;
@@ -579,25 +594,30 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
           if (w.row0 + t * kBM + tid >= w.n_valid) mask_limit = -1.0f;
           diag = diag || (j + 1) * kBN > w.n_valid || w.row0 + (t + 1) * kBM > w.n_valid;
         }
-        // bf16 P goes back over the first half of the columns this thread has just read
+        // bf16 P goes back over the first half of the columns this thread reads, 32 logits at a time
+        // (the packed values of a later run land on logits that an earlier run has consumed)
         const uint32_t tS = tmem + t * kBN + lane_off + g * kCols;
-        uint32_t sv[kCols];
-        tmem_ld_cols(tS, sv);
-        tmem_wait_ld();
-        uint32_t pk[kCols / 2];
         constexpr int kEmulateEvery = (D == 128) ? SIGATTN_FWD_EMULATE_D128
                                       : CAUSAL ? SIGATTN_FWD_EMULATE_D64 : SIGATTN_FWD_EMULATE_D64_UNMASKED;
-        if (ragged) {
-          const int key0 = jk * kBN;
-          const bool cut = key0 < key_lo[t] || key0 + kBN > key_hi[t];   // not wholly inside the row's range
-          sigmoid_cols<ALIBI, CAUSAL, kEmulateEvery, true>(sv, pk, p.scale_log2e, bias_t[t], slope_t[0], row_rel, g * kCols, cut,
-                                                   static_cast<float>(key_hi[t] - 1 - key0),
-                                                   static_cast<float>(key_lo[t] - key0));
-        } else {
-          sigmoid_cols<ALIBI, CAUSAL, kEmulateEvery>(sv, pk, p.scale_log2e, bias_t[PACKED ? t : 0], slope_t[PACKED ? t : 0],
-                                             row_rel, g * kCols, diag, mask_limit);
+#pragma unroll
+        for (int c = 0; c < kCols / kRun; ++c) {
+          uint32_t sv[kRun];
+          tmem_ld_cols(tS + c * kRun, sv);
+          tmem_wait_ld();
+          uint32_t pk[kRun / 2];
+          const int col0 = g * kCols + c * kRun;
+          if (ragged) {
+            const int key0 = jk * kBN;
+            const bool cut = key0 < key_lo[t] || key0 + kBN > key_hi[t];   // not wholly inside the row's range
+            sigmoid_cols<kRun, ALIBI, CAUSAL, kEmulateEvery, true>(sv, pk, p.scale_log2e, bias_t[t], slope_t[0], row_rel, col0,
+                                                           cut, static_cast<float>(key_hi[t] - 1 - key0),
+                                                           static_cast<float>(key_lo[t] - key0));
+          } else {
+            sigmoid_cols<kRun, ALIBI, CAUSAL, kEmulateEvery>(sv, pk, p.scale_log2e, bias_t[PACKED ? t : 0],
+                                                     slope_t[PACKED ? t : 0], row_rel, col0, diag, mask_limit);
+          }
+          tmem_st_cols(tS + c * (kRun / 2), pk);
         }
-        tmem_st_cols(tS, pk);
         tmem_wait_st();
         tc_fence_before_sync();
         mbar_arrive(smem_u32(&bars->p_full[t]));
@@ -608,55 +628,59 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
     // buffer, free once every logits MMA of the item is done; at D = 64 a buffer of its own) -> TMA store.  Each column group
     // converts its share of the D columns.
 #pragma unroll
-    for (int t = 0; t < 2; ++t) {
+    for (int t = 0; t < kTiles; ++t) {
       if (w.n[t] == 0) continue;
       if (!mbar_wait(smem_u32(&bars->o_full[t]), it[t] & 1, cta_err, 32 + t)) return;
       ++it[t];
       tc_fence_after_sync();
       uint8_t* stage = smem + (L::kOStaged ? L::kOOff : L::kQOff) + t * L::kTileBytes;
-      constexpr int kECols = D / kGroups;   // accumulator columns per thread
-      const uint32_t tO = tmem + 2 * kBN + t * D + lane_off + g * kECols;
-      uint32_t o[kECols];
-      tmem_ld_cols(tO, o);
-      tmem_wait_ld();
-      if (GENERAL && p.row_scale != nullptr) {
-        // sequence-length normalisation: one factor per query row (rows past the end are not stored)
-        const int row = w.row0 + t * kBM + tid;
-        const float r = row < p.N ? __ldg(p.row_scale + row) : 0.0f;
+      constexpr int kECols = D / kGroups;                 // accumulator columns per thread
+      constexpr int kERun = kECols > 32 ? 32 : kECols;    // converted this many at a time
+      // Partial result (split keys, or one shard of the keys): this item's rows are added, in fp32,
+      // into the accumulator - local scratch or another GPU's memory, plain vector reductions
+      // either way.  Whoever owns the accumulator converts the sums to bf16 afterwards.  The Q
+      // buffer is not needed for staging.
+      const bool to_acc = (PACKED || GENERAL) && p.split_ws != nullptr;
+      const int row = w.row0 + t * kBM + tid;
 #pragma unroll
-        for (int e = 0; e < kECols; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * r);
-      }
-      if ((PACKED || GENERAL) && p.split_ws != nullptr) {
-        // Partial result (split keys, or one shard of the keys): add this item's rows, in fp32,
-        // into the accumulator - local scratch or another GPU's memory, plain vector reductions
-        // either way.  Whoever owns the accumulator converts the sums to bf16 afterwards.  The Q
-        // buffer is not needed for staging.
-        const int row = w.row0 + t * kBM + tid;
-        if (row < p.N) {
-          float* dst = p.split_ws + (static_cast<size_t>(w.bh) * p.N + row) * D + g * kECols;
+      for (int ec = 0; ec < kECols / kERun; ++ec) {
+        const int col = g * kECols + ec * kERun;   // first of this run's columns
+        uint32_t o[kERun];
+        tmem_ld_cols(tmem + kTiles * kBN + t * D + lane_off + col, o);
+        tmem_wait_ld();
+        if (GENERAL && p.row_scale != nullptr) {
+          // sequence-length normalisation: one factor per query row (rows past the end are not stored)
+          const float r = row < p.N ? __ldg(p.row_scale + row) : 0.0f;
 #pragma unroll
-          for (int e = 0; e < kECols; e += 4)
-            red_add_v4_f32(dst + e, __uint_as_float(o[e]), __uint_as_float(o[e + 1]), __uint_as_float(o[e + 2]),
-                           __uint_as_float(o[e + 3]));
+          for (int e = 0; e < kERun; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * r);
         }
+        if (to_acc) {
+          if (row < p.N) {
+            float* dst = p.split_ws + (static_cast<size_t>(w.bh) * p.N + row) * D + col;
+#pragma unroll
+            for (int e = 0; e < kERun; e += 4)
+              red_add_v4_f32(dst + e, __uint_as_float(o[e]), __uint_as_float(o[e + 1]), __uint_as_float(o[e + 2]),
+                             __uint_as_float(o[e + 3]));
+          }
+        } else {
+          uint8_t* row_ptr = stage + (col >> 6) * L::kPanelBytes + tid * 128;
+#pragma unroll
+          for (int q4 = 0; q4 < kERun / 8; ++q4) {
+            uint4 val;
+            val.x = pack_bf16x2(__uint_as_float(o[8 * q4 + 0]), __uint_as_float(o[8 * q4 + 1]));
+            val.y = pack_bf16x2(__uint_as_float(o[8 * q4 + 2]), __uint_as_float(o[8 * q4 + 3]));
+            val.z = pack_bf16x2(__uint_as_float(o[8 * q4 + 4]), __uint_as_float(o[8 * q4 + 5]));
+            val.w = pack_bf16x2(__uint_as_float(o[8 * q4 + 6]), __uint_as_float(o[8 * q4 + 7]));
+            const int chunk = ((col & 63) >> 3) + q4;
+            *reinterpret_cast<uint4*>(row_ptr + ((chunk ^ (tid & 7)) * 16)) = val;
+          }
+        }
+      }
+      if (to_acc) {
         tc_fence_before_sync();
         mbar_arrive(smem_u32(&bars->o_empty[t]));
         if (!L::kOStaged && threadIdx.x == 0) mbar_arrive(smem_u32(&bars->q_empty[t]));   // all logits MMAs of the item are done
         continue;
-      }
-      {
-        const int col = g * kECols;           // first of this thread's columns
-        uint8_t* row_ptr = stage + (col >> 6) * L::kPanelBytes + tid * 128;
-#pragma unroll
-        for (int q4 = 0; q4 < kECols / 8; ++q4) {
-          uint4 val;
-          val.x = pack_bf16x2(__uint_as_float(o[8 * q4 + 0]), __uint_as_float(o[8 * q4 + 1]));
-          val.y = pack_bf16x2(__uint_as_float(o[8 * q4 + 2]), __uint_as_float(o[8 * q4 + 3]));
-          val.z = pack_bf16x2(__uint_as_float(o[8 * q4 + 4]), __uint_as_float(o[8 * q4 + 5]));
-          val.w = pack_bf16x2(__uint_as_float(o[8 * q4 + 6]), __uint_as_float(o[8 * q4 + 7]));
-          const int chunk = ((col & 63) >> 3) + q4;
-          *reinterpret_cast<uint4*>(row_ptr + ((chunk ^ (tid & 7)) * 16)) = val;
-        }
       }
       tc_fence_before_sync();
       mbar_arrive(smem_u32(&bars->o_empty[t]));
@@ -681,7 +705,7 @@ __device__ void fwd_act_role(const FwdParams& p, const CUtensorMap* tmO, uint8_t
 // ------------------------------------------------------------------ kernel
 
 template <int D, bool CAUSAL, bool ALIBI, int MODE>
-__global__ void __launch_bounds__(kFwdThreads, 1)
+__global__ void __launch_bounds__(kFwdThreads, kCtasPerSm)
 sigattn_fwd_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                         const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
                         const FwdParams p) {
@@ -722,7 +746,7 @@ sigattn_fwd_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
     tma_prefetch_desc(&tmO);
   }
   if (warp == kMmaWarp) {
-    tmem_alloc(smem_u32(&tmem_base_slot), 512);
+    tmem_alloc(smem_u32(&tmem_base_slot), kTmemCols);
     tmem_relinquish();
   }
   tc_fence_before_sync();
@@ -746,9 +770,10 @@ sigattn_fwd_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
     if (threadIdx.x == 0) atomicExch(p.status, 100 + cta_err);
     __nanosleep(100000);  // let copies in flight towards this CTA's shared memory land
   }
-  if (warp == kMmaWarp) tmem_dealloc(tmem, 512);
+  if (warp == kMmaWarp) tmem_dealloc(tmem, kTmemCols);
 }
 
+#if SIGATTN_FWD_TILES == 2
 // O (bf16) = the fp32 sums of the key splits: the pass that follows a split forward.
 __global__ void __launch_bounds__(256)
 sigattn_fwd_convert_o_kernel(const float4* __restrict__ ws, uint2* __restrict__ o, size_t n_vec4) {
@@ -762,6 +787,24 @@ sigattn_fwd_convert_o_kernel(const float4* __restrict__ ws, uint2* __restrict__ 
 // Number of key splits for a problem with `base_items` work items of `n_kv` key tiles each:
 // the count that minimises rounds of the persistent grid times tiles per item (plus about two
 // tiles' worth of per-item start-up and epilogue), each split keeping at least two key tiles.
+// Which shape serves a plain problem (the launcher's tile table).  Measured on B200, forward alone, us:
+//   B4 H12 N256 D64 (48 pair items)    one tile 13.3   two tiles 17.4
+//   B2 H8 N256 D128 (16)               14.3            17.4
+//   B8 H12 N197 D64 (96)               17.4            17.4
+//   B16 H12 N197 D64 (192)             23.6            25.6
+//   B24 / B32 H12 N197 D64 (288, 384)  27.6 / 34.8     25.6 / 31.7
+//   B3 / B8 H12 N577 D64 (108, 288)    23.6 / 42.0     21.5 / 37.8
+//   B4 H16 N384 D128 causal (128)      20.5            19.5
+// and on the benchmark configurations the two-tile shape is 5-16 % faster.  One tile per item pays when the
+// two-tile items leave more than half of the SMs empty and the sequence is too short for the keys of an item
+// to be divided (that division serves the long sequences with few heads); with N <= 128 both shapes are the same.
+bool fwd_single_tile_shape(const Problem& p, int num_sms) {
+  const bool plain_self = p.key_rows() == p.N && p.query_pos0() == 0 && p.kv_heads() == p.H;
+  const long long pair_items = static_cast<long long>(p.B) * p.H * ((p.N + 2 * kBM - 1) / (2 * kBM));
+  const int n_kv_tiles = (p.N + kBN - 1) / kBN;
+  return plain_self && p.N > kBM && n_kv_tiles < 4 && 2 * pair_items <= num_sms;
+}
+
 int choose_key_splits(int base_items, int n_kv, int num_sms) {
   int best = 1;
   long long best_cost = -1;
@@ -781,6 +824,7 @@ int choose_key_splits(int base_items, int n_kv, int num_sms) {
 // sees its counter run past what one launch can draw sets the device status word).
 constexpr int kSchedSlots = 1024;
 __device__ int g_fwd_sched_counters[kSchedSlots];
+#endif
 
 template <int D, bool CAUSAL, bool ALIBI, int MODE>
 int launch_fwd_variant(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtensorMap& tmO,
@@ -798,7 +842,8 @@ int launch_fwd_variant(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUt
     if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
     configured.fetch_or(bit, std::memory_order_relaxed);
   }
-  const int grid = fp.n_items < num_sms ? fp.n_items : num_sms;
+  const int slots = num_sms * kCtasPerSm;
+  const int grid = fp.n_items < slots ? fp.n_items : slots;
   kernel<<<grid, kFwdThreads, FwdSmem<D>::kDynBytes, stream>>>(tmQ, tmK, tmV, tmO, fp);
   *cuda_err = cudaGetLastError();
   return *cuda_err == cudaSuccess ? SIGATTN_OK : SIGATTN_ERR_CUDA;
@@ -806,6 +851,57 @@ int launch_fwd_variant(const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUt
 
 }  // namespace
 
+#if SIGATTN_FWD_TILES == 1
+// Plain problems only (no grouped heads, padded or unpadded batches, key shards or split keys).
+int launch_fwd_bf16_single(const void* q, const void* k, const void* v, void* o, const Problem& p, int* status,
+                           cudaStream_t stream, unsigned long long* launches, cudaError_t* cuda_err) {
+  int dev = 0, num_sms = 0;
+  *cuda_err = cudaGetDevice(&dev);
+  if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
+  *cuda_err = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
+  if (*cuda_err != cudaSuccess) return SIGATTN_ERR_CUDA;
+  const uint64_t BH = static_cast<uint64_t>(p.B) * p.H;
+  CUtensorMap tmQ, tmK, tmV, tmO;
+  const void* ptrs[4] = {q, k, v, o};
+  CUtensorMap* maps[4] = {&tmQ, &tmK, &tmV, &tmO};
+  for (int i = 0; i < 4; ++i) {
+    if (make_map_3d(maps[i], ptrs[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, BH, p.N, p.D, kBM, 64) != 0) {
+      *cuda_err = cudaErrorInvalidValue;
+      return SIGATTN_ERR_CUDA;
+    }
+  }
+  FwdParams fp = {};
+  fp.BH = static_cast<int>(BH);
+  fp.H = fp.H_kv = p.H;
+  fp.group = 1;
+  fp.pack_group = 1;
+  fp.N = p.N;
+  fp.pos0 = 0;
+  fp.n_pairs = (p.N + kBM - 1) / kBM;
+  fp.n_kv_total = (p.N + kBN - 1) / kBN;
+  fp.n_splits = 1;
+  fp.tiles_per_split = fp.n_kv_total;
+  fp.n_items = fp.n_pairs * fp.BH;
+  fp.scale_log2e = p.scale * kLog2e;
+  fp.bias_log2e = p.bias * kLog2e;
+  fp.bias_vec = p.bias_vec;
+  fp.slopes = p.slopes;
+  fp.status = status;
+  int rc;
+  const bool alibi = p.slopes != nullptr;
+#define SIGATTN_FWD_CASE(DD, CC, AA) rc = launch_fwd_variant<DD, CC, AA, 0>(tmQ, tmK, tmV, tmO, fp, num_sms, stream, cuda_err)
+  if (p.D == 128) {
+    if (p.causal) { if (alibi) SIGATTN_FWD_CASE(128, true, true); else SIGATTN_FWD_CASE(128, true, false); }
+    else          { if (alibi) SIGATTN_FWD_CASE(128, false, true); else SIGATTN_FWD_CASE(128, false, false); }
+  } else {
+    if (p.causal) { if (alibi) SIGATTN_FWD_CASE(64, true, true); else SIGATTN_FWD_CASE(64, true, false); }
+    else          { if (alibi) SIGATTN_FWD_CASE(64, false, true); else SIGATTN_FWD_CASE(64, false, false); }
+  }
+#undef SIGATTN_FWD_CASE
+  if (rc == SIGATTN_OK) *launches += 1;
+  return rc;
+}
+#else
 int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const Problem& p, int* status,
                     cudaStream_t stream, unsigned long long* launches, cudaError_t* cuda_err) {
   int dev = 0, num_sms = 0;
@@ -896,6 +992,8 @@ int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const 
   fp.sched_counter = nullptr;
   const bool general = !packed && (p.cu_seqlens != nullptr || p.seqlens != nullptr || p.row_scale != nullptr || accumulate ||
                                    o_splits > 1);
+  if (!packed && !general && fwd_single_tile_shape(p, num_sms))
+    return launch_fwd_bf16_single(q, k, v, o, p, status, stream, launches, cuda_err);
   if (general) {   // the general instantiations draw their work items from a counter
     static std::atomic<unsigned> next_slot{0};
     int* counters = nullptr;
@@ -945,6 +1043,7 @@ int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const 
   }
   return SIGATTN_OK;
 }
+#endif   // SIGATTN_FWD_TILES
 
 }  // namespace sigattn
 

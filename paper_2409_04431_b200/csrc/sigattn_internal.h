@@ -50,6 +50,11 @@ int launch_bwd_fp32(const float* q, const float* k, const float* v, const float*
 int launch_fwd_bf16(const void* q, const void* k, const void* v, void* o, const Problem& p, int* status,
                     cudaStream_t stream, unsigned long long* launches, cudaError_t* cuda_err);
 
+// The forward in its second shape: one query tile per work item, two thread blocks per SM.  Plain problems
+// only (self-attention with one key/value head per query head, no padded or unpadded batch, no accumulator).
+int launch_fwd_bf16_single(const void* q, const void* k, const void* v, void* o, const Problem& p, int* status,
+                           cudaStream_t stream, unsigned long long* launches, cudaError_t* cuda_err);
+
 int launch_bwd_bf16(const void* q, const void* k, const void* v, const void* d_o, void* dq, void* dk, void* dv,
                     const Problem& p, void* workspace, int* status, cudaStream_t stream,
                     unsigned long long* launches, cudaError_t* cuda_err);
