@@ -256,10 +256,12 @@ __device__ __forceinline__ uint64_t make_smem_desc_sw128(uint32_t smem_addr, uin
 }
 
 // Descriptor of the same matrix `byte_offset` bytes further on (a multiple of 16 that keeps
-// the address inside the 256 KB window): only the start-address field changes, so issuing
-// the k-steps of a product costs one 64-bit add each instead of rebuilding the descriptor.
+// the address inside the 256 KB window): only the start-address field, in the low word, changes and
+// no carry can leave it, so a k-step costs the issuing thread one 32-bit add per operand (a 64-bit add
+// is two dependent instructions, and every instruction of that thread counts).
 __device__ __forceinline__ uint64_t desc_advance(uint64_t desc, uint32_t byte_offset) {
-  return desc + static_cast<uint64_t>(byte_offset >> 4);
+  const uint32_t lo = static_cast<uint32_t>(desc) + (byte_offset >> 4);
+  return (desc & 0xFFFFFFFF00000000ull) | lo;
 }
 
 // 32-bit instruction descriptor for kind::f16 with bf16 inputs and fp32 accumulation.
