@@ -51,6 +51,7 @@ struct BwdSmem {
   static constexpr int kKOff = 0;
   static constexpr int kVOff = kTileBytes;
   // Q stages: two at D = 128 (shared memory is full); three at D = 64, where S^T runs two steps ahead
+  // (four, which would make stage and phase a mask and a shift, measured no faster)
   static constexpr int kQStages = (D == 64) ? 3 : 2;
   static constexpr int kQOff = 2 * kTileBytes;
   static constexpr int kDoOff = (2 + kQStages) * kTileBytes;   // one stage
@@ -342,12 +343,10 @@ __device__ void bwd_mma_role(const BwdParams& p, uint32_t smem_base, uint32_t tm
   const uint64_t dDo_mn = make_smem_desc_sw128(sDo, L::kPanelBytes, 1024);  // dO_i, MN-major (dV)
   const uint64_t dK_mn = make_smem_desc_sw128(sK, L::kPanelBytes, 1024);    // K_j, MN-major (dQ)
   const uint64_t dDs_mn = make_smem_desc_sw128(sDs, L::kPanelBytes, 1024);  // dS^T, MN-major (dQ)
-  uint64_t dQ_k[L::kQStages], dQ_mn[L::kQStages];
-#pragma unroll
-  for (int st = 0; st < L::kQStages; ++st) {
-    dQ_k[st] = make_smem_desc_sw128(smem_base + L::kQOff + st * L::kTileBytes, 16, 1024);                 // S^T
-    dQ_mn[st] = make_smem_desc_sw128(smem_base + L::kQOff + st * L::kTileBytes, L::kPanelBytes, 1024);    // dK
-  }
+  // Stage 0 of Q; the other stages are reached by advancing the start address (an array indexed by the
+  // stage at run time would live in local memory, and this thread pays for every load in full)
+  const uint64_t dQ_k0 = make_smem_desc_sw128(smem_base + L::kQOff, 16, 1024);                 // Q_i, K-major (S^T)
+  const uint64_t dQ_mn0 = make_smem_desc_sw128(smem_base + L::kQOff, L::kPanelBytes, 1024);    // Q_i, MN-major (dK)
   auto q_stage = [](uint32_t cnt) -> uint32_t { return cnt % L::kQStages; };
   auto q_phase = [](uint32_t cnt) -> uint32_t { return (cnt / L::kQStages) & 1; };
   // S^T of global step `step` from the Q tile with running number `qn`.  D = 64: the step's region A last
@@ -358,7 +357,7 @@ __device__ void bwd_mma_role(const BwdParams& p, uint32_t smem_base, uint32_t tm
         !mbar_wait(smem_u32(&bars->dq_empty[TM::r_index(step)]), (TM::r_use(step) & 1) ^ 1, cta_err, where + 20))
       return false;
     tc_fence_after_sync();
-    issue_kk(TM::a_col(step), dK_k, dQ_k[q_stage(qn)]);
+    issue_kk(TM::a_col(step), dK_k, desc_advance(dQ_k0, q_stage(qn) * L::kTileBytes));
     umma_commit(smem_u32(&bars->s_full[TM::r_index(step)]));
     return true;
   };
@@ -412,9 +411,10 @@ __device__ void bwd_mma_role(const BwdParams& p, uint32_t smem_base, uint32_t tm
       // one thread execute in issue order.
       if (!mbar_wait(smem_u32(&bars->ds_ready), step_cnt & 1, cta_err, 57)) return;
       tc_fence_after_sync();
+      const uint64_t q_mn = desc_advance(dQ_mn0, st * L::kTileBytes);
 #pragma unroll
       for (int ks = 0; ks < kT / 16; ++ks) {
-        umma_ts(tmem + TM::kDk, tmem + TM::kB + (ks >> 2) * 64 + (ks & 3) * 8, desc_advance(dQ_mn[st], ks * 2048),
+        umma_ts(tmem + TM::kDk, tmem + TM::kB + (ks >> 2) * 64 + (ks & 3) * 8, desc_advance(q_mn, ks * 2048),
                 kIdescAcc, (it > 0 || ks > 0));
       }
 #pragma unroll
