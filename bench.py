@@ -265,12 +265,14 @@ def time_side_workload(sa, torch, dev, cfg, steps, flush, peaks, bias=None, samp
     if sampler:
         sampler.start()
     kern = []
+    spin = getattr(torch.cuda, "_sleep", None)   # (a private helper of torch: used when present)
     for s in range(steps):
         flush.zero_()
         # A short spin on the device (it touches no memory) lets the host enqueue the whole step before the
         # device reaches it: the smallest configuration runs 0.03 ms per pass, less than the host needs to
         # issue one, and the events would otherwise time the host.
-        torch.cuda._sleep(200_000)
+        if spin is not None:
+            spin(200_000)
         e0[s].record()
         sa.sigattn_fwd(q, k, v, cfg.scale, bias, cfg.causal, slopes, out=o)
         e1[s].record()
